@@ -1,0 +1,139 @@
+/*
+ * ssm_scan.h -- C ABI of the B200 (sm_100a) selective-scan library.
+ *
+ * The library computes the selective state-space scan "S6" of Algorithm 2 (steps 5-6), forward and backward,
+ * fused with the skip term and the SiLU gate of the block it sits in (Section 3.4).  For every batch index b and
+ * channel d independently (Section 2, "Structure and Dimensions": diagonal A, one SSM per channel), with
+ * t = 1..L and n = 1..N:
+ *
+ *     a[t,n]  = exp(delta[b,t,d] * A[d,n])                                   discretization, Eq. 4 (A-bar)
+ *     h[t,n]  = a[t,n] * h[t-1,n] + delta[b,t,d] * B[b,t,n] * x[b,t,d]       recurrence, Eq. 2a; h[0,n] = 0
+ *     s[t]    = sum_n C[b,t,n] * h[t,n] + D_skip[d] * x[b,t,d]               readout, Eq. 2b, plus skip term
+ *     out[b,t,d] = s[t] * z[b,t,d] / (1 + exp(-z[b,t,d]))                    SiLU gate
+ *
+ * B-bar is delta*B (not the zero-order-hold expression of Eq. 4).  delta is the positive step size, i.e. the value
+ * AFTER the softplus of Algorithm 2 step 4.  The (batch, L, D, N) tensors a, B-bar and h never exist in device
+ * memory (Section 3.3); long sequences are split in time and the state is carried between the pieces
+ * (Appendix D, "we split the sequences into chunks").  The backward pass recomputes the states from saved or
+ * rebuilt checkpoint states instead of reading them (Section 3.3 and Appendix D, recomputation).
+ *
+ * Conventions common to all entry points
+ *   - Every pointer except `p` is DEVICE memory owned by the caller; the library never allocates, frees or keeps a
+ *     pointer after the call returns.  Scratch memory is the caller's `workspace` (size from the *_workspace_bytes
+ *     queries; at least 256-byte aligned; contents undefined between calls; calls that overlap on the GPU must not
+ *     share a workspace).
+ *   - Layouts are dense row-major: x, delta, z, out, dout, dx, ddelta, dz are [batch][L][D]; B, C, dB, dC are
+ *     [batch][L][N]; A, dA are [D][N]; D_skip, dD are [D].
+ *   - x, delta, B, C, z, out, dout, dx, ddelta, dB, dC, dz have the element type `io_dtype`; A, D_skip, dA, dD and
+ *     every state are float32; all arithmetic and accumulation is float32; results are rounded once to io_dtype
+ *     (round-to-nearest-even).
+ *   - Outputs are overwritten, never accumulated.  Inputs must not alias outputs.
+ *   - Calls enqueue work on `stream` and return without synchronising.  Argument errors are detected before
+ *     anything is launched and reported by the return value; nothing is written in that case.  A failed kernel
+ *     launch is reported as SSM_ERR_CUDA.
+ *   - N must be 1, 2, 4, 8 or 16 (Table 10 ablates exactly these state sizes).  All io pointers must be
+ *     aligned to the element size; 16-byte aligned pointers together with D % 8 == 0 select the vector path.
+ *   - Results are bitwise reproducible for fixed inputs, shape, flags and library build: every reduction (over n,
+ *     over channels for dB/dC, over batch and time for dA/dD) has a fixed order and no floating-point atomics
+ *     are used.
+ *   - NaN and Inf propagate; signs are not validated (A < 0 and delta > 0 are expected).
+ */
+#ifndef SSM_SCAN_H_
+#define SSM_SCAN_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#if defined(__GNUC__)
+#define SSM_API __attribute__((visibility("default")))
+#else
+#define SSM_API
+#endif
+
+typedef enum {
+  SSM_OK = 0,
+  SSM_ERR_INVALID_ARG = 1,  /* null required pointer, non-positive dimension, misaligned pointer, bad flag      */
+  SSM_ERR_UNSUPPORTED = 2,  /* N or dtype outside the supported set                                             */
+  SSM_ERR_WORKSPACE = 3,    /* workspace null / misaligned / smaller than the query reports                     */
+  SSM_ERR_CUDA = 4,         /* a CUDA runtime call or a kernel launch failed                                    */
+  SSM_ERR_TIMEOUT = 5       /* a bounded device-side wait gave up (reported through ssm_scan_check_status)      */
+} ssm_status_t;
+
+typedef enum { SSM_F32 = 0, SSM_BF16 = 1 } ssm_dtype_t;
+
+enum {
+  SSM_FLAG_HAS_Z = 1u,        /* z is given: out = s * silu(z); otherwise out = s and dz is not produced        */
+  SSM_FLAG_HAS_DSKIP = 2u,    /* D_skip is given; otherwise the skip term is absent and dD is not produced      */
+  SSM_FLAG_SAVE_STATES = 4u,  /* forward: also write the checkpoint states that backward starts its recomputation
+                                 from (Appendix D keeps "intermediate scan states" between chunks)             */
+  SSM_FLAG_GENERAL_A = 8u     /* do not use the fast path for rows of A that are arithmetic progressions in n   */
+};
+
+typedef struct {
+  int32_t batch, L, D, N;   /* all >= 1 */
+  int32_t io_dtype;         /* ssm_dtype_t */
+  uint32_t flags;           /* SSM_FLAG_* */
+} ssm_problem_t;
+
+/* Bytes of scratch memory ssm_scan_fwd / ssm_scan_bwd need for this problem (0 is possible).  Returns 0 for an
+ * invalid problem; the call itself then reports the error. */
+SSM_API size_t ssm_scan_fwd_workspace_bytes(const ssm_problem_t* p);
+SSM_API size_t ssm_scan_bwd_workspace_bytes(const ssm_problem_t* p);
+
+/* Bytes of the `saved_states` buffer: float32 states h at the start of every block of ssm_scan_checkpoint_steps()
+ * time steps, laid out [batch][ceil(L / steps)][D][N].  Independent of flags. */
+SSM_API size_t ssm_scan_saved_state_bytes(const ssm_problem_t* p);
+SSM_API int32_t ssm_scan_checkpoint_steps(void);
+
+/*
+ * Forward (Algorithm 2 steps 5-6, Eq. 2a/2b, Eq. 4's A-bar, skip term, gate).
+ *   x, delta, B, C        in, io_dtype, required
+ *   A                     in, float32 [D][N], required
+ *   D_skip                in, float32 [D]; required iff SSM_FLAG_HAS_DSKIP
+ *   z                     in, io_dtype; required iff SSM_FLAG_HAS_Z
+ *   out                   out, io_dtype [batch][L][D]
+ *   saved_states          out, float32, ssm_scan_saved_state_bytes(p) bytes; required iff SSM_FLAG_SAVE_STATES
+ *   workspace             scratch of at least ssm_scan_fwd_workspace_bytes(p) bytes (may be NULL if that is 0)
+ */
+SSM_API ssm_status_t ssm_scan_fwd(const ssm_problem_t* p, const void* x, const void* delta, const float* A, const void* B,
+                          const void* C, const float* D_skip, const void* z, void* out, void* saved_states,
+                          void* workspace, size_t workspace_bytes, void* stream /* cudaStream_t */);
+
+/*
+ * Backward: gradients of loss = sum(dout * out) with respect to every input (the adjoint of the four lines at
+ * the top; the states are recomputed on chip from checkpoint states, Section 3.3 "recomputation").
+ *   x, delta, A, B, C, D_skip, z   the forward inputs, same rules as above
+ *   dout                  in, io_dtype [batch][L][D], required
+ *   saved_states          in, float32, as written by ssm_scan_fwd with SSM_FLAG_SAVE_STATES for the same problem and
+ *                         inputs; NULL makes backward rebuild the checkpoints itself (one more forward sweep)
+ *   dx, ddelta            out, io_dtype [batch][L][D], required
+ *   dA                    out, float32 [D][N], required
+ *   dB, dC                out, io_dtype [batch][L][N], required
+ *   dD                    out, float32 [D]; may be NULL; written only with SSM_FLAG_HAS_DSKIP
+ *   dz                    out, io_dtype [batch][L][D]; may be NULL; written only with SSM_FLAG_HAS_Z
+ *   workspace             scratch of at least ssm_scan_bwd_workspace_bytes(p) bytes
+ */
+SSM_API ssm_status_t ssm_scan_bwd(const ssm_problem_t* p, const void* x, const void* delta, const float* A, const void* B,
+                          const void* C, const float* D_skip, const void* z, const void* dout,
+                          const void* saved_states, void* dx, void* ddelta, float* dA, void* dB, void* dC, float* dD,
+                          void* dz, void* workspace, size_t workspace_bytes, void* stream /* cudaStream_t */);
+
+/* Human-readable name of a status code (static storage). */
+SSM_API const char* ssm_status_string(ssm_status_t s);
+
+/*
+ * Describes how the library would run this problem: number of time segments the sequence is split into, steps per
+ * segment, channels per thread block and states per thread of the forward kernel.  Any output pointer may be NULL.
+ * Returns SSM_OK or the validation error.  Host-only; launches nothing.
+ */
+SSM_API ssm_status_t ssm_scan_plan(const ssm_problem_t* p, int32_t* n_segments, int32_t* segment_steps,
+                           int32_t* channels_per_block, int32_t* states_per_thread);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SSM_SCAN_H_ */

@@ -1,0 +1,221 @@
+"""Thin Python binding of the C ABI in include/ssm_scan.h (same names, argument marshalling only).
+
+Every step of the selective scan runs in the CUDA kernels of libssm_scan.so; torch is used for device memory and
+streams.  There is no CPU or eager fallback: if the library is missing or fails to load, importing a symbol raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import shutil
+
+import torch
+
+from . import build as _build
+
+SSM_OK = 0
+SSM_F32, SSM_BF16 = 0, 1
+SSM_FLAG_HAS_Z, SSM_FLAG_HAS_DSKIP, SSM_FLAG_SAVE_STATES, SSM_FLAG_GENERAL_A = 1, 2, 4, 8
+
+EXPORTED_SYMBOLS = (
+    "ssm_scan_fwd_workspace_bytes", "ssm_scan_bwd_workspace_bytes", "ssm_scan_saved_state_bytes",
+    "ssm_scan_checkpoint_steps", "ssm_scan_fwd", "ssm_scan_bwd", "ssm_status_string", "ssm_scan_plan",
+)
+
+
+class ssm_problem_t(ctypes.Structure):
+    _fields_ = [("batch", ctypes.c_int32), ("L", ctypes.c_int32), ("D", ctypes.c_int32), ("N", ctypes.c_int32),
+                ("io_dtype", ctypes.c_int32), ("flags", ctypes.c_uint32)]
+
+
+class SsmScanError(RuntimeError):
+    pass
+
+
+_lib = None
+
+
+def library_path() -> str:
+    return _build.LIB_PATH
+
+
+def load_library() -> ctypes.CDLL:
+    """dlopen libssm_scan.so (building it first if nvcc is present and the sources are newer)."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if _build.is_stale() and shutil.which(os.environ.get("NVCC", "nvcc")):
+        _build.build_library()
+    if not os.path.exists(_build.LIB_PATH):
+        raise SsmScanError(f"{_build.LIB_PATH} is missing and nvcc is not available to build it; "
+                           "there is no fallback path")
+    lib = ctypes.CDLL(_build.LIB_PATH)
+    P = ctypes.POINTER(ssm_problem_t)
+    vp, sz = ctypes.c_void_p, ctypes.c_size_t
+    for name in ("ssm_scan_fwd_workspace_bytes", "ssm_scan_bwd_workspace_bytes", "ssm_scan_saved_state_bytes"):
+        getattr(lib, name).restype = sz
+        getattr(lib, name).argtypes = [P]
+    lib.ssm_scan_checkpoint_steps.restype = ctypes.c_int32
+    lib.ssm_scan_checkpoint_steps.argtypes = []
+    lib.ssm_status_string.restype = ctypes.c_char_p
+    lib.ssm_status_string.argtypes = [ctypes.c_int]
+    lib.ssm_scan_plan.restype = ctypes.c_int
+    lib.ssm_scan_plan.argtypes = [P] + [ctypes.POINTER(ctypes.c_int32)] * 4
+    lib.ssm_scan_fwd.restype = ctypes.c_int
+    lib.ssm_scan_fwd.argtypes = [P] + [vp] * 9 + [vp, sz, vp]
+    lib.ssm_scan_bwd.restype = ctypes.c_int
+    lib.ssm_scan_bwd.argtypes = [P] + [vp] * 16 + [vp, sz, vp]
+    _lib = lib
+    return lib
+
+
+def status_string(code: int) -> str:
+    return load_library().ssm_status_string(int(code)).decode()
+
+
+def _check(code: int, what: str) -> None:
+    if code != SSM_OK:
+        raise SsmScanError(f"{what}: {status_string(code)}")
+
+
+def _io_dtype(t: torch.Tensor) -> int:
+    if t.dtype == torch.float32:
+        return SSM_F32
+    if t.dtype == torch.bfloat16:
+        return SSM_BF16
+    raise SsmScanError(f"io dtype must be float32 or bfloat16, got {t.dtype}")
+
+
+def make_problem(x: torch.Tensor, B: torch.Tensor, has_z: bool, has_dskip: bool, save_states: bool = False,
+                 general_A: bool = False) -> ssm_problem_t:
+    batch, L, D = x.shape
+    flags = (SSM_FLAG_HAS_Z if has_z else 0) | (SSM_FLAG_HAS_DSKIP if has_dskip else 0) \
+        | (SSM_FLAG_SAVE_STATES if save_states else 0) | (SSM_FLAG_GENERAL_A if general_A else 0)
+    return ssm_problem_t(batch, L, D, B.shape[-1], _io_dtype(x), flags)
+
+
+def _dev_ptr(t, name, shape=None, dtype=None):
+    if t is None:
+        return None
+    if not t.is_cuda:
+        raise SsmScanError(f"{name} must be a CUDA tensor")
+    if not t.is_contiguous():
+        raise SsmScanError(f"{name} must be contiguous")
+    if shape is not None and tuple(t.shape) != tuple(shape):
+        raise SsmScanError(f"{name} has shape {tuple(t.shape)}, expected {tuple(shape)}")
+    if dtype is not None and t.dtype != dtype:
+        raise SsmScanError(f"{name} has dtype {t.dtype}, expected {dtype}")
+    return ctypes.c_void_p(t.data_ptr())
+
+
+_workspaces: dict = {}
+
+
+def _workspace(nbytes: int, device, stream_ptr: int) -> torch.Tensor | None:
+    """Grow-only scratch buffer per (device, stream): calls on different streams never share scratch memory."""
+    if nbytes == 0:
+        return None
+    key = (str(device), int(stream_ptr))
+    ws = _workspaces.get(key)
+    if ws is None or ws.numel() < nbytes:
+        ws = torch.empty(nbytes, dtype=torch.uint8, device=device)
+        _workspaces[key] = ws
+    return ws
+
+
+def plan(problem: ssm_problem_t) -> dict:
+    lib = load_library()
+    v = [ctypes.c_int32() for _ in range(4)]
+    _check(lib.ssm_scan_plan(ctypes.byref(problem), *[ctypes.byref(c) for c in v]), "ssm_scan_plan")
+    return dict(zip(("n_segments", "segment_steps", "channels_per_block", "states_per_thread"), [c.value for c in v]))
+
+
+def checkpoint_steps() -> int:
+    return int(load_library().ssm_scan_checkpoint_steps())
+
+
+def fwd_workspace_bytes(problem: ssm_problem_t) -> int:
+    return int(load_library().ssm_scan_fwd_workspace_bytes(ctypes.byref(problem)))
+
+
+def bwd_workspace_bytes(problem: ssm_problem_t) -> int:
+    return int(load_library().ssm_scan_bwd_workspace_bytes(ctypes.byref(problem)))
+
+
+def saved_state_bytes(problem: ssm_problem_t) -> int:
+    return int(load_library().ssm_scan_saved_state_bytes(ctypes.byref(problem)))
+
+
+def ssm_scan_fwd(x, delta, A, B, C, D_skip=None, z=None, *, save_states=False, general_A=False, out=None,
+                 saved_states=None, workspace=None, stream=None):
+    """out = selective_scan(x, delta, A, B, C) (+ D_skip * x) (* silu(z)); see include/ssm_scan.h.
+
+    x, delta, z: (batch, L, D) io dtype; B, C: (batch, L, N) io dtype; A: (D, N) float32; D_skip: (D) float32.
+    Returns `out`, or `(out, saved_states)` with save_states=True.  Enqueues on `stream` (default: torch's current
+    stream) and does not synchronise.
+    """
+    lib = load_library()
+    prob = make_problem(x, B, z is not None, D_skip is not None, save_states, general_A)
+    batch, L, D, N = prob.batch, prob.L, prob.D, prob.N
+    io = x.dtype
+    if out is None:
+        out = torch.empty_like(x)
+    if save_states and saved_states is None:
+        saved_states = torch.empty(saved_state_bytes(prob) // 4, dtype=torch.float32, device=x.device)
+    stream_ptr = (stream if stream is not None else torch.cuda.current_stream(x.device)).cuda_stream
+    need = fwd_workspace_bytes(prob)
+    ws = workspace if workspace is not None else _workspace(need, x.device, stream_ptr)
+    code = lib.ssm_scan_fwd(
+        ctypes.byref(prob), _dev_ptr(x, "x", (batch, L, D), io), _dev_ptr(delta, "delta", (batch, L, D), io),
+        _dev_ptr(A, "A", (D, N), torch.float32), _dev_ptr(B, "B", (batch, L, N), io),
+        _dev_ptr(C, "C", (batch, L, N), io), _dev_ptr(D_skip, "D_skip", (D,), torch.float32),
+        _dev_ptr(z, "z", (batch, L, D), io), _dev_ptr(out, "out", (batch, L, D), io),
+        _dev_ptr(saved_states if save_states else None, "saved_states"),
+        _dev_ptr(ws, "workspace"), ctypes.c_size_t(0 if ws is None else ws.numel() * ws.element_size()),
+        ctypes.c_void_p(stream_ptr))
+    _check(code, "ssm_scan_fwd")
+    return (out, saved_states) if save_states else out
+
+
+def ssm_scan_bwd(x, delta, A, B, C, D_skip, z, dout, saved_states=None, *, general_A=False, workspace=None,
+                 stream=None, outputs=None):
+    """Gradients of sum(dout * out) w.r.t. x, delta, A, B, C, D_skip, z; see include/ssm_scan.h.
+
+    Returns a dict with dx, ddelta, dz (io dtype, (batch, L, D)); dB, dC (io dtype, (batch, L, N)); dA (float32, (D, N));
+    dD (float32, (D)).  dz / dD are None when z / D_skip is None.  `outputs` may pass preallocated tensors.
+    """
+    lib = load_library()
+    prob = make_problem(x, B, z is not None, D_skip is not None, False, general_A)
+    batch, L, D, N = prob.batch, prob.L, prob.D, prob.N
+    io = x.dtype
+    o = dict(outputs or {})
+    o.setdefault("dx", torch.empty_like(x))
+    o.setdefault("ddelta", torch.empty_like(x))
+    o.setdefault("dA", torch.empty((D, N), dtype=torch.float32, device=x.device))
+    o.setdefault("dB", torch.empty_like(B))
+    o.setdefault("dC", torch.empty_like(B))
+    if D_skip is not None:
+        o.setdefault("dD", torch.empty((D,), dtype=torch.float32, device=x.device))
+    else:
+        o["dD"] = None
+    if z is not None:
+        o.setdefault("dz", torch.empty_like(x))
+    else:
+        o["dz"] = None
+    stream_ptr = (stream if stream is not None else torch.cuda.current_stream(x.device)).cuda_stream
+    need = bwd_workspace_bytes(prob)
+    ws = workspace if workspace is not None else _workspace(need, x.device, stream_ptr)
+    code = lib.ssm_scan_bwd(
+        ctypes.byref(prob), _dev_ptr(x, "x", (batch, L, D), io), _dev_ptr(delta, "delta", (batch, L, D), io),
+        _dev_ptr(A, "A", (D, N), torch.float32), _dev_ptr(B, "B", (batch, L, N), io),
+        _dev_ptr(C, "C", (batch, L, N), io), _dev_ptr(D_skip, "D_skip", (D,), torch.float32),
+        _dev_ptr(z, "z", (batch, L, D), io), _dev_ptr(dout, "dout", (batch, L, D), io),
+        _dev_ptr(saved_states, "saved_states"),
+        _dev_ptr(o["dx"], "dx", (batch, L, D), io), _dev_ptr(o["ddelta"], "ddelta", (batch, L, D), io),
+        _dev_ptr(o["dA"], "dA", (D, N), torch.float32), _dev_ptr(o["dB"], "dB", (batch, L, N), io),
+        _dev_ptr(o["dC"], "dC", (batch, L, N), io), _dev_ptr(o["dD"], "dD", (D,), torch.float32),
+        _dev_ptr(o["dz"], "dz", (batch, L, D), io),
+        _dev_ptr(ws, "workspace"), ctypes.c_size_t(0 if ws is None else ws.numel() * ws.element_size()),
+        ctypes.c_void_p(stream_ptr))
+    _check(code, "ssm_scan_bwd")
+    return o

@@ -1,0 +1,327 @@
+// C ABI of the selective-scan library: argument validation, the time-split plan, the workspace layout and the
+// launch sequences.  See include/ssm_scan.h for the contract of every entry point.
+#include <algorithm>
+
+#include "ssm_common.cuh"
+
+namespace ssm {
+
+int fwd_channels_per_block(int N);
+int bwd_channels_per_block(int N);
+
+static inline size_t align_up(size_t v) { return (v + 255) & ~(size_t)255; }
+
+static ssm_status_t validate_problem(const ssm_problem_t* p) {
+  if (p == nullptr) return SSM_ERR_INVALID_ARG;
+  if (p->batch < 1 || p->L < 1 || p->D < 1 || p->N < 1) return SSM_ERR_INVALID_ARG;
+  if (p->flags & ~(uint32_t)(SSM_FLAG_HAS_Z | SSM_FLAG_HAS_DSKIP | SSM_FLAG_SAVE_STATES | SSM_FLAG_GENERAL_A))
+    return SSM_ERR_INVALID_ARG;
+  if (p->io_dtype != SSM_F32 && p->io_dtype != SSM_BF16) return SSM_ERR_UNSUPPORTED;
+  if (p->N != 1 && p->N != 2 && p->N != 4 && p->N != 8 && p->N != 16) return SSM_ERR_UNSUPPORTED;
+  if (p->batch > 65535) return SSM_ERR_UNSUPPORTED;  // batch is a grid z dimension
+  return SSM_OK;
+}
+
+// The sequence is split in time only when (batch, channel, state) parallelism alone would leave most of the GPU
+// idle: every time segment but the first costs one extra sweep of the recurrence.
+Plan make_plan(const ssm_problem_t& p) {
+  Plan pl{};
+  pl.nck = (p.L + kCkptSteps - 1) / kCkptSteps;
+  pl.fwd_cpt = 2;
+  pl.fwd_ch = fwd_channels_per_block(p.N);
+  pl.bwd_ch = bwd_channels_per_block(p.N);
+  pl.bwd_groups = (p.D + pl.bwd_ch - 1) / pl.bwd_ch;
+  const int S = p.N < 4 ? p.N : 4;
+  const long long groups = (long long)p.batch * ((p.D + pl.fwd_cpt - 1) / pl.fwd_cpt);  // thread groups
+  const long long warps = std::max<long long>(1, groups * (p.N / S) / 32);
+  const long long sub_partitions = 4LL * kNumSMs;
+  int nseg = 1;
+  if (warps < sub_partitions * 3 / 4) {
+    const long long want = (6 * sub_partitions + warps - 1) / warps;
+    const long long max_by_len = std::max(1, p.L / (4 * kCkptSteps));
+    nseg = (int)std::min<long long>(std::min(want, max_by_len), 65535);
+  }
+  int seg_steps = (p.L + nseg - 1) / nseg;
+  seg_steps = (seg_steps + kCkptSteps - 1) / kCkptSteps * kCkptSteps;
+  pl.seg_steps = seg_steps;
+  pl.nseg = (p.L + seg_steps - 1) / seg_steps;
+  return pl;
+}
+
+struct FwdWorkspace {
+  size_t seg_end, seg_dsum, h_start, total;
+};
+static FwdWorkspace fwd_layout(const ssm_problem_t& p, const Plan& pl) {
+  FwdWorkspace w{};
+  if (pl.nseg > 1) {
+    const size_t st = (size_t)p.batch * pl.nseg * p.D * p.N * sizeof(float);
+    w.seg_end = 0;
+    w.h_start = align_up(st);
+    w.seg_dsum = w.h_start + align_up(st);
+    w.total = w.seg_dsum + align_up((size_t)p.batch * pl.nseg * p.D * sizeof(float));
+  }
+  return w;
+}
+
+struct BwdWorkspace {
+  size_t dBC_part, dA_part, dD_part, ckpt, seg_local, seg_dsum, mu_in, fwd, total;
+};
+static BwdWorkspace bwd_layout(const ssm_problem_t& p, const Plan& pl) {
+  BwdWorkspace w{};
+  size_t off = 0;
+  auto take = [&](size_t bytes) {
+    const size_t at = off;
+    off += align_up(bytes);
+    return at;
+  };
+  const size_t bln = (size_t)p.batch * p.L * p.N;
+  const size_t parts = (size_t)p.batch * pl.nseg;
+  w.dBC_part = take((size_t)pl.bwd_groups * 2 * bln * sizeof(float));
+  w.dA_part = take(parts * p.D * p.N * sizeof(float));
+  w.dD_part = take(parts * p.D * sizeof(float));
+  w.ckpt = take((size_t)p.batch * pl.nck * p.D * p.N * sizeof(float));
+  if (pl.nseg > 1) {
+    const size_t st = parts * p.D * p.N * sizeof(float);
+    w.seg_local = take(st);
+    w.mu_in = take(st);
+    w.seg_dsum = take(parts * p.D * sizeof(float));
+  }
+  w.fwd = take(fwd_layout(p, pl).total);
+  w.total = off;
+  return w;
+}
+
+static bool aligned_to(const void* ptr, size_t a) { return (reinterpret_cast<uintptr_t>(ptr) % a) == 0; }
+
+static ssm_status_t check_ws(const void* ws, size_t have, size_t need) {
+  if (need == 0) return SSM_OK;
+  if (ws == nullptr || !aligned_to(ws, 256) || have < need) return SSM_ERR_WORKSPACE;
+  return SSM_OK;
+}
+
+// Runs the passes that establish the state at the start of every segment (nothing to do without a time split).
+static cudaError_t run_segment_starts(const ssm_problem_t& prob, const Plan& pl, FwdParams fp, char* ws,
+                                      const float** h_start, cudaStream_t s) {
+  *h_start = nullptr;
+  if (pl.nseg == 1) return cudaSuccess;
+  const FwdWorkspace w = fwd_layout(prob, pl);
+  fp.seg_end = reinterpret_cast<float*>(ws + w.seg_end);
+  fp.seg_dsum = reinterpret_cast<float*>(ws + w.seg_dsum);
+  fp.h_start = nullptr;
+  fp.ckpt = nullptr;
+  cudaError_t e = launch_fwd(prob, pl, fp, kFwdSummary, s);
+  if (e != cudaSuccess) return e;
+  CarryParams cp{};
+  cp.local = fp.seg_end;
+  cp.dsum = fp.seg_dsum;
+  cp.A = fp.A;
+  cp.carried = reinterpret_cast<float*>(ws + w.h_start);
+  cp.batch = prob.batch;
+  cp.nseg = pl.nseg;
+  cp.D = prob.D;
+  cp.N = prob.N;
+  cp.reverse = 0;
+  e = launch_carry(cp, s);
+  *h_start = cp.carried;
+  return e;
+}
+
+}  // namespace ssm
+
+using namespace ssm;
+
+extern "C" {
+
+size_t ssm_scan_fwd_workspace_bytes(const ssm_problem_t* p) {
+  if (validate_problem(p) != SSM_OK) return 0;
+  return fwd_layout(*p, make_plan(*p)).total;
+}
+
+size_t ssm_scan_bwd_workspace_bytes(const ssm_problem_t* p) {
+  if (validate_problem(p) != SSM_OK) return 0;
+  return bwd_layout(*p, make_plan(*p)).total;
+}
+
+size_t ssm_scan_saved_state_bytes(const ssm_problem_t* p) {
+  if (validate_problem(p) != SSM_OK) return 0;
+  const size_t nck = (size_t)(p->L + kCkptSteps - 1) / kCkptSteps;
+  return (size_t)p->batch * nck * p->D * p->N * sizeof(float);
+}
+
+int32_t ssm_scan_checkpoint_steps(void) { return kCkptSteps; }
+
+const char* ssm_status_string(ssm_status_t s) {
+  switch (s) {
+    case SSM_OK: return "SSM_OK";
+    case SSM_ERR_INVALID_ARG: return "SSM_ERR_INVALID_ARG: null or misaligned pointer, bad dimension or flag";
+    case SSM_ERR_UNSUPPORTED: return "SSM_ERR_UNSUPPORTED: N must be 1, 2, 4, 8 or 16 and io_dtype f32 or bf16";
+    case SSM_ERR_WORKSPACE: return "SSM_ERR_WORKSPACE: workspace missing, misaligned or too small";
+    case SSM_ERR_CUDA: return "SSM_ERR_CUDA: a CUDA call or kernel launch failed";
+    case SSM_ERR_TIMEOUT: return "SSM_ERR_TIMEOUT: a bounded device-side wait gave up";
+    default: return "unknown ssm_status_t";
+  }
+}
+
+ssm_status_t ssm_scan_plan(const ssm_problem_t* p, int32_t* n_segments, int32_t* segment_steps,
+                           int32_t* channels_per_block, int32_t* states_per_thread) {
+  const ssm_status_t st = validate_problem(p);
+  if (st != SSM_OK) return st;
+  const Plan pl = make_plan(*p);
+  if (n_segments) *n_segments = pl.nseg;
+  if (segment_steps) *segment_steps = pl.seg_steps;
+  if (channels_per_block) *channels_per_block = pl.fwd_ch;
+  if (states_per_thread) *states_per_thread = p->N < 4 ? p->N : 4;
+  return SSM_OK;
+}
+
+ssm_status_t ssm_scan_fwd(const ssm_problem_t* p, const void* x, const void* delta, const float* A, const void* B,
+                          const void* C, const float* D_skip, const void* z, void* out, void* saved_states,
+                          void* workspace, size_t workspace_bytes, void* stream) {
+  ssm_status_t st = validate_problem(p);
+  if (st != SSM_OK) return st;
+  const bool has_z = p->flags & SSM_FLAG_HAS_Z, has_d = p->flags & SSM_FLAG_HAS_DSKIP;
+  const bool save = p->flags & SSM_FLAG_SAVE_STATES;
+  if (!x || !delta || !A || !B || !C || !out) return SSM_ERR_INVALID_ARG;
+  if ((has_z && !z) || (has_d && !D_skip) || (save && !saved_states)) return SSM_ERR_INVALID_ARG;
+  const size_t esz = p->io_dtype == SSM_BF16 ? 2 : 4;
+  for (const void* q : {x, delta, B, C, z, (const void*)out})
+    if (q && !aligned_to(q, esz)) return SSM_ERR_INVALID_ARG;
+  for (const void* q : {(const void*)A, (const void*)D_skip, (const void*)saved_states})
+    if (q && !aligned_to(q, 4)) return SSM_ERR_INVALID_ARG;
+  const Plan pl = make_plan(*p);
+  st = check_ws(workspace, workspace_bytes, fwd_layout(*p, pl).total);
+  if (st != SSM_OK) return st;
+
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  FwdParams fp{};
+  fp.x = x;
+  fp.delta = delta;
+  fp.z = has_z ? z : nullptr;
+  fp.B = B;
+  fp.C = C;
+  fp.A = A;
+  fp.Dskip = has_d ? D_skip : nullptr;
+  fp.out = out;
+  fp.batch = p->batch;
+  fp.L = p->L;
+  fp.D = p->D;
+  fp.nseg = pl.nseg;
+  fp.seg_steps = pl.seg_steps;
+  fp.nck = pl.nck;
+  fp.general_A = (p->flags & SSM_FLAG_GENERAL_A) ? 1 : 0;
+  const float* h_start = nullptr;
+  if (run_segment_starts(*p, pl, fp, static_cast<char*>(workspace), &h_start, s) != cudaSuccess) return SSM_ERR_CUDA;
+  fp.h_start = h_start;
+  fp.ckpt = save ? static_cast<float*>(saved_states) : nullptr;
+  if (launch_fwd(*p, pl, fp, kFwdFull, s) != cudaSuccess) return SSM_ERR_CUDA;
+  return SSM_OK;
+}
+
+ssm_status_t ssm_scan_bwd(const ssm_problem_t* p, const void* x, const void* delta, const float* A, const void* B,
+                          const void* C, const float* D_skip, const void* z, const void* dout,
+                          const void* saved_states, void* dx, void* ddelta, float* dA, void* dB, void* dC, float* dD,
+                          void* dz, void* workspace, size_t workspace_bytes, void* stream) {
+  ssm_status_t st = validate_problem(p);
+  if (st != SSM_OK) return st;
+  const bool has_z = p->flags & SSM_FLAG_HAS_Z, has_d = p->flags & SSM_FLAG_HAS_DSKIP;
+  if (!x || !delta || !A || !B || !C || !dout || !dx || !ddelta || !dA || !dB || !dC) return SSM_ERR_INVALID_ARG;
+  if ((has_z && !z) || (has_d && !D_skip)) return SSM_ERR_INVALID_ARG;
+  const size_t esz = p->io_dtype == SSM_BF16 ? 2 : 4;
+  for (const void* q : {x, delta, B, C, z, dout, (const void*)dx, (const void*)ddelta, (const void*)dB,
+                        (const void*)dC, (const void*)dz})
+    if (q && !aligned_to(q, esz)) return SSM_ERR_INVALID_ARG;
+  for (const void* q : {(const void*)A, (const void*)D_skip, saved_states, (const void*)dA, (const void*)dD})
+    if (q && !aligned_to(q, 4)) return SSM_ERR_INVALID_ARG;
+  const Plan pl = make_plan(*p);
+  const BwdWorkspace w = bwd_layout(*p, pl);
+  st = check_ws(workspace, workspace_bytes, w.total);
+  if (st != SSM_OK) return st;
+
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  char* ws = static_cast<char*>(workspace);
+
+  // checkpoint states: the caller's, or rebuilt here with one more forward sweep
+  const float* ckpt = static_cast<const float*>(saved_states);
+  if (ckpt == nullptr) {
+    FwdParams fp{};
+    fp.x = x;
+    fp.delta = delta;
+    fp.B = B;
+    fp.C = C;
+    fp.A = A;
+    fp.batch = p->batch;
+    fp.L = p->L;
+    fp.D = p->D;
+    fp.nseg = pl.nseg;
+    fp.seg_steps = pl.seg_steps;
+    fp.nck = pl.nck;
+    fp.general_A = (p->flags & SSM_FLAG_GENERAL_A) ? 1 : 0;
+    const float* h_start = nullptr;
+    if (run_segment_starts(*p, pl, fp, ws + w.fwd, &h_start, s) != cudaSuccess) return SSM_ERR_CUDA;
+    fp.h_start = h_start;
+    fp.ckpt = reinterpret_cast<float*>(ws + w.ckpt);
+    if (launch_fwd(*p, pl, fp, kFwdCkptOnly, s) != cudaSuccess) return SSM_ERR_CUDA;
+    ckpt = fp.ckpt;
+  }
+
+  BwdParams bp{};
+  bp.x = x;
+  bp.delta = delta;
+  bp.z = has_z ? z : nullptr;
+  bp.B = B;
+  bp.C = C;
+  bp.A = A;
+  bp.Dskip = has_d ? D_skip : nullptr;
+  bp.dout = dout;
+  bp.ckpt = ckpt;
+  bp.dx = dx;
+  bp.ddelta = ddelta;
+  bp.dz = has_z ? dz : nullptr;
+  bp.dBC_part = reinterpret_cast<float*>(ws + w.dBC_part);
+  bp.dA_part = reinterpret_cast<float*>(ws + w.dA_part);
+  bp.dD_part = reinterpret_cast<float*>(ws + w.dD_part);
+  bp.batch = p->batch;
+  bp.L = p->L;
+  bp.D = p->D;
+  bp.nseg = pl.nseg;
+  bp.seg_steps = pl.seg_steps;
+  bp.nck = pl.nck;
+  bp.groups = pl.bwd_groups;
+
+  if (pl.nseg > 1) {
+    bp.seg_local = reinterpret_cast<float*>(ws + w.seg_local);
+    bp.seg_dsum = reinterpret_cast<float*>(ws + w.seg_dsum);
+    if (launch_bwd(*p, pl, bp, kBwdLocal, s) != cudaSuccess) return SSM_ERR_CUDA;
+    CarryParams cp{};
+    cp.local = bp.seg_local;
+    cp.dsum = bp.seg_dsum;
+    cp.A = A;
+    cp.carried = reinterpret_cast<float*>(ws + w.mu_in);
+    cp.batch = p->batch;
+    cp.nseg = pl.nseg;
+    cp.D = p->D;
+    cp.N = p->N;
+    cp.reverse = 1;
+    if (launch_carry(cp, s) != cudaSuccess) return SSM_ERR_CUDA;
+    bp.mu_in = cp.carried;
+  }
+  if (launch_bwd(*p, pl, bp, kBwdFull, s) != cudaSuccess) return SSM_ERR_CUDA;
+
+  ReduceParams rp{};
+  rp.dBC_part = bp.dBC_part;
+  rp.dB = dB;
+  rp.dC = dC;
+  rp.dA_part = bp.dA_part;
+  rp.dD_part = bp.dD_part;
+  rp.dA = dA;
+  rp.dD = has_d ? dD : nullptr;
+  rp.bln = (long long)p->batch * p->L * p->N;
+  rp.groups = pl.bwd_groups;
+  rp.parts = p->batch * pl.nseg;
+  rp.D = p->D;
+  rp.N = p->N;
+  if (launch_bwd_reduce(*p, rp, s) != cudaSuccess) return SSM_ERR_CUDA;
+  return SSM_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,141 @@
+// Shared declarations of the selective-scan kernels (sm_100a).  Internal to the library: nothing here is part of
+// the C ABI, and nothing here is used by the CPU oracle.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "ssm_scan.h"
+
+namespace ssm {
+
+// Time steps between two checkpoint states (the state h at the start of every such block is what backward restarts
+// its recomputation from).  Segment lengths of the time split are multiples of this.
+constexpr int kCkptSteps = 64;
+constexpr float kLog2e = 1.4426950408889634f;
+constexpr int kNumSMs = 148;
+
+// ---------------------------------------------------------------------------------------------- plan (host)
+struct Plan {
+  int nseg;        // time segments per sequence (1: a thread sweeps the whole sequence)
+  int seg_steps;   // steps per segment (multiple of kCkptSteps; the last segment may be shorter)
+  int nck;         // checkpoints per sequence = ceil(L / kCkptSteps)
+  int fwd_cpt;     // channels per thread, forward
+  int fwd_ch;      // channels per block, forward
+  int bwd_ch;      // channels per block, backward (= channel-group size of the dB/dC partial sums)
+  int bwd_groups;  // ceil(D / bwd_ch)
+};
+Plan make_plan(const ssm_problem_t& p);
+
+// ---------------------------------------------------------------------------------------------- kernel params
+struct FwdParams {
+  const void* x;
+  const void* delta;
+  const void* z;       // null: no gate
+  const void* B;
+  const void* C;
+  const float* A;
+  const float* Dskip;  // null: no skip term
+  void* out;           // FULL mode
+  const float* h_start;  // [batch][nseg][D][N] start state of each segment; null: zero
+  float* ckpt;           // [batch][nck][D][N] checkpoint states to write; null: none
+  float* seg_end;        // SUMMARY mode: [batch][nseg][D][N] end state of each segment started from zero
+  float* seg_dsum;       // SUMMARY mode: [batch][nseg][D] sum of delta over the segment
+  int batch, L, D, nseg, seg_steps, nck;
+  int general_A;       // 1: never take the arithmetic-progression fast path
+};
+
+struct CarryParams {
+  const float* local;   // [batch][nseg][D][N]: per-segment result computed with zero inflow (end state e, or l)
+  const float* dsum;    // [batch][nseg][D]: sum of delta over the segment
+  const float* A;       // [D][N]
+  float* carried;       // [batch][nseg][D][N]: inflow of each segment (forward: state before its first step;
+                        //                      reverse: adjoint flowing in from the following segment)
+  int batch, nseg, D, N;
+  int reverse;
+};
+
+struct BwdParams {
+  const void* x;
+  const void* delta;
+  const void* z;
+  const void* B;
+  const void* C;
+  const float* A;
+  const float* Dskip;
+  const void* dout;
+  const float* ckpt;      // [batch][nck][D][N]
+  const float* mu_in;     // [batch][nseg][D][N] adjoint inflow of each segment; null: zero
+  float* seg_local;       // LOCAL mode: [batch][nseg][D][N] adjoint leaving each segment with zero inflow
+  float* seg_dsum;        // LOCAL mode: [batch][nseg][D]
+  void* dx;
+  void* ddelta;
+  void* dz;               // null: not produced
+  float* dBC_part;        // [groups][2][batch*L*N] float partial sums over the channels of one block
+  float* dA_part;         // [batch*nseg][D][N]
+  float* dD_part;         // [batch*nseg][D]
+  int batch, L, D, nseg, seg_steps, nck, groups;
+};
+
+struct ReduceParams {
+  const float* dBC_part;  // [groups][2][rows*N]
+  void* dB;
+  void* dC;
+  const float* dA_part;   // [parts][D*N]
+  const float* dD_part;   // [parts][D]
+  float* dA;
+  float* dD;              // null: skip
+  long long bln;          // batch*L*N
+  int groups, parts, D, N;
+};
+
+cudaError_t launch_fwd(const ssm_problem_t& prob, const Plan& plan, const FwdParams& p, int mode, cudaStream_t s);
+cudaError_t launch_carry(const CarryParams& p, cudaStream_t s);
+cudaError_t launch_bwd(const ssm_problem_t& prob, const Plan& plan, const BwdParams& p, int mode, cudaStream_t s);
+cudaError_t launch_bwd_reduce(const ssm_problem_t& prob, const ReduceParams& p, cudaStream_t s);
+
+enum FwdMode { kFwdFull = 0, kFwdSummary = 1, kFwdCkptOnly = 2 };
+enum BwdMode { kBwdFull = 0, kBwdLocal = 1 };
+
+// ---------------------------------------------------------------------------------------------- device helpers
+#ifdef __CUDACC__
+__device__ __forceinline__ float ex2_approx(float v) {
+  float r;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(v));
+  return r;
+}
+__device__ __forceinline__ float rcp_approx(float v) {
+  float r;
+  asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(v));
+  return r;
+}
+
+template <typename IO>
+__device__ __forceinline__ float io_to_float(IO v);
+template <>
+__device__ __forceinline__ float io_to_float<float>(float v) { return v; }
+template <>
+__device__ __forceinline__ float io_to_float<__nv_bfloat16>(__nv_bfloat16 v) { return __bfloat162float(v); }
+
+template <typename IO>
+__device__ __forceinline__ IO float_to_io(float v);
+template <>
+__device__ __forceinline__ float float_to_io<float>(float v) { return v; }
+template <>
+__device__ __forceinline__ __nv_bfloat16 float_to_io<__nv_bfloat16>(float v) { return __float2bfloat16_rn(v); }
+
+// sigmoid(z) through one ex2 and one reciprocal
+__device__ __forceinline__ float sigmoid_fast(float z) { return rcp_approx(1.0f + ex2_approx(-kLog2e * z)); }
+
+// The associative operator of the recurrence h' = a h + b:  (a, b) o (a2, b2) = (a a2, a2 b + b2), i.e. "apply
+// (a, b) first, then (a2, b2)".
+struct AffinePair {
+  float a, b;
+};
+__device__ __forceinline__ AffinePair combine(AffinePair first, AffinePair second) {
+  return {first.a * second.a, fmaf(second.a, first.b, second.b)};
+}
+#endif
+
+}  // namespace ssm

@@ -1,0 +1,118 @@
+"""GPU parity on small shapes: the CUDA path through the C ABI against the fp64 oracle, element by element.
+
+Sizes are chosen so that the oracle takes well under a second while the kernels still see several tiles, ragged tails
+in time and in channels, every supported state size, both io dtypes, missing gate / skip term, and the time-split
+(segment carry) path in both directions.
+"""
+import numpy as np
+import pytest
+
+from paper_2312_00752_b200 import synth
+from tests import _gpu_util as U
+
+pytestmark = pytest.mark.gpu
+
+
+def _case(batch, L, D, N, io, dt=(1e-3, 1e-1), seed=0, cfg_id=9):
+    cfg = synth.ScanConfig("case", cfg_id, batch, L, D, N, io, dt[0], dt[1])
+    return cfg, synth.make_inputs(cfg, seed=seed)
+
+
+def test_config0_tiny_f32():
+    cfg = synth.CONFIGS[0]
+    inp = synth.make_inputs(cfg, seed=0)
+    dev = U.to_device(inp, cfg.io)
+    ref = U.oracle_fwd_bwd(inp)
+    for use_saved in (True, False):
+        got = U.gpu_fwd_bwd(dev, use_saved=use_saved)
+        U.assert_parity(got, ref, cfg.io, f"config0 saved={use_saved}")
+    got = U.gpu_fwd_bwd(dev, general_A=True)
+    U.assert_parity(got, ref, cfg.io, "config0 general-A path")
+
+
+@pytest.mark.parametrize("batch,L,D,N,io", [
+    (2, 100, 40, 16, "bf16"),     # ragged time tail, channel tail inside a block
+    (1, 1, 8, 16, "f32"),         # a single step
+    (3, 257, 24, 8, "f32"),       # one step past four checkpoint blocks
+    (2, 65, 7, 4, "bf16"),        # odd channel count
+    (1, 130, 33, 2, "f32"),
+    (2, 64, 70, 1, "bf16"),       # N = 1 (the setting of the gating theorem)
+    (1, 333, 129, 16, "f32"),     # channels straddle several blocks
+])
+def test_shapes_and_state_sizes(batch, L, D, N, io):
+    cfg, inp = _case(batch, L, D, N, io)
+    got = U.gpu_fwd_bwd(U.to_device(inp, io))
+    U.assert_parity(got, U.oracle_fwd_bwd(inp), io, f"{(batch, L, D, N, io)}")
+
+
+@pytest.mark.parametrize("gate,skip", [(False, True), (True, False), (False, False)])
+def test_optional_gate_and_skip(gate, skip):
+    cfg, inp = _case(2, 150, 48, 16, "f32")
+    if not gate:
+        inp["z"] = None
+    if not skip:
+        inp["D_skip"] = None
+    got = U.gpu_fwd_bwd(U.to_device(inp, "f32"))
+    assert (got["dz"] is None) == (not gate) and (got["dD"] is None) == (not skip)
+    U.assert_parity(got, U.oracle_fwd_bwd(inp), "f32", f"gate={gate} skip={skip}")
+
+
+@pytest.mark.parametrize("io,L,D", [("f32", 4096, 64), ("bf16", 5000, 40)])
+def test_time_split_carry(io, L, D):
+    """Few channels and a long sequence: the library splits time into segments and carries the state (forward) and
+    the adjoint (backward) across them."""
+    from paper_2312_00752_b200 import binding as K
+    cfg, inp = _case(1, L, D, 16, io, dt=(1e-4, 1e-2))
+    dev = U.to_device(inp, io)
+    plan = K.plan(K.make_problem(dev["x"], dev["B"], True, True))
+    assert plan["n_segments"] > 1
+    ref = U.oracle_fwd_bwd(inp)
+    for use_saved in (True, False):
+        got = U.gpu_fwd_bwd(dev, use_saved=use_saved)
+        U.assert_parity(got, ref, io, f"time split saved={use_saved}")
+
+
+def test_bitwise_determinism():
+    cfg, inp = _case(2, 700, 96, 16, "bf16")
+    dev = U.to_device(inp, "bf16")
+    a = U.gpu_fwd_bwd(dev)
+    for _ in range(3):
+        b = U.gpu_fwd_bwd(dev)
+        for k in a:
+            if a[k] is not None:
+                assert np.array_equal(a[k], b[k]), k
+
+
+def test_large_and_zero_steps():
+    """Section 3.5.2 limits on the device: a huge step resets the state, a zero step freezes it."""
+    cfg, inp = _case(1, 96, 16, 16, "f32")
+    inp["delta"][:, 10:20] = 50.0
+    inp["delta"][:, 40:60] = 0.0
+    got = U.gpu_fwd_bwd(U.to_device(inp, "f32"))
+    U.assert_parity(got, U.oracle_fwd_bwd(inp), "f32", "step-size limits")
+
+
+def test_outputs_outside_are_untouched():
+    """Guard bands around every output: the kernels write exactly the output extents."""
+    import torch
+    from paper_2312_00752_b200 import binding as K
+    cfg, inp = _case(2, 70, 24, 16, "bf16")
+    dev = U.to_device(inp, "bf16")
+    pad = 64
+
+    def guarded(like):
+        buf = torch.full((like.numel() + 2 * pad,), 7.0, dtype=like.dtype, device=like.device)
+        return buf, buf[pad:pad + like.numel()].view(like.shape)
+
+    gb_out, out = guarded(dev["x"])
+    K.ssm_scan_fwd(dev["x"], dev["delta"], dev["A"], dev["B"], dev["C"], dev["D_skip"], dev["z"], out=out)
+    bufs = {"out": gb_out}
+    outs = {}
+    for k, like in (("dx", dev["x"]), ("ddelta", dev["x"]), ("dz", dev["x"]), ("dB", dev["B"]), ("dC", dev["B"]),
+                    ("dA", dev["A"]), ("dD", dev["D_skip"])):
+        bufs[k], outs[k] = guarded(like)
+    K.ssm_scan_bwd(dev["x"], dev["delta"], dev["A"], dev["B"], dev["C"], dev["D_skip"], dev["z"], dev["dout"],
+                   outputs=outs)
+    torch.cuda.synchronize()
+    for k, b in bufs.items():
+        assert torch.all(b[:pad] == 7.0) and torch.all(b[-pad:] == 7.0), k

@@ -1,0 +1,74 @@
+"""Host-only checks of the C-ABI library: it loads, exports every declared symbol, and validates arguments before
+launching anything (no GPU needed: every call here returns before a CUDA call is made)."""
+import ctypes
+import os
+import re
+
+import pytest
+
+from paper_2312_00752_b200 import binding as K
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def _declared_symbols():
+    text = open(os.path.join(ROOT, "include", "ssm_scan.h")).read()
+    return sorted(set(re.findall(r"SSM_API[^;(]*?\b(ssm_\w+)\s*\(", text)))
+
+
+def test_library_exports_every_declared_symbol():
+    lib = K.load_library()
+    names = _declared_symbols()
+    assert set(names) == set(K.EXPORTED_SYMBOLS) and len(names) >= 8
+    for n in names:
+        assert getattr(lib, n) is not None
+
+
+def _prob(batch=2, L=100, D=64, N=16, io=K.SSM_BF16, flags=3):
+    return K.ssm_problem_t(batch, L, D, N, io, flags)
+
+
+def test_queries_and_plan():
+    assert K.checkpoint_steps() == 64
+    p = _prob(4, 2048, 5120)
+    assert K.saved_state_bytes(p) == 4 * 32 * 5120 * 16 * 4
+    pl = K.plan(p)
+    assert pl["n_segments"] == 1 and pl["segment_steps"] == 2048 and pl["states_per_thread"] == 4
+    assert K.fwd_workspace_bytes(p) == 0
+    assert K.bwd_workspace_bytes(p) > 0
+    long = _prob(1, 524288, 1536)
+    pl = K.plan(long)
+    assert pl["n_segments"] > 1 and pl["segment_steps"] % 64 == 0
+    assert pl["n_segments"] * pl["segment_steps"] >= 524288 > (pl["n_segments"] - 1) * pl["segment_steps"]
+    assert K.fwd_workspace_bytes(long) >= 2 * pl["n_segments"] * 1536 * 16 * 4
+
+
+@pytest.mark.parametrize("bad,code", [
+    (dict(N=3), 2), (dict(N=32), 2), (dict(io=5), 2), (dict(L=0), 1), (dict(batch=-1), 1), (dict(flags=1 << 9), 1),
+])
+def test_invalid_problems_are_rejected(bad, code):
+    lib = K.load_library()
+    p = _prob(**bad)
+    assert lib.ssm_scan_plan(ctypes.byref(p), None, None, None, None) == code
+    assert K.fwd_workspace_bytes(p) == 0 and K.bwd_workspace_bytes(p) == 0
+    one = ctypes.c_void_p(256)
+    assert lib.ssm_scan_fwd(ctypes.byref(p), one, one, one, one, one, one, one, one, None, None, 0, None) == code
+
+
+def test_null_misaligned_and_workspace_errors_before_launch():
+    lib = K.load_library()
+    p = _prob()
+    a = ctypes.c_void_p(4096)
+    args = [a] * 8
+    assert lib.ssm_scan_fwd(ctypes.byref(p), None, *args[1:], None, None, 0, None) == 1          # x missing
+    assert lib.ssm_scan_fwd(ctypes.byref(p), *args[:6], None, a, None, None, 0, None) == 1       # z flagged, missing
+    assert lib.ssm_scan_fwd(ctypes.byref(p), ctypes.c_void_p(4097), *args[1:], None, None, 0, None) == 1  # misaligned
+    ps = _prob(flags=7)
+    assert lib.ssm_scan_fwd(ctypes.byref(ps), *args, None, None, 0, None) == 1                   # saved_states missing
+    long = _prob(1, 524288, 1536)
+    assert lib.ssm_scan_fwd(ctypes.byref(long), *args, None, None, 0, None) == 3                 # workspace missing
+    assert lib.ssm_scan_fwd(ctypes.byref(long), *args, None, a, 16, None) == 3                   # workspace too small
+    b16 = [a] * 16
+    assert lib.ssm_scan_bwd(ctypes.byref(p), *b16, None, 0, None) == 3
+    assert lib.ssm_scan_bwd(ctypes.byref(p), *b16[:7], None, *b16[8:], None, 0, None) == 1       # dout missing
+    assert "WORKSPACE" in K.status_string(3) and K.status_string(0) == "SSM_OK"
