@@ -1,0 +1,347 @@
+#!/usr/bin/env python
+"""Benchmark of the selective-scan hot path (forward + backward) on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config I] [--impl ours|reference]
+
+A "step" is one pass of the whole hot path over one batch of synthetic input: ssm_scan_fwd (writing the checkpoint
+states) followed by ssm_scan_bwd, both through the C ABI.  The workload is the Mamba-2.8B layer shape
+(batch 4, L 2048, D 5120, N 16, bf16 io, fp32 state) unless --config picks another one.  The metric is elements/s
+with elements = batch * L * D.  One JSON line is printed by rank 0.
+
+With --impl reference the fp64 CPU oracle is timed instead, as it stands, on the host cores.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "selective-scan fwd+bwd elements/s (elements = batch*L*D); achieved HBM GB/s as % of measured B200 peak"
+FALLBACK_HBM_GBS = 6650.0
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--config", type=int, default=3, help="index into the five synthetic workloads")
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--general-A", action="store_true", help="perturb A so that no row is an arithmetic progression")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    return ap.parse_args()
+
+
+def algorithmic_bytes(cfg):
+    """Bytes the method itself must move per call (bf16/f32 io): forward reads x, delta, z, B, C and writes out;
+    backward reads x, delta, z, dout, B, C and writes dx, ddelta, dz, dB, dC; A, D_skip, dA, dD once."""
+    e = 2 if cfg.io == "bf16" else 4
+    el = cfg.elements
+    bln = cfg.batch * cfg.L * cfg.N
+    small = cfg.D * cfg.N * 4 + cfg.D * 4
+    fwd = 4 * e * el + 2 * e * bln + small
+    bwd = 7 * e * el + 4 * e * bln + 2 * small
+    return fwd, bwd
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs (read-only queries)."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.proc = None
+        self.lines = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.Q}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            threading.Thread(target=self._read, daemon=True).start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for ln in self.proc.stdout:
+            self.lines.append(ln.strip())
+
+    def stop(self) -> dict:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        time.sleep(0.15)
+        self.proc.terminate()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in self.lines:
+            parts = [p.strip() for p in ln.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0]))
+                mx.append(float(parts[1]))
+            except ValueError:
+                continue
+            for nm, v in zip(names, parts[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(nm)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def kernels_per_step(plan_info: dict) -> int:
+    """Kernel launches of one fwd (saving states) + bwd (given saved states) pass."""
+    if plan_info["n_segments"] == 1:
+        return 1 + 2            # forward; backward + reduction
+    return 3 + 4                # summary, carry, forward; local adjoint, carry, backward, reduction
+
+
+# ------------------------------------------------------------------------------------------------ oracle timing
+def time_oracle(cfg, host, budget_core_s=25.0):
+    """Times the fp64 oracle (fwd and fwd+bwd) on a bounded sample of the workload: whole batch entries, all channels
+    or the first `dsel` channels, sized for roughly `budget_core_s` core-seconds."""
+    from oracle import ssm_oracle as O
+    cores = O.threads_available()
+    est_core_s = cfg.elements * cfg.N * 45e-9            # ~45 ns per state step for fwd+bwd on one core
+    frac = min(1.0, budget_core_s / est_core_s)
+    if frac * cfg.batch >= 1.0:
+        nb, dsel = int(frac * cfg.batch), cfg.D
+    else:
+        nb, dsel = 1, min(cfg.D, max(64, int(cfg.D * frac * cfg.batch) // 64 * 64))
+    sl = lambda a: a[:nb, :, :dsel]
+    x, dl, z, g = sl(host["x"]), sl(host["delta"]), sl(host["z"]), sl(host["dout"])
+    B, C = host["B"][:nb], host["C"][:nb]
+    A, Dk = host["A"][:dsel], host["D_skip"][:dsel]
+    import numpy as np
+    x, dl, z, g = (np.ascontiguousarray(v) for v in (x, dl, z, g))
+    t0 = time.perf_counter()
+    O.scan_fwd(x, dl, A, B, C, D_skip=Dk, z=z)
+    t1 = time.perf_counter()
+    O.scan_bwd(x, dl, A, B, C, Dk, z, g)
+    t2 = time.perf_counter()
+    el = nb * cfg.L * dsel
+    return {"value": el / (t2 - t0), "unit": "elements/s", "cores": cores, "kind": "oracle",
+            "sample": f"batch entries 0..{nb - 1}, channels 0..{dsel - 1} of the workload ({el} elements), "
+                      f"fwd {t1 - t0:.2f} s + bwd {t2 - t1:.2f} s wall",
+            "fwd_elements_per_s": el / (t1 - t0)}
+
+
+def run_reference(args, cfg):
+    """The reference arm: the oracle, as it stands, on the host cores; rank 0 only."""
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    from paper_2312_00752_b200 import synth
+    host = synth.make_inputs(cfg, seed=0)
+    per_step = []
+    info = None
+    for i in range(args.warmup + args.steps):
+        info = time_oracle(cfg, host, budget_core_s=8.0)
+        if i >= args.warmup:
+            per_step.append(info["value"])
+        if sum(1.0 for _ in per_step) >= 1 and time.perf_counter() - _T0 > 240:
+            break
+    v = statistics.median(per_step)
+    line = {"impl": "reference", "metric": METRIC, "value": v, "unit": "elements/s", "n_gpus": args.gpus,
+            "steps": len(per_step), "warmup": args.warmup, "ms_per_step": None, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": cfg.name, "batch": cfg.batch, "L": cfg.L, "D": cfg.D, "N": cfg.N, "io": cfg.io},
+            "cpu_baseline": {"value": v, "unit": "elements/s", "cores": info["cores"], "kind": "oracle",
+                             "sample": info["sample"]},
+            "e2e": {"value": v, "unit": "elements/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+# ------------------------------------------------------------------------------------------------ our arm
+def run_ours(args, cfg):
+    import numpy as np
+    import torch
+    import torch.distributed as dist
+    from paper_2312_00752_b200 import binding as K, synth
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    assert torch.cuda.is_available(), "bench.py needs a CUDA device; there is no CPU fallback"
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    K.load_library()
+    io_t = torch.bfloat16 if cfg.io == "bf16" else torch.float32
+    # every rank owns a batch of the same shape (weak scaling, no data-path collective); ranks differ by seed
+    host = synth.make_inputs(cfg, seed=rank, perturb_A=0.01 if args.general_A else 0.0)
+    pinned = {k: torch.from_numpy(v).to(io_t if k not in ("A", "D_skip") else torch.float32).pin_memory()
+              for k, v in host.items()}
+    NSETS = 3
+    sets = []
+    for _ in range(NSETS):
+        sets.append({k: v.to(dev, non_blocking=True) for k, v in pinned.items()})
+    d0 = sets[0]
+    prob = K.make_problem(d0["x"], d0["B"], True, True, save_states=True)
+    plan_info = K.plan(prob)
+    out = torch.empty_like(d0["x"])
+    saved = torch.empty(K.saved_state_bytes(prob) // 4, dtype=torch.float32, device=dev)
+    grads = {"dx": torch.empty_like(d0["x"]), "ddelta": torch.empty_like(d0["x"]), "dz": torch.empty_like(d0["x"]),
+             "dB": torch.empty_like(d0["B"]), "dC": torch.empty_like(d0["B"]),
+             "dA": torch.empty_like(d0["A"]), "dD": torch.empty_like(d0["D_skip"])}
+    stream = torch.cuda.current_stream(dev)
+
+    def fwd(s):
+        K.ssm_scan_fwd(s["x"], s["delta"], s["A"], s["B"], s["C"], s["D_skip"], s["z"], save_states=True, out=out,
+                       saved_states=saved, stream=stream)
+
+    def bwd(s):
+        K.ssm_scan_bwd(s["x"], s["delta"], s["A"], s["B"], s["C"], s["D_skip"], s["z"], s["dout"], saved,
+                       outputs=grads, stream=stream)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize(dev)
+
+    for i in range(max(args.warmup, 3)):
+        fwd(sets[i % NSETS])
+        bwd(sets[i % NSETS])
+    barrier()
+
+    # ---- device-resident timing: K steps, CUDA events on the launching stream
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
+    sampler = ClockSampler(local)
+    sampler.start()
+    time.sleep(0.3)
+    barrier()
+    t_wall = time.perf_counter()
+    for i in range(args.steps):
+        s = sets[i % NSETS]
+        ev[i][0].record(stream)
+        fwd(s)
+        ev[i][1].record(stream)
+        bwd(s)
+        ev[i][2].record(stream)
+    barrier()
+    t_wall = time.perf_counter() - t_wall
+    clocks = sampler.stop()
+    total_ms = ev[0][0].elapsed_time(ev[-1][2])
+    fwd_ms = [e[0].elapsed_time(e[1]) for e in ev]
+    bwd_ms = [e[1].elapsed_time(e[2]) for e in ev]
+    ms_per_step = total_ms / args.steps
+    if world > 1:
+        t = torch.tensor([ms_per_step], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_per_step = float(t.item())
+
+    # ---- end to end: pinned host inputs -> device, fwd + bwd, every result back to pinned host memory
+    e2e = None
+    if not args.no_e2e:
+        hres = {k: torch.empty(v.shape, dtype=v.dtype).pin_memory() for k, v in {"out": out, **grads}.items()}
+        names_in = ("x", "delta", "z", "dout", "B", "C", "A", "D_skip")
+        h2d = sum(pinned[k].numel() * pinned[k].element_size() for k in names_in)
+        d2h = sum(v.numel() * v.element_size() for v in hres.values())
+        es = sets[0]
+
+        def e2e_step():
+            for k in names_in:
+                es[k].copy_(pinned[k], non_blocking=True)
+            fwd(es)
+            bwd(es)
+            hres["out"].copy_(out, non_blocking=True)
+            for k, v in grads.items():
+                hres[k].copy_(v, non_blocking=True)
+
+        e2e_step()
+        barrier()
+        n_e2e = max(3, min(args.steps, 10))
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        for _ in range(n_e2e):
+            e2e_step()
+        b.record(stream)
+        barrier()
+        e2e_ms = a.elapsed_time(b) / n_e2e
+        if world > 1:
+            t = torch.tensor([e2e_ms], device=dev, dtype=torch.float64)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            e2e_ms = float(t.item())
+        e2e = {"value": world * cfg.elements / (e2e_ms * 1e-3), "unit": "elements/s",
+               "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h), "ms_per_step": e2e_ms,
+               "steps": n_e2e}
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    fwd_bytes, bwd_bytes = algorithmic_bytes(cfg)
+    peak, peak_kind = measured_peaks()
+    f_ms, b_ms = statistics.mean(fwd_ms), statistics.mean(bwd_ms)
+    bwd_gbs = bwd_bytes / (b_ms * 1e-3) / 1e9
+    fwd_gbs = fwd_bytes / (f_ms * 1e-3) / 1e9
+    line = {
+        "metric": METRIC, "value": world * cfg.elements / (ms_per_step * 1e-3), "unit": "elements/s",
+        "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": f"{cfg.name} (config {cfg.cfg_id}): batch {cfg.batch}, L {cfg.L}, D {cfg.D}, N {cfg.N}, "
+                               f"{cfg.io} io, fp32 state; one step = ssm_scan_fwd (saving checkpoint states) + ssm_scan_bwd",
+                   "batch": cfg.batch, "L": cfg.L, "D": cfg.D, "N": cfg.N, "io": cfg.io,
+                   "A": "perturbed (general path)" if args.general_A else "S4D-Real -(n+1)",
+                   "l2": f"inputs larger than L2 (4 x {cfg.elements * (2 if cfg.io == 'bf16' else 4) / 1e6:.0f} MB) and "
+                         f"{NSETS} input sets rotated between steps",
+                   "plan": plan_info, "parallelism": "replicas" if world > 1 else "single"},
+        "clocks": clocks,
+        "gpu_launches": kernels_per_step(plan_info) * args.steps,
+        "fwd": {"ms": f_ms, "elements_per_s": cfg.elements / (f_ms * 1e-3), "algorithmic_bytes": fwd_bytes,
+                "achieved_gbs": fwd_gbs, "frac_of_hbm_peak": fwd_gbs / peak},
+        "bwd": {"ms": b_ms, "elements_per_s": cfg.elements / (b_ms * 1e-3), "algorithmic_bytes": bwd_bytes,
+                "achieved_gbs": bwd_gbs, "frac_of_hbm_peak": bwd_gbs / peak},
+        "roofline": {"bound": "hbm", "kernel": "ssm_scan_bwd call (backward kernel + its reduction kernel)",
+                     "achieved": bwd_gbs, "peak": peak, "peak_kind": f"{peak_kind} copy bandwidth",
+                     "unit": "GB/s", "frac": bwd_gbs / peak, "traffic": None},
+        "wall_s_timed_region": t_wall,
+    }
+    if e2e is not None:
+        line["e2e"] = e2e
+    if not args.no_cpu_baseline and world >= 1:
+        line["cpu_baseline"] = time_oracle(cfg, host)
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+_T0 = time.perf_counter()
+
+
+def main():
+    args = parse_args()
+    from paper_2312_00752_b200 import synth
+    cfg = synth.CONFIGS[args.config]
+    if args.impl == "reference":
+        run_reference(args, cfg)
+    else:
+        run_ours(args, cfg)
+
+
+if __name__ == "__main__":
+    main()
