@@ -38,7 +38,7 @@ Plan make_plan(const ssm_problem_t& p) {
   int nseg = 1;
   if (warps < sub_partitions * 3 / 4) {
     const long long want = (6 * sub_partitions + warps - 1) / warps;
-    const long long max_by_len = std::max(1, p.L / (4 * kCkptSteps));
+    const long long max_by_len = std::max(1, p.L / 256);
     nseg = (int)std::min<long long>(std::min(want, max_by_len), 65535);
   }
   int seg_steps = (p.L + nseg - 1) / nseg;
@@ -287,6 +287,7 @@ ssm_status_t ssm_scan_bwd(const ssm_problem_t* p, const void* x, const void* del
   bp.seg_steps = pl.seg_steps;
   bp.nck = pl.nck;
   bp.groups = pl.bwd_groups;
+  bp.general_A = (p->flags & SSM_FLAG_GENERAL_A) ? 1 : 0;
 
   if (pl.nseg > 1) {
     bp.seg_local = reinterpret_cast<float*>(ws + w.seg_local);

@@ -1,0 +1,416 @@
+// Backward selective scan, tuned path: bf16 io, N = 16, D % 8 == 0, 16-byte aligned pointers.
+// Same mathematics as ssm_bwd.cu (adjoint of Eq. 2a/2b with skip term and gate; states recomputed, Section 3.3).
+//
+// Mapping (as in the tuned forward kernel).  A thread owns 4 states of 2 adjacent channels as packed float2 pairs;
+// the 4 lanes of a quad cover the 16 states of the channel pair; a warp covers 16 channels, a block 32.
+//
+// Recomputation in two levels.  The block walks its segment backwards in tiles of 32 steps (one checkpoint block).
+// For a tile it first re-runs the recurrence from the checkpoint state over steps 0..23, keeping the states at steps
+// 8, 16 and 24 in registers; then, for the sub-blocks of 8 steps from last to first, it re-runs the 8 steps keeping
+// every h_t in registers and walks them backwards with the adjoint recurrence.  No state ever goes to shared or
+// global memory except the checkpoints.
+//
+// Sums.  The three per-(step, channel) sums over n (readout for dz, sum lam*B for dx and ddelta, sum w*A for
+// ddelta) are exchanged inside the quad in one batch per sub-block; afterwards every lane finalises 4 steps of one
+// channel.  dB and dC are summed over the two channels of a thread in registers, over the 8 quads of a warp through
+// a shared-memory transpose with a fixed order, over the 2 warps in ascending order, and leave the block as partial
+// sums that ssm_bwd_reduce_kernel adds in ascending block order.  dA and dD accumulate in registers over the whole
+// segment.  Everything is deterministic; there are no floating-point atomics.
+#include <type_traits>
+
+#include "ssm_common.cuh"
+
+namespace ssm {
+
+namespace {
+
+constexpr int kBT = 32;   // steps per tile = checkpoint spacing
+constexpr int kSB = 8;    // steps per register-resident sub-block
+static_assert(kBT == kCkptSteps, "the tuned backward kernel restarts from one checkpoint per tile");
+constexpr int kBwdFastWarps = 2;
+constexpr int kBwdFastThreads = kBwdFastWarps * 32;
+constexpr int kBwdFastCH = 16 * kBwdFastWarps;
+constexpr float kInvLog2e = 0.6931471805599453f;
+
+struct BwdFastSmem {
+  uint32_t x[2][kBT][kBwdFastCH / 2];   // bf16 pairs; the rows of a finished sub-block are reused for dx
+  uint32_t d[2][kBT][kBwdFastCH / 2];   // ... for ddelta
+  uint32_t z[2][kBT][kBwdFastCH / 2];   // ... for dz
+  uint32_t g[2][kBT][kBwdFastCH / 2];
+  uint32_t rawB[2][kBT][8];
+  uint32_t rawC[2][kBT][8];
+  float4 fB[kBT][4];
+  float4 fC[kBT][4];
+  float ds[kBT][kBwdFastCH];            // dout * silu(z)
+  float gsp[kBT][kBwdFastCH];           // dout * silu'(z)
+  float4 red[kBwdFastWarps][kSB][8][4][2];   // [warp][step][quad][lane in quad][dB quad | dC quad]
+  float acc[kBwdFastWarps][kBT][32];    // per-warp sums over its 16 channels: [step][dB 0..15 | dC 0..15]
+  float4 hsave[kBT / kSB][2][kBwdFastThreads];  // states at the sub-block boundaries, per thread and channel
+};
+
+}  // namespace
+
+__global__ void __launch_bounds__(kBwdFastThreads) ssm_bwd_fast_kernel(const BwdParams p) {
+  constexpr int THREADS = kBwdFastThreads;
+  constexpr int CH = kBwdFastCH;
+  constexpr int CHUNKS = CH / 8;
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  BwdFastSmem& sm = *reinterpret_cast<BwdFastSmem*>(smem_raw);
+
+  const __nv_bfloat16* __restrict__ gx = static_cast<const __nv_bfloat16*>(p.x);
+  const __nv_bfloat16* __restrict__ gd = static_cast<const __nv_bfloat16*>(p.delta);
+  const __nv_bfloat16* __restrict__ gz = static_cast<const __nv_bfloat16*>(p.z);
+  const __nv_bfloat16* __restrict__ gg = static_cast<const __nv_bfloat16*>(p.dout);
+  const __nv_bfloat16* __restrict__ gB = static_cast<const __nv_bfloat16*>(p.B);
+  const __nv_bfloat16* __restrict__ gC = static_cast<const __nv_bfloat16*>(p.C);
+  __nv_bfloat16* __restrict__ gdx = static_cast<__nv_bfloat16*>(p.dx);
+  __nv_bfloat16* __restrict__ gdd = static_cast<__nv_bfloat16*>(p.ddelta);
+  __nv_bfloat16* __restrict__ gdz = static_cast<__nv_bfloat16*>(p.dz);
+
+  const int tid = threadIdx.x;
+  const int lane = tid & 31, warp = tid >> 5;
+  const int j = lane & 3, quad = lane >> 2;
+  const int slot = warp * 8 + quad;      // channel pair within the block
+  const int d_cta = blockIdx.x * CH;
+  const int seg = blockIdx.y;
+  const int b = blockIdx.z;
+  const int D = p.D;
+  const int t_begin = seg * p.seg_steps;
+  const int t_end = min(p.L, t_begin + p.seg_steps);
+  const int ntiles = (t_end - t_begin + kBT - 1) / kBT;
+  const int d0 = d_cta + 2 * slot;
+  const bool valid = d0 < D;
+  const bool has_z = gz != nullptr;
+  // q = 0 is the channel whose sums this lane keeps (channel pq of the pair), q = 1 the one it hands to its neighbour
+  const int pq = j & 1, gq = j >> 1;
+  const uint32_t selA = pq ? 0x3244u : 0x1044u, selB = pq ? 0x1044u : 0x3244u;
+  auto chan = [&](int q) { return d0 + (q ^ pq); };
+
+  float2 A2[2][2], mu[2][2], dA2[2][2];
+  bool ap = true;
+#pragma unroll
+  for (int q = 0; q < 2; ++q) {
+    float4 a = make_float4(0.f, 0.f, 0.f, 0.f), m = a;
+    if (valid) {
+      a = *reinterpret_cast<const float4*>(p.A + (size_t)chan(q) * 16 + 4 * j);
+      if (p.mu_in != nullptr)
+        m = *reinterpret_cast<const float4*>(p.mu_in + (((size_t)b * p.nseg + seg) * D + chan(q)) * 16 + 4 * j);
+    }
+    const float step = a.y - a.x, tol = 1e-6f * fabsf(a.w);
+    ap = ap && fabsf(a.z - (a.x + 2.f * step)) <= tol && fabsf(a.w - (a.x + 3.f * step)) <= tol;
+    A2[q][0] = make_float2(a.x * kLog2e, a.y * kLog2e);
+    A2[q][1] = make_float2(a.z * kLog2e, a.w * kLog2e);
+    mu[q][0] = make_float2(m.x, m.y);
+    mu[q][1] = make_float2(m.z, m.w);
+    dA2[q][0] = dA2[q][1] = make_float2(0.f, 0.f);
+  }
+  ap = __all_sync(0xffffffffu, ap && !p.general_A);
+  const float Dk = (valid && p.Dskip != nullptr) ? p.Dskip[d0 + pq] : 0.f;
+  float dD_acc = 0.f;
+
+  auto issue_tile = [&](int i) {
+    if (i >= 0) {
+      const int st = i & 1;
+      const int t0 = t_begin + i * kBT;
+      const size_t row0 = (size_t)b * p.L + t0;
+      for (int c = tid; c < kBT * CHUNKS; c += THREADS) {
+        const int tt = c / CHUNKS, cc = c % CHUNKS;
+        const bool ok = (t0 + tt < t_end) && (d_cta + cc * 8 < D);
+        const size_t g = ok ? (row0 + tt) * D + d_cta + cc * 8 : 0;
+        cp_async16(&sm.x[st][tt][cc * 4], gx + g, ok);
+        cp_async16(&sm.d[st][tt][cc * 4], gd + g, ok);
+        cp_async16(&sm.z[st][tt][cc * 4], (has_z ? gz : gx) + g, ok && has_z);
+        cp_async16(&sm.g[st][tt][cc * 4], gg + g, ok);
+      }
+      for (int c = tid; c < kBT * 2; c += THREADS) {
+        const int tt = c >> 1, cc = c & 1;
+        const bool ok = t0 + tt < t_end;
+        const size_t g = ok ? (row0 + tt) * 16 + cc * 8 : 0;
+        cp_async16(&sm.rawB[st][tt][cc * 4], gB + g, ok);
+        cp_async16(&sm.rawC[st][tt][cc * 4], gC + g, ok);
+      }
+    }
+    cp_async_commit();
+  };
+
+  // decays of one step for channel q: general A or arithmetic-progression A (two exponentials)
+  auto decays = [&](float dt, int q, auto ap_tag, float2& a01, float2& a23) {
+    if (decltype(ap_tag)::value) {
+      const float a0 = ex2_approx(dt * A2[q][0].x);
+      const float r = ex2_approx(dt * (A2[q][0].y - A2[q][0].x));
+      const float r2 = r * r;
+      a01 = make_float2(a0, a0 * r);
+      a23 = f2mul(a01, f2dup(r2));
+    } else {
+      const float2 e01 = f2mul(f2dup(dt), A2[q][0]), e23 = f2mul(f2dup(dt), A2[q][1]);
+      a01 = make_float2(ex2_approx(e01.x), ex2_approx(e01.y));
+      a23 = make_float2(ex2_approx(e23.x), ex2_approx(e23.y));
+    }
+  };
+
+  auto process_tile = [&](int i, auto ap_tag, const float4 (&ck)[2]) {
+    const int st = i & 1;
+    // ---- level 1: states at the sub-block boundaries (steps 0, 8, 16, 24 of the tile), parked in shared memory
+    {
+      float2 h[2][2];
+#pragma unroll
+      for (int q = 0; q < 2; ++q) {
+        sm.hsave[0][q][tid] = ck[q];
+        h[q][0] = make_float2(ck[q].x, ck[q].y);
+        h[q][1] = make_float2(ck[q].z, ck[q].w);
+      }
+#pragma unroll 1
+    for (int sb = 0; sb < kBT / kSB - 1; ++sb) {
+#pragma unroll
+      for (int t = 0; t < kSB; ++t) {
+        const int tt = sb * kSB + t;
+        const uint32_t dw = sm.d[st][tt][slot], xw = sm.x[st][tt][slot];
+        const float4 Bq = sm.fB[tt][j];
+        const float2 dt2 = make_float2(bf16sel(dw, selA), bf16sel(dw, selB));
+        const float2 du = f2mul(dt2, make_float2(bf16sel(xw, selA), bf16sel(xw, selB)));
+        const float dtq[2] = {dt2.x, dt2.y}, duq[2] = {du.x, du.y};
+#pragma unroll
+        for (int q = 0; q < 2; ++q) {
+          float2 a01, a23;
+          decays(dtq[q], q, ap_tag, a01, a23);
+          h[q][0] = f2fma(a01, h[q][0], f2mul(f2dup(duq[q]), make_float2(Bq.x, Bq.y)));
+          h[q][1] = f2fma(a23, h[q][1], f2mul(f2dup(duq[q]), make_float2(Bq.z, Bq.w)));
+        }
+      }
+#pragma unroll
+      for (int q = 0; q < 2; ++q) sm.hsave[sb + 1][q][tid] = make_float4(h[q][0].x, h[q][0].y, h[q][1].x, h[q][1].y);
+    }
+    }
+    // ---- level 2: sub-blocks from last to first
+#pragma unroll 1
+    for (int sb = kBT / kSB - 1; sb >= 0; --sb) {
+      float2 hs0[2][2];  // state before the first step of the sub-block
+#pragma unroll
+      for (int q = 0; q < 2; ++q) {
+        const float4 v = sm.hsave[sb][q][tid];
+        hs0[q][0] = make_float2(v.x, v.y);
+        hs0[q][1] = make_float2(v.z, v.w);
+      }
+      float2 hist[kSB][2][2];
+      uint32_t dwk[kSB], xwk[kSB];
+      float yw[kSB], dxw[kSB], ddw[kSB];  // quad-pair sums of: readout, delta * sum lam B, sum w A + x sum lam B
+      {
+        float2 h[2][2] = {{hs0[0][0], hs0[0][1]}, {hs0[1][0], hs0[1][1]}};
+#pragma unroll
+        for (int t = 0; t < kSB; ++t) {
+          const int tt = sb * kSB + t;
+          dwk[t] = sm.d[st][tt][slot];
+          xwk[t] = sm.x[st][tt][slot];
+          const float4 Bq = sm.fB[tt][j], Cq = sm.fC[tt][j];
+          const float2 dt2 = make_float2(bf16sel(dwk[t], selA), bf16sel(dwk[t], selB));
+          const float2 du = f2mul(dt2, make_float2(bf16sel(xwk[t], selA), bf16sel(xwk[t], selB)));
+          const float dtq[2] = {dt2.x, dt2.y}, duq[2] = {du.x, du.y};
+          float y[2];
+#pragma unroll
+          for (int q = 0; q < 2; ++q) {
+            float2 a01, a23;
+            decays(dtq[q], q, ap_tag, a01, a23);
+            h[q][0] = f2fma(a01, h[q][0], f2mul(f2dup(duq[q]), make_float2(Bq.x, Bq.y)));
+            h[q][1] = f2fma(a23, h[q][1], f2mul(f2dup(duq[q]), make_float2(Bq.z, Bq.w)));
+            hist[t][q][0] = h[q][0];
+            hist[t][q][1] = h[q][1];
+            float2 yv = f2mul(make_float2(Cq.x, Cq.y), h[q][0]);
+            yv = f2fma(make_float2(Cq.z, Cq.w), h[q][1], yv);
+            y[q] = yv.x + yv.y;
+          }
+          yw[t] = y[0] + __shfl_xor_sync(0xffffffffu, y[1], 1);
+        }
+      }
+      // reverse recurrence over the sub-block
+#pragma unroll
+      for (int t = kSB - 1; t >= 0; --t) {
+        const int tt = sb * kSB + t;
+        const float4 Bq = sm.fB[tt][j], Cq = sm.fC[tt][j];
+        const float2 dt2 = make_float2(bf16sel(dwk[t], selA), bf16sel(dwk[t], selB));
+        const float2 u2 = make_float2(bf16sel(xwk[t], selA), bf16sel(xwk[t], selB));
+        const float2 du = f2mul(dt2, u2);
+        const float dtq[2] = {dt2.x, dt2.y}, uq[2] = {u2.x, u2.y}, duq[2] = {du.x, du.y};
+        const float dsq[2] = {sm.ds[tt][2 * slot + pq], sm.ds[tt][2 * slot + (pq ^ 1)]};
+        float2 dB01, dB23, dC01, dC23;
+        float dxp[2], ddp[2];
+#pragma unroll
+        for (int q = 0; q < 2; ++q) {
+          float2 a01, a23;
+          decays(dtq[q], q, ap_tag, a01, a23);
+          const float2 ds2 = f2dup(dsq[q]), du2 = f2dup(duq[q]);
+          const float2 lam01 = f2fma(make_float2(Cq.x, Cq.y), ds2, mu[q][0]);
+          const float2 lam23 = f2fma(make_float2(Cq.z, Cq.w), ds2, mu[q][1]);
+          if (q == 0) {
+            dC01 = f2mul(ds2, hist[t][q][0]);
+            dC23 = f2mul(ds2, hist[t][q][1]);
+            dB01 = f2mul(lam01, du2);
+            dB23 = f2mul(lam23, du2);
+          } else {
+            dC01 = f2fma(ds2, hist[t][q][0], dC01);
+            dC23 = f2fma(ds2, hist[t][q][1], dC23);
+            dB01 = f2fma(lam01, du2, dB01);
+            dB23 = f2fma(lam23, du2, dB23);
+          }
+          float2 lb = f2mul(lam01, make_float2(Bq.x, Bq.y));
+          lb = f2fma(lam23, make_float2(Bq.z, Bq.w), lb);
+          const float lamB = lb.x + lb.y;
+          mu[q][0] = f2mul(a01, lam01);
+          mu[q][1] = f2mul(a23, lam23);
+          const float2 hp0 = t > 0 ? hist[t > 0 ? t - 1 : 0][q][0] : hs0[q][0];
+          const float2 hp1 = t > 0 ? hist[t > 0 ? t - 1 : 0][q][1] : hs0[q][1];
+          const float2 w01 = f2mul(mu[q][0], hp0), w23 = f2mul(mu[q][1], hp1);
+          float2 wa = f2mul(w01, A2[q][0]);
+          wa = f2fma(w23, A2[q][1], wa);
+          dA2[q][0] = f2fma(w01, f2dup(dtq[q]), dA2[q][0]);
+          dA2[q][1] = f2fma(w23, f2dup(dtq[q]), dA2[q][1]);
+          dxp[q] = dtq[q] * lamB;
+          ddp[q] = fmaf(uq[q], lamB, (wa.x + wa.y) * kInvLog2e);
+        }
+        sm.red[warp][t][quad][j][0] = make_float4(dB01.x, dB01.y, dB23.x, dB23.y);
+        sm.red[warp][t][quad][j][1] = make_float4(dC01.x, dC01.y, dC23.x, dC23.y);
+        dxw[t] = dxp[0] + __shfl_xor_sync(0xffffffffu, dxp[1], 1);
+        ddw[t] = ddp[0] + __shfl_xor_sync(0xffffffffu, ddp[1], 1);
+      }
+      // second exchange: lanes j and j^2 hold sums of the same channel; the lower keeps steps 0..3, the upper 4..7
+      float ytot[4], dxtot[4], ddtot[4];
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const float ky = gq ? yw[4 + e] : yw[e], sy = gq ? yw[e] : yw[4 + e];
+        const float kx = gq ? dxw[4 + e] : dxw[e], sx = gq ? dxw[e] : dxw[4 + e];
+        const float kd = gq ? ddw[4 + e] : ddw[e], sd = gq ? ddw[e] : ddw[4 + e];
+        ytot[e] = ky + __shfl_xor_sync(0xffffffffu, sy, 2);
+        dxtot[e] = kx + __shfl_xor_sync(0xffffffffu, sx, 2);
+        ddtot[e] = kd + __shfl_xor_sync(0xffffffffu, sd, 2);
+      }
+      // finalise 4 steps of channel pq: the rows of this sub-block are no longer read as inputs by this quad
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const int tt = sb * kSB + 4 * gq + e;
+        const float u = __uint_as_float((uint32_t)reinterpret_cast<const uint16_t*>(&sm.x[st][tt][slot])[pq] << 16);
+        const float ds = sm.ds[tt][2 * slot + pq];
+        const float s = fmaf(Dk, u, ytot[e]);
+        dD_acc = fmaf(ds, u, dD_acc);
+        reinterpret_cast<__nv_bfloat16*>(&sm.x[st][tt][slot])[pq] = __float2bfloat16_rn(fmaf(ds, Dk, dxtot[e]));
+        reinterpret_cast<__nv_bfloat16*>(&sm.d[st][tt][slot])[pq] = __float2bfloat16_rn(ddtot[e]);
+        reinterpret_cast<__nv_bfloat16*>(&sm.z[st][tt][slot])[pq] = __float2bfloat16_rn(sm.gsp[tt][2 * slot + pq] * s);
+      }
+      // dB / dC: sum over the 8 quads of this warp, fixed order; lane -> (step = lane / 4, state quad = lane % 4)
+      __syncwarp();
+      {
+        const int tr = lane >> 2, jr = lane & 3;
+        float4 sb4 = sm.red[warp][tr][0][jr][0], sc4 = sm.red[warp][tr][0][jr][1];
+#pragma unroll
+        for (int qd = 1; qd < 8; ++qd) {
+          const float4 vb = sm.red[warp][tr][qd][jr][0], vc = sm.red[warp][tr][qd][jr][1];
+          sb4.x += vb.x; sb4.y += vb.y; sb4.z += vb.z; sb4.w += vb.w;
+          sc4.x += vc.x; sc4.y += vc.y; sc4.z += vc.z; sc4.w += vc.w;
+        }
+        *reinterpret_cast<float4*>(&sm.acc[warp][sb * kSB + tr][4 * jr]) = sb4;
+        *reinterpret_cast<float4*>(&sm.acc[warp][sb * kSB + tr][16 + 4 * jr]) = sc4;
+      }
+      __syncwarp();
+    }
+  };
+
+  // ---- tiles from last to first
+  issue_tile(ntiles - 1);
+  for (int i = ntiles - 1; i >= 0; --i) {
+    const int st = i & 1;
+    const int t0 = t_begin + i * kBT;
+    const size_t row0 = (size_t)b * p.L + t0;
+    float4 ck[2];
+#pragma unroll
+    for (int q = 0; q < 2; ++q)
+      ck[q] = valid ? *reinterpret_cast<const float4*>(p.ckpt + (((size_t)b * p.nck + t0 / kCkptSteps) * D + chan(q)) * 16 + 4 * j)
+                    : make_float4(0.f, 0.f, 0.f, 0.f);
+    cp_async_wait_all();
+    __syncthreads();
+    issue_tile(i - 1);
+    // widen B, C; per-element gate terms ds = dout * silu(z), gsp = dout * silu'(z)
+    for (int c = tid; c < kBT * 8; c += THREADS) {
+      const int tt = c >> 3, w = c & 7;
+      const uint32_t vb = sm.rawB[st][tt][w], vc = sm.rawC[st][tt][w];
+      reinterpret_cast<float2*>(&sm.fB[tt][0])[w] = make_float2(bf16lo(vb), bf16hi(vb));
+      reinterpret_cast<float2*>(&sm.fC[tt][0])[w] = make_float2(bf16lo(vc), bf16hi(vc));
+    }
+    for (int c = tid; c < kBT * (CH / 2); c += THREADS) {
+      const int tt = c / (CH / 2), w = c % (CH / 2);
+      const uint32_t zw = sm.z[st][tt][w], gw = sm.g[st][tt][w];
+      float2 dsv, gpv;
+      {
+        const float g0 = bf16lo(gw), g1 = bf16hi(gw);
+        if (has_z) {
+          const float z0 = bf16lo(zw), z1 = bf16hi(zw);
+          const float s0 = sigmoid_fast(z0), s1 = sigmoid_fast(z1);
+          dsv = make_float2(g0 * z0 * s0, g1 * z1 * s1);
+          gpv = make_float2(g0 * s0 * fmaf(z0, 1.f - s0, 1.f), g1 * s1 * fmaf(z1, 1.f - s1, 1.f));
+        } else {
+          dsv = make_float2(g0, g1);
+          gpv = make_float2(0.f, 0.f);
+        }
+      }
+      *reinterpret_cast<float2*>(&sm.ds[tt][2 * w]) = dsv;
+      *reinterpret_cast<float2*>(&sm.gsp[tt][2 * w]) = gpv;
+    }
+    __syncthreads();
+    if (ap) process_tile(i, std::true_type{}, ck);
+    else process_tile(i, std::false_type{}, ck);
+    __syncthreads();
+    // results of the tile: 16-byte stores of dx, ddelta, dz; block partial sums of dB, dC
+    for (int c = tid; c < kBT * CHUNKS; c += THREADS) {
+      const int tt = c / CHUNKS, cc = c % CHUNKS;
+      if (t0 + tt < t_end && d_cta + cc * 8 < D) {
+        const size_t g = (row0 + tt) * D + d_cta + cc * 8;
+        *reinterpret_cast<uint4*>(gdx + g) = *reinterpret_cast<const uint4*>(&sm.x[st][tt][cc * 4]);
+        *reinterpret_cast<uint4*>(gdd + g) = *reinterpret_cast<const uint4*>(&sm.d[st][tt][cc * 4]);
+        if (gdz != nullptr) *reinterpret_cast<uint4*>(gdz + g) = *reinterpret_cast<const uint4*>(&sm.z[st][tt][cc * 4]);
+      }
+    }
+    const size_t bln = (size_t)p.batch * p.L * 16;
+    for (int c = tid; c < kBT * 8; c += THREADS) {  // float4 granules: [step][dB 0..15 | dC 0..15]
+      const int tt = c >> 3, f = c & 7;
+      if (t0 + tt < t_end) {
+        float4 v = *reinterpret_cast<const float4*>(&sm.acc[0][tt][4 * f]);
+#pragma unroll
+        for (int w = 1; w < kBwdFastWarps; ++w) {
+          const float4 o = *reinterpret_cast<const float4*>(&sm.acc[w][tt][4 * f]);
+          v.x += o.x; v.y += o.y; v.z += o.z; v.w += o.w;
+        }
+        const int which = f >> 2;
+        *reinterpret_cast<float4*>(p.dBC_part + ((size_t)blockIdx.x * 2 + which) * bln + (row0 + tt) * 16 + 4 * (f & 3)) = v;
+      }
+    }
+  }
+  cp_async_wait_all();
+
+  if (valid) {
+    const size_t part = (size_t)b * p.nseg + seg;
+#pragma unroll
+    for (int q = 0; q < 2; ++q)
+      *reinterpret_cast<float4*>(p.dA_part + (part * D + chan(q)) * 16 + 4 * j) =
+          make_float4(dA2[q][0].x, dA2[q][0].y, dA2[q][1].x, dA2[q][1].y);
+  }
+  // dD: lanes j and j^2 accumulated disjoint steps of the same channel
+  dD_acc += __shfl_xor_sync(0xffffffffu, dD_acc, 2);
+  if (valid && j < 2) p.dD_part[((size_t)b * p.nseg + seg) * D + d0 + pq] = dD_acc;
+}
+
+bool bwd_fast_applicable(const ssm_problem_t& prob, const BwdParams& p) {
+  auto al16 = [](const void* q) { return q == nullptr || (reinterpret_cast<uintptr_t>(q) & 15) == 0; };
+  return prob.io_dtype == SSM_BF16 && prob.N == 16 && prob.D % 8 == 0 && al16(p.x) && al16(p.delta) && al16(p.z) &&
+         al16(p.B) && al16(p.C) && al16(p.dout) && al16(p.dx) && al16(p.ddelta) && al16(p.dz) && al16(p.A) &&
+         al16(p.ckpt) && al16(p.mu_in) && al16(p.dBC_part) && al16(p.dA_part);
+}
+
+int bwd_fast_channels_per_block() { return kBwdFastCH; }
+
+cudaError_t launch_bwd_fast(const Plan& plan, const BwdParams& p, cudaStream_t s) {
+  constexpr size_t smem = sizeof(BwdFastSmem);
+  cudaError_t e = cudaFuncSetAttribute(ssm_bwd_fast_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (e != cudaSuccess) return e;
+  dim3 grid((p.D + kBwdFastCH - 1) / kBwdFastCH, plan.nseg, p.batch);
+  ssm_bwd_fast_kernel<<<grid, kBwdFastThreads, smem, s>>>(p);
+  return cudaGetLastError();
+}
+
+}  // namespace ssm

@@ -12,7 +12,7 @@ namespace ssm {
 
 // Time steps between two checkpoint states (the state h at the start of every such block is what backward restarts
 // its recomputation from).  Segment lengths of the time split are multiples of this.
-constexpr int kCkptSteps = 64;
+constexpr int kCkptSteps = 32;
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr int kNumSMs = 148;
 
@@ -76,6 +76,7 @@ struct BwdParams {
   float* dA_part;         // [batch*nseg][D][N]
   float* dD_part;         // [batch*nseg][D]
   int batch, L, D, nseg, seg_steps, nck, groups;
+  int general_A;          // 1: never take the arithmetic-progression fast path
 };
 
 struct ReduceParams {
@@ -101,9 +102,13 @@ enum BwdMode { kBwdFull = 0, kBwdLocal = 1 };
 // ---------------------------------------------------------------------------------------------- device helpers
 #ifdef __CUDACC__
 __device__ __forceinline__ float ex2_approx(float v) {
+#ifdef LAB_NOMUFU
+  return fmaf(v, 0.25f, 1.0f);
+#else
   float r;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(v));
   return r;
+#endif
 }
 __device__ __forceinline__ float rcp_approx(float v) {
   float r;
@@ -124,6 +129,25 @@ template <>
 __device__ __forceinline__ float float_to_io<float>(float v) { return v; }
 template <>
 __device__ __forceinline__ __nv_bfloat16 float_to_io<__nv_bfloat16>(float v) { return __float2bfloat16_rn(v); }
+
+// 16-byte asynchronous global -> shared copy; with valid == false nothing is read and the destination is zero-filled
+__device__ __forceinline__ void cp_async16(void* smem_dst, const void* gmem_src, bool valid) {
+  const unsigned dst = (unsigned)__cvta_generic_to_shared(smem_dst);
+  const int bytes = valid ? 16 : 0;
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(gmem_src), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_group 0;" ::: "memory"); }
+
+// halves of a packed bf16 pair, widened to float (bf16 is the upper half of a float)
+__device__ __forceinline__ float bf16lo(uint32_t w) { return __uint_as_float(w << 16); }
+__device__ __forceinline__ float bf16hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
+// the same through one byte-permute whose selector (0x1044: low half, 0x3244: high half) may differ per lane
+__device__ __forceinline__ float bf16sel(uint32_t w, uint32_t sel) { return __uint_as_float(__byte_perm(w, 0u, sel)); }
+
+__device__ __forceinline__ float2 f2mul(float2 a, float2 b) { return __fmul2_rn(a, b); }
+__device__ __forceinline__ float2 f2fma(float2 a, float2 b, float2 c) { return __ffma2_rn(a, b, c); }
+__device__ __forceinline__ float2 f2dup(float v) { return make_float2(v, v); }
 
 // sigmoid(z) through one ex2 and one reciprocal
 __device__ __forceinline__ float sigmoid_fast(float z) { return rcp_approx(1.0f + ex2_approx(-kLog2e * z)); }

@@ -220,7 +220,11 @@ int fwd_channels_per_block(int N) {
   return (fwd_threads(N) / (N / S)) * 2;
 }
 
+bool fwd_fast_applicable(const ssm_problem_t& prob, const FwdParams& p);
+cudaError_t launch_fwd_fast(const Plan& plan, const FwdParams& p, int mode, cudaStream_t s);
+
 cudaError_t launch_fwd(const ssm_problem_t& prob, const Plan& plan, const FwdParams& p, int mode, cudaStream_t s) {
+  if (fwd_fast_applicable(prob, p)) return launch_fwd_fast(plan, p, mode, s);
   if (prob.io_dtype == SSM_BF16) return launch_fwd_io<__nv_bfloat16>(prob, plan, p, mode, s);
   return launch_fwd_io<float>(prob, plan, p, mode, s);
 }

@@ -1,0 +1,347 @@
+// Forward selective scan, tuned path: bf16 io, N = 16, D % 8 == 0, 16-byte aligned pointers.
+// Same mathematics and modes as ssm_fwd.cu (Algorithm 2 steps 5-6; Eq. 2a/2b; Eq. 4's A-bar; fused skip and gate).
+//
+// Mapping.  A thread owns 4 states of 2 adjacent channels (8 recurrences, held as packed float2 pairs so that the
+// multiply-adds issue as two-wide FP32 instructions); the 4 lanes of a quad cover the 16 states of the channel
+// pair; a warp covers 16 channels and sweeps time sequentially.  The sum over n of the readout is completed inside
+// the quad by a two-step exchange that leaves the total of channel 0 in even lanes and of channel 1 in odd lanes.
+//
+// Staging.  x, delta, z and B, C arrive by 16-byte cp.async into a three-stage ring of [32 steps x channels] tiles
+// (one __syncthreads per tile); B and C are widened to float once per block and tile, so the inner loop reads them
+// as 128-bit broadcast loads; the output tile is assembled in shared memory and written with 16-byte stores.
+//
+// Discretization.  a = 2^(delta * A * log2 e) with the hardware ex2.  When the four A values of a thread form an
+// arithmetic progression (as in the S4D-Real initialisation A_n = -(n+1)) the four decays are built from two
+// exponentials, a_{k} = a_0 r^k with r = 2^(delta * step * log2 e); the test is made per warp at run time and can
+// be disabled by SSM_FLAG_GENERAL_A.
+#include <cstdio>
+#include <type_traits>
+
+#include "ssm_common.cuh"
+
+namespace ssm {
+
+namespace {
+
+constexpr int kTT = 32;    // steps per tile
+constexpr int kNST = 3;    // ring stages
+
+template <int WARPS, bool FULL>
+struct FastSmem {
+  static constexpr int CH = 16 * WARPS;
+  uint32_t x[kNST][kTT][CH / 2];
+  uint32_t d[kNST][kTT][CH / 2];
+  uint32_t z[FULL ? kNST : 1][FULL ? kTT : 1][CH / 2];
+  uint32_t rawB[kNST][kTT][8];
+  uint32_t rawC[FULL ? kNST : 1][FULL ? kTT : 1][8];
+  float4 fB[2][kTT][4];
+  float4 fC[FULL ? 2 : 1][FULL ? kTT : 1][4];
+  uint32_t o[FULL ? 2 : 1][FULL ? kTT : 1][CH / 2];
+};
+
+}  // namespace
+
+template <int WARPS, int MODE>
+__global__ void __launch_bounds__(WARPS * 32) ssm_fwd_fast_kernel(const FwdParams p) {
+  constexpr bool FULL = (MODE == kFwdFull);
+  constexpr int THREADS = WARPS * 32;
+  constexpr int CH = 16 * WARPS;
+  constexpr int CHUNKS = CH / 8;  // 16-byte chunks per tile row
+  using Smem = FastSmem<WARPS, FULL>;
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  Smem& sm = *reinterpret_cast<Smem*>(smem_raw);
+
+  const __nv_bfloat16* __restrict__ gx = static_cast<const __nv_bfloat16*>(p.x);
+  const __nv_bfloat16* __restrict__ gd = static_cast<const __nv_bfloat16*>(p.delta);
+  const __nv_bfloat16* __restrict__ gz = static_cast<const __nv_bfloat16*>(p.z);
+  const __nv_bfloat16* __restrict__ gB = static_cast<const __nv_bfloat16*>(p.B);
+  const __nv_bfloat16* __restrict__ gC = static_cast<const __nv_bfloat16*>(p.C);
+  __nv_bfloat16* __restrict__ gout = static_cast<__nv_bfloat16*>(p.out);
+
+  const int tid = threadIdx.x;
+  const int lane = tid & 31;
+  const int j = lane & 3;
+  const int slot = (tid >> 5) * 8 + (lane >> 2);  // channel pair within the block
+  const int d_cta = blockIdx.x * CH;
+  const int seg = blockIdx.y;
+  const int b = blockIdx.z;
+  const int D = p.D;
+  const int t_begin = seg * p.seg_steps;
+  const int t_end = min(p.L, t_begin + p.seg_steps);
+  const int ntiles = (t_end - t_begin + kTT - 1) / kTT;
+  const int d0 = d_cta + 2 * slot;  // first channel of this quad's pair (D is even, so both are valid or neither)
+  const bool valid = d0 < D;
+  const int pq = j & 1, gq = j >> 1;
+  // A lane keeps the readout of channel pq of the pair and hands the other channel's partial sum to its neighbour,
+  // so it numbers its own channels q = 0 (channel pq) and q = 1 (channel 1 - pq); the byte-permute selectors below
+  // pick the matching half of a packed bf16 pair and widen it to float in one instruction.
+  const uint32_t selA = pq ? 0x3244u : 0x1044u, selB = pq ? 0x1044u : 0x3244u;
+  auto chan = [&](int q) { return d0 + (q ^ pq); };
+  const bool has_z = FULL && gz != nullptr;
+
+  // ---- per-thread constants and state
+  float2 A2[2][2];   // A * log2(e), states (4j, 4j+1) and (4j+2, 4j+3) of each channel
+  float2 h[2][2];
+  float dsum[2] = {0.f, 0.f};
+  bool ap = !p.general_A;
+#pragma unroll
+  for (int q = 0; q < 2; ++q) {
+    float4 a = make_float4(0.f, 0.f, 0.f, 0.f), hs = a;
+    if (valid) {
+      a = *reinterpret_cast<const float4*>(p.A + (size_t)chan(q) * 16 + 4 * j);
+      if (p.h_start != nullptr)
+        hs = *reinterpret_cast<const float4*>(p.h_start + (((size_t)b * p.nseg + seg) * D + chan(q)) * 16 + 4 * j);
+    }
+    const float step = a.y - a.x;
+    const float tol = 1e-6f * fabsf(a.w);
+    ap = ap && fabsf(a.z - (a.x + 2.f * step)) <= tol && fabsf(a.w - (a.x + 3.f * step)) <= tol;
+    A2[q][0] = make_float2(a.x * kLog2e, a.y * kLog2e);
+    A2[q][1] = make_float2(a.z * kLog2e, a.w * kLog2e);
+    h[q][0] = make_float2(hs.x, hs.y);
+    h[q][1] = make_float2(hs.z, hs.w);
+  }
+  ap = __all_sync(0xffffffffu, ap);
+  const float Dk = (FULL && valid && p.Dskip != nullptr) ? p.Dskip[d0 + pq] : 0.f;
+
+  auto issue_tile = [&](int i) {
+    if (i < ntiles) {
+      const int st = i % kNST;
+      const int t0 = t_begin + i * kTT;
+      const size_t row0 = (size_t)b * p.L + t0;
+      for (int c = tid; c < kTT * CHUNKS; c += THREADS) {
+        const int tt = c / CHUNKS, cc = c % CHUNKS;
+        const bool ok = (t0 + tt < t_end) && (d_cta + cc * 8 < D);
+        const size_t g = ok ? (row0 + tt) * D + d_cta + cc * 8 : 0;
+        cp_async16(&sm.x[st][tt][cc * 4], gx + g, ok);
+        cp_async16(&sm.d[st][tt][cc * 4], gd + g, ok);
+        if (FULL) cp_async16(&sm.z[st][tt][cc * 4], (has_z ? gz : gx) + g, ok && has_z);
+      }
+      for (int c = tid; c < kTT * 2; c += THREADS) {
+        const int tt = c >> 1, cc = c & 1;
+        const bool ok = t0 + tt < t_end;
+        const size_t g = ok ? (row0 + tt) * 16 + cc * 8 : 0;
+        cp_async16(&sm.rawB[st][tt][cc * 4], gB + g, ok);
+        if (FULL) cp_async16(&sm.rawC[st][tt][cc * 4], gC + g, ok);
+      }
+    }
+    cp_async_commit();
+  };
+  auto widen_BC = [&](int i) {  // tile i: bf16 -> float
+    if (i >= ntiles) return;
+    const int st = i % kNST, fb = i & 1;
+    for (int c = tid; c < kTT * 8; c += THREADS) {
+      const int tt = c >> 3, w = c & 7;
+      const uint32_t vb = sm.rawB[st][tt][w];
+      reinterpret_cast<float2*>(&sm.fB[fb][tt][0])[w] = make_float2(bf16lo(vb), bf16hi(vb));
+      if (FULL) {
+        const uint32_t vc = sm.rawC[st][tt][w];
+        reinterpret_cast<float2*>(&sm.fC[fb][tt][0])[w] = make_float2(bf16lo(vc), bf16hi(vc));
+      }
+    }
+  };
+  auto store_out = [&](int i) {  // tile i: shared -> global, 16 bytes per thread and iteration
+    if (!FULL) return;
+    const int t0 = t_begin + i * kTT;
+    const size_t row0 = (size_t)b * p.L + t0;
+    for (int c = tid; c < kTT * CHUNKS; c += THREADS) {
+      const int tt = c / CHUNKS, cc = c % CHUNKS;
+      if (t0 + tt < t_end && d_cta + cc * 8 < D)
+        *reinterpret_cast<uint4*>(gout + (row0 + tt) * D + d_cta + cc * 8) =
+            *reinterpret_cast<const uint4*>(&sm.o[i & 1][tt][cc * 4]);
+    }
+  };
+
+  // One tile of kTT steps, in sub-blocks of 4 steps: the loads of the next sub-block are issued before the
+  // shared-memory stores of the current one, and the readout sums of 4 steps x 2 channels are exchanged inside the
+  // quad in one batch, after which every lane finalises two (step, channel) values.  Rows past the end of the
+  // segment were zero-filled: delta = 0 gives a = 1 and no input, so they leave the state untouched.
+  auto compute_tile = [&](int i, auto ap_tag) {
+    constexpr bool AP = decltype(ap_tag)::value;
+    constexpr int SB = 4;  // the quad exchange below is written for exactly 4 steps
+    const int st = i % kNST, fb = i & 1;
+    float a0s[2], rs[2];  // AP path: A2 of the first state and of the step
+    if (AP) {
+#pragma unroll
+      for (int q = 0; q < 2; ++q) {
+        a0s[q] = A2[q][0].x;
+        rs[q] = A2[q][0].y - A2[q][0].x;
+      }
+    }
+    uint32_t dw[SB], xw[SB];
+    float4 Bq[SB], Cq[SB];
+    auto load_sb = [&](int tb) {
+#pragma unroll
+      for (int t = 0; t < SB; ++t) {
+        dw[t] = sm.d[st][tb + t][slot];
+        xw[t] = sm.x[st][tb + t][slot];
+        Bq[t] = sm.fB[fb][tb + t][j];
+        if (FULL) Cq[t] = sm.fC[fb][tb + t][j];
+      }
+    };
+    load_sb(0);
+#pragma unroll
+    for (int tb = 0; tb < kTT; tb += SB) {
+      // pass 1: discretization of the whole sub-block (independent work: decays a and inputs bx for 4 steps)
+      float2 a01[SB][2], a23[SB][2], bx01[SB][2], bx23[SB][2];
+#pragma unroll
+      for (int t = 0; t < SB; ++t) {
+        // q = 0 is this lane's kept channel (channel pq of the pair), q = 1 the one it hands to its neighbour
+        const float dt[2] = {__uint_as_float(__byte_perm(dw[t], 0, selA)), __uint_as_float(__byte_perm(dw[t], 0, selB))};
+        const float u[2] = {__uint_as_float(__byte_perm(xw[t], 0, selA)), __uint_as_float(__byte_perm(xw[t], 0, selB))};
+        const float2 du = f2mul(make_float2(dt[0], dt[1]), make_float2(u[0], u[1]));
+        const float duq[2] = {du.x, du.y};
+#pragma unroll
+        for (int q = 0; q < 2; ++q) {
+          if (AP) {
+            const float a0 = ex2_approx(dt[q] * a0s[q]);
+            const float r = ex2_approx(dt[q] * rs[q]);
+            const float r2 = r * r;
+            a01[t][q] = make_float2(a0, a0 * r);
+            a23[t][q] = f2mul(a01[t][q], make_float2(r2, r2));
+          } else {
+            const float2 dd = make_float2(dt[q], dt[q]);
+            const float2 e01 = f2mul(dd, A2[q][0]), e23 = f2mul(dd, A2[q][1]);
+            a01[t][q] = make_float2(ex2_approx(e01.x), ex2_approx(e01.y));
+            a23[t][q] = make_float2(ex2_approx(e23.x), ex2_approx(e23.y));
+          }
+          const float2 dq = make_float2(duq[q], duq[q]);
+          bx01[t][q] = f2mul(dq, make_float2(Bq[t].x, Bq[t].y));
+          bx23[t][q] = f2mul(dq, make_float2(Bq[t].z, Bq[t].w));
+          if (MODE == kFwdSummary) dsum[q] += dt[q];
+        }
+      }
+      // pass 2: the recurrence (4 independent packed chains) and the readout
+      float y[SB][2];
+#pragma unroll
+      for (int t = 0; t < SB; ++t) {
+#pragma unroll
+        for (int q = 0; q < 2; ++q) {
+          h[q][0] = f2fma(a01[t][q], h[q][0], bx01[t][q]);
+          h[q][1] = f2fma(a23[t][q], h[q][1], bx23[t][q]);
+          if (FULL) {
+            float2 yv = f2mul(make_float2(Cq[t].x, Cq[t].y), h[q][0]);
+            yv = f2fma(make_float2(Cq[t].z, Cq[t].w), h[q][1], yv);
+            y[t][q] = yv.x + yv.y;
+          }
+        }
+      }
+      if (tb + SB < kTT) load_sb(tb + SB);
+#ifdef LAB_NOEPI
+      if (FULL) { float acc = 0.f;
+#pragma unroll
+        for (int t = 0; t < SB; ++t) acc += y[t][0] + y[t][1];
+        if (acc == 123.456f) reinterpret_cast<__nv_bfloat16*>(&sm.o[fb][tb][slot])[pq] = __float2bfloat16_rn(acc); }
+      if (false) {
+#else
+      if (FULL) {
+#endif
+        float w[SB];
+#pragma unroll
+        for (int t = 0; t < SB; ++t) w[t] = y[t][0] + __shfl_xor_sync(0xffffffffu, y[t][1], 1);
+        // lanes j and j^2 hold the same channel: the lower one finishes steps 0,1 of the sub-block, the upper 2,3
+        float tot[2];
+#pragma unroll
+        for (int e = 0; e < 2; ++e) {
+          const float keep = gq ? w[2 + e] : w[e], send = gq ? w[e] : w[2 + e];
+          tot[e] = keep + __shfl_xor_sync(0xffffffffu, send, 2);
+        }
+#pragma unroll
+        for (int e = 0; e < 2; ++e) {
+          const int tt = tb + 2 * gq + e;
+          const uint32_t ub = reinterpret_cast<const uint16_t*>(&sm.x[st][tt][slot])[pq];
+          float s = fmaf(Dk, __uint_as_float(ub << 16), tot[e]);
+          if (has_z) {
+            const uint32_t zb = reinterpret_cast<const uint16_t*>(&sm.z[st][tt][slot])[pq];
+            const float zz = __uint_as_float(zb << 16);
+            s = s * zz * sigmoid_fast(zz);
+          }
+          reinterpret_cast<__nv_bfloat16*>(&sm.o[fb][tt][slot])[pq] = __float2bfloat16_rn(s);
+        }
+      }
+    }
+  };
+
+#ifdef LAB_TIMING
+  long long tk_wait = 0, tk_stage = 0, tk_comp = 0, tk0;
+#define TK(acc) { long long now_ = clock64(); acc += now_ - tk0; tk0 = now_; }
+#else
+#define TK(acc)
+#endif
+  // ---- pipeline
+  issue_tile(0);
+  cp_async_wait_all();
+  __syncthreads();
+  issue_tile(1);
+  widen_BC(0);
+#ifdef LAB_TIMING
+  tk0 = clock64();
+#endif
+  for (int i = 0; i < ntiles; ++i) {
+    cp_async_wait_all();
+    __syncthreads();
+    TK(tk_wait)
+    issue_tile(i + 2);
+    if (i >= 1) store_out(i - 1);
+    widen_BC(i + 1);
+    const int t0 = t_begin + i * kTT;
+    if (MODE != kFwdSummary && p.ckpt != nullptr && (t0 % kCkptSteps) == 0 && valid) {
+#pragma unroll
+      for (int q = 0; q < 2; ++q)
+        *reinterpret_cast<float4*>(p.ckpt + (((size_t)b * p.nck + t0 / kCkptSteps) * D + chan(q)) * 16 + 4 * j) =
+            make_float4(h[q][0].x, h[q][0].y, h[q][1].x, h[q][1].y);
+    }
+    TK(tk_stage)
+    if (ap) compute_tile(i, std::true_type{});
+    else compute_tile(i, std::false_type{});
+    TK(tk_comp)
+  }
+#ifdef LAB_TIMING
+  if (tid == 0 && blockIdx.x == 7 && blockIdx.z == 1) printf("cycles: wait %lld stage %lld compute %lld (tiles %d)\n", tk_wait, tk_stage, tk_comp, ntiles);
+#endif
+  cp_async_wait_all();
+  if (FULL) {
+    __syncthreads();
+    store_out(ntiles - 1);
+  }
+  if (MODE == kFwdSummary && valid) {
+#pragma unroll
+    for (int q = 0; q < 2; ++q) {
+      *reinterpret_cast<float4*>(p.seg_end + (((size_t)b * p.nseg + seg) * D + chan(q)) * 16 + 4 * j) =
+          make_float4(h[q][0].x, h[q][0].y, h[q][1].x, h[q][1].y);
+      if (j < 2 && q == 0) p.seg_dsum[((size_t)b * p.nseg + seg) * D + chan(0)] = dsum[0];
+    }
+  }
+}
+
+template <int WARPS, int MODE>
+static cudaError_t launch_fast(const Plan& plan, const FwdParams& p, cudaStream_t s) {
+  constexpr size_t smem = sizeof(FastSmem<WARPS, MODE == kFwdFull>);
+  constexpr int CH = 16 * WARPS;
+  if (smem > 48 * 1024) {
+    cudaError_t e = cudaFuncSetAttribute(ssm_fwd_fast_kernel<WARPS, MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         (int)smem);
+    if (e != cudaSuccess) return e;
+  }
+  dim3 grid((p.D + CH - 1) / CH, plan.nseg, p.batch);
+  ssm_fwd_fast_kernel<WARPS, MODE><<<grid, WARPS * 32, smem, s>>>(p);
+  return cudaGetLastError();
+}
+
+bool fwd_fast_applicable(const ssm_problem_t& prob, const FwdParams& p) {
+  auto al16 = [](const void* q) { return q == nullptr || (reinterpret_cast<uintptr_t>(q) & 15) == 0; };
+  return prob.io_dtype == SSM_BF16 && prob.N == 16 && prob.D % 8 == 0 && al16(p.x) && al16(p.delta) && al16(p.z) &&
+         al16(p.B) && al16(p.C) && al16(p.out) && al16(p.A) && al16(p.h_start) && al16(p.ckpt) && al16(p.seg_end);
+}
+
+cudaError_t launch_fwd_fast(const Plan& plan, const FwdParams& p, int mode, cudaStream_t s) {
+  switch (mode) {
+#ifndef LAB_WARPS
+#define LAB_WARPS 2
+#endif
+    case kFwdFull: return launch_fast<LAB_WARPS, kFwdFull>(plan, p, s);
+    case kFwdSummary: return launch_fast<LAB_WARPS, kFwdSummary>(plan, p, s);
+    default: return launch_fast<LAB_WARPS, kFwdCkptOnly>(plan, p, s);
+  }
+}
+
+}  // namespace ssm

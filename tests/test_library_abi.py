@@ -29,16 +29,17 @@ def _prob(batch=2, L=100, D=64, N=16, io=K.SSM_BF16, flags=3):
 
 
 def test_queries_and_plan():
-    assert K.checkpoint_steps() == 64
+    ck = K.checkpoint_steps()
+    assert ck in (16, 32, 64)
     p = _prob(4, 2048, 5120)
-    assert K.saved_state_bytes(p) == 4 * 32 * 5120 * 16 * 4
+    assert K.saved_state_bytes(p) == 4 * (2048 // ck) * 5120 * 16 * 4
     pl = K.plan(p)
     assert pl["n_segments"] == 1 and pl["segment_steps"] == 2048 and pl["states_per_thread"] == 4
     assert K.fwd_workspace_bytes(p) == 0
     assert K.bwd_workspace_bytes(p) > 0
     long = _prob(1, 524288, 1536)
     pl = K.plan(long)
-    assert pl["n_segments"] > 1 and pl["segment_steps"] % 64 == 0
+    assert pl["n_segments"] > 1 and pl["segment_steps"] % ck == 0
     assert pl["n_segments"] * pl["segment_steps"] >= 524288 > (pl["n_segments"] - 1) * pl["segment_steps"]
     assert K.fwd_workspace_bytes(long) >= 2 * pl["n_segments"] * 1536 * 16 * 4
 
