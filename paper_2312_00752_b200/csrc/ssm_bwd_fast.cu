@@ -5,10 +5,9 @@
 // the 4 lanes of a quad cover the 16 states of the channel pair; a warp covers 16 channels, a block 32.
 //
 // Recomputation in two levels.  The block walks its segment backwards in tiles of 32 steps (one checkpoint block).
-// For a tile it first re-runs the recurrence from the checkpoint state over steps 0..23, keeping the states at steps
-// 8, 16 and 24 in registers; then, for the sub-blocks of 8 steps from last to first, it re-runs the 8 steps keeping
-// every h_t in registers and walks them backwards with the adjoint recurrence.  No state ever goes to shared or
-// global memory except the checkpoints.
+// For a tile it first re-runs the recurrence from the checkpoint state over steps 0..23, parking the states at steps
+// 8, 16 and 24 in shared memory; then, for the sub-blocks of 8 steps from last to first, it re-runs the 8 steps keeping
+// every h_t in registers and walks them backwards with the adjoint recurrence.
 //
 // Sums.  The three per-(step, channel) sums over n (readout for dz, sum lam*B for dx and ddelta, sum w*A for
 // ddelta) are exchanged inside the quad in one batch per sub-block; afterwards every lane finalises 4 steps of one
@@ -26,6 +25,7 @@ namespace {
 
 constexpr int kBT = 32;   // steps per tile = checkpoint spacing
 constexpr int kSB = 8;    // steps per register-resident sub-block
+constexpr int kRB = 4;    // steps between two dB/dC transposes
 static_assert(kBT == kCkptSteps, "the tuned backward kernel restarts from one checkpoint per tile");
 constexpr int kBwdFastWarps = 2;
 constexpr int kBwdFastThreads = kBwdFastWarps * 32;
@@ -43,9 +43,9 @@ struct BwdFastSmem {
   float4 fC[kBT][4];
   float ds[kBT][kBwdFastCH];            // dout * silu(z)
   float gsp[kBT][kBwdFastCH];           // dout * silu'(z)
-  float4 red[kBwdFastWarps][kSB][8][4][2];   // [warp][step][quad][lane in quad][dB quad | dC quad]
+  float4 red[kBwdFastWarps][kRB][8][4][2];   // [warp][step][quad][lane in quad][dB quad | dC quad]
   float acc[kBwdFastWarps][kBT][32];    // per-warp sums over its 16 channels: [step][dB 0..15 | dC 0..15]
-  float4 hsave[kBT / kSB][2][kBwdFastThreads];  // states at the sub-block boundaries, per thread and channel
+  float4 hsave[kBT / kSB - 1][2][kBwdFastThreads];  // states at steps 8, 16, 24 of the tile, per thread and channel
 };
 
 }  // namespace
@@ -155,7 +155,6 @@ __global__ void __launch_bounds__(kBwdFastThreads) ssm_bwd_fast_kernel(const Bwd
       float2 h[2][2];
 #pragma unroll
       for (int q = 0; q < 2; ++q) {
-        sm.hsave[0][q][tid] = ck[q];
         h[q][0] = make_float2(ck[q].x, ck[q].y);
         h[q][1] = make_float2(ck[q].z, ck[q].w);
       }
@@ -178,7 +177,7 @@ __global__ void __launch_bounds__(kBwdFastThreads) ssm_bwd_fast_kernel(const Bwd
         }
       }
 #pragma unroll
-      for (int q = 0; q < 2; ++q) sm.hsave[sb + 1][q][tid] = make_float4(h[q][0].x, h[q][0].y, h[q][1].x, h[q][1].y);
+      for (int q = 0; q < 2; ++q) sm.hsave[sb][q][tid] = make_float4(h[q][0].x, h[q][0].y, h[q][1].x, h[q][1].y);
     }
     }
     // ---- level 2: sub-blocks from last to first
@@ -187,7 +186,7 @@ __global__ void __launch_bounds__(kBwdFastThreads) ssm_bwd_fast_kernel(const Bwd
       float2 hs0[2][2];  // state before the first step of the sub-block
 #pragma unroll
       for (int q = 0; q < 2; ++q) {
-        const float4 v = sm.hsave[sb][q][tid];
+        const float4 v = sb > 0 ? sm.hsave[sb > 0 ? sb - 1 : 0][q][tid] : ck[q];
         hs0[q][0] = make_float2(v.x, v.y);
         hs0[q][1] = make_float2(v.z, v.w);
       }
@@ -266,10 +265,24 @@ __global__ void __launch_bounds__(kBwdFastThreads) ssm_bwd_fast_kernel(const Bwd
           dxp[q] = dtq[q] * lamB;
           ddp[q] = fmaf(uq[q], lamB, (wa.x + wa.y) * kInvLog2e);
         }
-        sm.red[warp][t][quad][j][0] = make_float4(dB01.x, dB01.y, dB23.x, dB23.y);
-        sm.red[warp][t][quad][j][1] = make_float4(dC01.x, dC01.y, dC23.x, dC23.y);
+        sm.red[warp][t % kRB][quad][j][0] = make_float4(dB01.x, dB01.y, dB23.x, dB23.y);
+        sm.red[warp][t % kRB][quad][j][1] = make_float4(dC01.x, dC01.y, dC23.x, dC23.y);
         dxw[t] = dxp[0] + __shfl_xor_sync(0xffffffffu, dxp[1], 1);
         ddw[t] = ddp[0] + __shfl_xor_sync(0xffffffffu, ddp[1], 1);
+        if (t % kRB == 0) {
+          // dB / dC of steps t .. t+kRB-1: sum over the 8 quads of this warp in ascending order;
+          // lane -> (step = lane / 8, state quad = (lane / 2) % 4, dB or dC = lane % 2)
+          __syncwarp();
+          const int tr = lane >> 3, jr = (lane >> 1) & 3, hf = lane & 1;
+          float4 acc4 = sm.red[warp][tr][0][jr][hf];
+#pragma unroll
+          for (int qd = 1; qd < 8; ++qd) {
+            const float4 v = sm.red[warp][tr][qd][jr][hf];
+            acc4.x += v.x; acc4.y += v.y; acc4.z += v.z; acc4.w += v.w;
+          }
+          *reinterpret_cast<float4*>(&sm.acc[warp][sb * kSB + t + tr][16 * hf + 4 * jr]) = acc4;
+          __syncwarp();
+        }
       }
       // second exchange: lanes j and j^2 hold sums of the same channel; the lower keeps steps 0..3, the upper 4..7
       float ytot[4], dxtot[4], ddtot[4];
@@ -294,21 +307,6 @@ __global__ void __launch_bounds__(kBwdFastThreads) ssm_bwd_fast_kernel(const Bwd
         reinterpret_cast<__nv_bfloat16*>(&sm.d[st][tt][slot])[pq] = __float2bfloat16_rn(ddtot[e]);
         reinterpret_cast<__nv_bfloat16*>(&sm.z[st][tt][slot])[pq] = __float2bfloat16_rn(sm.gsp[tt][2 * slot + pq] * s);
       }
-      // dB / dC: sum over the 8 quads of this warp, fixed order; lane -> (step = lane / 4, state quad = lane % 4)
-      __syncwarp();
-      {
-        const int tr = lane >> 2, jr = lane & 3;
-        float4 sb4 = sm.red[warp][tr][0][jr][0], sc4 = sm.red[warp][tr][0][jr][1];
-#pragma unroll
-        for (int qd = 1; qd < 8; ++qd) {
-          const float4 vb = sm.red[warp][tr][qd][jr][0], vc = sm.red[warp][tr][qd][jr][1];
-          sb4.x += vb.x; sb4.y += vb.y; sb4.z += vb.z; sb4.w += vb.w;
-          sc4.x += vc.x; sc4.y += vc.y; sc4.z += vc.z; sc4.w += vc.w;
-        }
-        *reinterpret_cast<float4*>(&sm.acc[warp][sb * kSB + tr][4 * jr]) = sb4;
-        *reinterpret_cast<float4*>(&sm.acc[warp][sb * kSB + tr][16 + 4 * jr]) = sc4;
-      }
-      __syncwarp();
     }
   };
 

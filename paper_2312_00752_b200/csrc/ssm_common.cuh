@@ -102,13 +102,9 @@ enum BwdMode { kBwdFull = 0, kBwdLocal = 1 };
 // ---------------------------------------------------------------------------------------------- device helpers
 #ifdef __CUDACC__
 __device__ __forceinline__ float ex2_approx(float v) {
-#ifdef LAB_NOMUFU
-  return fmaf(v, 0.25f, 1.0f);
-#else
   float r;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(v));
   return r;
-#endif
 }
 __device__ __forceinline__ float rcp_approx(float v) {
   float r;

@@ -14,7 +14,6 @@
 // arithmetic progression (as in the S4D-Real initialisation A_n = -(n+1)) the four decays are built from two
 // exponentials, a_{k} = a_0 r^k with r = 2^(delta * step * log2 e); the test is made per warp at run time and can
 // be disabled by SSM_FLAG_GENERAL_A.
-#include <cstdio>
 #include <type_traits>
 
 #include "ssm_common.cuh"
@@ -25,6 +24,7 @@ namespace {
 
 constexpr int kTT = 32;    // steps per tile
 constexpr int kNST = 3;    // ring stages
+constexpr int kFwdFastWarps = 2;
 
 template <int WARPS, bool FULL>
 struct FastSmem {
@@ -226,15 +226,7 @@ __global__ void __launch_bounds__(WARPS * 32) ssm_fwd_fast_kernel(const FwdParam
         }
       }
       if (tb + SB < kTT) load_sb(tb + SB);
-#ifdef LAB_NOEPI
-      if (FULL) { float acc = 0.f;
-#pragma unroll
-        for (int t = 0; t < SB; ++t) acc += y[t][0] + y[t][1];
-        if (acc == 123.456f) reinterpret_cast<__nv_bfloat16*>(&sm.o[fb][tb][slot])[pq] = __float2bfloat16_rn(acc); }
-      if (false) {
-#else
       if (FULL) {
-#endif
         float w[SB];
 #pragma unroll
         for (int t = 0; t < SB; ++t) w[t] = y[t][0] + __shfl_xor_sync(0xffffffffu, y[t][1], 1);
@@ -261,25 +253,15 @@ __global__ void __launch_bounds__(WARPS * 32) ssm_fwd_fast_kernel(const FwdParam
     }
   };
 
-#ifdef LAB_TIMING
-  long long tk_wait = 0, tk_stage = 0, tk_comp = 0, tk0;
-#define TK(acc) { long long now_ = clock64(); acc += now_ - tk0; tk0 = now_; }
-#else
-#define TK(acc)
-#endif
   // ---- pipeline
   issue_tile(0);
   cp_async_wait_all();
   __syncthreads();
   issue_tile(1);
   widen_BC(0);
-#ifdef LAB_TIMING
-  tk0 = clock64();
-#endif
   for (int i = 0; i < ntiles; ++i) {
     cp_async_wait_all();
     __syncthreads();
-    TK(tk_wait)
     issue_tile(i + 2);
     if (i >= 1) store_out(i - 1);
     widen_BC(i + 1);
@@ -290,14 +272,9 @@ __global__ void __launch_bounds__(WARPS * 32) ssm_fwd_fast_kernel(const FwdParam
         *reinterpret_cast<float4*>(p.ckpt + (((size_t)b * p.nck + t0 / kCkptSteps) * D + chan(q)) * 16 + 4 * j) =
             make_float4(h[q][0].x, h[q][0].y, h[q][1].x, h[q][1].y);
     }
-    TK(tk_stage)
     if (ap) compute_tile(i, std::true_type{});
     else compute_tile(i, std::false_type{});
-    TK(tk_comp)
   }
-#ifdef LAB_TIMING
-  if (tid == 0 && blockIdx.x == 7 && blockIdx.z == 1) printf("cycles: wait %lld stage %lld compute %lld (tiles %d)\n", tk_wait, tk_stage, tk_comp, ntiles);
-#endif
   cp_async_wait_all();
   if (FULL) {
     __syncthreads();
@@ -335,12 +312,9 @@ bool fwd_fast_applicable(const ssm_problem_t& prob, const FwdParams& p) {
 
 cudaError_t launch_fwd_fast(const Plan& plan, const FwdParams& p, int mode, cudaStream_t s) {
   switch (mode) {
-#ifndef LAB_WARPS
-#define LAB_WARPS 2
-#endif
-    case kFwdFull: return launch_fast<LAB_WARPS, kFwdFull>(plan, p, s);
-    case kFwdSummary: return launch_fast<LAB_WARPS, kFwdSummary>(plan, p, s);
-    default: return launch_fast<LAB_WARPS, kFwdCkptOnly>(plan, p, s);
+    case kFwdFull: return launch_fast<kFwdFastWarps, kFwdFull>(plan, p, s);
+    case kFwdSummary: return launch_fast<kFwdFastWarps, kFwdSummary>(plan, p, s);
+    default: return launch_fast<kFwdFastWarps, kFwdCkptOnly>(plan, p, s);
   }
 }
 
