@@ -27,6 +27,9 @@ if ROOT not in sys.path:
 
 METRIC = "selective-scan fwd+bwd elements/s (elements = batch*L*D); achieved HBM GB/s as % of measured B200 peak"
 FALLBACK_HBM_GBS = 6650.0
+# DRAM bytes (read + write) of one launch of the dominant kernel from an ncu capture at the bench workload itself
+# (profiles/ssm_bwd_fast_kernel_mamba2p8b_layer.md); None where no capture exists.
+NCU_TRAFFIC_BYTES = {3: 420.6e6 + 380.5e6}
 
 
 def parse_args():
@@ -108,6 +111,22 @@ class ClockSampler:
                     reasons.add(nm)
         return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
                 "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def max_over_ranks(value: float, device="cpu") -> float:
+    """Slowest rank's value (the whole job is as slow as its slowest replica); identity for a single process."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return float(value)
+    t = torch.tensor([value], device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def job_value(elements_per_rank: int, world: int, ms_per_step: float) -> float:
+    """Whole-job throughput of `world` replicas that each process `elements_per_rank` per step (weak scaling)."""
+    return world * elements_per_rank / (ms_per_step * 1e-3)
 
 
 def kernels_per_step(plan_info: dict) -> int:
@@ -247,11 +266,7 @@ def run_ours(args, cfg):
     total_ms = ev[0][0].elapsed_time(ev[-1][2])
     fwd_ms = [e[0].elapsed_time(e[1]) for e in ev]
     bwd_ms = [e[1].elapsed_time(e[2]) for e in ev]
-    ms_per_step = total_ms / args.steps
-    if world > 1:
-        t = torch.tensor([ms_per_step], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_per_step = float(t.item())
+    ms_per_step = max_over_ranks(total_ms / args.steps, dev)
 
     # ---- end to end: pinned host inputs -> device, fwd + bwd, every result back to pinned host memory
     e2e = None
@@ -280,12 +295,8 @@ def run_ours(args, cfg):
             e2e_step()
         b.record(stream)
         barrier()
-        e2e_ms = a.elapsed_time(b) / n_e2e
-        if world > 1:
-            t = torch.tensor([e2e_ms], device=dev, dtype=torch.float64)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            e2e_ms = float(t.item())
-        e2e = {"value": world * cfg.elements / (e2e_ms * 1e-3), "unit": "elements/s",
+        e2e_ms = max_over_ranks(a.elapsed_time(b) / n_e2e, dev)
+        e2e = {"value": job_value(cfg.elements, world, e2e_ms), "unit": "elements/s",
                "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h), "ms_per_step": e2e_ms,
                "steps": n_e2e}
 
@@ -300,7 +311,7 @@ def run_ours(args, cfg):
     bwd_gbs = bwd_bytes / (b_ms * 1e-3) / 1e9
     fwd_gbs = fwd_bytes / (f_ms * 1e-3) / 1e9
     line = {
-        "metric": METRIC, "value": world * cfg.elements / (ms_per_step * 1e-3), "unit": "elements/s",
+        "metric": METRIC, "value": job_value(cfg.elements, world, ms_per_step), "unit": "elements/s",
         "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
         "config": {"workload": f"{cfg.name} (config {cfg.cfg_id}): batch {cfg.batch}, L {cfg.L}, D {cfg.D}, N {cfg.N}, "
@@ -318,7 +329,9 @@ def run_ours(args, cfg):
                 "achieved_gbs": bwd_gbs, "frac_of_hbm_peak": bwd_gbs / peak},
         "roofline": {"bound": "hbm", "kernel": "ssm_scan_bwd call (backward kernel + its reduction kernel)",
                      "achieved": bwd_gbs, "peak": peak, "peak_kind": f"{peak_kind} copy bandwidth",
-                     "unit": "GB/s", "frac": bwd_gbs / peak, "traffic": None},
+                     "unit": "GB/s", "frac": bwd_gbs / peak,
+                     "traffic": NCU_TRAFFIC_BYTES.get(cfg.cfg_id) if not args.general_A else None,
+                     "algorithmic_bytes": bwd_bytes},
         "wall_s_timed_region": t_wall,
     }
     if e2e is not None:
