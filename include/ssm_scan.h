@@ -122,6 +122,29 @@ SSM_API ssm_status_t ssm_scan_bwd(const ssm_problem_t* p, const void* x, const v
                           const void* saved_states, void* dx, void* ddelta, float* dA, void* dB, void* dC, float* dD,
                           void* dz, void* workspace, size_t workspace_bytes, void* stream /* cudaStream_t */);
 
+/*
+ * Forward without any caller-provided scratch memory.  (The paper has no counterpart: this entry point exists for
+ * the integration of the library, not for the method.)
+ *
+ * It is for callers that are not allowed to allocate device memory at the point where they call the scan -- for
+ * example a layer plug-in that receives only its input and output buffers from a host framework and must not
+ * allocate while enqueueing work, because a device allocation synchronises the GPU, or an application whose memory
+ * budget is fixed at start-up.  Same arguments and results as ssm_scan_fwd, minus the workspace: the scratch memory
+ * of the time-split forward path is a fixed array of SSM_STATIC_SCRATCH_BYTES bytes inside the library's device
+ * image, present on every GPU that loads the library until the process exits.
+ *   - A problem whose ssm_scan_fwd_workspace_bytes() exceeds SSM_STATIC_SCRATCH_BYTES is refused with
+ *     SSM_ERR_WORKSPACE before anything is launched; use ssm_scan_fwd with your own workspace for those.
+ *   - The call allocates and frees nothing.  The first call on a device looks up the device address of the array
+ *     (with that device current) and keeps it; make that first call outside any stream capture.
+ *   - All calls on a device share the one array: two calls that can overlap on the GPU (different streams, no
+ *     dependency between them) race on it and must be ordered by the caller.  The array keeps the contents of the last
+ *     call; the kernels overwrite every word of it before they read it, so nothing needs clearing in between.
+ */
+#define SSM_STATIC_SCRATCH_BYTES (4u << 20)
+SSM_API ssm_status_t ssm_scan_fwd_static(const ssm_problem_t* p, const void* x, const void* delta, const float* A,
+                                         const void* B, const void* C, const float* D_skip, const void* z, void* out,
+                                         void* saved_states, void* stream /* cudaStream_t */);
+
 /* Human-readable name of a status code (static storage). */
 SSM_API const char* ssm_status_string(ssm_status_t s);
 

@@ -20,7 +20,9 @@ SSM_FLAG_HAS_Z, SSM_FLAG_HAS_DSKIP, SSM_FLAG_SAVE_STATES, SSM_FLAG_GENERAL_A = 1
 EXPORTED_SYMBOLS = (
     "ssm_scan_fwd_workspace_bytes", "ssm_scan_bwd_workspace_bytes", "ssm_scan_saved_state_bytes",
     "ssm_scan_checkpoint_steps", "ssm_scan_fwd", "ssm_scan_bwd", "ssm_status_string", "ssm_scan_plan",
+    "ssm_scan_fwd_static",
 )
+SSM_STATIC_SCRATCH_BYTES = 4 << 20
 
 
 class ssm_problem_t(ctypes.Structure):
@@ -65,6 +67,8 @@ def load_library() -> ctypes.CDLL:
     lib.ssm_scan_fwd.argtypes = [P] + [vp] * 9 + [vp, sz, vp]
     lib.ssm_scan_bwd.restype = ctypes.c_int
     lib.ssm_scan_bwd.argtypes = [P] + [vp] * 16 + [vp, sz, vp]
+    lib.ssm_scan_fwd_static.restype = ctypes.c_int
+    lib.ssm_scan_fwd_static.argtypes = [P] + [vp] * 9 + [vp]
     _lib = lib
     return lib
 
@@ -174,6 +178,31 @@ def ssm_scan_fwd(x, delta, A, B, C, D_skip=None, z=None, *, save_states=False, g
         _dev_ptr(ws, "workspace"), ctypes.c_size_t(0 if ws is None else ws.numel() * ws.element_size()),
         ctypes.c_void_p(stream_ptr))
     _check(code, "ssm_scan_fwd")
+    return (out, saved_states) if save_states else out
+
+
+def ssm_scan_fwd_static(x, delta, A, B, C, D_skip=None, z=None, *, save_states=False, general_A=False, out=None,
+                        saved_states=None, stream=None):
+    """ssm_scan_fwd for callers that may not allocate: no workspace argument, and this wrapper allocates none either
+    when `out` (and `saved_states`, if asked for) are passed in.  The scratch memory is the fixed array inside the
+    library (SSM_STATIC_SCRATCH_BYTES); a problem that needs more raises SsmScanError (SSM_ERR_WORKSPACE).  Calls that
+    may overlap on the GPU must be ordered by the caller, because they share that array."""
+    lib = load_library()
+    prob = make_problem(x, B, z is not None, D_skip is not None, save_states, general_A)
+    batch, L, D, N = prob.batch, prob.L, prob.D, prob.N
+    io = x.dtype
+    if out is None:
+        out = torch.empty_like(x)
+    if save_states and saved_states is None:
+        saved_states = torch.empty(saved_state_bytes(prob) // 4, dtype=torch.float32, device=x.device)
+    stream_ptr = (stream if stream is not None else torch.cuda.current_stream(x.device)).cuda_stream
+    code = lib.ssm_scan_fwd_static(
+        ctypes.byref(prob), _dev_ptr(x, "x", (batch, L, D), io), _dev_ptr(delta, "delta", (batch, L, D), io),
+        _dev_ptr(A, "A", (D, N), torch.float32), _dev_ptr(B, "B", (batch, L, N), io),
+        _dev_ptr(C, "C", (batch, L, N), io), _dev_ptr(D_skip, "D_skip", (D,), torch.float32),
+        _dev_ptr(z, "z", (batch, L, D), io), _dev_ptr(out, "out", (batch, L, D), io),
+        _dev_ptr(saved_states if save_states else None, "saved_states"), ctypes.c_void_p(stream_ptr))
+    _check(code, "ssm_scan_fwd_static")
     return (out, saved_states) if save_states else out
 
 
