@@ -1,18 +1,20 @@
 // Forward selective scan, tuned path: bf16 io, N = 16, D % 8 == 0, 16-byte aligned pointers.
 // Same mathematics and modes as ssm_fwd.cu (Algorithm 2 steps 5-6; Eq. 2a/2b; Eq. 4's A-bar; fused skip and gate).
 //
-// Mapping.  A thread owns 4 states of 2 adjacent channels (8 recurrences, held as packed float2 pairs so that the
-// multiply-adds issue as two-wide FP32 instructions); the 4 lanes of a quad cover the 16 states of the channel
+// Mapping.  A compute thread owns 4 states of 2 adjacent channels (8 recurrences, held as packed float2 pairs so that
+// the multiply-adds issue as two-wide FP32 instructions); the 4 lanes of a quad cover the 16 states of the channel
 // pair; a warp covers 16 channels and sweeps time sequentially.  The sum over n of the readout is completed inside
-// the quad by a two-step exchange that leaves the total of channel 0 in even lanes and of channel 1 in odd lanes.
+// the quad by a batched two-step exchange, after which every lane holds the totals of two (step, channel) pairs.
 //
-// Staging.  x, delta, z and B, C arrive by 16-byte cp.async into a three-stage ring of [32 steps x channels] tiles
-// (one __syncthreads per tile); B and C are widened to float once per block and tile, so the inner loop reads them
-// as 128-bit broadcast loads; the output tile is assembled in shared memory and written with 16-byte stores.
+// Warp roles.  A block has WARPS compute warps and one service warp.  The service warp issues the 16-byte cp.async
+// copies of x, delta, z, B, C into a three-stage ring of [32 steps x channels] tiles, widens B and C to float, and
+// finishes the previous tile: it adds the skip term to the readout totals the compute warps left in shared memory,
+// applies the SiLU gate, rounds to bf16 and writes the output tile with 16-byte stores -- all while the compute warps
+// run the recurrence of the current tile.  The two roles meet at one block-wide barrier per tile.
 //
 // Discretization.  a = 2^(delta * A * log2 e) with the hardware ex2.  When the four A values of a thread form an
 // arithmetic progression (as in the S4D-Real initialisation A_n = -(n+1)) the four decays are built from two
-// exponentials, a_{k} = a_0 r^k with r = 2^(delta * step * log2 e); the test is made per warp at run time and can
+// exponentials, a_k = a_0 r^k with r = 2^(delta * step * log2 e); the test is made per warp at run time and can
 // be disabled by SSM_FLAG_GENERAL_A.
 #include <type_traits>
 
@@ -24,7 +26,6 @@ namespace {
 
 constexpr int kTT = 32;    // steps per tile
 constexpr int kNST = 3;    // ring stages
-constexpr int kFwdFastWarps = 2;
 
 template <int WARPS, bool FULL>
 struct FastSmem {
@@ -36,32 +37,30 @@ struct FastSmem {
   uint32_t rawC[FULL ? kNST : 1][FULL ? kTT : 1][8];
   float4 fB[2][kTT][4];
   float4 fC[FULL ? 2 : 1][FULL ? kTT : 1][4];
-  uint32_t o[FULL ? 2 : 1][FULL ? kTT : 1][CH / 2];
+  float yp[FULL ? 2 : 1][FULL ? kTT : 1][CH];      // readout totals sum_n C h of a tile, per (step, channel)
+  uint32_t o[FULL ? kTT : 1][CH / 2];              // output tile (bf16 pairs), owned by the service warp
 };
+
+__device__ __forceinline__ void block_barrier(int nthreads) {
+  asm volatile("bar.sync 1, %0;" ::"r"(nthreads) : "memory");
+}
+__device__ __forceinline__ void cp_async_wait_but_one() { asm volatile("cp.async.wait_group 1;" ::: "memory"); }
 
 }  // namespace
 
 template <int WARPS, int MODE>
-__global__ void __launch_bounds__(WARPS * 32) ssm_fwd_fast_kernel(const FwdParams p) {
+__global__ void __launch_bounds__((WARPS + 1) * 32) ssm_fwd_fast_kernel(const FwdParams p) {
   constexpr bool FULL = (MODE == kFwdFull);
-  constexpr int THREADS = WARPS * 32;
+  constexpr int THREADS = (WARPS + 1) * 32;
   constexpr int CH = 16 * WARPS;
-  constexpr int CHUNKS = CH / 8;  // 16-byte chunks per tile row
+  constexpr int CHUNKS = CH / 8;              // 16-byte chunks per tile row
+  constexpr int ROWS_PER_PASS = 32 / CHUNKS;  // tile rows one pass of the staging warp covers
   using Smem = FastSmem<WARPS, FULL>;
   extern __shared__ __align__(16) unsigned char smem_raw[];
   Smem& sm = *reinterpret_cast<Smem*>(smem_raw);
 
-  const __nv_bfloat16* __restrict__ gx = static_cast<const __nv_bfloat16*>(p.x);
-  const __nv_bfloat16* __restrict__ gd = static_cast<const __nv_bfloat16*>(p.delta);
-  const __nv_bfloat16* __restrict__ gz = static_cast<const __nv_bfloat16*>(p.z);
-  const __nv_bfloat16* __restrict__ gB = static_cast<const __nv_bfloat16*>(p.B);
-  const __nv_bfloat16* __restrict__ gC = static_cast<const __nv_bfloat16*>(p.C);
-  __nv_bfloat16* __restrict__ gout = static_cast<__nv_bfloat16*>(p.out);
-
   const int tid = threadIdx.x;
-  const int lane = tid & 31;
-  const int j = lane & 3;
-  const int slot = (tid >> 5) * 8 + (lane >> 2);  // channel pair within the block
+  const int lane = tid & 31, warp = tid >> 5;
   const int d_cta = blockIdx.x * CH;
   const int seg = blockIdx.y;
   const int b = blockIdx.z;
@@ -69,6 +68,119 @@ __global__ void __launch_bounds__(WARPS * 32) ssm_fwd_fast_kernel(const FwdParam
   const int t_begin = seg * p.seg_steps;
   const int t_end = min(p.L, t_begin + p.seg_steps);
   const int ntiles = (t_end - t_begin + kTT - 1) / kTT;
+  const bool has_z = FULL && p.z != nullptr;
+
+  if (warp == WARPS) {
+    // ================================================================== service warp
+    const __nv_bfloat16* __restrict__ gx = static_cast<const __nv_bfloat16*>(p.x);
+    const __nv_bfloat16* __restrict__ gd = static_cast<const __nv_bfloat16*>(p.delta);
+    const __nv_bfloat16* __restrict__ gz = static_cast<const __nv_bfloat16*>(p.z);
+    const __nv_bfloat16* __restrict__ gB = static_cast<const __nv_bfloat16*>(p.B);
+    const __nv_bfloat16* __restrict__ gC = static_cast<const __nv_bfloat16*>(p.C);
+    __nv_bfloat16* __restrict__ gout = static_cast<__nv_bfloat16*>(p.out);
+    const int cc = lane % CHUNKS, r0 = lane / CHUNKS;  // this lane's chunk column and first row of every pass
+    const bool col_ok = d_cta + cc * 8 < D;
+    const size_t seg_row0 = (size_t)b * p.L + t_begin;
+
+    auto issue_tile = [&](int i) {
+      if (i < ntiles) {
+        const int st = i % kNST;
+        const int t0 = t_begin + i * kTT;
+        const size_t row0 = seg_row0 + (size_t)i * kTT;
+#pragma unroll
+        for (int k = 0; k < kTT / ROWS_PER_PASS; ++k) {
+          const int tt = r0 + k * ROWS_PER_PASS;
+          const bool ok = col_ok && (t0 + tt < t_end);
+          const size_t g = ok ? (row0 + tt) * D + d_cta + cc * 8 : 0;
+          cp_async16(&sm.x[st][tt][cc * 4], gx + g, ok);
+          cp_async16(&sm.d[st][tt][cc * 4], gd + g, ok);
+          if (FULL) cp_async16(&sm.z[st][tt][cc * 4], (has_z ? gz : gx) + g, ok && has_z);
+        }
+#pragma unroll
+        for (int k = 0; k < 2; ++k) {
+          const int c = lane + 32 * k;
+          const int tt = c >> 1, hc = c & 1;
+          const bool ok = t0 + tt < t_end;
+          const size_t g = ok ? (row0 + tt) * 16 + hc * 8 : 0;
+          cp_async16(&sm.rawB[st][tt][hc * 4], gB + g, ok);
+          if (FULL) cp_async16(&sm.rawC[st][tt][hc * 4], gC + g, ok);
+        }
+      }
+      cp_async_commit();
+    };
+    auto widen_BC = [&](int i) {  // tile i: bf16 -> float
+      if (i >= ntiles) return;
+      const int st = i % kNST, fb = i & 1;
+#pragma unroll
+      for (int k = 0; k < kTT * 8 / 32; ++k) {
+        const int c = lane + 32 * k;
+        const int tt = c >> 3, w = c & 7;
+        const uint32_t vb = sm.rawB[st][tt][w];
+        reinterpret_cast<float2*>(&sm.fB[fb][tt][0])[w] = make_float2(bf16lo(vb), bf16hi(vb));
+        if (FULL) {
+          const uint32_t vc = sm.rawC[st][tt][w];
+          reinterpret_cast<float2*>(&sm.fC[fb][tt][0])[w] = make_float2(bf16lo(vc), bf16hi(vc));
+        }
+      }
+    };
+    // skip term, gate and rounding of tile i (its readout totals are complete), then the 16-byte stores
+    const int eslot = lane % (CH / 2), et0 = lane / (CH / 2);   // this lane's channel pair and first step
+    constexpr int ESTEP = 32 / (CH / 2);
+    float2 Dk2 = make_float2(0.f, 0.f);
+    if (FULL && p.Dskip != nullptr && d_cta + 2 * eslot < D)
+      Dk2 = *reinterpret_cast<const float2*>(p.Dskip + d_cta + 2 * eslot);
+    auto finish_tile = [&](int i) {
+      if (!FULL) return;
+      const int st = i % kNST, yb = i & 1;
+#pragma unroll 4
+      for (int tt = et0; tt < kTT; tt += ESTEP) {
+        const float2 y = *reinterpret_cast<const float2*>(&sm.yp[yb][tt][2 * eslot]);
+        const uint32_t xw = sm.x[st][tt][eslot];
+        float s0 = fmaf(Dk2.x, bf16lo(xw), y.x), s1 = fmaf(Dk2.y, bf16hi(xw), y.y);
+        if (has_z) {
+          const uint32_t zw = sm.z[st][tt][eslot];
+          const float z0 = bf16lo(zw), z1 = bf16hi(zw);
+          s0 = s0 * z0 * sigmoid_fast(z0);
+          s1 = s1 * z1 * sigmoid_fast(z1);
+        }
+        const __nv_bfloat162 r = __floats2bfloat162_rn(s0, s1);
+        sm.o[tt][eslot] = *reinterpret_cast<const uint32_t*>(&r);
+      }
+      __syncwarp();
+      const int t0 = t_begin + i * kTT;
+      const size_t row0 = seg_row0 + (size_t)i * kTT;
+#pragma unroll
+      for (int k = 0; k < kTT / ROWS_PER_PASS; ++k) {
+        const int tt = r0 + k * ROWS_PER_PASS;
+        if (col_ok && t0 + tt < t_end)
+          *reinterpret_cast<uint4*>(gout + (row0 + tt) * D + d_cta + cc * 8) =
+              *reinterpret_cast<const uint4*>(&sm.o[tt][cc * 4]);
+      }
+      __syncwarp();
+    };
+
+    issue_tile(0);
+    issue_tile(1);
+    cp_async_wait_but_one();
+    __syncwarp();
+    widen_BC(0);
+    for (int i = 0; i < ntiles; ++i) {
+      block_barrier(THREADS);  // tile i is staged; the compute warps are done with tile i-1
+      if (i >= 1) finish_tile(i - 1);  // reads x and z of the ring stage that tile i+2 is about to overwrite
+      issue_tile(i + 2);
+      cp_async_wait_but_one();
+      __syncwarp();
+      widen_BC(i + 1);
+    }
+    cp_async_wait_all();
+    block_barrier(THREADS);
+    finish_tile(ntiles - 1);
+    return;
+  }
+
+  // ==================================================================== compute warps
+  const int j = lane & 3;
+  const int slot = warp * 8 + (lane >> 2);  // channel pair within the block
   const int d0 = d_cta + 2 * slot;  // first channel of this quad's pair (D is even, so both are valid or neither)
   const bool valid = d0 < D;
   const int pq = j & 1, gq = j >> 1;
@@ -77,7 +189,6 @@ __global__ void __launch_bounds__(WARPS * 32) ssm_fwd_fast_kernel(const FwdParam
   // pick the matching half of a packed bf16 pair and widen it to float in one instruction.
   const uint32_t selA = pq ? 0x3244u : 0x1044u, selB = pq ? 0x1044u : 0x3244u;
   auto chan = [&](int q) { return d0 + (q ^ pq); };
-  const bool has_z = FULL && gz != nullptr;
 
   // ---- per-thread constants and state
   float2 A2[2][2];   // A * log2(e), states (4j, 4j+1) and (4j+2, 4j+3) of each channel
@@ -101,59 +212,11 @@ __global__ void __launch_bounds__(WARPS * 32) ssm_fwd_fast_kernel(const FwdParam
     h[q][1] = make_float2(hs.z, hs.w);
   }
   ap = __all_sync(0xffffffffu, ap);
-  const float Dk = (FULL && valid && p.Dskip != nullptr) ? p.Dskip[d0 + pq] : 0.f;
 
-  auto issue_tile = [&](int i) {
-    if (i < ntiles) {
-      const int st = i % kNST;
-      const int t0 = t_begin + i * kTT;
-      const size_t row0 = (size_t)b * p.L + t0;
-      for (int c = tid; c < kTT * CHUNKS; c += THREADS) {
-        const int tt = c / CHUNKS, cc = c % CHUNKS;
-        const bool ok = (t0 + tt < t_end) && (d_cta + cc * 8 < D);
-        const size_t g = ok ? (row0 + tt) * D + d_cta + cc * 8 : 0;
-        cp_async16(&sm.x[st][tt][cc * 4], gx + g, ok);
-        cp_async16(&sm.d[st][tt][cc * 4], gd + g, ok);
-        if (FULL) cp_async16(&sm.z[st][tt][cc * 4], (has_z ? gz : gx) + g, ok && has_z);
-      }
-      for (int c = tid; c < kTT * 2; c += THREADS) {
-        const int tt = c >> 1, cc = c & 1;
-        const bool ok = t0 + tt < t_end;
-        const size_t g = ok ? (row0 + tt) * 16 + cc * 8 : 0;
-        cp_async16(&sm.rawB[st][tt][cc * 4], gB + g, ok);
-        if (FULL) cp_async16(&sm.rawC[st][tt][cc * 4], gC + g, ok);
-      }
-    }
-    cp_async_commit();
-  };
-  auto widen_BC = [&](int i) {  // tile i: bf16 -> float
-    if (i >= ntiles) return;
-    const int st = i % kNST, fb = i & 1;
-    for (int c = tid; c < kTT * 8; c += THREADS) {
-      const int tt = c >> 3, w = c & 7;
-      const uint32_t vb = sm.rawB[st][tt][w];
-      reinterpret_cast<float2*>(&sm.fB[fb][tt][0])[w] = make_float2(bf16lo(vb), bf16hi(vb));
-      if (FULL) {
-        const uint32_t vc = sm.rawC[st][tt][w];
-        reinterpret_cast<float2*>(&sm.fC[fb][tt][0])[w] = make_float2(bf16lo(vc), bf16hi(vc));
-      }
-    }
-  };
-  auto store_out = [&](int i) {  // tile i: shared -> global, 16 bytes per thread and iteration
-    if (!FULL) return;
-    const int t0 = t_begin + i * kTT;
-    const size_t row0 = (size_t)b * p.L + t0;
-    for (int c = tid; c < kTT * CHUNKS; c += THREADS) {
-      const int tt = c / CHUNKS, cc = c % CHUNKS;
-      if (t0 + tt < t_end && d_cta + cc * 8 < D)
-        *reinterpret_cast<uint4*>(gout + (row0 + tt) * D + d_cta + cc * 8) =
-            *reinterpret_cast<const uint4*>(&sm.o[i & 1][tt][cc * 4]);
-    }
-  };
 
   // One tile of kTT steps, in sub-blocks of 4 steps: the loads of the next sub-block are issued before the
   // shared-memory stores of the current one, and the readout sums of 4 steps x 2 channels are exchanged inside the
-  // quad in one batch, after which every lane finalises two (step, channel) values.  Rows past the end of the
+  // quad in one batch, after which every lane leaves the totals of two (step, channel) pairs in shared memory for the service warp.  Rows past the end of the
   // segment were zero-filled: delta = 0 gives a = 1 and no input, so they leave the state untouched.
   auto compute_tile = [&](int i, auto ap_tag) {
     constexpr bool AP = decltype(ap_tag)::value;
@@ -237,34 +300,14 @@ __global__ void __launch_bounds__(WARPS * 32) ssm_fwd_fast_kernel(const FwdParam
           const float keep = gq ? w[2 + e] : w[e], send = gq ? w[e] : w[2 + e];
           tot[e] = keep + __shfl_xor_sync(0xffffffffu, send, 2);
         }
-#pragma unroll
-        for (int e = 0; e < 2; ++e) {
-          const int tt = tb + 2 * gq + e;
-          const uint32_t ub = reinterpret_cast<const uint16_t*>(&sm.x[st][tt][slot])[pq];
-          float s = fmaf(Dk, __uint_as_float(ub << 16), tot[e]);
-          if (has_z) {
-            const uint32_t zb = reinterpret_cast<const uint16_t*>(&sm.z[st][tt][slot])[pq];
-            const float zz = __uint_as_float(zb << 16);
-            s = s * zz * sigmoid_fast(zz);
-          }
-          reinterpret_cast<__nv_bfloat16*>(&sm.o[fb][tt][slot])[pq] = __float2bfloat16_rn(s);
-        }
+        sm.yp[fb][tb + 2 * gq][2 * slot + pq] = tot[0];
+        sm.yp[fb][tb + 2 * gq + 1][2 * slot + pq] = tot[1];
       }
     }
   };
 
-  // ---- pipeline
-  issue_tile(0);
-  cp_async_wait_all();
-  __syncthreads();
-  issue_tile(1);
-  widen_BC(0);
   for (int i = 0; i < ntiles; ++i) {
-    cp_async_wait_all();
-    __syncthreads();
-    issue_tile(i + 2);
-    if (i >= 1) store_out(i - 1);
-    widen_BC(i + 1);
+    block_barrier(THREADS);
     const int t0 = t_begin + i * kTT;
     if (MODE != kFwdSummary && p.ckpt != nullptr && (t0 % kCkptSteps) == 0 && valid) {
 #pragma unroll
@@ -275,11 +318,7 @@ __global__ void __launch_bounds__(WARPS * 32) ssm_fwd_fast_kernel(const FwdParam
     if (ap) compute_tile(i, std::true_type{});
     else compute_tile(i, std::false_type{});
   }
-  cp_async_wait_all();
-  if (FULL) {
-    __syncthreads();
-    store_out(ntiles - 1);
-  }
+  block_barrier(THREADS);
   if (MODE == kFwdSummary && valid) {
 #pragma unroll
     for (int q = 0; q < 2; ++q) {
@@ -300,7 +339,7 @@ static cudaError_t launch_fast(const Plan& plan, const FwdParams& p, cudaStream_
     if (e != cudaSuccess) return e;
   }
   dim3 grid((p.D + CH - 1) / CH, plan.nseg, p.batch);
-  ssm_fwd_fast_kernel<WARPS, MODE><<<grid, WARPS * 32, smem, s>>>(p);
+  ssm_fwd_fast_kernel<WARPS, MODE><<<grid, (WARPS + 1) * 32, smem, s>>>(p);
   return cudaGetLastError();
 }
 
@@ -309,6 +348,8 @@ bool fwd_fast_applicable(const ssm_problem_t& prob, const FwdParams& p) {
   return prob.io_dtype == SSM_BF16 && prob.N == 16 && prob.D % 8 == 0 && al16(p.x) && al16(p.delta) && al16(p.z) &&
          al16(p.B) && al16(p.C) && al16(p.out) && al16(p.A) && al16(p.h_start) && al16(p.ckpt) && al16(p.seg_end);
 }
+
+constexpr int kFwdFastWarps = 2;
 
 cudaError_t launch_fwd_fast(const Plan& plan, const FwdParams& p, int mode, cudaStream_t s) {
   switch (mode) {
