@@ -60,7 +60,7 @@ typedef enum {
   SSM_ERR_UNSUPPORTED = 2,  /* N or dtype outside the supported set                                             */
   SSM_ERR_WORKSPACE = 3,    /* workspace null / misaligned / smaller than the query reports                     */
   SSM_ERR_CUDA = 4,         /* a CUDA runtime call or a kernel launch failed                                    */
-  SSM_ERR_TIMEOUT = 5       /* a bounded device-side wait gave up (reported through ssm_scan_check_status)      */
+  SSM_ERR_TIMEOUT = 5       /* a bounded device-side wait gave up (reported by ssm_scan_check_status)           */
 } ssm_status_t;
 
 typedef enum { SSM_F32 = 0, SSM_BF16 = 1 } ssm_dtype_t;
@@ -70,7 +70,10 @@ enum {
   SSM_FLAG_HAS_DSKIP = 2u,    /* D_skip is given; otherwise the skip term is absent and dD is not produced      */
   SSM_FLAG_SAVE_STATES = 4u,  /* forward: also write the checkpoint states that backward starts its recomputation
                                  from (Appendix D keeps "intermediate scan states" between chunks)             */
-  SSM_FLAG_GENERAL_A = 8u     /* do not use the fast path for rows of A that are arithmetic progressions in n   */
+  SSM_FLAG_GENERAL_A = 8u,    /* do not use the fast path for rows of A that are arithmetic progressions in n   */
+  SSM_FLAG_TEST_WITHHOLD = 16u /* test hook for the bounded waits: the tuned backward kernel never publishes its
+                                 hand-off flags and polls only 1000 times, so every dependent tile gives up and
+                                 ssm_scan_check_status reports SSM_ERR_TIMEOUT; the gradients are then undefined  */
 };
 
 typedef struct {
@@ -121,6 +124,15 @@ SSM_API ssm_status_t ssm_scan_bwd(const ssm_problem_t* p, const void* x, const v
                           const void* C, const float* D_skip, const void* z, const void* dout,
                           const void* saved_states, void* dx, void* ddelta, float* dA, void* dB, void* dC, float* dD,
                           void* dz, void* workspace, size_t workspace_bytes, void* stream /* cudaStream_t */);
+
+/*
+ * Reads back whether the last ssm_scan_bwd on this workspace completed.  The tuned backward kernel passes the adjoint
+ * from one tile of a channel group to the next through a hand-off buffer and waits (with a bounded number of polls)
+ * for the tile it depends on; if such a wait ever gives up, every block stops and an abort word is left in the
+ * workspace.  This call synchronises `stream`, copies that word to the host and returns SSM_ERR_TIMEOUT if it is set
+ * (the gradients of that call are then incomplete), SSM_OK otherwise.  `p` and `workspace` must be those of the call.
+ */
+SSM_API ssm_status_t ssm_scan_check_status(const ssm_problem_t* p, const void* workspace, void* stream /* cudaStream_t */);
 
 /*
  * Forward without any caller-provided scratch memory.  (The paper has no counterpart: this entry point exists for

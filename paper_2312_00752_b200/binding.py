@@ -15,12 +15,12 @@ from . import build as _build
 
 SSM_OK = 0
 SSM_F32, SSM_BF16 = 0, 1
-SSM_FLAG_HAS_Z, SSM_FLAG_HAS_DSKIP, SSM_FLAG_SAVE_STATES, SSM_FLAG_GENERAL_A = 1, 2, 4, 8
+SSM_FLAG_HAS_Z, SSM_FLAG_HAS_DSKIP, SSM_FLAG_SAVE_STATES, SSM_FLAG_GENERAL_A, SSM_FLAG_TEST_WITHHOLD = 1, 2, 4, 8, 16
 
 EXPORTED_SYMBOLS = (
     "ssm_scan_fwd_workspace_bytes", "ssm_scan_bwd_workspace_bytes", "ssm_scan_saved_state_bytes",
     "ssm_scan_checkpoint_steps", "ssm_scan_fwd", "ssm_scan_bwd", "ssm_status_string", "ssm_scan_plan",
-    "ssm_scan_fwd_static",
+    "ssm_scan_fwd_static", "ssm_scan_check_status",
 )
 SSM_STATIC_SCRATCH_BYTES = 4 << 20
 
@@ -67,6 +67,8 @@ def load_library() -> ctypes.CDLL:
     lib.ssm_scan_fwd.argtypes = [P] + [vp] * 9 + [vp, sz, vp]
     lib.ssm_scan_bwd.restype = ctypes.c_int
     lib.ssm_scan_bwd.argtypes = [P] + [vp] * 16 + [vp, sz, vp]
+    lib.ssm_scan_check_status.restype = ctypes.c_int
+    lib.ssm_scan_check_status.argtypes = [P, vp, vp]
     lib.ssm_scan_fwd_static.restype = ctypes.c_int
     lib.ssm_scan_fwd_static.argtypes = [P] + [vp] * 9 + [vp]
     _lib = lib
@@ -181,6 +183,19 @@ def ssm_scan_fwd(x, delta, A, B, C, D_skip=None, z=None, *, save_states=False, g
     return (out, saved_states) if save_states else out
 
 
+def check_status(problem: ssm_problem_t, workspace: torch.Tensor, stream=None) -> None:
+    """Synchronises the stream and raises SsmScanError if the last backward call on `workspace` gave up a wait."""
+    stream_ptr = (stream if stream is not None else torch.cuda.current_stream(workspace.device)).cuda_stream
+    _check(load_library().ssm_scan_check_status(ctypes.byref(problem), ctypes.c_void_p(workspace.data_ptr()),
+                                                ctypes.c_void_p(stream_ptr)), "ssm_scan_check_status")
+
+
+def last_bwd_workspace(device, stream=None):
+    """The cached workspace tensor the binding used for calls on (device, stream), or None."""
+    stream_ptr = (stream if stream is not None else torch.cuda.current_stream(device)).cuda_stream
+    return _workspaces.get((str(device), int(stream_ptr)))
+
+
 def ssm_scan_fwd_static(x, delta, A, B, C, D_skip=None, z=None, *, save_states=False, general_A=False, out=None,
                         saved_states=None, stream=None):
     """ssm_scan_fwd for callers that may not allocate: no workspace argument, and this wrapper allocates none either
@@ -207,7 +222,7 @@ def ssm_scan_fwd_static(x, delta, A, B, C, D_skip=None, z=None, *, save_states=F
 
 
 def ssm_scan_bwd(x, delta, A, B, C, D_skip, z, dout, saved_states=None, *, general_A=False, workspace=None,
-                 stream=None, outputs=None):
+                 stream=None, outputs=None, extra_flags=0):
     """Gradients of sum(dout * out) w.r.t. x, delta, A, B, C, D_skip, z; see include/ssm_scan.h.
 
     Returns a dict with dx, ddelta, dz (io dtype, (batch, L, D)); dB, dC (io dtype, (batch, L, N)); dA (float32, (D, N));
@@ -215,6 +230,7 @@ def ssm_scan_bwd(x, delta, A, B, C, D_skip, z, dout, saved_states=None, *, gener
     """
     lib = load_library()
     prob = make_problem(x, B, z is not None, D_skip is not None, False, general_A)
+    prob.flags |= int(extra_flags)
     batch, L, D, N = prob.batch, prob.L, prob.D, prob.N
     io = x.dtype
     o = dict(outputs or {})

@@ -8,13 +8,14 @@ namespace ssm {
 
 int fwd_channels_per_block(int N);
 int bwd_channels_per_block(int N);
+size_t bwd_fast_handoff_bytes_per_chain();
 
 static inline size_t align_up(size_t v) { return (v + 255) & ~(size_t)255; }
 
 static ssm_status_t validate_problem(const ssm_problem_t* p) {
   if (p == nullptr) return SSM_ERR_INVALID_ARG;
   if (p->batch < 1 || p->L < 1 || p->D < 1 || p->N < 1) return SSM_ERR_INVALID_ARG;
-  if (p->flags & ~(uint32_t)(SSM_FLAG_HAS_Z | SSM_FLAG_HAS_DSKIP | SSM_FLAG_SAVE_STATES | SSM_FLAG_GENERAL_A))
+  if (p->flags & ~(uint32_t)(SSM_FLAG_HAS_Z | SSM_FLAG_HAS_DSKIP | SSM_FLAG_SAVE_STATES | SSM_FLAG_GENERAL_A | SSM_FLAG_TEST_WITHHOLD))
     return SSM_ERR_INVALID_ARG;
   if (p->io_dtype != SSM_F32 && p->io_dtype != SSM_BF16) return SSM_ERR_UNSUPPORTED;
   if (p->N != 1 && p->N != 2 && p->N != 4 && p->N != 8 && p->N != 16) return SSM_ERR_UNSUPPORTED;
@@ -64,7 +65,7 @@ static FwdWorkspace fwd_layout(const ssm_problem_t& p, const Plan& pl) {
 }
 
 struct BwdWorkspace {
-  size_t dBC_part, dA_part, dD_part, ckpt, seg_local, seg_dsum, mu_in, fwd, total;
+  size_t dBC_part, dA_part, dD_part, ckpt, seg_local, seg_dsum, mu_in, fwd, sched, handoff, total;
 };
 static BwdWorkspace bwd_layout(const ssm_problem_t& p, const Plan& pl) {
   BwdWorkspace w{};
@@ -87,6 +88,9 @@ static BwdWorkspace bwd_layout(const ssm_problem_t& p, const Plan& pl) {
     w.seg_dsum = take(parts * p.D * sizeof(float));
   }
   w.fwd = take(fwd_layout(p, pl).total);
+  const size_t chains = parts * pl.bwd_groups;   // (batch, segment, channel group) chains of the tuned kernel
+  w.sched = take((64 + chains) * sizeof(int));
+  w.handoff = take(chains * bwd_fast_handoff_bytes_per_chain());
   w.total = off;
   return w;
 }
@@ -160,6 +164,20 @@ const char* ssm_status_string(ssm_status_t s) {
     case SSM_ERR_TIMEOUT: return "SSM_ERR_TIMEOUT: a bounded device-side wait gave up";
     default: return "unknown ssm_status_t";
   }
+}
+
+ssm_status_t ssm_scan_check_status(const ssm_problem_t* p, const void* workspace, void* stream) {
+  const ssm_status_t st = validate_problem(p);
+  if (st != SSM_OK) return st;
+  if (workspace == nullptr) return SSM_ERR_WORKSPACE;
+  const BwdWorkspace w = bwd_layout(*p, make_plan(*p));
+  int word = 0;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  if (cudaMemcpyAsync(&word, static_cast<const char*>(workspace) + w.sched + sizeof(int), sizeof(int),
+                      cudaMemcpyDeviceToHost, s) != cudaSuccess)
+    return SSM_ERR_CUDA;
+  if (cudaStreamSynchronize(s) != cudaSuccess) return SSM_ERR_CUDA;
+  return word != 0 ? SSM_ERR_TIMEOUT : SSM_OK;
 }
 
 ssm_status_t ssm_scan_plan(const ssm_problem_t* p, int32_t* n_segments, int32_t* segment_steps,
@@ -288,6 +306,12 @@ ssm_status_t ssm_scan_bwd(const ssm_problem_t* p, const void* x, const void* del
   bp.nck = pl.nck;
   bp.groups = pl.bwd_groups;
   bp.general_A = (p->flags & SSM_FLAG_GENERAL_A) ? 1 : 0;
+  bp.test_withhold = (p->flags & SSM_FLAG_TEST_WITHHOLD) ? 1 : 0;
+  bp.sched = reinterpret_cast<int*>(ws + w.sched);
+  bp.handoff = reinterpret_cast<float4*>(ws + w.handoff);
+  // scheduling words of the tuned kernel (claim counter, abort word, one progress flag per chain) start at zero; the
+  // abort word is also what ssm_scan_check_status reads, whichever kernel runs
+  if (cudaMemsetAsync(ws + w.sched, 0, w.handoff - w.sched, s) != cudaSuccess) return SSM_ERR_CUDA;
 
   if (pl.nseg > 1) {
     bp.seg_local = reinterpret_cast<float*>(ws + w.seg_local);

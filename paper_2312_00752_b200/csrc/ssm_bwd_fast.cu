@@ -9,6 +9,13 @@
 // 8, 16 and 24 in shared memory; then, for the sub-blocks of 8 steps from last to first, it re-runs the 8 steps keeping
 // every h_t in registers and walks them backwards with the adjoint recurrence.
 //
+// Scheduling.  The kernel is persistent: blocks claim work items (channel group, tile) from a global counter in an
+// order in which the tile that a tile depends on (the next tile in time of the same channel group) is always claimed
+// earlier, so whoever holds it is already running; the adjoint mu and the dA / dD accumulators cross from one tile
+// to the next through a small hand-off buffer in L2 and a release/acquire flag per channel group.  This keeps every
+// SM busy to the end whatever the ratio of blocks to SMs is.  Every wait is bounded: after a fixed number of polls a
+// block raises an abort word that all blocks observe, and the host reports SSM_ERR_TIMEOUT.
+//
 // Sums.  The three per-(step, channel) sums over n (readout for dz, sum lam*B for dx and ddelta, sum w*A for
 // ddelta) are exchanged inside the quad in one batch per sub-block; afterwards every lane finalises 4 steps of one
 // channel.  dB and dC are summed over the two channels of a thread in registers, over the 8 quads of a warp through
@@ -31,6 +38,8 @@ constexpr int kBwdFastWarps = 2;
 constexpr int kBwdFastThreads = kBwdFastWarps * 32;
 constexpr int kBwdFastCH = 16 * kBwdFastWarps;
 constexpr float kInvLog2e = 0.6931471805599453f;
+constexpr int kHandoffVec = 5;            // float4 per thread: mu (2), dA (2), dD (1)
+constexpr int kSpinLimit = 1 << 22;       // polls of a dependency flag before giving up (each poll sleeps ~100 ns)
 
 struct BwdFastSmem {
   uint32_t x[2][kBT][kBwdFastCH / 2];   // bf16 pairs; the rows of a finished sub-block are reused for dx
@@ -45,8 +54,19 @@ struct BwdFastSmem {
   float gsp[kBT][kBwdFastCH];           // dout * silu'(z)
   float4 red[kBwdFastWarps][kRB][8][4][2];   // [warp][step][quad][lane in quad][dB quad | dC quad]
   float acc[kBwdFastWarps][kBT][32];    // per-warp sums over its 16 channels: [step][dB 0..15 | dC 0..15]
+  int sched[4];                         // [0] current item, [1] next item, [2] abort
   float4 hsave[kBT / kSB - 1][2][kBwdFastThreads];  // states at steps 8, 16, 24 of the tile, per thread and channel
 };
+
+
+__device__ __forceinline__ int ld_acquire(const int* p) {
+  int v;
+  asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+  return v;
+}
+__device__ __forceinline__ void st_release(int* p, int v) {
+  asm volatile("st.release.gpu.global.s32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
 
 }  // namespace
 
@@ -71,52 +91,49 @@ __global__ void __launch_bounds__(kBwdFastThreads) ssm_bwd_fast_kernel(const Bwd
   const int lane = tid & 31, warp = tid >> 5;
   const int j = lane & 3, quad = lane >> 2;
   const int slot = warp * 8 + quad;      // channel pair within the block
-  const int d_cta = blockIdx.x * CH;
-  const int seg = blockIdx.y;
-  const int b = blockIdx.z;
   const int D = p.D;
-  const int t_begin = seg * p.seg_steps;
-  const int t_end = min(p.L, t_begin + p.seg_steps);
-  const int ntiles = (t_end - t_begin + kBT - 1) / kBT;
-  const int d0 = d_cta + 2 * slot;
-  const bool valid = d0 < D;
   const bool has_z = gz != nullptr;
   // q = 0 is the channel whose sums this lane keeps (channel pq of the pair), q = 1 the one it hands to its neighbour
   const int pq = j & 1, gq = j >> 1;
   const uint32_t selA = pq ? 0x3244u : 0x1044u, selB = pq ? 0x1044u : 0x3244u;
-  auto chan = [&](int q) { return d0 + (q ^ pq); };
 
-  float2 A2[2][2], mu[2][2], dA2[2][2];
-  bool ap = true;
-#pragma unroll
-  for (int q = 0; q < 2; ++q) {
-    float4 a = make_float4(0.f, 0.f, 0.f, 0.f), m = a;
-    if (valid) {
-      a = *reinterpret_cast<const float4*>(p.A + (size_t)chan(q) * 16 + 4 * j);
-      if (p.mu_in != nullptr)
-        m = *reinterpret_cast<const float4*>(p.mu_in + (((size_t)b * p.nseg + seg) * D + chan(q)) * 16 + 4 * j);
-    }
-    const float step = a.y - a.x, tol = 1e-6f * fabsf(a.w);
-    ap = ap && fabsf(a.z - (a.x + 2.f * step)) <= tol && fabsf(a.w - (a.x + 3.f * step)) <= tol;
-    A2[q][0] = make_float2(a.x * kLog2e, a.y * kLog2e);
-    A2[q][1] = make_float2(a.z * kLog2e, a.w * kLog2e);
-    mu[q][0] = make_float2(m.x, m.y);
-    mu[q][1] = make_float2(m.z, m.w);
-    dA2[q][0] = dA2[q][1] = make_float2(0.f, 0.f);
-  }
-  ap = __all_sync(0xffffffffu, ap && !p.general_A);
-  const float Dk = (valid && p.Dskip != nullptr) ? p.Dskip[d0 + pq] : 0.f;
-  float dD_acc = 0.f;
+  // ---- work items: chain = (batch, segment, channel group); item = (order within the chain, chain), order-major
+  const int groups = (D + CH - 1) / CH;
+  const int chains = p.batch * p.nseg * groups;
+  const int tiles_max = p.seg_steps / kBT;
+  const int total_items = chains * tiles_max;
+  int* const sched_counter = p.sched;
+  int* const sched_abort = p.sched + 1;
+  int* const sched_flags = p.sched + 64;
 
-  auto issue_tile = [&](int i) {
-    if (i >= 0) {
-      const int st = i & 1;
-      const int t0 = t_begin + i * kBT;
-      const size_t row0 = (size_t)b * p.L + t0;
+  struct Item {
+    int chain, ord, b, seg, grp, d_cta, t_begin, t_end, ntiles, tile, t0;
+    bool live;   // false: the chain has fewer tiles than tiles_max and this order does not exist
+  };
+  auto decode = [&](int id) {
+    Item it;
+    it.ord = id / chains;
+    it.chain = id - it.ord * chains;
+    it.grp = it.chain % groups;
+    const int bs = it.chain / groups;
+    it.seg = bs % p.nseg;
+    it.b = bs / p.nseg;
+    it.d_cta = it.grp * CH;
+    it.t_begin = it.seg * p.seg_steps;
+    it.t_end = min(p.L, it.t_begin + p.seg_steps);
+    it.ntiles = (it.t_end - it.t_begin + kBT - 1) / kBT;
+    it.live = id < total_items && it.ord < it.ntiles;
+    it.tile = it.ntiles - 1 - it.ord;               // tiles run from last to first
+    it.t0 = it.t_begin + it.tile * kBT;
+    return it;
+  };
+  auto issue_item = [&](const Item& it, int st) {   // inputs of one tile into ring stage st
+    if (it.live) {
+      const size_t row0 = (size_t)it.b * p.L + it.t0;
       for (int c = tid; c < kBT * CHUNKS; c += THREADS) {
         const int tt = c / CHUNKS, cc = c % CHUNKS;
-        const bool ok = (t0 + tt < t_end) && (d_cta + cc * 8 < D);
-        const size_t g = ok ? (row0 + tt) * D + d_cta + cc * 8 : 0;
+        const bool ok = (it.t0 + tt < it.t_end) && (it.d_cta + cc * 8 < D);
+        const size_t g = ok ? (row0 + tt) * D + it.d_cta + cc * 8 : 0;
         cp_async16(&sm.x[st][tt][cc * 4], gx + g, ok);
         cp_async16(&sm.d[st][tt][cc * 4], gd + g, ok);
         cp_async16(&sm.z[st][tt][cc * 4], (has_z ? gz : gx) + g, ok && has_z);
@@ -124,7 +141,7 @@ __global__ void __launch_bounds__(kBwdFastThreads) ssm_bwd_fast_kernel(const Bwd
       }
       for (int c = tid; c < kBT * 2; c += THREADS) {
         const int tt = c >> 1, cc = c & 1;
-        const bool ok = t0 + tt < t_end;
+        const bool ok = it.t0 + tt < it.t_end;
         const size_t g = ok ? (row0 + tt) * 16 + cc * 8 : 0;
         cp_async16(&sm.rawB[st][tt][cc * 4], gB + g, ok);
         cp_async16(&sm.rawC[st][tt][cc * 4], gC + g, ok);
@@ -132,6 +149,13 @@ __global__ void __launch_bounds__(kBwdFastThreads) ssm_bwd_fast_kernel(const Bwd
     }
     cp_async_commit();
   };
+
+  // ---- state of the chain being processed (set per item)
+  float2 A2[2][2], mu[2][2], dA2[2][2];
+  float Dk = 0.f, dD_acc = 0.f;
+  int d0 = 0;
+  bool valid = false;
+  auto chan = [&](int q) { return d0 + (q ^ pq); };
 
   // decays of one step for channel q: general A or arithmetic-progression A (two exponentials)
   auto decays = [&](float dt, int q, auto ap_tag, float2& a01, float2& a23) {
@@ -148,8 +172,7 @@ __global__ void __launch_bounds__(kBwdFastThreads) ssm_bwd_fast_kernel(const Bwd
     }
   };
 
-  auto process_tile = [&](int i, auto ap_tag, const float4 (&ck)[2]) {
-    const int st = i & 1;
+  auto process_tile = [&](int st, auto ap_tag, const float4 (&ck)[2]) {
     // ---- level 1: states at the sub-block boundaries (steps 0, 8, 16, 24 of the tile), parked in shared memory
     {
       float2 h[2][2];
@@ -310,32 +333,96 @@ __global__ void __launch_bounds__(kBwdFastThreads) ssm_bwd_fast_kernel(const Bwd
     }
   };
 
-  // ---- tiles from last to first
-  issue_tile(ntiles - 1);
-  for (int i = ntiles - 1; i >= 0; --i) {
-    const int st = i & 1;
-    const int t0 = t_begin + i * kBT;
-    const size_t row0 = (size_t)b * p.L + t0;
-    float4 ck[2];
-#pragma unroll
-    for (int q = 0; q < 2; ++q)
-      ck[q] = valid ? *reinterpret_cast<const float4*>(p.ckpt + (((size_t)b * p.nck + t0 / kCkptSteps) * D + chan(q)) * 16 + 4 * j)
-                    : make_float4(0.f, 0.f, 0.f, 0.f);
-    cp_async_wait_all();
-    __syncthreads();
-    issue_tile(i - 1);
-    // widen B, C; per-element gate terms ds = dout * silu(z), gsp = dout * silu'(z)
-    for (int c = tid; c < kBT * 8; c += THREADS) {
-      const int tt = c >> 3, w = c & 7;
-      const uint32_t vb = sm.rawB[st][tt][w], vc = sm.rawC[st][tt][w];
-      reinterpret_cast<float2*>(&sm.fB[tt][0])[w] = make_float2(bf16lo(vb), bf16hi(vb));
-      reinterpret_cast<float2*>(&sm.fC[tt][0])[w] = make_float2(bf16lo(vc), bf16hi(vc));
+
+  // ---- persistent loop over claimed items
+  if (tid == 0) {
+    sm.sched[0] = atomicAdd(sched_counter, 1);
+    sm.sched[2] = 0;
+  }
+  __syncthreads();
+  Item cur = decode(sm.sched[0]);
+  int st = 0;
+  issue_item(cur, st);
+  while (cur.chain + cur.ord * chains < total_items) {
+    if (tid == 0) sm.sched[1] = atomicAdd(sched_counter, 1);   // claim ahead: its inputs are prefetched below
+    if (cur.live) {
+      d0 = cur.d_cta + 2 * slot;
+      valid = d0 < D;
     }
-    for (int c = tid; c < kBT * (CH / 2); c += THREADS) {
-      const int tt = c / (CH / 2), w = c % (CH / 2);
-      const uint32_t zw = sm.z[st][tt][w], gw = sm.g[st][tt][w];
-      float2 dsv, gpv;
-      {
+    float4 ck[2] = {make_float4(0.f, 0.f, 0.f, 0.f), make_float4(0.f, 0.f, 0.f, 0.f)};
+    bool ap = !p.general_A;
+    if (cur.live) {
+      // per-chain constants and the checkpoint state of this tile
+#pragma unroll
+      for (int q = 0; q < 2; ++q) {
+        float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (valid) {
+          a = *reinterpret_cast<const float4*>(p.A + (size_t)chan(q) * 16 + 4 * j);
+          ck[q] = *reinterpret_cast<const float4*>(p.ckpt + (((size_t)cur.b * p.nck + cur.t0 / kCkptSteps) * D + chan(q)) * 16 + 4 * j);
+        }
+        const float step = a.y - a.x, tol = 1e-6f * fabsf(a.w);
+        ap = ap && fabsf(a.z - (a.x + 2.f * step)) <= tol && fabsf(a.w - (a.x + 3.f * step)) <= tol;
+        A2[q][0] = make_float2(a.x * kLog2e, a.y * kLog2e);
+        A2[q][1] = make_float2(a.z * kLog2e, a.w * kLog2e);
+      }
+      Dk = (valid && p.Dskip != nullptr) ? p.Dskip[d0 + pq] : 0.f;
+      // carried values: from the segment's inflow for the first tile in order, else from the tile before in order
+      if (cur.ord == 0) {
+#pragma unroll
+        for (int q = 0; q < 2; ++q) {
+          float4 m = make_float4(0.f, 0.f, 0.f, 0.f);
+          if (valid && p.mu_in != nullptr)
+            m = *reinterpret_cast<const float4*>(p.mu_in + (((size_t)cur.b * p.nseg + cur.seg) * D + chan(q)) * 16 + 4 * j);
+          mu[q][0] = make_float2(m.x, m.y);
+          mu[q][1] = make_float2(m.z, m.w);
+          dA2[q][0] = dA2[q][1] = make_float2(0.f, 0.f);
+        }
+        dD_acc = 0.f;
+      } else {
+        if (tid == 0) {
+          int spins = 0;
+          while (ld_acquire(sched_flags + cur.chain) < cur.ord) {
+            __nanosleep(100);
+            if (++spins > (p.test_withhold ? 1000 : kSpinLimit) || ld_acquire(sched_abort) != 0) {
+              atomicExch(sched_abort, 1);
+              sm.sched[2] = 1;
+              break;
+            }
+          }
+        }
+      }
+    }
+    ap = __all_sync(0xffffffffu, ap);
+    cp_async_wait_all();
+    __syncthreads();                       // inputs of this tile landed; sched[1], sched[2] and the dependency are visible
+    if (sm.sched[2] != 0) {                // a bounded wait gave up somewhere: every block leaves
+      cp_async_wait_all();
+      return;
+    }
+    const Item nxt = decode(sm.sched[1]);
+    issue_item(nxt, st ^ 1);
+    if (cur.live) {
+      if (cur.ord > 0) {
+        const float4* hb = p.handoff + ((size_t)cur.chain * THREADS + tid) * kHandoffVec;
+        const float4 m0 = __ldcg(hb), m1 = __ldcg(hb + 1), a0 = __ldcg(hb + 2), a1 = __ldcg(hb + 3), dd = __ldcg(hb + 4);
+        mu[0][0] = make_float2(m0.x, m0.y); mu[0][1] = make_float2(m0.z, m0.w);
+        mu[1][0] = make_float2(m1.x, m1.y); mu[1][1] = make_float2(m1.z, m1.w);
+        dA2[0][0] = make_float2(a0.x, a0.y); dA2[0][1] = make_float2(a0.z, a0.w);
+        dA2[1][0] = make_float2(a1.x, a1.y); dA2[1][1] = make_float2(a1.z, a1.w);
+        dD_acc = dd.x;
+      }
+      const size_t row0 = (size_t)cur.b * p.L + cur.t0;
+      // widen B, C; per-element gate terms ds = dout * silu(z), gsp = dout * silu'(z)
+      for (int c = tid; c < kBT * 8; c += THREADS) {
+        const int tt = c >> 3, w = c & 7;
+        const uint32_t vb = sm.rawB[st][tt][w], vc = sm.rawC[st][tt][w];
+        reinterpret_cast<float2*>(&sm.fB[tt][0])[w] = make_float2(bf16lo(vb), bf16hi(vb));
+        reinterpret_cast<float2*>(&sm.fC[tt][0])[w] = make_float2(bf16lo(vc), bf16hi(vc));
+      }
+      for (int c = tid; c < kBT * (CH / 2); c += THREADS) {
+        const int tt = c / (CH / 2), w = c % (CH / 2);
+        const uint32_t zw = sm.z[st][tt][w], gw = sm.g[st][tt][w];
+        float2 dsv, gpv;
         const float g0 = bf16lo(gw), g1 = bf16hi(gw);
         if (has_z) {
           const float z0 = bf16lo(zw), z1 = bf16hi(zw);
@@ -346,67 +433,94 @@ __global__ void __launch_bounds__(kBwdFastThreads) ssm_bwd_fast_kernel(const Bwd
           dsv = make_float2(g0, g1);
           gpv = make_float2(0.f, 0.f);
         }
+        *reinterpret_cast<float2*>(&sm.ds[tt][2 * w]) = dsv;
+        *reinterpret_cast<float2*>(&sm.gsp[tt][2 * w]) = gpv;
       }
-      *reinterpret_cast<float2*>(&sm.ds[tt][2 * w]) = dsv;
-      *reinterpret_cast<float2*>(&sm.gsp[tt][2 * w]) = gpv;
-    }
-    __syncthreads();
-    if (ap) process_tile(i, std::true_type{}, ck);
-    else process_tile(i, std::false_type{}, ck);
-    __syncthreads();
-    // results of the tile: 16-byte stores of dx, ddelta, dz; block partial sums of dB, dC
-    for (int c = tid; c < kBT * CHUNKS; c += THREADS) {
-      const int tt = c / CHUNKS, cc = c % CHUNKS;
-      if (t0 + tt < t_end && d_cta + cc * 8 < D) {
-        const size_t g = (row0 + tt) * D + d_cta + cc * 8;
-        *reinterpret_cast<uint4*>(gdx + g) = *reinterpret_cast<const uint4*>(&sm.x[st][tt][cc * 4]);
-        *reinterpret_cast<uint4*>(gdd + g) = *reinterpret_cast<const uint4*>(&sm.d[st][tt][cc * 4]);
-        if (gdz != nullptr) *reinterpret_cast<uint4*>(gdz + g) = *reinterpret_cast<const uint4*>(&sm.z[st][tt][cc * 4]);
-      }
-    }
-    const size_t bln = (size_t)p.batch * p.L * 16;
-    for (int c = tid; c < kBT * 8; c += THREADS) {  // float4 granules: [step][dB 0..15 | dC 0..15]
-      const int tt = c >> 3, f = c & 7;
-      if (t0 + tt < t_end) {
-        float4 v = *reinterpret_cast<const float4*>(&sm.acc[0][tt][4 * f]);
-#pragma unroll
-        for (int w = 1; w < kBwdFastWarps; ++w) {
-          const float4 o = *reinterpret_cast<const float4*>(&sm.acc[w][tt][4 * f]);
-          v.x += o.x; v.y += o.y; v.z += o.z; v.w += o.w;
+      __syncthreads();
+      if (ap) process_tile(st, std::true_type{}, ck);
+      else process_tile(st, std::false_type{}, ck);
+      __syncthreads();
+      // results of the tile: 16-byte stores of dx, ddelta, dz; block partial sums of dB, dC
+      for (int c = tid; c < kBT * CHUNKS; c += THREADS) {
+        const int tt = c / CHUNKS, cc = c % CHUNKS;
+        if (cur.t0 + tt < cur.t_end && cur.d_cta + cc * 8 < D) {
+          const size_t g = (row0 + tt) * D + cur.d_cta + cc * 8;
+          *reinterpret_cast<uint4*>(gdx + g) = *reinterpret_cast<const uint4*>(&sm.x[st][tt][cc * 4]);
+          *reinterpret_cast<uint4*>(gdd + g) = *reinterpret_cast<const uint4*>(&sm.d[st][tt][cc * 4]);
+          if (gdz != nullptr) *reinterpret_cast<uint4*>(gdz + g) = *reinterpret_cast<const uint4*>(&sm.z[st][tt][cc * 4]);
         }
-        const int which = f >> 2;
-        *reinterpret_cast<float4*>(p.dBC_part + ((size_t)blockIdx.x * 2 + which) * bln + (row0 + tt) * 16 + 4 * (f & 3)) = v;
+      }
+      const size_t bln = (size_t)p.batch * p.L * 16;
+      for (int c = tid; c < kBT * 8; c += THREADS) {  // float4 granules: [step][dB 0..15 | dC 0..15]
+        const int tt = c >> 3, f = c & 7;
+        if (cur.t0 + tt < cur.t_end) {
+          float4 v = *reinterpret_cast<const float4*>(&sm.acc[0][tt][4 * f]);
+#pragma unroll
+          for (int w = 1; w < kBwdFastWarps; ++w) {
+            const float4 o = *reinterpret_cast<const float4*>(&sm.acc[w][tt][4 * f]);
+            v.x += o.x; v.y += o.y; v.z += o.z; v.w += o.w;
+          }
+          const int which = f >> 2;
+          *reinterpret_cast<float4*>(p.dBC_part + ((size_t)cur.grp * 2 + which) * bln + (row0 + tt) * 16 + 4 * (f & 3)) = v;
+        }
+      }
+      if (cur.ord + 1 < cur.ntiles) {
+        // hand the carried values to whoever runs the next tile of this chain
+        float4* hb = p.handoff + ((size_t)cur.chain * THREADS + tid) * kHandoffVec;
+        __stcg(hb, make_float4(mu[0][0].x, mu[0][0].y, mu[0][1].x, mu[0][1].y));
+        __stcg(hb + 1, make_float4(mu[1][0].x, mu[1][0].y, mu[1][1].x, mu[1][1].y));
+        __stcg(hb + 2, make_float4(dA2[0][0].x, dA2[0][0].y, dA2[0][1].x, dA2[0][1].y));
+        __stcg(hb + 3, make_float4(dA2[1][0].x, dA2[1][0].y, dA2[1][1].x, dA2[1][1].y));
+        __stcg(hb + 4, make_float4(dD_acc, 0.f, 0.f, 0.f));
+        __threadfence();
+        __syncthreads();
+        if (tid == 0 && !p.test_withhold) st_release(sched_flags + cur.chain, cur.ord + 1);
+      } else {
+        // first tile in time: the chain is complete
+        if (valid) {
+          const size_t part = (size_t)cur.b * p.nseg + cur.seg;
+#pragma unroll
+          for (int q = 0; q < 2; ++q)
+            *reinterpret_cast<float4*>(p.dA_part + (part * D + chan(q)) * 16 + 4 * j) =
+                make_float4(dA2[q][0].x, dA2[q][0].y, dA2[q][1].x, dA2[q][1].y);
+        }
+        // dD: lanes j and j^2 accumulated disjoint steps of the same channel
+        const float dsum2 = dD_acc + __shfl_xor_sync(0xffffffffu, dD_acc, 2);
+        if (valid && j < 2) p.dD_part[((size_t)cur.b * p.nseg + cur.seg) * D + d0 + pq] = dsum2;
       }
     }
+    cur = nxt;
+    st ^= 1;
   }
   cp_async_wait_all();
-
-  if (valid) {
-    const size_t part = (size_t)b * p.nseg + seg;
-#pragma unroll
-    for (int q = 0; q < 2; ++q)
-      *reinterpret_cast<float4*>(p.dA_part + (part * D + chan(q)) * 16 + 4 * j) =
-          make_float4(dA2[q][0].x, dA2[q][0].y, dA2[q][1].x, dA2[q][1].y);
-  }
-  // dD: lanes j and j^2 accumulated disjoint steps of the same channel
-  dD_acc += __shfl_xor_sync(0xffffffffu, dD_acc, 2);
-  if (valid && j < 2) p.dD_part[((size_t)b * p.nseg + seg) * D + d0 + pq] = dD_acc;
 }
 
 bool bwd_fast_applicable(const ssm_problem_t& prob, const BwdParams& p) {
   auto al16 = [](const void* q) { return q == nullptr || (reinterpret_cast<uintptr_t>(q) & 15) == 0; };
-  return prob.io_dtype == SSM_BF16 && prob.N == 16 && prob.D % 8 == 0 && al16(p.x) && al16(p.delta) && al16(p.z) &&
-         al16(p.B) && al16(p.C) && al16(p.dout) && al16(p.dx) && al16(p.ddelta) && al16(p.dz) && al16(p.A) &&
-         al16(p.ckpt) && al16(p.mu_in) && al16(p.dBC_part) && al16(p.dA_part);
+  return prob.io_dtype == SSM_BF16 && prob.N == 16 && prob.D % 8 == 0 && p.seg_steps % kBT == 0 && al16(p.x) &&
+         al16(p.delta) && al16(p.z) && al16(p.B) && al16(p.C) && al16(p.dout) && al16(p.dx) && al16(p.ddelta) &&
+         al16(p.dz) && al16(p.A) && al16(p.ckpt) && al16(p.mu_in) && al16(p.dBC_part) && al16(p.dA_part) &&
+         p.sched != nullptr && p.handoff != nullptr;
 }
 
 int bwd_fast_channels_per_block() { return kBwdFastCH; }
+size_t bwd_fast_handoff_bytes_per_chain() { return sizeof(float4) * kHandoffVec * kBwdFastThreads; }
 
 cudaError_t launch_bwd_fast(const Plan& plan, const BwdParams& p, cudaStream_t s) {
   constexpr size_t smem = sizeof(BwdFastSmem);
   cudaError_t e = cudaFuncSetAttribute(ssm_bwd_fast_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
-  dim3 grid((p.D + kBwdFastCH - 1) / kBwdFastCH, plan.nseg, p.batch);
+  int dev = 0, sms = 0, per_sm = 0;
+  if ((e = cudaGetDevice(&dev)) != cudaSuccess) return e;
+  if ((e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
+  if ((e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, ssm_bwd_fast_kernel, kBwdFastThreads, smem)) != cudaSuccess)
+    return e;
+  const int groups = (p.D + kBwdFastCH - 1) / kBwdFastCH;
+  const long long chains = (long long)p.batch * plan.nseg * groups;
+  const long long items = chains * (plan.seg_steps / kBT);
+  const long long resident = (long long)sms * (per_sm > 0 ? per_sm : 1);
+  const unsigned grid = (unsigned)(items < resident ? items : resident);
+  // the claim counter, the abort word and the flag of every chain were zeroed by the caller (ssm_scan_bwd)
   ssm_bwd_fast_kernel<<<grid, kBwdFastThreads, smem, s>>>(p);
   return cudaGetLastError();
 }

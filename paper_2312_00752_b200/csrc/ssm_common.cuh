@@ -77,6 +77,9 @@ struct BwdParams {
   float* dD_part;         // [batch*nseg][D]
   int batch, L, D, nseg, seg_steps, nck, groups;
   int general_A;          // 1: never take the arithmetic-progression fast path
+  int test_withhold;      // test hook: never publish hand-off flags, poll only 1000 times
+  int* sched;             // tuned kernel: [0] claim counter, [1] abort word, [64 + chain] progress flag per chain
+  float4* handoff;        // tuned kernel: carried values between consecutive tiles of a chain
 };
 
 struct ReduceParams {

@@ -47,6 +47,10 @@ def gpu_fwd_bwd(dev: dict, use_saved=True, general_A=False):
     res = {"out": to_host(out)}
     if dev.get("dout") is not None:
         g = K.ssm_scan_bwd(*args, dev["dout"], saved, general_A=general_A)
+        ws = K.last_bwd_workspace(dev["x"].device)
+        if ws is not None:
+            K.check_status(K.make_problem(dev["x"], dev["B"], dev.get("z") is not None, dev.get("D_skip") is not None,
+                                          False, general_A), ws)
         for k, v in g.items():
             res[k] = None if v is None else to_host(v)
     return res

@@ -116,3 +116,22 @@ def test_outputs_outside_are_untouched():
     torch.cuda.synchronize()
     for k, b in bufs.items():
         assert torch.all(b[:pad] == 7.0) and torch.all(b[-pad:] == 7.0), k
+
+
+def test_bounded_wait_reports_timeout_and_the_context_survives():
+    """Failure detection without a GPU fault: with the test hook the tuned backward kernel never publishes its hand-off
+    flags, so every dependent tile polls its (short) limit, gives up and raises the abort word; the host reads
+    SSM_ERR_TIMEOUT, and the next ordinary call on the same context is correct."""
+    import torch
+    from paper_2312_00752_b200 import binding as K
+    cfg, inp = _case(2, 256, 64, 16, "bf16")
+    dev = U.to_device(inp, "bf16")
+    args = (dev["x"], dev["delta"], dev["A"], dev["B"], dev["C"], dev["D_skip"], dev["z"])
+    K.ssm_scan_bwd(*args, dev["dout"], None, extra_flags=K.SSM_FLAG_TEST_WITHHOLD)
+    ws = K.last_bwd_workspace(dev["x"].device)
+    prob = K.make_problem(dev["x"], dev["B"], True, True)
+    with pytest.raises(K.SsmScanError, match="TIMEOUT"):
+        K.check_status(prob, ws)
+    torch.cuda.synchronize()
+    got = U.gpu_fwd_bwd(dev)                      # checks the status itself and must be clean again
+    U.assert_parity(got, U.oracle_fwd_bwd(inp), "bf16", "after a timed-out call")
