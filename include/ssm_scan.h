@@ -107,6 +107,30 @@ SSM_API ssm_status_t ssm_scan_fwd(const ssm_problem_t* p, const void* x, const v
                           void* workspace, size_t workspace_bytes, void* stream /* cudaStream_t */);
 
 /*
+ * Forward with a carried-in and a carried-out state, for processing a long sequence in pieces or for handing a prompt
+ * over to token-by-token generation (Appendix D: with the intermediate scan states one can continue the scan with the
+ * next chunk; Section 2: the recurrent mode of Eq. 2).  Same as ssm_scan_fwd, plus
+ *   h0        in, float32 [batch][D][N]: the state before the first step (NULL: zero)
+ *   h_last    out, float32 [batch][D][N]: the state after the last step (NULL: not wanted)
+ * Checkpoint states written with SSM_FLAG_SAVE_STATES include the effect of h0, so ssm_scan_bwd given those saved
+ * states returns the gradients of this call's inputs; the gradient with respect to h0 itself is not produced, and
+ * ssm_scan_bwd without saved states assumes h0 = 0.
+ */
+SSM_API ssm_status_t ssm_scan_fwd_state(const ssm_problem_t* p, const void* x, const void* delta, const float* A,
+                                        const void* B, const void* C, const float* D_skip, const void* z,
+                                        const float* h0, void* out, float* h_last, void* saved_states,
+                                        void* workspace, size_t workspace_bytes, void* stream /* cudaStream_t */);
+
+/*
+ * One recurrent step (Eq. 2a/2b evaluated for a single t, the mode used for autoregressive inference): p->L must be
+ * 1; x, delta, z, out are [batch][D], B, C are [batch][N] (io_dtype), A [D][N], D_skip [D]; the float32 state
+ * h [batch][D][N] is read and overwritten with the state after the step.  Needs no workspace.
+ */
+SSM_API ssm_status_t ssm_step(const ssm_problem_t* p, const void* x, const void* delta, const float* A, const void* B,
+                              const void* C, const float* D_skip, const void* z, float* h, void* out,
+                              void* stream /* cudaStream_t */);
+
+/*
  * Backward: gradients of loss = sum(dout * out) with respect to every input (the adjoint of the four lines at
  * the top; the states are recomputed on chip from checkpoint states, Section 3.3 "recomputation").
  *   x, delta, A, B, C, D_skip, z   the forward inputs, same rules as above

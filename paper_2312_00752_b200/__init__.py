@@ -4,11 +4,11 @@
 seeded input generator in `synth`) does not need torch or the compiled library.
 """
 
-__all__ = ["ssm_scan_fwd", "ssm_scan_bwd", "ssm_scan_fwd_static", "binding", "synth", "build"]
+__all__ = ["ssm_scan_fwd", "ssm_scan_bwd", "ssm_scan_fwd_static", "ssm_step", "binding", "synth", "build"]
 
 
 def __getattr__(name):
-    if name in ("ssm_scan_fwd", "ssm_scan_bwd", "ssm_scan_fwd_static"):
+    if name in ("ssm_scan_fwd", "ssm_scan_bwd", "ssm_scan_fwd_static", "ssm_step"):
         from . import binding
         return getattr(binding, name)
     if name in ("binding", "synth", "build"):

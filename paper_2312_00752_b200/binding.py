@@ -20,7 +20,7 @@ SSM_FLAG_HAS_Z, SSM_FLAG_HAS_DSKIP, SSM_FLAG_SAVE_STATES, SSM_FLAG_GENERAL_A, SS
 EXPORTED_SYMBOLS = (
     "ssm_scan_fwd_workspace_bytes", "ssm_scan_bwd_workspace_bytes", "ssm_scan_saved_state_bytes",
     "ssm_scan_checkpoint_steps", "ssm_scan_fwd", "ssm_scan_bwd", "ssm_status_string", "ssm_scan_plan",
-    "ssm_scan_fwd_static", "ssm_scan_check_status",
+    "ssm_scan_fwd_static", "ssm_scan_check_status", "ssm_scan_fwd_state", "ssm_step",
 )
 SSM_STATIC_SCRATCH_BYTES = 4 << 20
 
@@ -67,6 +67,10 @@ def load_library() -> ctypes.CDLL:
     lib.ssm_scan_fwd.argtypes = [P] + [vp] * 9 + [vp, sz, vp]
     lib.ssm_scan_bwd.restype = ctypes.c_int
     lib.ssm_scan_bwd.argtypes = [P] + [vp] * 16 + [vp, sz, vp]
+    lib.ssm_scan_fwd_state.restype = ctypes.c_int
+    lib.ssm_scan_fwd_state.argtypes = [P] + [vp] * 11 + [vp, sz, vp]
+    lib.ssm_step.restype = ctypes.c_int
+    lib.ssm_step.argtypes = [P] + [vp] * 10
     lib.ssm_scan_check_status.restype = ctypes.c_int
     lib.ssm_scan_check_status.argtypes = [P, vp, vp]
     lib.ssm_scan_fwd_static.restype = ctypes.c_int
@@ -153,12 +157,14 @@ def saved_state_bytes(problem: ssm_problem_t) -> int:
 
 
 def ssm_scan_fwd(x, delta, A, B, C, D_skip=None, z=None, *, save_states=False, general_A=False, out=None,
-                 saved_states=None, workspace=None, stream=None):
+                 saved_states=None, workspace=None, stream=None, h0=None, h_last=None):
     """out = selective_scan(x, delta, A, B, C) (+ D_skip * x) (* silu(z)); see include/ssm_scan.h.
 
     x, delta, z: (batch, L, D) io dtype; B, C: (batch, L, N) io dtype; A: (D, N) float32; D_skip: (D) float32.
     Returns `out`, or `(out, saved_states)` with save_states=True.  Enqueues on `stream` (default: torch's current
-    stream) and does not synchronise.
+    stream) and does not synchronise.  `h0` (batch, D, N) float32 is the state before the first step (default zero);
+    if a float32 tensor `h_last` (batch, D, N) is passed it receives the state after the last step
+    (ssm_scan_fwd_state).
     """
     lib = load_library()
     prob = make_problem(x, B, z is not None, D_skip is not None, save_states, general_A)
@@ -171,16 +177,39 @@ def ssm_scan_fwd(x, delta, A, B, C, D_skip=None, z=None, *, save_states=False, g
     stream_ptr = (stream if stream is not None else torch.cuda.current_stream(x.device)).cuda_stream
     need = fwd_workspace_bytes(prob)
     ws = workspace if workspace is not None else _workspace(need, x.device, stream_ptr)
-    code = lib.ssm_scan_fwd(
+    code = lib.ssm_scan_fwd_state(
         ctypes.byref(prob), _dev_ptr(x, "x", (batch, L, D), io), _dev_ptr(delta, "delta", (batch, L, D), io),
         _dev_ptr(A, "A", (D, N), torch.float32), _dev_ptr(B, "B", (batch, L, N), io),
         _dev_ptr(C, "C", (batch, L, N), io), _dev_ptr(D_skip, "D_skip", (D,), torch.float32),
-        _dev_ptr(z, "z", (batch, L, D), io), _dev_ptr(out, "out", (batch, L, D), io),
+        _dev_ptr(z, "z", (batch, L, D), io), _dev_ptr(h0, "h0", (batch, D, N), torch.float32),
+        _dev_ptr(out, "out", (batch, L, D), io), _dev_ptr(h_last, "h_last", (batch, D, N), torch.float32),
         _dev_ptr(saved_states if save_states else None, "saved_states"),
         _dev_ptr(ws, "workspace"), ctypes.c_size_t(0 if ws is None else ws.numel() * ws.element_size()),
         ctypes.c_void_p(stream_ptr))
-    _check(code, "ssm_scan_fwd")
+    _check(code, "ssm_scan_fwd_state")
     return (out, saved_states) if save_states else out
+
+
+def ssm_step(x, delta, A, B, C, D_skip, z, h, *, out=None, stream=None):
+    """One recurrent step: x, delta, z (batch, D), B, C (batch, N) io dtype; h (batch, D, N) float32 is updated in
+    place.  Returns out (batch, D)."""
+    lib = load_library()
+    batch, D = x.shape
+    N = B.shape[-1]
+    prob = ssm_problem_t(batch, 1, D, N, _io_dtype(x),
+                         (SSM_FLAG_HAS_Z if z is not None else 0) | (SSM_FLAG_HAS_DSKIP if D_skip is not None else 0))
+    io = x.dtype
+    if out is None:
+        out = torch.empty_like(x)
+    stream_ptr = (stream if stream is not None else torch.cuda.current_stream(x.device)).cuda_stream
+    code = lib.ssm_step(
+        ctypes.byref(prob), _dev_ptr(x, "x", (batch, D), io), _dev_ptr(delta, "delta", (batch, D), io),
+        _dev_ptr(A, "A", (D, N), torch.float32), _dev_ptr(B, "B", (batch, N), io), _dev_ptr(C, "C", (batch, N), io),
+        _dev_ptr(D_skip, "D_skip", (D,), torch.float32), _dev_ptr(z, "z", (batch, D), io),
+        _dev_ptr(h, "h", (batch, D, N), torch.float32), _dev_ptr(out, "out", (batch, D), io),
+        ctypes.c_void_p(stream_ptr))
+    _check(code, "ssm_step")
+    return out
 
 
 def check_status(problem: ssm_problem_t, workspace: torch.Tensor, stream=None) -> None:

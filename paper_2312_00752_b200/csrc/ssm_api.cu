@@ -105,20 +105,22 @@ static ssm_status_t check_ws(const void* ws, size_t have, size_t need) {
 
 // Runs the passes that establish the state at the start of every segment (nothing to do without a time split).
 static cudaError_t run_segment_starts(const ssm_problem_t& prob, const Plan& pl, FwdParams fp, char* ws,
-                                      const float** h_start, cudaStream_t s) {
-  *h_start = nullptr;
+                                      const float* h0, const float** h_start, cudaStream_t s) {
+  *h_start = h0;  // one segment: [batch][1][D][N] is the layout of the caller's initial state
   if (pl.nseg == 1) return cudaSuccess;
   const FwdWorkspace w = fwd_layout(prob, pl);
   fp.seg_end = reinterpret_cast<float*>(ws + w.seg_end);
   fp.seg_dsum = reinterpret_cast<float*>(ws + w.seg_dsum);
   fp.h_start = nullptr;
   fp.ckpt = nullptr;
+  fp.h_last = nullptr;
   cudaError_t e = launch_fwd(prob, pl, fp, kFwdSummary, s);
   if (e != cudaSuccess) return e;
   CarryParams cp{};
   cp.local = fp.seg_end;
   cp.dsum = fp.seg_dsum;
   cp.A = fp.A;
+  cp.init = h0;
   cp.carried = reinterpret_cast<float*>(ws + w.h_start);
   cp.batch = prob.batch;
   cp.nseg = pl.nseg;
@@ -192,9 +194,10 @@ ssm_status_t ssm_scan_plan(const ssm_problem_t* p, int32_t* n_segments, int32_t*
   return SSM_OK;
 }
 
-ssm_status_t ssm_scan_fwd(const ssm_problem_t* p, const void* x, const void* delta, const float* A, const void* B,
-                          const void* C, const float* D_skip, const void* z, void* out, void* saved_states,
-                          void* workspace, size_t workspace_bytes, void* stream) {
+ssm_status_t ssm_scan_fwd_state(const ssm_problem_t* p, const void* x, const void* delta, const float* A,
+                                const void* B, const void* C, const float* D_skip, const void* z, const float* h0,
+                                void* out, float* h_last, void* saved_states, void* workspace, size_t workspace_bytes,
+                                void* stream) {
   ssm_status_t st = validate_problem(p);
   if (st != SSM_OK) return st;
   const bool has_z = p->flags & SSM_FLAG_HAS_Z, has_d = p->flags & SSM_FLAG_HAS_DSKIP;
@@ -204,7 +207,7 @@ ssm_status_t ssm_scan_fwd(const ssm_problem_t* p, const void* x, const void* del
   const size_t esz = p->io_dtype == SSM_BF16 ? 2 : 4;
   for (const void* q : {x, delta, B, C, z, (const void*)out})
     if (q && !aligned_to(q, esz)) return SSM_ERR_INVALID_ARG;
-  for (const void* q : {(const void*)A, (const void*)D_skip, (const void*)saved_states})
+  for (const void* q : {(const void*)A, (const void*)D_skip, (const void*)saved_states, (const void*)h0, (const void*)h_last})
     if (q && !aligned_to(q, 4)) return SSM_ERR_INVALID_ARG;
   const Plan pl = make_plan(*p);
   st = check_ws(workspace, workspace_bytes, fwd_layout(*p, pl).total);
@@ -228,10 +231,48 @@ ssm_status_t ssm_scan_fwd(const ssm_problem_t* p, const void* x, const void* del
   fp.nck = pl.nck;
   fp.general_A = (p->flags & SSM_FLAG_GENERAL_A) ? 1 : 0;
   const float* h_start = nullptr;
-  if (run_segment_starts(*p, pl, fp, static_cast<char*>(workspace), &h_start, s) != cudaSuccess) return SSM_ERR_CUDA;
+  if (run_segment_starts(*p, pl, fp, static_cast<char*>(workspace), h0, &h_start, s) != cudaSuccess) return SSM_ERR_CUDA;
   fp.h_start = h_start;
+  fp.h_last = h_last;
   fp.ckpt = save ? static_cast<float*>(saved_states) : nullptr;
   if (launch_fwd(*p, pl, fp, kFwdFull, s) != cudaSuccess) return SSM_ERR_CUDA;
+  return SSM_OK;
+}
+
+ssm_status_t ssm_scan_fwd(const ssm_problem_t* p, const void* x, const void* delta, const float* A, const void* B,
+                          const void* C, const float* D_skip, const void* z, void* out, void* saved_states,
+                          void* workspace, size_t workspace_bytes, void* stream) {
+  return ssm_scan_fwd_state(p, x, delta, A, B, C, D_skip, z, nullptr, out, nullptr, saved_states, workspace,
+                            workspace_bytes, stream);
+}
+
+ssm_status_t ssm_step(const ssm_problem_t* p, const void* x, const void* delta, const float* A, const void* B,
+                      const void* C, const float* D_skip, const void* z, float* h, void* out, void* stream) {
+  ssm_status_t st = validate_problem(p);
+  if (st != SSM_OK) return st;
+  if (p->L != 1) return SSM_ERR_INVALID_ARG;
+  const bool has_z = p->flags & SSM_FLAG_HAS_Z, has_d = p->flags & SSM_FLAG_HAS_DSKIP;
+  if (!x || !delta || !A || !B || !C || !h || !out) return SSM_ERR_INVALID_ARG;
+  if ((has_z && !z) || (has_d && !D_skip)) return SSM_ERR_INVALID_ARG;
+  const size_t esz = p->io_dtype == SSM_BF16 ? 2 : 4;
+  for (const void* q : {x, delta, B, C, z, (const void*)out})
+    if (q && !aligned_to(q, esz)) return SSM_ERR_INVALID_ARG;
+  for (const void* q : {(const void*)A, (const void*)D_skip, (const void*)h})
+    if (q && !aligned_to(q, 4)) return SSM_ERR_INVALID_ARG;
+  StepParams sp{};
+  sp.x = x;
+  sp.delta = delta;
+  sp.z = has_z ? z : nullptr;
+  sp.B = B;
+  sp.C = C;
+  sp.A = A;
+  sp.Dskip = has_d ? D_skip : nullptr;
+  sp.h = h;
+  sp.out = out;
+  sp.batch = p->batch;
+  sp.D = p->D;
+  sp.N = p->N;
+  if (launch_step(*p, sp, static_cast<cudaStream_t>(stream)) != cudaSuccess) return SSM_ERR_CUDA;
   return SSM_OK;
 }
 
@@ -275,7 +316,7 @@ ssm_status_t ssm_scan_bwd(const ssm_problem_t* p, const void* x, const void* del
     fp.nck = pl.nck;
     fp.general_A = (p->flags & SSM_FLAG_GENERAL_A) ? 1 : 0;
     const float* h_start = nullptr;
-    if (run_segment_starts(*p, pl, fp, ws + w.fwd, &h_start, s) != cudaSuccess) return SSM_ERR_CUDA;
+    if (run_segment_starts(*p, pl, fp, ws + w.fwd, nullptr, &h_start, s) != cudaSuccess) return SSM_ERR_CUDA;
     fp.h_start = h_start;
     fp.ckpt = reinterpret_cast<float*>(ws + w.ckpt);
     if (launch_fwd(*p, pl, fp, kFwdCkptOnly, s) != cudaSuccess) return SSM_ERR_CUDA;

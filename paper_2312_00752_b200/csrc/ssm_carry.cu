@@ -3,7 +3,7 @@
 //
 // A segment g that starts from a zero state ends in a local state e_g, and multiplies whatever state it was given by
 // P_g = prod_t a_t = exp(A_n * sum_{t in g} delta_t).  The true state before segment g+1 is therefore
-//     H_{g+1} = P_g * H_g + e_g,   H_0 = 0,
+//     H_{g+1} = P_g * H_g + e_g,   H_0 = the caller's initial state (zero if none),
 // i.e. an exclusive scan over segments of the pairs (P_g, e_g) under the operator
 // (a, b) o (a', b') = (a a', a' b + b').  The adjoint that flows backwards through the segments obeys the same law
 // in reversed order, with the same P_g.
@@ -42,10 +42,11 @@ __global__ void __launch_bounds__(kCarryCols* kCarryRanges) ssm_carry_kernel(con
   }
   s_agg[r][threadIdx.x] = agg;
   __syncthreads();
-  AffinePair pre{1.f, 0.f};  // everything before this thread's range
+  // everything before this thread's range, starting from what flows into the first segment
+  AffinePair pre{1.f, (valid && p.init != nullptr) ? p.init[(size_t)b * DN + col] : 0.f};
   for (int rr = 0; rr < r; ++rr) pre = combine(pre, s_agg[rr][threadIdx.x]);
   if (valid) {
-    float carry = pre.b;  // exclusive scan started from a zero state
+    float carry = pre.b;  // exclusive scan
     for (int i = i0; i < i1; ++i) {
       const size_t sg = (size_t)b * p.nseg + seg_of(i);
       p.carried[sg * DN + col] = carry;

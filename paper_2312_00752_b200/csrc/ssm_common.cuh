@@ -42,6 +42,7 @@ struct FwdParams {
   float* ckpt;           // [batch][nck][D][N] checkpoint states to write; null: none
   float* seg_end;        // SUMMARY mode: [batch][nseg][D][N] end state of each segment started from zero
   float* seg_dsum;       // SUMMARY mode: [batch][nseg][D] sum of delta over the segment
+  float* h_last;         // FULL mode: [batch][D][N] state after the last step; null: not wanted
   int batch, L, D, nseg, seg_steps, nck;
   int general_A;       // 1: never take the arithmetic-progression fast path
 };
@@ -50,6 +51,7 @@ struct CarryParams {
   const float* local;   // [batch][nseg][D][N]: per-segment result computed with zero inflow (end state e, or l)
   const float* dsum;    // [batch][nseg][D]: sum of delta over the segment
   const float* A;       // [D][N]
+  const float* init;    // [batch][D][N]: what flows into the first segment in scan order; null: zero
   float* carried;       // [batch][nseg][D][N]: inflow of each segment (forward: state before its first step;
                         //                      reverse: adjoint flowing in from the following segment)
   int batch, nseg, D, N;
@@ -98,6 +100,20 @@ cudaError_t launch_fwd(const ssm_problem_t& prob, const Plan& plan, const FwdPar
 cudaError_t launch_carry(const CarryParams& p, cudaStream_t s);
 cudaError_t launch_bwd(const ssm_problem_t& prob, const Plan& plan, const BwdParams& p, int mode, cudaStream_t s);
 cudaError_t launch_bwd_reduce(const ssm_problem_t& prob, const ReduceParams& p, cudaStream_t s);
+
+struct StepParams {
+  const void* x;        // [batch][D]
+  const void* delta;    // [batch][D]
+  const void* z;        // [batch][D] or null
+  const void* B;        // [batch][N]
+  const void* C;        // [batch][N]
+  const float* A;       // [D][N]
+  const float* Dskip;   // [D] or null
+  float* h;             // [batch][D][N], updated in place
+  void* out;            // [batch][D]
+  int batch, D, N;
+};
+cudaError_t launch_step(const ssm_problem_t& prob, const StepParams& p, cudaStream_t s);
 
 enum FwdMode { kFwdFull = 0, kFwdSummary = 1, kFwdCkptOnly = 2 };
 enum BwdMode { kBwdFull = 0, kBwdLocal = 1 };

@@ -174,6 +174,16 @@ __global__ void __launch_bounds__(fwd_threads(N)) ssm_fwd_kernel(const FwdParams
     }
   }
 
+  if (MODE == kFwdFull && p.h_last != nullptr && seg == p.nseg - 1) {
+#pragma unroll
+    for (int q = 0; q < CPT; ++q) {
+      const int d = d_thr + q;
+      if (d < D) {
+#pragma unroll
+        for (int k = 0; k < S; ++k) p.h_last[((size_t)b * D + d) * N + j * S + k] = h[q][k];
+      }
+    }
+  }
   if (MODE == kFwdSummary) {
 #pragma unroll
     for (int q = 0; q < CPT; ++q) {

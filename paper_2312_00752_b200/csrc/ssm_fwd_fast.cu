@@ -318,6 +318,12 @@ __global__ void __launch_bounds__((WARPS + 1) * 32) ssm_fwd_fast_kernel(const Fw
     else compute_tile(i, std::false_type{});
   }
   block_barrier(THREADS);
+  if (MODE == kFwdFull && p.h_last != nullptr && seg == p.nseg - 1 && valid) {
+#pragma unroll
+    for (int q = 0; q < 2; ++q)
+      *reinterpret_cast<float4*>(p.h_last + ((size_t)b * D + chan(q)) * 16 + 4 * j) =
+          make_float4(h[q][0].x, h[q][0].y, h[q][1].x, h[q][1].y);
+  }
   if (MODE == kFwdSummary && valid) {
 #pragma unroll
     for (int q = 0; q < 2; ++q) {
@@ -345,7 +351,7 @@ static cudaError_t launch_fast(const Plan& plan, const FwdParams& p, cudaStream_
 bool fwd_fast_applicable(const ssm_problem_t& prob, const FwdParams& p) {
   auto al16 = [](const void* q) { return q == nullptr || (reinterpret_cast<uintptr_t>(q) & 15) == 0; };
   return prob.io_dtype == SSM_BF16 && prob.N == 16 && prob.D % 8 == 0 && al16(p.x) && al16(p.delta) && al16(p.z) &&
-         al16(p.B) && al16(p.C) && al16(p.out) && al16(p.A) && al16(p.h_start) && al16(p.ckpt) && al16(p.seg_end);
+         al16(p.B) && al16(p.C) && al16(p.out) && al16(p.A) && al16(p.h_start) && al16(p.ckpt) && al16(p.seg_end) && al16(p.h_last);
 }
 
 // Two compute warps (32 channels) per block measured best on all three layer shapes (1, 3 and 4 were 3-35 % slower).
