@@ -25,6 +25,8 @@
  *   dC[t,n] += ds[t] h[t,n];   dD += ds[t] x[t];   dB[t,n] += lam[t,n] delta[t] x[t]
  *   dx[t]   = ds[t] D_skip + delta[t] sum_n lam[t,n] B[t,n]
  *   w[t,n]  = lam[t,n] h[t-1,n] a[t,n];   ddelta[t] = sum_n w[t,n] A[n] + x[t] sum_n lam[t,n] B[t,n];   dA[n] += w[t,n] delta[t]
+ * With the softplus switch the input is the pre-activation v, delta = softplus(v + delta_bias[d]), ddelta is the
+ * gradient of v (the line above times sigmoid(v + delta_bias[d])) and dbias[d] = sum over batch and time of ddelta.
  * Sums over channels (dB, dC) and over batch (dA, dD) are taken in a fixed order that does not depend on the
  * number of threads: channels are grouped in blocks of ORACLE_CH_BLOCK, each block accumulates in ascending channel
  * order into its own buffer, and the buffers are added in ascending block order.
@@ -47,6 +49,8 @@ typedef struct {
   int32_t has_z;      /* 0: out = s (no gate) */
   int32_t has_dskip;  /* 0: skip term absent */
   int32_t zoh_bbar;   /* 1: zero-order-hold B-bar of Eq. 4 (forward only; used by the gating-theorem pin) */
+  int32_t softplus;   /* 1: `delta` holds the pre-activation v and the step size is softplus(v + delta_bias[d])
+                         (Algorithm 2 step 4: Delta = tau_Delta(Parameter + s_Delta(x)), tau_Delta = softplus) */
   int32_t nthreads;   /* <= 0: all available */
 } oracle_dims_t;
 
@@ -69,6 +73,8 @@ int ssm_oracle_threads_available(void) {
 
 static inline double silu(double z) { return z / (1.0 + exp(-z)); }
 static inline double sigmoid(double z) { return 1.0 / (1.0 + exp(-z)); }
+/* softplus(v) = log(1 + e^v), written so that neither large nor very negative v loses accuracy */
+static inline double softplus(double v) { return (v > 0.0 ? v : 0.0) + log1p(exp(-fabs(v))); }
 
 /* ------------------------------------------------------------------------------------------------------------
  * The two entry-point families differ only in the storage type of the (batch, L, *) inputs.
@@ -77,7 +83,8 @@ static inline double sigmoid(double z) { return 1.0 / (1.0 + exp(-z)); }
   /* forward: out (batch,L,D); optional s_pre (pre-gate readout, batch,L,D); optional h_last (batch,D,N) */      \
   int ssm_oracle_fwd_##SUFFIX(const oracle_dims_t* p, const REAL* x, const REAL* delta, const double* A,         \
                               const REAL* B, const REAL* C, const double* D_skip, const REAL* z,                 \
-                              const double* h0, double* out, double* s_pre, double* h_last) {                    \
+                              const double* h0, const double* delta_bias, double* out, double* s_pre,            \
+                              double* h_last) {                                                                  \
     if (!p || p->batch < 1 || p->L < 1 || p->D < 1 || p->N < 1) return 1;                                         \
     const int64_t L = p->L, D = p->D, N = p->N;                                                                  \
     const int64_t items = (int64_t)p->batch * D;                                                                 \
@@ -90,7 +97,8 @@ static inline double sigmoid(double z) { return 1.0 / (1.0 + exp(-z)); }
       for (int64_t n = 0; n < N; ++n) h[n] = h0 ? h0[(b * D + d) * N + n] : 0.0;                                 \
       for (int64_t t = 0; t < L; ++t) {                                                                          \
         const int64_t e = (b * L + t) * D + d;                                                                   \
-        const double dt = (double)delta[e], u = (double)x[e];                                                    \
+        const double dv = (double)delta[e] + (delta_bias ? delta_bias[d] : 0.0);                                 \
+        const double dt = p->softplus ? softplus(dv) : dv, u = (double)x[e];                                     \
         const REAL* Bt = B + (b * L + t) * N;                                                                    \
         const REAL* Ct = C + (b * L + t) * N;                                                                    \
         double s = 0.0;                                                                                          \
@@ -115,8 +123,8 @@ static inline double sigmoid(double z) { return 1.0 / (1.0 + exp(-z)); }
   /* backward: every output is overwritten; dD and dz may be NULL */                                             \
   int ssm_oracle_bwd_##SUFFIX(const oracle_dims_t* p, const REAL* x, const REAL* delta, const double* A,         \
                               const REAL* B, const REAL* C, const double* D_skip, const REAL* z,                 \
-                              const REAL* dout, double* dx, double* ddelta, double* dA, double* dB, double* dC,  \
-                              double* dD, double* dz) {                                                          \
+                              const REAL* dout, const double* delta_bias, double* dx, double* ddelta,           \
+                              double* dA, double* dB, double* dC, double* dD, double* dz, double* dbias) {       \
     if (!p || p->batch < 1 || p->L < 1 || p->D < 1 || p->N < 1 || p->zoh_bbar) return 1;                          \
     const int64_t L = p->L, D = p->D, N = p->N, NB = p->batch;                                                   \
     const int64_t nblk = (D + ORACLE_CH_BLOCK - 1) / ORACLE_CH_BLOCK;                                            \
@@ -125,8 +133,9 @@ static inline double sigmoid(double z) { return 1.0 / (1.0 + exp(-z)); }
     (void)nt;                                                                                                    \
     double* dA_part = (double*)calloc((size_t)(NB * D * N), sizeof(double));     /* [b][d][n] */                 \
     double* dD_part = (double*)calloc((size_t)(NB * D), sizeof(double));         /* [b][d]    */                 \
+    double* dbias_part = (double*)calloc((size_t)(NB * D), sizeof(double));      /* [b][d]    */                 \
     double* dBC_part = (double*)calloc((size_t)(items * L * N * 2), sizeof(double)); /* [b][blk][2][t][n] */     \
-    int fail = (!dA_part || !dD_part || !dBC_part);                                                              \
+    int fail = (!dA_part || !dD_part || !dBC_part || !dbias_part);                                                              \
     if (!fail) {                                                                                                 \
       _Pragma("omp parallel for schedule(dynamic, 1) num_threads(nt)")                                           \
       for (int64_t it = 0; it < items; ++it) {                                                                   \
@@ -142,7 +151,8 @@ static inline double sigmoid(double z) { return 1.0 / (1.0 + exp(-z)); }
           for (int64_t n = 0; n < N; ++n) hs[n] = 0.0;                                                           \
           for (int64_t t = 1; t <= L; ++t) {                                                                     \
             const int64_t e = (b * L + (t - 1)) * D + d;                                                         \
-            const double dt = (double)delta[e], u = (double)x[e];                                                \
+            const double dv = (double)delta[e] + (delta_bias ? delta_bias[d] : 0.0);                             \
+            const double dt = p->softplus ? softplus(dv) : dv, u = (double)x[e];                                 \
             const REAL* Bt = B + (b * L + (t - 1)) * N;                                                          \
             const REAL* Ct = C + (b * L + (t - 1)) * N;                                                          \
             double s = 0.0;                                                                                      \
@@ -156,10 +166,11 @@ static inline double sigmoid(double z) { return 1.0 / (1.0 + exp(-z)); }
             ss[t] = s;                                                                                           \
           }                                                                                                      \
           for (int64_t n = 0; n < N; ++n) lam[n] = 0.0;                                                          \
-          double dD_acc = 0.0;                                                                                   \
+          double dD_acc = 0.0, dbias_acc = 0.0;                                                                  \
           for (int64_t t = L; t >= 1; --t) {                                                                     \
             const int64_t e = (b * L + (t - 1)) * D + d;                                                         \
-            const double dt = (double)delta[e], u = (double)x[e], g = (double)dout[e];                           \
+            const double dv = (double)delta[e] + (delta_bias ? delta_bias[d] : 0.0);                             \
+            const double dt = p->softplus ? softplus(dv) : dv, u = (double)x[e], g = (double)dout[e];            \
             const REAL* Bt = B + (b * L + (t - 1)) * N;                                                          \
             const REAL* Ct = C + (b * L + (t - 1)) * N;                                                          \
             double ds;                                                                                           \
@@ -184,10 +195,13 @@ static inline double sigmoid(double z) { return 1.0 / (1.0 + exp(-z)); }
               lam[n] = as[t * N + n] * l;                                                                        \
             }                                                                                                    \
             dx[e] = (p->has_dskip ? ds * D_skip[d] : 0.0) + dt * lamB;                                           \
-            ddelta[e] = wA + u * lamB;                                                                           \
+            /* with the softplus, ddelta is the gradient of the pre-activation: d softplus(v)/dv = sigmoid(v) */ \
+            ddelta[e] = (wA + u * lamB) * (p->softplus ? sigmoid(dv) : 1.0);                                     \
+            dbias_acc += ddelta[e];                                                                              \
             dD_acc += ds * u;                                                                                    \
           }                                                                                                      \
           dD_part[b * D + d] = dD_acc;                                                                           \
+          dbias_part[b * D + d] = dbias_acc;                                                                     \
         }                                                                                                        \
         free(hs); free(as); free(ss);                                                                            \
       }                                                                                                          \
@@ -217,9 +231,14 @@ static inline double sigmoid(double z) { return 1.0 / (1.0 + exp(-z)); }
           for (int64_t b = 0; b < NB; ++b) sd += dD_part[b * D + d];                                             \
           dD[d] = p->has_dskip ? sd : 0.0;                                                                       \
         }                                                                                                        \
+        if (dbias) {                                                                                             \
+          double sb = 0.0;                                                                                       \
+          for (int64_t b = 0; b < NB; ++b) sb += dbias_part[b * D + d];                                          \
+          dbias[d] = sb;                                                                                         \
+        }                                                                                                        \
       }                                                                                                          \
     }                                                                                                            \
-    free(dA_part); free(dD_part); free(dBC_part);                                                                \
+    free(dA_part); free(dD_part); free(dBC_part); free(dbias_part);                                                                \
     return fail ? 2 : 0;                                                                                         \
   }
 

@@ -25,7 +25,7 @@ _lib = None
 class _Dims(ctypes.Structure):
     _fields_ = [("batch", ctypes.c_int32), ("L", ctypes.c_int32), ("D", ctypes.c_int32), ("N", ctypes.c_int32),
                 ("has_z", ctypes.c_int32), ("has_dskip", ctypes.c_int32), ("zoh_bbar", ctypes.c_int32),
-                ("nthreads", ctypes.c_int32)]
+                ("softplus", ctypes.c_int32), ("nthreads", ctypes.c_int32)]
 
 
 def build(force: bool = False) -> str:
@@ -69,12 +69,13 @@ def _storage_dtype(x):
 
 
 def scan_fwd(x, delta, A, B, C, D_skip=None, z=None, h0=None, zoh=False, nthreads=0,
-             return_pregate=False, return_h_last=False):
+             return_pregate=False, return_h_last=False, delta_softplus=False, delta_bias=None):
     """Sequential fp64 selective scan (Algorithm 2 steps 5-6, Eq. 2, Eq. 4) + skip term + SiLU gate.
 
     x, delta, z: (batch, L, D); B, C: (batch, L, N); A: (D, N); D_skip: (D); h0: (batch, D, N) or None.
     Inputs stored as float32 are upcast exactly; anything else is taken as float64.  Returns float64 `out`
-    (and, if asked, the pre-gate readout s and the final state h_L).
+    (and, if asked, the pre-gate readout s and the final state h_L).  With delta_softplus the argument `delta` is
+    the pre-activation and the step size is softplus(delta + delta_bias[d]) (Algorithm 2 step 4).
     """
     lib = _load()
     st = _storage_dtype(x)
@@ -89,10 +90,12 @@ def scan_fwd(x, delta, A, B, C, D_skip=None, z=None, h0=None, zoh=False, nthread
     out = np.empty((batch, L, D), dtype=np.float64)
     s_pre = np.empty((batch, L, D), dtype=np.float64) if return_pregate else None
     h_last = np.empty((batch, D, N), dtype=np.float64) if return_h_last else None
-    dims = _Dims(batch, L, D, N, int(z is not None), int(D_skip is not None), int(bool(zoh)), int(nthreads))
+    bias = None if delta_bias is None else np.ascontiguousarray(delta_bias, dtype=np.float64)
+    dims = _Dims(batch, L, D, N, int(z is not None), int(D_skip is not None), int(bool(zoh)), int(bool(delta_softplus)),
+                 int(nthreads))
     fn = lib.ssm_oracle_fwd_f32 if st == np.float32 else lib.ssm_oracle_fwd_f64
     rc = fn(ctypes.byref(dims), _ptr(io["x"]), _ptr(io["delta"]), _ptr(A64), _ptr(io["B"]), _ptr(io["C"]),
-            _ptr(Dk), _ptr(io["z"]), _ptr(H0), _ptr(out), _ptr(s_pre), _ptr(h_last))
+            _ptr(Dk), _ptr(io["z"]), _ptr(H0), _ptr(bias), _ptr(out), _ptr(s_pre), _ptr(h_last))
     if rc != 0:
         raise RuntimeError(f"ssm_oracle_fwd failed with code {rc}")
     res = (out,)
@@ -103,11 +106,12 @@ def scan_fwd(x, delta, A, B, C, D_skip=None, z=None, h0=None, zoh=False, nthread
     return res[0] if len(res) == 1 else res
 
 
-def scan_bwd(x, delta, A, B, C, D_skip, z, dout, nthreads=0):
+def scan_bwd(x, delta, A, B, C, D_skip, z, dout, nthreads=0, delta_softplus=False, delta_bias=None):
     """Analytic adjoint of scan_fwd for loss = sum(dout * out), sequential, fp64.
 
     Returns a dict with dx, ddelta, dz (batch, L, D); dB, dC (batch, L, N); dA (D, N); dD (D) -- all float64.
-    dz is zero when z is None, dD is zero when D_skip is None.
+    dz is zero when z is None, dD is zero when D_skip is None.  With delta_softplus, `delta` is the pre-activation,
+    ddelta its gradient, and the dict also holds ddelta_bias (D) = ddelta summed over batch and time.
     """
     lib = _load()
     st = _storage_dtype(x)
@@ -121,11 +125,13 @@ def scan_bwd(x, delta, A, B, C, D_skip, z, dout, nthreads=0):
     g["dC"] = np.empty((batch, L, N), dtype=np.float64)
     g["dA"] = np.empty((D, N), dtype=np.float64)
     g["dD"] = np.empty((D,), dtype=np.float64)
-    dims = _Dims(batch, L, D, N, int(z is not None), int(D_skip is not None), 0, int(nthreads))
+    g["ddelta_bias"] = np.empty((D,), dtype=np.float64)
+    bias = None if delta_bias is None else np.ascontiguousarray(delta_bias, dtype=np.float64)
+    dims = _Dims(batch, L, D, N, int(z is not None), int(D_skip is not None), 0, int(bool(delta_softplus)), int(nthreads))
     fn = lib.ssm_oracle_bwd_f32 if st == np.float32 else lib.ssm_oracle_bwd_f64
     rc = fn(ctypes.byref(dims), _ptr(io["x"]), _ptr(io["delta"]), _ptr(A64), _ptr(io["B"]), _ptr(io["C"]), _ptr(Dk),
-            _ptr(io["z"]), _ptr(io["dout"]), _ptr(g["dx"]), _ptr(g["ddelta"]), _ptr(g["dA"]), _ptr(g["dB"]),
-            _ptr(g["dC"]), _ptr(g["dD"]), _ptr(g["dz"]))
+            _ptr(io["z"]), _ptr(io["dout"]), _ptr(bias), _ptr(g["dx"]), _ptr(g["ddelta"]), _ptr(g["dA"]), _ptr(g["dB"]),
+            _ptr(g["dC"]), _ptr(g["dD"]), _ptr(g["dz"]), _ptr(g["ddelta_bias"]))
     if rc != 0:
         raise RuntimeError(f"ssm_oracle_bwd failed with code {rc}")
     return g

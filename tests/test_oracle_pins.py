@@ -279,3 +279,53 @@ def test_f32_storage_matches_f64_and_threads_do_not_matter():
                     dout.astype(np.float64), nthreads=8)
     for k in g1:
         assert np.array_equal(g1[k], g8[k]), k
+
+
+# --------------------------------------------------------------------------------------------------------------
+# Step size through the softplus (Algorithm 2 step 4: Delta = softplus(Parameter + s_Delta(x))).
+def test_softplus_switch_equals_precomputed_step_and_gating_theorem():
+    batch, L, D, N = 2, 30, 4, 3
+    p = _rand_problem(batch, L, D, N)
+    v = RNG.standard_normal((batch, L, D)) * 3.0 - 2.0
+    bias = RNG.standard_normal(D)
+    step = np.logaddexp(0.0, v + bias)                          # library softplus, another route than the oracle's
+    a = O.scan_fwd(p["x"], v, p["A"], p["B"], p["C"], D_skip=p["D_skip"], z=p["z"], delta_softplus=True, delta_bias=bias)
+    b = O.scan_fwd(p["x"], step, p["A"], p["B"], p["C"], D_skip=p["D_skip"], z=p["z"])
+    np.testing.assert_allclose(a, b, rtol=1e-13, atol=1e-14)
+    # Theorem 1 stated on the pre-activation: N = 1, A = -1, B = C = 1, zero-order hold  =>  gate g = sigmoid(v)
+    x = RNG.standard_normal((batch, L, D))
+    ones = np.ones((batch, L, 1))
+    g = 1.0 / (1.0 + np.exp(-v))
+    h = np.zeros((batch, D))
+    ref = np.empty((batch, L, D))
+    for t in range(L):
+        h = (1.0 - g[:, t]) * h + g[:, t] * x[:, t]
+        ref[:, t] = h
+    got = O.scan_fwd(x, v, -np.ones((D, 1)), ones, ones, zoh=True, delta_softplus=True)
+    np.testing.assert_allclose(got, ref, rtol=1e-12, atol=1e-13)
+
+
+def test_softplus_gradients_match_finite_differences():
+    batch, L, D, N = 2, 10, 3, 4
+    p = _rand_problem(batch, L, D, N)
+    v = RNG.standard_normal((batch, L, D)) * 2.0 - 1.0
+    bias = RNG.standard_normal(D)
+    dout = RNG.standard_normal((batch, L, D))
+    g = O.scan_bwd(p["x"], v, p["A"], p["B"], p["C"], p["D_skip"], p["z"], dout, delta_softplus=True, delta_bias=bias)
+
+    def loss(vv, bb):
+        return float((dout * O.scan_fwd(p["x"], vv, p["A"], p["B"], p["C"], D_skip=p["D_skip"], z=p["z"],
+                                        delta_softplus=True, delta_bias=bb)).sum())
+    eps = 1e-6
+    for trial in range(3):
+        dv, db = RNG.standard_normal(v.shape), RNG.standard_normal(D)
+        fd_v = (loss(v + eps * dv, bias) - loss(v - eps * dv, bias)) / (2 * eps)
+        fd_b = (loss(v, bias + eps * db) - loss(v, bias - eps * db)) / (2 * eps)
+        assert abs(fd_v - (g["ddelta"] * dv).sum()) <= 1e-6 * max(1.0, abs(fd_v))
+        assert abs(fd_b - (g["ddelta_bias"] * db).sum()) <= 1e-6 * max(1.0, abs(fd_b))
+    # the other gradients equal those of the unfused problem with the precomputed step size
+    step = np.logaddexp(0.0, v + bias)
+    g0 = O.scan_bwd(p["x"], step, p["A"], p["B"], p["C"], p["D_skip"], p["z"], dout)
+    for k in ("dx", "dz", "dA", "dB", "dC", "dD"):
+        np.testing.assert_allclose(g[k], g0[k], rtol=1e-11, atol=1e-12)
+    np.testing.assert_allclose(g["ddelta"], g0["ddelta"] / (1.0 + np.exp(-(v + bias))), rtol=1e-11, atol=1e-12)
