@@ -71,6 +71,7 @@ enum {
   SSM_FLAG_SAVE_STATES = 4u,  /* forward: also write the checkpoint states that backward starts its recomputation
                                  from (Appendix D keeps "intermediate scan states" between chunks)             */
   SSM_FLAG_GENERAL_A = 8u,    /* do not use the fast path for rows of A that are arithmetic progressions in n   */
+  SSM_FLAG_DELTA_SOFTPLUS = 32u, /* ssm_scan_*_fused_dt: the step size is softplus(delta_pre + delta_bias[d])         */
   SSM_FLAG_TEST_WITHHOLD = 16u /* test hook for the bounded waits: the tuned backward kernel never publishes its
                                  hand-off flags and polls only 1000 times, so every dependent tile gives up and
                                  ssm_scan_check_status reports SSM_ERR_TIMEOUT; the gradients are then undefined  */
@@ -120,6 +121,32 @@ SSM_API ssm_status_t ssm_scan_fwd_state(const ssm_problem_t* p, const void* x, c
                                         const void* B, const void* C, const float* D_skip, const void* z,
                                         const float* h0, void* out, float* h_last, void* saved_states,
                                         void* workspace, size_t workspace_bytes, void* stream /* cudaStream_t */);
+
+/*
+ * Forward and backward with the step-size activation fused in (Algorithm 2 step 4: Delta = tau_Delta(Parameter +
+ * s_Delta(x)) with tau_Delta = softplus, Section 3.2; the bias initialisation of Section 3.6 is that Parameter).
+ * `delta_pre` [batch][L][D] (io_dtype) is the output of the projection s_Delta, `delta_bias` float32 [D] the parameter
+ * (NULL: zero); the step size used by the scan is
+ *     delta = softplus(delta_pre + delta_bias[d])     with SSM_FLAG_DELTA_SOFTPLUS,
+ *     delta = delta_pre + delta_bias[d]               without it,
+ * evaluated in float32 and never rounded to io_dtype, which saves the separate elementwise pass over [batch][L][D] in
+ * each direction.  Everything else is as in ssm_scan_fwd_state / ssm_scan_bwd.  The backward returns
+ *     ddelta_pre   io_dtype [batch][L][D]: gradient of the pre-activation (ddelta * sigmoid(delta_pre + bias) with the
+ *                  softplus),
+ *     ddelta_bias  float32 [D], may be NULL: ddelta_pre summed over batch and time (fixed order).
+ * These calls currently run the generic kernels for every shape (the tuned bf16 kernels take the step size as given).
+ */
+SSM_API ssm_status_t ssm_scan_fwd_fused_dt(const ssm_problem_t* p, const void* x, const void* delta_pre,
+                                           const float* delta_bias, const float* A, const void* B, const void* C,
+                                           const float* D_skip, const void* z, const float* h0, void* out,
+                                           float* h_last, void* saved_states, void* workspace, size_t workspace_bytes,
+                                           void* stream /* cudaStream_t */);
+SSM_API ssm_status_t ssm_scan_bwd_fused_dt(const ssm_problem_t* p, const void* x, const void* delta_pre,
+                                           const float* delta_bias, const float* A, const void* B, const void* C,
+                                           const float* D_skip, const void* z, const void* dout,
+                                           const void* saved_states, void* dx, void* ddelta_pre, float* ddelta_bias,
+                                           float* dA, void* dB, void* dC, float* dD, void* dz, void* workspace,
+                                           size_t workspace_bytes, void* stream /* cudaStream_t */);
 
 /*
  * One recurrent step (Eq. 2a/2b evaluated for a single t, the mode used for autoregressive inference): p->L must be

@@ -16,11 +16,13 @@ from . import build as _build
 SSM_OK = 0
 SSM_F32, SSM_BF16 = 0, 1
 SSM_FLAG_HAS_Z, SSM_FLAG_HAS_DSKIP, SSM_FLAG_SAVE_STATES, SSM_FLAG_GENERAL_A, SSM_FLAG_TEST_WITHHOLD = 1, 2, 4, 8, 16
+SSM_FLAG_DELTA_SOFTPLUS = 32
 
 EXPORTED_SYMBOLS = (
     "ssm_scan_fwd_workspace_bytes", "ssm_scan_bwd_workspace_bytes", "ssm_scan_saved_state_bytes",
     "ssm_scan_checkpoint_steps", "ssm_scan_fwd", "ssm_scan_bwd", "ssm_status_string", "ssm_scan_plan",
     "ssm_scan_fwd_static", "ssm_scan_check_status", "ssm_scan_fwd_state", "ssm_step",
+    "ssm_scan_fwd_fused_dt", "ssm_scan_bwd_fused_dt",
 )
 SSM_STATIC_SCRATCH_BYTES = 4 << 20
 
@@ -69,6 +71,10 @@ def load_library() -> ctypes.CDLL:
     lib.ssm_scan_bwd.argtypes = [P] + [vp] * 16 + [vp, sz, vp]
     lib.ssm_scan_fwd_state.restype = ctypes.c_int
     lib.ssm_scan_fwd_state.argtypes = [P] + [vp] * 11 + [vp, sz, vp]
+    lib.ssm_scan_fwd_fused_dt.restype = ctypes.c_int
+    lib.ssm_scan_fwd_fused_dt.argtypes = [P] + [vp] * 12 + [vp, sz, vp]
+    lib.ssm_scan_bwd_fused_dt.restype = ctypes.c_int
+    lib.ssm_scan_bwd_fused_dt.argtypes = [P] + [vp] * 18 + [vp, sz, vp]
     lib.ssm_step.restype = ctypes.c_int
     lib.ssm_step.argtypes = [P] + [vp] * 10
     lib.ssm_scan_check_status.restype = ctypes.c_int
@@ -188,6 +194,69 @@ def ssm_scan_fwd(x, delta, A, B, C, D_skip=None, z=None, *, save_states=False, g
         ctypes.c_void_p(stream_ptr))
     _check(code, "ssm_scan_fwd_state")
     return (out, saved_states) if save_states else out
+
+
+def ssm_scan_fwd_fused_dt(x, delta_pre, delta_bias, A, B, C, D_skip=None, z=None, *, softplus=True, save_states=False,
+                          out=None, saved_states=None, stream=None, h0=None, h_last=None):
+    """Forward with the step-size activation fused: delta = softplus(delta_pre + delta_bias) (or the plain sum with
+    softplus=False), in float32.  Otherwise as ssm_scan_fwd."""
+    lib = load_library()
+    prob = make_problem(x, B, z is not None, D_skip is not None, save_states, False)
+    if softplus:
+        prob.flags |= SSM_FLAG_DELTA_SOFTPLUS
+    batch, L, D, N = prob.batch, prob.L, prob.D, prob.N
+    io = x.dtype
+    if out is None:
+        out = torch.empty_like(x)
+    if save_states and saved_states is None:
+        saved_states = torch.empty(saved_state_bytes(prob) // 4, dtype=torch.float32, device=x.device)
+    stream_ptr = (stream if stream is not None else torch.cuda.current_stream(x.device)).cuda_stream
+    ws = _workspace(fwd_workspace_bytes(prob), x.device, stream_ptr)
+    code = lib.ssm_scan_fwd_fused_dt(
+        ctypes.byref(prob), _dev_ptr(x, "x", (batch, L, D), io), _dev_ptr(delta_pre, "delta_pre", (batch, L, D), io),
+        _dev_ptr(delta_bias, "delta_bias", (D,), torch.float32), _dev_ptr(A, "A", (D, N), torch.float32),
+        _dev_ptr(B, "B", (batch, L, N), io), _dev_ptr(C, "C", (batch, L, N), io),
+        _dev_ptr(D_skip, "D_skip", (D,), torch.float32), _dev_ptr(z, "z", (batch, L, D), io),
+        _dev_ptr(h0, "h0", (batch, D, N), torch.float32), _dev_ptr(out, "out", (batch, L, D), io),
+        _dev_ptr(h_last, "h_last", (batch, D, N), torch.float32),
+        _dev_ptr(saved_states if save_states else None, "saved_states"),
+        _dev_ptr(ws, "workspace"), ctypes.c_size_t(0 if ws is None else ws.numel() * ws.element_size()),
+        ctypes.c_void_p(stream_ptr))
+    _check(code, "ssm_scan_fwd_fused_dt")
+    return (out, saved_states) if save_states else out
+
+
+def ssm_scan_bwd_fused_dt(x, delta_pre, delta_bias, A, B, C, D_skip, z, dout, saved_states=None, *, softplus=True,
+                          stream=None):
+    """Backward of ssm_scan_fwd_fused_dt.  Returns the dict of ssm_scan_bwd with `ddelta` the gradient of delta_pre
+    and an extra `ddelta_bias` (D,) float32."""
+    lib = load_library()
+    prob = make_problem(x, B, z is not None, D_skip is not None, False, False)
+    if softplus:
+        prob.flags |= SSM_FLAG_DELTA_SOFTPLUS
+    batch, L, D, N = prob.batch, prob.L, prob.D, prob.N
+    io = x.dtype
+    o = {"dx": torch.empty_like(x), "ddelta": torch.empty_like(x),
+         "ddelta_bias": torch.empty((D,), dtype=torch.float32, device=x.device),
+         "dA": torch.empty((D, N), dtype=torch.float32, device=x.device), "dB": torch.empty_like(B),
+         "dC": torch.empty_like(B),
+         "dD": torch.empty((D,), dtype=torch.float32, device=x.device) if D_skip is not None else None,
+         "dz": torch.empty_like(x) if z is not None else None}
+    stream_ptr = (stream if stream is not None else torch.cuda.current_stream(x.device)).cuda_stream
+    ws = _workspace(bwd_workspace_bytes(prob), x.device, stream_ptr)
+    code = lib.ssm_scan_bwd_fused_dt(
+        ctypes.byref(prob), _dev_ptr(x, "x", (batch, L, D), io), _dev_ptr(delta_pre, "delta_pre", (batch, L, D), io),
+        _dev_ptr(delta_bias, "delta_bias", (D,), torch.float32), _dev_ptr(A, "A", (D, N), torch.float32),
+        _dev_ptr(B, "B", (batch, L, N), io), _dev_ptr(C, "C", (batch, L, N), io),
+        _dev_ptr(D_skip, "D_skip", (D,), torch.float32), _dev_ptr(z, "z", (batch, L, D), io),
+        _dev_ptr(dout, "dout", (batch, L, D), io), _dev_ptr(saved_states, "saved_states"),
+        _dev_ptr(o["dx"], "dx"), _dev_ptr(o["ddelta"], "ddelta"), _dev_ptr(o["ddelta_bias"], "ddelta_bias"),
+        _dev_ptr(o["dA"], "dA"), _dev_ptr(o["dB"], "dB"), _dev_ptr(o["dC"], "dC"), _dev_ptr(o["dD"], "dD"),
+        _dev_ptr(o["dz"], "dz"),
+        _dev_ptr(ws, "workspace"), ctypes.c_size_t(0 if ws is None else ws.numel() * ws.element_size()),
+        ctypes.c_void_p(stream_ptr))
+    _check(code, "ssm_scan_bwd_fused_dt")
+    return o
 
 
 def ssm_step(x, delta, A, B, C, D_skip, z, h, *, out=None, stream=None):

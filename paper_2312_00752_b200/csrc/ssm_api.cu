@@ -15,7 +15,8 @@ static inline size_t align_up(size_t v) { return (v + 255) & ~(size_t)255; }
 static ssm_status_t validate_problem(const ssm_problem_t* p) {
   if (p == nullptr) return SSM_ERR_INVALID_ARG;
   if (p->batch < 1 || p->L < 1 || p->D < 1 || p->N < 1) return SSM_ERR_INVALID_ARG;
-  if (p->flags & ~(uint32_t)(SSM_FLAG_HAS_Z | SSM_FLAG_HAS_DSKIP | SSM_FLAG_SAVE_STATES | SSM_FLAG_GENERAL_A | SSM_FLAG_TEST_WITHHOLD))
+  if (p->flags & ~(uint32_t)(SSM_FLAG_HAS_Z | SSM_FLAG_HAS_DSKIP | SSM_FLAG_SAVE_STATES | SSM_FLAG_GENERAL_A | SSM_FLAG_TEST_WITHHOLD |
+                             SSM_FLAG_DELTA_SOFTPLUS))
     return SSM_ERR_INVALID_ARG;
   if (p->io_dtype != SSM_F32 && p->io_dtype != SSM_BF16) return SSM_ERR_UNSUPPORTED;
   if (p->N != 1 && p->N != 2 && p->N != 4 && p->N != 8 && p->N != 16) return SSM_ERR_UNSUPPORTED;
@@ -65,7 +66,7 @@ static FwdWorkspace fwd_layout(const ssm_problem_t& p, const Plan& pl) {
 }
 
 struct BwdWorkspace {
-  size_t dBC_part, dA_part, dD_part, ckpt, seg_local, seg_dsum, mu_in, fwd, sched, handoff, total;
+  size_t dBC_part, dA_part, dD_part, dbias_part, ckpt, seg_local, seg_dsum, mu_in, fwd, sched, handoff, total;
 };
 static BwdWorkspace bwd_layout(const ssm_problem_t& p, const Plan& pl) {
   BwdWorkspace w{};
@@ -80,6 +81,7 @@ static BwdWorkspace bwd_layout(const ssm_problem_t& p, const Plan& pl) {
   w.dBC_part = take((size_t)pl.bwd_groups * 2 * bln * sizeof(float));
   w.dA_part = take(parts * p.D * p.N * sizeof(float));
   w.dD_part = take(parts * p.D * sizeof(float));
+  w.dbias_part = take(parts * p.D * sizeof(float));
   w.ckpt = take((size_t)p.batch * pl.nck * p.D * p.N * sizeof(float));
   if (pl.nseg > 1) {
     const size_t st = parts * p.D * p.N * sizeof(float);
@@ -194,10 +196,10 @@ ssm_status_t ssm_scan_plan(const ssm_problem_t* p, int32_t* n_segments, int32_t*
   return SSM_OK;
 }
 
-ssm_status_t ssm_scan_fwd_state(const ssm_problem_t* p, const void* x, const void* delta, const float* A,
-                                const void* B, const void* C, const float* D_skip, const void* z, const float* h0,
-                                void* out, float* h_last, void* saved_states, void* workspace, size_t workspace_bytes,
-                                void* stream) {
+static ssm_status_t fwd_impl(const ssm_problem_t* p, const void* x, const void* delta, const float* delta_bias,
+                             const float* A, const void* B, const void* C, const float* D_skip, const void* z,
+                             const float* h0, void* out, float* h_last, void* saved_states, void* workspace,
+                             size_t workspace_bytes, void* stream) {
   ssm_status_t st = validate_problem(p);
   if (st != SSM_OK) return st;
   const bool has_z = p->flags & SSM_FLAG_HAS_Z, has_d = p->flags & SSM_FLAG_HAS_DSKIP;
@@ -207,7 +209,8 @@ ssm_status_t ssm_scan_fwd_state(const ssm_problem_t* p, const void* x, const voi
   const size_t esz = p->io_dtype == SSM_BF16 ? 2 : 4;
   for (const void* q : {x, delta, B, C, z, (const void*)out})
     if (q && !aligned_to(q, esz)) return SSM_ERR_INVALID_ARG;
-  for (const void* q : {(const void*)A, (const void*)D_skip, (const void*)saved_states, (const void*)h0, (const void*)h_last})
+  for (const void* q : {(const void*)A, (const void*)D_skip, (const void*)saved_states, (const void*)h0, (const void*)h_last,
+                        (const void*)delta_bias})
     if (q && !aligned_to(q, 4)) return SSM_ERR_INVALID_ARG;
   const Plan pl = make_plan(*p);
   st = check_ws(workspace, workspace_bytes, fwd_layout(*p, pl).total);
@@ -230,6 +233,8 @@ ssm_status_t ssm_scan_fwd_state(const ssm_problem_t* p, const void* x, const voi
   fp.seg_steps = pl.seg_steps;
   fp.nck = pl.nck;
   fp.general_A = (p->flags & SSM_FLAG_GENERAL_A) ? 1 : 0;
+  fp.delta_bias = delta_bias;
+  fp.softplus = (p->flags & SSM_FLAG_DELTA_SOFTPLUS) ? 1 : 0;
   const float* h_start = nullptr;
   if (run_segment_starts(*p, pl, fp, static_cast<char*>(workspace), h0, &h_start, s) != cudaSuccess) return SSM_ERR_CUDA;
   fp.h_start = h_start;
@@ -239,11 +244,27 @@ ssm_status_t ssm_scan_fwd_state(const ssm_problem_t* p, const void* x, const voi
   return SSM_OK;
 }
 
+ssm_status_t ssm_scan_fwd_state(const ssm_problem_t* p, const void* x, const void* delta, const float* A,
+                                const void* B, const void* C, const float* D_skip, const void* z, const float* h0,
+                                void* out, float* h_last, void* saved_states, void* workspace, size_t workspace_bytes,
+                                void* stream) {
+  return fwd_impl(p, x, delta, nullptr, A, B, C, D_skip, z, h0, out, h_last, saved_states, workspace, workspace_bytes,
+                  stream);
+}
+
 ssm_status_t ssm_scan_fwd(const ssm_problem_t* p, const void* x, const void* delta, const float* A, const void* B,
                           const void* C, const float* D_skip, const void* z, void* out, void* saved_states,
                           void* workspace, size_t workspace_bytes, void* stream) {
-  return ssm_scan_fwd_state(p, x, delta, A, B, C, D_skip, z, nullptr, out, nullptr, saved_states, workspace,
-                            workspace_bytes, stream);
+  return fwd_impl(p, x, delta, nullptr, A, B, C, D_skip, z, nullptr, out, nullptr, saved_states, workspace,
+                  workspace_bytes, stream);
+}
+
+ssm_status_t ssm_scan_fwd_fused_dt(const ssm_problem_t* p, const void* x, const void* delta_pre,
+                                   const float* delta_bias, const float* A, const void* B, const void* C,
+                                   const float* D_skip, const void* z, const float* h0, void* out, float* h_last,
+                                   void* saved_states, void* workspace, size_t workspace_bytes, void* stream) {
+  return fwd_impl(p, x, delta_pre, delta_bias, A, B, C, D_skip, z, h0, out, h_last, saved_states, workspace,
+                  workspace_bytes, stream);
 }
 
 ssm_status_t ssm_step(const ssm_problem_t* p, const void* x, const void* delta, const float* A, const void* B,
@@ -276,10 +297,11 @@ ssm_status_t ssm_step(const ssm_problem_t* p, const void* x, const void* delta, 
   return SSM_OK;
 }
 
-ssm_status_t ssm_scan_bwd(const ssm_problem_t* p, const void* x, const void* delta, const float* A, const void* B,
-                          const void* C, const float* D_skip, const void* z, const void* dout,
-                          const void* saved_states, void* dx, void* ddelta, float* dA, void* dB, void* dC, float* dD,
-                          void* dz, void* workspace, size_t workspace_bytes, void* stream) {
+static ssm_status_t bwd_impl(const ssm_problem_t* p, const void* x, const void* delta, const float* delta_bias,
+                             const float* A, const void* B, const void* C, const float* D_skip, const void* z,
+                             const void* dout, const void* saved_states, void* dx, void* ddelta, float* ddelta_bias,
+                             float* dA, void* dB, void* dC, float* dD, void* dz, void* workspace,
+                             size_t workspace_bytes, void* stream) {
   ssm_status_t st = validate_problem(p);
   if (st != SSM_OK) return st;
   const bool has_z = p->flags & SSM_FLAG_HAS_Z, has_d = p->flags & SSM_FLAG_HAS_DSKIP;
@@ -289,7 +311,8 @@ ssm_status_t ssm_scan_bwd(const ssm_problem_t* p, const void* x, const void* del
   for (const void* q : {x, delta, B, C, z, dout, (const void*)dx, (const void*)ddelta, (const void*)dB,
                         (const void*)dC, (const void*)dz})
     if (q && !aligned_to(q, esz)) return SSM_ERR_INVALID_ARG;
-  for (const void* q : {(const void*)A, (const void*)D_skip, saved_states, (const void*)dA, (const void*)dD})
+  for (const void* q : {(const void*)A, (const void*)D_skip, saved_states, (const void*)dA, (const void*)dD,
+                        (const void*)delta_bias, (const void*)ddelta_bias})
     if (q && !aligned_to(q, 4)) return SSM_ERR_INVALID_ARG;
   const Plan pl = make_plan(*p);
   const BwdWorkspace w = bwd_layout(*p, pl);
@@ -315,6 +338,8 @@ ssm_status_t ssm_scan_bwd(const ssm_problem_t* p, const void* x, const void* del
     fp.seg_steps = pl.seg_steps;
     fp.nck = pl.nck;
     fp.general_A = (p->flags & SSM_FLAG_GENERAL_A) ? 1 : 0;
+    fp.delta_bias = delta_bias;
+    fp.softplus = (p->flags & SSM_FLAG_DELTA_SOFTPLUS) ? 1 : 0;
     const float* h_start = nullptr;
     if (run_segment_starts(*p, pl, fp, ws + w.fwd, nullptr, &h_start, s) != cudaSuccess) return SSM_ERR_CUDA;
     fp.h_start = h_start;
@@ -348,6 +373,9 @@ ssm_status_t ssm_scan_bwd(const ssm_problem_t* p, const void* x, const void* del
   bp.groups = pl.bwd_groups;
   bp.general_A = (p->flags & SSM_FLAG_GENERAL_A) ? 1 : 0;
   bp.test_withhold = (p->flags & SSM_FLAG_TEST_WITHHOLD) ? 1 : 0;
+  bp.delta_bias = delta_bias;
+  bp.softplus = (p->flags & SSM_FLAG_DELTA_SOFTPLUS) ? 1 : 0;
+  bp.dbias_part = ddelta_bias != nullptr ? reinterpret_cast<float*>(ws + w.dbias_part) : nullptr;
   bp.sched = reinterpret_cast<int*>(ws + w.sched);
   bp.handoff = reinterpret_cast<float4*>(ws + w.handoff);
   // scheduling words of the tuned kernel (claim counter, abort word, one progress flag per chain) start at zero; the
@@ -381,6 +409,8 @@ ssm_status_t ssm_scan_bwd(const ssm_problem_t* p, const void* x, const void* del
   rp.dD_part = bp.dD_part;
   rp.dA = dA;
   rp.dD = has_d ? dD : nullptr;
+  rp.dbias_part = bp.dbias_part;
+  rp.dbias = ddelta_bias;
   rp.bln = (long long)p->batch * p->L * p->N;
   rp.groups = pl.bwd_groups;
   rp.parts = p->batch * pl.nseg;
@@ -388,6 +418,23 @@ ssm_status_t ssm_scan_bwd(const ssm_problem_t* p, const void* x, const void* del
   rp.N = p->N;
   if (launch_bwd_reduce(*p, rp, s) != cudaSuccess) return SSM_ERR_CUDA;
   return SSM_OK;
+}
+
+ssm_status_t ssm_scan_bwd(const ssm_problem_t* p, const void* x, const void* delta, const float* A, const void* B,
+                          const void* C, const float* D_skip, const void* z, const void* dout,
+                          const void* saved_states, void* dx, void* ddelta, float* dA, void* dB, void* dC, float* dD,
+                          void* dz, void* workspace, size_t workspace_bytes, void* stream) {
+  return bwd_impl(p, x, delta, nullptr, A, B, C, D_skip, z, dout, saved_states, dx, ddelta, nullptr, dA, dB, dC, dD, dz,
+                  workspace, workspace_bytes, stream);
+}
+
+ssm_status_t ssm_scan_bwd_fused_dt(const ssm_problem_t* p, const void* x, const void* delta_pre,
+                                   const float* delta_bias, const float* A, const void* B, const void* C,
+                                   const float* D_skip, const void* z, const void* dout, const void* saved_states,
+                                   void* dx, void* ddelta_pre, float* ddelta_bias, float* dA, void* dB, void* dC,
+                                   float* dD, void* dz, void* workspace, size_t workspace_bytes, void* stream) {
+  return bwd_impl(p, x, delta_pre, delta_bias, A, B, C, D_skip, z, dout, saved_states, dx, ddelta_pre, ddelta_bias, dA,
+                  dB, dC, dD, dz, workspace, workspace_bytes, stream);
 }
 
 }  // extern "C"

@@ -80,8 +80,9 @@ __global__ void __launch_bounds__(BwdGeom<N>::THREADS) ssm_bwd_kernel(const BwdP
   const bool has_z = gz != nullptr;
 
   float Ar[S], A2[S], mu[S], dA[S];
-  float dD_acc = 0.f;
+  float dD_acc = 0.f, dbias_acc = 0.f;
   const float Dk = (valid && p.Dskip != nullptr) ? p.Dskip[d] : 0.f;
+  const float dbias = (valid && p.delta_bias != nullptr) ? p.delta_bias[d] : 0.f;
 #pragma unroll
   for (int k = 0; k < S; ++k) {
     Ar[k] = valid ? p.A[(size_t)d * N + j * S + k] : 0.f;
@@ -122,7 +123,8 @@ __global__ void __launch_bounds__(BwdGeom<N>::THREADS) ssm_bwd_kernel(const BwdP
 
     // ---- recompute h_1 .. h_nt of this block and the pre-gate readout s_t
     for (int tt = 0; tt < nt; ++tt) {
-      const float dt = io_to_float<IO>(s_d[tt * CH + slot]);
+      float dt = io_to_float<IO>(s_d[tt * CH + slot]) + dbias;
+      if (p.softplus) dt = softplus_precise(dt);
       const float u = io_to_float<IO>(s_x[tt * CH + slot]);
       const float du = dt * u;
       float y = 0.f;
@@ -141,7 +143,8 @@ __global__ void __launch_bounds__(BwdGeom<N>::THREADS) ssm_bwd_kernel(const BwdP
 
     // ---- reverse recurrence over the block
     for (int tt = nt - 1; tt >= 0; --tt) {
-      const float dt = io_to_float<IO>(s_d[tt * CH + slot]);
+      const float dv = io_to_float<IO>(s_d[tt * CH + slot]) + dbias;
+      const float dt = p.softplus ? softplus_precise(dv) : dv;
       const float u = io_to_float<IO>(s_x[tt * CH + slot]);
       const float g = io_to_float<IO>(s_g[tt * CH + slot]);
       const float du = dt * u;
@@ -192,8 +195,11 @@ __global__ void __launch_bounds__(BwdGeom<N>::THREADS) ssm_bwd_kernel(const BwdP
       }
       if (j == 0) {
         dD_acc = fmaf(ds, u, dD_acc);
+        // with the softplus the gradient goes to the pre-activation: d softplus(v)/dv = sigmoid(v)
+        const float ddv = fmaf(u, lamB, wA) * (p.softplus ? 1.f / (1.f + __expf(-dv)) : 1.f);
+        dbias_acc += ddv;
         s_x[tt * CH + slot] = float_to_io<IO>(fmaf(ds, Dk, dt * lamB));
-        s_d[tt * CH + slot] = float_to_io<IO>(fmaf(u, lamB, wA));
+        s_d[tt * CH + slot] = float_to_io<IO>(ddv);
         s_z[tt * CH + slot] = float_to_io<IO>(dzv);
       }
     }
@@ -223,6 +229,7 @@ __global__ void __launch_bounds__(BwdGeom<N>::THREADS) ssm_bwd_kernel(const BwdP
 #pragma unroll
     for (int k = 0; k < S; ++k) p.dA_part[(part * D + d) * N + j * S + k] = dA[k];
     if (j == 0) p.dD_part[part * D + d] = dD_acc;
+    if (j == 0 && p.dbias_part != nullptr) p.dbias_part[part * D + d] = dbias_acc;
   }
 }
 
@@ -252,6 +259,7 @@ __global__ void __launch_bounds__(BwdGeom<N>::THREADS) ssm_bwd_local_kernel(cons
   const bool has_z = gz != nullptr;
 
   float A2[S], mu[S], dsum = 0.f;
+  const float dbias = (valid && p.delta_bias != nullptr) ? p.delta_bias[d] : 0.f;
 #pragma unroll
   for (int k = 0; k < S; ++k) {
     A2[k] = valid ? p.A[(size_t)d * N + j * S + k] * kLog2e : 0.f;
@@ -274,7 +282,8 @@ __global__ void __launch_bounds__(BwdGeom<N>::THREADS) ssm_bwd_local_kernel(cons
     for (int i = tid; i < T * N; i += kBwdThreads) s_C[i] = (i / N < nt) ? io_to_float<IO>(gC[row0 * N + i]) : 0.f;
     __syncthreads();
     for (int tt = nt - 1; tt >= 0; --tt) {
-      const float dt = io_to_float<IO>(s_d[tt * CH + slot]);
+      float dt = io_to_float<IO>(s_d[tt * CH + slot]) + dbias;
+      if (p.softplus) dt = softplus_precise(dt);
       float ds = io_to_float<IO>(s_g[tt * CH + slot]);
       if (has_z) {
         const float zz = io_to_float<IO>(s_z[tt * CH + slot]);
@@ -317,6 +326,11 @@ __global__ void __launch_bounds__(256) ssm_bwd_reduce_kernel(const ReduceParams 
     float sd = 0.f;
     for (int q = 0; q < p.parts; ++q) sd += p.dD_part[(size_t)q * p.D + i];
     p.dD[i] = sd;
+  }
+  if (p.dbias != nullptr && i < p.D) {
+    float sb = 0.f;
+    for (int q = 0; q < p.parts; ++q) sb += p.dbias_part[(size_t)q * p.D + i];
+    p.dbias[i] = sb;
   }
 }
 

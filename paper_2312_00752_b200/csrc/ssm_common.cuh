@@ -43,6 +43,8 @@ struct FwdParams {
   float* seg_end;        // SUMMARY mode: [batch][nseg][D][N] end state of each segment started from zero
   float* seg_dsum;       // SUMMARY mode: [batch][nseg][D] sum of delta over the segment
   float* h_last;         // FULL mode: [batch][D][N] state after the last step; null: not wanted
+  const float* delta_bias;  // [D] added to delta before the softplus; null: none
+  int softplus;          // 1: `delta` is the pre-activation, the step size is softplus(delta + delta_bias)
   int batch, L, D, nseg, seg_steps, nck;
   int general_A;       // 1: never take the arithmetic-progression fast path
 };
@@ -79,6 +81,9 @@ struct BwdParams {
   float* dD_part;         // [batch*nseg][D]
   int batch, L, D, nseg, seg_steps, nck, groups;
   int general_A;          // 1: never take the arithmetic-progression fast path
+  const float* delta_bias;  // as in FwdParams
+  int softplus;
+  float* dbias_part;      // [batch*nseg][D] sums of the pre-activation gradient; null: not wanted
   int test_withhold;      // test hook: never publish hand-off flags, poll only 1000 times
   int* sched;             // tuned kernel: [0] claim counter, [1] abort word, [64 + chain] progress flag per chain
   float4* handoff;        // tuned kernel: carried values between consecutive tiles of a chain
@@ -92,6 +97,8 @@ struct ReduceParams {
   const float* dD_part;   // [parts][D]
   float* dA;
   float* dD;              // null: skip
+  const float* dbias_part;  // [parts][D]
+  float* dbias;           // null: skip
   long long bln;          // batch*L*N
   int groups, parts, D, N;
 };
@@ -163,6 +170,9 @@ __device__ __forceinline__ float bf16sel(uint32_t w, uint32_t sel) { return __ui
 __device__ __forceinline__ float2 f2mul(float2 a, float2 b) { return __fmul2_rn(a, b); }
 __device__ __forceinline__ float2 f2fma(float2 a, float2 b, float2 c) { return __ffma2_rn(a, b, c); }
 __device__ __forceinline__ float2 f2dup(float v) { return make_float2(v, v); }
+
+// softplus(v) = log(1 + e^v) = max(v, 0) + log1p(e^-|v|) with the precise library log1p (generic kernels)
+__device__ __forceinline__ float softplus_precise(float v) { return fmaxf(v, 0.f) + log1pf(__expf(-fabsf(v))); }
 
 // sigmoid(z) through one ex2 and one reciprocal
 __device__ __forceinline__ float sigmoid_fast(float z) { return rcp_approx(1.0f + ex2_approx(-kLog2e * z)); }

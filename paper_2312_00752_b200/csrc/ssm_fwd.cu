@@ -56,12 +56,13 @@ __global__ void __launch_bounds__(fwd_threads(N)) ssm_fwd_kernel(const FwdParams
   const int d_thr = d_cta + slot * CPT;
   const int D = p.D;
 
-  float A2[CPT][S], h[CPT][S], dsum[CPT];
+  float A2[CPT][S], h[CPT][S], dsum[CPT], dbias[CPT];
 #pragma unroll
   for (int q = 0; q < CPT; ++q) {
     const int d = d_thr + q;
     const bool valid = d < D;
     dsum[q] = 0.f;
+    dbias[q] = (valid && p.delta_bias != nullptr) ? p.delta_bias[d] : 0.f;
 #pragma unroll
     for (int k = 0; k < S; ++k) {
       A2[q][k] = valid ? p.A[(size_t)d * N + j * S + k] * kLog2e : 0.f;
@@ -126,7 +127,8 @@ __global__ void __launch_bounds__(fwd_threads(N)) ssm_fwd_kernel(const FwdParams
       float y[CPT], u[CPT];
 #pragma unroll
       for (int q = 0; q < CPT; ++q) {
-        const float dt = io_to_float<IO>(s_d[tt][slot * CPT + q]);
+        float dt = io_to_float<IO>(s_d[tt][slot * CPT + q]) + dbias[q];
+        if (p.softplus) dt = softplus_precise(dt);
         u[q] = io_to_float<IO>(s_x[tt][slot * CPT + q]);
         const float du = dt * u[q];
         if (MODE == kFwdSummary) dsum[q] += dt;

@@ -1,0 +1,51 @@
+"""Step size through the fused softplus (Algorithm 2 step 4) on the GPU against the oracle, forward and backward."""
+import numpy as np
+import pytest
+
+from paper_2312_00752_b200 import synth
+from tests import _gpu_util as U
+
+pytestmark = pytest.mark.gpu
+
+
+def _pre_activation_case(batch, L, D, N, io, seed=0):
+    """Inputs of a workload with `delta` replaced by a pre-activation and a per-channel bias: the pre-activation is
+    the small noise term of the recipe (rounded to the io dtype), the bias is softplus^-1 of the per-channel target
+    step (float32), so that softplus(pre + bias) has the recipe's distribution."""
+    cfg = synth.ScanConfig("fused_dt", 13, batch, L, D, N, io, 1e-3, 1e-1)
+    inp = synth.make_inputs(cfg, seed=seed)
+    rng = np.random.default_rng(100 + seed)
+    tau = synth.channel_tau(cfg, seed)
+    bias = (tau + np.log(-np.expm1(-tau))).astype(np.float32)
+    pre = synth.round_to_io(0.1 * rng.standard_normal((batch, L, D)), io)
+    inp["delta"] = pre
+    return inp, bias
+
+
+@pytest.mark.parametrize("batch,L,D,N,io", [(2, 130, 40, 16, "bf16"), (1, 200, 24, 8, "f32"), (1, 4200, 32, 16, "f32")])
+@pytest.mark.parametrize("softplus", [True, False])
+def test_fused_step_size_forward_backward(batch, L, D, N, io, softplus):
+    import torch
+    from oracle import ssm_oracle as O
+    from paper_2312_00752_b200 import binding as K
+    inp, bias = _pre_activation_case(batch, L, D, N, io)
+    if not softplus:
+        bias = np.abs(bias) * 0.01 + 0.05          # keeps delta_pre + bias positive
+        inp["delta"] = synth.round_to_io(np.abs(inp["delta"]) * 0.1, io)
+    dev = U.to_device(inp, io)
+    dbias = torch.from_numpy(bias).cuda()
+    args = (dev["x"], dev["delta"], dbias, dev["A"], dev["B"], dev["C"], dev["D_skip"], dev["z"])
+    out, saved = K.ssm_scan_fwd_fused_dt(*args, softplus=softplus, save_states=True)
+    g = K.ssm_scan_bwd_fused_dt(*args, dev["dout"], saved, softplus=softplus)
+    ref_out = O.scan_fwd(inp["x"], inp["delta"], inp["A"], inp["B"], inp["C"], D_skip=inp["D_skip"], z=inp["z"],
+                         delta_softplus=softplus, delta_bias=bias)
+    ref = O.scan_bwd(inp["x"], inp["delta"], inp["A"], inp["B"], inp["C"], inp["D_skip"], inp["z"], inp["dout"],
+                     delta_softplus=softplus, delta_bias=bias)
+    tol = U.TOL[io]
+    assert U.rel_err(U.to_host(out), ref_out) <= tol["out"]
+    for k in ("dx", "ddelta", "ddelta_bias", "dz", "dB", "dC", "dA", "dD"):
+        assert U.rel_err(U.to_host(g[k]), ref[k]) <= tol["grad"], k
+    # without saved states the backward rebuilds the checkpoints with the same fused step size
+    g2 = K.ssm_scan_bwd_fused_dt(*args, dev["dout"], None, softplus=softplus)
+    for k in ("dx", "ddelta", "ddelta_bias", "dA"):
+        assert U.rel_err(U.to_host(g2[k]), ref[k]) <= tol["grad"], k
