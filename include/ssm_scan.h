@@ -134,7 +134,8 @@ SSM_API ssm_status_t ssm_scan_fwd_state(const ssm_problem_t* p, const void* x, c
  *     ddelta_pre   io_dtype [batch][L][D]: gradient of the pre-activation (ddelta * sigmoid(delta_pre + bias) with the
  *                  softplus),
  *     ddelta_bias  float32 [D], may be NULL: ddelta_pre summed over batch and time (fixed order).
- * These calls currently run the generic kernels for every shape (the tuned bf16 kernels take the step size as given).
+ * The forward call runs the tuned bf16 kernel where ssm_scan_fwd would; the backward call currently runs the generic
+ * kernels for every shape.
  */
 SSM_API ssm_status_t ssm_scan_fwd_fused_dt(const ssm_problem_t* p, const void* x, const void* delta_pre,
                                            const float* delta_bias, const float* A, const void* B, const void* C,

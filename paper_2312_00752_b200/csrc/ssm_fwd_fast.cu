@@ -12,6 +12,10 @@
 // applies the SiLU gate, rounds to bf16 and writes the output tile with 16-byte stores -- all while the compute warps
 // run the recurrence of the current tile.  The two roles meet at one block-wide barrier per tile.
 //
+// Step size.  With a bias and/or the softplus of Algorithm 2 step 4 fused in (template flag SP), every compute warp
+// turns the staged pre-activations of its own 16 channels into float step sizes, half a tile at a time and once per
+// element, in a strip of shared memory of its own; its lanes then read those instead of unpacking bf16.
+//
 // Discretization.  a = 2^(delta * A * log2 e) with the hardware ex2.  When the four A values of a thread form an
 // arithmetic progression (as in the S4D-Real initialisation A_n = -(n+1)) the four decays are built from two
 // exponentials, a_k = a_0 r^k with r = 2^(delta * step * log2 e); the test is made per warp at run time and can
@@ -26,21 +30,33 @@ namespace {
 
 constexpr int kTT = 32;    // steps per tile
 constexpr int kNST = 3;    // ring stages
+constexpr int kHalf = 16;  // steps whose fused step sizes a compute warp prepares at a time
 
-template <int WARPS, bool FULL>
+template <int WARPS, bool FULL, bool SP>
 struct FastSmem {
   static constexpr int CH = 16 * WARPS;
   uint32_t x[kNST][kTT][CH / 2];
   uint32_t d[kNST][kTT][CH / 2];
   uint32_t z[FULL ? kNST : 1][FULL ? kTT : 1][CH / 2];
-  uint32_t rawB[kNST][kTT][8];
-  uint32_t rawC[FULL ? kNST : 1][FULL ? kTT : 1][8];
+  uint32_t rawB[2][kTT][8];                        // widened one tile ahead: two stages
+  uint32_t rawC[FULL ? 2 : 1][FULL ? kTT : 1][8];
   float4 fB[2][kTT][4];
   float4 fC[FULL ? 2 : 1][FULL ? kTT : 1][4];
+  float dF[SP ? WARPS : 1][SP ? kHalf : 1][16];    // SP: step sizes after bias and softplus of half a tile, per warp
   float yp[FULL ? 2 : 1][FULL ? kTT : 1][CH];      // readout totals sum_n C h of a tile, per (step, channel)
   uint32_t o[FULL ? kTT : 1][CH / 2];              // output tile (bf16 pairs), owned by the service warp
   float Dsk[CH];                                   // D_skip of the block's channels
 };
+
+// softplus(v) = max(v, 0) + log1p(e^-|v|) for the tuned path: for small e = e^-|v| a short series (relative error
+// below 2e-7), otherwise the hardware logarithm (absolute error ~2e-7 on a value above 0.06)
+__device__ __forceinline__ float softplus_fast(float v) {
+  const float e = ex2_approx(-fabsf(v) * kLog2e);
+  const float series = e * fmaf(e, fmaf(e, fmaf(e, fmaf(e, 0.2f, -0.25f), 0.33333334f), -0.5f), 1.f);
+  float lg;
+  asm("lg2.approx.ftz.f32 %0, %1;" : "=f"(lg) : "f"(1.f + e));
+  return fmaxf(v, 0.f) + (e < 0.0625f ? series : lg * 0.6931471805599453f);
+}
 
 __device__ __forceinline__ void block_barrier(int nthreads) {
   asm volatile("bar.sync 1, %0;" ::"r"(nthreads) : "memory");
@@ -49,13 +65,13 @@ __device__ __forceinline__ void cp_async_wait_but_one() { asm volatile("cp.async
 
 }  // namespace
 
-template <int WARPS, int MODE>
+template <int WARPS, int MODE, bool SP>
 __global__ void __launch_bounds__((WARPS + 1) * 32) ssm_fwd_fast_kernel(const FwdParams p) {
   constexpr bool FULL = (MODE == kFwdFull);
   constexpr int THREADS = (WARPS + 1) * 32;
   constexpr int CH = 16 * WARPS;
   constexpr int CHUNKS = CH / 8;              // 16-byte chunks per tile row
-  using Smem = FastSmem<WARPS, FULL>;
+  using Smem = FastSmem<WARPS, FULL, SP>;
   extern __shared__ __align__(16) unsigned char smem_raw[];
   Smem& sm = *reinterpret_cast<Smem*>(smem_raw);
 
@@ -100,32 +116,31 @@ __global__ void __launch_bounds__((WARPS + 1) * 32) ssm_fwd_fast_kernel(const Fw
           const int tt = c >> 1, hc = c & 1;
           const bool ok = t0 + tt < t_end;
           const size_t g = ok ? (row0 + tt) * 16 + hc * 8 : 0;
-          cp_async16(&sm.rawB[st][tt][hc * 4], gB + g, ok);
-          if (FULL) cp_async16(&sm.rawC[st][tt][hc * 4], gC + g, ok);
+          cp_async16(&sm.rawB[i & 1][tt][hc * 4], gB + g, ok);
+          if (FULL) cp_async16(&sm.rawC[i & 1][tt][hc * 4], gC + g, ok);
         }
       }
       cp_async_commit();
     };
     auto widen_BC = [&](int i) {  // tile i: bf16 -> float
       if (i >= ntiles) return;
-      const int st = i % kNST, fb = i & 1;
+      const int fb = i & 1;
 #pragma unroll
       for (int k = 0; k < kTT * 8 / 32; ++k) {
         const int c = lane + 32 * k;
         const int tt = c >> 3, w = c & 7;
-        const uint32_t vb = sm.rawB[st][tt][w];
+        const uint32_t vb = sm.rawB[fb][tt][w];
         reinterpret_cast<float2*>(&sm.fB[fb][tt][0])[w] = make_float2(bf16lo(vb), bf16hi(vb));
         if (FULL) {
-          const uint32_t vc = sm.rawC[st][tt][w];
+          const uint32_t vc = sm.rawC[fb][tt][w];
           reinterpret_cast<float2*>(&sm.fC[fb][tt][0])[w] = make_float2(bf16lo(vc), bf16hi(vc));
         }
       }
     };
     // skip term, gate and rounding of tile i (its readout totals are complete), then the 16-byte stores
-    if (FULL) {
-      for (int c = lane; c < CH; c += 32) sm.Dsk[c] = (p.Dskip != nullptr && d_cta + c < D) ? p.Dskip[d_cta + c] : 0.f;
-      __syncwarp();
-    }
+    for (int c = lane; c < CH; c += 32)
+      if (FULL) sm.Dsk[c] = (p.Dskip != nullptr && d_cta + c < D) ? p.Dskip[d_cta + c] : 0.f;
+    __syncwarp();
     auto finish_tile = [&](int i) {
       if (!FULL) return;
       const int st = i % kNST, yb = i & 1;
@@ -211,6 +226,15 @@ __global__ void __launch_bounds__((WARPS + 1) * 32) ssm_fwd_fast_kernel(const Fw
     h[q][1] = make_float2(hs.z, hs.w);
   }
   ap = __all_sync(0xffffffffu, ap);
+  // SP: in the step-size stage below a lane always handles channel pair (lane % 8) of its warp
+  float bias0 = 0.f, bias1 = 0.f;
+  if (SP && p.delta_bias != nullptr) {
+    const int c = d_cta + warp * 16 + 2 * (lane & 7);
+    if (c < D) {
+      bias0 = p.delta_bias[c];
+      bias1 = p.delta_bias[c + 1];
+    }
+  }
 
 
   // One tile of kTT steps, in sub-blocks of 4 steps: the loads of the next sub-block are issued before the
@@ -230,11 +254,32 @@ __global__ void __launch_bounds__((WARPS + 1) * 32) ssm_fwd_fast_kernel(const Fw
       }
     }
     uint32_t dw[SB], xw[SB];
+    float2 dfv[SB];   // SP: the step sizes of the channel pair, float
     float4 Bq[SB], Cq[SB];
+    // SP: step sizes of steps [half * kHalf, +kHalf) of this warp's 16 channels: bf16 pre-activation + bias, softplus,
+    // float, into the warp's own strip (4 pairs per lane); rows past the end of the segment stay identity steps
+    auto prepare_dt = [&](int half) {
+      __syncwarp();
+#pragma unroll
+      for (int k = 0; k < kHalf / 4; ++k) {
+        const int tt = (lane >> 3) + 4 * k, sl = lane & 7;
+        const uint32_t w = sm.d[st][half * kHalf + tt][warp * 8 + sl];
+        float v0 = bf16lo(w) + bias0, v1 = bf16hi(w) + bias1;
+        if (p.softplus) {
+          v0 = softplus_fast(v0);
+          v1 = softplus_fast(v1);
+        }
+        const bool live = t_begin + i * kTT + half * kHalf + tt < t_end;
+        *reinterpret_cast<float2*>(&sm.dF[warp][tt][2 * sl]) = live ? make_float2(v0, v1) : make_float2(0.f, 0.f);
+      }
+      __syncwarp();
+    };
     auto load_sb = [&](int tb) {
+      if (SP && tb % kHalf == 0) prepare_dt(tb / kHalf);
 #pragma unroll
       for (int t = 0; t < SB; ++t) {
-        dw[t] = sm.d[st][tb + t][slot];
+        if (SP) dfv[t] = *reinterpret_cast<const float2*>(&sm.dF[warp][(tb + t) % kHalf][2 * (lane >> 2)]);
+        else dw[t] = sm.d[st][tb + t][slot];
         xw[t] = sm.x[st][tb + t][slot];
         Bq[t] = sm.fB[fb][tb + t][j];
         if (FULL) Cq[t] = sm.fC[fb][tb + t][j];
@@ -248,7 +293,8 @@ __global__ void __launch_bounds__((WARPS + 1) * 32) ssm_fwd_fast_kernel(const Fw
 #pragma unroll
       for (int t = 0; t < SB; ++t) {
         // q = 0 is this lane's kept channel (channel pq of the pair), q = 1 the one it hands to its neighbour
-        const float dt[2] = {__uint_as_float(__byte_perm(dw[t], 0, selA)), __uint_as_float(__byte_perm(dw[t], 0, selB))};
+        const float dt[2] = {SP ? (pq ? dfv[t].y : dfv[t].x) : __uint_as_float(__byte_perm(dw[t], 0, selA)),
+                             SP ? (pq ? dfv[t].x : dfv[t].y) : __uint_as_float(__byte_perm(dw[t], 0, selB))};
         const float u[2] = {__uint_as_float(__byte_perm(xw[t], 0, selA)), __uint_as_float(__byte_perm(xw[t], 0, selB))};
         const float2 du = f2mul(make_float2(dt[0], dt[1]), make_float2(u[0], u[1]));
         const float duq[2] = {du.x, du.y};
@@ -334,23 +380,29 @@ __global__ void __launch_bounds__((WARPS + 1) * 32) ssm_fwd_fast_kernel(const Fw
   }
 }
 
-template <int WARPS, int MODE>
-static cudaError_t launch_fast(const Plan& plan, const FwdParams& p, cudaStream_t s) {
-  constexpr size_t smem = sizeof(FastSmem<WARPS, MODE == kFwdFull>);
+template <int WARPS, int MODE, bool SP>
+static cudaError_t launch_fast_sp(const Plan& plan, const FwdParams& p, cudaStream_t s) {
+  constexpr size_t smem = sizeof(FastSmem<WARPS, MODE == kFwdFull, SP>);
   constexpr int CH = 16 * WARPS;
   if (smem > 48 * 1024) {
-    cudaError_t e = cudaFuncSetAttribute(ssm_fwd_fast_kernel<WARPS, MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         (int)smem);
+    cudaError_t e = cudaFuncSetAttribute(ssm_fwd_fast_kernel<WARPS, MODE, SP>,
+                                         cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
   }
   dim3 grid((p.D + CH - 1) / CH, plan.nseg, p.batch);
-  ssm_fwd_fast_kernel<WARPS, MODE><<<grid, (WARPS + 1) * 32, smem, s>>>(p);
+  ssm_fwd_fast_kernel<WARPS, MODE, SP><<<grid, (WARPS + 1) * 32, smem, s>>>(p);
   return cudaGetLastError();
+}
+
+// SP: the step size goes through the bias / softplus stage of the service warp
+template <int WARPS, int MODE>
+static cudaError_t launch_fast(const Plan& plan, const FwdParams& p, cudaStream_t s) {
+  if (p.softplus || p.delta_bias != nullptr) return launch_fast_sp<WARPS, MODE, true>(plan, p, s);
+  return launch_fast_sp<WARPS, MODE, false>(plan, p, s);
 }
 
 bool fwd_fast_applicable(const ssm_problem_t& prob, const FwdParams& p) {
   auto al16 = [](const void* q) { return q == nullptr || (reinterpret_cast<uintptr_t>(q) & 15) == 0; };
-  if (p.softplus || p.delta_bias != nullptr) return false;  // the tuned kernel takes the step size as given
   return prob.io_dtype == SSM_BF16 && prob.N == 16 && prob.D % 8 == 0 && al16(p.x) && al16(p.delta) && al16(p.z) &&
          al16(p.B) && al16(p.C) && al16(p.out) && al16(p.A) && al16(p.h_start) && al16(p.ckpt) && al16(p.seg_end) && al16(p.h_last);
 }
