@@ -134,8 +134,7 @@ SSM_API ssm_status_t ssm_scan_fwd_state(const ssm_problem_t* p, const void* x, c
  *     ddelta_pre   io_dtype [batch][L][D]: gradient of the pre-activation (ddelta * sigmoid(delta_pre + bias) with the
  *                  softplus),
  *     ddelta_bias  float32 [D], may be NULL: ddelta_pre summed over batch and time (fixed order).
- * The forward call runs the tuned bf16 kernel where ssm_scan_fwd would; the backward call currently runs the generic
- * kernels for every shape.
+ * Both calls run the tuned bf16 kernels wherever ssm_scan_fwd / ssm_scan_bwd would.
  */
 SSM_API ssm_status_t ssm_scan_fwd_fused_dt(const ssm_problem_t* p, const void* x, const void* delta_pre,
                                            const float* delta_bias, const float* A, const void* B, const void* C,

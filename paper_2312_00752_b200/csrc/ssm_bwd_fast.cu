@@ -51,7 +51,7 @@ struct BwdFastSmem {
   float4 fB[kBT][4];
   float4 fC[kBT][4];
   float ds[kBT][kBwdFastCH];            // dout * silu(z)
-  float gsp[kBT][kBwdFastCH];           // dout * silu'(z)
+  float gsp[kBT][kBwdFastCH];           // dout * silu'(z); with the fused step size: the step size itself, float
   float4 red[kBwdFastWarps][kRB][8][4][2];   // [warp][step][quad][lane in quad][dB quad | dC quad]
   float acc[kBwdFastWarps][kBT][32];    // per-warp sums over its 16 channels: [step][dB 0..15 | dC 0..15]
   int sched[4];                         // [0] current item, [1] next item, [2] abort
@@ -70,6 +70,7 @@ __device__ __forceinline__ void st_release(int* p, int v) {
 
 }  // namespace
 
+template <bool SP>
 __global__ void __launch_bounds__(kBwdFastThreads) ssm_bwd_fast_kernel(const BwdParams p) {
   constexpr int THREADS = kBwdFastThreads;
   constexpr int CH = kBwdFastCH;
@@ -153,6 +154,7 @@ __global__ void __launch_bounds__(kBwdFastThreads) ssm_bwd_fast_kernel(const Bwd
   // ---- state of the chain being processed (set per item)
   float2 A2[2][2], mu[2][2], dA2[2][2];
   float Dk = 0.f, dD_acc = 0.f;
+  float bias_pq = 0.f, dbias_acc = 0.f;   // SP: bias of the kept channel, sum of the pre-activation gradient
   int d0 = 0;
   bool valid = false;
   auto chan = [&](int q) { return d0 + (q ^ pq); };
@@ -172,6 +174,16 @@ __global__ void __launch_bounds__(kBwdFastThreads) ssm_bwd_fast_kernel(const Bwd
     }
   };
 
+  // step sizes of the lane's channel pair at tile row tt as (kept channel, handed channel)
+  auto step_sizes = [&](int st, int tt, uint32_t dw) {
+    if (SP) {
+      const float2 f = *reinterpret_cast<const float2*>(&sm.gsp[tt][2 * slot]);
+      return pq ? make_float2(f.y, f.x) : f;
+    }
+    (void)st;
+    return make_float2(bf16sel(dw, selA), bf16sel(dw, selB));
+  };
+
   auto process_tile = [&](int st, auto ap_tag, const float4 (&ck)[2]) {
     // ---- level 1: states at the sub-block boundaries (steps 0, 8, 16, 24 of the tile), parked in shared memory
     {
@@ -186,9 +198,9 @@ __global__ void __launch_bounds__(kBwdFastThreads) ssm_bwd_fast_kernel(const Bwd
 #pragma unroll
       for (int t = 0; t < kSB; ++t) {
         const int tt = sb * kSB + t;
-        const uint32_t dw = sm.d[st][tt][slot], xw = sm.x[st][tt][slot];
+        const uint32_t dw = SP ? 0u : sm.d[st][tt][slot], xw = sm.x[st][tt][slot];
         const float4 Bq = sm.fB[tt][j];
-        const float2 dt2 = make_float2(bf16sel(dw, selA), bf16sel(dw, selB));
+        const float2 dt2 = step_sizes(st, tt, dw);
         const float2 du = f2mul(dt2, make_float2(bf16sel(xw, selA), bf16sel(xw, selB)));
         const float dtq[2] = {dt2.x, dt2.y}, duq[2] = {du.x, du.y};
 #pragma unroll
@@ -221,10 +233,10 @@ __global__ void __launch_bounds__(kBwdFastThreads) ssm_bwd_fast_kernel(const Bwd
 #pragma unroll
         for (int t = 0; t < kSB; ++t) {
           const int tt = sb * kSB + t;
-          dwk[t] = sm.d[st][tt][slot];
+          dwk[t] = SP ? 0u : sm.d[st][tt][slot];
           xwk[t] = sm.x[st][tt][slot];
           const float4 Bq = sm.fB[tt][j], Cq = sm.fC[tt][j];
-          const float2 dt2 = make_float2(bf16sel(dwk[t], selA), bf16sel(dwk[t], selB));
+          const float2 dt2 = step_sizes(st, tt, dwk[t]);
           const float2 du = f2mul(dt2, make_float2(bf16sel(xwk[t], selA), bf16sel(xwk[t], selB)));
           const float dtq[2] = {dt2.x, dt2.y}, duq[2] = {du.x, du.y};
           float y[2];
@@ -248,7 +260,7 @@ __global__ void __launch_bounds__(kBwdFastThreads) ssm_bwd_fast_kernel(const Bwd
       for (int t = kSB - 1; t >= 0; --t) {
         const int tt = sb * kSB + t;
         const float4 Bq = sm.fB[tt][j], Cq = sm.fC[tt][j];
-        const float2 dt2 = make_float2(bf16sel(dwk[t], selA), bf16sel(dwk[t], selB));
+        const float2 dt2 = step_sizes(st, tt, dwk[t]);
         const float2 u2 = make_float2(bf16sel(xwk[t], selA), bf16sel(xwk[t], selB));
         const float2 du = f2mul(dt2, u2);
         const float dtq[2] = {dt2.x, dt2.y}, uq[2] = {u2.x, u2.y}, duq[2] = {du.x, du.y};
@@ -327,8 +339,24 @@ __global__ void __launch_bounds__(kBwdFastThreads) ssm_bwd_fast_kernel(const Bwd
         const float s = fmaf(Dk, u, ytot[e]);
         dD_acc = fmaf(ds, u, dD_acc);
         reinterpret_cast<__nv_bfloat16*>(&sm.x[st][tt][slot])[pq] = __float2bfloat16_rn(fmaf(ds, Dk, dxtot[e]));
-        reinterpret_cast<__nv_bfloat16*>(&sm.d[st][tt][slot])[pq] = __float2bfloat16_rn(ddtot[e]);
-        reinterpret_cast<__nv_bfloat16*>(&sm.z[st][tt][slot])[pq] = __float2bfloat16_rn(sm.gsp[tt][2 * slot + pq] * s);
+        float ddv = ddtot[e], gsp;
+        if (SP) {
+          // the gate derivative is rebuilt here (its array holds the step sizes); the gradient goes to the
+          // pre-activation v: d softplus(v) / dv = sigmoid(v)
+          const float gf = __uint_as_float((uint32_t)reinterpret_cast<const uint16_t*>(&sm.g[st][tt][slot])[pq] << 16);
+          const float zf = __uint_as_float((uint32_t)reinterpret_cast<const uint16_t*>(&sm.z[st][tt][slot])[pq] << 16);
+          const float sg = sigmoid_fast(zf);
+          gsp = has_z ? gf * sg * fmaf(zf, 1.f - sg, 1.f) : 0.f;
+          if (p.softplus) {
+            const float v = __uint_as_float((uint32_t)reinterpret_cast<const uint16_t*>(&sm.d[st][tt][slot])[pq] << 16) + bias_pq;
+            ddv *= sigmoid_fast(v);
+          }
+          dbias_acc += ddv;
+        } else {
+          gsp = sm.gsp[tt][2 * slot + pq];
+        }
+        reinterpret_cast<__nv_bfloat16*>(&sm.d[st][tt][slot])[pq] = __float2bfloat16_rn(ddv);
+        reinterpret_cast<__nv_bfloat16*>(&sm.z[st][tt][slot])[pq] = __float2bfloat16_rn(gsp * s);
       }
     }
   };
@@ -366,6 +394,7 @@ __global__ void __launch_bounds__(kBwdFastThreads) ssm_bwd_fast_kernel(const Bwd
         A2[q][1] = make_float2(a.z * kLog2e, a.w * kLog2e);
       }
       Dk = (valid && p.Dskip != nullptr) ? p.Dskip[d0 + pq] : 0.f;
+      if (SP) bias_pq = (valid && p.delta_bias != nullptr) ? p.delta_bias[d0 + pq] : 0.f;
       // carried values: from the segment's inflow for the first tile in order, else from the tile before in order
       if (cur.ord == 0) {
 #pragma unroll
@@ -378,6 +407,7 @@ __global__ void __launch_bounds__(kBwdFastThreads) ssm_bwd_fast_kernel(const Bwd
           dA2[q][0] = dA2[q][1] = make_float2(0.f, 0.f);
         }
         dD_acc = 0.f;
+        dbias_acc = 0.f;
       } else {
         if (tid == 0) {
           int spins = 0;
@@ -410,6 +440,7 @@ __global__ void __launch_bounds__(kBwdFastThreads) ssm_bwd_fast_kernel(const Bwd
         dA2[0][0] = make_float2(a0.x, a0.y); dA2[0][1] = make_float2(a0.z, a0.w);
         dA2[1][0] = make_float2(a1.x, a1.y); dA2[1][1] = make_float2(a1.z, a1.w);
         dD_acc = dd.x;
+        if (SP) dbias_acc = dd.y;
       }
       const size_t row0 = (size_t)cur.b * p.L + cur.t0;
       // widen B, C; per-element gate terms ds = dout * silu(z), gsp = dout * silu'(z)
@@ -434,6 +465,18 @@ __global__ void __launch_bounds__(kBwdFastThreads) ssm_bwd_fast_kernel(const Bwd
           gpv = make_float2(0.f, 0.f);
         }
         *reinterpret_cast<float2*>(&sm.ds[tt][2 * w]) = dsv;
+        if (SP) {
+          // step size of Algorithm 2 step 4 from the pre-activation; rows past the end stay identity steps
+          const uint32_t dw = sm.d[st][tt][w];
+          const int c0 = cur.d_cta + 2 * w;
+          const bool chan_ok = c0 < D && p.delta_bias != nullptr;
+          float v0 = bf16lo(dw) + (chan_ok ? p.delta_bias[c0] : 0.f), v1 = bf16hi(dw) + (chan_ok ? p.delta_bias[c0 + 1] : 0.f);
+          if (p.softplus) {
+            v0 = softplus_fast(v0);
+            v1 = softplus_fast(v1);
+          }
+          gpv = (cur.t0 + tt < cur.t_end) ? make_float2(v0, v1) : make_float2(0.f, 0.f);
+        }
         *reinterpret_cast<float2*>(&sm.gsp[tt][2 * w]) = gpv;
       }
       __syncthreads();
@@ -471,7 +514,7 @@ __global__ void __launch_bounds__(kBwdFastThreads) ssm_bwd_fast_kernel(const Bwd
         __stcg(hb + 1, make_float4(mu[1][0].x, mu[1][0].y, mu[1][1].x, mu[1][1].y));
         __stcg(hb + 2, make_float4(dA2[0][0].x, dA2[0][0].y, dA2[0][1].x, dA2[0][1].y));
         __stcg(hb + 3, make_float4(dA2[1][0].x, dA2[1][0].y, dA2[1][1].x, dA2[1][1].y));
-        __stcg(hb + 4, make_float4(dD_acc, 0.f, 0.f, 0.f));
+        __stcg(hb + 4, make_float4(dD_acc, SP ? dbias_acc : 0.f, 0.f, 0.f));
         __threadfence();
         __syncthreads();
         if (tid == 0 && !p.test_withhold) st_release(sched_flags + cur.chain, cur.ord + 1);
@@ -487,6 +530,11 @@ __global__ void __launch_bounds__(kBwdFastThreads) ssm_bwd_fast_kernel(const Bwd
         // dD: lanes j and j^2 accumulated disjoint steps of the same channel
         const float dsum2 = dD_acc + __shfl_xor_sync(0xffffffffu, dD_acc, 2);
         if (valid && j < 2) p.dD_part[((size_t)cur.b * p.nseg + cur.seg) * D + d0 + pq] = dsum2;
+        if (SP) {
+          const float bsum2 = dbias_acc + __shfl_xor_sync(0xffffffffu, dbias_acc, 2);
+          if (valid && j < 2 && p.dbias_part != nullptr)
+            p.dbias_part[((size_t)cur.b * p.nseg + cur.seg) * D + d0 + pq] = bsum2;
+        }
       }
     }
     cur = nxt;
@@ -497,7 +545,6 @@ __global__ void __launch_bounds__(kBwdFastThreads) ssm_bwd_fast_kernel(const Bwd
 
 bool bwd_fast_applicable(const ssm_problem_t& prob, const BwdParams& p) {
   auto al16 = [](const void* q) { return q == nullptr || (reinterpret_cast<uintptr_t>(q) & 15) == 0; };
-  if (p.softplus || p.delta_bias != nullptr) return false;  // the tuned kernel takes the step size as given
   return prob.io_dtype == SSM_BF16 && prob.N == 16 && prob.D % 8 == 0 && p.seg_steps % kBT == 0 && al16(p.x) &&
          al16(p.delta) && al16(p.z) && al16(p.B) && al16(p.C) && al16(p.dout) && al16(p.dx) && al16(p.ddelta) &&
          al16(p.dz) && al16(p.A) && al16(p.ckpt) && al16(p.mu_in) && al16(p.dBC_part) && al16(p.dA_part) &&
@@ -507,14 +554,15 @@ bool bwd_fast_applicable(const ssm_problem_t& prob, const BwdParams& p) {
 int bwd_fast_channels_per_block() { return kBwdFastCH; }
 size_t bwd_fast_handoff_bytes_per_chain() { return sizeof(float4) * kHandoffVec * kBwdFastThreads; }
 
-cudaError_t launch_bwd_fast(const Plan& plan, const BwdParams& p, cudaStream_t s) {
+template <bool SP>
+static cudaError_t launch_bwd_fast_sp(const Plan& plan, const BwdParams& p, cudaStream_t s) {
   constexpr size_t smem = sizeof(BwdFastSmem);
-  cudaError_t e = cudaFuncSetAttribute(ssm_bwd_fast_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  cudaError_t e = cudaFuncSetAttribute(ssm_bwd_fast_kernel<SP>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
   int dev = 0, sms = 0, per_sm = 0;
   if ((e = cudaGetDevice(&dev)) != cudaSuccess) return e;
   if ((e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
-  if ((e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, ssm_bwd_fast_kernel, kBwdFastThreads, smem)) != cudaSuccess)
+  if ((e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, ssm_bwd_fast_kernel<SP>, kBwdFastThreads, smem)) != cudaSuccess)
     return e;
   const int groups = (p.D + kBwdFastCH - 1) / kBwdFastCH;
   const long long chains = (long long)p.batch * plan.nseg * groups;
@@ -522,8 +570,14 @@ cudaError_t launch_bwd_fast(const Plan& plan, const BwdParams& p, cudaStream_t s
   const long long resident = (long long)sms * (per_sm > 0 ? per_sm : 1);
   const unsigned grid = (unsigned)(items < resident ? items : resident);
   // the claim counter, the abort word and the flag of every chain were zeroed by the caller (ssm_scan_bwd)
-  ssm_bwd_fast_kernel<<<grid, kBwdFastThreads, smem, s>>>(p);
+  ssm_bwd_fast_kernel<SP><<<grid, kBwdFastThreads, smem, s>>>(p);
   return cudaGetLastError();
+}
+
+// SP: the step size is bias + pre-activation, through the softplus if asked (Algorithm 2 step 4)
+cudaError_t launch_bwd_fast(const Plan& plan, const BwdParams& p, cudaStream_t s) {
+  if (p.softplus || p.delta_bias != nullptr) return launch_bwd_fast_sp<true>(plan, p, s);
+  return launch_bwd_fast_sp<false>(plan, p, s);
 }
 
 }  // namespace ssm

@@ -171,6 +171,16 @@ __device__ __forceinline__ float2 f2mul(float2 a, float2 b) { return __fmul2_rn(
 __device__ __forceinline__ float2 f2fma(float2 a, float2 b, float2 c) { return __ffma2_rn(a, b, c); }
 __device__ __forceinline__ float2 f2dup(float v) { return make_float2(v, v); }
 
+// softplus(v) = max(v, 0) + log1p(e^-|v|) for the tuned path: for small e = e^-|v| a short series (relative error
+// below 2e-7), otherwise the hardware logarithm (absolute error ~2e-7 on a value above 0.06)
+__device__ __forceinline__ float softplus_fast(float v) {
+  const float e = ex2_approx(-fabsf(v) * kLog2e);
+  const float series = e * fmaf(e, fmaf(e, fmaf(e, fmaf(e, 0.2f, -0.25f), 0.33333334f), -0.5f), 1.f);
+  float lg;
+  asm("lg2.approx.ftz.f32 %0, %1;" : "=f"(lg) : "f"(1.f + e));
+  return fmaxf(v, 0.f) + (e < 0.0625f ? series : lg * 0.6931471805599453f);
+}
+
 // softplus(v) = log(1 + e^v) = max(v, 0) + log1p(e^-|v|) with the precise library log1p (generic kernels)
 __device__ __forceinline__ float softplus_precise(float v) { return fmaxf(v, 0.f) + log1pf(__expf(-fabsf(v))); }
 

@@ -48,16 +48,6 @@ struct FastSmem {
   float Dsk[CH];                                   // D_skip of the block's channels
 };
 
-// softplus(v) = max(v, 0) + log1p(e^-|v|) for the tuned path: for small e = e^-|v| a short series (relative error
-// below 2e-7), otherwise the hardware logarithm (absolute error ~2e-7 on a value above 0.06)
-__device__ __forceinline__ float softplus_fast(float v) {
-  const float e = ex2_approx(-fabsf(v) * kLog2e);
-  const float series = e * fmaf(e, fmaf(e, fmaf(e, fmaf(e, 0.2f, -0.25f), 0.33333334f), -0.5f), 1.f);
-  float lg;
-  asm("lg2.approx.ftz.f32 %0, %1;" : "=f"(lg) : "f"(1.f + e));
-  return fmaxf(v, 0.f) + (e < 0.0625f ? series : lg * 0.6931471805599453f);
-}
-
 __device__ __forceinline__ void block_barrier(int nthreads) {
   asm volatile("bar.sync 1, %0;" ::"r"(nthreads) : "memory");
 }

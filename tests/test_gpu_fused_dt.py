@@ -22,7 +22,8 @@ def _pre_activation_case(batch, L, D, N, io, seed=0):
     return inp, bias
 
 
-@pytest.mark.parametrize("batch,L,D,N,io", [(2, 130, 40, 16, "bf16"), (1, 200, 24, 8, "f32"), (1, 4200, 32, 16, "f32")])
+@pytest.mark.parametrize("batch,L,D,N,io", [(2, 130, 40, 16, "bf16"), (1, 200, 24, 8, "f32"), (1, 4200, 32, 16, "f32"), (1, 4200, 48, 16, "bf16"),
+                                           (3, 1000, 328, 16, "bf16")])
 @pytest.mark.parametrize("softplus", [True, False])
 def test_fused_step_size_forward_backward(batch, L, D, N, io, softplus):
     import torch
