@@ -25,6 +25,10 @@
  *   dC[t,n] += ds[t] h[t,n];   dD += ds[t] x[t];   dB[t,n] += lam[t,n] delta[t] x[t]
  *   dx[t]   = ds[t] D_skip + delta[t] sum_n lam[t,n] B[t,n]
  *   w[t,n]  = lam[t,n] h[t-1,n] a[t,n];   ddelta[t] = sum_n w[t,n] A[n] + x[t] sum_n lam[t,n] B[t,n];   dA[n] += w[t,n] delta[t]
+ * With the ZOH rule write bbar = E B with the input gain E(delta, A) = (exp(delta A) - 1) / A (E = delta at A = 0),
+ * whose partial derivatives are dE/ddelta = a and dE/dA = (delta a - E) / A (delta^2 / 2 at A = 0).  Then
+ *   dB[t,n] += lam E x;   dx[t] = ds D_skip + sum_n lam E B;
+ *   ddelta[t] = sum_n w A + x sum_n lam a B;   dA[n] += w delta + lam (dE/dA) B x.
  * With the softplus switch the input is the pre-activation v, delta = softplus(v + delta_bias[d]), ddelta is the
  * gradient of v (the line above times sigmoid(v + delta_bias[d])) and dbias[d] = sum over batch and time of ddelta.
  * Sums over channels (dB, dC) and over batch (dA, dD) are taken in a fixed order that does not depend on the
@@ -48,7 +52,7 @@ typedef struct {
   int32_t batch, L, D, N;
   int32_t has_z;      /* 0: out = s (no gate) */
   int32_t has_dskip;  /* 0: skip term absent */
-  int32_t zoh_bbar;   /* 1: zero-order-hold B-bar of Eq. 4 (forward only; used by the gating-theorem pin) */
+  int32_t zoh_bbar;   /* 1: zero-order-hold B-bar of Eq. 4 instead of delta * B */
   int32_t softplus;   /* 1: `delta` holds the pre-activation v and the step size is softplus(v + delta_bias[d])
                          (Algorithm 2 step 4: Delta = tau_Delta(Parameter + s_Delta(x)), tau_Delta = softplus) */
   int32_t nthreads;   /* <= 0: all available */
@@ -75,6 +79,14 @@ static inline double silu(double z) { return z / (1.0 + exp(-z)); }
 static inline double sigmoid(double z) { return 1.0 / (1.0 + exp(-z)); }
 /* softplus(v) = log(1 + e^v), written so that neither large nor very negative v loses accuracy */
 static inline double softplus(double v) { return (v > 0.0 ? v : 0.0) + log1p(exp(-fabs(v))); }
+/* input gain of the ZOH rule (Eq. 4 for diagonal A): E = (exp(dt A) - 1) / A, and its derivative in A */
+static inline double zoh_gain(double dt, double An) { return An != 0.0 ? expm1(dt * An) / An : dt; }
+static inline double zoh_gain_dA(double dt, double An) {
+  const double xx = dt * An;
+  if (fabs(xx) < 1e-3) /* (x e^x - e^x + 1) / x^2 = 1/2 + x/3 + x^2/8 + x^3/30 + ... : no cancellation near 0 */
+    return dt * dt * (0.5 + xx * (1.0 / 3.0 + xx * (0.125 + xx * (1.0 / 30.0 + xx / 144.0))));
+  return (dt * exp(xx) - expm1(xx) / An) / An;
+}
 
 /* ------------------------------------------------------------------------------------------------------------
  * The two entry-point families differ only in the storage type of the (batch, L, *) inputs.
@@ -106,7 +118,7 @@ static inline double softplus(double v) { return (v > 0.0 ? v : 0.0) + log1p(exp
           const double An = A[d * N + n];                                                                        \
           const double a = exp(dt * An);                                                                         \
           double bbar;                                                                                           \
-          if (p->zoh_bbar) bbar = (An != 0.0 ? (a - 1.0) / An : dt) * (double)Bt[n];                             \
+          if (p->zoh_bbar) bbar = zoh_gain(dt, An) * (double)Bt[n];                                              \
           else             bbar = dt * (double)Bt[n];                                                            \
           h[n] = a * h[n] + bbar * u;                                                                            \
           s += (double)Ct[n] * h[n];                                                                             \
@@ -125,7 +137,7 @@ static inline double softplus(double v) { return (v > 0.0 ? v : 0.0) + log1p(exp
                               const REAL* B, const REAL* C, const double* D_skip, const REAL* z,                 \
                               const REAL* dout, const double* delta_bias, double* dx, double* ddelta,           \
                               double* dA, double* dB, double* dC, double* dD, double* dz, double* dbias) {       \
-    if (!p || p->batch < 1 || p->L < 1 || p->D < 1 || p->N < 1 || p->zoh_bbar) return 1;                          \
+    if (!p || p->batch < 1 || p->L < 1 || p->D < 1 || p->N < 1) return 1;                                         \
     const int64_t L = p->L, D = p->D, N = p->N, NB = p->batch;                                                   \
     const int64_t nblk = (D + ORACLE_CH_BLOCK - 1) / ORACLE_CH_BLOCK;                                            \
     const int64_t items = NB * nblk;                                                                             \
@@ -159,7 +171,8 @@ static inline double softplus(double v) { return (v > 0.0 ? v : 0.0) + log1p(exp
             for (int64_t n = 0; n < N; ++n) {                                                                    \
               const double a = exp(dt * A[d * N + n]);                                                           \
               as[t * N + n] = a;                                                                                 \
-              hs[t * N + n] = a * hs[(t - 1) * N + n] + dt * (double)Bt[n] * u;                                  \
+              const double E = p->zoh_bbar ? zoh_gain(dt, A[d * N + n]) : dt;                                    \
+              hs[t * N + n] = a * hs[(t - 1) * N + n] + E * (double)Bt[n] * u;                                   \
               s += (double)Ct[n] * hs[t * N + n];                                                                \
             }                                                                                                    \
             if (p->has_dskip) s += D_skip[d] * u;                                                                \
@@ -182,21 +195,27 @@ static inline double softplus(double v) { return (v > 0.0 ? v : 0.0) + log1p(exp
               ds = g;                                                                                            \
               if (dz) dz[e] = 0.0;                                                                               \
             }                                                                                                    \
-            double lamB = 0.0, wA = 0.0;                                                                         \
+            /* lamEB = sum lam E B (input gradient), lamGB = sum lam (dE/ddelta) B (step-size gradient) */     \
+            double lamEB = 0.0, lamGB = 0.0, wA = 0.0;                                                           \
             for (int64_t n = 0; n < N; ++n) {                                                                    \
               /* lam currently holds a[t+1] * lam[t+1] (zero for t = L) */                                       \
               const double l = (double)Ct[n] * ds + lam[n];                                                      \
+              const double An = A[d * N + n], a = as[t * N + n];                                                 \
+              const double E = p->zoh_bbar ? zoh_gain(dt, An) : dt;                                              \
+              const double dE_ddt = p->zoh_bbar ? a : 1.0;                                                       \
+              const double dE_dA = p->zoh_bbar ? zoh_gain_dA(dt, An) : 0.0;                                      \
               dCp[(t - 1) * N + n] += ds * hs[t * N + n];                                                        \
-              dBp[(t - 1) * N + n] += l * dt * u;                                                                \
-              lamB += l * (double)Bt[n];                                                                         \
-              const double w = l * hs[(t - 1) * N + n] * as[t * N + n];                                          \
-              wA += w * A[d * N + n];                                                                            \
-              dA_part[(b * D + d) * N + n] += w * dt;                                                            \
-              lam[n] = as[t * N + n] * l;                                                                        \
+              dBp[(t - 1) * N + n] += l * E * u;                                                                 \
+              lamEB += l * E * (double)Bt[n];                                                                    \
+              lamGB += l * dE_ddt * (double)Bt[n];                                                               \
+              const double w = l * hs[(t - 1) * N + n] * a;                                                      \
+              wA += w * An;                                                                                      \
+              dA_part[(b * D + d) * N + n] += w * dt + l * dE_dA * (double)Bt[n] * u;                            \
+              lam[n] = a * l;                                                                                    \
             }                                                                                                    \
-            dx[e] = (p->has_dskip ? ds * D_skip[d] : 0.0) + dt * lamB;                                           \
+            dx[e] = (p->has_dskip ? ds * D_skip[d] : 0.0) + lamEB;                                               \
             /* with the softplus, ddelta is the gradient of the pre-activation: d softplus(v)/dv = sigmoid(v) */ \
-            ddelta[e] = (wA + u * lamB) * (p->softplus ? sigmoid(dv) : 1.0);                                     \
+            ddelta[e] = (wA + u * lamGB) * (p->softplus ? sigmoid(dv) : 1.0);                                    \
             dbias_acc += ddelta[e];                                                                              \
             dD_acc += ds * u;                                                                                    \
           }                                                                                                      \

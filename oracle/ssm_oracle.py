@@ -106,12 +106,13 @@ def scan_fwd(x, delta, A, B, C, D_skip=None, z=None, h0=None, zoh=False, nthread
     return res[0] if len(res) == 1 else res
 
 
-def scan_bwd(x, delta, A, B, C, D_skip, z, dout, nthreads=0, delta_softplus=False, delta_bias=None):
+def scan_bwd(x, delta, A, B, C, D_skip, z, dout, nthreads=0, delta_softplus=False, delta_bias=None, zoh=False):
     """Analytic adjoint of scan_fwd for loss = sum(dout * out), sequential, fp64.
 
     Returns a dict with dx, ddelta, dz (batch, L, D); dB, dC (batch, L, N); dA (D, N); dD (D) -- all float64.
     dz is zero when z is None, dD is zero when D_skip is None.  With delta_softplus, `delta` is the pre-activation,
-    ddelta its gradient, and the dict also holds ddelta_bias (D) = ddelta summed over batch and time.
+    ddelta its gradient, and the dict also holds ddelta_bias (D) = ddelta summed over batch and time.  `zoh` selects
+    the zero-order-hold B-bar of Eq. 4 as in scan_fwd.
     """
     lib = _load()
     st = _storage_dtype(x)
@@ -127,7 +128,8 @@ def scan_bwd(x, delta, A, B, C, D_skip, z, dout, nthreads=0, delta_softplus=Fals
     g["dD"] = np.empty((D,), dtype=np.float64)
     g["ddelta_bias"] = np.empty((D,), dtype=np.float64)
     bias = None if delta_bias is None else np.ascontiguousarray(delta_bias, dtype=np.float64)
-    dims = _Dims(batch, L, D, N, int(z is not None), int(D_skip is not None), 0, int(bool(delta_softplus)), int(nthreads))
+    dims = _Dims(batch, L, D, N, int(z is not None), int(D_skip is not None), int(bool(zoh)), int(bool(delta_softplus)),
+                 int(nthreads))
     fn = lib.ssm_oracle_bwd_f32 if st == np.float32 else lib.ssm_oracle_bwd_f64
     rc = fn(ctypes.byref(dims), _ptr(io["x"]), _ptr(io["delta"]), _ptr(A64), _ptr(io["B"]), _ptr(io["C"]), _ptr(Dk),
             _ptr(io["z"]), _ptr(io["dout"]), _ptr(bias), _ptr(g["dx"]), _ptr(g["ddelta"]), _ptr(g["dA"]), _ptr(g["dB"]),

@@ -329,3 +329,53 @@ def test_softplus_gradients_match_finite_differences():
     for k in ("dx", "dz", "dA", "dB", "dC", "dD"):
         np.testing.assert_allclose(g[k], g0[k], rtol=1e-11, atol=1e-12)
     np.testing.assert_allclose(g["ddelta"], g0["ddelta"] / (1.0 + np.exp(-(v + bias))), rtol=1e-11, atol=1e-12)
+
+
+# --------------------------------------------------------------------------------------------------------------
+# Zero-order-hold B-bar (Eq. 4) -- forward against a library matrix exponential, backward against finite differences.
+def test_zoh_is_the_exact_solution_for_held_inputs():
+    # Eq. 1a with the input held constant over a step of length delta: [h; 1](t + delta) = expm(delta * M) [h; 1](t),
+    # M = [[diag(A), B x], [0, 0]].  The library matrix exponential knows nothing of the closed form (e^{dA} - 1) / A.
+    from scipy.linalg import expm
+    L, N = 9, 3
+    p = _rand_problem(1, L, 1, N)
+    p["A"][0, 1] = 0.0                      # the removable singularity of (e^{dA} - 1) / A
+    got, s_pre = O.scan_fwd(p["x"], p["delta"], p["A"], p["B"], p["C"], zoh=True, return_pregate=True)
+    h = np.zeros(N)
+    for t in range(L):
+        M = np.zeros((N + 1, N + 1))
+        M[:N, :N] = np.diag(p["A"][0])
+        M[:N, N] = p["B"][0, t] * p["x"][0, t, 0]
+        h = (expm(p["delta"][0, t, 0] * M) @ np.append(h, 1.0))[:N]
+        assert abs(s_pre[0, t, 0] - p["C"][0, t] @ h) <= 1e-12 * max(1.0, abs(s_pre[0, t, 0]))
+
+
+@pytest.mark.parametrize("small_steps", [False, True])
+def test_zoh_gradients_match_finite_differences(small_steps):
+    batch, L, D, N = 2, 10, 3, 4
+    p = _rand_problem(batch, L, D, N, dt_scale=2e-3 if small_steps else 0.5)   # both branches of dE/dA
+    p["A"][1, 2] = 0.0
+    dout = RNG.standard_normal((batch, L, D))
+    g = O.scan_bwd(p["x"], p["delta"], p["A"], p["B"], p["C"], p["D_skip"], p["z"], dout, zoh=True)
+
+    def loss(q):
+        return float((dout * O.scan_fwd(q["x"], q["delta"], q["A"], q["B"], q["C"], D_skip=q["D_skip"], z=q["z"],
+                                        zoh=True)).sum())
+    names = {"x": "dx", "delta": "ddelta", "A": "dA", "B": "dB", "C": "dC", "D_skip": "dD", "z": "dz"}
+    for key, gname in names.items():
+        eps = 1e-6 * max(1.0, float(np.abs(p[key]).max())) if key != "delta" else 1e-6 * float(p["delta"].mean())
+        for trial in range(3):
+            v = RNG.standard_normal(p[key].shape)
+            pp, pm = dict(p), dict(p)
+            pp[key] = p[key] + eps * v
+            pm[key] = p[key] - eps * v
+            fd = (loss(pp) - loss(pm)) / (2 * eps)
+            an = float((g[gname] * v).sum())
+            assert abs(fd - an) <= 2e-6 * max(1.0, abs(an)), (key, fd, an)
+    # the entry with A = 0 on its own (the limit delta^2 / 2 of dE/dA)
+    e = np.zeros_like(p["A"])
+    e[1, 2] = 1e-6
+    pp, pm = dict(p), dict(p)
+    pp["A"], pm["A"] = p["A"] + e, p["A"] - e
+    fd = (loss(pp) - loss(pm)) / 2e-6
+    assert abs(fd - g["dA"][1, 2]) <= 2e-6 * max(1.0, abs(fd))
