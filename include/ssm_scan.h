@@ -72,6 +72,9 @@ enum {
                                  from (Appendix D keeps "intermediate scan states" between chunks)             */
   SSM_FLAG_GENERAL_A = 8u,    /* do not use the fast path for rows of A that are arithmetic progressions in n   */
   SSM_FLAG_DELTA_SOFTPLUS = 32u, /* ssm_scan_*_fused_dt: the step size is softplus(delta_pre + delta_bias[d])         */
+  SSM_FLAG_ZOH_BBAR = 64u,    /* B-bar = (exp(delta A) - 1) / A * B, the zero-order hold of Eq. 4 (delta * B at A = 0),
+                                 instead of the default delta * B; honoured by every call; such problems run on
+                                 the generic kernels                                                             */
   SSM_FLAG_TEST_WITHHOLD = 16u /* test hook for the bounded waits: the tuned backward kernel never publishes its
                                  hand-off flags and polls only 1000 times, so every dependent tile gives up and
                                  ssm_scan_check_status reports SSM_ERR_TIMEOUT; the gradients are then undefined  */

@@ -17,6 +17,7 @@ SSM_OK = 0
 SSM_F32, SSM_BF16 = 0, 1
 SSM_FLAG_HAS_Z, SSM_FLAG_HAS_DSKIP, SSM_FLAG_SAVE_STATES, SSM_FLAG_GENERAL_A, SSM_FLAG_TEST_WITHHOLD = 1, 2, 4, 8, 16
 SSM_FLAG_DELTA_SOFTPLUS = 32
+SSM_FLAG_ZOH_BBAR = 64
 
 EXPORTED_SYMBOLS = (
     "ssm_scan_fwd_workspace_bytes", "ssm_scan_bwd_workspace_bytes", "ssm_scan_saved_state_bytes",
@@ -103,10 +104,11 @@ def _io_dtype(t: torch.Tensor) -> int:
 
 
 def make_problem(x: torch.Tensor, B: torch.Tensor, has_z: bool, has_dskip: bool, save_states: bool = False,
-                 general_A: bool = False) -> ssm_problem_t:
+                 general_A: bool = False, zoh: bool = False) -> ssm_problem_t:
     batch, L, D = x.shape
     flags = (SSM_FLAG_HAS_Z if has_z else 0) | (SSM_FLAG_HAS_DSKIP if has_dskip else 0) \
-        | (SSM_FLAG_SAVE_STATES if save_states else 0) | (SSM_FLAG_GENERAL_A if general_A else 0)
+        | (SSM_FLAG_SAVE_STATES if save_states else 0) | (SSM_FLAG_GENERAL_A if general_A else 0) \
+        | (SSM_FLAG_ZOH_BBAR if zoh else 0)
     return ssm_problem_t(batch, L, D, B.shape[-1], _io_dtype(x), flags)
 
 
@@ -162,18 +164,18 @@ def saved_state_bytes(problem: ssm_problem_t) -> int:
     return int(load_library().ssm_scan_saved_state_bytes(ctypes.byref(problem)))
 
 
-def ssm_scan_fwd(x, delta, A, B, C, D_skip=None, z=None, *, save_states=False, general_A=False, out=None,
+def ssm_scan_fwd(x, delta, A, B, C, D_skip=None, z=None, *, save_states=False, general_A=False, zoh=False, out=None,
                  saved_states=None, workspace=None, stream=None, h0=None, h_last=None):
     """out = selective_scan(x, delta, A, B, C) (+ D_skip * x) (* silu(z)); see include/ssm_scan.h.
 
     x, delta, z: (batch, L, D) io dtype; B, C: (batch, L, N) io dtype; A: (D, N) float32; D_skip: (D) float32.
     Returns `out`, or `(out, saved_states)` with save_states=True.  Enqueues on `stream` (default: torch's current
-    stream) and does not synchronise.  `h0` (batch, D, N) float32 is the state before the first step (default zero);
+    stream) and does not synchronise.  zoh=True selects the zero-order-hold B-bar of Eq. 4.  `h0` (batch, D, N) float32 is the state before the first step (default zero);
     if a float32 tensor `h_last` (batch, D, N) is passed it receives the state after the last step
     (ssm_scan_fwd_state).
     """
     lib = load_library()
-    prob = make_problem(x, B, z is not None, D_skip is not None, save_states, general_A)
+    prob = make_problem(x, B, z is not None, D_skip is not None, save_states, general_A, zoh)
     batch, L, D, N = prob.batch, prob.L, prob.D, prob.N
     io = x.dtype
     if out is None:
@@ -259,14 +261,15 @@ def ssm_scan_bwd_fused_dt(x, delta_pre, delta_bias, A, B, C, D_skip, z, dout, sa
     return o
 
 
-def ssm_step(x, delta, A, B, C, D_skip, z, h, *, out=None, stream=None):
+def ssm_step(x, delta, A, B, C, D_skip, z, h, *, zoh=False, out=None, stream=None):
     """One recurrent step: x, delta, z (batch, D), B, C (batch, N) io dtype; h (batch, D, N) float32 is updated in
     place.  Returns out (batch, D)."""
     lib = load_library()
     batch, D = x.shape
     N = B.shape[-1]
     prob = ssm_problem_t(batch, 1, D, N, _io_dtype(x),
-                         (SSM_FLAG_HAS_Z if z is not None else 0) | (SSM_FLAG_HAS_DSKIP if D_skip is not None else 0))
+                         (SSM_FLAG_HAS_Z if z is not None else 0) | (SSM_FLAG_HAS_DSKIP if D_skip is not None else 0)
+                         | (SSM_FLAG_ZOH_BBAR if zoh else 0))
     io = x.dtype
     if out is None:
         out = torch.empty_like(x)
@@ -319,7 +322,7 @@ def ssm_scan_fwd_static(x, delta, A, B, C, D_skip=None, z=None, *, save_states=F
     return (out, saved_states) if save_states else out
 
 
-def ssm_scan_bwd(x, delta, A, B, C, D_skip, z, dout, saved_states=None, *, general_A=False, workspace=None,
+def ssm_scan_bwd(x, delta, A, B, C, D_skip, z, dout, saved_states=None, *, general_A=False, zoh=False, workspace=None,
                  stream=None, outputs=None, extra_flags=0):
     """Gradients of sum(dout * out) w.r.t. x, delta, A, B, C, D_skip, z; see include/ssm_scan.h.
 
@@ -327,7 +330,7 @@ def ssm_scan_bwd(x, delta, A, B, C, D_skip, z, dout, saved_states=None, *, gener
     dD (float32, (D)).  dz / dD are None when z / D_skip is None.  `outputs` may pass preallocated tensors.
     """
     lib = load_library()
-    prob = make_problem(x, B, z is not None, D_skip is not None, False, general_A)
+    prob = make_problem(x, B, z is not None, D_skip is not None, False, general_A, zoh)
     prob.flags |= int(extra_flags)
     batch, L, D, N = prob.batch, prob.L, prob.D, prob.N
     io = x.dtype

@@ -16,7 +16,7 @@ static ssm_status_t validate_problem(const ssm_problem_t* p) {
   if (p == nullptr) return SSM_ERR_INVALID_ARG;
   if (p->batch < 1 || p->L < 1 || p->D < 1 || p->N < 1) return SSM_ERR_INVALID_ARG;
   if (p->flags & ~(uint32_t)(SSM_FLAG_HAS_Z | SSM_FLAG_HAS_DSKIP | SSM_FLAG_SAVE_STATES | SSM_FLAG_GENERAL_A | SSM_FLAG_TEST_WITHHOLD |
-                             SSM_FLAG_DELTA_SOFTPLUS))
+                             SSM_FLAG_DELTA_SOFTPLUS | SSM_FLAG_ZOH_BBAR))
     return SSM_ERR_INVALID_ARG;
   if (p->io_dtype != SSM_F32 && p->io_dtype != SSM_BF16) return SSM_ERR_UNSUPPORTED;
   if (p->N != 1 && p->N != 2 && p->N != 4 && p->N != 8 && p->N != 16) return SSM_ERR_UNSUPPORTED;
@@ -233,6 +233,7 @@ static ssm_status_t fwd_impl(const ssm_problem_t* p, const void* x, const void* 
   fp.seg_steps = pl.seg_steps;
   fp.nck = pl.nck;
   fp.general_A = (p->flags & SSM_FLAG_GENERAL_A) ? 1 : 0;
+  fp.zoh = (p->flags & SSM_FLAG_ZOH_BBAR) ? 1 : 0;
   fp.delta_bias = delta_bias;
   fp.softplus = (p->flags & SSM_FLAG_DELTA_SOFTPLUS) ? 1 : 0;
   const float* h_start = nullptr;
@@ -293,6 +294,7 @@ ssm_status_t ssm_step(const ssm_problem_t* p, const void* x, const void* delta, 
   sp.batch = p->batch;
   sp.D = p->D;
   sp.N = p->N;
+  sp.zoh = (p->flags & SSM_FLAG_ZOH_BBAR) ? 1 : 0;
   if (launch_step(*p, sp, static_cast<cudaStream_t>(stream)) != cudaSuccess) return SSM_ERR_CUDA;
   return SSM_OK;
 }
@@ -338,6 +340,7 @@ static ssm_status_t bwd_impl(const ssm_problem_t* p, const void* x, const void* 
     fp.seg_steps = pl.seg_steps;
     fp.nck = pl.nck;
     fp.general_A = (p->flags & SSM_FLAG_GENERAL_A) ? 1 : 0;
+    fp.zoh = (p->flags & SSM_FLAG_ZOH_BBAR) ? 1 : 0;
     fp.delta_bias = delta_bias;
     fp.softplus = (p->flags & SSM_FLAG_DELTA_SOFTPLUS) ? 1 : 0;
     const float* h_start = nullptr;
@@ -372,6 +375,7 @@ static ssm_status_t bwd_impl(const ssm_problem_t* p, const void* x, const void* 
   bp.nck = pl.nck;
   bp.groups = pl.bwd_groups;
   bp.general_A = (p->flags & SSM_FLAG_GENERAL_A) ? 1 : 0;
+  bp.zoh = (p->flags & SSM_FLAG_ZOH_BBAR) ? 1 : 0;
   bp.test_withhold = (p->flags & SSM_FLAG_TEST_WITHHOLD) ? 1 : 0;
   bp.delta_bias = delta_bias;
   bp.softplus = (p->flags & SSM_FLAG_DELTA_SOFTPLUS) ? 1 : 0;

@@ -130,8 +130,15 @@ __global__ void __launch_bounds__(BwdGeom<N>::THREADS) ssm_bwd_kernel(const BwdP
       float y = 0.f;
 #pragma unroll
       for (int k = 0; k < S; ++k) {
-        const float a = ex2_approx(dt * A2[k]);
-        h[k] = fmaf(a, h[k], du * s_B[tt * N + j * S + k]);
+        float a, bx = du * s_B[tt * N + j * S + k];
+        if (p.zoh) {
+          float E;
+          zoh_discretize(dt, Ar[k], a, E);
+          bx = E * u * s_B[tt * N + j * S + k];
+        } else {
+          a = ex2_approx(dt * A2[k]);
+        }
+        h[k] = fmaf(a, h[k], bx);
         y = fmaf(s_C[tt * N + j * S + k], h[k], y);
         s_h[((size_t)(tt + 1) * CH + slot) * N + j * S + k] = h[k];
       }
@@ -155,7 +162,9 @@ __global__ void __launch_bounds__(BwdGeom<N>::THREADS) ssm_bwd_kernel(const BwdP
         ds = g * zz * sg;
         dzv = g * s_s[tt * CH + slot] * sg * fmaf(zz, 1.f - sg, 1.f);
       }
-      float lamB = 0.f, wA = 0.f;
+      // lamB = sum_n lam B (default rule; with ZOH sum_n lam E B, the input gradient), lamGB = sum_n lam a B (ZOH
+      // only: the step-size gradient through E, dE/ddelta = a)
+      float lamB = 0.f, lamGB = 0.f, wA = 0.f;
       float dBp[S], dCp[S];
 #pragma unroll
       for (int k = 0; k < S; ++k) {
@@ -164,9 +173,20 @@ __global__ void __launch_bounds__(BwdGeom<N>::THREADS) ssm_bwd_kernel(const BwdP
         const float Bn = s_B[tt * N + j * S + k];
         const float lam = fmaf(s_C[tt * N + j * S + k], ds, mu[k]);
         dCp[k] = ds * ht;
-        dBp[k] = lam * du;
-        lamB = fmaf(lam, Bn, lamB);
-        const float a = ex2_approx(dt * A2[k]);
+        float a;
+        if (p.zoh) {
+          // B-bar = E B with E = (a - 1) / A: dE/ddelta = a, dE/dA = (dt a - E) / A
+          float E;
+          zoh_discretize(dt, Ar[k], a, E);
+          dBp[k] = lam * E * u;
+          lamB = fmaf(lam * E, Bn, lamB);
+          lamGB = fmaf(lam * a, Bn, lamGB);
+          dA[k] = fmaf(lam * zoh_gain_dA(dt, Ar[k], a, E), Bn * u, dA[k]);
+        } else {
+          a = ex2_approx(dt * A2[k]);
+          dBp[k] = lam * du;
+          lamB = fmaf(lam, Bn, lamB);
+        }
         mu[k] = a * lam;
         const float w = mu[k] * hp;
         wA = fmaf(w, Ar[k], wA);
@@ -175,6 +195,7 @@ __global__ void __launch_bounds__(BwdGeom<N>::THREADS) ssm_bwd_kernel(const BwdP
 #pragma unroll
       for (int m = LPC / 2; m >= 1; m >>= 1) {
         lamB += __shfl_xor_sync(0xffffffffu, lamB, m);
+        lamGB += __shfl_xor_sync(0xffffffffu, lamGB, m);
         wA += __shfl_xor_sync(0xffffffffu, wA, m);
       }
       // sum dB/dC over the channels held by this warp (lanes that share j)
@@ -196,9 +217,9 @@ __global__ void __launch_bounds__(BwdGeom<N>::THREADS) ssm_bwd_kernel(const BwdP
       if (j == 0) {
         dD_acc = fmaf(ds, u, dD_acc);
         // with the softplus the gradient goes to the pre-activation: d softplus(v)/dv = sigmoid(v)
-        const float ddv = fmaf(u, lamB, wA) * (p.softplus ? 1.f / (1.f + __expf(-dv)) : 1.f);
+        const float ddv = fmaf(u, p.zoh ? lamGB : lamB, wA) * (p.softplus ? 1.f / (1.f + __expf(-dv)) : 1.f);
         dbias_acc += ddv;
-        s_x[tt * CH + slot] = float_to_io<IO>(fmaf(ds, Dk, dt * lamB));
+        s_x[tt * CH + slot] = float_to_io<IO>(fmaf(ds, Dk, p.zoh ? lamB : dt * lamB));
         s_d[tt * CH + slot] = float_to_io<IO>(ddv);
         s_z[tt * CH + slot] = float_to_io<IO>(dzv);
       }

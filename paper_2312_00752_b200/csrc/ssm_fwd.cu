@@ -56,7 +56,7 @@ __global__ void __launch_bounds__(fwd_threads(N)) ssm_fwd_kernel(const FwdParams
   const int d_thr = d_cta + slot * CPT;
   const int D = p.D;
 
-  float A2[CPT][S], h[CPT][S], dsum[CPT], dbias[CPT];
+  float A2[CPT][S], Ar[CPT][S], h[CPT][S], dsum[CPT], dbias[CPT];
 #pragma unroll
   for (int q = 0; q < CPT; ++q) {
     const int d = d_thr + q;
@@ -65,7 +65,8 @@ __global__ void __launch_bounds__(fwd_threads(N)) ssm_fwd_kernel(const FwdParams
     dbias[q] = (valid && p.delta_bias != nullptr) ? p.delta_bias[d] : 0.f;
 #pragma unroll
     for (int k = 0; k < S; ++k) {
-      A2[q][k] = valid ? p.A[(size_t)d * N + j * S + k] * kLog2e : 0.f;
+      Ar[q][k] = valid ? p.A[(size_t)d * N + j * S + k] : 0.f;
+      A2[q][k] = Ar[q][k] * kLog2e;
       h[q][k] = (valid && p.h_start != nullptr)
                     ? p.h_start[(((size_t)b * p.nseg + seg) * D + d) * N + j * S + k]
                     : 0.f;
@@ -135,8 +136,15 @@ __global__ void __launch_bounds__(fwd_threads(N)) ssm_fwd_kernel(const FwdParams
         y[q] = 0.f;
 #pragma unroll
         for (int k = 0; k < S; ++k) {
-          const float a = ex2_approx(dt * A2[q][k]);
-          h[q][k] = fmaf(a, h[q][k], du * Bv[k]);
+          float a, bx = du * Bv[k];
+          if (p.zoh) {
+            float E;
+            zoh_discretize(dt, Ar[q][k], a, E);
+            bx = E * u[q] * Bv[k];
+          } else {
+            a = ex2_approx(dt * A2[q][k]);
+          }
+          h[q][k] = fmaf(a, h[q][k], bx);
           if constexpr (kReadout) y[q] = fmaf(Cv[k], h[q][k], y[q]);
         }
       }

@@ -1,6 +1,7 @@
 // One recurrent step of the selective SSM (the recurrent mode of Eq. 2 used for autoregressive inference, Section 2
 // "Computation"): for every (batch, channel)
 //     h[n] <- exp(delta * A[n]) * h[n] + delta * x * B[n];   out = (sum_n C[n] h[n] + D_skip * x) * silu(z)
+// (or with the zero-order-hold B-bar of Eq. 4 in place of delta * B),
 // with the state h [batch][D][N] updated in place.  Constant time per token, no history.
 //
 // The work is a single pass over the state (2 * 4 N bytes per channel against a few bytes of inputs), so the kernel is
@@ -42,8 +43,15 @@ __global__ void __launch_bounds__(128) ssm_step_kernel(const StepParams p) {
   float y = 0.f;
 #pragma unroll
   for (int k = 0; k < N; ++k) {
-    const float a = ex2_approx(dt * (av[k] * kLog2e));
-    hv[k] = fmaf(a, hv[k], du * io_to_float<IO>(__ldg(gB + k)));
+    float a, bx = du * io_to_float<IO>(__ldg(gB + k));
+    if (p.zoh) {
+      float E;
+      zoh_discretize(dt, av[k], a, E);
+      bx = E * u * io_to_float<IO>(__ldg(gB + k));
+    } else {
+      a = ex2_approx(dt * (av[k] * kLog2e));
+    }
+    hv[k] = fmaf(a, hv[k], bx);
     y = fmaf(io_to_float<IO>(__ldg(gC + k)), hv[k], y);
   }
   if (N % 4 == 0) {

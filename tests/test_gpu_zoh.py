@@ -1,0 +1,90 @@
+"""Zero-order-hold B-bar (Eq. 4: B-bar = (exp(delta A) - 1) / A * B) on the GPU against the oracle: forward, backward,
+the single recurrent step, and the gated-recurrence special case of Theorem 1."""
+import numpy as np
+import pytest
+
+from paper_2312_00752_b200 import synth
+from tests import _gpu_util as U
+
+pytestmark = pytest.mark.gpu
+
+
+def _case(batch, L, D, N, io, dt=(1e-3, 1e-1), seed=0):
+    cfg = synth.ScanConfig("zoh", 14, batch, L, D, N, io, dt[0], dt[1])
+    inp = synth.make_inputs(cfg, seed=seed)
+    inp["A"] = inp["A"].copy()
+    inp["A"][0, 0] = 0.0            # the removable singularity: B-bar = delta * B there
+    return inp
+
+
+@pytest.mark.parametrize("batch,L,D,N,io,dt", [
+    (2, 130, 40, 16, "bf16", (1e-3, 1e-1)),
+    (1, 200, 24, 8, "f32", (1e-3, 1e-1)),
+    (2, 97, 33, 4, "f32", (5e-2, 2.0)),        # large steps: the two rules differ by O(1)
+    (1, 4200, 32, 16, "f32", (1e-4, 1e-2)),    # time split: segment summaries and both carries under ZOH
+    (1, 64, 16, 1, "bf16", (1e-2, 1.0)),
+])
+def test_zoh_forward_backward(batch, L, D, N, io, dt):
+    from oracle import ssm_oracle as O
+    from paper_2312_00752_b200 import binding as K
+    inp = _case(batch, L, D, N, io, dt)
+    dev = U.to_device(inp, io)
+    args = (dev["x"], dev["delta"], dev["A"], dev["B"], dev["C"], dev["D_skip"], dev["z"])
+    out, saved = K.ssm_scan_fwd(*args, save_states=True, zoh=True)
+    g = K.ssm_scan_bwd(*args, dev["dout"], saved, zoh=True)
+    ref_out = O.scan_fwd(inp["x"], inp["delta"], inp["A"], inp["B"], inp["C"], D_skip=inp["D_skip"], z=inp["z"], zoh=True)
+    ref = O.scan_bwd(inp["x"], inp["delta"], inp["A"], inp["B"], inp["C"], inp["D_skip"], inp["z"], inp["dout"], zoh=True)
+    tol = U.TOL[io]
+    assert U.rel_err(U.to_host(out), ref_out) <= tol["out"]
+    for k in U.GRADS:
+        assert U.rel_err(U.to_host(g[k]), ref[k]) <= tol["grad"], k
+    # the flag is not a no-op: the default rule gives a different answer where delta * A is not small
+    if dt[1] >= 1.0:
+        plain = O.scan_fwd(inp["x"], inp["delta"], inp["A"], inp["B"], inp["C"], D_skip=inp["D_skip"], z=inp["z"])
+        assert U.rel_err(U.to_host(out), plain) > 0.03
+    # backward without saved states rebuilds the checkpoints under the same rule
+    g2 = K.ssm_scan_bwd(*args, dev["dout"], None, zoh=True)
+    for k in ("dx", "ddelta", "dA", "dB"):
+        assert U.rel_err(U.to_host(g2[k]), ref[k]) <= tol["grad"], k
+
+
+def test_zoh_gated_recurrence_of_theorem_1():
+    # N = 1, A = -1, B = C = 1, delta = softplus(v): h_t = (1 - g_t) h_{t-1} + g_t x_t with g = sigmoid(v)
+    import torch
+    from paper_2312_00752_b200 import binding as K
+    rng = np.random.default_rng(5)
+    batch, L, D = 2, 150, 24
+    v = rng.standard_normal((batch, L, D)) * 2.0
+    x = rng.standard_normal((batch, L, D)).astype(np.float32)
+    delta = np.log1p(np.exp(v)).astype(np.float32)
+    g = -np.expm1(-delta.astype(np.float64))          # 1 - exp(-delta), the gate the rounded step size stands for
+    h = np.zeros((batch, D))
+    ref = np.empty((batch, L, D))
+    for t in range(L):
+        h = (1.0 - g[:, t]) * h + g[:, t] * x[:, t]
+        ref[:, t] = h
+    ones = torch.ones((batch, L, 1), dtype=torch.float32, device="cuda")
+    A = -torch.ones((D, 1), dtype=torch.float32, device="cuda")
+    out = K.ssm_scan_fwd(torch.from_numpy(x).cuda(), torch.from_numpy(delta).cuda(), A, ones, ones, zoh=True)
+    assert U.rel_err(U.to_host(out), ref) <= 1e-5
+
+
+@pytest.mark.parametrize("batch,D,N,io", [(3, 40, 16, "bf16"), (2, 33, 8, "f32")])
+def test_zoh_step_by_step_equals_scan(batch, D, N, io):
+    import torch
+    from oracle import ssm_oracle as O
+    from paper_2312_00752_b200 import binding as K
+    T = 20
+    inp = _case(batch, T, D, N, io, (5e-2, 1.0))
+    dev = U.to_device(inp, io)
+    ref_out, ref_h = O.scan_fwd(inp["x"], inp["delta"], inp["A"], inp["B"], inp["C"], D_skip=inp["D_skip"], z=inp["z"],
+                                zoh=True, return_h_last=True)
+    h = torch.zeros((batch, D, N), dtype=torch.float32, device="cuda")
+    outs = []
+    for t in range(T):
+        outs.append(K.ssm_step(dev["x"][:, t].contiguous(), dev["delta"][:, t].contiguous(), dev["A"],
+                               dev["B"][:, t].contiguous(), dev["C"][:, t].contiguous(), dev["D_skip"],
+                               dev["z"][:, t].contiguous(), h, zoh=True))
+    got = np.stack([U.to_host(o) for o in outs], axis=1)
+    assert U.rel_err(got, ref_out) <= U.TOL[io]["out"]
+    assert U.rel_err(U.to_host(h), ref_h) <= 1e-5
