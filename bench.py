@@ -57,6 +57,21 @@ def algorithmic_bytes(cfg):
     return fwd, bwd
 
 
+# ALU peaks of one B200 from its unit counts and clocks: 148 SMs x 128 FP32 lanes x 1.965 GHz (a multiply-add counts
+# as one lane-operation) and 148 SMs x 16 special-function results per clock
+FP32_LANE_OPS_PER_S = 148 * 128 * 1.965e9
+MUFU_OPS_PER_S = 148 * 16 * 1.965e9
+
+
+def algorithmic_alu_ops(cfg):
+    """FP32 lane-operations and exponentials the method itself needs per element (batch, step, channel): forward
+    4 per state (discretize 2, recurrence 1, readout 1) + 14 per element (delta * x, skip, gate, converts) and one
+    exponential per state + 1 (gate); backward 13 per state (recompute 3, lambda 2, dC 1, w 2, dA 1, ddelta 1,
+    lambda * B 1, dB 1, cross-channel sums 1) + 30 per element and one exponential per state + 3."""
+    n = cfg.N
+    return {"fwd_fp32": 4 * n + 14, "fwd_exp": n + 1, "bwd_fp32": 13 * n + 30, "bwd_exp": n + 3}
+
+
 def measured_peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     try:
@@ -279,16 +294,12 @@ def run_ours(args, cfg):
         names_in = ("x", "delta", "z", "dout", "B", "C", "A", "D_skip")
         h2d = sum(pinned[k].numel() * pinned[k].element_size() for k in names_in)
         d2h = sum(v.numel() * v.element_size() for v in hres.values())
-        es = sets[0]
+        arena = torch.empty(K.host_arena_bytes(prob), dtype=torch.uint8, device=dev)
 
-        def e2e_step():
-            for k in names_in:
-                es[k].copy_(pinned[k], non_blocking=True)
-            fwd(es)
-            bwd(es)
-            hres["out"].copy_(out, non_blocking=True)
-            for k, v in grads.items():
-                hres[k].copy_(v, non_blocking=True)
+        def e2e_step():   # one library call: host buffers in, host buffers out, copies pipelined with the kernels
+            K.ssm_scan_fwd_bwd_host(pinned["x"], pinned["delta"], pinned["A"], pinned["B"], pinned["C"],
+                                    pinned["D_skip"], pinned["z"], pinned["dout"], device=dev, arena=arena,
+                                    outputs=hres, stream=stream)
 
         e2e_step()
         barrier()
@@ -302,7 +313,8 @@ def run_ours(args, cfg):
         e2e_ms = max_over_ranks(a.elapsed_time(b) / n_e2e, dev)
         e2e = {"value": job_value(cfg.elements, world, e2e_ms), "unit": "elements/s",
                "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h), "ms_per_step": e2e_ms,
-               "steps": n_e2e}
+               "steps": n_e2e, "api": "ssm_scan_fwd_bwd_host (pinned host buffers in and out, batch pipelined over "
+                                      "copy-in / compute / copy-out streams)"}
 
     if rank != 0:
         if world > 1:
@@ -314,6 +326,13 @@ def run_ours(args, cfg):
     f_ms, b_ms = statistics.mean(fwd_ms), statistics.mean(bwd_ms)
     bwd_gbs = bwd_bytes / (b_ms * 1e-3) / 1e9
     fwd_gbs = fwd_bytes / (f_ms * 1e-3) / 1e9
+    alu = algorithmic_alu_ops(cfg)
+
+    def alu_fracs(direction, ms):
+        per_s = cfg.elements / (ms * 1e-3)
+        return {"frac_of_fp32_lane_peak": per_s * alu[direction + "_fp32"] / FP32_LANE_OPS_PER_S,
+                "frac_of_mufu_peak": per_s * alu[direction + "_exp"] / MUFU_OPS_PER_S}
+
     line = {
         "metric": METRIC, "value": job_value(cfg.elements, world, ms_per_step), "unit": "elements/s",
         "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step,
@@ -328,14 +347,21 @@ def run_ours(args, cfg):
         "clocks": clocks,
         "gpu_launches": kernels_per_step(plan_info) * args.steps,
         "fwd": {"ms": f_ms, "elements_per_s": cfg.elements / (f_ms * 1e-3), "algorithmic_bytes": fwd_bytes,
-                "achieved_gbs": fwd_gbs, "frac_of_hbm_peak": fwd_gbs / peak},
+                "achieved_gbs": fwd_gbs, "frac_of_hbm_peak": fwd_gbs / peak, **alu_fracs("fwd", f_ms)},
         "bwd": {"ms": b_ms, "elements_per_s": cfg.elements / (b_ms * 1e-3), "algorithmic_bytes": bwd_bytes,
-                "achieved_gbs": bwd_gbs, "frac_of_hbm_peak": bwd_gbs / peak},
+                "achieved_gbs": bwd_gbs, "frac_of_hbm_peak": bwd_gbs / peak, **alu_fracs("bwd", b_ms)},
         "roofline": {"bound": "hbm", "kernel": "ssm_scan_bwd call (backward kernel + its reduction kernel)",
                      "achieved": bwd_gbs, "peak": peak, "peak_kind": f"{peak_kind} copy bandwidth",
                      "unit": "GB/s", "frac": bwd_gbs / peak,
                      "traffic": NCU_TRAFFIC_BYTES.get(cfg.cfg_id) if not args.general_A else None,
                      "algorithmic_bytes": bwd_bytes},
+        # the same launch against the ALU roof that actually binds it (algorithmic FP32 lane-operations per second
+        # over lanes x clock); the HBM figure above is the metric, this one says how far the kernel is from its bound
+        "roofline_alu": {"bound": "alu", "kernel": "ssm_scan_bwd call",
+                         "achieved": cfg.elements / (b_ms * 1e-3) * alu["bwd_fp32"] / 1e12,
+                         "peak": FP32_LANE_OPS_PER_S / 1e12, "unit": "T lane-op/s (FP32, FMA = 1)",
+                         "frac": alu_fracs("bwd", b_ms)["frac_of_fp32_lane_peak"],
+                         "ops_per_element": alu["bwd_fp32"]},
         "wall_s_timed_region": t_wall,
     }
     # the single recurrent step (decode): one pass over the float32 state, batch 64 at the same width

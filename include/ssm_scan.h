@@ -211,6 +211,34 @@ SSM_API ssm_status_t ssm_scan_fwd_static(const ssm_problem_t* p, const void* x, 
                                          const void* B, const void* C, const float* D_skip, const void* z, void* out,
                                          void* saved_states, void* stream /* cudaStream_t */);
 
+/*
+ * Forward + backward of one batch held in HOST memory, copies included (the paper has no counterpart: its kernels
+ * start from tensors already in HBM).  Equivalent to copying every input to the device, calling ssm_scan_fwd with
+ * SSM_FLAG_SAVE_STATES and ssm_scan_bwd with those states, and copying every result back; the batch is cut into up
+ * to 8 pieces whose copies in, computation and copies out overlap on three streams (the batch entries are
+ * independent, Section 2 "Structure and Dimensions").
+ *   x, delta, z, dout, B, C, A, D_skip      in, HOST pointers, layouts and dtypes as for ssm_scan_fwd / ssm_scan_bwd
+ *   out, dx, ddelta, dz, dB, dC, dA, dD     out, HOST pointers, every element overwritten; dz / dD are required iff
+ *                                           SSM_FLAG_HAS_Z / SSM_FLAG_HAS_DSKIP
+ *   device_arena   DEVICE scratch of at least ssm_scan_host_arena_bytes(p) bytes, 256-byte aligned, caller-owned
+ *   stream         the call is ordered after everything already enqueued on it, and work enqueued on it afterwards
+ *                  is ordered after every copy of this call; the call itself does not wait for the GPU
+ * Host buffers should be page-locked: with pageable memory the results are the same but the copies do not overlap.
+ * The host buffers and the arena must stay valid and untouched until the stream has passed the call.  dA and dD are
+ * summed over the pieces in ascending order, so they can differ in the last bit from one ssm_scan_bwd call over the
+ * whole batch; everything else is identical.  The library keeps two helper streams per device (created on first use)
+ * and allocates no device memory.  Flags other than HAS_Z, HAS_DSKIP, GENERAL_A and ZOH_BBAR are ignored.
+ * Errors: SSM_ERR_INVALID_ARG / SSM_ERR_UNSUPPORTED as for the device calls, SSM_ERR_WORKSPACE for a short, NULL or
+ * misaligned arena (nothing is enqueued), SSM_ERR_CUDA if a runtime call fails (the stream is still ordered after
+ * whatever had been enqueued).
+ */
+SSM_API size_t ssm_scan_host_arena_bytes(const ssm_problem_t* p);
+SSM_API ssm_status_t ssm_scan_fwd_bwd_host(const ssm_problem_t* p, const void* x, const void* delta, const float* A,
+                                           const void* B, const void* C, const float* D_skip, const void* z,
+                                           const void* dout, void* out, void* dx, void* ddelta, float* dA, void* dB,
+                                           void* dC, float* dD, void* dz, void* device_arena, size_t arena_bytes,
+                                           void* stream /* cudaStream_t */);
+
 /* Human-readable name of a status code (static storage). */
 SSM_API const char* ssm_status_string(ssm_status_t s);
 

@@ -23,7 +23,7 @@ EXPORTED_SYMBOLS = (
     "ssm_scan_fwd_workspace_bytes", "ssm_scan_bwd_workspace_bytes", "ssm_scan_saved_state_bytes",
     "ssm_scan_checkpoint_steps", "ssm_scan_fwd", "ssm_scan_bwd", "ssm_status_string", "ssm_scan_plan",
     "ssm_scan_fwd_static", "ssm_scan_check_status", "ssm_scan_fwd_state", "ssm_step",
-    "ssm_scan_fwd_fused_dt", "ssm_scan_bwd_fused_dt",
+    "ssm_scan_fwd_fused_dt", "ssm_scan_bwd_fused_dt", "ssm_scan_host_arena_bytes", "ssm_scan_fwd_bwd_host",
 )
 SSM_STATIC_SCRATCH_BYTES = 4 << 20
 
@@ -57,7 +57,8 @@ def load_library() -> ctypes.CDLL:
     lib = ctypes.CDLL(_build.LIB_PATH)
     P = ctypes.POINTER(ssm_problem_t)
     vp, sz = ctypes.c_void_p, ctypes.c_size_t
-    for name in ("ssm_scan_fwd_workspace_bytes", "ssm_scan_bwd_workspace_bytes", "ssm_scan_saved_state_bytes"):
+    for name in ("ssm_scan_fwd_workspace_bytes", "ssm_scan_bwd_workspace_bytes", "ssm_scan_saved_state_bytes",
+                 "ssm_scan_host_arena_bytes"):
         getattr(lib, name).restype = sz
         getattr(lib, name).argtypes = [P]
     lib.ssm_scan_checkpoint_steps.restype = ctypes.c_int32
@@ -80,6 +81,8 @@ def load_library() -> ctypes.CDLL:
     lib.ssm_step.argtypes = [P] + [vp] * 10
     lib.ssm_scan_check_status.restype = ctypes.c_int
     lib.ssm_scan_check_status.argtypes = [P, vp, vp]
+    lib.ssm_scan_fwd_bwd_host.restype = ctypes.c_int
+    lib.ssm_scan_fwd_bwd_host.argtypes = [P] + [vp] * 16 + [vp, sz, vp]
     lib.ssm_scan_fwd_static.restype = ctypes.c_int
     lib.ssm_scan_fwd_static.argtypes = [P] + [vp] * 9 + [vp]
     _lib = lib
@@ -365,3 +368,55 @@ def ssm_scan_bwd(x, delta, A, B, C, D_skip, z, dout, saved_states=None, *, gener
         ctypes.c_void_p(stream_ptr))
     _check(code, "ssm_scan_bwd")
     return o
+
+
+def _host_ptr(t, name, shape, dtype):
+    if t is None:
+        return None
+    if t.is_cuda:
+        raise SsmScanError(f"{name} must be a host tensor")
+    if not t.is_contiguous() or tuple(t.shape) != tuple(shape) or t.dtype != dtype:
+        raise SsmScanError(f"{name}: expected a contiguous host tensor of shape {tuple(shape)} and dtype {dtype}")
+    return ctypes.c_void_p(t.data_ptr())
+
+
+def host_arena_bytes(problem: ssm_problem_t) -> int:
+    return int(load_library().ssm_scan_host_arena_bytes(ctypes.byref(problem)))
+
+
+def ssm_scan_fwd_bwd_host(x, delta, A, B, C, D_skip, z, dout, *, device, arena=None, outputs=None, stream=None,
+                          general_A=False, zoh=False):
+    """Forward + backward of host tensors (page-locked for the copies to overlap), copies included
+    (ssm_scan_fwd_bwd_host).  Returns a dict of host tensors out, dx, ddelta, dz, dB, dC, dA, dD; pass `outputs` to
+    reuse page-locked result tensors and `arena` (a uint8 CUDA tensor of host_arena_bytes) to reuse the device scratch.
+    Enqueues on `stream` (default: torch's current stream of `device`) and does not synchronise."""
+    lib = load_library()
+    device = torch.device(device)
+    batch, L, D = x.shape
+    N = B.shape[-1]
+    prob = make_problem(x, B, z is not None, D_skip is not None, False, general_A, zoh)
+    io = x.dtype
+    need = host_arena_bytes(prob)
+    if arena is None:
+        arena = torch.empty(need, dtype=torch.uint8, device=device)
+    if outputs is None:
+        mk = lambda shape, dt: torch.empty(shape, dtype=dt).pin_memory()
+        outputs = {"out": mk((batch, L, D), io), "dx": mk((batch, L, D), io), "ddelta": mk((batch, L, D), io),
+                   "dz": mk((batch, L, D), io) if z is not None else None, "dB": mk((batch, L, N), io),
+                   "dC": mk((batch, L, N), io), "dA": mk((D, N), torch.float32),
+                   "dD": mk((D,), torch.float32) if D_skip is not None else None}
+    stream_ptr = (stream if stream is not None else torch.cuda.current_stream(device)).cuda_stream
+    f32 = torch.float32
+    with torch.cuda.device(device):
+        code = lib.ssm_scan_fwd_bwd_host(
+            ctypes.byref(prob), _host_ptr(x, "x", (batch, L, D), io), _host_ptr(delta, "delta", (batch, L, D), io),
+            _host_ptr(A, "A", (D, N), f32), _host_ptr(B, "B", (batch, L, N), io), _host_ptr(C, "C", (batch, L, N), io),
+            _host_ptr(D_skip, "D_skip", (D,), f32), _host_ptr(z, "z", (batch, L, D), io),
+            _host_ptr(dout, "dout", (batch, L, D), io),
+            _host_ptr(outputs["out"], "out", (batch, L, D), io), _host_ptr(outputs["dx"], "dx", (batch, L, D), io),
+            _host_ptr(outputs["ddelta"], "ddelta", (batch, L, D), io), _host_ptr(outputs["dA"], "dA", (D, N), f32),
+            _host_ptr(outputs["dB"], "dB", (batch, L, N), io), _host_ptr(outputs["dC"], "dC", (batch, L, N), io),
+            _host_ptr(outputs.get("dD"), "dD", (D,), f32), _host_ptr(outputs.get("dz"), "dz", (batch, L, D), io),
+            _dev_ptr(arena, "device_arena"), ctypes.c_size_t(arena.numel()), ctypes.c_void_p(stream_ptr))
+    _check(code, "ssm_scan_fwd_bwd_host")
+    return outputs
