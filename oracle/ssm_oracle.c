@@ -29,6 +29,9 @@
  * whose partial derivatives are dE/ddelta = a and dE/dA = (delta a - E) / A (delta^2 / 2 at A = 0).  Then
  *   dB[t,n] += lam E x;   dx[t] = ds D_skip + sum_n lam E B;
  *   ddelta[t] = sum_n w A + x sum_n lam a B;   dA[n] += w delta + lam (dE/dA) B x.
+ * With an initial state h0 and an adjoint dh_last flowing into the last state from outside (a later piece of the
+ * same sequence), h[0] = h0, the reverse recurrence starts from a[L+1] lam[L+1] := dh_last, and the gradient of h0 is
+ * dh0[n] = a[1,n] lam[1,n].
  * With the softplus switch the input is the pre-activation v, delta = softplus(v + delta_bias[d]), ddelta is the
  * gradient of v (the line above times sigmoid(v + delta_bias[d])) and dbias[d] = sum over batch and time of ddelta.
  * Sums over channels (dB, dC) and over batch (dA, dD) are taken in a fixed order that does not depend on the
@@ -135,8 +138,9 @@ static inline double zoh_gain_dA(double dt, double An) {
   /* backward: every output is overwritten; dD and dz may be NULL */                                             \
   int ssm_oracle_bwd_##SUFFIX(const oracle_dims_t* p, const REAL* x, const REAL* delta, const double* A,         \
                               const REAL* B, const REAL* C, const double* D_skip, const REAL* z,                 \
-                              const REAL* dout, const double* delta_bias, double* dx, double* ddelta,           \
-                              double* dA, double* dB, double* dC, double* dD, double* dz, double* dbias) {       \
+                              const REAL* dout, const double* delta_bias, const double* h0,                    \
+                              const double* dh_last, double* dx, double* ddelta, double* dA, double* dB,       \
+                              double* dC, double* dD, double* dz, double* dbias, double* dh0) {                  \
     if (!p || p->batch < 1 || p->L < 1 || p->D < 1 || p->N < 1) return 1;                                         \
     const int64_t L = p->L, D = p->D, N = p->N, NB = p->batch;                                                   \
     const int64_t nblk = (D + ORACLE_CH_BLOCK - 1) / ORACLE_CH_BLOCK;                                            \
@@ -155,12 +159,12 @@ static inline double zoh_gain_dA(double dt, double An) {
         const int64_t d0 = blk * ORACLE_CH_BLOCK, d1 = (d0 + ORACLE_CH_BLOCK < D) ? d0 + ORACLE_CH_BLOCK : D;    \
         double* dBp = dBC_part + it * L * N * 2;                                                                 \
         double* dCp = dBp + L * N;                                                                               \
-        double* hs = (double*)malloc((size_t)((L + 1) * N) * sizeof(double));  /* h[0..L][n], h[0] = 0 */        \
+        double* hs = (double*)malloc((size_t)((L + 1) * N) * sizeof(double));  /* h[0..L][n] */                  \
         double* as = (double*)malloc((size_t)((L + 1) * N) * sizeof(double));  /* a[1..L][n] */                  \
         double* ss = (double*)malloc((size_t)(L + 1) * sizeof(double));        /* s[1..L] */                     \
         double lam[p->N];                                                                                        \
         for (int64_t d = d0; d < d1; ++d) {                                                                      \
-          for (int64_t n = 0; n < N; ++n) hs[n] = 0.0;                                                           \
+          for (int64_t n = 0; n < N; ++n) hs[n] = h0 ? h0[(b * D + d) * N + n] : 0.0;                            \
           for (int64_t t = 1; t <= L; ++t) {                                                                     \
             const int64_t e = (b * L + (t - 1)) * D + d;                                                         \
             const double dv = (double)delta[e] + (delta_bias ? delta_bias[d] : 0.0);                             \
@@ -178,7 +182,7 @@ static inline double zoh_gain_dA(double dt, double An) {
             if (p->has_dskip) s += D_skip[d] * u;                                                                \
             ss[t] = s;                                                                                           \
           }                                                                                                      \
-          for (int64_t n = 0; n < N; ++n) lam[n] = 0.0;                                                          \
+          for (int64_t n = 0; n < N; ++n) lam[n] = dh_last ? dh_last[(b * D + d) * N + n] : 0.0;                 \
           double dD_acc = 0.0, dbias_acc = 0.0;                                                                  \
           for (int64_t t = L; t >= 1; --t) {                                                                     \
             const int64_t e = (b * L + (t - 1)) * D + d;                                                         \
@@ -219,6 +223,7 @@ static inline double zoh_gain_dA(double dt, double An) {
             dbias_acc += ddelta[e];                                                                              \
             dD_acc += ds * u;                                                                                    \
           }                                                                                                      \
+          if (dh0) for (int64_t n = 0; n < N; ++n) dh0[(b * D + d) * N + n] = lam[n];                            \
           dD_part[b * D + d] = dD_acc;                                                                           \
           dbias_part[b * D + d] = dbias_acc;                                                                     \
         }                                                                                                        \

@@ -106,13 +106,15 @@ def scan_fwd(x, delta, A, B, C, D_skip=None, z=None, h0=None, zoh=False, nthread
     return res[0] if len(res) == 1 else res
 
 
-def scan_bwd(x, delta, A, B, C, D_skip, z, dout, nthreads=0, delta_softplus=False, delta_bias=None, zoh=False):
+def scan_bwd(x, delta, A, B, C, D_skip, z, dout, nthreads=0, delta_softplus=False, delta_bias=None, zoh=False,
+             h0=None, dh_last=None):
     """Analytic adjoint of scan_fwd for loss = sum(dout * out), sequential, fp64.
 
     Returns a dict with dx, ddelta, dz (batch, L, D); dB, dC (batch, L, N); dA (D, N); dD (D) -- all float64.
     dz is zero when z is None, dD is zero when D_skip is None.  With delta_softplus, `delta` is the pre-activation,
     ddelta its gradient, and the dict also holds ddelta_bias (D) = ddelta summed over batch and time.  `zoh` selects
-    the zero-order-hold B-bar of Eq. 4 as in scan_fwd.
+    the zero-order-hold B-bar of Eq. 4 as in scan_fwd.  `h0` (batch, D, N) is the state before the first step and
+    `dh_last` (batch, D, N) a gradient that reaches the last state from outside; the dict holds dh0 (batch, D, N).
     """
     lib = _load()
     st = _storage_dtype(x)
@@ -127,13 +129,19 @@ def scan_bwd(x, delta, A, B, C, D_skip, z, dout, nthreads=0, delta_softplus=Fals
     g["dA"] = np.empty((D, N), dtype=np.float64)
     g["dD"] = np.empty((D,), dtype=np.float64)
     g["ddelta_bias"] = np.empty((D,), dtype=np.float64)
+    g["dh0"] = np.empty((batch, D, N), dtype=np.float64)
+    H0 = None if h0 is None else np.ascontiguousarray(h0, dtype=np.float64)
+    dHL = None if dh_last is None else np.ascontiguousarray(dh_last, dtype=np.float64)
+    assert H0 is None or H0.shape == (batch, D, N)
+    assert dHL is None or dHL.shape == (batch, D, N)
     bias = None if delta_bias is None else np.ascontiguousarray(delta_bias, dtype=np.float64)
     dims = _Dims(batch, L, D, N, int(z is not None), int(D_skip is not None), int(bool(zoh)), int(bool(delta_softplus)),
                  int(nthreads))
     fn = lib.ssm_oracle_bwd_f32 if st == np.float32 else lib.ssm_oracle_bwd_f64
     rc = fn(ctypes.byref(dims), _ptr(io["x"]), _ptr(io["delta"]), _ptr(A64), _ptr(io["B"]), _ptr(io["C"]), _ptr(Dk),
-            _ptr(io["z"]), _ptr(io["dout"]), _ptr(bias), _ptr(g["dx"]), _ptr(g["ddelta"]), _ptr(g["dA"]), _ptr(g["dB"]),
-            _ptr(g["dC"]), _ptr(g["dD"]), _ptr(g["dz"]), _ptr(g["ddelta_bias"]))
+            _ptr(io["z"]), _ptr(io["dout"]), _ptr(bias), _ptr(H0), _ptr(dHL), _ptr(g["dx"]), _ptr(g["ddelta"]),
+            _ptr(g["dA"]), _ptr(g["dB"]), _ptr(g["dC"]), _ptr(g["dD"]), _ptr(g["dz"]), _ptr(g["ddelta_bias"]),
+            _ptr(g["dh0"]))
     if rc != 0:
         raise RuntimeError(f"ssm_oracle_bwd failed with code {rc}")
     return g

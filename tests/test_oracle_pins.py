@@ -379,3 +379,50 @@ def test_zoh_gradients_match_finite_differences(small_steps):
     pp["A"], pm["A"] = p["A"] + e, p["A"] - e
     fd = (loss(pp) - loss(pm)) / 2e-6
     assert abs(fd - g["dA"][1, 2]) <= 2e-6 * max(1.0, abs(fd))
+
+
+# --------------------------------------------------------------------------------------------------------------
+# Backward with a carried-in state and an adjoint arriving at the last state.
+def test_backward_in_two_pieces_equals_one_backward():
+    # The gradient of a sequence equals the gradients of its two pieces when the second piece starts from the first
+    # piece's last state and hands the first piece the gradient of that state (chain rule across the cut).
+    batch, L, D, N, m = 2, 23, 3, 4, 9
+    p = _rand_problem(batch, L, D, N)
+    dout = RNG.standard_normal((batch, L, D))
+    whole = O.scan_bwd(p["x"], p["delta"], p["A"], p["B"], p["C"], p["D_skip"], p["z"], dout)
+    cut = lambda a, lo, hi: a[:, lo:hi]
+    first = {k: cut(p[k], 0, m) for k in ("x", "delta", "B", "C", "z")}
+    second = {k: cut(p[k], m, L) for k in ("x", "delta", "B", "C", "z")}
+    _, h_m = O.scan_fwd(first["x"], first["delta"], p["A"], first["B"], first["C"], D_skip=p["D_skip"], z=first["z"],
+                        return_h_last=True)
+    g2 = O.scan_bwd(second["x"], second["delta"], p["A"], second["B"], second["C"], p["D_skip"], second["z"],
+                    dout[:, m:], h0=h_m)
+    g1 = O.scan_bwd(first["x"], first["delta"], p["A"], first["B"], first["C"], p["D_skip"], first["z"],
+                    dout[:, :m], dh_last=g2["dh0"])
+    for k in ("dx", "ddelta", "dz", "dB", "dC"):
+        np.testing.assert_allclose(np.concatenate([g1[k], g2[k]], axis=1), whole[k], rtol=1e-11, atol=1e-12)
+    for k in ("dA", "dD"):
+        np.testing.assert_allclose(g1[k] + g2[k], whole[k], rtol=1e-11, atol=1e-12)
+    assert np.all(whole["dh0"] == g1["dh0"]) or np.allclose(whole["dh0"], g1["dh0"], rtol=1e-11, atol=1e-13)
+
+
+def test_initial_state_gradient_matches_finite_differences():
+    batch, L, D, N = 2, 8, 3, 4
+    p = _rand_problem(batch, L, D, N)
+    h0 = RNG.standard_normal((batch, D, N))
+    dhl = RNG.standard_normal((batch, D, N))
+    dout = RNG.standard_normal((batch, L, D))
+
+    def loss(hh, xx=None):
+        out, hl = O.scan_fwd(p["x"] if xx is None else xx, p["delta"], p["A"], p["B"], p["C"], D_skip=p["D_skip"],
+                             z=p["z"], h0=hh, return_h_last=True)
+        return float((dout * out).sum() + (dhl * hl).sum())
+    g = O.scan_bwd(p["x"], p["delta"], p["A"], p["B"], p["C"], p["D_skip"], p["z"], dout, h0=h0, dh_last=dhl)
+    eps = 1e-6
+    for trial in range(3):
+        v = RNG.standard_normal(h0.shape)
+        fd = (loss(h0 + eps * v) - loss(h0 - eps * v)) / (2 * eps)
+        assert abs(fd - (g["dh0"] * v).sum()) <= 1e-6 * max(1.0, abs(fd))
+        vx = RNG.standard_normal(p["x"].shape)       # dh_last must reach the other gradients too
+        fd = (loss(h0, p["x"] + eps * vx) - loss(h0, p["x"] - eps * vx)) / (2 * eps)
+        assert abs(fd - (g["dx"] * vx).sum()) <= 1e-6 * max(1.0, abs(fd))
