@@ -117,8 +117,8 @@ SSM_API ssm_status_t ssm_scan_fwd(const ssm_problem_t* p, const void* x, const v
  *   h0        in, float32 [batch][D][N]: the state before the first step (NULL: zero)
  *   h_last    out, float32 [batch][D][N]: the state after the last step (NULL: not wanted)
  * Checkpoint states written with SSM_FLAG_SAVE_STATES include the effect of h0, so ssm_scan_bwd given those saved
- * states returns the gradients of this call's inputs; the gradient with respect to h0 itself is not produced, and
- * ssm_scan_bwd without saved states assumes h0 = 0.
+ * states returns the gradients of this call's inputs; ssm_scan_bwd_state also returns the gradient with respect to
+ * h0 and accepts h0 when it has to rebuild the checkpoints (plain ssm_scan_bwd without saved states assumes h0 = 0).
  */
 SSM_API ssm_status_t ssm_scan_fwd_state(const ssm_problem_t* p, const void* x, const void* delta, const float* A,
                                         const void* B, const void* C, const float* D_skip, const void* z,
@@ -178,6 +178,25 @@ SSM_API ssm_status_t ssm_scan_bwd(const ssm_problem_t* p, const void* x, const v
                           const void* C, const float* D_skip, const void* z, const void* dout,
                           const void* saved_states, void* dx, void* ddelta, float* dA, void* dB, void* dC, float* dD,
                           void* dz, void* workspace, size_t workspace_bytes, void* stream /* cudaStream_t */);
+
+/*
+ * Backward of a piece of a longer sequence (the counterpart of ssm_scan_fwd_state; Appendix D: the scan is continued
+ * chunk by chunk through the intermediate states, and the chain rule crosses a cut the same way).  Same as
+ * ssm_scan_bwd, plus
+ *   h0        in, float32 [batch][D][N]: the state before the first step, as given to ssm_scan_fwd_state (NULL: zero);
+ *             only read when saved_states is NULL (saved states already contain its effect)
+ *   dh_last   in, float32 [batch][D][N]: gradient of the loss with respect to the state after the last step that
+ *             arrives from outside this piece (the dh0 of the following piece); NULL: zero
+ *   dh0       out, float32 [batch][D][N]: gradient with respect to h0; NULL: not wanted
+ * Walking the pieces of a sequence from last to first, passing each piece's dh0 as the previous piece's dh_last, gives
+ * the gradients of the whole sequence (dA and dD of the pieces add up).
+ */
+SSM_API ssm_status_t ssm_scan_bwd_state(const ssm_problem_t* p, const void* x, const void* delta, const float* A,
+                                        const void* B, const void* C, const float* D_skip, const void* z,
+                                        const void* dout, const float* h0, const float* dh_last,
+                                        const void* saved_states, void* dx, void* ddelta, float* dA, void* dB, void* dC,
+                                        float* dD, void* dz, float* dh0, void* workspace, size_t workspace_bytes,
+                                        void* stream /* cudaStream_t */);
 
 /*
  * Reads back whether the last ssm_scan_bwd on this workspace completed.  The tuned backward kernel passes the adjoint

@@ -24,6 +24,7 @@ EXPORTED_SYMBOLS = (
     "ssm_scan_checkpoint_steps", "ssm_scan_fwd", "ssm_scan_bwd", "ssm_status_string", "ssm_scan_plan",
     "ssm_scan_fwd_static", "ssm_scan_check_status", "ssm_scan_fwd_state", "ssm_step",
     "ssm_scan_fwd_fused_dt", "ssm_scan_bwd_fused_dt", "ssm_scan_host_arena_bytes", "ssm_scan_fwd_bwd_host",
+    "ssm_scan_bwd_state",
 )
 SSM_STATIC_SCRATCH_BYTES = 4 << 20
 
@@ -71,6 +72,8 @@ def load_library() -> ctypes.CDLL:
     lib.ssm_scan_fwd.argtypes = [P] + [vp] * 9 + [vp, sz, vp]
     lib.ssm_scan_bwd.restype = ctypes.c_int
     lib.ssm_scan_bwd.argtypes = [P] + [vp] * 16 + [vp, sz, vp]
+    lib.ssm_scan_bwd_state.restype = ctypes.c_int
+    lib.ssm_scan_bwd_state.argtypes = [P] + [vp] * 19 + [vp, sz, vp]
     lib.ssm_scan_fwd_state.restype = ctypes.c_int
     lib.ssm_scan_fwd_state.argtypes = [P] + [vp] * 11 + [vp, sz, vp]
     lib.ssm_scan_fwd_fused_dt.restype = ctypes.c_int
@@ -326,11 +329,14 @@ def ssm_scan_fwd_static(x, delta, A, B, C, D_skip=None, z=None, *, save_states=F
 
 
 def ssm_scan_bwd(x, delta, A, B, C, D_skip, z, dout, saved_states=None, *, general_A=False, zoh=False, workspace=None,
-                 stream=None, outputs=None, extra_flags=0):
+                 stream=None, outputs=None, extra_flags=0, h0=None, dh_last=None, want_dh0=False):
     """Gradients of sum(dout * out) w.r.t. x, delta, A, B, C, D_skip, z; see include/ssm_scan.h.
 
     Returns a dict with dx, ddelta, dz (io dtype, (batch, L, D)); dB, dC (io dtype, (batch, L, N)); dA (float32, (D, N));
     dD (float32, (D)).  dz / dD are None when z / D_skip is None.  `outputs` may pass preallocated tensors.
+    With h0, dh_last or want_dh0 the call goes through ssm_scan_bwd_state: h0 / dh_last (batch, D, N) float32 are the
+    state before the first step and the gradient arriving at the state after the last step, and the dict also holds
+    dh0 (batch, D, N) float32.
     """
     lib = load_library()
     prob = make_problem(x, B, z is not None, D_skip is not None, False, general_A, zoh)
@@ -354,6 +360,24 @@ def ssm_scan_bwd(x, delta, A, B, C, D_skip, z, dout, saved_states=None, *, gener
     stream_ptr = (stream if stream is not None else torch.cuda.current_stream(x.device)).cuda_stream
     need = bwd_workspace_bytes(prob)
     ws = workspace if workspace is not None else _workspace(need, x.device, stream_ptr)
+    if h0 is not None or dh_last is not None or want_dh0:
+        f32 = torch.float32
+        if want_dh0:
+            o.setdefault("dh0", torch.empty((batch, D, N), dtype=f32, device=x.device))
+        code = lib.ssm_scan_bwd_state(
+            ctypes.byref(prob), _dev_ptr(x, "x", (batch, L, D), io), _dev_ptr(delta, "delta", (batch, L, D), io),
+            _dev_ptr(A, "A", (D, N), f32), _dev_ptr(B, "B", (batch, L, N), io), _dev_ptr(C, "C", (batch, L, N), io),
+            _dev_ptr(D_skip, "D_skip", (D,), f32), _dev_ptr(z, "z", (batch, L, D), io),
+            _dev_ptr(dout, "dout", (batch, L, D), io), _dev_ptr(h0, "h0", (batch, D, N), f32),
+            _dev_ptr(dh_last, "dh_last", (batch, D, N), f32), _dev_ptr(saved_states, "saved_states"),
+            _dev_ptr(o["dx"], "dx", (batch, L, D), io), _dev_ptr(o["ddelta"], "ddelta", (batch, L, D), io),
+            _dev_ptr(o["dA"], "dA", (D, N), f32), _dev_ptr(o["dB"], "dB", (batch, L, N), io),
+            _dev_ptr(o["dC"], "dC", (batch, L, N), io), _dev_ptr(o["dD"], "dD", (D,), f32),
+            _dev_ptr(o["dz"], "dz", (batch, L, D), io), _dev_ptr(o.get("dh0"), "dh0", (batch, D, N), f32),
+            _dev_ptr(ws, "workspace"), ctypes.c_size_t(0 if ws is None else ws.numel() * ws.element_size()),
+            ctypes.c_void_p(stream_ptr))
+        _check(code, "ssm_scan_bwd_state")
+        return o
     code = lib.ssm_scan_bwd(
         ctypes.byref(prob), _dev_ptr(x, "x", (batch, L, D), io), _dev_ptr(delta, "delta", (batch, L, D), io),
         _dev_ptr(A, "A", (D, N), torch.float32), _dev_ptr(B, "B", (batch, L, N), io),

@@ -301,9 +301,9 @@ ssm_status_t ssm_step(const ssm_problem_t* p, const void* x, const void* delta, 
 
 static ssm_status_t bwd_impl(const ssm_problem_t* p, const void* x, const void* delta, const float* delta_bias,
                              const float* A, const void* B, const void* C, const float* D_skip, const void* z,
-                             const void* dout, const void* saved_states, void* dx, void* ddelta, float* ddelta_bias,
-                             float* dA, void* dB, void* dC, float* dD, void* dz, void* workspace,
-                             size_t workspace_bytes, void* stream) {
+                             const void* dout, const float* h0, const float* dh_last, const void* saved_states,
+                             void* dx, void* ddelta, float* ddelta_bias, float* dA, void* dB, void* dC, float* dD,
+                             void* dz, float* dh0, void* workspace, size_t workspace_bytes, void* stream) {
   ssm_status_t st = validate_problem(p);
   if (st != SSM_OK) return st;
   const bool has_z = p->flags & SSM_FLAG_HAS_Z, has_d = p->flags & SSM_FLAG_HAS_DSKIP;
@@ -314,7 +314,8 @@ static ssm_status_t bwd_impl(const ssm_problem_t* p, const void* x, const void* 
                         (const void*)dC, (const void*)dz})
     if (q && !aligned_to(q, esz)) return SSM_ERR_INVALID_ARG;
   for (const void* q : {(const void*)A, (const void*)D_skip, saved_states, (const void*)dA, (const void*)dD,
-                        (const void*)delta_bias, (const void*)ddelta_bias})
+                        (const void*)delta_bias, (const void*)ddelta_bias, (const void*)h0, (const void*)dh_last,
+                        (const void*)dh0})
     if (q && !aligned_to(q, 4)) return SSM_ERR_INVALID_ARG;
   const Plan pl = make_plan(*p);
   const BwdWorkspace w = bwd_layout(*p, pl);
@@ -344,7 +345,7 @@ static ssm_status_t bwd_impl(const ssm_problem_t* p, const void* x, const void* 
     fp.delta_bias = delta_bias;
     fp.softplus = (p->flags & SSM_FLAG_DELTA_SOFTPLUS) ? 1 : 0;
     const float* h_start = nullptr;
-    if (run_segment_starts(*p, pl, fp, ws + w.fwd, nullptr, &h_start, s) != cudaSuccess) return SSM_ERR_CUDA;
+    if (run_segment_starts(*p, pl, fp, ws + w.fwd, h0, &h_start, s) != cudaSuccess) return SSM_ERR_CUDA;
     fp.h_start = h_start;
     fp.ckpt = reinterpret_cast<float*>(ws + w.ckpt);
     if (launch_fwd(*p, pl, fp, kFwdCkptOnly, s) != cudaSuccess) return SSM_ERR_CUDA;
@@ -379,6 +380,8 @@ static ssm_status_t bwd_impl(const ssm_problem_t* p, const void* x, const void* 
   bp.test_withhold = (p->flags & SSM_FLAG_TEST_WITHHOLD) ? 1 : 0;
   bp.delta_bias = delta_bias;
   bp.softplus = (p->flags & SSM_FLAG_DELTA_SOFTPLUS) ? 1 : 0;
+  bp.dh0 = dh0;
+  bp.mu_in = dh_last;  // one segment: [batch][1][D][N] is the layout of the caller's adjoint
   bp.dbias_part = ddelta_bias != nullptr ? reinterpret_cast<float*>(ws + w.dbias_part) : nullptr;
   bp.sched = reinterpret_cast<int*>(ws + w.sched);
   bp.handoff = reinterpret_cast<float4*>(ws + w.handoff);
@@ -400,6 +403,7 @@ static ssm_status_t bwd_impl(const ssm_problem_t* p, const void* x, const void* 
     cp.D = p->D;
     cp.N = p->N;
     cp.reverse = 1;
+    cp.init = dh_last;
     if (launch_carry(cp, s) != cudaSuccess) return SSM_ERR_CUDA;
     bp.mu_in = cp.carried;
   }
@@ -428,8 +432,17 @@ ssm_status_t ssm_scan_bwd(const ssm_problem_t* p, const void* x, const void* del
                           const void* C, const float* D_skip, const void* z, const void* dout,
                           const void* saved_states, void* dx, void* ddelta, float* dA, void* dB, void* dC, float* dD,
                           void* dz, void* workspace, size_t workspace_bytes, void* stream) {
-  return bwd_impl(p, x, delta, nullptr, A, B, C, D_skip, z, dout, saved_states, dx, ddelta, nullptr, dA, dB, dC, dD, dz,
-                  workspace, workspace_bytes, stream);
+  return bwd_impl(p, x, delta, nullptr, A, B, C, D_skip, z, dout, nullptr, nullptr, saved_states, dx, ddelta, nullptr,
+                  dA, dB, dC, dD, dz, nullptr, workspace, workspace_bytes, stream);
+}
+
+ssm_status_t ssm_scan_bwd_state(const ssm_problem_t* p, const void* x, const void* delta, const float* A, const void* B,
+                                const void* C, const float* D_skip, const void* z, const void* dout, const float* h0,
+                                const float* dh_last, const void* saved_states, void* dx, void* ddelta, float* dA,
+                                void* dB, void* dC, float* dD, void* dz, float* dh0, void* workspace,
+                                size_t workspace_bytes, void* stream) {
+  return bwd_impl(p, x, delta, nullptr, A, B, C, D_skip, z, dout, h0, dh_last, saved_states, dx, ddelta, nullptr, dA,
+                  dB, dC, dD, dz, dh0, workspace, workspace_bytes, stream);
 }
 
 ssm_status_t ssm_scan_bwd_fused_dt(const ssm_problem_t* p, const void* x, const void* delta_pre,
@@ -437,8 +450,8 @@ ssm_status_t ssm_scan_bwd_fused_dt(const ssm_problem_t* p, const void* x, const 
                                    const float* D_skip, const void* z, const void* dout, const void* saved_states,
                                    void* dx, void* ddelta_pre, float* ddelta_bias, float* dA, void* dB, void* dC,
                                    float* dD, void* dz, void* workspace, size_t workspace_bytes, void* stream) {
-  return bwd_impl(p, x, delta_pre, delta_bias, A, B, C, D_skip, z, dout, saved_states, dx, ddelta_pre, ddelta_bias, dA,
-                  dB, dC, dD, dz, workspace, workspace_bytes, stream);
+  return bwd_impl(p, x, delta_pre, delta_bias, A, B, C, D_skip, z, dout, nullptr, nullptr, saved_states, dx, ddelta_pre,
+                  ddelta_bias, dA, dB, dC, dD, dz, nullptr, workspace, workspace_bytes, stream);
 }
 
 }  // extern "C"

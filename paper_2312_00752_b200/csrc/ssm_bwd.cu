@@ -251,6 +251,10 @@ __global__ void __launch_bounds__(BwdGeom<N>::THREADS) ssm_bwd_kernel(const BwdP
     for (int k = 0; k < S; ++k) p.dA_part[(part * D + d) * N + j * S + k] = dA[k];
     if (j == 0) p.dD_part[part * D + d] = dD_acc;
     if (j == 0 && p.dbias_part != nullptr) p.dbias_part[part * D + d] = dbias_acc;
+    if (seg == 0 && p.dh0 != nullptr) {
+#pragma unroll
+      for (int k = 0; k < S; ++k) p.dh0[((size_t)b * D + d) * N + j * S + k] = mu[k];
+    }
   }
 }
 

@@ -527,6 +527,13 @@ __global__ void __launch_bounds__(kBwdFastThreads) ssm_bwd_fast_kernel(const Bwd
             *reinterpret_cast<float4*>(p.dA_part + (part * D + chan(q)) * 16 + 4 * j) =
                 make_float4(dA2[q][0].x, dA2[q][0].y, dA2[q][1].x, dA2[q][1].y);
         }
+        if (valid && cur.seg == 0 && p.dh0 != nullptr) {
+          // the adjoint that leaves the first step is the gradient of the initial state
+#pragma unroll
+          for (int q = 0; q < 2; ++q)
+            *reinterpret_cast<float4*>(p.dh0 + ((size_t)cur.b * D + chan(q)) * 16 + 4 * j) =
+                make_float4(mu[q][0].x, mu[q][0].y, mu[q][1].x, mu[q][1].y);
+        }
         // dD: lanes j and j^2 accumulated disjoint steps of the same channel
         const float dsum2 = dD_acc + __shfl_xor_sync(0xffffffffu, dD_acc, 2);
         if (valid && j < 2) p.dD_part[((size_t)cur.b * p.nseg + cur.seg) * D + d0 + pq] = dsum2;
@@ -548,7 +555,7 @@ bool bwd_fast_applicable(const ssm_problem_t& prob, const BwdParams& p) {
   if (p.zoh) return false;  // the tuned kernel implements the default rule B-bar = delta * B only
   return prob.io_dtype == SSM_BF16 && prob.N == 16 && prob.D % 8 == 0 && p.seg_steps % kBT == 0 && al16(p.x) &&
          al16(p.delta) && al16(p.z) && al16(p.B) && al16(p.C) && al16(p.dout) && al16(p.dx) && al16(p.ddelta) &&
-         al16(p.dz) && al16(p.A) && al16(p.ckpt) && al16(p.mu_in) && al16(p.dBC_part) && al16(p.dA_part) &&
+         al16(p.dz) && al16(p.A) && al16(p.ckpt) && al16(p.mu_in) && al16(p.dh0) && al16(p.dBC_part) && al16(p.dA_part) &&
          p.sched != nullptr && p.handoff != nullptr;
 }
 

@@ -85,6 +85,8 @@ struct BwdParams {
   const float* delta_bias;  // as in FwdParams
   int softplus;
   float* dbias_part;      // [batch*nseg][D] sums of the pre-activation gradient; null: not wanted
+  float* dh0;             // [batch][D][N] gradient of the initial state (the adjoint mu that leaves the first step);
+                          // null: not wanted
   int zoh;                // as in FwdParams
   int test_withhold;      // test hook: never publish hand-off flags, poll only 1000 times
   int* sched;             // tuned kernel: [0] claim counter, [1] abort word, [64 + chain] progress flag per chain

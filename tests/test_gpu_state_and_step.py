@@ -106,3 +106,41 @@ def test_saved_states_carry_h0_into_backward():
     g = K.ssm_scan_bwd(*args2, sl("dout", cut, L), saved)
     for k in ("dx", "ddelta", "dz", "dB", "dC"):
         assert U.rel_err(U.to_host(g[k]), ref[k][:, cut:]) <= U.TOL[io]["grad"], k
+
+
+@pytest.mark.parametrize("batch,L,D,N,io,cut,saved", [
+    (2, 300, 40, 16, "bf16", 130, True),       # tuned kernels
+    (2, 300, 40, 16, "bf16", 130, False),      # ... with the checkpoints rebuilt from h0
+    (1, 200, 24, 8, "f32", 77, True),          # generic kernels
+    (1, 200, 24, 8, "f32", 77, False),
+    (1, 6000, 64, 16, "bf16", 2048, True),     # both pieces split time: dh_last enters the reverse carry
+])
+def test_backward_in_two_pieces(batch, L, D, N, io, cut, saved):
+    import torch
+    from oracle import ssm_oracle as O
+    from paper_2312_00752_b200 import binding as K
+    cfg = synth.ScanConfig("state", 12, batch, L, D, N, io, *((1e-4, 1e-2) if L > 1000 else (1e-3, 1e-1)))
+    inp = synth.make_inputs(cfg, seed=3)
+    dev = U.to_device(inp, io)
+    ref = O.scan_bwd(inp["x"], inp["delta"], inp["A"], inp["B"], inp["C"], inp["D_skip"], inp["z"], inp["dout"])
+    sl = lambda k, a, b: dev[k][:, a:b].contiguous()
+    piece = lambda a, b: (sl("x", a, b), sl("delta", a, b), dev["A"], sl("B", a, b), sl("C", a, b), dev["D_skip"],
+                          sl("z", a, b))
+    h_mid = torch.empty((batch, D, N), dtype=torch.float32, device="cuda")
+    _, sv1 = K.ssm_scan_fwd(*piece(0, cut), save_states=True, h_last=h_mid)
+    _, sv2 = K.ssm_scan_fwd(*piece(cut, L), save_states=True, h0=h_mid)
+    g2 = K.ssm_scan_bwd(*piece(cut, L), sl("dout", cut, L), sv2 if saved else None, h0=h_mid, want_dh0=True)
+    g1 = K.ssm_scan_bwd(*piece(0, cut), sl("dout", 0, cut), sv1 if saved else None, dh_last=g2["dh0"], want_dh0=True)
+    tol = U.TOL[io]["grad"]
+    for k in ("dx", "ddelta", "dz", "dB", "dC"):
+        got = np.concatenate([U.to_host(g1[k]), U.to_host(g2[k])], axis=1)
+        assert U.rel_err(got, ref[k]) <= tol, k
+    for k in ("dA", "dD"):
+        assert U.rel_err(U.to_host(g1[k]) + U.to_host(g2[k]), ref[k]) <= tol, k
+    # the gradient of the state at the cut, against the oracle's for the second piece alone
+    mid = {k: (v[:, cut:] if v.ndim == 3 and v.shape[1] == L else v) for k, v in inp.items()}
+    _, h_m = O.scan_fwd(inp["x"][:, :cut], inp["delta"][:, :cut], inp["A"], inp["B"][:, :cut], inp["C"][:, :cut],
+                        D_skip=inp["D_skip"], z=inp["z"][:, :cut], return_h_last=True)
+    r2 = O.scan_bwd(mid["x"], mid["delta"], mid["A"], mid["B"], mid["C"], mid["D_skip"], mid["z"], mid["dout"], h0=h_m)
+    assert U.rel_err(U.to_host(g2["dh0"]), r2["dh0"]) <= (1e-4 if io == "f32" else 3e-2)
+    assert U.rel_err(U.to_host(g1["dh0"]), ref["dh0"]) <= (1e-4 if io == "f32" else 3e-2)
