@@ -24,9 +24,17 @@ EXPORTED_SYMBOLS = (
     "ssm_scan_checkpoint_steps", "ssm_scan_fwd", "ssm_scan_bwd", "ssm_status_string", "ssm_scan_plan",
     "ssm_scan_fwd_static", "ssm_scan_check_status", "ssm_scan_fwd_state", "ssm_step",
     "ssm_scan_fwd_fused_dt", "ssm_scan_bwd_fused_dt", "ssm_scan_host_arena_bytes", "ssm_scan_fwd_bwd_host",
-    "ssm_scan_bwd_state",
+    "ssm_scan_bwd_state", "ssm_conv1d_fwd", "ssm_conv1d_bwd_workspace_bytes", "ssm_conv1d_bwd",
 )
 SSM_STATIC_SCRATCH_BYTES = 4 << 20
+
+
+SSM_CONV_FLAG_SILU, SSM_CONV_FLAG_HAS_BIAS = 1, 2
+
+
+class ssm_conv_problem_t(ctypes.Structure):
+    _fields_ = [("batch", ctypes.c_int32), ("L", ctypes.c_int32), ("D", ctypes.c_int32), ("width", ctypes.c_int32),
+                ("io_dtype", ctypes.c_int32), ("flags", ctypes.c_uint32)]
 
 
 class ssm_problem_t(ctypes.Structure):
@@ -72,6 +80,13 @@ def load_library() -> ctypes.CDLL:
     lib.ssm_scan_fwd.argtypes = [P] + [vp] * 9 + [vp, sz, vp]
     lib.ssm_scan_bwd.restype = ctypes.c_int
     lib.ssm_scan_bwd.argtypes = [P] + [vp] * 16 + [vp, sz, vp]
+    CP = ctypes.POINTER(ssm_conv_problem_t)
+    lib.ssm_conv1d_fwd.restype = ctypes.c_int
+    lib.ssm_conv1d_fwd.argtypes = [CP] + [vp] * 5 + [vp]
+    lib.ssm_conv1d_bwd_workspace_bytes.restype = sz
+    lib.ssm_conv1d_bwd_workspace_bytes.argtypes = [CP]
+    lib.ssm_conv1d_bwd.restype = ctypes.c_int
+    lib.ssm_conv1d_bwd.argtypes = [CP] + [vp] * 9 + [vp, sz, vp]
     lib.ssm_scan_bwd_state.restype = ctypes.c_int
     lib.ssm_scan_bwd_state.argtypes = [P] + [vp] * 19 + [vp, sz, vp]
     lib.ssm_scan_fwd_state.restype = ctypes.c_int
@@ -444,3 +459,57 @@ def ssm_scan_fwd_bwd_host(x, delta, A, B, C, D_skip, z, dout, *, device, arena=N
             _dev_ptr(arena, "device_arena"), ctypes.c_size_t(arena.numel()), ctypes.c_void_p(stream_ptr))
     _check(code, "ssm_scan_fwd_bwd_host")
     return outputs
+
+
+def make_conv_problem(x: torch.Tensor, w: torch.Tensor, silu: bool, has_bias: bool) -> ssm_conv_problem_t:
+    batch, L, D = x.shape
+    return ssm_conv_problem_t(batch, L, D, w.shape[1], _io_dtype(x),
+                              (SSM_CONV_FLAG_SILU if silu else 0) | (SSM_CONV_FLAG_HAS_BIAS if has_bias else 0))
+
+
+def ssm_conv1d_fwd(x, w, bias=None, *, silu=True, x_prev=None, out=None, stream=None):
+    """y = silu(causal depthwise conv1d(x; w) + bias), see include/ssm_conv1d.h.  x (batch, L, D) io dtype; w (D, W)
+    float32 with the last tap on the current step; bias (D) float32 or None; x_prev (batch, W-1, D) io dtype or None."""
+    lib = load_library()
+    prob = make_conv_problem(x, w, silu, bias is not None)
+    batch, L, D, W = prob.batch, prob.L, prob.D, prob.width
+    io = x.dtype
+    if out is None:
+        out = torch.empty_like(x)
+    stream_ptr = (stream if stream is not None else torch.cuda.current_stream(x.device)).cuda_stream
+    code = lib.ssm_conv1d_fwd(ctypes.byref(prob), _dev_ptr(x, "x", (batch, L, D), io),
+                              _dev_ptr(w, "w", (D, W), torch.float32), _dev_ptr(bias, "bias", (D,), torch.float32),
+                              _dev_ptr(x_prev, "x_prev", (batch, W - 1, D), io), _dev_ptr(out, "y", (batch, L, D), io),
+                              ctypes.c_void_p(stream_ptr))
+    _check(code, "ssm_conv1d_fwd")
+    return out
+
+
+def ssm_conv1d_bwd(x, w, bias, dy, *, silu=True, x_prev=None, want_dx_prev=False, outputs=None, stream=None):
+    """Gradients of sum(dy * y) of ssm_conv1d_fwd: dict with dx (io dtype), dw (D, W) and dbias (D) float32 (dbias None
+    without bias), and dx_prev (batch, W-1, D) if asked for."""
+    lib = load_library()
+    prob = make_conv_problem(x, w, silu, bias is not None)
+    batch, L, D, W = prob.batch, prob.L, prob.D, prob.width
+    io = x.dtype
+    o = dict(outputs or {})
+    o.setdefault("dx", torch.empty_like(x))
+    o.setdefault("dw", torch.empty((D, W), dtype=torch.float32, device=x.device))
+    if bias is not None:
+        o.setdefault("dbias", torch.empty((D,), dtype=torch.float32, device=x.device))
+    else:
+        o["dbias"] = None
+    if want_dx_prev and W > 1:
+        o.setdefault("dx_prev", torch.empty((batch, W - 1, D), dtype=io, device=x.device))
+    stream_ptr = (stream if stream is not None else torch.cuda.current_stream(x.device)).cuda_stream
+    ws = _workspace(int(lib.ssm_conv1d_bwd_workspace_bytes(ctypes.byref(prob))), x.device, stream_ptr)
+    code = lib.ssm_conv1d_bwd(ctypes.byref(prob), _dev_ptr(x, "x", (batch, L, D), io),
+                              _dev_ptr(w, "w", (D, W), torch.float32), _dev_ptr(bias, "bias", (D,), torch.float32),
+                              _dev_ptr(x_prev, "x_prev", (batch, W - 1, D), io), _dev_ptr(dy, "dy", (batch, L, D), io),
+                              _dev_ptr(o["dx"], "dx", (batch, L, D), io), _dev_ptr(o["dw"], "dw", (D, W), torch.float32),
+                              _dev_ptr(o["dbias"], "dbias", (D,), torch.float32),
+                              _dev_ptr(o.get("dx_prev"), "dx_prev", (batch, W - 1, D), io),
+                              _dev_ptr(ws, "workspace"), ctypes.c_size_t(0 if ws is None else ws.numel() * ws.element_size()),
+                              ctypes.c_void_p(stream_ptr))
+    _check(code, "ssm_conv1d_bwd")
+    return o

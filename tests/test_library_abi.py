@@ -12,7 +12,8 @@ ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 
 
 def _declared_symbols():
-    text = open(os.path.join(ROOT, "include", "ssm_scan.h")).read()
+    import glob
+    text = "".join(open(h).read() for h in sorted(glob.glob(os.path.join(ROOT, "include", "*.h"))))
     return sorted(set(re.findall(r"SSM_API[^;(]*?\b(ssm_\w+)\s*\(", text)))
 
 
@@ -73,3 +74,21 @@ def test_null_misaligned_and_workspace_errors_before_launch():
     assert lib.ssm_scan_bwd(ctypes.byref(p), *b16, None, 0, None) == 3
     assert lib.ssm_scan_bwd(ctypes.byref(p), *b16[:7], None, *b16[8:], None, 0, None) == 1       # dout missing
     assert "WORKSPACE" in K.status_string(3) and K.status_string(0) == "SSM_OK"
+
+
+def test_conv1d_argument_errors_before_launch():
+    lib = K.load_library()
+    a = ctypes.c_void_p(4096)
+    ok = K.ssm_conv_problem_t(2, 100, 64, 4, K.SSM_BF16, 3)
+    assert lib.ssm_conv1d_fwd(ctypes.byref(ok), None, a, a, None, a, None) == 1                  # x missing
+    assert lib.ssm_conv1d_fwd(ctypes.byref(ok), a, a, None, None, a, None) == 1                  # bias flagged, missing
+    for bad, code in [(dict(width=5), 2), (dict(width=0), 2), (dict(io=7), 2), (dict(L=0), 1), (dict(flags=8), 1)]:
+        f = dict(batch=2, L=100, D=64, width=4, io=K.SSM_BF16, flags=3)
+        f.update(bad)
+        p = K.ssm_conv_problem_t(f["batch"], f["L"], f["D"], f["width"], f["io"], f["flags"])
+        assert lib.ssm_conv1d_fwd(ctypes.byref(p), a, a, a, None, a, None) == code
+        assert lib.ssm_conv1d_bwd_workspace_bytes(ctypes.byref(p)) == 0
+    need = lib.ssm_conv1d_bwd_workspace_bytes(ctypes.byref(ok))
+    assert need == 2 * 4 * 64 * 5 * 4                                                            # room for 4 chunks of 32 steps
+    assert lib.ssm_conv1d_bwd(ctypes.byref(ok), a, a, a, None, a, a, a, a, None, None, 0, None) == 3
+    assert lib.ssm_conv1d_bwd(ctypes.byref(ok), a, a, a, None, a, a, a, a, None, a, need - 1, None) == 3
