@@ -388,6 +388,37 @@ def run_ours(args, cfg):
                                "note": "state (42 MB) stays in L2 between repetitions; a launch-latency-sized kernel"}
     except Exception as exc:  # the headline numbers do not depend on this extra
         line["decode_step"] = {"error": str(exc)}
+    # the neighbour of the scan on the SSM branch: short causal depthwise convolution + SiLU (HBM-bound streaming kernels)
+    try:
+        cw = torch.randn((cfg.D, 4), device=dev) * 0.5
+        cb = torch.randn((cfg.D,), device=dev) * 0.1
+        cy = torch.empty_like(d0["x"])
+        cg = {"dx": grads["dx"], "dw": torch.empty_like(cw), "dbias": torch.empty_like(cb)}
+
+        def time_calls(fn, n=30):
+            for i in range(5):
+                fn(i)
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            for i in range(n):
+                fn(i)
+            b.record(stream)
+            torch.cuda.synchronize(dev)
+            return a.elapsed_time(b) / n * 1e3
+
+        f_us = time_calls(lambda i: K.ssm_conv1d_fwd(sets[i % NSETS]["x"], cw, cb, out=cy, stream=stream))
+        b_us = time_calls(lambda i: K.ssm_conv1d_bwd(sets[i % NSETS]["x"], cw, cb, sets[i % NSETS]["dout"], outputs=cg,
+                                                     stream=stream))
+        esz = 2 if cfg.io == "bf16" else 4
+        fb, bb = 2 * esz * cfg.elements, 3 * esz * cfg.elements
+        line["conv1d"] = {"width": 4, "fwd_us": f_us, "bwd_us": b_us, "fwd_algorithmic_bytes": fb,
+                          "bwd_algorithmic_bytes": bb, "fwd_gbs": fb / (f_us * 1e-6) / 1e9,
+                          "bwd_gbs": bb / (b_us * 1e-6) / 1e9, "fwd_frac_of_hbm_peak": fb / (f_us * 1e-6) / 1e9 / peak,
+                          "bwd_frac_of_hbm_peak": bb / (b_us * 1e-6) / 1e9 / peak,
+                          "note": "ssm_conv1d_fwd / ssm_conv1d_bwd (incl. its reduction kernel) on the workload's x and "
+                                  "dout, input sets rotated; includes the host cost of one Python call per launch"}
+    except Exception as exc:  # the headline numbers do not depend on this extra
+        line["conv1d"] = {"error": str(exc)}
     if e2e is not None:
         line["e2e"] = e2e
     if not args.no_cpu_baseline and world >= 1:

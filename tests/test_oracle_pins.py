@@ -426,3 +426,25 @@ def test_initial_state_gradient_matches_finite_differences():
         vx = RNG.standard_normal(p["x"].shape)       # dh_last must reach the other gradients too
         fd = (loss(h0, p["x"] + eps * vx) - loss(h0, p["x"] - eps * vx)) / (2 * eps)
         assert abs(fd - (g["dx"] * vx).sum()) <= 1e-6 * max(1.0, abs(fd))
+
+
+# --------------------------------------------------------------------------------------------------------------
+# Regression anchor: the stored outputs of the oracle on a tiny seeded problem (tests/golden/, written by a committed
+# script that calls only the oracle; the paper prints no worked example to store instead).
+def test_oracle_reproduces_its_stored_tiny_problem():
+    import importlib.util
+    import os
+    here = os.path.join(os.path.dirname(os.path.abspath(__file__)), "golden")
+    spec = importlib.util.spec_from_file_location("make_golden", os.path.join(here, "make_golden.py"))
+    mg = importlib.util.module_from_spec(spec)
+    spec.loader.exec_module(mg)
+    now = mg.compute()
+    seen = set()
+    for line in open(os.path.join(here, "scan_tiny.txt")):
+        if line.startswith("#"):
+            continue
+        name, shape, *vals = line.split()
+        ref = np.array([float(v) for v in vals]).reshape([int(s) for s in shape.split("x")])
+        np.testing.assert_allclose(now[name], ref, rtol=1e-13, atol=1e-15, err_msg=name)
+        seen.add(name)
+    assert seen == set(now)
