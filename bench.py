@@ -42,6 +42,8 @@ def parse_args():
     ap.add_argument("--general-A", action="store_true", help="perturb A so that no row is an arithmetic progression")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-extras", action="store_true",
+                    help="skip the decode-step and conv1d measurements that follow the timed region")
     return ap.parse_args()
 
 
@@ -366,6 +368,8 @@ def run_ours(args, cfg):
     }
     # the single recurrent step (decode): one pass over the float32 state, batch 64 at the same width
     try:
+        if args.no_extras:
+            raise RuntimeError("skipped (--no-extras)")
         sb = 64
         hs = torch.zeros((sb, cfg.D, cfg.N), dtype=torch.float32, device=dev)
         xs = torch.randn((sb, cfg.D), device=dev).to(io_t)
@@ -390,6 +394,8 @@ def run_ours(args, cfg):
         line["decode_step"] = {"error": str(exc)}
     # the neighbour of the scan on the SSM branch: short causal depthwise convolution + SiLU (HBM-bound streaming kernels)
     try:
+        if args.no_extras:
+            raise RuntimeError("skipped (--no-extras)")
         cw = torch.randn((cfg.D, 4), device=dev) * 0.5
         cb = torch.randn((cfg.D,), device=dev) * 0.1
         cy = torch.empty_like(d0["x"])
