@@ -135,3 +135,15 @@ def test_bounded_wait_reports_timeout_and_the_context_survives():
     torch.cuda.synchronize()
     got = U.gpu_fwd_bwd(dev)                      # checks the status itself and must be clean again
     U.assert_parity(got, U.oracle_fwd_bwd(inp), "bf16", "after a timed-out call")
+
+
+def test_smoke_entry_point_runs():
+    # the repository's smoke check (one small forward + backward against the oracle) must keep working as the oracle
+    # and the binding grow
+    import importlib.util
+    import os
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    spec = importlib.util.spec_from_file_location("graft_entry", os.path.join(root, "__graft_entry__.py"))
+    mod = importlib.util.module_from_spec(spec)
+    spec.loader.exec_module(mod)
+    mod.smoke()
