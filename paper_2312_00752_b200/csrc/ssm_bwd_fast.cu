@@ -185,11 +185,19 @@ __global__ void __launch_bounds__(kBwdFastThreads) ssm_bwd_fast_kernel(const Bwd
   };
 
   auto process_tile = [&](int st, auto ap_tag, const float4 (&ck)[2]) {
+    // The raw B / C rows of this ring stage were widened by the staging pass and are dead until the stage is refilled
+    // two tiles from now: the checkpoint state waits there (one float4 per thread and channel) until the first
+    // sub-block needs it again, instead of in registers.
+    float4* const park[2] = {reinterpret_cast<float4*>(&sm.rawB[st][0][0]), reinterpret_cast<float4*>(&sm.rawC[st][0][0])};
+    static_assert(sizeof(sm.rawB[0]) == sizeof(float4) * kBwdFastThreads, "one float4 per thread fits a raw B stage");
+    // start state of sub-block sb, from where level 1 (or the checkpoint) left it
+    auto start_state = [&](int sb, int q) { return sb > 0 ? sm.hsave[sb - 1][q][tid] : park[q][tid]; };
     // ---- level 1: states at the sub-block boundaries (steps 0, 8, 16, 24 of the tile), parked in shared memory
     {
       float2 h[2][2];
 #pragma unroll
       for (int q = 0; q < 2; ++q) {
+        park[q][tid] = ck[q];
         h[q][0] = make_float2(ck[q].x, ck[q].y);
         h[q][1] = make_float2(ck[q].z, ck[q].w);
       }
@@ -218,26 +226,24 @@ __global__ void __launch_bounds__(kBwdFastThreads) ssm_bwd_fast_kernel(const Bwd
     // ---- level 2: sub-blocks from last to first
 #pragma unroll 1
     for (int sb = kBT / kSB - 1; sb >= 0; --sb) {
-      float2 hs0[2][2];  // state before the first step of the sub-block
-#pragma unroll
-      for (int q = 0; q < 2; ++q) {
-        const float4 v = sb > 0 ? sm.hsave[sb > 0 ? sb - 1 : 0][q][tid] : ck[q];
-        hs0[q][0] = make_float2(v.x, v.y);
-        hs0[q][1] = make_float2(v.z, v.w);
-      }
       float2 hist[kSB][2][2];
-      uint32_t dwk[kSB], xwk[kSB];
+      // (the x and step-size words are re-read from shared memory in the reverse pass: registers are the scarce resource)
       float yw[kSB], dxw[kSB], ddw[kSB];  // quad-pair sums of: readout, delta * sum lam B, sum w A + x sum lam B
       {
-        float2 h[2][2] = {{hs0[0][0], hs0[0][1]}, {hs0[1][0], hs0[1][1]}};
+        float2 h[2][2];
+#pragma unroll
+        for (int q = 0; q < 2; ++q) {
+          const float4 v = start_state(sb, q);
+          h[q][0] = make_float2(v.x, v.y);
+          h[q][1] = make_float2(v.z, v.w);
+        }
 #pragma unroll
         for (int t = 0; t < kSB; ++t) {
           const int tt = sb * kSB + t;
-          dwk[t] = SP ? 0u : sm.d[st][tt][slot];
-          xwk[t] = sm.x[st][tt][slot];
+          const uint32_t xw = sm.x[st][tt][slot];
           const float4 Bq = sm.fB[tt][j], Cq = sm.fC[tt][j];
-          const float2 dt2 = step_sizes(st, tt, dwk[t]);
-          const float2 du = f2mul(dt2, make_float2(bf16sel(xwk[t], selA), bf16sel(xwk[t], selB)));
+          const float2 dt2 = step_sizes(st, tt, SP ? 0u : sm.d[st][tt][slot]);
+          const float2 du = f2mul(dt2, make_float2(bf16sel(xw, selA), bf16sel(xw, selB)));
           const float dtq[2] = {dt2.x, dt2.y}, duq[2] = {du.x, du.y};
           float y[2];
 #pragma unroll
@@ -255,13 +261,36 @@ __global__ void __launch_bounds__(kBwdFastThreads) ssm_bwd_fast_kernel(const Bwd
           yw[t] = y[0] + __shfl_xor_sync(0xffffffffu, y[1], 1);
         }
       }
+      // The readout totals are complete: finish them now (second exchange: lanes j and j^2 hold sums of the same
+      // channel, the lower keeps steps 0..3, the upper 4..7) and write dz, so that they do not occupy registers
+      // during the reverse recurrence.  The z rows of the tile were consumed by the staging pass.
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const float ky = gq ? yw[4 + e] : yw[e], sy = gq ? yw[e] : yw[4 + e];
+        const float ytot = ky + __shfl_xor_sync(0xffffffffu, sy, 2);
+        const int tt = sb * kSB + 4 * gq + e;
+        const float u = __uint_as_float((uint32_t)reinterpret_cast<const uint16_t*>(&sm.x[st][tt][slot])[pq] << 16);
+        const float s = fmaf(Dk, u, ytot);
+        float gsp;
+        if (SP) {
+          // the gate derivative is rebuilt here (its array holds the step sizes)
+          const float gf = __uint_as_float((uint32_t)reinterpret_cast<const uint16_t*>(&sm.g[st][tt][slot])[pq] << 16);
+          const float zf = __uint_as_float((uint32_t)reinterpret_cast<const uint16_t*>(&sm.z[st][tt][slot])[pq] << 16);
+          const float sg = sigmoid_fast(zf);
+          gsp = has_z ? gf * sg * fmaf(zf, 1.f - sg, 1.f) : 0.f;
+        } else {
+          gsp = sm.gsp[tt][2 * slot + pq];
+        }
+        reinterpret_cast<__nv_bfloat16*>(&sm.z[st][tt][slot])[pq] = __float2bfloat16_rn(gsp * s);
+      }
       // reverse recurrence over the sub-block
 #pragma unroll
       for (int t = kSB - 1; t >= 0; --t) {
         const int tt = sb * kSB + t;
         const float4 Bq = sm.fB[tt][j], Cq = sm.fC[tt][j];
-        const float2 dt2 = step_sizes(st, tt, dwk[t]);
-        const float2 u2 = make_float2(bf16sel(xwk[t], selA), bf16sel(xwk[t], selB));
+        const float2 dt2 = step_sizes(st, tt, SP ? 0u : sm.d[st][tt][slot]);
+        const uint32_t xw = sm.x[st][tt][slot];
+        const float2 u2 = make_float2(bf16sel(xw, selA), bf16sel(xw, selB));
         const float2 du = f2mul(dt2, u2);
         const float dtq[2] = {dt2.x, dt2.y}, uq[2] = {u2.x, u2.y}, duq[2] = {du.x, du.y};
         const float dsq[2] = {sm.ds[tt][2 * slot + pq], sm.ds[tt][2 * slot + (pq ^ 1)]};
@@ -290,8 +319,15 @@ __global__ void __launch_bounds__(kBwdFastThreads) ssm_bwd_fast_kernel(const Bwd
           const float lamB = lb.x + lb.y;
           mu[q][0] = f2mul(a01, lam01);
           mu[q][1] = f2mul(a23, lam23);
-          const float2 hp0 = t > 0 ? hist[t > 0 ? t - 1 : 0][q][0] : hs0[q][0];
-          const float2 hp1 = t > 0 ? hist[t > 0 ? t - 1 : 0][q][1] : hs0[q][1];
+          float2 hp0, hp1;   // h_{t-1}: the step before in registers, or the sub-block's start state (read again)
+          if (t > 0) {
+            hp0 = hist[t > 0 ? t - 1 : 0][q][0];
+            hp1 = hist[t > 0 ? t - 1 : 0][q][1];
+          } else {
+            const float4 v = start_state(sb, q);
+            hp0 = make_float2(v.x, v.y);
+            hp1 = make_float2(v.z, v.w);
+          }
           const float2 w01 = f2mul(mu[q][0], hp0), w23 = f2mul(mu[q][1], hp1);
           float2 wa = f2mul(w01, A2[q][0]);
           wa = f2fma(w23, A2[q][1], wa);
@@ -320,13 +356,11 @@ __global__ void __launch_bounds__(kBwdFastThreads) ssm_bwd_fast_kernel(const Bwd
         }
       }
       // second exchange: lanes j and j^2 hold sums of the same channel; the lower keeps steps 0..3, the upper 4..7
-      float ytot[4], dxtot[4], ddtot[4];
+      float dxtot[4], ddtot[4];
 #pragma unroll
       for (int e = 0; e < 4; ++e) {
-        const float ky = gq ? yw[4 + e] : yw[e], sy = gq ? yw[e] : yw[4 + e];
         const float kx = gq ? dxw[4 + e] : dxw[e], sx = gq ? dxw[e] : dxw[4 + e];
         const float kd = gq ? ddw[4 + e] : ddw[e], sd = gq ? ddw[e] : ddw[4 + e];
-        ytot[e] = ky + __shfl_xor_sync(0xffffffffu, sy, 2);
         dxtot[e] = kx + __shfl_xor_sync(0xffffffffu, sx, 2);
         ddtot[e] = kd + __shfl_xor_sync(0xffffffffu, sd, 2);
       }
@@ -336,27 +370,18 @@ __global__ void __launch_bounds__(kBwdFastThreads) ssm_bwd_fast_kernel(const Bwd
         const int tt = sb * kSB + 4 * gq + e;
         const float u = __uint_as_float((uint32_t)reinterpret_cast<const uint16_t*>(&sm.x[st][tt][slot])[pq] << 16);
         const float ds = sm.ds[tt][2 * slot + pq];
-        const float s = fmaf(Dk, u, ytot[e]);
         dD_acc = fmaf(ds, u, dD_acc);
         reinterpret_cast<__nv_bfloat16*>(&sm.x[st][tt][slot])[pq] = __float2bfloat16_rn(fmaf(ds, Dk, dxtot[e]));
-        float ddv = ddtot[e], gsp;
+        float ddv = ddtot[e];
         if (SP) {
-          // the gate derivative is rebuilt here (its array holds the step sizes); the gradient goes to the
-          // pre-activation v: d softplus(v) / dv = sigmoid(v)
-          const float gf = __uint_as_float((uint32_t)reinterpret_cast<const uint16_t*>(&sm.g[st][tt][slot])[pq] << 16);
-          const float zf = __uint_as_float((uint32_t)reinterpret_cast<const uint16_t*>(&sm.z[st][tt][slot])[pq] << 16);
-          const float sg = sigmoid_fast(zf);
-          gsp = has_z ? gf * sg * fmaf(zf, 1.f - sg, 1.f) : 0.f;
+          // the gradient goes to the pre-activation v: d softplus(v) / dv = sigmoid(v)
           if (p.softplus) {
             const float v = __uint_as_float((uint32_t)reinterpret_cast<const uint16_t*>(&sm.d[st][tt][slot])[pq] << 16) + bias_pq;
             ddv *= sigmoid_fast(v);
           }
           dbias_acc += ddv;
-        } else {
-          gsp = sm.gsp[tt][2 * slot + pq];
         }
         reinterpret_cast<__nv_bfloat16*>(&sm.d[st][tt][slot])[pq] = __float2bfloat16_rn(ddv);
-        reinterpret_cast<__nv_bfloat16*>(&sm.z[st][tt][slot])[pq] = __float2bfloat16_rn(gsp * s);
       }
     }
   };
@@ -431,6 +456,17 @@ __global__ void __launch_bounds__(kBwdFastThreads) ssm_bwd_fast_kernel(const Bwd
     }
     const Item nxt = decode(sm.sched[1]);
     issue_item(nxt, st ^ 1);
+    if (nxt.live) {
+      // the checkpoint state of the next tile is needed the moment that tile starts: pull it into L2 now
+      const int dn = nxt.d_cta + 2 * slot;
+      if (dn < D) {
+#pragma unroll
+        for (int q = 0; q < 2; ++q) {
+          const float* ckp = p.ckpt + (((size_t)nxt.b * p.nck + nxt.t0 / kCkptSteps) * D + dn + q) * 16 + 4 * j;
+          asm volatile("prefetch.global.L2 [%0];" ::"l"(ckp));
+        }
+      }
+    }
     if (cur.live) {
       if (cur.ord > 0) {
         const float4* hb = p.handoff + ((size_t)cur.chain * THREADS + tid) * kHandoffVec;
