@@ -50,6 +50,29 @@ Plan make_plan(const ssm_problem_t& p) {
   return pl;
 }
 
+// The backward pass splits time on its own terms.  Its unit of work is a chain (batch entry, segment, group of 32
+// channels) walked by one block of the persistent kernel, 4 blocks per SM; a problem with fewer chains than resident
+// blocks (the 130M layer shape: 384 for 592) leaves SMs idle and every chain sequential, and the extra adjoint pre-pass
+// that a split needs costs about a third of a forward sweep.  So: no split while the chains nearly fill the GPU,
+// otherwise enough segments for about 3 chains per resident block (segments of at least 256 steps).  The checkpoint
+// states do not depend on the split, so forward and backward may disagree about it.
+Plan make_bwd_plan(const ssm_problem_t& p) {
+  Plan pl = make_plan(p);
+  const long long chains = (long long)p.batch * pl.bwd_groups;
+  const long long resident = 4LL * kNumSMs;
+  int nseg = 1;
+  if (chains * 10 < resident * 9) {
+    const long long want = (3 * resident + chains - 1) / chains;
+    const long long max_by_len = std::max(1, p.L / 256);
+    nseg = (int)std::min<long long>(std::min(want, max_by_len), 65535);
+  }
+  int seg_steps = (p.L + nseg - 1) / nseg;
+  seg_steps = (seg_steps + kCkptSteps - 1) / kCkptSteps * kCkptSteps;
+  pl.seg_steps = seg_steps;
+  pl.nseg = (p.L + seg_steps - 1) / seg_steps;
+  return pl;
+}
+
 struct FwdWorkspace {
   size_t seg_end, seg_dsum, h_start, total;
 };
@@ -68,7 +91,7 @@ static FwdWorkspace fwd_layout(const ssm_problem_t& p, const Plan& pl) {
 struct BwdWorkspace {
   size_t dBC_part, dA_part, dD_part, dbias_part, ckpt, seg_local, seg_dsum, mu_in, fwd, sched, handoff, total;
 };
-static BwdWorkspace bwd_layout(const ssm_problem_t& p, const Plan& pl) {
+static BwdWorkspace bwd_layout(const ssm_problem_t& p, const Plan& pl, const Plan& pl_fwd) {
   BwdWorkspace w{};
   size_t off = 0;
   auto take = [&](size_t bytes) {
@@ -89,7 +112,7 @@ static BwdWorkspace bwd_layout(const ssm_problem_t& p, const Plan& pl) {
     w.mu_in = take(st);
     w.seg_dsum = take(parts * p.D * sizeof(float));
   }
-  w.fwd = take(fwd_layout(p, pl).total);
+  w.fwd = take(fwd_layout(p, pl_fwd).total);   // the forward sweep that rebuilds checkpoints uses the forward split
   const size_t chains = parts * pl.bwd_groups;   // (batch, segment, channel group) chains of the tuned kernel
   w.sched = take((64 + chains) * sizeof(int));
   w.handoff = take(chains * bwd_fast_handoff_bytes_per_chain());
@@ -147,7 +170,7 @@ size_t ssm_scan_fwd_workspace_bytes(const ssm_problem_t* p) {
 
 size_t ssm_scan_bwd_workspace_bytes(const ssm_problem_t* p) {
   if (validate_problem(p) != SSM_OK) return 0;
-  return bwd_layout(*p, make_plan(*p)).total;
+  return bwd_layout(*p, make_bwd_plan(*p), make_plan(*p)).total;
 }
 
 size_t ssm_scan_saved_state_bytes(const ssm_problem_t* p) {
@@ -174,7 +197,7 @@ ssm_status_t ssm_scan_check_status(const ssm_problem_t* p, const void* workspace
   const ssm_status_t st = validate_problem(p);
   if (st != SSM_OK) return st;
   if (workspace == nullptr) return SSM_ERR_WORKSPACE;
-  const BwdWorkspace w = bwd_layout(*p, make_plan(*p));
+  const BwdWorkspace w = bwd_layout(*p, make_bwd_plan(*p), make_plan(*p));
   int word = 0;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   if (cudaMemcpyAsync(&word, static_cast<const char*>(workspace) + w.sched + sizeof(int), sizeof(int),
@@ -317,8 +340,8 @@ static ssm_status_t bwd_impl(const ssm_problem_t* p, const void* x, const void* 
                         (const void*)delta_bias, (const void*)ddelta_bias, (const void*)h0, (const void*)dh_last,
                         (const void*)dh0})
     if (q && !aligned_to(q, 4)) return SSM_ERR_INVALID_ARG;
-  const Plan pl = make_plan(*p);
-  const BwdWorkspace w = bwd_layout(*p, pl);
+  const Plan pl = make_bwd_plan(*p), pl_fwd = make_plan(*p);
+  const BwdWorkspace w = bwd_layout(*p, pl, pl_fwd);
   st = check_ws(workspace, workspace_bytes, w.total);
   if (st != SSM_OK) return st;
 
@@ -337,18 +360,18 @@ static ssm_status_t bwd_impl(const ssm_problem_t* p, const void* x, const void* 
     fp.batch = p->batch;
     fp.L = p->L;
     fp.D = p->D;
-    fp.nseg = pl.nseg;
-    fp.seg_steps = pl.seg_steps;
-    fp.nck = pl.nck;
+    fp.nseg = pl_fwd.nseg;
+    fp.seg_steps = pl_fwd.seg_steps;
+    fp.nck = pl_fwd.nck;
     fp.general_A = (p->flags & SSM_FLAG_GENERAL_A) ? 1 : 0;
     fp.zoh = (p->flags & SSM_FLAG_ZOH_BBAR) ? 1 : 0;
     fp.delta_bias = delta_bias;
     fp.softplus = (p->flags & SSM_FLAG_DELTA_SOFTPLUS) ? 1 : 0;
     const float* h_start = nullptr;
-    if (run_segment_starts(*p, pl, fp, ws + w.fwd, h0, &h_start, s) != cudaSuccess) return SSM_ERR_CUDA;
+    if (run_segment_starts(*p, pl_fwd, fp, ws + w.fwd, h0, &h_start, s) != cudaSuccess) return SSM_ERR_CUDA;
     fp.h_start = h_start;
     fp.ckpt = reinterpret_cast<float*>(ws + w.ckpt);
-    if (launch_fwd(*p, pl, fp, kFwdCkptOnly, s) != cudaSuccess) return SSM_ERR_CUDA;
+    if (launch_fwd(*p, pl_fwd, fp, kFwdCkptOnly, s) != cudaSuccess) return SSM_ERR_CUDA;
     ckpt = fp.ckpt;
   }
 

@@ -393,8 +393,12 @@ int bwd_channels_per_block(int) { return 32; }
 bool bwd_fast_applicable(const ssm_problem_t& prob, const BwdParams& p);
 cudaError_t launch_bwd_fast(const Plan& plan, const BwdParams& p, cudaStream_t s);
 
+bool bwd_local_fast_applicable(const ssm_problem_t& prob, const BwdParams& p);
+cudaError_t launch_bwd_local_fast(const Plan& plan, const BwdParams& p, cudaStream_t s);
+
 cudaError_t launch_bwd(const ssm_problem_t& prob, const Plan& plan, const BwdParams& p, int mode, cudaStream_t s) {
   if (mode == kBwdFull && bwd_fast_applicable(prob, p)) return launch_bwd_fast(plan, p, s);
+  if (mode == kBwdLocal && bwd_local_fast_applicable(prob, p)) return launch_bwd_local_fast(plan, p, s);
   if (prob.io_dtype == SSM_BF16) return launch_bwd_io<__nv_bfloat16>(prob, plan, p, mode, s);
   return launch_bwd_io<float>(prob, plan, p, mode, s);
 }
