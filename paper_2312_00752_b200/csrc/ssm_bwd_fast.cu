@@ -589,6 +589,9 @@ __global__ void __launch_bounds__(kBwdFastThreads) ssm_bwd_fast_kernel(const Bwd
 bool bwd_fast_applicable(const ssm_problem_t& prob, const BwdParams& p) {
   auto al16 = [](const void* q) { return q == nullptr || (reinterpret_cast<uintptr_t>(q) & 15) == 0; };
   if (p.zoh) return false;  // the tuned kernel implements the default rule B-bar = delta * B only
+  // work items are numbered with 32-bit integers (one spare bit for the claims that run past the end)
+  const long long items = (long long)p.batch * p.nseg * ((p.D + kBwdFastCH - 1) / kBwdFastCH) * (p.seg_steps / kBT);
+  if (items > (1LL << 30)) return false;
   return prob.io_dtype == SSM_BF16 && prob.N == 16 && prob.D % 8 == 0 && p.seg_steps % kBT == 0 && al16(p.x) &&
          al16(p.delta) && al16(p.z) && al16(p.B) && al16(p.C) && al16(p.dout) && al16(p.dx) && al16(p.ddelta) &&
          al16(p.dz) && al16(p.A) && al16(p.ckpt) && al16(p.mu_in) && al16(p.dh0) && al16(p.dBC_part) && al16(p.dA_part) &&

@@ -32,6 +32,7 @@ struct LocalSmem {
   uint32_t rawC[2][kTT][8];
   float4 fC[2][kTT][4];
   float ds[kWarps][kHalf][16];
+  float dt[kWarps][kHalf][16];   // fused step size only: softplus(delta_pre + bias) of half a tile, per warp
 };
 
 __device__ __forceinline__ void block_barrier() { asm volatile("bar.sync 1, %0;" ::"r"(kThreads) : "memory"); }
@@ -39,6 +40,8 @@ __device__ __forceinline__ void cp_async_wait_but_one() { asm volatile("cp.async
 
 }  // namespace
 
+// SP: `delta` holds the pre-activation and the step size is delta + bias, through the softplus if asked (Algorithm 2 step 4)
+template <bool SP>
 __global__ void __launch_bounds__(kThreads) ssm_bwd_local_fast_kernel(const BwdParams p) {
   __shared__ __align__(16) LocalSmem sm;
   const int tid = threadIdx.x;
@@ -135,6 +138,15 @@ __global__ void __launch_bounds__(kThreads) ssm_bwd_local_fast_kernel(const BwdP
     mu[q][0] = mu[q][1] = make_float2(0.f, 0.f);
   }
   ap = __all_sync(0xffffffffu, ap);
+  // SP: in the preparation stage below a lane always handles channel pair (lane % 8) of its warp
+  float bias0 = 0.f, bias1 = 0.f;
+  if (SP && p.delta_bias != nullptr) {
+    const int c = d_cta + warp * 16 + 2 * (lane & 7);
+    if (c < D) {
+      bias0 = p.delta_bias[c];
+      bias1 = p.delta_bias[c + 1];
+    }
+  }
 
   auto compute_tile = [&](int i, auto ap_tag) {
     constexpr bool AP = decltype(ap_tag)::value;
@@ -155,15 +167,34 @@ __global__ void __launch_bounds__(kThreads) ssm_bwd_local_fast_kernel(const BwdP
           v1 *= z1 * sigmoid_fast(z1);
         }
         *reinterpret_cast<float2*>(&sm.ds[warp][tt][2 * sl]) = make_float2(v0, v1);
+        if (SP) {
+          const uint32_t dw = sm.d[st][half * kHalf + tt][warp * 8 + sl];
+          float s0 = bf16lo(dw) + bias0, s1 = bf16hi(dw) + bias1;
+          if (p.softplus) {
+            s0 = softplus_fast(s0);
+            s1 = softplus_fast(s1);
+          }
+          // rows past the end of the segment must stay identity steps
+          const bool live = t_begin + (ntiles - 1 - i) * kTT + half * kHalf + tt < t_end;
+          *reinterpret_cast<float2*>(&sm.dt[warp][tt][2 * sl]) = live ? make_float2(s0, s1) : make_float2(0.f, 0.f);
+        }
       }
       __syncwarp();
 #pragma unroll
       for (int t = kHalf - 1; t >= 0; --t) {
         const int row = half * kHalf + t;
-        const uint32_t dw = sm.d[st][row][slot];
         const float2 dsv = *reinterpret_cast<const float2*>(&sm.ds[warp][t][2 * (lane >> 2)]);
         const float4 Cq = sm.fC[fb][row][j];
-        const float dt[2] = {bf16sel(dw, selA), bf16sel(dw, selB)};
+        float dt[2];
+        if (SP) {
+          const float2 f = *reinterpret_cast<const float2*>(&sm.dt[warp][t][2 * (lane >> 2)]);
+          dt[0] = pq ? f.y : f.x;
+          dt[1] = pq ? f.x : f.y;
+        } else {
+          const uint32_t dw = sm.d[st][row][slot];
+          dt[0] = bf16sel(dw, selA);
+          dt[1] = bf16sel(dw, selB);
+        }
         const float dsq[2] = {pq ? dsv.y : dsv.x, pq ? dsv.x : dsv.y};
 #pragma unroll
         for (int q = 0; q < 2; ++q) {
@@ -206,14 +237,14 @@ __global__ void __launch_bounds__(kThreads) ssm_bwd_local_fast_kernel(const BwdP
 
 bool bwd_local_fast_applicable(const ssm_problem_t& prob, const BwdParams& p) {
   auto al16 = [](const void* q) { return q == nullptr || (reinterpret_cast<uintptr_t>(q) & 15) == 0; };
-  if (p.softplus || p.delta_bias != nullptr) return false;   // the fused step size runs on the generic kernel here
   return prob.io_dtype == SSM_BF16 && prob.N == 16 && prob.D % 8 == 0 && al16(p.delta) && al16(p.z) && al16(p.dout) &&
          al16(p.C) && al16(p.A) && al16(p.seg_local);
 }
 
 cudaError_t launch_bwd_local_fast(const Plan& plan, const BwdParams& p, cudaStream_t s) {
   dim3 grid((p.D + kCH - 1) / kCH, plan.nseg, p.batch);
-  ssm_bwd_local_fast_kernel<<<grid, kThreads, 0, s>>>(p);
+  if (p.softplus || p.delta_bias != nullptr) ssm_bwd_local_fast_kernel<true><<<grid, kThreads, 0, s>>>(p);
+  else ssm_bwd_local_fast_kernel<false><<<grid, kThreads, 0, s>>>(p);
   return cudaGetLastError();
 }
 
