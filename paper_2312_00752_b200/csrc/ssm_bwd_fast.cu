@@ -9,6 +9,11 @@
 // 8, 16 and 24 in shared memory; then, for the sub-blocks of 8 steps from last to first, it re-runs the 8 steps keeping
 // every h_t in registers and walks them backwards with the adjoint recurrence.
 //
+// Registers are the scarce resource (255 per thread, 4 blocks per SM, and almost no L1 left beside 54 KB of shared
+// memory per block, so a spill costs an L2 round trip): whatever can wait in shared memory does -- the input words of a
+// step are read again in the reverse pass, the checkpoint state waits in a staging buffer that is dead by then, and
+// the readout is finished before the reverse pass starts.
+//
 // Scheduling.  The kernel is persistent: blocks claim work items (channel group, tile) from a global counter in an
 // order in which the tile that a tile depends on (the next tile in time of the same channel group) is always claimed
 // earlier, so whoever holds it is already running; the adjoint mu and the dA / dD accumulators cross from one tile
@@ -17,8 +22,9 @@
 // block raises an abort word that all blocks observe, and the host reports SSM_ERR_TIMEOUT.
 //
 // Sums.  The three per-(step, channel) sums over n (readout for dz, sum lam*B for dx and ddelta, sum w*A for
-// ddelta) are exchanged inside the quad in one batch per sub-block; afterwards every lane finalises 4 steps of one
-// channel.  dB and dC are summed over the two channels of a thread in registers, over the 8 quads of a warp through
+// ddelta) are exchanged inside the quad in batches per sub-block, after which every lane finalises 4 steps of one
+// channel (the readout and dz before the reverse pass, dx and ddelta after it).  dB and dC are summed over the two
+// channels of a thread in registers, over the 8 quads of a warp through
 // a shared-memory transpose with a fixed order, over the 2 warps in ascending order, and leave the block as partial
 // sums that ssm_bwd_reduce_kernel adds in ascending block order.  dA and dD accumulate in registers over the whole
 // segment.  Everything is deterministic; there are no floating-point atomics.
