@@ -218,6 +218,19 @@ __device__ __forceinline__ float zoh_gain_dA(float dt, float A, float a, float E
   return __fdividef(fmaf(dt, a, -E), A);
 }
 
+// tanh through the hardware unit (one special-function operation; relative error about 2^-11: bf16 io only)
+__device__ __forceinline__ float tanh_approx(float v) {
+  float r;
+  asm("tanh.approx.f32 %0, %1;" : "=f"(r) : "f"(v));
+  return r;
+}
+// s * silu(z) for a pair of elements with the hardware tanh: silu(z) = z/2 + z/2 tanh(z/2)
+__device__ __forceinline__ float2 gate_pair_tanh(float2 s, float2 z) {
+  const float2 hz = f2mul(z, f2dup(0.5f));
+  const float2 sl = f2fma(hz, make_float2(tanh_approx(hz.x), tanh_approx(hz.y)), hz);
+  return f2mul(s, sl);
+}
+
 // sigmoid(z) through one ex2 and one reciprocal
 __device__ __forceinline__ float sigmoid_fast(float z) { return rcp_approx(1.0f + ex2_approx(-kLog2e * z)); }
 

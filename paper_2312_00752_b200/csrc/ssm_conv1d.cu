@@ -273,11 +273,6 @@ __device__ __forceinline__ void store4(float* __restrict__ p, const float2 (&v)[
   *reinterpret_cast<float4*>(p) = make_float4(v[0].x, v[0].y, v[1].x, v[1].y);
 }
 
-__device__ __forceinline__ float tanh_approx(float v) {
-  float r;
-  asm("tanh.approx.f32 %0, %1;" : "=f"(r) : "f"(v));
-  return r;
-}
 // sigmoid of a pair.  FAST: 1/2 + 1/2 tanh(v/2) with the hardware tanh (one special-function operation instead of two;
 // relative error about 2^-11, used for bf16 io only, whose own rounding is 2^-9); otherwise ex2 + reciprocal.
 template <bool FAST>

@@ -140,14 +140,12 @@ __global__ void __launch_bounds__((WARPS + 1) * 32) ssm_fwd_fast_kernel(const Fw
         const float2 y = *reinterpret_cast<const float2*>(&sm.yp[yb][tt][2 * eslot]);
         const float2 Dk2 = *reinterpret_cast<const float2*>(&sm.Dsk[2 * eslot]);
         const uint32_t xw = sm.x[st][tt][eslot];
-        float s0 = fmaf(Dk2.x, bf16lo(xw), y.x), s1 = fmaf(Dk2.y, bf16hi(xw), y.y);
+        float2 s2 = f2fma(Dk2, make_float2(bf16lo(xw), bf16hi(xw)), y);
         if (has_z) {
           const uint32_t zw = sm.z[st][tt][eslot];
-          const float z0 = bf16lo(zw), z1 = bf16hi(zw);
-          s0 = s0 * z0 * sigmoid_fast(z0);
-          s1 = s1 * z1 * sigmoid_fast(z1);
+          s2 = gate_pair_tanh(s2, make_float2(bf16lo(zw), bf16hi(zw)));
         }
-        const __nv_bfloat162 r = __floats2bfloat162_rn(s0, s1);
+        const __nv_bfloat162 r = __floats2bfloat162_rn(s2.x, s2.y);
         sm.o[tt][eslot] = *reinterpret_cast<const uint32_t*>(&r);
       }
       __syncwarp();
