@@ -38,6 +38,9 @@ def test_config0_tiny_f32():
     (1, 130, 33, 2, "f32"),
     (2, 64, 70, 1, "bf16"),       # N = 1 (the setting of the gating theorem)
     (1, 333, 129, 16, "f32"),     # channels straddle several blocks
+    (1, 1, 8, 16, "bf16"),        # tuned kernels: a single step in a single partial channel block
+    (2, 31, 16, 16, "bf16"),      # tuned kernels: one step short of a tile
+    (1, 33, 72, 16, "bf16"),      # tuned kernels: one step past a tile, channel blocks 32 + 32 + 8
 ])
 def test_shapes_and_state_sizes(batch, L, D, N, io):
     cfg, inp = _case(batch, L, D, N, io)
@@ -45,16 +48,17 @@ def test_shapes_and_state_sizes(batch, L, D, N, io):
     U.assert_parity(got, U.oracle_fwd_bwd(inp), io, f"{(batch, L, D, N, io)}")
 
 
+@pytest.mark.parametrize("io", ["f32", "bf16"])     # generic and tuned kernels
 @pytest.mark.parametrize("gate,skip", [(False, True), (True, False), (False, False)])
-def test_optional_gate_and_skip(gate, skip):
-    cfg, inp = _case(2, 150, 48, 16, "f32")
+def test_optional_gate_and_skip(gate, skip, io):
+    cfg, inp = _case(2, 150, 48, 16, io)
     if not gate:
         inp["z"] = None
     if not skip:
         inp["D_skip"] = None
-    got = U.gpu_fwd_bwd(U.to_device(inp, "f32"))
+    got = U.gpu_fwd_bwd(U.to_device(inp, io))
     assert (got["dz"] is None) == (not gate) and (got["dD"] is None) == (not skip)
-    U.assert_parity(got, U.oracle_fwd_bwd(inp), "f32", f"gate={gate} skip={skip}")
+    U.assert_parity(got, U.oracle_fwd_bwd(inp), io, f"gate={gate} skip={skip} {io}")
 
 
 @pytest.mark.parametrize("io,L,D", [("f32", 4096, 64), ("bf16", 5000, 40)])
