@@ -151,3 +151,22 @@ def test_smoke_entry_point_runs():
     mod = importlib.util.module_from_spec(spec)
     spec.loader.exec_module(mod)
     mod.smoke()
+
+
+def test_pointers_off_the_16_byte_grid_take_the_generic_kernels():
+    # bf16 / N = 16 tensors whose addresses are only 8-byte aligned: the tuned kernels do not apply, the results must
+    # be the same within tolerance (and the call must not fault on a misaligned 16-byte access)
+    import torch
+    cfg, inp = _case(2, 100, 40, 16, "bf16")
+    dev = U.to_device(inp, "bf16")
+
+    def shifted(t):   # same values at an address that is 8 bytes past a 16-byte boundary
+        buf = torch.empty(t.numel() + 8, dtype=t.dtype, device=t.device)
+        off = 4 if t.dtype == torch.bfloat16 else 2
+        v = buf[off:off + t.numel()].view(t.shape)
+        v.copy_(t)
+        assert v.data_ptr() % 16 == 8 and v.is_contiguous()
+        return v
+    dev2 = {k: (shifted(v) if v is not None else None) for k, v in dev.items()}
+    got = U.gpu_fwd_bwd(dev2)
+    U.assert_parity(got, U.oracle_fwd_bwd(inp), "bf16", "misaligned")
