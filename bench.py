@@ -392,6 +392,26 @@ def run_ours(args, cfg):
                                "note": "state (42 MB) stays in L2 between repetitions; a launch-latency-sized kernel"}
     except Exception as exc:  # the headline numbers do not depend on this extra
         line["decode_step"] = {"error": str(exc)}
+    # forward only, no checkpoint states written (the prefill use of the scan)
+    try:
+        if args.no_extras:
+            raise RuntimeError("skipped (--no-extras)")
+        for i in range(3):
+            K.ssm_scan_fwd(sets[i % NSETS]["x"], sets[i % NSETS]["delta"], d0["A"], sets[i % NSETS]["B"],
+                           sets[i % NSETS]["C"], d0["D_skip"], sets[i % NSETS]["z"], out=out, stream=stream)
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        for i in range(20):
+            s_ = sets[i % NSETS]
+            K.ssm_scan_fwd(s_["x"], s_["delta"], s_["A"], s_["B"], s_["C"], s_["D_skip"], s_["z"], out=out, stream=stream)
+        b.record(stream)
+        torch.cuda.synchronize(dev)
+        p_ms = a.elapsed_time(b) / 20
+        line["prefill_fwd"] = {"ms": p_ms, "elements_per_s": cfg.elements / (p_ms * 1e-3),
+                               "frac_of_hbm_peak": fwd_bytes / (p_ms * 1e-3) / 1e9 / peak,
+                               "note": "ssm_scan_fwd without SSM_FLAG_SAVE_STATES"}
+    except Exception as exc:
+        line["prefill_fwd"] = {"error": str(exc)}
     # the neighbour of the scan on the SSM branch: short causal depthwise convolution + SiLU (HBM-bound streaming kernels)
     try:
         if args.no_extras:
