@@ -24,7 +24,7 @@ constexpr int kConvThreads = 64;
 constexpr int kConvMinSteps = 32;   // time steps per thread and chunk: chosen per launch between these two so that the
 constexpr int kConvMaxSteps = 128;  // grid fills the GPU a whole number of times (see choose_steps)
 constexpr int kConvAheadFwd = 8;    // rows loaded before the first of them is used
-constexpr int kConvAheadBwd = 4;    // (two tensors per row in the backward kernel)
+constexpr int kConvAheadBwd = 8;    // (two tensors per row in the backward kernel; 2, 4, 8, 16 measured: 78, 64, 60, 83 us)
 
 struct ConvParams {
   const void* x;
@@ -330,12 +330,20 @@ __global__ void __launch_bounds__(kConvThreads) ssm_conv1d_fwd_vec4_kernel(const
   const IO* __restrict__ xp = static_cast<const IO*>(p.x) + ((size_t)b * p.L + t0) * p.D + c0;
   IO* __restrict__ yp = static_cast<IO*>(p.y) + ((size_t)b * p.L + t0) * p.D + c0;
   const size_t stride = (size_t)p.D;
-  auto batch = [&](int n, auto full_tag) {   // n rows (n == A when full_tag is true)
+  // Rows are fetched one batch ahead: while a batch is computed the loads of the next one are in flight.
+  Raw4<IO> nxt[A];
+  auto fetch = [&](int t) {   // rows t .. t+A-1 of the chunk
+#pragma unroll
+    for (int u = 0; u < A; ++u)
+      if (t + u < t1) nxt[u] = load_raw4(xp + u * stride);
+    xp += A * stride;
+  };
+  auto batch = [&](int t, int n, auto full_tag) {   // n rows from t (n == A when full_tag is true)
     constexpr bool FULL = decltype(full_tag)::value;
     Raw4<IO> raw[A];
 #pragma unroll
-    for (int u = 0; u < A; ++u)
-      if (FULL || u < n) raw[u] = load_raw4(xp + u * stride);
+    for (int u = 0; u < A; ++u) raw[u] = nxt[u];
+    fetch(t + A);
 #pragma unroll
     for (int u = 0; u < A; ++u) {
       if (FULL || u < n) {
@@ -354,12 +362,12 @@ __global__ void __launch_bounds__(kConvThreads) ssm_conv1d_fwd_vec4_kernel(const
         store4(yp + u * stride, o);
       }
     }
-    xp += A * stride;
     yp += A * stride;
   };
+  fetch(t0);
   int t = t0;
-  for (; t + A <= t1; t += A) batch(A, std::true_type{});
-  if (t < t1) batch(t1 - t, std::false_type{});
+  for (; t + A <= t1; t += A) batch(t, A, std::true_type{});
+  if (t < t1) batch(t, t1 - t, std::false_type{});
 }
 
 template <typename IO, int W, bool SILU, bool FAST>
@@ -391,19 +399,31 @@ __global__ void __launch_bounds__(kConvThreads) ssm_conv1d_bwd_vec4_kernel(const
   IO* __restrict__ dxp = static_cast<IO*>(p.dx) + ((size_t)b * p.L + t0 - (W - 1)) * p.D + c0;   // row of s = t - (W-1)
   // dx[s] needs dpre[s .. s+W-1]: the walk runs W-1 steps past the chunk (dpre is zero past the end of the sequence)
   const int t_stop = t1 + (W - 1);
+  // Rows are fetched one batch ahead: while batch t is computed the loads of batch t + A are in flight.
+  Raw4<IO> nx[A], ng[A];   // the next batch, still in its loaded form
+  auto fetch = [&](int t) {   // rows t .. t+A-1 (zeros outside the walk or past the end of the sequence)
+#pragma unroll
+    for (int u = 0; u < A; ++u) {
+      if (t + u < t_stop && t + u < p.L) {
+        nx[u] = load_raw4(xp + u * stride);
+        ng[u] = load_raw4(gp + u * stride);
+      } else {
+        zero4(nx[u]);
+        zero4(ng[u]);
+      }
+    }
+    xp += A * stride;
+    gp += A * stride;
+  };
   auto batch = [&](int t, auto full_tag) {   // rows t .. t+A-1; FULL: all of them inside the chunk and the sequence
     constexpr bool FULL = decltype(full_tag)::value;
     Raw4<IO> rx[A], rg[A];
 #pragma unroll
     for (int u = 0; u < A; ++u) {
-      if (FULL || (t + u < t_stop && t + u < p.L)) {
-        rx[u] = load_raw4(xp + u * stride);
-        rg[u] = load_raw4(gp + u * stride);
-      } else {
-        zero4(rx[u]);
-        zero4(rg[u]);
-      }
+      rx[u] = nx[u];
+      rg[u] = ng[u];
     }
+    fetch(t + A);
 #pragma unroll
     for (int u = 0; u < A; ++u) {
       const int tt = t + u;
@@ -448,10 +468,9 @@ __global__ void __launch_bounds__(kConvThreads) ssm_conv1d_bwd_vec4_kernel(const
         }
       }
     }
-    xp += A * stride;
-    gp += A * stride;
     dxp += A * stride;
   };
+  fetch(t0);
   int t = t0;
   for (; t + A <= t1; t += A) batch(t, std::true_type{});
   for (; t < t_stop; t += A) batch(t, std::false_type{});
