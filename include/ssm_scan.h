@@ -75,6 +75,10 @@ enum {
   SSM_FLAG_ZOH_BBAR = 64u,    /* B-bar = (exp(delta A) - 1) / A * B, the zero-order hold of Eq. 4 (delta * B at A = 0),
                                  instead of the default delta * B; honoured by every call; such problems run on
                                  the generic kernels                                                             */
+  SSM_FLAG_STATIC_B = 256u,   /* B is not input-dependent (Algorithm 1; the selective-parameter ablation, Table 7): B is a float32
+                                 parameter [D][N] like A instead of io_dtype [batch][L][N], and dB is float32 [D][N],
+                                 summed over batch and time.  Generic kernels.                                    */
+  SSM_FLAG_STATIC_C = 512u,   /* the same for C and dC                                                            */
   SSM_FLAG_TEST_WITHHOLD = 16u /* test hook for the bounded waits: the tuned backward kernel never publishes its
                                  hand-off flags and polls only 1000 times, so every dependent tile gives up and
                                  ssm_scan_check_status reports SSM_ERR_TIMEOUT; the gradients are then undefined  */

@@ -18,6 +18,7 @@ SSM_F32, SSM_BF16 = 0, 1
 SSM_FLAG_HAS_Z, SSM_FLAG_HAS_DSKIP, SSM_FLAG_SAVE_STATES, SSM_FLAG_GENERAL_A, SSM_FLAG_TEST_WITHHOLD = 1, 2, 4, 8, 16
 SSM_FLAG_DELTA_SOFTPLUS = 32
 SSM_FLAG_ZOH_BBAR = 64
+SSM_FLAG_STATIC_B, SSM_FLAG_STATIC_C = 256, 512
 
 EXPORTED_SYMBOLS = (
     "ssm_scan_fwd_workspace_bytes", "ssm_scan_bwd_workspace_bytes", "ssm_scan_saved_state_bytes",
@@ -125,11 +126,13 @@ def _io_dtype(t: torch.Tensor) -> int:
 
 
 def make_problem(x: torch.Tensor, B: torch.Tensor, has_z: bool, has_dskip: bool, save_states: bool = False,
-                 general_A: bool = False, zoh: bool = False) -> ssm_problem_t:
+                 general_A: bool = False, zoh: bool = False, static_B: bool = False,
+                 static_C: bool = False) -> ssm_problem_t:
     batch, L, D = x.shape
     flags = (SSM_FLAG_HAS_Z if has_z else 0) | (SSM_FLAG_HAS_DSKIP if has_dskip else 0) \
         | (SSM_FLAG_SAVE_STATES if save_states else 0) | (SSM_FLAG_GENERAL_A if general_A else 0) \
-        | (SSM_FLAG_ZOH_BBAR if zoh else 0)
+        | (SSM_FLAG_ZOH_BBAR if zoh else 0) | (SSM_FLAG_STATIC_B if static_B else 0) \
+        | (SSM_FLAG_STATIC_C if static_C else 0)
     return ssm_problem_t(batch, L, D, B.shape[-1], _io_dtype(x), flags)
 
 
@@ -186,7 +189,7 @@ def saved_state_bytes(problem: ssm_problem_t) -> int:
 
 
 def ssm_scan_fwd(x, delta, A, B, C, D_skip=None, z=None, *, save_states=False, general_A=False, zoh=False, out=None,
-                 saved_states=None, workspace=None, stream=None, h0=None, h_last=None):
+                 saved_states=None, workspace=None, stream=None, h0=None, h_last=None, static_B=False, static_C=False):
     """out = selective_scan(x, delta, A, B, C) (+ D_skip * x) (* silu(z)); see include/ssm_scan.h.
 
     x, delta, z: (batch, L, D) io dtype; B, C: (batch, L, N) io dtype; A: (D, N) float32; D_skip: (D) float32.
@@ -196,9 +199,11 @@ def ssm_scan_fwd(x, delta, A, B, C, D_skip=None, z=None, *, save_states=False, g
     (ssm_scan_fwd_state).
     """
     lib = load_library()
-    prob = make_problem(x, B, z is not None, D_skip is not None, save_states, general_A, zoh)
+    prob = make_problem(x, B, z is not None, D_skip is not None, save_states, general_A, zoh, static_B, static_C)
     batch, L, D, N = prob.batch, prob.L, prob.D, prob.N
     io = x.dtype
+    bshape, bdt = ((D, N), torch.float32) if static_B else ((batch, L, N), io)   # static: a parameter like A
+    cshape, cdt = ((D, N), torch.float32) if static_C else ((batch, L, N), io)
     if out is None:
         out = torch.empty_like(x)
     if save_states and saved_states is None:
@@ -208,8 +213,8 @@ def ssm_scan_fwd(x, delta, A, B, C, D_skip=None, z=None, *, save_states=False, g
     ws = workspace if workspace is not None else _workspace(need, x.device, stream_ptr)
     code = lib.ssm_scan_fwd_state(
         ctypes.byref(prob), _dev_ptr(x, "x", (batch, L, D), io), _dev_ptr(delta, "delta", (batch, L, D), io),
-        _dev_ptr(A, "A", (D, N), torch.float32), _dev_ptr(B, "B", (batch, L, N), io),
-        _dev_ptr(C, "C", (batch, L, N), io), _dev_ptr(D_skip, "D_skip", (D,), torch.float32),
+        _dev_ptr(A, "A", (D, N), torch.float32), _dev_ptr(B, "B", bshape, bdt),
+        _dev_ptr(C, "C", cshape, cdt), _dev_ptr(D_skip, "D_skip", (D,), torch.float32),
         _dev_ptr(z, "z", (batch, L, D), io), _dev_ptr(h0, "h0", (batch, D, N), torch.float32),
         _dev_ptr(out, "out", (batch, L, D), io), _dev_ptr(h_last, "h_last", (batch, D, N), torch.float32),
         _dev_ptr(saved_states if save_states else None, "saved_states"),
@@ -282,7 +287,7 @@ def ssm_scan_bwd_fused_dt(x, delta_pre, delta_bias, A, B, C, D_skip, z, dout, sa
     return o
 
 
-def ssm_step(x, delta, A, B, C, D_skip, z, h, *, zoh=False, out=None, stream=None):
+def ssm_step(x, delta, A, B, C, D_skip, z, h, *, zoh=False, out=None, stream=None, static_B=False, static_C=False):
     """One recurrent step: x, delta, z (batch, D), B, C (batch, N) io dtype; h (batch, D, N) float32 is updated in
     place.  Returns out (batch, D)."""
     lib = load_library()
@@ -290,14 +295,17 @@ def ssm_step(x, delta, A, B, C, D_skip, z, h, *, zoh=False, out=None, stream=Non
     N = B.shape[-1]
     prob = ssm_problem_t(batch, 1, D, N, _io_dtype(x),
                          (SSM_FLAG_HAS_Z if z is not None else 0) | (SSM_FLAG_HAS_DSKIP if D_skip is not None else 0)
-                         | (SSM_FLAG_ZOH_BBAR if zoh else 0))
+                         | (SSM_FLAG_ZOH_BBAR if zoh else 0) | (SSM_FLAG_STATIC_B if static_B else 0)
+                         | (SSM_FLAG_STATIC_C if static_C else 0))
     io = x.dtype
     if out is None:
         out = torch.empty_like(x)
     stream_ptr = (stream if stream is not None else torch.cuda.current_stream(x.device)).cuda_stream
     code = lib.ssm_step(
         ctypes.byref(prob), _dev_ptr(x, "x", (batch, D), io), _dev_ptr(delta, "delta", (batch, D), io),
-        _dev_ptr(A, "A", (D, N), torch.float32), _dev_ptr(B, "B", (batch, N), io), _dev_ptr(C, "C", (batch, N), io),
+        _dev_ptr(A, "A", (D, N), torch.float32),
+        _dev_ptr(B, "B", (D, N) if static_B else (batch, N), torch.float32 if static_B else io),
+        _dev_ptr(C, "C", (D, N) if static_C else (batch, N), torch.float32 if static_C else io),
         _dev_ptr(D_skip, "D_skip", (D,), torch.float32), _dev_ptr(z, "z", (batch, D), io),
         _dev_ptr(h, "h", (batch, D, N), torch.float32), _dev_ptr(out, "out", (batch, D), io),
         ctypes.c_void_p(stream_ptr))
@@ -344,26 +352,30 @@ def ssm_scan_fwd_static(x, delta, A, B, C, D_skip=None, z=None, *, save_states=F
 
 
 def ssm_scan_bwd(x, delta, A, B, C, D_skip, z, dout, saved_states=None, *, general_A=False, zoh=False, workspace=None,
-                 stream=None, outputs=None, extra_flags=0, h0=None, dh_last=None, want_dh0=False):
+                 stream=None, outputs=None, extra_flags=0, h0=None, dh_last=None, want_dh0=False, static_B=False,
+                 static_C=False):
     """Gradients of sum(dout * out) w.r.t. x, delta, A, B, C, D_skip, z; see include/ssm_scan.h.
 
     Returns a dict with dx, ddelta, dz (io dtype, (batch, L, D)); dB, dC (io dtype, (batch, L, N)); dA (float32, (D, N));
     dD (float32, (D)).  dz / dD are None when z / D_skip is None.  `outputs` may pass preallocated tensors.
     With h0, dh_last or want_dh0 the call goes through ssm_scan_bwd_state: h0 / dh_last (batch, D, N) float32 are the
     state before the first step and the gradient arriving at the state after the last step, and the dict also holds
-    dh0 (batch, D, N) float32.
+    dh0 (batch, D, N) float32.  With static_B / static_C, B / C is a float32 (D, N) parameter and dB / dC is its
+    float32 (D, N) gradient.
     """
     lib = load_library()
-    prob = make_problem(x, B, z is not None, D_skip is not None, False, general_A, zoh)
+    prob = make_problem(x, B, z is not None, D_skip is not None, False, general_A, zoh, static_B, static_C)
     prob.flags |= int(extra_flags)
     batch, L, D, N = prob.batch, prob.L, prob.D, prob.N
     io = x.dtype
+    bshape, bdt = ((D, N), torch.float32) if static_B else ((batch, L, N), io)
+    cshape, cdt = ((D, N), torch.float32) if static_C else ((batch, L, N), io)
     o = dict(outputs or {})
     o.setdefault("dx", torch.empty_like(x))
     o.setdefault("ddelta", torch.empty_like(x))
     o.setdefault("dA", torch.empty((D, N), dtype=torch.float32, device=x.device))
     o.setdefault("dB", torch.empty_like(B))
-    o.setdefault("dC", torch.empty_like(B))
+    o.setdefault("dC", torch.empty_like(C))
     if D_skip is not None:
         o.setdefault("dD", torch.empty((D,), dtype=torch.float32, device=x.device))
     else:
@@ -381,13 +393,13 @@ def ssm_scan_bwd(x, delta, A, B, C, D_skip, z, dout, saved_states=None, *, gener
             o.setdefault("dh0", torch.empty((batch, D, N), dtype=f32, device=x.device))
         code = lib.ssm_scan_bwd_state(
             ctypes.byref(prob), _dev_ptr(x, "x", (batch, L, D), io), _dev_ptr(delta, "delta", (batch, L, D), io),
-            _dev_ptr(A, "A", (D, N), f32), _dev_ptr(B, "B", (batch, L, N), io), _dev_ptr(C, "C", (batch, L, N), io),
+            _dev_ptr(A, "A", (D, N), f32), _dev_ptr(B, "B", bshape, bdt), _dev_ptr(C, "C", cshape, cdt),
             _dev_ptr(D_skip, "D_skip", (D,), f32), _dev_ptr(z, "z", (batch, L, D), io),
             _dev_ptr(dout, "dout", (batch, L, D), io), _dev_ptr(h0, "h0", (batch, D, N), f32),
             _dev_ptr(dh_last, "dh_last", (batch, D, N), f32), _dev_ptr(saved_states, "saved_states"),
             _dev_ptr(o["dx"], "dx", (batch, L, D), io), _dev_ptr(o["ddelta"], "ddelta", (batch, L, D), io),
-            _dev_ptr(o["dA"], "dA", (D, N), f32), _dev_ptr(o["dB"], "dB", (batch, L, N), io),
-            _dev_ptr(o["dC"], "dC", (batch, L, N), io), _dev_ptr(o["dD"], "dD", (D,), f32),
+            _dev_ptr(o["dA"], "dA", (D, N), f32), _dev_ptr(o["dB"], "dB", bshape, bdt),
+            _dev_ptr(o["dC"], "dC", cshape, cdt), _dev_ptr(o["dD"], "dD", (D,), f32),
             _dev_ptr(o["dz"], "dz", (batch, L, D), io), _dev_ptr(o.get("dh0"), "dh0", (batch, D, N), f32),
             _dev_ptr(ws, "workspace"), ctypes.c_size_t(0 if ws is None else ws.numel() * ws.element_size()),
             ctypes.c_void_p(stream_ptr))
@@ -395,13 +407,13 @@ def ssm_scan_bwd(x, delta, A, B, C, D_skip, z, dout, saved_states=None, *, gener
         return o
     code = lib.ssm_scan_bwd(
         ctypes.byref(prob), _dev_ptr(x, "x", (batch, L, D), io), _dev_ptr(delta, "delta", (batch, L, D), io),
-        _dev_ptr(A, "A", (D, N), torch.float32), _dev_ptr(B, "B", (batch, L, N), io),
-        _dev_ptr(C, "C", (batch, L, N), io), _dev_ptr(D_skip, "D_skip", (D,), torch.float32),
+        _dev_ptr(A, "A", (D, N), torch.float32), _dev_ptr(B, "B", bshape, bdt),
+        _dev_ptr(C, "C", cshape, cdt), _dev_ptr(D_skip, "D_skip", (D,), torch.float32),
         _dev_ptr(z, "z", (batch, L, D), io), _dev_ptr(dout, "dout", (batch, L, D), io),
         _dev_ptr(saved_states, "saved_states"),
         _dev_ptr(o["dx"], "dx", (batch, L, D), io), _dev_ptr(o["ddelta"], "ddelta", (batch, L, D), io),
-        _dev_ptr(o["dA"], "dA", (D, N), torch.float32), _dev_ptr(o["dB"], "dB", (batch, L, N), io),
-        _dev_ptr(o["dC"], "dC", (batch, L, N), io), _dev_ptr(o["dD"], "dD", (D,), torch.float32),
+        _dev_ptr(o["dA"], "dA", (D, N), torch.float32), _dev_ptr(o["dB"], "dB", bshape, bdt),
+        _dev_ptr(o["dC"], "dC", cshape, cdt), _dev_ptr(o["dD"], "dD", (D,), torch.float32),
         _dev_ptr(o["dz"], "dz", (batch, L, D), io),
         _dev_ptr(ws, "workspace"), ctypes.c_size_t(0 if ws is None else ws.numel() * ws.element_size()),
         ctypes.c_void_p(stream_ptr))

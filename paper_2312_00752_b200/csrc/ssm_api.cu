@@ -16,7 +16,7 @@ static ssm_status_t validate_problem(const ssm_problem_t* p) {
   if (p == nullptr) return SSM_ERR_INVALID_ARG;
   if (p->batch < 1 || p->L < 1 || p->D < 1 || p->N < 1) return SSM_ERR_INVALID_ARG;
   if (p->flags & ~(uint32_t)(SSM_FLAG_HAS_Z | SSM_FLAG_HAS_DSKIP | SSM_FLAG_SAVE_STATES | SSM_FLAG_GENERAL_A | SSM_FLAG_TEST_WITHHOLD |
-                             SSM_FLAG_DELTA_SOFTPLUS | SSM_FLAG_ZOH_BBAR))
+                             SSM_FLAG_DELTA_SOFTPLUS | SSM_FLAG_ZOH_BBAR | SSM_FLAG_STATIC_B | SSM_FLAG_STATIC_C))
     return SSM_ERR_INVALID_ARG;
   if (p->io_dtype != SSM_F32 && p->io_dtype != SSM_BF16) return SSM_ERR_UNSUPPORTED;
   if (p->N != 1 && p->N != 2 && p->N != 4 && p->N != 8 && p->N != 16) return SSM_ERR_UNSUPPORTED;
@@ -90,6 +90,7 @@ static FwdWorkspace fwd_layout(const ssm_problem_t& p, const Plan& pl) {
 
 struct BwdWorkspace {
   size_t dBC_part, dA_part, dD_part, dbias_part, ckpt, seg_local, seg_dsum, mu_in, fwd, sched, handoff, total;
+  size_t dBs_part, dCs_part;   // static B / C
 };
 static BwdWorkspace bwd_layout(const ssm_problem_t& p, const Plan& pl, const Plan& pl_fwd) {
   BwdWorkspace w{};
@@ -116,11 +117,19 @@ static BwdWorkspace bwd_layout(const ssm_problem_t& p, const Plan& pl, const Pla
   const size_t chains = parts * pl.bwd_groups;   // (batch, segment, channel group) chains of the tuned kernel
   w.sched = take((64 + chains) * sizeof(int));
   w.handoff = take(chains * bwd_fast_handoff_bytes_per_chain());
+  if (p.flags & SSM_FLAG_STATIC_B) w.dBs_part = take(parts * p.D * p.N * sizeof(float));
+  if (p.flags & SSM_FLAG_STATIC_C) w.dCs_part = take(parts * p.D * p.N * sizeof(float));
   w.total = off;
   return w;
 }
 
 static bool aligned_to(const void* ptr, size_t a) { return (reinterpret_cast<uintptr_t>(ptr) % a) == 0; }
+// static B / C (and their gradients) are float32 whatever the io dtype
+static bool static_bc_aligned(const ssm_problem_t& p, const void* B, const void* C, const void* dB, const void* dC) {
+  const bool sb = p.flags & SSM_FLAG_STATIC_B, sc = p.flags & SSM_FLAG_STATIC_C;
+  return (!sb || (aligned_to(B, 4) && (dB == nullptr || aligned_to(dB, 4)))) &&
+         (!sc || (aligned_to(C, 4) && (dC == nullptr || aligned_to(dC, 4))));
+}
 
 static ssm_status_t check_ws(const void* ws, size_t have, size_t need) {
   if (need == 0) return SSM_OK;
@@ -232,6 +241,7 @@ static ssm_status_t fwd_impl(const ssm_problem_t* p, const void* x, const void* 
   const size_t esz = p->io_dtype == SSM_BF16 ? 2 : 4;
   for (const void* q : {x, delta, B, C, z, (const void*)out})
     if (q && !aligned_to(q, esz)) return SSM_ERR_INVALID_ARG;
+  if (!static_bc_aligned(*p, B, C, nullptr, nullptr)) return SSM_ERR_INVALID_ARG;
   for (const void* q : {(const void*)A, (const void*)D_skip, (const void*)saved_states, (const void*)h0, (const void*)h_last,
                         (const void*)delta_bias})
     if (q && !aligned_to(q, 4)) return SSM_ERR_INVALID_ARG;
@@ -257,6 +267,8 @@ static ssm_status_t fwd_impl(const ssm_problem_t* p, const void* x, const void* 
   fp.nck = pl.nck;
   fp.general_A = (p->flags & SSM_FLAG_GENERAL_A) ? 1 : 0;
   fp.zoh = (p->flags & SSM_FLAG_ZOH_BBAR) ? 1 : 0;
+  fp.static_B = (p->flags & SSM_FLAG_STATIC_B) ? 1 : 0;
+  fp.static_C = (p->flags & SSM_FLAG_STATIC_C) ? 1 : 0;
   fp.delta_bias = delta_bias;
   fp.softplus = (p->flags & SSM_FLAG_DELTA_SOFTPLUS) ? 1 : 0;
   const float* h_start = nullptr;
@@ -302,6 +314,7 @@ ssm_status_t ssm_step(const ssm_problem_t* p, const void* x, const void* delta, 
   const size_t esz = p->io_dtype == SSM_BF16 ? 2 : 4;
   for (const void* q : {x, delta, B, C, z, (const void*)out})
     if (q && !aligned_to(q, esz)) return SSM_ERR_INVALID_ARG;
+  if (!static_bc_aligned(*p, B, C, nullptr, nullptr)) return SSM_ERR_INVALID_ARG;
   for (const void* q : {(const void*)A, (const void*)D_skip, (const void*)h})
     if (q && !aligned_to(q, 4)) return SSM_ERR_INVALID_ARG;
   StepParams sp{};
@@ -318,6 +331,8 @@ ssm_status_t ssm_step(const ssm_problem_t* p, const void* x, const void* delta, 
   sp.D = p->D;
   sp.N = p->N;
   sp.zoh = (p->flags & SSM_FLAG_ZOH_BBAR) ? 1 : 0;
+  sp.static_B = (p->flags & SSM_FLAG_STATIC_B) ? 1 : 0;
+  sp.static_C = (p->flags & SSM_FLAG_STATIC_C) ? 1 : 0;
   if (launch_step(*p, sp, static_cast<cudaStream_t>(stream)) != cudaSuccess) return SSM_ERR_CUDA;
   return SSM_OK;
 }
@@ -336,6 +351,7 @@ static ssm_status_t bwd_impl(const ssm_problem_t* p, const void* x, const void* 
   for (const void* q : {x, delta, B, C, z, dout, (const void*)dx, (const void*)ddelta, (const void*)dB,
                         (const void*)dC, (const void*)dz})
     if (q && !aligned_to(q, esz)) return SSM_ERR_INVALID_ARG;
+  if (!static_bc_aligned(*p, B, C, dB, dC)) return SSM_ERR_INVALID_ARG;
   for (const void* q : {(const void*)A, (const void*)D_skip, saved_states, (const void*)dA, (const void*)dD,
                         (const void*)delta_bias, (const void*)ddelta_bias, (const void*)h0, (const void*)dh_last,
                         (const void*)dh0})
@@ -365,6 +381,8 @@ static ssm_status_t bwd_impl(const ssm_problem_t* p, const void* x, const void* 
     fp.nck = pl_fwd.nck;
     fp.general_A = (p->flags & SSM_FLAG_GENERAL_A) ? 1 : 0;
     fp.zoh = (p->flags & SSM_FLAG_ZOH_BBAR) ? 1 : 0;
+    fp.static_B = (p->flags & SSM_FLAG_STATIC_B) ? 1 : 0;
+    fp.static_C = (p->flags & SSM_FLAG_STATIC_C) ? 1 : 0;
     fp.delta_bias = delta_bias;
     fp.softplus = (p->flags & SSM_FLAG_DELTA_SOFTPLUS) ? 1 : 0;
     const float* h_start = nullptr;
@@ -400,6 +418,10 @@ static ssm_status_t bwd_impl(const ssm_problem_t* p, const void* x, const void* 
   bp.groups = pl.bwd_groups;
   bp.general_A = (p->flags & SSM_FLAG_GENERAL_A) ? 1 : 0;
   bp.zoh = (p->flags & SSM_FLAG_ZOH_BBAR) ? 1 : 0;
+  bp.static_B = (p->flags & SSM_FLAG_STATIC_B) ? 1 : 0;
+  bp.static_C = (p->flags & SSM_FLAG_STATIC_C) ? 1 : 0;
+  bp.dBs_part = bp.static_B ? reinterpret_cast<float*>(ws + w.dBs_part) : nullptr;
+  bp.dCs_part = bp.static_C ? reinterpret_cast<float*>(ws + w.dCs_part) : nullptr;
   bp.test_withhold = (p->flags & SSM_FLAG_TEST_WITHHOLD) ? 1 : 0;
   bp.delta_bias = delta_bias;
   bp.softplus = (p->flags & SSM_FLAG_DELTA_SOFTPLUS) ? 1 : 0;
@@ -434,8 +456,12 @@ static ssm_status_t bwd_impl(const ssm_problem_t* p, const void* x, const void* 
 
   ReduceParams rp{};
   rp.dBC_part = bp.dBC_part;
-  rp.dB = dB;
-  rp.dC = dC;
+  rp.dB = bp.static_B ? nullptr : dB;   // static B / C: float32 [D][N] sums over batch and time instead
+  rp.dC = bp.static_C ? nullptr : dC;
+  rp.dBs = bp.static_B ? static_cast<float*>(dB) : nullptr;
+  rp.dCs = bp.static_C ? static_cast<float*>(dC) : nullptr;
+  rp.dBs_part = bp.dBs_part;
+  rp.dCs_part = bp.dCs_part;
   rp.dA_part = bp.dA_part;
   rp.dD_part = bp.dD_part;
   rp.dA = dA;

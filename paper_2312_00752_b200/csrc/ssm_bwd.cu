@@ -80,12 +80,16 @@ __global__ void __launch_bounds__(BwdGeom<N>::THREADS) ssm_bwd_kernel(const BwdP
   const bool has_z = gz != nullptr;
 
   float Ar[S], A2[S], mu[S], dA[S];
+  float Bst[S], Cst[S], dBs[S], dCs[S];   // static B / C (parameters [D][N]) and their gradient sums over time
   float dD_acc = 0.f, dbias_acc = 0.f;
   const float Dk = (valid && p.Dskip != nullptr) ? p.Dskip[d] : 0.f;
   const float dbias = (valid && p.delta_bias != nullptr) ? p.delta_bias[d] : 0.f;
 #pragma unroll
   for (int k = 0; k < S; ++k) {
     Ar[k] = valid ? p.A[(size_t)d * N + j * S + k] : 0.f;
+    Bst[k] = (valid && p.static_B) ? static_cast<const float*>(p.B)[(size_t)d * N + j * S + k] : 0.f;
+    Cst[k] = (valid && p.static_C) ? static_cast<const float*>(p.C)[(size_t)d * N + j * S + k] : 0.f;
+    dBs[k] = dCs[k] = 0.f;
     A2[k] = Ar[k] * kLog2e;
     mu[k] = (valid && p.mu_in != nullptr) ? p.mu_in[(((size_t)b * p.nseg + seg) * D + d) * N + j * S + k] : 0.f;
     dA[k] = 0.f;
@@ -110,8 +114,8 @@ __global__ void __launch_bounds__(BwdGeom<N>::THREADS) ssm_bwd_kernel(const BwdP
     }
     for (int i = tid; i < T * N; i += kBwdThreads) {
       const bool ok = i / N < nt;
-      s_B[i] = ok ? io_to_float<IO>(gB[row0 * N + i]) : 0.f;
-      s_C[i] = ok ? io_to_float<IO>(gC[row0 * N + i]) : 0.f;
+      s_B[i] = (ok && !p.static_B) ? io_to_float<IO>(gB[row0 * N + i]) : 0.f;
+      s_C[i] = (ok && !p.static_C) ? io_to_float<IO>(gC[row0 * N + i]) : 0.f;
     }
     float h[S];
 #pragma unroll
@@ -130,16 +134,17 @@ __global__ void __launch_bounds__(BwdGeom<N>::THREADS) ssm_bwd_kernel(const BwdP
       float y = 0.f;
 #pragma unroll
       for (int k = 0; k < S; ++k) {
-        float a, bx = du * s_B[tt * N + j * S + k];
+        const float Bk = p.static_B ? Bst[k] : s_B[tt * N + j * S + k];
+        float a, bx = du * Bk;
         if (p.zoh) {
           float E;
           zoh_discretize(dt, Ar[k], a, E);
-          bx = E * u * s_B[tt * N + j * S + k];
+          bx = E * u * Bk;
         } else {
           a = ex2_approx(dt * A2[k]);
         }
         h[k] = fmaf(a, h[k], bx);
-        y = fmaf(s_C[tt * N + j * S + k], h[k], y);
+        y = fmaf(p.static_C ? Cst[k] : s_C[tt * N + j * S + k], h[k], y);
         s_h[((size_t)(tt + 1) * CH + slot) * N + j * S + k] = h[k];
       }
 #pragma unroll
@@ -170,8 +175,8 @@ __global__ void __launch_bounds__(BwdGeom<N>::THREADS) ssm_bwd_kernel(const BwdP
       for (int k = 0; k < S; ++k) {
         const float ht = s_h[((size_t)(tt + 1) * CH + slot) * N + j * S + k];
         const float hp = s_h[((size_t)tt * CH + slot) * N + j * S + k];
-        const float Bn = s_B[tt * N + j * S + k];
-        const float lam = fmaf(s_C[tt * N + j * S + k], ds, mu[k]);
+        const float Bn = p.static_B ? Bst[k] : s_B[tt * N + j * S + k];
+        const float lam = fmaf(p.static_C ? Cst[k] : s_C[tt * N + j * S + k], ds, mu[k]);
         dCp[k] = ds * ht;
         float a;
         if (p.zoh) {
@@ -187,6 +192,8 @@ __global__ void __launch_bounds__(BwdGeom<N>::THREADS) ssm_bwd_kernel(const BwdP
           dBp[k] = lam * du;
           lamB = fmaf(lam, Bn, lamB);
         }
+        dBs[k] += dBp[k];   // static B / C: the same terms summed over time instead of over channels
+        dCs[k] += dCp[k];
         mu[k] = a * lam;
         const float w = mu[k] * hp;
         wA = fmaf(w, Ar[k], wA);
@@ -251,6 +258,11 @@ __global__ void __launch_bounds__(BwdGeom<N>::THREADS) ssm_bwd_kernel(const BwdP
     for (int k = 0; k < S; ++k) p.dA_part[(part * D + d) * N + j * S + k] = dA[k];
     if (j == 0) p.dD_part[part * D + d] = dD_acc;
     if (j == 0 && p.dbias_part != nullptr) p.dbias_part[part * D + d] = dbias_acc;
+#pragma unroll
+    for (int k = 0; k < S; ++k) {
+      if (p.static_B) p.dBs_part[(part * D + d) * N + j * S + k] = dBs[k];
+      if (p.static_C) p.dCs_part[(part * D + d) * N + j * S + k] = dCs[k];
+    }
     if (seg == 0 && p.dh0 != nullptr) {
 #pragma unroll
       for (int k = 0; k < S; ++k) p.dh0[((size_t)b * D + d) * N + j * S + k] = mu[k];
@@ -283,11 +295,12 @@ __global__ void __launch_bounds__(BwdGeom<N>::THREADS) ssm_bwd_local_kernel(cons
   const int t_end = min(p.L, t_begin + p.seg_steps);
   const bool has_z = gz != nullptr;
 
-  float A2[S], mu[S], dsum = 0.f;
+  float A2[S], mu[S], Cst[S], dsum = 0.f;
   const float dbias = (valid && p.delta_bias != nullptr) ? p.delta_bias[d] : 0.f;
 #pragma unroll
   for (int k = 0; k < S; ++k) {
     A2[k] = valid ? p.A[(size_t)d * N + j * S + k] * kLog2e : 0.f;
+    Cst[k] = (valid && p.static_C) ? static_cast<const float*>(p.C)[(size_t)d * N + j * S + k] : 0.f;
     mu[k] = 0.f;
   }
   for (int kb = (t_end - 1) / T; kb >= t_begin / T; --kb) {
@@ -304,7 +317,8 @@ __global__ void __launch_bounds__(BwdGeom<N>::THREADS) ssm_bwd_local_kernel(cons
       s_z[i] = (ok && has_z) ? gz[g] : zero;
       s_g[i] = ok ? gg[g] : zero;
     }
-    for (int i = tid; i < T * N; i += kBwdThreads) s_C[i] = (i / N < nt) ? io_to_float<IO>(gC[row0 * N + i]) : 0.f;
+    for (int i = tid; i < T * N; i += kBwdThreads)
+      s_C[i] = (i / N < nt && !p.static_C) ? io_to_float<IO>(gC[row0 * N + i]) : 0.f;
     __syncthreads();
     for (int tt = nt - 1; tt >= 0; --tt) {
       float dt = io_to_float<IO>(s_d[tt * CH + slot]) + dbias;
@@ -316,7 +330,8 @@ __global__ void __launch_bounds__(BwdGeom<N>::THREADS) ssm_bwd_local_kernel(cons
       }
       dsum += dt;
 #pragma unroll
-      for (int k = 0; k < S; ++k) mu[k] = ex2_approx(dt * A2[k]) * fmaf(s_C[tt * N + j * S + k], ds, mu[k]);
+      for (int k = 0; k < S; ++k)
+        mu[k] = ex2_approx(dt * A2[k]) * fmaf(p.static_C ? Cst[k] : s_C[tt * N + j * S + k], ds, mu[k]);
     }
   }
   if (valid) {
@@ -338,14 +353,24 @@ __global__ void __launch_bounds__(256) ssm_bwd_reduce_kernel(const ReduceParams 
       sb += p.dBC_part[((size_t)g * 2 + 0) * p.bln + i];
       sc += p.dBC_part[((size_t)g * 2 + 1) * p.bln + i];
     }
-    static_cast<IO*>(p.dB)[i] = float_to_io<IO>(sb);
-    static_cast<IO*>(p.dC)[i] = float_to_io<IO>(sc);
+    if (p.dB != nullptr) static_cast<IO*>(p.dB)[i] = float_to_io<IO>(sb);
+    if (p.dC != nullptr) static_cast<IO*>(p.dC)[i] = float_to_io<IO>(sc);
   }
   const long long dn = (long long)p.D * p.N;
   if (i < dn) {
     float sa = 0.f;
     for (int q = 0; q < p.parts; ++q) sa += p.dA_part[(size_t)q * dn + i];
     p.dA[i] = sa;
+    if (p.dBs != nullptr) {
+      float v = 0.f;
+      for (int q = 0; q < p.parts; ++q) v += p.dBs_part[(size_t)q * dn + i];
+      p.dBs[i] = v;
+    }
+    if (p.dCs != nullptr) {
+      float v = 0.f;
+      for (int q = 0; q < p.parts; ++q) v += p.dCs_part[(size_t)q * dn + i];
+      p.dCs[i] = v;
+    }
   }
   if (p.dD != nullptr && i < p.D) {
     float sd = 0.f;

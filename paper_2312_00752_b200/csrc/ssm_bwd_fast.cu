@@ -594,7 +594,7 @@ __global__ void __launch_bounds__(kBwdFastThreads) ssm_bwd_fast_kernel(const Bwd
 
 bool bwd_fast_applicable(const ssm_problem_t& prob, const BwdParams& p) {
   auto al16 = [](const void* q) { return q == nullptr || (reinterpret_cast<uintptr_t>(q) & 15) == 0; };
-  if (p.zoh) return false;  // the tuned kernel implements the default rule B-bar = delta * B only
+  if (p.zoh || p.static_B || p.static_C) return false;  // default rule and input-dependent B, C only
   // work items are numbered with 32-bit integers (one spare bit for the claims that run past the end)
   const long long items = (long long)p.batch * p.nseg * ((p.D + kBwdFastCH - 1) / kBwdFastCH) * (p.seg_steps / kBT);
   if (items > (1LL << 30)) return false;

@@ -237,6 +237,7 @@ __global__ void __launch_bounds__(kThreads) ssm_bwd_local_fast_kernel(const BwdP
 
 bool bwd_local_fast_applicable(const ssm_problem_t& prob, const BwdParams& p) {
   auto al16 = [](const void* q) { return q == nullptr || (reinterpret_cast<uintptr_t>(q) & 15) == 0; };
+  if (p.static_C) return false;
   return prob.io_dtype == SSM_BF16 && prob.N == 16 && prob.D % 8 == 0 && al16(p.delta) && al16(p.z) && al16(p.dout) &&
          al16(p.C) && al16(p.A) && al16(p.seg_local);
 }

@@ -48,6 +48,7 @@ struct FwdParams {
   int batch, L, D, nseg, seg_steps, nck;
   int general_A;       // 1: never take the arithmetic-progression fast path
   int zoh;             // 1: B-bar = (exp(delta A) - 1) / A * B (Eq. 4) instead of delta * B
+  int static_B, static_C;  // 1: B / C is a float32 [D][N] parameter (not input-dependent: Algorithm 1) instead of [batch][L][N]
 };
 
 struct CarryParams {
@@ -88,6 +89,9 @@ struct BwdParams {
   float* dh0;             // [batch][D][N] gradient of the initial state (the adjoint mu that leaves the first step);
                           // null: not wanted
   int zoh;                // as in FwdParams
+  int static_B, static_C;  // as in FwdParams
+  float* dBs_part;        // static B: [batch*nseg][D][N] per-thread sums over time of the dB terms
+  float* dCs_part;        // static C: same for dC
   int test_withhold;      // test hook: never publish hand-off flags, poll only 1000 times
   int* sched;             // tuned kernel: [0] claim counter, [1] abort word, [64 + chain] progress flag per chain
   float4* handoff;        // tuned kernel: carried values between consecutive tiles of a chain
@@ -105,6 +109,10 @@ struct ReduceParams {
   float* dbias;           // null: skip
   long long bln;          // batch*L*N
   int groups, parts, D, N;
+  const float* dBs_part;  // static B / C: [parts][D*N] partial sums; null: B / C are input-dependent
+  const float* dCs_part;
+  float* dBs;             // static B: float32 [D][N] (then dB above is null)
+  float* dCs;
 };
 
 cudaError_t launch_fwd(const ssm_problem_t& prob, const Plan& plan, const FwdParams& p, int mode, cudaStream_t s);
@@ -124,6 +132,7 @@ struct StepParams {
   void* out;            // [batch][D]
   int batch, D, N;
   int zoh;              // as in FwdParams
+  int static_B, static_C;  // as in FwdParams
 };
 cudaError_t launch_step(const ssm_problem_t& prob, const StepParams& p, cudaStream_t s);
 

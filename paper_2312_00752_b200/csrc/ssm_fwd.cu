@@ -57,6 +57,7 @@ __global__ void __launch_bounds__(fwd_threads(N)) ssm_fwd_kernel(const FwdParams
   const int D = p.D;
 
   float A2[CPT][S], Ar[CPT][S], h[CPT][S], dsum[CPT], dbias[CPT];
+  float Bst[CPT][S], Cst[CPT][S];   // static B / C (parameters [D][N]): this thread's entries
 #pragma unroll
   for (int q = 0; q < CPT; ++q) {
     const int d = d_thr + q;
@@ -66,6 +67,8 @@ __global__ void __launch_bounds__(fwd_threads(N)) ssm_fwd_kernel(const FwdParams
 #pragma unroll
     for (int k = 0; k < S; ++k) {
       Ar[q][k] = valid ? p.A[(size_t)d * N + j * S + k] : 0.f;
+      Bst[q][k] = (valid && p.static_B) ? static_cast<const float*>(p.B)[(size_t)d * N + j * S + k] : 0.f;
+      Cst[q][k] = (valid && p.static_C) ? static_cast<const float*>(p.C)[(size_t)d * N + j * S + k] : 0.f;
       A2[q][k] = Ar[q][k] * kLog2e;
       h[q][k] = (valid && p.h_start != nullptr)
                     ? p.h_start[(((size_t)b * p.nseg + seg) * D + d) * N + j * S + k]
@@ -100,8 +103,8 @@ __global__ void __launch_bounds__(fwd_threads(N)) ssm_fwd_kernel(const FwdParams
       const int tt = i / N, n = i % N;
       const bool ok = tt < nt;
       const size_t g = (row0 + tt) * N + n;
-      s_B[tt][n] = ok ? io_to_float<IO>(gB[g]) : 0.f;
-      if constexpr (kReadout) s_C[tt][n] = ok ? io_to_float<IO>(gC[g]) : 0.f;
+      s_B[tt][n] = (ok && !p.static_B) ? io_to_float<IO>(gB[g]) : 0.f;
+      if constexpr (kReadout) s_C[tt][n] = (ok && !p.static_C) ? io_to_float<IO>(gC[g]) : 0.f;
     }
     if (MODE != kFwdSummary && p.ckpt != nullptr && (t0 % kCkptSteps) == 0) {
       const int kc = t0 / kCkptSteps;
@@ -136,16 +139,17 @@ __global__ void __launch_bounds__(fwd_threads(N)) ssm_fwd_kernel(const FwdParams
         y[q] = 0.f;
 #pragma unroll
         for (int k = 0; k < S; ++k) {
-          float a, bx = du * Bv[k];
+          const float Bk = p.static_B ? Bst[q][k] : Bv[k];
+          float a, bx = du * Bk;
           if (p.zoh) {
             float E;
             zoh_discretize(dt, Ar[q][k], a, E);
-            bx = E * u[q] * Bv[k];
+            bx = E * u[q] * Bk;
           } else {
             a = ex2_approx(dt * A2[q][k]);
           }
           h[q][k] = fmaf(a, h[q][k], bx);
-          if constexpr (kReadout) y[q] = fmaf(Cv[k], h[q][k], y[q]);
+          if constexpr (kReadout) y[q] = fmaf(p.static_C ? Cst[q][k] : Cv[k], h[q][k], y[q]);
         }
       }
       if constexpr (kReadout) {

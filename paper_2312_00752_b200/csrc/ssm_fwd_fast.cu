@@ -391,7 +391,7 @@ static cudaError_t launch_fast(const Plan& plan, const FwdParams& p, cudaStream_
 
 bool fwd_fast_applicable(const ssm_problem_t& prob, const FwdParams& p) {
   auto al16 = [](const void* q) { return q == nullptr || (reinterpret_cast<uintptr_t>(q) & 15) == 0; };
-  if (p.zoh) return false;  // the tuned kernel implements the default rule B-bar = delta * B only
+  if (p.zoh || p.static_B || p.static_C) return false;  // default rule and input-dependent B, C only
   return prob.io_dtype == SSM_BF16 && prob.N == 16 && prob.D % 8 == 0 && al16(p.x) && al16(p.delta) && al16(p.z) &&
          al16(p.B) && al16(p.C) && al16(p.out) && al16(p.A) && al16(p.h_start) && al16(p.ckpt) && al16(p.seg_end) && al16(p.h_last);
 }

@@ -19,6 +19,8 @@ __global__ void __launch_bounds__(128) ssm_step_kernel(const StepParams p) {
   const size_t e = (size_t)b * p.D + d;
   const IO* __restrict__ gB = static_cast<const IO*>(p.B) + (size_t)b * N;
   const IO* __restrict__ gC = static_cast<const IO*>(p.C) + (size_t)b * N;
+  const float* __restrict__ sB = static_cast<const float*>(p.B) + (size_t)d * N;   // static B / C: float32 [D][N]
+  const float* __restrict__ sC = static_cast<const float*>(p.C) + (size_t)d * N;
   const float dt = io_to_float<IO>(static_cast<const IO*>(p.delta)[e]);
   const float u = io_to_float<IO>(static_cast<const IO*>(p.x)[e]);
   const float du = dt * u;
@@ -43,16 +45,17 @@ __global__ void __launch_bounds__(128) ssm_step_kernel(const StepParams p) {
   float y = 0.f;
 #pragma unroll
   for (int k = 0; k < N; ++k) {
-    float a, bx = du * io_to_float<IO>(__ldg(gB + k));
+    const float Bk = p.static_B ? __ldg(sB + k) : io_to_float<IO>(__ldg(gB + k));
+    float a, bx = du * Bk;
     if (p.zoh) {
       float E;
       zoh_discretize(dt, av[k], a, E);
-      bx = E * u * io_to_float<IO>(__ldg(gB + k));
+      bx = E * u * Bk;
     } else {
       a = ex2_approx(dt * (av[k] * kLog2e));
     }
     hv[k] = fmaf(a, hv[k], bx);
-    y = fmaf(io_to_float<IO>(__ldg(gC + k)), hv[k], y);
+    y = fmaf(p.static_C ? __ldg(sC + k) : io_to_float<IO>(__ldg(gC + k)), hv[k], y);
   }
   if (N % 4 == 0) {
 #pragma unroll
