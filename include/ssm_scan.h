@@ -11,19 +11,19 @@
  *     s[t]    = sum_n C[b,t,n] * h[t,n] + D_skip[d] * x[b,t,d]               readout, Eq. 2b, plus skip term
  *     out[b,t,d] = s[t] * z[b,t,d] / (1 + exp(-z[b,t,d]))                    SiLU gate
  *
- * B-bar is delta*B (not the zero-order-hold expression of Eq. 4).  delta is the positive step size, i.e. the value
- * AFTER the softplus of Algorithm 2 step 4.  The (batch, L, D, N) tensors a, B-bar and h never exist in device
+ * B-bar is delta*B unless SSM_FLAG_ZOH_BBAR asks for the zero-order-hold expression of Eq. 4.  delta is the positive
+ * step size, i.e. the value AFTER the softplus of Algorithm 2 step 4 (the *_fused_dt calls take the pre-activation).  The (batch, L, D, N) tensors a, B-bar and h never exist in device
  * memory (Section 3.3); long sequences are split in time and the state is carried between the pieces
  * (Appendix D, "we split the sequences into chunks").  The backward pass recomputes the states from saved or
  * rebuilt checkpoint states instead of reading them (Section 3.3 and Appendix D, recomputation).
  *
  * Conventions common to all entry points
- *   - Every pointer except `p` is DEVICE memory owned by the caller; the library never allocates, frees or keeps a
+ *   - Every pointer except `p` is DEVICE memory owned by the caller (ssm_scan_fwd_bwd_host alone takes host buffers); the library never allocates, frees or keeps a
  *     pointer after the call returns.  Scratch memory is the caller's `workspace` (size from the *_workspace_bytes
  *     queries; at least 256-byte aligned; contents undefined between calls; calls that overlap on the GPU must not
  *     share a workspace).
  *   - Layouts are dense row-major: x, delta, z, out, dout, dx, ddelta, dz are [batch][L][D]; B, C, dB, dC are
- *     [batch][L][N]; A, dA are [D][N]; D_skip, dD are [D].
+ *     [batch][L][N] (float32 [D][N] with SSM_FLAG_STATIC_B / _C); A, dA are [D][N]; D_skip, dD are [D].
  *   - x, delta, B, C, z, out, dout, dx, ddelta, dB, dC, dz have the element type `io_dtype`; A, D_skip, dA, dD and
  *     every state are float32; all arithmetic and accumulation is float32; results are rounded once to io_dtype
  *     (round-to-nearest-even).
