@@ -73,8 +73,7 @@ enum {
   SSM_FLAG_GENERAL_A = 8u,    /* do not use the fast path for rows of A that are arithmetic progressions in n   */
   SSM_FLAG_DELTA_SOFTPLUS = 32u, /* ssm_scan_*_fused_dt: the step size is softplus(delta_pre + delta_bias[d])         */
   SSM_FLAG_ZOH_BBAR = 64u,    /* B-bar = (exp(delta A) - 1) / A * B, the zero-order hold of Eq. 4 (delta * B at A = 0),
-                                 instead of the default delta * B; honoured by every call; such problems run on
-                                 the generic kernels                                                             */
+                                 instead of the default delta * B; honoured by every call                        */
   SSM_FLAG_STATIC_B = 256u,   /* B is not input-dependent (Algorithm 1; the selective-parameter ablation, Table 7): B is a float32
                                  parameter [D][N] like A instead of io_dtype [batch][L][N], and dB is float32 [D][N],
                                  summed over batch and time.  Generic kernels.                                    */

@@ -76,7 +76,8 @@ __device__ __forceinline__ void st_release(int* p, int v) {
 
 }  // namespace
 
-template <bool SP>
+// ZOH: B-bar = E B with E = (a - 1) / A (Eq. 4; E = delta where A = 0) instead of delta * B
+template <bool SP, bool ZOH>
 __global__ void __launch_bounds__(kBwdFastThreads) ssm_bwd_fast_kernel(const BwdParams p) {
   constexpr int THREADS = kBwdFastThreads;
   constexpr int CH = kBwdFastCH;
@@ -159,6 +160,8 @@ __global__ void __launch_bounds__(kBwdFastThreads) ssm_bwd_fast_kernel(const Bwd
 
   // ---- state of the chain being processed (set per item)
   float2 A2[2][2], mu[2][2], dA2[2][2];
+  float2 invA[ZOH ? 2 : 1][2];   // ZOH: 1 / A (0 where A = 0)
+  bool zeroA = false;            // ZOH: some A of this warp is exactly 0 (then the slower exact form of E is used)
   float Dk = 0.f, dD_acc = 0.f;
   float bias_pq = 0.f, dbias_acc = 0.f;   // SP: bias of the kept channel, sum of the pre-activation gradient
   int d0 = 0;
@@ -177,6 +180,43 @@ __global__ void __launch_bounds__(kBwdFastThreads) ssm_bwd_fast_kernel(const Bwd
       const float2 e01 = f2mul(f2dup(dt), A2[q][0]), e23 = f2mul(f2dup(dt), A2[q][1]);
       a01 = make_float2(ex2_approx(e01.x), ex2_approx(e01.y));
       a23 = make_float2(ex2_approx(e23.x), ex2_approx(e23.y));
+    }
+  };
+
+  // ZOH input gain of channel q: E = (a - 1) / A, and E = dt where A = 0
+  auto gain = [&](float dt, int q, float2 a01, float2 a23, float2& E01, float2& E23) {
+    E01 = f2mul(f2fma(a01, f2dup(1.f), f2dup(-1.f)), invA[ZOH ? q : 0][0]);
+    E23 = f2mul(f2fma(a23, f2dup(1.f), f2dup(-1.f)), invA[ZOH ? q : 0][1]);
+    if (zeroA) {
+      if (A2[q][0].x == 0.f) E01.x = dt;
+      if (A2[q][0].y == 0.f) E01.y = dt;
+      if (A2[q][1].x == 0.f) E23.x = dt;
+      if (A2[q][1].y == 0.f) E23.y = dt;
+    }
+  };
+  // dE/dA = (dt a - E) / A, and dt^2 / 2 where A = 0
+  auto gain_dA = [&](float dt, int q, float2 a01, float2 a23, float2 E01, float2 E23, float2& G01, float2& G23) {
+    const float2 dd = f2dup(dt);
+    G01 = f2mul(f2fma(dd, a01, f2mul(E01, f2dup(-1.f))), invA[ZOH ? q : 0][0]);
+    G23 = f2mul(f2fma(dd, a23, f2mul(E23, f2dup(-1.f))), invA[ZOH ? q : 0][1]);
+    if (zeroA) {
+      const float hv = 0.5f * dt * dt;
+      if (A2[q][0].x == 0.f) G01.x = hv;
+      if (A2[q][0].y == 0.f) G01.y = hv;
+      if (A2[q][1].x == 0.f) G23.x = hv;
+      if (A2[q][1].y == 0.f) G23.y = hv;
+    }
+  };
+  // input term of the recurrence for channel q: bx = delta x B, or E x B under ZOH
+  auto input_term = [&](float dt, float xu, float dxu, int q, float2 a01, float2 a23, float4 Bq, float2& b01, float2& b23) {
+    if (ZOH) {
+      float2 E01, E23;
+      gain(dt, q, a01, a23, E01, E23);
+      b01 = f2mul(f2mul(E01, f2dup(xu)), make_float2(Bq.x, Bq.y));
+      b23 = f2mul(f2mul(E23, f2dup(xu)), make_float2(Bq.z, Bq.w));
+    } else {
+      b01 = f2mul(f2dup(dxu), make_float2(Bq.x, Bq.y));
+      b23 = f2mul(f2dup(dxu), make_float2(Bq.z, Bq.w));
     }
   };
 
@@ -215,14 +255,16 @@ __global__ void __launch_bounds__(kBwdFastThreads) ssm_bwd_fast_kernel(const Bwd
         const uint32_t dw = SP ? 0u : sm.d[st][tt][slot], xw = sm.x[st][tt][slot];
         const float4 Bq = sm.fB[tt][j];
         const float2 dt2 = step_sizes(st, tt, dw);
-        const float2 du = f2mul(dt2, make_float2(bf16sel(xw, selA), bf16sel(xw, selB)));
-        const float dtq[2] = {dt2.x, dt2.y}, duq[2] = {du.x, du.y};
+        const float2 u2 = make_float2(bf16sel(xw, selA), bf16sel(xw, selB));
+        const float2 du = f2mul(dt2, u2);
+        const float dtq[2] = {dt2.x, dt2.y}, uq[2] = {u2.x, u2.y}, duq[2] = {du.x, du.y};
 #pragma unroll
         for (int q = 0; q < 2; ++q) {
-          float2 a01, a23;
+          float2 a01, a23, b01, b23;
           decays(dtq[q], q, ap_tag, a01, a23);
-          h[q][0] = f2fma(a01, h[q][0], f2mul(f2dup(duq[q]), make_float2(Bq.x, Bq.y)));
-          h[q][1] = f2fma(a23, h[q][1], f2mul(f2dup(duq[q]), make_float2(Bq.z, Bq.w)));
+          input_term(dtq[q], uq[q], duq[q], q, a01, a23, Bq, b01, b23);
+          h[q][0] = f2fma(a01, h[q][0], b01);
+          h[q][1] = f2fma(a23, h[q][1], b23);
         }
       }
 #pragma unroll
@@ -249,15 +291,17 @@ __global__ void __launch_bounds__(kBwdFastThreads) ssm_bwd_fast_kernel(const Bwd
           const uint32_t xw = sm.x[st][tt][slot];
           const float4 Bq = sm.fB[tt][j], Cq = sm.fC[tt][j];
           const float2 dt2 = step_sizes(st, tt, SP ? 0u : sm.d[st][tt][slot]);
-          const float2 du = f2mul(dt2, make_float2(bf16sel(xw, selA), bf16sel(xw, selB)));
-          const float dtq[2] = {dt2.x, dt2.y}, duq[2] = {du.x, du.y};
+          const float2 u2 = make_float2(bf16sel(xw, selA), bf16sel(xw, selB));
+          const float2 du = f2mul(dt2, u2);
+          const float dtq[2] = {dt2.x, dt2.y}, uq[2] = {u2.x, u2.y}, duq[2] = {du.x, du.y};
           float y[2];
 #pragma unroll
           for (int q = 0; q < 2; ++q) {
-            float2 a01, a23;
+            float2 a01, a23, b01, b23;
             decays(dtq[q], q, ap_tag, a01, a23);
-            h[q][0] = f2fma(a01, h[q][0], f2mul(f2dup(duq[q]), make_float2(Bq.x, Bq.y)));
-            h[q][1] = f2fma(a23, h[q][1], f2mul(f2dup(duq[q]), make_float2(Bq.z, Bq.w)));
+            input_term(dtq[q], uq[q], duq[q], q, a01, a23, Bq, b01, b23);
+            h[q][0] = f2fma(a01, h[q][0], b01);
+            h[q][1] = f2fma(a23, h[q][1], b23);
             hist[t][q][0] = h[q][0];
             hist[t][q][1] = h[q][1];
             float2 yv = f2mul(make_float2(Cq.x, Cq.y), h[q][0]);
@@ -309,20 +353,28 @@ __global__ void __launch_bounds__(kBwdFastThreads) ssm_bwd_fast_kernel(const Bwd
           const float2 ds2 = f2dup(dsq[q]), du2 = f2dup(duq[q]);
           const float2 lam01 = f2fma(make_float2(Cq.x, Cq.y), ds2, mu[q][0]);
           const float2 lam23 = f2fma(make_float2(Cq.z, Cq.w), ds2, mu[q][1]);
+          // with ZOH the input weight of a state is E x instead of delta x: lE = lam E takes the place of lam below
+          float2 E01, E23, lw01 = lam01, lw23 = lam23, xw2 = du2;
+          if (ZOH) {
+            gain(dtq[q], q, a01, a23, E01, E23);
+            lw01 = f2mul(lam01, E01);
+            lw23 = f2mul(lam23, E23);
+            xw2 = f2dup(uq[q]);
+          }
           if (q == 0) {
             dC01 = f2mul(ds2, hist[t][q][0]);
             dC23 = f2mul(ds2, hist[t][q][1]);
-            dB01 = f2mul(lam01, du2);
-            dB23 = f2mul(lam23, du2);
+            dB01 = f2mul(lw01, xw2);
+            dB23 = f2mul(lw23, xw2);
           } else {
             dC01 = f2fma(ds2, hist[t][q][0], dC01);
             dC23 = f2fma(ds2, hist[t][q][1], dC23);
-            dB01 = f2fma(lam01, du2, dB01);
-            dB23 = f2fma(lam23, du2, dB23);
+            dB01 = f2fma(lw01, xw2, dB01);
+            dB23 = f2fma(lw23, xw2, dB23);
           }
-          float2 lb = f2mul(lam01, make_float2(Bq.x, Bq.y));
-          lb = f2fma(lam23, make_float2(Bq.z, Bq.w), lb);
-          const float lamB = lb.x + lb.y;
+          float2 lb = f2mul(lw01, make_float2(Bq.x, Bq.y));
+          lb = f2fma(lw23, make_float2(Bq.z, Bq.w), lb);
+          const float lamB = lb.x + lb.y;   // sum lam B (default rule), sum lam E B (ZOH)
           mu[q][0] = f2mul(a01, lam01);
           mu[q][1] = f2mul(a23, lam23);
           float2 hp0, hp1;   // h_{t-1}: the step before in registers, or the sub-block's start state (read again)
@@ -339,8 +391,21 @@ __global__ void __launch_bounds__(kBwdFastThreads) ssm_bwd_fast_kernel(const Bwd
           wa = f2fma(w23, A2[q][1], wa);
           dA2[q][0] = f2fma(w01, f2dup(dtq[q]), dA2[q][0]);
           dA2[q][1] = f2fma(w23, f2dup(dtq[q]), dA2[q][1]);
-          dxp[q] = dtq[q] * lamB;
-          ddp[q] = fmaf(uq[q], lamB, (wa.x + wa.y) * kInvLog2e);
+          if (ZOH) {
+            // dE/ddelta = a: the step-size gradient through E is x sum mu B; dE/dA adds lam (dE/dA) B x to dA
+            float2 mb = f2mul(mu[q][0], make_float2(Bq.x, Bq.y));
+            mb = f2fma(mu[q][1], make_float2(Bq.z, Bq.w), mb);
+            float2 G01, G23;
+            gain_dA(dtq[q], q, a01, a23, E01, E23, G01, G23);
+            const float2 uu = f2dup(uq[q]);
+            dA2[q][0] = f2fma(f2mul(lam01, G01), f2mul(make_float2(Bq.x, Bq.y), uu), dA2[q][0]);
+            dA2[q][1] = f2fma(f2mul(lam23, G23), f2mul(make_float2(Bq.z, Bq.w), uu), dA2[q][1]);
+            dxp[q] = lamB;
+            ddp[q] = fmaf(uq[q], mb.x + mb.y, (wa.x + wa.y) * kInvLog2e);
+          } else {
+            dxp[q] = dtq[q] * lamB;
+            ddp[q] = fmaf(uq[q], lamB, (wa.x + wa.y) * kInvLog2e);
+          }
         }
         sm.red[warp][t % kRB][quad][j][0] = make_float4(dB01.x, dB01.y, dB23.x, dB23.y);
         sm.red[warp][t % kRB][quad][j][1] = make_float4(dC01.x, dC01.y, dC23.x, dC23.y);
@@ -423,6 +488,12 @@ __global__ void __launch_bounds__(kBwdFastThreads) ssm_bwd_fast_kernel(const Bwd
         ap = ap && fabsf(a.z - (a.x + 2.f * step)) <= tol && fabsf(a.w - (a.x + 3.f * step)) <= tol;
         A2[q][0] = make_float2(a.x * kLog2e, a.y * kLog2e);
         A2[q][1] = make_float2(a.z * kLog2e, a.w * kLog2e);
+        if (ZOH) {
+          auto inv = [](float v) { return v != 0.f ? 1.f / v : 0.f; };
+          invA[q][0] = make_float2(inv(a.x), inv(a.y));
+          invA[q][1] = make_float2(inv(a.z), inv(a.w));
+          zeroA = zeroA || a.x == 0.f || a.y == 0.f || a.z == 0.f || a.w == 0.f;
+        }
       }
       Dk = (valid && p.Dskip != nullptr) ? p.Dskip[d0 + pq] : 0.f;
       if (SP) bias_pq = (valid && p.delta_bias != nullptr) ? p.delta_bias[d0 + pq] : 0.f;
@@ -454,6 +525,7 @@ __global__ void __launch_bounds__(kBwdFastThreads) ssm_bwd_fast_kernel(const Bwd
       }
     }
     ap = __all_sync(0xffffffffu, ap);
+    if (ZOH) zeroA = __any_sync(0xffffffffu, zeroA);
     cp_async_wait_all();
     __syncthreads();                       // inputs of this tile landed; sched[1], sched[2] and the dependency are visible
     if (sm.sched[2] != 0) {                // a bounded wait gave up somewhere: every block leaves
@@ -594,7 +666,7 @@ __global__ void __launch_bounds__(kBwdFastThreads) ssm_bwd_fast_kernel(const Bwd
 
 bool bwd_fast_applicable(const ssm_problem_t& prob, const BwdParams& p) {
   auto al16 = [](const void* q) { return q == nullptr || (reinterpret_cast<uintptr_t>(q) & 15) == 0; };
-  if (p.zoh || p.static_B || p.static_C) return false;  // default rule and input-dependent B, C only
+  if (p.static_B || p.static_C) return false;  // input-dependent B, C only
   // work items are numbered with 32-bit integers (one spare bit for the claims that run past the end)
   const long long items = (long long)p.batch * p.nseg * ((p.D + kBwdFastCH - 1) / kBwdFastCH) * (p.seg_steps / kBT);
   if (items > (1LL << 30)) return false;
@@ -607,15 +679,15 @@ bool bwd_fast_applicable(const ssm_problem_t& prob, const BwdParams& p) {
 int bwd_fast_channels_per_block() { return kBwdFastCH; }
 size_t bwd_fast_handoff_bytes_per_chain() { return sizeof(float4) * kHandoffVec * kBwdFastThreads; }
 
-template <bool SP>
+template <bool SP, bool ZOH>
 static cudaError_t launch_bwd_fast_sp(const Plan& plan, const BwdParams& p, cudaStream_t s) {
   constexpr size_t smem = sizeof(BwdFastSmem);
-  cudaError_t e = cudaFuncSetAttribute(ssm_bwd_fast_kernel<SP>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  cudaError_t e = cudaFuncSetAttribute(ssm_bwd_fast_kernel<SP, ZOH>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
   int dev = 0, sms = 0, per_sm = 0;
   if ((e = cudaGetDevice(&dev)) != cudaSuccess) return e;
   if ((e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
-  if ((e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, ssm_bwd_fast_kernel<SP>, kBwdFastThreads, smem)) != cudaSuccess)
+  if ((e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, ssm_bwd_fast_kernel<SP, ZOH>, kBwdFastThreads, smem)) != cudaSuccess)
     return e;
   const int groups = (p.D + kBwdFastCH - 1) / kBwdFastCH;
   const long long chains = (long long)p.batch * plan.nseg * groups;
@@ -623,14 +695,15 @@ static cudaError_t launch_bwd_fast_sp(const Plan& plan, const BwdParams& p, cuda
   const long long resident = (long long)sms * (per_sm > 0 ? per_sm : 1);
   const unsigned grid = (unsigned)(items < resident ? items : resident);
   // the claim counter, the abort word and the flag of every chain were zeroed by the caller (ssm_scan_bwd)
-  ssm_bwd_fast_kernel<SP><<<grid, kBwdFastThreads, smem, s>>>(p);
+  ssm_bwd_fast_kernel<SP, ZOH><<<grid, kBwdFastThreads, smem, s>>>(p);
   return cudaGetLastError();
 }
 
 // SP: the step size is bias + pre-activation, through the softplus if asked (Algorithm 2 step 4)
 cudaError_t launch_bwd_fast(const Plan& plan, const BwdParams& p, cudaStream_t s) {
-  if (p.softplus || p.delta_bias != nullptr) return launch_bwd_fast_sp<true>(plan, p, s);
-  return launch_bwd_fast_sp<false>(plan, p, s);
+  const bool sp = p.softplus || p.delta_bias != nullptr;
+  if (p.zoh) return sp ? launch_bwd_fast_sp<true, true>(plan, p, s) : launch_bwd_fast_sp<false, true>(plan, p, s);
+  return sp ? launch_bwd_fast_sp<true, false>(plan, p, s) : launch_bwd_fast_sp<false, false>(plan, p, s);
 }
 
 }  // namespace ssm

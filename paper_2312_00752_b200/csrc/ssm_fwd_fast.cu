@@ -55,7 +55,7 @@ __device__ __forceinline__ void cp_async_wait_but_one() { asm volatile("cp.async
 
 }  // namespace
 
-template <int WARPS, int MODE, bool SP>
+template <int WARPS, int MODE, bool SP, bool ZOH>
 __global__ void __launch_bounds__((WARPS + 1) * 32) ssm_fwd_fast_kernel(const FwdParams p) {
   constexpr bool FULL = (MODE == kFwdFull);
   constexpr int THREADS = (WARPS + 1) * 32;
@@ -195,6 +195,9 @@ __global__ void __launch_bounds__((WARPS + 1) * 32) ssm_fwd_fast_kernel(const Fw
   // ---- per-thread constants and state
   float2 A2[2][2];   // A * log2(e), states (4j, 4j+1) and (4j+2, 4j+3) of each channel
   float2 h[2][2];
+  // ZOH: B-bar = E B with the input gain E = (a - 1) / A (Eq. 4), and E = delta where A = 0: 1 / A (0 where A = 0)
+  // and the indicator of A = 0
+  float2 invA[ZOH ? 2 : 1][2], zeroA[ZOH ? 2 : 1][2];
   float dsum[2] = {0.f, 0.f};
   bool ap = !p.general_A;
 #pragma unroll
@@ -212,6 +215,14 @@ __global__ void __launch_bounds__((WARPS + 1) * 32) ssm_fwd_fast_kernel(const Fw
     A2[q][1] = make_float2(a.z * kLog2e, a.w * kLog2e);
     h[q][0] = make_float2(hs.x, hs.y);
     h[q][1] = make_float2(hs.z, hs.w);
+    if (ZOH) {
+      auto inv = [](float v) { return v != 0.f ? 1.f / v : 0.f; };
+      auto isz = [](float v) { return v != 0.f ? 0.f : 1.f; };
+      invA[q][0] = make_float2(inv(a.x), inv(a.y));
+      invA[q][1] = make_float2(inv(a.z), inv(a.w));
+      zeroA[q][0] = make_float2(isz(a.x), isz(a.y));
+      zeroA[q][1] = make_float2(isz(a.z), isz(a.w));
+    }
   }
   ap = __all_sync(0xffffffffu, ap);
   // SP: in the step-size stage below a lane always handles channel pair (lane % 8) of its warp
@@ -300,9 +311,17 @@ __global__ void __launch_bounds__((WARPS + 1) * 32) ssm_fwd_fast_kernel(const Fw
             a01[t][q] = make_float2(ex2_approx(e01.x), ex2_approx(e01.y));
             a23[t][q] = make_float2(ex2_approx(e23.x), ex2_approx(e23.y));
           }
-          const float2 dq = make_float2(duq[q], duq[q]);
-          bx01[t][q] = f2mul(dq, make_float2(Bq[t].x, Bq[t].y));
-          bx23[t][q] = f2mul(dq, make_float2(Bq[t].z, Bq[t].w));
+          if (ZOH) {
+            const float2 dd = f2dup(dt[q]), uu = f2dup(u[q]), m1 = f2dup(-1.f), one = f2dup(1.f);
+            const float2 E01 = f2fma(f2fma(a01[t][q], one, m1), invA[q][0], f2mul(zeroA[q][0], dd));
+            const float2 E23 = f2fma(f2fma(a23[t][q], one, m1), invA[q][1], f2mul(zeroA[q][1], dd));
+            bx01[t][q] = f2mul(f2mul(E01, uu), make_float2(Bq[t].x, Bq[t].y));
+            bx23[t][q] = f2mul(f2mul(E23, uu), make_float2(Bq[t].z, Bq[t].w));
+          } else {
+            const float2 dq = make_float2(duq[q], duq[q]);
+            bx01[t][q] = f2mul(dq, make_float2(Bq[t].x, Bq[t].y));
+            bx23[t][q] = f2mul(dq, make_float2(Bq[t].z, Bq[t].w));
+          }
           if (MODE == kFwdSummary) dsum[q] += dt[q];
         }
       }
@@ -368,18 +387,25 @@ __global__ void __launch_bounds__((WARPS + 1) * 32) ssm_fwd_fast_kernel(const Fw
   }
 }
 
-template <int WARPS, int MODE, bool SP>
-static cudaError_t launch_fast_sp(const Plan& plan, const FwdParams& p, cudaStream_t s) {
+template <int WARPS, int MODE, bool SP, bool ZOH>
+static cudaError_t launch_fast_variant(const Plan& plan, const FwdParams& p, cudaStream_t s) {
   constexpr size_t smem = sizeof(FastSmem<WARPS, MODE == kFwdFull, SP>);
   constexpr int CH = 16 * WARPS;
   if (smem > 48 * 1024) {
-    cudaError_t e = cudaFuncSetAttribute(ssm_fwd_fast_kernel<WARPS, MODE, SP>,
+    cudaError_t e = cudaFuncSetAttribute(ssm_fwd_fast_kernel<WARPS, MODE, SP, ZOH>,
                                          cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
   }
   dim3 grid((p.D + CH - 1) / CH, plan.nseg, p.batch);
-  ssm_fwd_fast_kernel<WARPS, MODE, SP><<<grid, (WARPS + 1) * 32, smem, s>>>(p);
+  ssm_fwd_fast_kernel<WARPS, MODE, SP, ZOH><<<grid, (WARPS + 1) * 32, smem, s>>>(p);
   return cudaGetLastError();
+}
+
+// ZOH: the zero-order-hold B-bar of Eq. 4 instead of delta * B
+template <int WARPS, int MODE, bool SP>
+static cudaError_t launch_fast_sp(const Plan& plan, const FwdParams& p, cudaStream_t s) {
+  if (p.zoh) return launch_fast_variant<WARPS, MODE, SP, true>(plan, p, s);
+  return launch_fast_variant<WARPS, MODE, SP, false>(plan, p, s);
 }
 
 // SP: the step size goes through the bias / softplus stage of the service warp
@@ -391,7 +417,7 @@ static cudaError_t launch_fast(const Plan& plan, const FwdParams& p, cudaStream_
 
 bool fwd_fast_applicable(const ssm_problem_t& prob, const FwdParams& p) {
   auto al16 = [](const void* q) { return q == nullptr || (reinterpret_cast<uintptr_t>(q) & 15) == 0; };
-  if (p.zoh || p.static_B || p.static_C) return false;  // default rule and input-dependent B, C only
+  if (p.static_B || p.static_C) return false;  // input-dependent B, C only
   return prob.io_dtype == SSM_BF16 && prob.N == 16 && prob.D % 8 == 0 && al16(p.x) && al16(p.delta) && al16(p.z) &&
          al16(p.B) && al16(p.C) && al16(p.out) && al16(p.A) && al16(p.h_start) && al16(p.ckpt) && al16(p.seg_end) && al16(p.h_last);
 }

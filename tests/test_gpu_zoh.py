@@ -23,6 +23,8 @@ def _case(batch, L, D, N, io, dt=(1e-3, 1e-1), seed=0):
     (2, 97, 33, 4, "f32", (5e-2, 2.0)),        # large steps: the two rules differ by O(1)
     (1, 4200, 32, 16, "f32", (1e-4, 1e-2)),    # time split: segment summaries and both carries under ZOH
     (1, 64, 16, 1, "bf16", (1e-2, 1.0)),
+    (2, 200, 64, 16, "bf16", (5e-2, 2.0)),     # tuned kernels, large steps
+    (1, 4200, 48, 16, "bf16", (1e-4, 1e-2)),   # tuned kernels with a time split
 ])
 def test_zoh_forward_backward(batch, L, D, N, io, dt):
     from oracle import ssm_oracle as O
