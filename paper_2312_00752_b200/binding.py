@@ -225,11 +225,11 @@ def ssm_scan_fwd(x, delta, A, B, C, D_skip=None, z=None, *, save_states=False, g
 
 
 def ssm_scan_fwd_fused_dt(x, delta_pre, delta_bias, A, B, C, D_skip=None, z=None, *, softplus=True, save_states=False,
-                          out=None, saved_states=None, stream=None, h0=None, h_last=None):
+                          out=None, saved_states=None, stream=None, h0=None, h_last=None, zoh=False):
     """Forward with the step-size activation fused: delta = softplus(delta_pre + delta_bias) (or the plain sum with
     softplus=False), in float32.  Otherwise as ssm_scan_fwd."""
     lib = load_library()
-    prob = make_problem(x, B, z is not None, D_skip is not None, save_states, False)
+    prob = make_problem(x, B, z is not None, D_skip is not None, save_states, False, zoh)
     if softplus:
         prob.flags |= SSM_FLAG_DELTA_SOFTPLUS
     batch, L, D, N = prob.batch, prob.L, prob.D, prob.N
@@ -255,11 +255,11 @@ def ssm_scan_fwd_fused_dt(x, delta_pre, delta_bias, A, B, C, D_skip=None, z=None
 
 
 def ssm_scan_bwd_fused_dt(x, delta_pre, delta_bias, A, B, C, D_skip, z, dout, saved_states=None, *, softplus=True,
-                          stream=None):
+                          stream=None, zoh=False):
     """Backward of ssm_scan_fwd_fused_dt.  Returns the dict of ssm_scan_bwd with `ddelta` the gradient of delta_pre
     and an extra `ddelta_bias` (D,) float32."""
     lib = load_library()
-    prob = make_problem(x, B, z is not None, D_skip is not None, False, False)
+    prob = make_problem(x, B, z is not None, D_skip is not None, False, False, zoh)
     if softplus:
         prob.flags |= SSM_FLAG_DELTA_SOFTPLUS
     batch, L, D, N = prob.batch, prob.L, prob.D, prob.N

@@ -50,3 +50,25 @@ def test_fused_step_size_forward_backward(batch, L, D, N, io, softplus):
     g2 = K.ssm_scan_bwd_fused_dt(*args, dev["dout"], None, softplus=softplus)
     for k in ("dx", "ddelta", "ddelta_bias", "dA"):
         assert U.rel_err(U.to_host(g2[k]), ref[k]) <= tol["grad"], k
+
+
+@pytest.mark.parametrize("batch,L,D,N,io", [(2, 130, 40, 16, "bf16"), (1, 100, 24, 8, "f32")])
+def test_fused_step_size_with_the_zoh_rule(batch, L, D, N, io):
+    # both options at once: delta = softplus(v + bias) and B-bar = (exp(delta A) - 1) / A * B
+    import torch
+    from oracle import ssm_oracle as O
+    from paper_2312_00752_b200 import binding as K
+    inp, bias = _pre_activation_case(batch, L, D, N, io)
+    dev = U.to_device(inp, io)
+    dbias = torch.from_numpy(bias).cuda()
+    args = (dev["x"], dev["delta"], dbias, dev["A"], dev["B"], dev["C"], dev["D_skip"], dev["z"])
+    out, saved = K.ssm_scan_fwd_fused_dt(*args, save_states=True, zoh=True)
+    g = K.ssm_scan_bwd_fused_dt(*args, dev["dout"], saved, zoh=True)
+    ref_out = O.scan_fwd(inp["x"], inp["delta"], inp["A"], inp["B"], inp["C"], D_skip=inp["D_skip"], z=inp["z"],
+                         delta_softplus=True, delta_bias=bias, zoh=True)
+    ref = O.scan_bwd(inp["x"], inp["delta"], inp["A"], inp["B"], inp["C"], inp["D_skip"], inp["z"], inp["dout"],
+                     delta_softplus=True, delta_bias=bias, zoh=True)
+    tol = U.TOL[io]
+    assert U.rel_err(U.to_host(out), ref_out) <= tol["out"]
+    for k in ("dx", "ddelta", "ddelta_bias", "dz", "dB", "dC", "dA", "dD"):
+        assert U.rel_err(U.to_host(g[k]), ref[k]) <= tol["grad"], k
