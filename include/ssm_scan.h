@@ -154,6 +154,16 @@ SSM_API ssm_status_t ssm_scan_bwd_fused_dt(const ssm_problem_t* p, const void* x
                                            float* dA, void* dB, void* dC, float* dD, void* dz, void* workspace,
                                            size_t workspace_bytes, void* stream /* cudaStream_t */);
 
+/* ssm_scan_bwd_fused_dt for a piece of a longer sequence: h0, dh_last and dh0 as in ssm_scan_bwd_state. */
+SSM_API ssm_status_t ssm_scan_bwd_fused_dt_state(const ssm_problem_t* p, const void* x, const void* delta_pre,
+                                                 const float* delta_bias, const float* A, const void* B,
+                                                 const void* C, const float* D_skip, const void* z,
+                                                 const void* dout, const float* h0, const float* dh_last,
+                                                 const void* saved_states, void* dx, void* ddelta_pre,
+                                                 float* ddelta_bias, float* dA, void* dB, void* dC, float* dD,
+                                                 void* dz, float* dh0, void* workspace, size_t workspace_bytes,
+                                                 void* stream /* cudaStream_t */);
+
 /*
  * One recurrent step (Eq. 2a/2b evaluated for a single t, the mode used for autoregressive inference): p->L must be
  * 1; x, delta, z, out are [batch][D], B, C are [batch][N] (io_dtype), A [D][N], D_skip [D]; the float32 state

@@ -25,7 +25,7 @@ EXPORTED_SYMBOLS = (
     "ssm_scan_checkpoint_steps", "ssm_scan_fwd", "ssm_scan_bwd", "ssm_status_string", "ssm_scan_plan",
     "ssm_scan_fwd_static", "ssm_scan_check_status", "ssm_scan_fwd_state", "ssm_step",
     "ssm_scan_fwd_fused_dt", "ssm_scan_bwd_fused_dt", "ssm_scan_host_arena_bytes", "ssm_scan_fwd_bwd_host",
-    "ssm_scan_bwd_state", "ssm_conv1d_fwd", "ssm_conv1d_bwd_workspace_bytes", "ssm_conv1d_bwd",
+    "ssm_scan_bwd_state", "ssm_scan_bwd_fused_dt_state", "ssm_conv1d_fwd", "ssm_conv1d_bwd_workspace_bytes", "ssm_conv1d_bwd",
 )
 SSM_STATIC_SCRATCH_BYTES = 4 << 20
 
@@ -88,6 +88,8 @@ def load_library() -> ctypes.CDLL:
     lib.ssm_conv1d_bwd_workspace_bytes.argtypes = [CP]
     lib.ssm_conv1d_bwd.restype = ctypes.c_int
     lib.ssm_conv1d_bwd.argtypes = [CP] + [vp] * 9 + [vp, sz, vp]
+    lib.ssm_scan_bwd_fused_dt_state.restype = ctypes.c_int
+    lib.ssm_scan_bwd_fused_dt_state.argtypes = [P] + [vp] * 21 + [vp, sz, vp]
     lib.ssm_scan_bwd_state.restype = ctypes.c_int
     lib.ssm_scan_bwd_state.argtypes = [P] + [vp] * 19 + [vp, sz, vp]
     lib.ssm_scan_fwd_state.restype = ctypes.c_int
@@ -255,9 +257,9 @@ def ssm_scan_fwd_fused_dt(x, delta_pre, delta_bias, A, B, C, D_skip=None, z=None
 
 
 def ssm_scan_bwd_fused_dt(x, delta_pre, delta_bias, A, B, C, D_skip, z, dout, saved_states=None, *, softplus=True,
-                          stream=None, zoh=False):
+                          stream=None, zoh=False, h0=None, dh_last=None, want_dh0=False):
     """Backward of ssm_scan_fwd_fused_dt.  Returns the dict of ssm_scan_bwd with `ddelta` the gradient of delta_pre
-    and an extra `ddelta_bias` (D,) float32."""
+    and an extra `ddelta_bias` (D,) float32.  h0, dh_last, want_dh0 as in ssm_scan_bwd (ssm_scan_bwd_fused_dt_state)."""
     lib = load_library()
     prob = make_problem(x, B, z is not None, D_skip is not None, False, False, zoh)
     if softplus:
@@ -272,6 +274,23 @@ def ssm_scan_bwd_fused_dt(x, delta_pre, delta_bias, A, B, C, D_skip, z, dout, sa
          "dz": torch.empty_like(x) if z is not None else None}
     stream_ptr = (stream if stream is not None else torch.cuda.current_stream(x.device)).cuda_stream
     ws = _workspace(bwd_workspace_bytes(prob), x.device, stream_ptr)
+    if h0 is not None or dh_last is not None or want_dh0:
+        f32 = torch.float32
+        if want_dh0:
+            o["dh0"] = torch.empty((batch, D, N), dtype=f32, device=x.device)
+        code = lib.ssm_scan_bwd_fused_dt_state(
+            ctypes.byref(prob), _dev_ptr(x, "x", (batch, L, D), io), _dev_ptr(delta_pre, "delta_pre", (batch, L, D), io),
+            _dev_ptr(delta_bias, "delta_bias", (D,), f32), _dev_ptr(A, "A", (D, N), f32),
+            _dev_ptr(B, "B", (batch, L, N), io), _dev_ptr(C, "C", (batch, L, N), io), _dev_ptr(D_skip, "D_skip", (D,), f32),
+            _dev_ptr(z, "z", (batch, L, D), io), _dev_ptr(dout, "dout", (batch, L, D), io),
+            _dev_ptr(h0, "h0", (batch, D, N), f32), _dev_ptr(dh_last, "dh_last", (batch, D, N), f32),
+            _dev_ptr(saved_states, "saved_states"), _dev_ptr(o["dx"], "dx"), _dev_ptr(o["ddelta"], "ddelta"),
+            _dev_ptr(o["ddelta_bias"], "ddelta_bias"), _dev_ptr(o["dA"], "dA"), _dev_ptr(o["dB"], "dB"),
+            _dev_ptr(o["dC"], "dC"), _dev_ptr(o["dD"], "dD"), _dev_ptr(o["dz"], "dz"), _dev_ptr(o.get("dh0"), "dh0"),
+            _dev_ptr(ws, "workspace"), ctypes.c_size_t(0 if ws is None else ws.numel() * ws.element_size()),
+            ctypes.c_void_p(stream_ptr))
+        _check(code, "ssm_scan_bwd_fused_dt_state")
+        return o
     code = lib.ssm_scan_bwd_fused_dt(
         ctypes.byref(prob), _dev_ptr(x, "x", (batch, L, D), io), _dev_ptr(delta_pre, "delta_pre", (batch, L, D), io),
         _dev_ptr(delta_bias, "delta_bias", (D,), torch.float32), _dev_ptr(A, "A", (D, N), torch.float32),

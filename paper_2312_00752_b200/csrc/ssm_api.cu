@@ -494,6 +494,16 @@ ssm_status_t ssm_scan_bwd_state(const ssm_problem_t* p, const void* x, const voi
                   dB, dC, dD, dz, dh0, workspace, workspace_bytes, stream);
 }
 
+ssm_status_t ssm_scan_bwd_fused_dt_state(const ssm_problem_t* p, const void* x, const void* delta_pre,
+                                         const float* delta_bias, const float* A, const void* B, const void* C,
+                                         const float* D_skip, const void* z, const void* dout, const float* h0,
+                                         const float* dh_last, const void* saved_states, void* dx, void* ddelta_pre,
+                                         float* ddelta_bias, float* dA, void* dB, void* dC, float* dD, void* dz,
+                                         float* dh0, void* workspace, size_t workspace_bytes, void* stream) {
+  return bwd_impl(p, x, delta_pre, delta_bias, A, B, C, D_skip, z, dout, h0, dh_last, saved_states, dx, ddelta_pre,
+                  ddelta_bias, dA, dB, dC, dD, dz, dh0, workspace, workspace_bytes, stream);
+}
+
 ssm_status_t ssm_scan_bwd_fused_dt(const ssm_problem_t* p, const void* x, const void* delta_pre,
                                    const float* delta_bias, const float* A, const void* B, const void* C,
                                    const float* D_skip, const void* z, const void* dout, const void* saved_states,

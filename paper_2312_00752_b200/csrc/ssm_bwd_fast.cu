@@ -230,7 +230,8 @@ __global__ void __launch_bounds__(kBwdFastThreads) ssm_bwd_fast_kernel(const Bwd
     return make_float2(bf16sel(dw, selA), bf16sel(dw, selB));
   };
 
-  auto process_tile = [&](int st, auto ap_tag, const float4 (&ck)[2]) {
+  // nlive: rows of the tile inside the segment (the rest were zero-filled and are identity steps)
+  auto process_tile = [&](int st, auto ap_tag, const float4 (&ck)[2], int nlive) {
     // The raw B / C rows of this ring stage were widened by the staging pass and are dead until the stage is refilled
     // two tiles from now: the checkpoint state waits there (one float4 per thread and channel) until the first
     // sub-block needs it again, instead of in registers.
@@ -450,7 +451,8 @@ __global__ void __launch_bounds__(kBwdFastThreads) ssm_bwd_fast_kernel(const Bwd
             const float v = __uint_as_float((uint32_t)reinterpret_cast<const uint16_t*>(&sm.d[st][tt][slot])[pq] << 16) + bias_pq;
             ddv *= sigmoid_fast(v);
           }
-          dbias_acc += ddv;
+          // (a padded row still sees the adjoint that flows through it, so its value is not zero)
+          if (tt < nlive) dbias_acc += ddv;
         }
         reinterpret_cast<__nv_bfloat16*>(&sm.d[st][tt][slot])[pq] = __float2bfloat16_rn(ddv);
       }
@@ -594,8 +596,8 @@ __global__ void __launch_bounds__(kBwdFastThreads) ssm_bwd_fast_kernel(const Bwd
         *reinterpret_cast<float2*>(&sm.gsp[tt][2 * w]) = gpv;
       }
       __syncthreads();
-      if (ap) process_tile(st, std::true_type{}, ck);
-      else process_tile(st, std::false_type{}, ck);
+      if (ap) process_tile(st, std::true_type{}, ck, cur.t_end - cur.t0);
+      else process_tile(st, std::false_type{}, ck, cur.t_end - cur.t0);
       __syncthreads();
       // results of the tile: 16-byte stores of dx, ddelta, dz; block partial sums of dB, dC
       for (int c = tid; c < kBT * CHUNKS; c += THREADS) {

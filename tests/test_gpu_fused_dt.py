@@ -72,3 +72,30 @@ def test_fused_step_size_with_the_zoh_rule(batch, L, D, N, io):
     assert U.rel_err(U.to_host(out), ref_out) <= tol["out"]
     for k in ("dx", "ddelta", "ddelta_bias", "dz", "dB", "dC", "dA", "dD"):
         assert U.rel_err(U.to_host(g[k]), ref[k]) <= tol["grad"], k
+
+
+def test_fused_step_size_backward_in_two_pieces():
+    # the chunked use (carried state, adjoint handed back across the cut) together with the fused step size
+    import torch
+    from oracle import ssm_oracle as O
+    from paper_2312_00752_b200 import binding as K
+    batch, L, D, N, io, cut = 2, 300, 40, 16, "bf16", 130
+    inp, bias = _pre_activation_case(batch, L, D, N, io)
+    dev = U.to_device(inp, io)
+    dbias = torch.from_numpy(bias).cuda()
+    ref = O.scan_bwd(inp["x"], inp["delta"], inp["A"], inp["B"], inp["C"], inp["D_skip"], inp["z"], inp["dout"],
+                     delta_softplus=True, delta_bias=bias)
+    sl = lambda k, a, b: dev[k][:, a:b].contiguous()
+    piece = lambda a, b: (sl("x", a, b), sl("delta", a, b), dbias, dev["A"], sl("B", a, b), sl("C", a, b), dev["D_skip"],
+                          sl("z", a, b))
+    h_mid = torch.empty((batch, D, N), dtype=torch.float32, device="cuda")
+    _, sv1 = K.ssm_scan_fwd_fused_dt(*piece(0, cut), save_states=True, h_last=h_mid)
+    _, sv2 = K.ssm_scan_fwd_fused_dt(*piece(cut, L), save_states=True, h0=h_mid)
+    g2 = K.ssm_scan_bwd_fused_dt(*piece(cut, L), sl("dout", cut, L), sv2, h0=h_mid, want_dh0=True)
+    g1 = K.ssm_scan_bwd_fused_dt(*piece(0, cut), sl("dout", 0, cut), sv1, dh_last=g2["dh0"])
+    tol = U.TOL[io]["grad"]
+    for k in ("dx", "ddelta", "dz", "dB", "dC"):
+        got = np.concatenate([U.to_host(g1[k]), U.to_host(g2[k])], axis=1)
+        assert U.rel_err(got, ref[k]) <= tol, k
+    for k in ("dA", "dD", "ddelta_bias"):
+        assert U.rel_err(U.to_host(g1[k]) + U.to_host(g2[k]), ref[k]) <= tol, k
