@@ -72,3 +72,21 @@ def test_host_call_twice_on_one_arena_and_argument_errors():
     with pytest.raises(K.SsmScanError):
         K.ssm_scan_fwd_bwd_host(h1["x"].cuda(), h1["delta"], h1["A"], h1["B"], h1["C"], h1["D_skip"], h1["z"],
                                 h1["dout"], device="cuda:0")
+
+
+def test_host_call_honours_the_zoh_flag():
+    import torch
+    from paper_2312_00752_b200 import binding as K
+    cfg = synth.ScanConfig("host", 15, 3, 100, 32, 16, "bf16", 5e-2, 1.0)
+    inp = synth.make_inputs(cfg, seed=4)
+    h = _host_tensors(inp, "bf16")
+    res = K.ssm_scan_fwd_bwd_host(h["x"], h["delta"], h["A"], h["B"], h["C"], h["D_skip"], h["z"], h["dout"],
+                                  device="cuda:0", zoh=True)
+    torch.cuda.synchronize()
+    dev = U.to_device(inp, "bf16")
+    args = (dev["x"], dev["delta"], dev["A"], dev["B"], dev["C"], dev["D_skip"], dev["z"])
+    out, saved = K.ssm_scan_fwd(*args, save_states=True, zoh=True)
+    g = K.ssm_scan_bwd(*args, dev["dout"], saved, zoh=True)
+    assert torch.equal(res["out"], out.cpu()) and torch.equal(res["dx"], g["dx"].cpu())
+    plain = K.ssm_scan_fwd(*args)
+    assert not torch.equal(out, plain)

@@ -90,3 +90,28 @@ def test_zoh_step_by_step_equals_scan(batch, D, N, io):
     got = np.stack([U.to_host(o) for o in outs], axis=1)
     assert U.rel_err(got, ref_out) <= U.TOL[io]["out"]
     assert U.rel_err(U.to_host(h), ref_h) <= 1e-5
+
+
+@pytest.mark.parametrize("batch,L,D,N,io,cut", [(2, 300, 40, 16, "bf16", 130), (1, 150, 24, 8, "f32", 70)])
+def test_zoh_backward_in_two_pieces(batch, L, D, N, io, cut):
+    # carried state and adjoint across a cut under the ZOH rule (ragged last tiles with an adjoint flowing through)
+    import torch
+    from oracle import ssm_oracle as O
+    from paper_2312_00752_b200 import binding as K
+    inp = _case(batch, L, D, N, io, (5e-3, 0.5))
+    dev = U.to_device(inp, io)
+    ref = O.scan_bwd(inp["x"], inp["delta"], inp["A"], inp["B"], inp["C"], inp["D_skip"], inp["z"], inp["dout"], zoh=True)
+    sl = lambda k, a, b: dev[k][:, a:b].contiguous()
+    piece = lambda a, b: (sl("x", a, b), sl("delta", a, b), dev["A"], sl("B", a, b), sl("C", a, b), dev["D_skip"],
+                          sl("z", a, b))
+    h_mid = torch.empty((batch, D, N), dtype=torch.float32, device="cuda")
+    _, sv1 = K.ssm_scan_fwd(*piece(0, cut), save_states=True, h_last=h_mid, zoh=True)
+    _, sv2 = K.ssm_scan_fwd(*piece(cut, L), save_states=True, h0=h_mid, zoh=True)
+    g2 = K.ssm_scan_bwd(*piece(cut, L), sl("dout", cut, L), sv2, h0=h_mid, want_dh0=True, zoh=True)
+    g1 = K.ssm_scan_bwd(*piece(0, cut), sl("dout", 0, cut), sv1, dh_last=g2["dh0"], want_dh0=True, zoh=True)
+    tol = U.TOL[io]["grad"]
+    for k in ("dx", "ddelta", "dz", "dB", "dC"):
+        assert U.rel_err(np.concatenate([U.to_host(g1[k]), U.to_host(g2[k])], axis=1), ref[k]) <= tol, k
+    for k in ("dA", "dD"):
+        assert U.rel_err(U.to_host(g1[k]) + U.to_host(g2[k]), ref[k]) <= tol, k
+    assert U.rel_err(U.to_host(g1["dh0"]), ref["dh0"]) <= (1e-4 if io == "f32" else 3e-2)
