@@ -74,12 +74,12 @@ def test_fused_step_size_with_the_zoh_rule(batch, L, D, N, io):
         assert U.rel_err(U.to_host(g[k]), ref[k]) <= tol["grad"], k
 
 
-def test_fused_step_size_backward_in_two_pieces():
+@pytest.mark.parametrize("batch,L,D,N,io,cut", [(2, 300, 40, 16, "bf16", 130), (1, 6000, 64, 16, "bf16", 2048)])
+def test_fused_step_size_backward_in_two_pieces(batch, L, D, N, io, cut):
     # the chunked use (carried state, adjoint handed back across the cut) together with the fused step size
     import torch
     from oracle import ssm_oracle as O
     from paper_2312_00752_b200 import binding as K
-    batch, L, D, N, io, cut = 2, 300, 40, 16, "bf16", 130
     inp, bias = _pre_activation_case(batch, L, D, N, io)
     dev = U.to_device(inp, io)
     dbias = torch.from_numpy(bias).cuda()
