@@ -77,3 +77,39 @@ def test_conv1d_layer_shape_sampled_and_deterministic():
     assert U.rel_err(U.to_host(r1["dx"][:, :, ch]), ref["dx"]) <= 3e-2
     assert U.rel_err(U.to_host(r1["dw"][ch]), ref["dw"]) <= 3e-2
     assert U.rel_err(U.to_host(r1["dbias"][ch]), ref["dbias"]) <= 3e-2
+
+
+def _draw_conv(rng):
+    return dict(io=str(rng.choice(["bf16", "f32"])), W=int(rng.integers(1, 5)), D=int(rng.choice([4, 8, 20, 64, 260, 7, 33])),
+                L=int(rng.choice([1, 2, 3, 5, 31, 32, 33, 64, 127, 129, 300])), batch=int(rng.integers(1, 4)),
+                silu=bool(rng.integers(0, 2)), bias=bool(rng.integers(0, 2)), prev=bool(rng.integers(0, 2)))
+
+
+CONV_CASES = [_draw_conv(np.random.default_rng([2312, 754, i])) for i in range(48)]
+
+
+@pytest.mark.parametrize("c", CONV_CASES, ids=[f"{i}" for i in range(len(CONV_CASES))])
+def test_conv1d_random_problem(c):
+    import torch
+    from oracle import conv_oracle as CO
+    from paper_2312_00752_b200 import binding as K
+    x, w, b, dy, xp = _case(c["batch"], c["L"], c["D"], c["W"], c["io"], seed=3, prev=c["prev"])
+    if not c["bias"]:
+        b = None
+    dt = torch.bfloat16 if c["io"] == "bf16" else torch.float32
+    tx, tdy = torch.from_numpy(x).cuda().to(dt), torch.from_numpy(dy).cuda().to(dt)
+    txp = None if xp is None else torch.from_numpy(xp).cuda().to(dt)
+    tw = torch.from_numpy(w).cuda()
+    tb = None if b is None else torch.from_numpy(b).cuda()
+    y = K.ssm_conv1d_fwd(tx, tw, tb, silu=c["silu"], x_prev=txp)
+    g = K.ssm_conv1d_bwd(tx, tw, tb, tdy, silu=c["silu"], x_prev=txp, want_dx_prev=True)
+    ref_y = CO.conv1d_fwd(x, w, b, silu=c["silu"], x_prev=xp)
+    ref = CO.conv1d_bwd(x, w, b, dy, silu=c["silu"], x_prev=xp)
+    tol = U.TOL[c["io"]]
+    assert U.rel_err(U.to_host(y), ref_y) <= tol["out"], c
+    assert U.rel_err(U.to_host(g["dx"]), ref["dx"]) <= tol["grad"], c
+    assert U.rel_err(U.to_host(g["dw"]), ref["dw"]) <= tol["grad"], c
+    if b is not None:
+        assert U.rel_err(U.to_host(g["dbias"]), ref["dbias"]) <= tol["grad"], c
+    if c["W"] > 1 and xp is not None:
+        assert U.rel_err(U.to_host(g["dx_prev"]), ref["dx_prev"]) <= tol["grad"], c
