@@ -29,7 +29,7 @@ METRIC = "selective-scan fwd+bwd elements/s (elements = batch*L*D); achieved HBM
 FALLBACK_HBM_GBS = 6650.0
 # DRAM bytes (read + write) of one launch of the dominant kernel from an ncu capture at the bench workload itself
 # (profiles/ssm_bwd_fast_kernel_mamba2p8b_layer.md); None where no capture exists.
-NCU_TRAFFIC_BYTES = {3: 420.4e6 + 380.7e6}
+NCU_TRAFFIC_BYTES = {3: 420.4e6 + 383.9e6}
 
 
 def parse_args():
