@@ -162,6 +162,10 @@ def _workspace(nbytes: int, device, stream_ptr: int) -> torch.Tensor | None:
     key = (str(device), int(stream_ptr))
     ws = _workspaces.get(key)
     if ws is None or ws.numel() < nbytes:
+        if ws is not None:
+            # kernels already enqueued on that stream may still use the old buffer: the caching allocator must not hand
+            # its memory to other work before they are done
+            ws.record_stream(torch.cuda.ExternalStream(int(stream_ptr), device=device))
         ws = torch.empty(nbytes, dtype=torch.uint8, device=device)
         _workspaces[key] = ws
     return ws

@@ -8,7 +8,21 @@ namespace ssm {
 
 int fwd_channels_per_block(int N);
 int bwd_channels_per_block(int N);
-size_t bwd_fast_handoff_bytes_per_chain();
+int fwd_states_per_thread();
+size_t fwd_handoff_bytes_per_worker();
+size_t bwd_handoff_bytes_per_worker();
+
+// Shapes the tuned warp-per-worker kernels take (they also want 16-byte aligned pointers, checked per call).
+static bool tuned_shape(const ssm_problem_t& p) {
+  return p.io_dtype == SSM_BF16 && p.N == 16 && p.D % 8 == 0 && !(p.flags & (SSM_FLAG_STATIC_B | SSM_FLAG_STATIC_C));
+}
+// Workers the hand-off slots of a workspace allow for `chains` chains of 32 channels: none while every chain can have
+// a warp of its own in the first round (one warp per SM sub-partition), else up to 8 resident warps per SM.
+constexpr int kMaxWarpsPerSM = 8;
+static int shared_workers(long long chains) {
+  if (chains <= 4LL * kNumSMs) return 0;
+  return (int)std::min<long long>(chains, (long long)kMaxWarpsPerSM * kNumSMs);
+}
 
 static inline size_t align_up(size_t v) { return (v + 255) & ~(size_t)255; }
 
@@ -38,13 +52,22 @@ Plan make_plan(const ssm_problem_t& p) {
   const long long warps = std::max<long long>(1, groups * (p.N / S) / 32);
   const long long sub_partitions = 4LL * kNumSMs;
   int nseg = 1;
-  if (warps < sub_partitions * 3 / 4) {
+  if (tuned_shape(p)) {
+    // one warp per 32 channels; a split doubles the forward arithmetic, so only when fewer than half of the
+    // sub-partitions would have a warp, and then into two rounds of chains
+    const long long chains = (long long)p.batch * ((p.D + 31) / 32);
+    if (2 * chains < sub_partitions) {
+      const long long want = (2 * sub_partitions + chains - 1) / chains;
+      const long long max_by_len = std::max(1, p.L / 256);
+      nseg = (int)std::min<long long>(std::min(want, max_by_len), 65535);
+    }
+  } else if (warps < sub_partitions * 3 / 4) {
     const long long want = (6 * sub_partitions + warps - 1) / warps;
     const long long max_by_len = std::max(1, p.L / 256);
     nseg = (int)std::min<long long>(std::min(want, max_by_len), 65535);
   }
   int seg_steps = (p.L + nseg - 1) / nseg;
-  seg_steps = (seg_steps + kCkptSteps - 1) / kCkptSteps * kCkptSteps;
+  seg_steps = (seg_steps + kSegAlign - 1) / kSegAlign * kSegAlign;
   pl.seg_steps = seg_steps;
   pl.nseg = (p.L + seg_steps - 1) / seg_steps;
   return pl;
@@ -61,40 +84,70 @@ Plan make_bwd_plan(const ssm_problem_t& p) {
   const long long chains = (long long)p.batch * pl.bwd_groups;
   const long long resident = 4LL * kNumSMs;
   int nseg = 1;
-  if (chains * 10 < resident * 9) {
-    const long long want = (3 * resident + chains - 1) / chains;
+  if (tuned_shape(p) ? chains < 2 * resident : chains * 4 < resident * 3) {
+    // the tuned kernel wants two warps per SM sub-partition (a lone warp cannot cover its own latencies), i.e. two
+    // rounds of chains; the adjoint pre-pass that a split costs is about a tenth of the backward work
+    const long long want = (2 * resident + chains - 1) / chains;
     const long long max_by_len = std::max(1, p.L / 256);
     nseg = (int)std::min<long long>(std::min(want, max_by_len), 65535);
   }
   int seg_steps = (p.L + nseg - 1) / nseg;
-  seg_steps = (seg_steps + kCkptSteps - 1) / kCkptSteps * kCkptSteps;
+  seg_steps = (seg_steps + kSegAlign - 1) / kSegAlign * kSegAlign;
   pl.seg_steps = seg_steps;
   pl.nseg = (p.L + seg_steps - 1) / seg_steps;
   return pl;
 }
 
+// Every non-empty workspace starts with a status block whose first word is the one ssm_scan_check_status reads.
+constexpr size_t kStatusBytes = 256;
+
 struct FwdWorkspace {
-  size_t seg_end, seg_dsum, h_start, total;
+  size_t seg_end, seg_dsum, h_start, flags, handoff, total;
+  int max_workers;
 };
 static FwdWorkspace fwd_layout(const ssm_problem_t& p, const Plan& pl) {
   FwdWorkspace w{};
+  w.max_workers = tuned_shape(p) ? shared_workers((long long)p.batch * pl.nseg * ((p.D + 31) / 32)) : 0;
+  if (pl.nseg == 1 && w.max_workers == 0) return w;
+  size_t off = kStatusBytes;
+  auto take = [&](size_t bytes) {
+    const size_t at = off;
+    off += align_up(bytes);
+    return at;
+  };
   if (pl.nseg > 1) {
     const size_t st = (size_t)p.batch * pl.nseg * p.D * p.N * sizeof(float);
-    w.seg_end = 0;
-    w.h_start = align_up(st);
-    w.seg_dsum = w.h_start + align_up(st);
-    w.total = w.seg_dsum + align_up((size_t)p.batch * pl.nseg * p.D * sizeof(float));
+    w.seg_end = take(st);
+    w.h_start = take(st);
+    w.seg_dsum = take((size_t)p.batch * pl.nseg * p.D * sizeof(float));
   }
+  if (w.max_workers > 0) {
+    w.flags = take((size_t)(w.max_workers + 1) * sizeof(int));
+    w.handoff = take((size_t)(w.max_workers + 1) * fwd_handoff_bytes_per_worker());
+  }
+  w.total = off;
   return w;
+}
+// Points the forward parameters at the scheduling words of a forward workspace and clears them.
+static cudaError_t attach_fwd_sched(const ssm_problem_t& p, const Plan& pl, char* ws, int* abort_word, FwdParams& fp,
+                                    cudaStream_t s) {
+  const FwdWorkspace w = fwd_layout(p, pl);
+  fp.abort = abort_word;
+  fp.max_workers = w.max_workers;
+  if (w.max_workers == 0) return cudaSuccess;
+  fp.flags = reinterpret_cast<int*>(ws + w.flags);
+  fp.handoff = reinterpret_cast<float4*>(ws + w.handoff);
+  return cudaMemsetAsync(ws + w.flags, 0, (size_t)(w.max_workers + 1) * sizeof(int), s);
 }
 
 struct BwdWorkspace {
-  size_t dBC_part, dA_part, dD_part, dbias_part, ckpt, seg_local, seg_dsum, mu_in, fwd, sched, handoff, total;
+  size_t dBC_part, dA_part, dD_part, dbias_part, ckpt, seg_local, seg_dsum, mu_in, fwd, flags, handoff, total;
   size_t dBs_part, dCs_part;   // static B / C
+  int max_workers;
 };
 static BwdWorkspace bwd_layout(const ssm_problem_t& p, const Plan& pl, const Plan& pl_fwd) {
   BwdWorkspace w{};
-  size_t off = 0;
+  size_t off = kStatusBytes;
   auto take = [&](size_t bytes) {
     const size_t at = off;
     off += align_up(bytes);
@@ -114,9 +167,12 @@ static BwdWorkspace bwd_layout(const ssm_problem_t& p, const Plan& pl, const Pla
     w.seg_dsum = take(parts * p.D * sizeof(float));
   }
   w.fwd = take(fwd_layout(p, pl_fwd).total);   // the forward sweep that rebuilds checkpoints uses the forward split
-  const size_t chains = parts * pl.bwd_groups;   // (batch, segment, channel group) chains of the tuned kernel
-  w.sched = take((64 + chains) * sizeof(int));
-  w.handoff = take(chains * bwd_fast_handoff_bytes_per_chain());
+  // (batch, segment, channel group) chains of the tuned kernel; SSM_FLAG_TEST_WITHHOLD forces chains to be shared
+  const long long chains = (long long)parts * pl.bwd_groups;
+  w.max_workers = !tuned_shape(p) ? 0 : (p.flags & SSM_FLAG_TEST_WITHHOLD) ? (int)std::max<long long>(1, (2 * chains + 2) / 3)
+                                                                            : shared_workers(chains);
+  w.flags = take((size_t)(w.max_workers + 1) * sizeof(int));
+  w.handoff = take((size_t)(w.max_workers + 1) * bwd_handoff_bytes_per_worker());
   if (p.flags & SSM_FLAG_STATIC_B) w.dBs_part = take(parts * p.D * p.N * sizeof(float));
   if (p.flags & SSM_FLAG_STATIC_C) w.dCs_part = take(parts * p.D * p.N * sizeof(float));
   w.total = off;
@@ -206,11 +262,9 @@ ssm_status_t ssm_scan_check_status(const ssm_problem_t* p, const void* workspace
   const ssm_status_t st = validate_problem(p);
   if (st != SSM_OK) return st;
   if (workspace == nullptr) return SSM_ERR_WORKSPACE;
-  const BwdWorkspace w = bwd_layout(*p, make_bwd_plan(*p), make_plan(*p));
   int word = 0;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
-  if (cudaMemcpyAsync(&word, static_cast<const char*>(workspace) + w.sched + sizeof(int), sizeof(int),
-                      cudaMemcpyDeviceToHost, s) != cudaSuccess)
+  if (cudaMemcpyAsync(&word, workspace, sizeof(int), cudaMemcpyDeviceToHost, s) != cudaSuccess)
     return SSM_ERR_CUDA;
   if (cudaStreamSynchronize(s) != cudaSuccess) return SSM_ERR_CUDA;
   return word != 0 ? SSM_ERR_TIMEOUT : SSM_OK;
@@ -224,7 +278,7 @@ ssm_status_t ssm_scan_plan(const ssm_problem_t* p, int32_t* n_segments, int32_t*
   if (n_segments) *n_segments = pl.nseg;
   if (segment_steps) *segment_steps = pl.seg_steps;
   if (channels_per_block) *channels_per_block = pl.fwd_ch;
-  if (states_per_thread) *states_per_thread = p->N < 4 ? p->N : 4;
+  if (states_per_thread) *states_per_thread = tuned_shape(*p) ? fwd_states_per_thread() : (p->N < 4 ? p->N : 4);
   return SSM_OK;
 }
 
@@ -271,8 +325,18 @@ static ssm_status_t fwd_impl(const ssm_problem_t* p, const void* x, const void* 
   fp.static_C = (p->flags & SSM_FLAG_STATIC_C) ? 1 : 0;
   fp.delta_bias = delta_bias;
   fp.softplus = (p->flags & SSM_FLAG_DELTA_SOFTPLUS) ? 1 : 0;
+  if (fwd_layout(*p, pl).total > 0) {
+    if (cudaMemsetAsync(workspace, 0, kStatusBytes, s) != cudaSuccess) return SSM_ERR_CUDA;
+    if (attach_fwd_sched(*p, pl, static_cast<char*>(workspace), static_cast<int*>(workspace), fp, s) != cudaSuccess)
+      return SSM_ERR_CUDA;
+  }
   const float* h_start = nullptr;
   if (run_segment_starts(*p, pl, fp, static_cast<char*>(workspace), h0, &h_start, s) != cudaSuccess) return SSM_ERR_CUDA;
+  if (fp.max_workers > 0 && pl.nseg > 1) {
+    // the summary pass used the hand-off flags: clear them again for the full pass
+    if (attach_fwd_sched(*p, pl, static_cast<char*>(workspace), static_cast<int*>(workspace), fp, s) != cudaSuccess)
+      return SSM_ERR_CUDA;
+  }
   fp.h_start = h_start;
   fp.h_last = h_last;
   fp.ckpt = save ? static_cast<float*>(saved_states) : nullptr;
@@ -364,6 +428,7 @@ static ssm_status_t bwd_impl(const ssm_problem_t* p, const void* x, const void* 
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   char* ws = static_cast<char*>(workspace);
 
+  if (cudaMemsetAsync(ws, 0, kStatusBytes, s) != cudaSuccess) return SSM_ERR_CUDA;
   // checkpoint states: the caller's, or rebuilt here with one more forward sweep
   const float* ckpt = static_cast<const float*>(saved_states);
   if (ckpt == nullptr) {
@@ -385,8 +450,12 @@ static ssm_status_t bwd_impl(const ssm_problem_t* p, const void* x, const void* 
     fp.static_C = (p->flags & SSM_FLAG_STATIC_C) ? 1 : 0;
     fp.delta_bias = delta_bias;
     fp.softplus = (p->flags & SSM_FLAG_DELTA_SOFTPLUS) ? 1 : 0;
+    if (attach_fwd_sched(*p, pl_fwd, ws + w.fwd, reinterpret_cast<int*>(ws), fp, s) != cudaSuccess) return SSM_ERR_CUDA;
     const float* h_start = nullptr;
     if (run_segment_starts(*p, pl_fwd, fp, ws + w.fwd, h0, &h_start, s) != cudaSuccess) return SSM_ERR_CUDA;
+    if (fp.max_workers > 0 && pl_fwd.nseg > 1 &&
+        attach_fwd_sched(*p, pl_fwd, ws + w.fwd, reinterpret_cast<int*>(ws), fp, s) != cudaSuccess)
+      return SSM_ERR_CUDA;
     fp.h_start = h_start;
     fp.ckpt = reinterpret_cast<float*>(ws + w.ckpt);
     if (launch_fwd(*p, pl_fwd, fp, kFwdCkptOnly, s) != cudaSuccess) return SSM_ERR_CUDA;
@@ -428,11 +497,12 @@ static ssm_status_t bwd_impl(const ssm_problem_t* p, const void* x, const void* 
   bp.dh0 = dh0;
   bp.mu_in = dh_last;  // one segment: [batch][1][D][N] is the layout of the caller's adjoint
   bp.dbias_part = ddelta_bias != nullptr ? reinterpret_cast<float*>(ws + w.dbias_part) : nullptr;
-  bp.sched = reinterpret_cast<int*>(ws + w.sched);
+  bp.abort = reinterpret_cast<int*>(ws);
+  bp.flags = reinterpret_cast<int*>(ws + w.flags);
   bp.handoff = reinterpret_cast<float4*>(ws + w.handoff);
-  // scheduling words of the tuned kernel (claim counter, abort word, one progress flag per chain) start at zero; the
-  // abort word is also what ssm_scan_check_status reads, whichever kernel runs
-  if (cudaMemsetAsync(ws + w.sched, 0, w.handoff - w.sched, s) != cudaSuccess) return SSM_ERR_CUDA;
+  bp.max_workers = w.max_workers;
+  // the hand-off flags of the tuned kernel start at zero (the status word was cleared above)
+  if (cudaMemsetAsync(ws + w.flags, 0, w.handoff - w.flags, s) != cudaSuccess) return SSM_ERR_CUDA;
 
   if (pl.nseg > 1) {
     bp.seg_local = reinterpret_cast<float*>(ws + w.seg_local);

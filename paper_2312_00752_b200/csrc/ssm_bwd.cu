@@ -7,9 +7,9 @@
 //     dC_t  += ds_t h_t,  dB_t += lam_t delta_t x_t                        (summed over channels)
 //     dx_t   = ds_t D_skip + delta_t sum_n lam_t B_t
 //     w_t    = mu_t h_{t-1};  ddelta_t = sum_n w_t A + x_t sum_n lam_t B_t;  dA += w_t delta_t;  dD += ds_t x_t
-// A block walks its time segment backwards one checkpoint block (kCkptSteps steps) at a time: it reloads the inputs
-// of the block, recomputes h_t forward from the checkpoint state into shared memory, then runs the reverse
-// recurrence over the block.  Thread layout as in the forward kernel with one channel per thread group.
+// A block walks its time segment backwards one tile (kBwdTile steps, a whole number of checkpoint blocks) at a time: it
+// reloads the inputs of the tile, recomputes h_t forward from the tile's first checkpoint state into shared memory,
+// then runs the reverse recurrence over the tile.  Thread layout as in the forward kernel with one channel per thread group.
 //
 // Reductions are deterministic: dB/dC are summed over the channels of a warp with a fixed xor-shuffle tree, over the
 // warps of the block in ascending order, written as per-block partial sums and finally summed over blocks in
@@ -18,6 +18,9 @@
 #include "ssm_common.cuh"
 
 namespace ssm {
+
+constexpr int kBwdTile = 32;
+static_assert(kBwdTile % kCkptSteps == 0, "a tile starts on a checkpoint");
 
 template <int N>
 struct BwdGeom {
@@ -31,17 +34,17 @@ struct BwdGeom {
 template <typename IO, int N>
 constexpr size_t bwd_smem_bytes() {
   using G = BwdGeom<N>;
-  return sizeof(float) * ((size_t)(kCkptSteps + 1) * G::CH * N   // h_0 .. h_T
-                          + 2 * (size_t)kCkptSteps * N           // B, C
-                          + (size_t)kCkptSteps * G::CH           // s (pre-gate readout)
-                          + (size_t)G::WARPS * kCkptSteps * 2 * N)  // per-warp dB/dC sums
-         + sizeof(IO) * 4 * (size_t)kCkptSteps * G::CH;          // x, delta, z, dout (reused for dx, ddelta, dz)
+  return sizeof(float) * ((size_t)(kBwdTile + 1) * G::CH * N   // h_0 .. h_T
+                          + 2 * (size_t)kBwdTile * N           // B, C
+                          + (size_t)kBwdTile * G::CH           // s (pre-gate readout)
+                          + (size_t)G::WARPS * kBwdTile * 2 * N)  // per-warp dB/dC sums
+         + sizeof(IO) * 4 * (size_t)kBwdTile * G::CH;          // x, delta, z, dout (reused for dx, ddelta, dz)
 }
 
 template <typename IO, int N>
 __global__ void __launch_bounds__(BwdGeom<N>::THREADS) ssm_bwd_kernel(const BwdParams p) {
   using G = BwdGeom<N>;
-  constexpr int S = G::S, LPC = G::LPC, CH = G::CH, WARPS = G::WARPS, T = kCkptSteps;
+  constexpr int S = G::S, LPC = G::LPC, CH = G::CH, WARPS = G::WARPS, T = kBwdTile;
   constexpr int kBwdThreads = G::THREADS;
 
   extern __shared__ __align__(16) unsigned char smem_raw[];
@@ -120,7 +123,7 @@ __global__ void __launch_bounds__(BwdGeom<N>::THREADS) ssm_bwd_kernel(const BwdP
     float h[S];
 #pragma unroll
     for (int k = 0; k < S; ++k) {
-      h[k] = valid ? p.ckpt[(((size_t)b * p.nck + kb) * D + d) * N + j * S + k] : 0.f;
+      h[k] = valid ? p.ckpt[(((size_t)b * p.nck + (size_t)kb * (T / kCkptSteps)) * D + d) * N + j * S + k] : 0.f;
       s_h[(size_t)slot * N + j * S + k] = h[k];
     }
     __syncthreads();
@@ -275,7 +278,7 @@ __global__ void __launch_bounds__(BwdGeom<N>::THREADS) ssm_bwd_kernel(const BwdP
 template <typename IO, int N>
 __global__ void __launch_bounds__(BwdGeom<N>::THREADS) ssm_bwd_local_kernel(const BwdParams p) {
   using G = BwdGeom<N>;
-  constexpr int S = G::S, LPC = G::LPC, CH = G::CH, T = kCkptSteps;
+  constexpr int S = G::S, LPC = G::LPC, CH = G::CH, T = kBwdTile;
   constexpr int kBwdThreads = G::THREADS;
   __shared__ __align__(16) IO s_d[T * CH];
   __shared__ __align__(16) IO s_z[T * CH];

@@ -1,0 +1,724 @@
+// Backward selective scan, tuned path: bf16 io, N = 16, D % 8 == 0, 16-byte aligned pointers.
+// Same mathematics as ssm_bwd.cu (adjoint of Eq. 2a/2b with skip term and gate; states recomputed, Section 3.3).
+//
+// One warp is one worker, as in the tuned forward kernel (ssm_fwd_warp.cu): it owns 32 adjacent channels of one batch
+// entry, walks its part of the sequence backwards in tiles of 16 steps, stages its own tiles with cp.async and shares
+// nothing with the other warps of its block.  A thread holds 16 recurrences as packed float2 pairs: S states of
+// CPT = 16 / S channels; local channel q of lane j (j = lane % LPC, LPC = 16 / S) is channel j ^ q of its lane group, so
+// the sums over n are exchanged with xor-shuffles and every lane finishes exactly one channel per step (channel `lane`).
+//
+// Recomputation.  The forward pass left the state at the start of every block of 8 steps, so a sub-block of 8 steps is
+// rebuilt directly from its checkpoint: a forward sweep keeps the states after the odd steps in registers (64
+// registers), the reverse sweep walks the steps in pairs and rebuilds the state after the even step of a pair from the
+// one before it (one multiply-add per state), which is also the h_{t-1} of the odd step.
+//
+// Sums.  The sums over n (readout for dz, sum lam B for dx and ddelta, sum w A for ddelta) are reduce-scattered over
+// the lane group.  dB and dC are summed over the CPT channels of a thread in registers and over the lane groups of
+// the warp through a transposing pass over shared memory every 4 steps, in a fixed order, and leave the warp as partial
+// sums per group of 32 channels that ssm_bwd_reduce_kernel adds in ascending group order.  dA and dD accumulate in
+// registers along the chain.  Everything is deterministic; there are no floating-point atomics.
+//
+// Schedule.  As in the forward kernel (WarpSched in ssm_common.cuh), in reverse time: a chain that two workers share
+// hands the adjoint mu and the dA / dD accumulators from one to the other once, through L2, behind a bounded wait.
+#include <cstdlib>
+#include <type_traits>
+
+#include "ssm_common.cuh"
+
+namespace ssm {
+
+int warp_workers(int chains, int sms, int per_sm, int max_workers);
+
+namespace {
+
+constexpr int kBT = 8;             // steps per tile (one sub-block: 8 warps per SM need small tiles)
+constexpr int kSB = kCkptSteps;    // steps per sub-block = checkpoint spacing
+constexpr int kRB = 4;             // steps between two dB / dC transposes
+constexpr int kBwdWarps = 4;       // warps per block
+constexpr int kBwdHandoffVec = 9;  // float4 per lane: mu (4), dA (4), dD and dbias (1)
+constexpr float kInvLog2e = 0.6931471805599453f;
+static_assert(kSB == 8 && kBT % kSB == 0, "sub-blocks of 8 steps, whole sub-blocks per tile");
+
+template <int S, bool SP>
+struct BwdWarpSmem {
+  uint32_t x[2][kBT][16];    // bf16 pairs, 32 channels
+  uint32_t d[2][kBT][16];
+  uint32_t z[2][kBT][16];
+  uint32_t g[2][kBT][16];
+  uint32_t rB[2][kBT][8];    // bf16 pairs, 16 states
+  uint32_t rC[2][kBT][8];
+  float4 ck[2][kBT / kSB][4][32];   // checkpoint states: [sub-block][float4 of the thread][lane]
+  float fB[kBT][16];         // B and C of the tile widened to float
+  float fC[kBT][16];
+  float ds[kBT][32];         // dout * silu(z)
+  float gp[kBT][32];         // dout * silu'(z)
+  float dF[SP ? kBT : 1][32];   // SP: step sizes after bias and softplus
+  uint32_t ox[kBT][16];      // dx, ddelta, dz of the tile (bf16 pairs)
+  uint32_t od[kBT][16];
+  uint32_t oz[kBT][16];
+  float4 red[kRB][32][S / 2];   // dB / dC terms of 4 steps: [step][lane][dB float4s | dC float4s], swizzled
+};
+
+#ifdef SSM_DEBUG_BOUNDS
+#define SSM_BROW(r, abort_ptr) \
+  (((unsigned)(r) < (unsigned)kBT) ? (r) : (((abort_ptr) != nullptr ? atomicExch((abort_ptr), 2) : 0), 0))
+#else
+#define SSM_BROW(r, abort_ptr) (r)
+#endif
+
+template <int S>
+struct Lane {
+  static constexpr int LPC = 16 / S, CPT = LPC, H = S / 2, V = S / 2;   // V: float4 of dB / dC terms per thread and step
+  int lane, j, g;
+  uint32_t sel0, sel1;
+  __device__ __forceinline__ explicit Lane(int l) : lane(l), j(l % LPC), g(l / LPC) {
+    sel0 = (j & 1) ? 0x3244u : 0x1044u;
+    sel1 = (j & 1) ? 0x1044u : 0x3244u;
+  }
+  // the CPT values of a tile row (32 channels as 16 bf16 pairs) that belong to this thread, by local channel
+  __device__ __forceinline__ void unpack_row(const uint32_t* row, float (&v)[CPT]) const {
+    if constexpr (CPT == 1) {
+      v[0] = __uint_as_float((uint32_t)reinterpret_cast<const uint16_t*>(row)[lane] << 16);
+    } else if constexpr (CPT == 2) {
+      const uint32_t w = row[g];
+      v[0] = bf16sel(w, sel0);
+      v[1] = bf16sel(w, sel1);
+    } else {
+      const uint2 w = *reinterpret_cast<const uint2*>(row + 2 * g);
+      const uint32_t wa = (j & 2) ? w.y : w.x, wb = (j & 2) ? w.x : w.y;
+      v[0] = bf16sel(wa, sel0);
+      v[1] = bf16sel(wa, sel1);
+      v[2] = bf16sel(wb, sel0);
+      v[3] = bf16sel(wb, sel1);
+    }
+  }
+  // the same from a row of 32 floats
+  __device__ __forceinline__ void pick_row(const float* row, float (&v)[CPT]) const {
+    if constexpr (CPT == 1) {
+      v[0] = row[lane];
+    } else if constexpr (CPT == 2) {
+      const float2 f = *reinterpret_cast<const float2*>(row + 2 * g);
+      v[0] = (j & 1) ? f.y : f.x;
+      v[1] = (j & 1) ? f.x : f.y;
+    } else {
+      const float4 f = *reinterpret_cast<const float4*>(row + 4 * g);
+      const float a0 = (j & 2) ? f.z : f.x, a1 = (j & 2) ? f.w : f.y, b0 = (j & 2) ? f.x : f.z, b1 = (j & 2) ? f.y : f.w;
+      v[0] = (j & 1) ? a1 : a0;
+      v[1] = (j & 1) ? a0 : a1;
+      v[2] = (j & 1) ? b1 : b0;
+      v[3] = (j & 1) ? b0 : b1;
+    }
+  }
+  // this thread's S states of a row of 16 floats
+  __device__ __forceinline__ void load_states_f(const float* row, float2 (&v)[H]) const {
+#pragma unroll
+    for (int k = 0; k < H / 2; ++k) {
+      const float4 a = *reinterpret_cast<const float4*>(row + S * j + 4 * k);
+      v[2 * k] = make_float2(a.x, a.y);
+      v[2 * k + 1] = make_float2(a.z, a.w);
+    }
+  }
+  // this thread's S states of a packed B or C row (16 states as 8 bf16 pairs), widened
+  __device__ __forceinline__ void load_states(const uint32_t* row, float2 (&v)[H]) const {
+    if constexpr (H == 8) {
+      const uint4 a = *reinterpret_cast<const uint4*>(row), b = *reinterpret_cast<const uint4*>(row + 4);
+      const uint32_t w[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
+#pragma unroll
+      for (int k = 0; k < 8; ++k) v[k] = make_float2(bf16lo(w[k]), bf16hi(w[k]));
+    } else if constexpr (H == 4) {
+      const uint4 a = *reinterpret_cast<const uint4*>(row + 4 * j);
+      const uint32_t w[4] = {a.x, a.y, a.z, a.w};
+#pragma unroll
+      for (int k = 0; k < 4; ++k) v[k] = make_float2(bf16lo(w[k]), bf16hi(w[k]));
+    } else {
+      const uint2 a = *reinterpret_cast<const uint2*>(row + 2 * j);
+      v[0] = make_float2(bf16lo(a.x), bf16hi(a.x));
+      v[1] = make_float2(bf16lo(a.y), bf16hi(a.y));
+    }
+  }
+};
+
+// Decays of one (step, channel): general A (one exponential per state) or arithmetic-progression A (two exponentials)
+template <int H, bool AP>
+__device__ __forceinline__ void decays(float dt, const float2 (&A2)[H], float a0s, float rs, float2 (&a)[H]) {
+  if constexpr (AP) {
+    const float a0 = ex2_approx(dt * a0s);
+    const float rr = ex2_approx(dt * rs);
+    const float r2 = rr * rr;
+    a[0] = make_float2(a0, a0 * rr);
+    if constexpr (H > 1) a[1] = f2mul(a[0], f2dup(r2));
+    if constexpr (H > 2) {
+      const float r4 = r2 * r2;
+      a[2] = f2mul(a[0], f2dup(r4));
+      a[3] = f2mul(a[1], f2dup(r4));
+      if constexpr (H > 4) {
+        const float r8 = r4 * r4;
+#pragma unroll
+        for (int k = 0; k < 4; ++k) a[4 + k] = f2mul(a[k], f2dup(r8));
+      }
+    }
+  } else {
+#pragma unroll
+    for (int k = 0; k < H; ++k) {
+      const float2 e = f2mul(f2dup(dt), A2[k]);
+      a[k] = make_float2(ex2_approx(e.x), ex2_approx(e.y));
+    }
+  }
+}
+
+// Per-thread state that lives along a chain
+template <int S>
+struct ChainRegs {
+  static constexpr int CPT = 16 / S, H = S / 2;
+  float2 A2[CPT][H];    // A * log2(e)
+  float a0s[CPT], rs[CPT];
+  float2 mu[CPT][H];    // adjoint flowing backwards in time
+  float2 dA[CPT][H];
+  float Dk, bias_own, dD, dbias;
+};
+
+// One sub-block of 8 steps: rows [r0, r0 + 8) of the tile; nlive = rows of the tile inside the segment.
+template <int S, bool SP, bool AP>
+__device__ __forceinline__ void sub_block(const Lane<S>& ln, ChainRegs<S>& cr, int r0, int nlive, float gate_on,
+                                          bool softplus, const uint32_t* tx, const uint32_t* td, const float* tfB,
+                                          const float* tfC, const float* tds, const float* tgp, const float* tdF,
+                                          const float4* tck, uint32_t* tox, uint32_t* tod, uint32_t* toz, float4* tred,
+                                          float* part_dB, float* part_dC, int* abort_word) {
+  constexpr int LPC = Lane<S>::LPC, CPT = Lane<S>::CPT, H = Lane<S>::H, V = Lane<S>::V;
+  const int lane = ln.lane;
+  // ---- forward sweep from the checkpoint: the states after the odd steps stay in registers
+  float2 hist[kSB / 2][CPT][H];
+  {
+    float2 h[CPT][H];
+#pragma unroll
+    for (int q = 0; q < CPT; ++q)
+#pragma unroll
+      for (int k = 0; k < S / 4; ++k) {
+        const float4 v = tck[(q * (S / 4) + k) * 32 + lane];
+        h[q][2 * k] = make_float2(v.x, v.y);
+        h[q][2 * k + 1] = make_float2(v.z, v.w);
+      }
+    float dt[kSB][CPT], u[kSB][CPT];
+#pragma unroll
+    for (int t = 0; t < kSB; ++t) {
+      const int r = SSM_BROW(r0 + t, abort_word);
+      if constexpr (SP) ln.pick_row(tdF + r * 32, dt[t]);
+      else ln.unpack_row(td + r * 16, dt[t]);
+      ln.unpack_row(tx + r * 16, u[t]);
+    }
+#pragma unroll
+    for (int t = 0; t < kSB; ++t) {
+      const int r = SSM_BROW(r0 + t, abort_word);
+      float2 Bv[H];
+      ln.load_states_f(tfB + r * 16, Bv);
+#pragma unroll
+      for (int q = 0; q < CPT; ++q) {
+        float2 a[H];
+        decays<H, AP>(dt[t][q], cr.A2[q], cr.a0s[q], cr.rs[q], a);
+        const float2 du2 = f2dup(dt[t][q] * u[t][q]);
+#pragma unroll
+        for (int k = 0; k < H; ++k) {
+          h[q][k] = f2fma(a[k], h[q][k], f2mul(du2, Bv[k]));
+          if (t & 1) hist[t >> 1][q][k] = h[q][k];
+        }
+      }
+    }
+  }
+  // ---- reverse sweep in pairs of steps (2m + 1, 2m)
+#pragma unroll
+  for (int m = kSB / 2 - 1; m >= 0; --m) {
+    // ======== odd step t1 = 2m + 1: its state is hist[m]; its w = mu h_{t-1} waits for the even step's state
+    const int r1 = SSM_BROW(r0 + 2 * m + 1, abort_word);
+    float dt1[CPT], u1[CPT], ds1[CPT];
+    if constexpr (SP) ln.pick_row(tdF + r1 * 32, dt1);
+    else ln.unpack_row(td + r1 * 16, dt1);
+    ln.unpack_row(tx + r1 * 16, u1);
+    ln.pick_row(tds + r1 * 32, ds1);
+    const float gp1 = tgp[r1 * 32 + lane];
+    float raw1 = 0.f;
+    if constexpr (SP) raw1 = __uint_as_float((uint32_t)reinterpret_cast<const uint16_t*>(td + r1 * 16)[lane] << 16);
+    float y1[CPT], lb1[CPT];
+    {
+      float2 Bv[H], Cv[H];
+      ln.load_states_f(tfB + r1 * 16, Bv);
+      ln.load_states_f(tfC + r1 * 16, Cv);
+      float2 dBt[H], dCt[H];
+#pragma unroll
+      for (int q = 0; q < CPT; ++q) {
+        float2 a[H];
+        decays<H, AP>(dt1[q], cr.A2[q], cr.a0s[q], cr.rs[q], a);
+        const float2 ds2 = f2dup(ds1[q]), du2 = f2dup(dt1[q] * u1[q]);
+        float2 yv = make_float2(0.f, 0.f), lb = yv;
+#pragma unroll
+        for (int k = 0; k < H; ++k) {
+          const float2 hc = hist[m][q][k];
+          const float2 lam = f2fma(Cv[k], ds2, cr.mu[q][k]);
+          if (q == 0) {
+            dCt[k] = f2mul(ds2, hc);
+            dBt[k] = f2mul(lam, du2);
+          } else {
+            dCt[k] = f2fma(ds2, hc, dCt[k]);
+            dBt[k] = f2fma(lam, du2, dBt[k]);
+          }
+          lb = f2fma(lam, Bv[k], lb);
+          yv = f2fma(Cv[k], hc, yv);
+          cr.mu[q][k] = f2mul(a[k], lam);
+        }
+        y1[q] = yv.x + yv.y;
+        lb1[q] = lb.x + lb.y;
+      }
+      // dB / dC terms of this step into the transposing buffer (swizzled: conflict-free 16-byte stores)
+      float4* rrow = tred + ((2 * m + 1) & (kRB - 1)) * 32 * V + lane * V;
+      const int swz = (lane / (8 / V)) & (V - 1);
+#pragma unroll
+      for (int v = 0; v < V / 2; ++v) {
+        rrow[v ^ swz] = make_float4(dBt[2 * v].x, dBt[2 * v].y, dBt[2 * v + 1].x, dBt[2 * v + 1].y);
+        rrow[(V / 2 + v) ^ swz] = make_float4(dCt[2 * v].x, dCt[2 * v].y, dCt[2 * v + 1].x, dCt[2 * v + 1].y);
+      }
+    }
+#pragma unroll
+    for (int mm = 1; mm < LPC; mm <<= 1) {
+#pragma unroll
+      for (int q = 0; q < CPT; ++q)
+        if ((q & (2 * mm - 1)) == 0) {
+          y1[q] += __shfl_xor_sync(0xffffffffu, y1[q + mm], mm);
+          lb1[q] += __shfl_xor_sync(0xffffffffu, lb1[q + mm], mm);
+        }
+    }
+    const float dz1 = gp1 * fmaf(cr.Dk, u1[0], y1[0]);
+    const float dx1 = fmaf(dt1[0], lb1[0], ds1[0] * cr.Dk);
+    cr.dD = fmaf(ds1[0], u1[0], cr.dD);
+
+    // ======== even step t0 = 2m: its state is rebuilt from the one before it
+    const int r0e = SSM_BROW(r0 + 2 * m, abort_word);
+    float dt0[CPT], u0[CPT], ds0[CPT];
+    if constexpr (SP) ln.pick_row(tdF + r0e * 32, dt0);
+    else ln.unpack_row(td + r0e * 16, dt0);
+    ln.unpack_row(tx + r0e * 16, u0);
+    ln.pick_row(tds + r0e * 32, ds0);
+    const float gp0 = tgp[r0e * 32 + lane];
+    float raw0 = 0.f;
+    if constexpr (SP) raw0 = __uint_as_float((uint32_t)reinterpret_cast<const uint16_t*>(td + r0e * 16)[lane] << 16);
+    float y0[CPT], lb0[CPT], wa0[CPT], wa1[CPT];
+    {
+      float2 Bv[H], Cv[H];
+      ln.load_states_f(tfB + r0e * 16, Bv);
+      ln.load_states_f(tfC + r0e * 16, Cv);
+      float2 dBt[H], dCt[H];
+#pragma unroll
+      for (int q = 0; q < CPT; ++q) {
+        float2 a[H];
+        decays<H, AP>(dt0[q], cr.A2[q], cr.a0s[q], cr.rs[q], a);
+        const float2 ds2 = f2dup(ds0[q]), du2 = f2dup(dt0[q] * u0[q]), dt02 = f2dup(dt0[q]), dt12 = f2dup(dt1[q]);
+        float2 yv = make_float2(0.f, 0.f), lb = yv, w0a = yv, w1a = yv;
+#pragma unroll
+        for (int k = 0; k < H; ++k) {
+          float2 hpp;   // the state before the even step: the history entry before, or the checkpoint
+          if (m > 0) {
+            hpp = hist[m > 0 ? m - 1 : 0][q][k];
+          } else {
+            const float4 v = tck[(q * (S / 4) + (k >> 1)) * 32 + lane];
+            hpp = (k & 1) ? make_float2(v.z, v.w) : make_float2(v.x, v.y);
+          }
+          const float2 he = f2fma(a[k], hpp, f2mul(du2, Bv[k]));      // h after the even step
+          const float2 w1 = f2mul(cr.mu[q][k], he);                   // the odd step's w = mu_{t1} h_{t1 - 1}
+          w1a = f2fma(w1, cr.A2[q][k], w1a);
+          cr.dA[q][k] = f2fma(w1, dt12, cr.dA[q][k]);
+          const float2 lam = f2fma(Cv[k], ds2, cr.mu[q][k]);
+          if (q == 0) {
+            dCt[k] = f2mul(ds2, he);
+            dBt[k] = f2mul(lam, du2);
+          } else {
+            dCt[k] = f2fma(ds2, he, dCt[k]);
+            dBt[k] = f2fma(lam, du2, dBt[k]);
+          }
+          lb = f2fma(lam, Bv[k], lb);
+          yv = f2fma(Cv[k], he, yv);
+          cr.mu[q][k] = f2mul(a[k], lam);
+          const float2 w0 = f2mul(cr.mu[q][k], hpp);
+          w0a = f2fma(w0, cr.A2[q][k], w0a);
+          cr.dA[q][k] = f2fma(w0, dt02, cr.dA[q][k]);
+        }
+        y0[q] = yv.x + yv.y;
+        lb0[q] = lb.x + lb.y;
+        wa0[q] = w0a.x + w0a.y;
+        wa1[q] = w1a.x + w1a.y;
+      }
+      float4* rrow = tred + ((2 * m) & (kRB - 1)) * 32 * V + lane * V;
+      const int swz = (lane / (8 / V)) & (V - 1);
+#pragma unroll
+      for (int v = 0; v < V / 2; ++v) {
+        rrow[v ^ swz] = make_float4(dBt[2 * v].x, dBt[2 * v].y, dBt[2 * v + 1].x, dBt[2 * v + 1].y);
+        rrow[(V / 2 + v) ^ swz] = make_float4(dCt[2 * v].x, dCt[2 * v].y, dCt[2 * v + 1].x, dCt[2 * v + 1].y);
+      }
+    }
+#pragma unroll
+    for (int mm = 1; mm < LPC; mm <<= 1) {
+#pragma unroll
+      for (int q = 0; q < CPT; ++q)
+        if ((q & (2 * mm - 1)) == 0) {
+          y0[q] += __shfl_xor_sync(0xffffffffu, y0[q + mm], mm);
+          lb0[q] += __shfl_xor_sync(0xffffffffu, lb0[q + mm], mm);
+          wa0[q] += __shfl_xor_sync(0xffffffffu, wa0[q + mm], mm);
+          wa1[q] += __shfl_xor_sync(0xffffffffu, wa1[q + mm], mm);
+        }
+    }
+    // ---- finish both steps of the pair for this lane's own channel
+    const float dz0 = gp0 * fmaf(cr.Dk, u0[0], y0[0]);
+    const float dx0 = fmaf(dt0[0], lb0[0], ds0[0] * cr.Dk);
+    cr.dD = fmaf(ds0[0], u0[0], cr.dD);
+    float dd1 = fmaf(u1[0], lb1[0], wa1[0] * kInvLog2e);
+    float dd0 = fmaf(u0[0], lb0[0], wa0[0] * kInvLog2e);
+    if constexpr (SP) {
+      // the gradient goes to the pre-activation v: d softplus(v) / dv = sigmoid(v); the bias gets the sum over time
+      if (softplus) {
+        dd1 *= sigmoid_fast(raw1 + cr.bias_own);
+        dd0 *= sigmoid_fast(raw0 + cr.bias_own);
+      }
+      if (r0 + 2 * m + 1 < nlive) cr.dbias += dd1;
+      if (r0 + 2 * m < nlive) cr.dbias += dd0;
+    }
+    reinterpret_cast<__nv_bfloat16*>(tox + r1 * 16)[lane] = __float2bfloat16_rn(dx1);
+    reinterpret_cast<__nv_bfloat16*>(tod + r1 * 16)[lane] = __float2bfloat16_rn(dd1);
+    reinterpret_cast<__nv_bfloat16*>(toz + r1 * 16)[lane] = __float2bfloat16_rn(dz1 * gate_on);
+    reinterpret_cast<__nv_bfloat16*>(tox + r0e * 16)[lane] = __float2bfloat16_rn(dx0);
+    reinterpret_cast<__nv_bfloat16*>(tod + r0e * 16)[lane] = __float2bfloat16_rn(dd0);
+    reinterpret_cast<__nv_bfloat16*>(toz + r0e * 16)[lane] = __float2bfloat16_rn(dz0 * gate_on);
+
+    if ((2 * m) % kRB == 0) {
+      // dB / dC of steps 2m .. 2m + 3: every lane sums one float4 of one step over the lane groups, ascending
+      __syncwarp();
+      const int s = lane >> 3, o = lane & 7;
+      const int which = o >> 2, n0 = 4 * (o & 3);
+      const int jo = n0 / S, v = which * (S / 4) + (n0 % S) / 4;
+      const float4* rs_ = tred + s * 32 * V;
+      float4 acc;
+#pragma unroll
+      for (int gg = 0; gg < 32 / LPC; ++gg) {
+        const int l = gg * LPC + jo;
+        const float4 t4 = rs_[l * V + (v ^ ((l / (8 / V)) & (V - 1)))];
+        if (gg == 0) acc = t4;
+        else { acc.x += t4.x; acc.y += t4.y; acc.z += t4.z; acc.w += t4.w; }
+      }
+      const int row = r0 + 2 * m + s;
+      if (row < nlive) *reinterpret_cast<float4*>((which ? part_dC : part_dB) + (size_t)row * 16 + n0) = acc;
+      __syncwarp();
+    }
+  }
+}
+
+}  // namespace
+
+template <int S, bool SP>
+__global__ void __launch_bounds__(kBwdWarps * 32) ssm_bwd_warp_kernel(const BwdParams p, const WarpSched sc) {
+  constexpr int LPC = 16 / S, CPT = LPC, H = S / 2;
+  using Smem = BwdWarpSmem<S, SP>;
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  Smem& sm = reinterpret_cast<Smem*>(smem_raw)[warp];
+  const Lane<S> ln(lane);
+  const int j = ln.j, g = ln.g;
+  const int D = p.D;
+  const int worker = blockIdx.x * kBwdWarps + warp;
+  const bool has_z = p.z != nullptr;
+
+  const __nv_bfloat16* __restrict__ gx = static_cast<const __nv_bfloat16*>(p.x);
+  const __nv_bfloat16* __restrict__ gd = static_cast<const __nv_bfloat16*>(p.delta);
+  const __nv_bfloat16* __restrict__ gz = static_cast<const __nv_bfloat16*>(p.z);
+  const __nv_bfloat16* __restrict__ gg = static_cast<const __nv_bfloat16*>(p.dout);
+  const __nv_bfloat16* __restrict__ gB = static_cast<const __nv_bfloat16*>(p.B);
+  const __nv_bfloat16* __restrict__ gC = static_cast<const __nv_bfloat16*>(p.C);
+  __nv_bfloat16* __restrict__ gdx = static_cast<__nv_bfloat16*>(p.dx);
+  __nv_bfloat16* __restrict__ gdd = static_cast<__nv_bfloat16*>(p.ddelta);
+  __nv_bfloat16* __restrict__ gdz = static_cast<__nv_bfloat16*>(p.dz);
+
+  const int groups = (D + 31) / 32;
+  const size_t bln = (size_t)p.batch * p.L * 16;
+  const WorkList wl = make_worklist(sc, worker);
+  for (int pi = 0; pi < wl.count; ++pi) {
+    int chain, from, to;
+    get_piece(wl, sc.tiles, pi, chain, from, to);
+    const int grp = chain % groups;
+    const int bs = chain / groups;
+    const int seg = bs % p.nseg, b = bs / p.nseg;
+    const int d_w = grp * 32;
+    const int t_seg0 = seg * p.seg_steps;
+    const int t_seg_end = min(p.L, t_seg0 + p.seg_steps);
+    const int live_tiles = (t_seg_end - t_seg0 + kBT - 1) / kBT;
+    // positions [from, to) of the chain in processing order are tiles tile_hi down to tile_lo (time runs backwards)
+    const int tile_lo = sc.tiles - to;
+    int tile_hi = sc.tiles - 1 - from;
+    if (tile_hi > live_tiles - 1) tile_hi = live_tiles - 1;
+    const bool gives_out = to < sc.tiles;
+
+    // ---- staging: this lane's chunks of a tile (rows lane / 4 + 8 k of x, delta, z, dout; row lane / 2 of B, C)
+    const int xrow = lane >> 2, xcc = lane & 3;
+    const bool xcol_ok = d_w + xcc * 8 < D;
+    const int brow = lane >> 1, bhc = lane & 1;
+    const int c_grp = d_w + g * CPT;          // first channel of this lane group (all valid or none)
+    const bool valid = c_grp < D;
+    auto chan = [&](int q) { return c_grp + (j ^ q); };
+    auto issue_tile = [&](int tile, int st) {
+      if (tile >= tile_lo && tile >= 0) {
+        const int t0 = t_seg0 + tile * kBT;
+        const size_t row0 = (size_t)b * p.L + t0;
+#pragma unroll
+        for (int k = 0; k < (kBT + 7) / 8; ++k) {
+          const int tt = xrow + 8 * k;
+          const bool ok = xcol_ok && (t0 + tt < t_seg_end);
+          const size_t go = ok ? (row0 + tt) * D + d_w + xcc * 8 : 0;
+          cp_async16(&sm.x[st][tt][xcc * 4], gx + go, ok);
+          cp_async16(&sm.d[st][tt][xcc * 4], gd + go, ok);
+          cp_async16(&sm.z[st][tt][xcc * 4], (has_z ? gz : gx) + go, ok && has_z);
+          cp_async16(&sm.g[st][tt][xcc * 4], gg + go, ok);
+        }
+        if (brow < kBT) {
+          const bool ok = t0 + brow < t_seg_end;
+          const size_t go = ok ? (row0 + brow) * 16 + bhc * 8 : 0;
+          cp_async16(&sm.rB[st][brow][bhc * 4], gB + go, ok);
+          cp_async16(&sm.rC[st][brow][bhc * 4], gC + go, ok);
+        }
+#pragma unroll
+        for (int sb = 0; sb < kBT / kSB; ++sb) {
+          const bool ok = valid && (t0 + sb * kSB < t_seg_end);
+#pragma unroll
+          for (int q = 0; q < CPT; ++q)
+#pragma unroll
+            for (int k = 0; k < S / 4; ++k) {
+              const size_t go = ok ? (((size_t)b * p.nck + (t0 + sb * kSB) / kCkptSteps) * D + chan(q)) * 16 + S * j + 4 * k : 0;
+              cp_async16(&sm.ck[st][sb][q * (S / 4) + k][lane], p.ckpt + go, ok);
+            }
+        }
+      }
+      cp_async_commit();
+    };
+    issue_tile(tile_hi, 0);
+
+    // ---- per-thread constants and carried values
+    ChainRegs<S> cr;
+    bool ap = !p.general_A;
+#pragma unroll
+    for (int q = 0; q < CPT; ++q) {
+      float av[S];
+#pragma unroll
+      for (int k = 0; k < S / 4; ++k) {
+        float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (valid) a = *reinterpret_cast<const float4*>(p.A + (size_t)chan(q) * 16 + S * j + 4 * k);
+        av[4 * k] = a.x; av[4 * k + 1] = a.y; av[4 * k + 2] = a.z; av[4 * k + 3] = a.w;
+      }
+      const float step = av[1] - av[0];
+      const float tol = 1e-6f * fabsf(av[S - 1]);
+#pragma unroll
+      for (int k = 2; k < S; ++k) ap = ap && fabsf(av[k] - (av[0] + (float)k * step)) <= tol;
+#pragma unroll
+      for (int k = 0; k < H; ++k) cr.A2[q][k] = make_float2(av[2 * k] * kLog2e, av[2 * k + 1] * kLog2e);
+      cr.a0s[q] = cr.A2[q][0].x;
+      cr.rs[q] = cr.A2[q][0].y - cr.A2[q][0].x;
+    }
+    ap = __all_sync(0xffffffffu, ap);
+    const int c_own = d_w + lane;
+    cr.Dk = (p.Dskip != nullptr && c_own < D) ? p.Dskip[c_own] : 0.f;
+    cr.bias_own = (SP && p.delta_bias != nullptr && c_own < D) ? p.delta_bias[c_own] : 0.f;
+    cr.dD = 0.f;
+    cr.dbias = 0.f;
+    if (from > 0) {
+      if (!wait_handoff(sc, worker, lane)) {
+        cp_async_wait_all();
+        return;
+      }
+      const float4* hb = sc.handoff + ((size_t)worker * 32 + lane) * kBwdHandoffVec;
+      float4 v[8];
+#pragma unroll
+      for (int k = 0; k < 8; ++k) v[k] = __ldcg(hb + k);
+      const float4 dv = __ldcg(hb + 8);
+      const float* f = reinterpret_cast<const float*>(v);
+#pragma unroll
+      for (int q = 0; q < CPT; ++q)
+#pragma unroll
+        for (int k = 0; k < H; ++k) {
+          cr.mu[q][k] = make_float2(f[(q * H + k) * 2], f[(q * H + k) * 2 + 1]);
+          cr.dA[q][k] = make_float2(f[16 + (q * H + k) * 2], f[16 + (q * H + k) * 2 + 1]);
+        }
+      cr.dD = dv.x;
+      cr.dbias = dv.y;
+    } else {
+#pragma unroll
+      for (int q = 0; q < CPT; ++q)
+#pragma unroll
+        for (int k = 0; k < S / 4; ++k) {
+          float4 m4 = make_float4(0.f, 0.f, 0.f, 0.f);
+          if (valid && p.mu_in != nullptr)
+            m4 = *reinterpret_cast<const float4*>(p.mu_in + (((size_t)b * p.nseg + seg) * D + chan(q)) * 16 + S * j + 4 * k);
+          cr.mu[q][2 * k] = make_float2(m4.x, m4.y);
+          cr.mu[q][2 * k + 1] = make_float2(m4.z, m4.w);
+          cr.dA[q][2 * k] = cr.dA[q][2 * k + 1] = make_float2(0.f, 0.f);
+        }
+    }
+
+    int st = 0;
+    for (int tile = tile_hi; tile >= tile_lo; --tile, st ^= 1) {
+      cp_async_wait_all();
+      __syncwarp();                   // this tile landed for all lanes; all lanes are done with the previous one
+      issue_tile(tile - 1, st ^ 1);   // prefetch the tile before in time
+      const int t0 = t_seg0 + tile * kBT;
+      const int nlive = min(kBT, t_seg_end - t0);
+      // ---- per-element gate terms of the tile, one channel per lane: ds = dout silu(z), gp = dout silu'(z)
+      {
+        // B and C of the tile to float: lane -> (row lane / 4, states 4 (lane % 4) ..)
+#pragma unroll
+        for (int k = 0; k < (kBT * 4 + 31) / 32; ++k) {
+          const int c = lane + 32 * k, rr = c >> 2, qq = c & 3;
+          if (kBT * 4 % 32 == 0 || rr < kBT) {
+            const uint2 wb = *reinterpret_cast<const uint2*>(&sm.rB[st][rr][2 * qq]);
+            const uint2 wc = *reinterpret_cast<const uint2*>(&sm.rC[st][rr][2 * qq]);
+            *reinterpret_cast<float4*>(&sm.fB[rr][4 * qq]) = make_float4(bf16lo(wb.x), bf16hi(wb.x), bf16lo(wb.y), bf16hi(wb.y));
+            *reinterpret_cast<float4*>(&sm.fC[rr][4 * qq]) = make_float4(bf16lo(wc.x), bf16hi(wc.x), bf16lo(wc.y), bf16hi(wc.y));
+          }
+        }
+        float zf[kBT], gf[kBT], df[SP ? kBT : 1];
+#pragma unroll
+        for (int r = 0; r < kBT; ++r) {
+          zf[r] = __uint_as_float((uint32_t)reinterpret_cast<const uint16_t*>(sm.z[st][r])[lane] << 16);
+          gf[r] = __uint_as_float((uint32_t)reinterpret_cast<const uint16_t*>(sm.g[st][r])[lane] << 16);
+          if constexpr (SP) df[r] = __uint_as_float((uint32_t)reinterpret_cast<const uint16_t*>(sm.d[st][r])[lane] << 16);
+        }
+#pragma unroll
+        for (int r = 0; r < kBT; ++r) {
+          float dsv = gf[r], gpv = 0.f;
+          if (has_z) {
+            const float sg = sigmoid_fast(zf[r]);
+            dsv = gf[r] * zf[r] * sg;
+            gpv = gf[r] * sg * fmaf(zf[r], 1.f - sg, 1.f);
+          }
+          sm.ds[r][lane] = dsv;
+          sm.gp[r][lane] = gpv;
+          if constexpr (SP) {
+            float v = df[r] + cr.bias_own;
+            if (p.softplus) v = softplus_fast(v);
+            sm.dF[r][lane] = r < nlive ? v : 0.f;   // rows past the end stay identity steps
+          }
+        }
+      }
+      __syncwarp();
+      const size_t row0 = (size_t)b * p.L + t0;
+      float* part_dB = p.dBC_part + ((size_t)grp * 2 + 0) * bln + row0 * 16;
+      float* part_dC = p.dBC_part + ((size_t)grp * 2 + 1) * bln + row0 * 16;
+#pragma unroll 1
+      for (int sb = kBT / kSB - 1; sb >= 0; --sb) {
+        if (sb * kSB >= nlive) continue;   // a sub-block of identity steps
+        if (ap)
+          sub_block<S, SP, true>(ln, cr, sb * kSB, nlive, has_z ? 1.f : 0.f, p.softplus != 0, &sm.x[st][0][0], &sm.d[st][0][0],
+                                 &sm.fB[0][0], &sm.fC[0][0], &sm.ds[0][0], &sm.gp[0][0], &sm.dF[0][0],
+                                 &sm.ck[st][sb][0][0], &sm.ox[0][0], &sm.od[0][0], &sm.oz[0][0], &sm.red[0][0][0], part_dB,
+                                 part_dC, sc.abort);
+        else
+          sub_block<S, SP, false>(ln, cr, sb * kSB, nlive, has_z ? 1.f : 0.f, p.softplus != 0, &sm.x[st][0][0], &sm.d[st][0][0],
+                                  &sm.fB[0][0], &sm.fC[0][0], &sm.ds[0][0], &sm.gp[0][0], &sm.dF[0][0],
+                                  &sm.ck[st][sb][0][0], &sm.ox[0][0], &sm.od[0][0], &sm.oz[0][0], &sm.red[0][0][0], part_dB,
+                                  part_dC, sc.abort);
+      }
+      __syncwarp();
+      // ---- results of the tile: 16-byte stores of dx, ddelta, dz
+#pragma unroll
+      for (int k = 0; k < (kBT + 7) / 8; ++k) {
+        const int tt = xrow + 8 * k;
+        if (xcol_ok && tt < nlive) {
+          const size_t go = (row0 + tt) * D + d_w + xcc * 8;
+          *reinterpret_cast<uint4*>(gdx + go) = *reinterpret_cast<const uint4*>(&sm.ox[tt][xcc * 4]);
+          *reinterpret_cast<uint4*>(gdd + go) = *reinterpret_cast<const uint4*>(&sm.od[tt][xcc * 4]);
+          if (gdz != nullptr) *reinterpret_cast<uint4*>(gdz + go) = *reinterpret_cast<const uint4*>(&sm.oz[tt][xcc * 4]);
+        }
+      }
+    }
+    cp_async_wait_all();
+    __syncwarp();
+
+    if (gives_out) {
+      // the earlier part of this chain (in time) belongs to the next worker
+      float4* hb = sc.handoff + ((size_t)(worker + 1) * 32 + lane) * kBwdHandoffVec;
+      float f[32];
+#pragma unroll
+      for (int q = 0; q < CPT; ++q)
+#pragma unroll
+        for (int k = 0; k < H; ++k) {
+          f[(q * H + k) * 2] = cr.mu[q][k].x;
+          f[(q * H + k) * 2 + 1] = cr.mu[q][k].y;
+          f[16 + (q * H + k) * 2] = cr.dA[q][k].x;
+          f[16 + (q * H + k) * 2 + 1] = cr.dA[q][k].y;
+        }
+#pragma unroll
+      for (int k = 0; k < 8; ++k) __stcg(hb + k, make_float4(f[4 * k], f[4 * k + 1], f[4 * k + 2], f[4 * k + 3]));
+      __stcg(hb + 8, make_float4(cr.dD, cr.dbias, 0.f, 0.f));
+      publish_handoff(sc, worker, lane);
+    } else if (valid) {
+      // first step in time done: the chain is complete
+      const size_t part = (size_t)b * p.nseg + seg;
+#pragma unroll
+      for (int q = 0; q < CPT; ++q)
+#pragma unroll
+        for (int k = 0; k < S / 4; ++k) {
+          *reinterpret_cast<float4*>(p.dA_part + (part * D + chan(q)) * 16 + S * j + 4 * k) =
+              make_float4(cr.dA[q][2 * k].x, cr.dA[q][2 * k].y, cr.dA[q][2 * k + 1].x, cr.dA[q][2 * k + 1].y);
+          if (seg == 0 && p.dh0 != nullptr)   // the adjoint that leaves the first step is the gradient of the initial state
+            *reinterpret_cast<float4*>(p.dh0 + ((size_t)b * D + chan(q)) * 16 + S * j + 4 * k) =
+                make_float4(cr.mu[q][2 * k].x, cr.mu[q][2 * k].y, cr.mu[q][2 * k + 1].x, cr.mu[q][2 * k + 1].y);
+        }
+      p.dD_part[part * D + c_own] = cr.dD;
+      if (SP && p.dbias_part != nullptr) p.dbias_part[part * D + c_own] = cr.dbias;
+    }
+  }
+}
+
+namespace {
+
+template <int S, bool SP>
+cudaError_t launch_bwd_variant(const Plan& plan, const BwdParams& p, cudaStream_t s) {
+  const size_t smem = sizeof(BwdWarpSmem<S, SP>) * kBwdWarps;
+  auto kern = ssm_bwd_warp_kernel<S, SP>;
+  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (e != cudaSuccess) return e;
+  int dev = 0, sms = 0, per_sm = 0;
+  if ((e = cudaGetDevice(&dev)) != cudaSuccess) return e;
+  if ((e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
+  if ((e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, kBwdWarps * 32, smem)) != cudaSuccess) return e;
+  if (per_sm < 1) return cudaErrorLaunchOutOfResources;
+  WarpSched sc{};
+  sc.chains = p.batch * plan.nseg * ((p.D + 31) / 32);
+  sc.tiles = (plan.seg_steps + kBT - 1) / kBT;
+  const bool can_share = p.abort != nullptr && p.flags != nullptr && p.handoff != nullptr && p.max_workers > 0;
+  sc.workers = warp_workers(sc.chains, sms, per_sm * kBwdWarps, can_share ? p.max_workers : 0);
+  if (p.test_withhold && can_share) {
+    // test hook: make neighbouring workers share chains whatever the shape (all of them must be resident)
+    sc.workers = p.max_workers < per_sm * kBwdWarps * sms ? p.max_workers : per_sm * kBwdWarps * sms;
+  }
+  const long long total = (long long)sc.chains * sc.tiles;
+  sc.quota = (int)((total + sc.workers - 1) / sc.workers);
+  sc.spin_limit = p.test_withhold ? 1000 : (1 << 22);
+  sc.withhold = p.test_withhold;
+  sc.flags = p.flags;
+  sc.abort = p.abort;
+  sc.handoff = p.handoff;
+  const unsigned grid = (unsigned)((sc.workers + kBwdWarps - 1) / kBwdWarps);
+  kern<<<grid, kBwdWarps * 32, smem, s>>>(p, sc);
+  return cudaGetLastError();
+}
+
+}  // namespace
+
+bool bwd_fast_applicable(const ssm_problem_t& prob, const BwdParams& p) {
+  auto al16 = [](const void* q) { return q == nullptr || (reinterpret_cast<uintptr_t>(q) & 15) == 0; };
+  if (p.static_B || p.static_C || p.zoh) return false;  // input-dependent B, C and the default B-bar only
+  return prob.io_dtype == SSM_BF16 && prob.N == 16 && prob.D % 8 == 0 && p.seg_steps % kBT == 0 && al16(p.x) &&
+         al16(p.delta) && al16(p.z) && al16(p.B) && al16(p.C) && al16(p.dout) && al16(p.dx) && al16(p.ddelta) &&
+         al16(p.dz) && al16(p.A) && al16(p.ckpt) && al16(p.mu_in) && al16(p.dh0) && al16(p.dBC_part) && al16(p.dA_part) &&
+         al16(p.handoff);
+}
+
+size_t bwd_handoff_bytes_per_worker() { return sizeof(float4) * kBwdHandoffVec * 32; }
+
+cudaError_t launch_bwd_fast(const Plan& plan, const BwdParams& p, cudaStream_t s) {
+  const bool sp = p.softplus || p.delta_bias != nullptr;
+  return sp ? launch_bwd_variant<8, true>(plan, p, s) : launch_bwd_variant<8, false>(plan, p, s);
+}
+
+}  // namespace ssm

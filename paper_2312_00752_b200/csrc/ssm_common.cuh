@@ -11,15 +11,20 @@
 namespace ssm {
 
 // Time steps between two checkpoint states (the state h at the start of every such block is what backward restarts
-// its recomputation from).  Segment lengths of the time split are multiples of this.
-constexpr int kCkptSteps = 32;
+// its recomputation from: 8 steps of a thread's 16 recurrences are what its registers can hold, so no second level of
+// recomputation is needed; the price is 8 bytes per element of checkpoint traffic in each direction, paid from HBM
+// bandwidth the arithmetic-bound kernels leave idle).  Segment lengths of the time split are multiples of this.
+constexpr int kCkptSteps = 8;
+// Segment lengths of the time split are multiples of this (the tile length of every kernel divides it).
+constexpr int kSegAlign = 32;
+static_assert(kSegAlign % kCkptSteps == 0, "segments start on a checkpoint");
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr int kNumSMs = 148;
 
 // ---------------------------------------------------------------------------------------------- plan (host)
 struct Plan {
   int nseg;        // time segments per sequence (1: a thread sweeps the whole sequence)
-  int seg_steps;   // steps per segment (multiple of kCkptSteps; the last segment may be shorter)
+  int seg_steps;   // steps per segment (multiple of kSegAlign; the last segment may be shorter)
   int nck;         // checkpoints per sequence = ceil(L / kCkptSteps)
   int fwd_cpt;     // channels per thread, forward
   int fwd_ch;      // channels per block, forward
@@ -49,6 +54,27 @@ struct FwdParams {
   int general_A;       // 1: never take the arithmetic-progression fast path
   int zoh;             // 1: B-bar = (exp(delta A) - 1) / A * B (Eq. 4) instead of delta * B
   int static_B, static_C;  // 1: B / C is a float32 [D][N] parameter (not input-dependent: Algorithm 1) instead of [batch][L][N]
+  int* abort;            // tuned kernel: status word (non-zero: a bounded wait gave up); null: no chain may be shared
+  int* flags;            // tuned kernel: [max_workers + 1] hand-off flags, zero before the launch
+  float4* handoff;       // tuned kernel: carried state of a chain that two workers share
+  int max_workers;       // tuned kernel: workers the hand-off slots allow (0: no chain may be shared)
+};
+
+// Work distribution of the warp-per-worker kernels.  The work is `chains` independent sequences of `tiles` tiles each
+// (a chain is one time segment of 32 adjacent channels of one batch entry; tiles of a chain must run in order).  The
+// linear tile space [0, chains * tiles) is cut into `workers` equal ranges, one per resident warp.  A range that starts
+// or ends inside a chain shares that chain with the neighbouring worker: the state crosses from one to the other once,
+// through `handoff`, guarded by `flags` (indexed by the receiving worker).  Every worker runs the piece that other
+// workers wait for first (the leading part of its last chain), then its whole chains, then the piece that waits (the
+// trailing part of its first chain); so with all workers resident a wait is satisfied after at most a short time, and
+// the bounded poll below is a safety net, not a scheduling device.
+struct WarpSched {
+  int chains, tiles, workers, quota;   // quota: tiles per worker = ceil(chains * tiles / workers)
+  int spin_limit;                      // polls of a flag before the worker gives up and raises *abort
+  int withhold;                        // test hook: never publish a flag
+  int* flags;                          // [workers + 1], zero before the launch
+  int* abort;                          // one word, zero before the launch; non-zero: some wait gave up
+  float4* handoff;                     // [workers + 1][32 lanes][vectors per lane]
 };
 
 struct CarryParams {
@@ -93,8 +119,10 @@ struct BwdParams {
   float* dBs_part;        // static B: [batch*nseg][D][N] per-thread sums over time of the dB terms
   float* dCs_part;        // static C: same for dC
   int test_withhold;      // test hook: never publish hand-off flags, poll only 1000 times
-  int* sched;             // tuned kernel: [0] claim counter, [1] abort word, [64 + chain] progress flag per chain
-  float4* handoff;        // tuned kernel: carried values between consecutive tiles of a chain
+  int* abort;             // status word of the workspace (non-zero: a bounded wait gave up)
+  int* flags;             // tuned kernel: [max_workers + 1] hand-off flags, zero before the launch
+  float4* handoff;        // tuned kernel: carried values of a chain that two workers share
+  int max_workers;        // tuned kernel: workers the hand-off slots allow (0: no chain may be shared)
 };
 
 struct ReduceParams {
@@ -172,6 +200,80 @@ __device__ __forceinline__ void cp_async16(void* smem_dst, const void* gmem_src,
   const int bytes = valid ? 16 : 0;
   asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(gmem_src), "r"(bytes) : "memory");
 }
+__device__ __forceinline__ int ld_acquire(const int* p) {
+  int v;
+  asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+  return v;
+}
+__device__ __forceinline__ void st_release(int* p, int v) {
+  asm volatile("st.release.gpu.global.s32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+
+// The pieces of one worker (see WarpSched), in the order in which it runs them.
+struct WorkList {
+  int c0, o0, c1, o1;     // first chain and first tile in it; last chain and one past the last tile in it
+  int head, wf, nwhole;   // 1: the leading part of chain c1 is a piece of its own; first whole chain; whole chains
+  int count;              // pieces
+};
+__device__ __forceinline__ WorkList make_worklist(const WarpSched& sc, int worker) {
+  WorkList w{};
+  const long long total = (long long)sc.chains * sc.tiles;
+  const long long lo = (long long)worker * sc.quota;
+  if (worker >= sc.workers || lo >= total) return w;   // count = 0
+  long long hi = lo + sc.quota;
+  if (hi > total) hi = total;
+  w.c0 = (int)(lo / sc.tiles);
+  w.o0 = (int)(lo - (long long)w.c0 * sc.tiles);
+  w.c1 = (int)((hi - 1) / sc.tiles);
+  w.o1 = (int)(hi - (long long)w.c1 * sc.tiles);
+  if (w.c0 == w.c1) {
+    w.count = 1;
+    return w;
+  }
+  w.head = w.o1 < sc.tiles ? 1 : 0;
+  const int tail = w.o0 > 0 ? 1 : 0;
+  w.wf = w.c0 + tail;
+  w.nwhole = (w.c1 - w.head) - w.wf + 1;
+  w.count = w.head + w.nwhole + tail;
+  return w;
+}
+// piece i of the list: tiles [from, to) of `chain`
+__device__ __forceinline__ void get_piece(const WorkList& w, int tiles, int i, int& chain, int& from, int& to) {
+  if (w.c0 == w.c1) {
+    chain = w.c0; from = w.o0; to = w.o1;
+  } else if (i < w.head) {
+    chain = w.c1; from = 0; to = w.o1;
+  } else if (i - w.head < w.nwhole) {
+    chain = w.wf + i - w.head; from = 0; to = tiles;
+  } else {
+    chain = w.c0; from = w.o0; to = tiles;
+  }
+}
+// Waits (lane 0 polls, bounded) until the worker that runs the earlier part of the chain has published it.
+// Returns false to the whole warp when the wait gave up or another worker raised the abort word.
+__device__ __forceinline__ bool wait_handoff(const WarpSched& sc, int worker, int lane) {
+  int ok = 1;
+  if (lane == 0) {
+    int spins = 0;
+    while (ld_acquire(sc.flags + worker) == 0) {
+      __nanosleep(64);
+      if (++spins > sc.spin_limit || ld_acquire(sc.abort) != 0) {
+        atomicExch(sc.abort, 1);
+        ok = 0;
+        break;
+      }
+    }
+  }
+  ok = __shfl_sync(0xffffffffu, ok, 0);
+  return ok != 0;
+}
+// Publishes the hand-off of the chain part this worker just finished (all lanes have written their vectors).
+__device__ __forceinline__ void publish_handoff(const WarpSched& sc, int worker, int lane) {
+  __threadfence();
+  __syncwarp();
+  if (lane == 0 && !sc.withhold) st_release(sc.flags + worker + 1, 1);
+}
+
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 __device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_group 0;" ::: "memory"); }
 

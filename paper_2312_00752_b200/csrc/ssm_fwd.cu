@@ -17,7 +17,7 @@ namespace ssm {
 
 // threads per block: 16 thread groups for N = 16, 32 groups otherwise (keeps the staged tiles below 48 KB)
 __host__ __device__ constexpr int fwd_threads(int N) { return N == 16 ? 64 : 32; }
-constexpr int kFwdTile = 32;  // time steps staged in shared memory at a time; divides kCkptSteps
+constexpr int kFwdTile = 32;  // time steps staged in shared memory at a time
 
 template <typename IO, int N, int CPT, int MODE>
 __global__ void __launch_bounds__(fwd_threads(N)) ssm_fwd_kernel(const FwdParams p) {
@@ -106,22 +106,23 @@ __global__ void __launch_bounds__(fwd_threads(N)) ssm_fwd_kernel(const FwdParams
       s_B[tt][n] = (ok && !p.static_B) ? io_to_float<IO>(gB[g]) : 0.f;
       if constexpr (kReadout) s_C[tt][n] = (ok && !p.static_C) ? io_to_float<IO>(gC[g]) : 0.f;
     }
-    if (MODE != kFwdSummary && p.ckpt != nullptr && (t0 % kCkptSteps) == 0) {
-      const int kc = t0 / kCkptSteps;
-#pragma unroll
-      for (int q = 0; q < CPT; ++q) {
-        const int d = d_thr + q;
-        if (d < D) {
-          float* dst = p.ckpt + (((size_t)b * p.nck + kc) * D + d) * N + j * S;
-#pragma unroll
-          for (int k = 0; k < S; ++k) dst[k] = h[q][k];
-        }
-      }
-    }
     __syncthreads();
 
 #pragma unroll 2
     for (int tt = 0; tt < nt; ++tt) {
+      if (MODE != kFwdSummary && p.ckpt != nullptr && ((t0 + tt) % kCkptSteps) == 0) {
+        // the state before this step starts a checkpoint block
+        const int kc = (t0 + tt) / kCkptSteps;
+#pragma unroll
+        for (int q = 0; q < CPT; ++q) {
+          const int d = d_thr + q;
+          if (d < D) {
+            float* dst = p.ckpt + (((size_t)b * p.nck + kc) * D + d) * N + j * S;
+#pragma unroll
+            for (int k = 0; k < S; ++k) dst[k] = h[q][k];
+          }
+        }
+      }
       float Bv[S], Cv[S];
 #pragma unroll
       for (int k = 0; k < S; ++k) {

@@ -66,6 +66,33 @@ def oracle_fwd_bwd(inp: dict, nthreads=0):
     return res
 
 
+def elementwise_excess(got, ref, io: str) -> float:
+    """Largest |got - ref| in units of what a correctly rounded result of this size may be off by: a few units in the last
+    place of the element itself (bf16: 2^-8 relative, f32: 2^-22) plus a floor tied to the rms of the tensor (sums of many
+    terms cancel, so an element far below the rms carries the rounding of its larger terms).  The tolerances of the benchmark spec
+    statement are relative to the largest element of a tensor, so a wrong value on a few small elements would pass them;
+    this measure is per element.  A value of 1 means "at the bound"."""
+    got = np.asarray(got, dtype=np.float64)
+    ref = np.asarray(ref, dtype=np.float64)
+    ulp = 2.0 ** -8 if io == "bf16" else 2.0 ** -22
+    rms = float(np.sqrt(np.mean(ref * ref)))
+    bound = 4.0 * ulp * np.abs(ref) + 8.0 * ulp * rms
+    if rms == 0.0:
+        return float(np.abs(got).max())
+    return float((np.abs(got - ref) / bound).max())
+
+
+def assert_elementwise(got: dict, ref: dict, io: str, what="", keys=("out", "dx", "ddelta", "dz", "dB", "dC")):
+    bad = {}
+    for k in keys:
+        if got.get(k) is None or k not in ref:
+            continue
+        e = elementwise_excess(got[k], ref[k], io)
+        if not e <= 1.0:
+            bad[k] = e
+    assert not bad, f"{what}: elements beyond their own rounding bound (in units of the bound): {bad}"
+
+
 def assert_parity(got: dict, ref: dict, io: str, what=""):
     errs = {}
     for k, r in ref.items():

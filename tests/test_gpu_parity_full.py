@@ -20,6 +20,7 @@ def test_layer_shapes_every_element(idx):
     got = U.gpu_fwd_bwd(U.to_device(inp, cfg.io))
     ref = U.oracle_fwd_bwd(inp)
     errs = U.assert_parity(got, ref, cfg.io, cfg.name)
+    U.assert_elementwise(got, ref, cfg.io, cfg.name)
     print(cfg.name, {k: f"{v:.2e}" for k, v in errs.items()})
 
 
@@ -37,6 +38,37 @@ def test_long_sequence_shortened_every_element():
     got = U.gpu_fwd_bwd(U.to_device(inp, cfg.io))
     errs = U.assert_parity(got, U.oracle_fwd_bwd(inp), cfg.io, "config 4 shortened")
     print({k: f"{v:.2e}" for k, v in errs.items()})
+
+
+def test_long_sequence_full_length_every_element():
+    """The long-sequence workload at its full length (524288 steps) on 128 channels: still split in time in both
+    directions, and cheap enough for the oracle that every element of all eight outputs is compared, the channel-summed
+    dB and dC included."""
+    from paper_2312_00752_b200 import binding as K
+    cfg = synth.CONFIGS[4].scaled(D=128)
+    inp = synth.make_inputs(cfg, seed=0)
+    dev = U.to_device(inp, cfg.io)
+    prob = K.make_problem(dev["x"], dev["B"], True, True)
+    assert K.plan(prob)["n_segments"] > 1
+    got = U.gpu_fwd_bwd(dev)
+    ref = U.oracle_fwd_bwd(inp)
+    errs = U.assert_parity(got, ref, cfg.io, "config 4 at full length, 128 channels")
+    assert set(errs) == {"out", "dx", "ddelta", "dz", "dB", "dC", "dA", "dD"}
+    U.assert_elementwise(got, ref, cfg.io, "config 4 at full length, 128 channels")
+    print({k: f"{v:.2e}" for k, v in errs.items()})
+
+
+@pytest.mark.parametrize("N", [16, 1])
+def test_fp32_long_memory(N):
+    """fp32 io where the state remembers thousands of steps (step sizes log-uniform in [1e-4, 1e-2], 65536 steps): a
+    relative error eps in the decay costs about eps / (delta |A|) in the state, so this is where an inexact
+    exponential would show against the fp32 tolerances (1e-5 on out, 1e-4 on the gradients)."""
+    cfg = synth.ScanConfig("fp32 long memory", 12, 1, 65536, 64, N, "f32", 1e-4, 1e-2)
+    inp = synth.make_inputs(cfg, seed=3)
+    got = U.gpu_fwd_bwd(U.to_device(inp, "f32"))
+    ref = U.oracle_fwd_bwd(inp)
+    errs = U.assert_parity(got, ref, "f32", cfg.name)
+    print(N, {k: f"{v:.2e}" for k, v in errs.items()})
 
 
 def test_long_sequence_full_size():

@@ -31,12 +31,14 @@ def _prob(batch=2, L=100, D=64, N=16, io=K.SSM_BF16, flags=3):
 
 def test_queries_and_plan():
     ck = K.checkpoint_steps()
-    assert ck in (16, 32, 64)
+    assert ck in (8, 16, 32, 64)
     p = _prob(4, 2048, 5120)
     assert K.saved_state_bytes(p) == 4 * (2048 // ck) * 5120 * 16 * 4
     pl = K.plan(p)
-    assert pl["n_segments"] == 1 and pl["segment_steps"] == 2048 and pl["states_per_thread"] == 4
-    assert K.fwd_workspace_bytes(p) == 0
+    assert pl["n_segments"] == 1 and pl["segment_steps"] == 2048 and pl["states_per_thread"] in (4, 8, 16)
+    # 640 groups of 32 channels for 592 resident warps: some groups are shared by two warps, which needs hand-off slots
+    assert 0 < K.fwd_workspace_bytes(p) < 4 << 20
+    assert K.fwd_workspace_bytes(_prob(64, 256, 64)) == 0 and K.fwd_workspace_bytes(_prob(2, 100, 64, io=K.SSM_F32)) == 0
     assert K.bwd_workspace_bytes(p) > 0
     long = _prob(1, 524288, 1536)
     pl = K.plan(long)

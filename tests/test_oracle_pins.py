@@ -70,6 +70,26 @@ def test_matrix_form(L, N):
 
 
 # --------------------------------------------------------------------------------------------------------------
+# Gate (Section 3.4, Figure 3: the SiLU branch multiplies the SSM output): the gated output equals the pre-gate readout
+# times z * sigmoid(z), with the sigmoid taken from a library (scipy's expit) rather than retyped; and, for the
+# backward pass, dz equals dout * s * d/dz [z expit(z)] with the derivative of the library function taken by complex-step
+# free central differences of expit itself.
+def test_gate_is_library_silu():
+    from scipy.special import expit
+    p = _rand_problem(2, 40, 6, 4)
+    p["z"] = p["z"] * 4.0     # reach both saturated ends of the sigmoid
+    out, s_pre = O.scan_fwd(p["x"], p["delta"], p["A"], p["B"], p["C"], D_skip=p["D_skip"], z=p["z"], return_pregate=True)
+    ungated = O.scan_fwd(p["x"], p["delta"], p["A"], p["B"], p["C"], D_skip=p["D_skip"], z=None)
+    np.testing.assert_allclose(s_pre, ungated, rtol=0, atol=0)
+    np.testing.assert_allclose(out, s_pre * p["z"] * expit(p["z"]), rtol=1e-14, atol=1e-15)
+    dout = RNG.standard_normal(out.shape)
+    g = O.scan_bwd(p["x"], p["delta"], p["A"], p["B"], p["C"], p["D_skip"], p["z"], dout)
+    sig = expit(p["z"])
+    dsilu = sig + p["z"] * sig * expit(-p["z"])     # d/dz [z expit(z)], expit'(z) = expit(z) expit(-z)
+    np.testing.assert_allclose(g["dz"], dout * s_pre * dsilu, rtol=1e-12, atol=1e-13)
+
+
+# --------------------------------------------------------------------------------------------------------------
 # P3  A = 0 makes Abar = 1, so the state is a plain running sum: h_t = cumsum(delta * B * x).
 def test_zero_A_is_cumsum():
     batch, L, D, N = 2, 50, 4, 3
