@@ -9,6 +9,8 @@ namespace ssm {
 int fwd_channels_per_block(int N);
 int bwd_channels_per_block(int N);
 int fwd_states_per_thread();
+int bwd_fast_channels_per_warp();
+bool bwd_fast_applicable(const ssm_problem_t& prob, const BwdParams& p);
 size_t fwd_handoff_bytes_per_worker();
 size_t bwd_handoff_bytes_per_worker();
 
@@ -17,8 +19,8 @@ static bool tuned_shape(const ssm_problem_t& p) {
   return p.io_dtype == SSM_BF16 && p.N == 16 && p.D % 8 == 0 && !(p.flags & (SSM_FLAG_STATIC_B | SSM_FLAG_STATIC_C));
 }
 // Workers the hand-off slots of a workspace allow for `chains` chains of 32 channels: none while every chain can have
-// a warp of its own in the first round (one warp per SM sub-partition), else up to 8 resident warps per SM.
-constexpr int kMaxWarpsPerSM = 8;
+// a warp of its own in the first round (one warp per SM sub-partition), else up to 12 resident warps per SM.
+constexpr int kMaxWarpsPerSM = 12;
 static int shared_workers(long long chains) {
   if (chains <= 4LL * kNumSMs) return 0;
   return (int)std::min<long long>(chains, (long long)kMaxWarpsPerSM * kNumSMs);
@@ -81,6 +83,11 @@ Plan make_plan(const ssm_problem_t& p) {
 // states do not depend on the split, so forward and backward may disagree about it.
 Plan make_bwd_plan(const ssm_problem_t& p) {
   Plan pl = make_plan(p);
+  if (tuned_shape(p)) {
+    // the tuned kernel's chains (and the channel groups of its dB / dC partial sums) are narrower than the generic ones
+    pl.bwd_ch = bwd_fast_channels_per_warp();
+    pl.bwd_groups = (p.D + pl.bwd_ch - 1) / pl.bwd_ch;
+  }
   const long long chains = (long long)p.batch * pl.bwd_groups;
   const long long resident = 4LL * kNumSMs;
   int nseg = 1;
@@ -522,6 +529,8 @@ static ssm_status_t bwd_impl(const ssm_problem_t* p, const void* x, const void* 
     if (launch_carry(cp, s) != cudaSuccess) return SSM_ERR_CUDA;
     bp.mu_in = cp.carried;
   }
+  // the generic kernel (taken when a pointer is not 16-byte aligned) writes one partial sum per 32 channels
+  if (!bwd_fast_applicable(*p, bp)) bp.groups = (p->D + bwd_channels_per_block(p->N) - 1) / bwd_channels_per_block(p->N);
   if (launch_bwd(*p, pl, bp, kBwdFull, s) != cudaSuccess) return SSM_ERR_CUDA;
 
   ReduceParams rp{};
@@ -539,7 +548,7 @@ static ssm_status_t bwd_impl(const ssm_problem_t* p, const void* x, const void* 
   rp.dbias_part = bp.dbias_part;
   rp.dbias = ddelta_bias;
   rp.bln = (long long)p->batch * p->L * p->N;
-  rp.groups = pl.bwd_groups;
+  rp.groups = bp.groups;
   rp.parts = p->batch * pl.nseg;
   rp.D = p->D;
   rp.N = p->N;

@@ -291,7 +291,8 @@ __global__ void __launch_bounds__(BwdGeom<N>::THREADS) ssm_bwd_local_kernel(cons
   const IO* __restrict__ gC = static_cast<const IO*>(p.C);
   const int tid = threadIdx.x;
   const int j = tid % LPC, slot = tid / LPC;
-  const int d_cta = blockIdx.x * CH, seg = blockIdx.y, b = blockIdx.z;
+  // (segment 0 has no earlier segment to hand its adjoint to: it is not computed)
+  const int d_cta = blockIdx.x * CH, seg = blockIdx.y + 1, b = blockIdx.z;
   const int D = p.D, d = d_cta + slot;
   const bool valid = d < D;
   const int t_begin = seg * p.seg_steps;
@@ -393,6 +394,8 @@ static cudaError_t launch_bwd_n(const Plan& plan, const BwdParams& p, int mode, 
   dim3 grid((p.D + G::CH - 1) / G::CH, plan.nseg, p.batch);
   constexpr int kBwdThreads = G::THREADS;
   if (mode == kBwdLocal) {
+    if (plan.nseg < 2) return cudaSuccess;
+    grid.y = plan.nseg - 1;
     ssm_bwd_local_kernel<IO, N><<<grid, kBwdThreads, 0, s>>>(p);
     return cudaGetLastError();
   }

@@ -47,7 +47,7 @@ __global__ void __launch_bounds__(kThreads) ssm_bwd_local_fast_kernel(const BwdP
   const int tid = threadIdx.x;
   const int lane = tid & 31, warp = tid >> 5;
   const int d_cta = blockIdx.x * kCH;
-  const int seg = blockIdx.y;
+  const int seg = blockIdx.y + 1;   // segment 0 has no earlier segment to hand its adjoint to: it is not computed
   const int b = blockIdx.z;
   const int D = p.D;
   const int t_begin = seg * p.seg_steps;
@@ -243,7 +243,8 @@ bool bwd_local_fast_applicable(const ssm_problem_t& prob, const BwdParams& p) {
 }
 
 cudaError_t launch_bwd_local_fast(const Plan& plan, const BwdParams& p, cudaStream_t s) {
-  dim3 grid((p.D + kCH - 1) / kCH, plan.nseg, p.batch);
+  if (plan.nseg < 2) return cudaSuccess;
+  dim3 grid((p.D + kCH - 1) / kCH, plan.nseg - 1, p.batch);
   if (p.softplus || p.delta_bias != nullptr) ssm_bwd_local_fast_kernel<true><<<grid, kThreads, 0, s>>>(p);
   else ssm_bwd_local_fast_kernel<false><<<grid, kThreads, 0, s>>>(p);
   return cudaGetLastError();

@@ -1,11 +1,15 @@
 // Backward selective scan, tuned path: bf16 io, N = 16, D % 8 == 0, 16-byte aligned pointers.
 // Same mathematics as ssm_bwd.cu (adjoint of Eq. 2a/2b with skip term and gate; states recomputed, Section 3.3).
 //
-// One warp is one worker, as in the tuned forward kernel (ssm_fwd_warp.cu): it owns 32 adjacent channels of one batch
-// entry, walks its part of the sequence backwards in tiles of 16 steps, stages its own tiles with cp.async and shares
-// nothing with the other warps of its block.  A thread holds 16 recurrences as packed float2 pairs: S states of
-// CPT = 16 / S channels; local channel q of lane j (j = lane % LPC, LPC = 16 / S) is channel j ^ q of its lane group, so
-// the sums over n are exchanged with xor-shuffles and every lane finishes exactly one channel per step (channel `lane`).
+// One warp is one worker, as in the tuned forward kernel (ssm_fwd_warp.cu): it owns CW adjacent channels of one batch
+// entry, walks its part of the sequence backwards in tiles of 8 steps, stages its own tiles with cp.async and shares
+// nothing with the other warps of its block.  A thread holds S states of CPT channels as packed float2 pairs; the
+// LPC = 16 / S lanes of a group cover the 16 states of the group's channels.  With CPT = LPC (16 recurrences per thread,
+// CW = 32) local channel q of lane j (j = lane % LPC) is channel j ^ q of the group, so the sums over n are
+// reduce-scattered with xor-shuffles and every lane finishes exactly one channel per step (channel `lane`).  With
+// S = 8, CPT = 1 (8 recurrences per thread, CW = 16) the two lanes of a group share one channel, the sums are completed
+// in both, and lane j finishes the steps of parity j; this mapping needs half the registers, so twice as many warps are
+// resident, and a problem has twice as many chains to give them.
 //
 // Recomputation.  The forward pass left the state at the start of every block of 8 steps, so a sub-block of 8 steps is
 // rebuilt directly from its checkpoint: a forward sweep keeps the states after the odd steps in registers (64
@@ -35,28 +39,30 @@ constexpr int kBT = 8;             // steps per tile (one sub-block: 8 warps per
 constexpr int kSB = kCkptSteps;    // steps per sub-block = checkpoint spacing
 constexpr int kRB = 4;             // steps between two dB / dC transposes
 constexpr int kBwdWarps = 4;       // warps per block
+constexpr int kBwdFastChannels = 32;   // channels per warp of the mapping the launcher picks
 constexpr int kBwdHandoffVec = 9;  // float4 per lane: mu (4), dA (4), dD and dbias (1)
 constexpr float kInvLog2e = 0.6931471805599453f;
 static_assert(kSB == 8 && kBT % kSB == 0, "sub-blocks of 8 steps, whole sub-blocks per tile");
 
-template <int S, bool SP>
+template <int S, int CPT, bool SP>
 struct BwdWarpSmem {
-  uint32_t x[2][kBT][16];    // bf16 pairs, 32 channels
-  uint32_t d[2][kBT][16];
-  uint32_t z[2][kBT][16];
-  uint32_t g[2][kBT][16];
-  uint32_t rB[2][kBT][8];    // bf16 pairs, 16 states
+  static constexpr int CW = (32 / (16 / S)) * CPT;   // channels per warp
+  uint32_t x[2][kBT][CW / 2];    // bf16 pairs
+  uint32_t d[2][kBT][CW / 2];
+  uint32_t z[2][kBT][CW / 2];
+  uint32_t g[2][kBT][CW / 2];
+  uint32_t rB[2][kBT][8];        // bf16 pairs, 16 states
   uint32_t rC[2][kBT][8];
-  float4 ck[2][kBT / kSB][4][32];   // checkpoint states: [sub-block][float4 of the thread][lane]
-  float fB[kBT][16];         // B and C of the tile widened to float
+  float4 ck[2][kBT / kSB][CPT * S / 4][32];   // checkpoint states: [sub-block][float4 of the thread][lane]
+  float fB[kBT][16];             // B and C of the tile widened to float
   float fC[kBT][16];
-  float ds[kBT][32];         // dout * silu(z)
-  float gp[kBT][32];         // dout * silu'(z)
-  float dF[SP ? kBT : 1][32];   // SP: step sizes after bias and softplus
-  uint32_t ox[kBT][16];      // dx, ddelta, dz of the tile (bf16 pairs)
-  uint32_t od[kBT][16];
-  uint32_t oz[kBT][16];
-  float4 red[kRB][32][S / 2];   // dB / dC terms of 4 steps: [step][lane][dB float4s | dC float4s], swizzled
+  float ds[kBT][CW];             // dout * silu(z)
+  float gp[kBT][CW];             // dout * silu'(z)
+  float dF[SP ? kBT : 1][CW];    // SP: step sizes after bias and softplus
+  uint32_t ox[kBT][CW / 2];      // dx, ddelta, dz of the tile (bf16 pairs)
+  uint32_t od[kBT][CW / 2];
+  uint32_t oz[kBT][CW / 2];
+  float4 red[kRB][32][S / 2];    // dB / dC terms of 4 steps: [step][lane][dB float4s | dC float4s], swizzled
 };
 
 #ifdef SSM_DEBUG_BOUNDS
@@ -66,18 +72,24 @@ struct BwdWarpSmem {
 #define SSM_BROW(r, abort_ptr) (r)
 #endif
 
-template <int S>
+template <int S, int CPT_>
 struct Lane {
-  static constexpr int LPC = 16 / S, CPT = LPC, H = S / 2, V = S / 2;   // V: float4 of dB / dC terms per thread and step
-  int lane, j, g;
+  static constexpr int LPC = 16 / S, CPT = CPT_, H = S / 2, V = S / 2;   // V: float4 of dB / dC terms per thread and step
+  static constexpr int CW = (32 / LPC) * CPT;       // channels per warp
+  static constexpr bool OWN = (CPT == LPC);          // every lane finishes its own channel (else: parity of the step)
+  static_assert(OWN || (CPT == 1 && LPC == 2), "supported mappings");
+  int lane, j, g, co;    // co: the channel (within the warp) this lane finishes
   uint32_t sel0, sel1;
   __device__ __forceinline__ explicit Lane(int l) : lane(l), j(l % LPC), g(l / LPC) {
+    co = OWN ? lane : g;
     sel0 = (j & 1) ? 0x3244u : 0x1044u;
     sel1 = (j & 1) ? 0x1044u : 0x3244u;
   }
-  // the CPT values of a tile row (32 channels as 16 bf16 pairs) that belong to this thread, by local channel
+  // the CPT values of a tile row (CW channels as bf16 pairs) that belong to this thread, by local channel
   __device__ __forceinline__ void unpack_row(const uint32_t* row, float (&v)[CPT]) const {
-    if constexpr (CPT == 1) {
+    if constexpr (!OWN) {
+      v[0] = __uint_as_float((uint32_t)reinterpret_cast<const uint16_t*>(row)[g] << 16);
+    } else if constexpr (CPT == 1) {
       v[0] = __uint_as_float((uint32_t)reinterpret_cast<const uint16_t*>(row)[lane] << 16);
     } else if constexpr (CPT == 2) {
       const uint32_t w = row[g];
@@ -92,9 +104,11 @@ struct Lane {
       v[3] = bf16sel(wb, sel1);
     }
   }
-  // the same from a row of 32 floats
+  // the same from a row of CW floats
   __device__ __forceinline__ void pick_row(const float* row, float (&v)[CPT]) const {
-    if constexpr (CPT == 1) {
+    if constexpr (!OWN) {
+      v[0] = row[g];
+    } else if constexpr (CPT == 1) {
       v[0] = row[lane];
     } else if constexpr (CPT == 2) {
       const float2 f = *reinterpret_cast<const float2*>(row + 2 * g);
@@ -167,9 +181,9 @@ __device__ __forceinline__ void decays(float dt, const float2 (&A2)[H], float a0
 }
 
 // Per-thread state that lives along a chain
-template <int S>
+template <int S, int CPT>
 struct ChainRegs {
-  static constexpr int CPT = 16 / S, H = S / 2;
+  static constexpr int H = S / 2;
   float2 A2[CPT][H];    // A * log2(e)
   float a0s[CPT], rs[CPT];
   float2 mu[CPT][H];    // adjoint flowing backwards in time
@@ -178,13 +192,15 @@ struct ChainRegs {
 };
 
 // One sub-block of 8 steps: rows [r0, r0 + 8) of the tile; nlive = rows of the tile inside the segment.
-template <int S, bool SP, bool AP>
-__device__ __forceinline__ void sub_block(const Lane<S>& ln, ChainRegs<S>& cr, int r0, int nlive, float gate_on,
+template <int S, int CPT, bool SP, bool AP>
+__device__ __forceinline__ void sub_block(const Lane<S, CPT>& ln, ChainRegs<S, CPT>& cr, int r0, int nlive, float gate_on,
                                           bool softplus, const uint32_t* tx, const uint32_t* td, const float* tfB,
                                           const float* tfC, const float* tds, const float* tgp, const float* tdF,
                                           const float4* tck, uint32_t* tox, uint32_t* tod, uint32_t* toz, float4* tred,
                                           float* part_dB, float* part_dC, int* abort_word) {
-  constexpr int LPC = Lane<S>::LPC, CPT = Lane<S>::CPT, H = Lane<S>::H, V = Lane<S>::V;
+  using LN = Lane<S, CPT>;
+  constexpr int LPC = LN::LPC, H = LN::H, V = LN::V, CW = LN::CW, WPR = CW / 2;
+  constexpr bool OWN = LN::OWN;
   const int lane = ln.lane;
   // ---- forward sweep from the checkpoint: the states after the odd steps stay in registers
   float2 hist[kSB / 2][CPT][H];
@@ -202,9 +218,9 @@ __device__ __forceinline__ void sub_block(const Lane<S>& ln, ChainRegs<S>& cr, i
 #pragma unroll
     for (int t = 0; t < kSB; ++t) {
       const int r = SSM_BROW(r0 + t, abort_word);
-      if constexpr (SP) ln.pick_row(tdF + r * 32, dt[t]);
-      else ln.unpack_row(td + r * 16, dt[t]);
-      ln.unpack_row(tx + r * 16, u[t]);
+      if constexpr (SP) ln.pick_row(tdF + r * CW, dt[t]);
+      else ln.unpack_row(td + r * WPR, dt[t]);
+      ln.unpack_row(tx + r * WPR, u[t]);
     }
 #pragma unroll
     for (int t = 0; t < kSB; ++t) {
@@ -230,13 +246,13 @@ __device__ __forceinline__ void sub_block(const Lane<S>& ln, ChainRegs<S>& cr, i
     // ======== odd step t1 = 2m + 1: its state is hist[m]; its w = mu h_{t-1} waits for the even step's state
     const int r1 = SSM_BROW(r0 + 2 * m + 1, abort_word);
     float dt1[CPT], u1[CPT], ds1[CPT];
-    if constexpr (SP) ln.pick_row(tdF + r1 * 32, dt1);
-    else ln.unpack_row(td + r1 * 16, dt1);
-    ln.unpack_row(tx + r1 * 16, u1);
-    ln.pick_row(tds + r1 * 32, ds1);
-    const float gp1 = tgp[r1 * 32 + lane];
+    if constexpr (SP) ln.pick_row(tdF + r1 * CW, dt1);
+    else ln.unpack_row(td + r1 * WPR, dt1);
+    ln.unpack_row(tx + r1 * WPR, u1);
+    ln.pick_row(tds + r1 * CW, ds1);
+    const float gp1 = tgp[r1 * CW + ln.co];
     float raw1 = 0.f;
-    if constexpr (SP) raw1 = __uint_as_float((uint32_t)reinterpret_cast<const uint16_t*>(td + r1 * 16)[lane] << 16);
+    if constexpr (SP) raw1 = __uint_as_float((uint32_t)reinterpret_cast<const uint16_t*>(td + r1 * WPR)[ln.co] << 16);
     float y1[CPT], lb1[CPT];
     {
       float2 Bv[H], Cv[H];
@@ -276,29 +292,31 @@ __device__ __forceinline__ void sub_block(const Lane<S>& ln, ChainRegs<S>& cr, i
         rrow[(V / 2 + v) ^ swz] = make_float4(dCt[2 * v].x, dCt[2 * v].y, dCt[2 * v + 1].x, dCt[2 * v + 1].y);
       }
     }
+    if constexpr (OWN) {
 #pragma unroll
-    for (int mm = 1; mm < LPC; mm <<= 1) {
+      for (int mm = 1; mm < LPC; mm <<= 1) {
 #pragma unroll
-      for (int q = 0; q < CPT; ++q)
-        if ((q & (2 * mm - 1)) == 0) {
-          y1[q] += __shfl_xor_sync(0xffffffffu, y1[q + mm], mm);
-          lb1[q] += __shfl_xor_sync(0xffffffffu, lb1[q + mm], mm);
-        }
+        for (int q = 0; q < CPT; ++q)
+          if ((q & (2 * mm - 1)) == 0) {
+            y1[q] += __shfl_xor_sync(0xffffffffu, y1[q + mm], mm);
+            lb1[q] += __shfl_xor_sync(0xffffffffu, lb1[q + mm], mm);
+          }
+      }
+    } else {
+      y1[0] += __shfl_xor_sync(0xffffffffu, y1[0], 1);
+      lb1[0] += __shfl_xor_sync(0xffffffffu, lb1[0], 1);
     }
-    const float dz1 = gp1 * fmaf(cr.Dk, u1[0], y1[0]);
-    const float dx1 = fmaf(dt1[0], lb1[0], ds1[0] * cr.Dk);
-    cr.dD = fmaf(ds1[0], u1[0], cr.dD);
 
     // ======== even step t0 = 2m: its state is rebuilt from the one before it
     const int r0e = SSM_BROW(r0 + 2 * m, abort_word);
     float dt0[CPT], u0[CPT], ds0[CPT];
-    if constexpr (SP) ln.pick_row(tdF + r0e * 32, dt0);
-    else ln.unpack_row(td + r0e * 16, dt0);
-    ln.unpack_row(tx + r0e * 16, u0);
-    ln.pick_row(tds + r0e * 32, ds0);
-    const float gp0 = tgp[r0e * 32 + lane];
+    if constexpr (SP) ln.pick_row(tdF + r0e * CW, dt0);
+    else ln.unpack_row(td + r0e * WPR, dt0);
+    ln.unpack_row(tx + r0e * WPR, u0);
+    ln.pick_row(tds + r0e * CW, ds0);
+    const float gp0 = tgp[r0e * CW + ln.co];
     float raw0 = 0.f;
-    if constexpr (SP) raw0 = __uint_as_float((uint32_t)reinterpret_cast<const uint16_t*>(td + r0e * 16)[lane] << 16);
+    if constexpr (SP) raw0 = __uint_as_float((uint32_t)reinterpret_cast<const uint16_t*>(td + r0e * WPR)[ln.co] << 16);
     float y0[CPT], lb0[CPT], wa0[CPT], wa1[CPT];
     {
       float2 Bv[H], Cv[H];
@@ -352,38 +370,65 @@ __device__ __forceinline__ void sub_block(const Lane<S>& ln, ChainRegs<S>& cr, i
         rrow[(V / 2 + v) ^ swz] = make_float4(dCt[2 * v].x, dCt[2 * v].y, dCt[2 * v + 1].x, dCt[2 * v + 1].y);
       }
     }
+    if constexpr (OWN) {
 #pragma unroll
-    for (int mm = 1; mm < LPC; mm <<= 1) {
+      for (int mm = 1; mm < LPC; mm <<= 1) {
 #pragma unroll
-      for (int q = 0; q < CPT; ++q)
-        if ((q & (2 * mm - 1)) == 0) {
-          y0[q] += __shfl_xor_sync(0xffffffffu, y0[q + mm], mm);
-          lb0[q] += __shfl_xor_sync(0xffffffffu, lb0[q + mm], mm);
-          wa0[q] += __shfl_xor_sync(0xffffffffu, wa0[q + mm], mm);
-          wa1[q] += __shfl_xor_sync(0xffffffffu, wa1[q + mm], mm);
-        }
-    }
-    // ---- finish both steps of the pair for this lane's own channel
-    const float dz0 = gp0 * fmaf(cr.Dk, u0[0], y0[0]);
-    const float dx0 = fmaf(dt0[0], lb0[0], ds0[0] * cr.Dk);
-    cr.dD = fmaf(ds0[0], u0[0], cr.dD);
-    float dd1 = fmaf(u1[0], lb1[0], wa1[0] * kInvLog2e);
-    float dd0 = fmaf(u0[0], lb0[0], wa0[0] * kInvLog2e);
-    if constexpr (SP) {
-      // the gradient goes to the pre-activation v: d softplus(v) / dv = sigmoid(v); the bias gets the sum over time
-      if (softplus) {
-        dd1 *= sigmoid_fast(raw1 + cr.bias_own);
-        dd0 *= sigmoid_fast(raw0 + cr.bias_own);
+        for (int q = 0; q < CPT; ++q)
+          if ((q & (2 * mm - 1)) == 0) {
+            y0[q] += __shfl_xor_sync(0xffffffffu, y0[q + mm], mm);
+            lb0[q] += __shfl_xor_sync(0xffffffffu, lb0[q + mm], mm);
+            wa0[q] += __shfl_xor_sync(0xffffffffu, wa0[q + mm], mm);
+            wa1[q] += __shfl_xor_sync(0xffffffffu, wa1[q + mm], mm);
+          }
       }
-      if (r0 + 2 * m + 1 < nlive) cr.dbias += dd1;
-      if (r0 + 2 * m < nlive) cr.dbias += dd0;
+      // ---- finish both steps of the pair for this lane's own channel
+      const float dz1 = gp1 * fmaf(cr.Dk, u1[0], y1[0]);
+      const float dx1 = fmaf(dt1[0], lb1[0], ds1[0] * cr.Dk);
+      const float dz0 = gp0 * fmaf(cr.Dk, u0[0], y0[0]);
+      const float dx0 = fmaf(dt0[0], lb0[0], ds0[0] * cr.Dk);
+      cr.dD = fmaf(ds1[0], u1[0], cr.dD);
+      cr.dD = fmaf(ds0[0], u0[0], cr.dD);
+      float dd1 = fmaf(u1[0], lb1[0], wa1[0] * kInvLog2e);
+      float dd0 = fmaf(u0[0], lb0[0], wa0[0] * kInvLog2e);
+      if constexpr (SP) {
+        // the gradient goes to the pre-activation v: d softplus(v) / dv = sigmoid(v); the bias gets the sum over time
+        if (softplus) {
+          dd1 *= sigmoid_fast(raw1 + cr.bias_own);
+          dd0 *= sigmoid_fast(raw0 + cr.bias_own);
+        }
+        if (r0 + 2 * m + 1 < nlive) cr.dbias += dd1;
+        if (r0 + 2 * m < nlive) cr.dbias += dd0;
+      }
+      reinterpret_cast<__nv_bfloat16*>(tox + r1 * WPR)[lane] = __float2bfloat16_rn(dx1);
+      reinterpret_cast<__nv_bfloat16*>(tod + r1 * WPR)[lane] = __float2bfloat16_rn(dd1);
+      reinterpret_cast<__nv_bfloat16*>(toz + r1 * WPR)[lane] = __float2bfloat16_rn(dz1 * gate_on);
+      reinterpret_cast<__nv_bfloat16*>(tox + r0e * WPR)[lane] = __float2bfloat16_rn(dx0);
+      reinterpret_cast<__nv_bfloat16*>(tod + r0e * WPR)[lane] = __float2bfloat16_rn(dd0);
+      reinterpret_cast<__nv_bfloat16*>(toz + r0e * WPR)[lane] = __float2bfloat16_rn(dz0 * gate_on);
+    } else {
+      // both lanes of the group complete the sums; lane 1 finishes the odd step of the pair, lane 0 the even one
+      y0[0] += __shfl_xor_sync(0xffffffffu, y0[0], 1);
+      lb0[0] += __shfl_xor_sync(0xffffffffu, lb0[0], 1);
+      wa0[0] += __shfl_xor_sync(0xffffffffu, wa0[0], 1);
+      wa1[0] += __shfl_xor_sync(0xffffffffu, wa1[0], 1);
+      const bool odd = ln.j != 0;
+      const float ym = odd ? y1[0] : y0[0], lbm = odd ? lb1[0] : lb0[0], wam = odd ? wa1[0] : wa0[0];
+      const float um = odd ? u1[0] : u0[0], dtm = odd ? dt1[0] : dt0[0], dsm = odd ? ds1[0] : ds0[0];
+      const float gpm = odd ? gp1 : gp0;
+      const int rm = odd ? r1 : r0e;
+      const float dzm = gpm * fmaf(cr.Dk, um, ym);
+      const float dxm = fmaf(dtm, lbm, dsm * cr.Dk);
+      cr.dD = fmaf(dsm, um, cr.dD);
+      float ddm = fmaf(um, lbm, wam * kInvLog2e);
+      if constexpr (SP) {
+        if (softplus) ddm *= sigmoid_fast((odd ? raw1 : raw0) + cr.bias_own);
+        if (r0 + 2 * m + (odd ? 1 : 0) < nlive) cr.dbias += ddm;
+      }
+      reinterpret_cast<__nv_bfloat16*>(tox + rm * WPR)[ln.co] = __float2bfloat16_rn(dxm);
+      reinterpret_cast<__nv_bfloat16*>(tod + rm * WPR)[ln.co] = __float2bfloat16_rn(ddm);
+      reinterpret_cast<__nv_bfloat16*>(toz + rm * WPR)[ln.co] = __float2bfloat16_rn(dzm * gate_on);
     }
-    reinterpret_cast<__nv_bfloat16*>(tox + r1 * 16)[lane] = __float2bfloat16_rn(dx1);
-    reinterpret_cast<__nv_bfloat16*>(tod + r1 * 16)[lane] = __float2bfloat16_rn(dd1);
-    reinterpret_cast<__nv_bfloat16*>(toz + r1 * 16)[lane] = __float2bfloat16_rn(dz1 * gate_on);
-    reinterpret_cast<__nv_bfloat16*>(tox + r0e * 16)[lane] = __float2bfloat16_rn(dx0);
-    reinterpret_cast<__nv_bfloat16*>(tod + r0e * 16)[lane] = __float2bfloat16_rn(dd0);
-    reinterpret_cast<__nv_bfloat16*>(toz + r0e * 16)[lane] = __float2bfloat16_rn(dz0 * gate_on);
 
     if ((2 * m) % kRB == 0) {
       // dB / dC of steps 2m .. 2m + 3: every lane sums one float4 of one step over the lane groups, ascending
@@ -409,14 +454,17 @@ __device__ __forceinline__ void sub_block(const Lane<S>& ln, ChainRegs<S>& cr, i
 
 }  // namespace
 
-template <int S, bool SP>
-__global__ void __launch_bounds__(kBwdWarps * 32) ssm_bwd_warp_kernel(const BwdParams p, const WarpSched sc) {
-  constexpr int LPC = 16 / S, CPT = LPC, H = S / 2;
-  using Smem = BwdWarpSmem<S, SP>;
+template <int S, int CPT, bool SP>
+__global__ void __launch_bounds__(kBwdWarps * 32, (CPT == 16 / S) ? 2 : 3)
+    ssm_bwd_warp_kernel(const BwdParams p, const WarpSched sc) {
+  using LN = Lane<S, CPT>;
+  constexpr int H = S / 2, CW = LN::CW, WPR = CW / 2, NV = CPT * S / 4;   // NV: float4 of a thread's states
+  constexpr bool OWN = LN::OWN;
+  using Smem = BwdWarpSmem<S, CPT, SP>;
   extern __shared__ __align__(16) unsigned char smem_raw[];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   Smem& sm = reinterpret_cast<Smem*>(smem_raw)[warp];
-  const Lane<S> ln(lane);
+  const LN ln(lane);
   const int j = ln.j, g = ln.g;
   const int D = p.D;
   const int worker = blockIdx.x * kBwdWarps + warp;
@@ -432,7 +480,7 @@ __global__ void __launch_bounds__(kBwdWarps * 32) ssm_bwd_warp_kernel(const BwdP
   __nv_bfloat16* __restrict__ gdd = static_cast<__nv_bfloat16*>(p.ddelta);
   __nv_bfloat16* __restrict__ gdz = static_cast<__nv_bfloat16*>(p.dz);
 
-  const int groups = (D + 31) / 32;
+  const int groups = (D + CW - 1) / CW;
   const size_t bln = (size_t)p.batch * p.L * 16;
   const WorkList wl = make_worklist(sc, worker);
   for (int pi = 0; pi < wl.count; ++pi) {
@@ -441,7 +489,7 @@ __global__ void __launch_bounds__(kBwdWarps * 32) ssm_bwd_warp_kernel(const BwdP
     const int grp = chain % groups;
     const int bs = chain / groups;
     const int seg = bs % p.nseg, b = bs / p.nseg;
-    const int d_w = grp * 32;
+    const int d_w = grp * CW;
     const int t_seg0 = seg * p.seg_steps;
     const int t_seg_end = min(p.L, t_seg0 + p.seg_steps);
     const int live_tiles = (t_seg_end - t_seg0 + kBT - 1) / kBT;
@@ -451,32 +499,35 @@ __global__ void __launch_bounds__(kBwdWarps * 32) ssm_bwd_warp_kernel(const BwdP
     if (tile_hi > live_tiles - 1) tile_hi = live_tiles - 1;
     const bool gives_out = to < sc.tiles;
 
-    // ---- staging: this lane's chunks of a tile (rows lane / 4 + 8 k of x, delta, z, dout; row lane / 2 of B, C)
-    const int xrow = lane >> 2, xcc = lane & 3;
-    const bool xcol_ok = d_w + xcc * 8 < D;
-    const int brow = lane >> 1, bhc = lane & 1;
-    const int c_grp = d_w + g * CPT;          // first channel of this lane group (all valid or none)
-    const bool valid = c_grp < D;
-    auto chan = [&](int q) { return c_grp + (j ^ q); };
+    // ---- staging: 16-byte chunks of the tile rows (CW / 8 per row of x, delta, z, dout; 2 per row of B, C)
+    constexpr int CPR = CW / 8;                 // chunks per row
+    constexpr int XCH = kBT * CPR;              // chunks per tensor and tile
+    const int c_grp = d_w + g * CPT;            // first channel of this lane group
+    const bool valid = c_grp < D;               // (CPT channels: all valid or none, D is a multiple of 8)
+    auto chan = [&](int q) { return OWN ? c_grp + (j ^ q) : c_grp; };
     auto issue_tile = [&](int tile, int st) {
       if (tile >= tile_lo && tile >= 0) {
         const int t0 = t_seg0 + tile * kBT;
         const size_t row0 = (size_t)b * p.L + t0;
 #pragma unroll
-        for (int k = 0; k < (kBT + 7) / 8; ++k) {
-          const int tt = xrow + 8 * k;
-          const bool ok = xcol_ok && (t0 + tt < t_seg_end);
-          const size_t go = ok ? (row0 + tt) * D + d_w + xcc * 8 : 0;
-          cp_async16(&sm.x[st][tt][xcc * 4], gx + go, ok);
-          cp_async16(&sm.d[st][tt][xcc * 4], gd + go, ok);
-          cp_async16(&sm.z[st][tt][xcc * 4], (has_z ? gz : gx) + go, ok && has_z);
-          cp_async16(&sm.g[st][tt][xcc * 4], gg + go, ok);
+        for (int k = 0; k < (XCH + 31) / 32; ++k) {
+          const int c = lane + 32 * k;
+          if (XCH % 32 == 0 || c < XCH) {
+            const int tt = c / CPR, cc = c % CPR;
+            const bool ok = (d_w + cc * 8 < D) && (t0 + tt < t_seg_end);
+            const size_t go = ok ? (row0 + tt) * D + d_w + cc * 8 : 0;
+            cp_async16(&sm.x[st][tt][cc * 4], gx + go, ok);
+            cp_async16(&sm.d[st][tt][cc * 4], gd + go, ok);
+            cp_async16(&sm.z[st][tt][cc * 4], (has_z ? gz : gx) + go, ok && has_z);
+            cp_async16(&sm.g[st][tt][cc * 4], gg + go, ok);
+          }
         }
-        if (brow < kBT) {
-          const bool ok = t0 + brow < t_seg_end;
-          const size_t go = ok ? (row0 + brow) * 16 + bhc * 8 : 0;
-          cp_async16(&sm.rB[st][brow][bhc * 4], gB + go, ok);
-          cp_async16(&sm.rC[st][brow][bhc * 4], gC + go, ok);
+        if (lane < kBT * 2) {
+          const int tt = lane >> 1, hc = lane & 1;
+          const bool ok = t0 + tt < t_seg_end;
+          const size_t go = ok ? (row0 + tt) * 16 + hc * 8 : 0;
+          cp_async16(&sm.rB[st][tt][hc * 4], gB + go, ok);
+          cp_async16(&sm.rC[st][tt][hc * 4], gC + go, ok);
         }
 #pragma unroll
         for (int sb = 0; sb < kBT / kSB; ++sb) {
@@ -495,7 +546,7 @@ __global__ void __launch_bounds__(kBwdWarps * 32) ssm_bwd_warp_kernel(const BwdP
     issue_tile(tile_hi, 0);
 
     // ---- per-thread constants and carried values
-    ChainRegs<S> cr;
+    ChainRegs<S, CPT> cr;
     bool ap = !p.general_A;
 #pragma unroll
     for (int q = 0; q < CPT; ++q) {
@@ -516,7 +567,7 @@ __global__ void __launch_bounds__(kBwdWarps * 32) ssm_bwd_warp_kernel(const BwdP
       cr.rs[q] = cr.A2[q][0].y - cr.A2[q][0].x;
     }
     ap = __all_sync(0xffffffffu, ap);
-    const int c_own = d_w + lane;
+    const int c_own = d_w + ln.co;
     cr.Dk = (p.Dskip != nullptr && c_own < D) ? p.Dskip[c_own] : 0.f;
     cr.bias_own = (SP && p.delta_bias != nullptr && c_own < D) ? p.delta_bias[c_own] : 0.f;
     cr.dD = 0.f;
@@ -527,17 +578,17 @@ __global__ void __launch_bounds__(kBwdWarps * 32) ssm_bwd_warp_kernel(const BwdP
         return;
       }
       const float4* hb = sc.handoff + ((size_t)worker * 32 + lane) * kBwdHandoffVec;
-      float4 v[8];
+      float4 v[2 * NV];
 #pragma unroll
-      for (int k = 0; k < 8; ++k) v[k] = __ldcg(hb + k);
-      const float4 dv = __ldcg(hb + 8);
+      for (int k = 0; k < 2 * NV; ++k) v[k] = __ldcg(hb + k);
+      const float4 dv = __ldcg(hb + 2 * NV);
       const float* f = reinterpret_cast<const float*>(v);
 #pragma unroll
       for (int q = 0; q < CPT; ++q)
 #pragma unroll
         for (int k = 0; k < H; ++k) {
           cr.mu[q][k] = make_float2(f[(q * H + k) * 2], f[(q * H + k) * 2 + 1]);
-          cr.dA[q][k] = make_float2(f[16 + (q * H + k) * 2], f[16 + (q * H + k) * 2 + 1]);
+          cr.dA[q][k] = make_float2(f[4 * NV + (q * H + k) * 2], f[4 * NV + (q * H + k) * 2 + 1]);
         }
       cr.dD = dv.x;
       cr.dbias = dv.y;
@@ -562,7 +613,6 @@ __global__ void __launch_bounds__(kBwdWarps * 32) ssm_bwd_warp_kernel(const BwdP
       issue_tile(tile - 1, st ^ 1);   // prefetch the tile before in time
       const int t0 = t_seg0 + tile * kBT;
       const int nlive = min(kBT, t_seg_end - t0);
-      // ---- per-element gate terms of the tile, one channel per lane: ds = dout silu(z), gp = dout silu'(z)
       {
         // B and C of the tile to float: lane -> (row lane / 4, states 4 (lane % 4) ..)
 #pragma unroll
@@ -575,27 +625,34 @@ __global__ void __launch_bounds__(kBwdWarps * 32) ssm_bwd_warp_kernel(const BwdP
             *reinterpret_cast<float4*>(&sm.fC[rr][4 * qq]) = make_float4(bf16lo(wc.x), bf16hi(wc.x), bf16lo(wc.y), bf16hi(wc.y));
           }
         }
-        float zf[kBT], gf[kBT], df[SP ? kBT : 1];
+        // per-element gate terms of the tile: ds = dout silu(z), gp = dout silu'(z); element e = lane + 32 i
+        constexpr int EPL = kBT * CW / 32;   // elements per lane
+        float zf[EPL], gf[EPL], df[SP ? EPL : 1];
 #pragma unroll
-        for (int r = 0; r < kBT; ++r) {
-          zf[r] = __uint_as_float((uint32_t)reinterpret_cast<const uint16_t*>(sm.z[st][r])[lane] << 16);
-          gf[r] = __uint_as_float((uint32_t)reinterpret_cast<const uint16_t*>(sm.g[st][r])[lane] << 16);
-          if constexpr (SP) df[r] = __uint_as_float((uint32_t)reinterpret_cast<const uint16_t*>(sm.d[st][r])[lane] << 16);
+        for (int i = 0; i < EPL; ++i) {
+          const int e = lane + 32 * i, r = e / CW, c = e % CW;
+          zf[i] = __uint_as_float((uint32_t)reinterpret_cast<const uint16_t*>(sm.z[st][r])[c] << 16);
+          gf[i] = __uint_as_float((uint32_t)reinterpret_cast<const uint16_t*>(sm.g[st][r])[c] << 16);
+          if constexpr (SP) df[i] = __uint_as_float((uint32_t)reinterpret_cast<const uint16_t*>(sm.d[st][r])[c] << 16);
         }
+        // (with 32 channels per warp an element's channel is this lane's own; with 16 it is lane % 16)
+        const int c_el = d_w + lane % CW;
+        const float bias_el = (SP && p.delta_bias != nullptr && c_el < D) ? p.delta_bias[c_el] : 0.f;
 #pragma unroll
-        for (int r = 0; r < kBT; ++r) {
-          float dsv = gf[r], gpv = 0.f;
+        for (int i = 0; i < EPL; ++i) {
+          const int e = lane + 32 * i, r = e / CW, c = e % CW;
+          float dsv = gf[i], gpv = 0.f;
           if (has_z) {
-            const float sg = sigmoid_fast(zf[r]);
-            dsv = gf[r] * zf[r] * sg;
-            gpv = gf[r] * sg * fmaf(zf[r], 1.f - sg, 1.f);
+            const float sg = sigmoid_fast(zf[i]);
+            dsv = gf[i] * zf[i] * sg;
+            gpv = gf[i] * sg * fmaf(zf[i], 1.f - sg, 1.f);
           }
-          sm.ds[r][lane] = dsv;
-          sm.gp[r][lane] = gpv;
+          sm.ds[r][c] = dsv;
+          sm.gp[r][c] = gpv;
           if constexpr (SP) {
-            float v = df[r] + cr.bias_own;
+            float v = df[i] + bias_el;
             if (p.softplus) v = softplus_fast(v);
-            sm.dF[r][lane] = r < nlive ? v : 0.f;   // rows past the end stay identity steps
+            sm.dF[r][c] = r < nlive ? v : 0.f;   // rows past the end stay identity steps
           }
         }
       }
@@ -607,26 +664,27 @@ __global__ void __launch_bounds__(kBwdWarps * 32) ssm_bwd_warp_kernel(const BwdP
       for (int sb = kBT / kSB - 1; sb >= 0; --sb) {
         if (sb * kSB >= nlive) continue;   // a sub-block of identity steps
         if (ap)
-          sub_block<S, SP, true>(ln, cr, sb * kSB, nlive, has_z ? 1.f : 0.f, p.softplus != 0, &sm.x[st][0][0], &sm.d[st][0][0],
-                                 &sm.fB[0][0], &sm.fC[0][0], &sm.ds[0][0], &sm.gp[0][0], &sm.dF[0][0],
-                                 &sm.ck[st][sb][0][0], &sm.ox[0][0], &sm.od[0][0], &sm.oz[0][0], &sm.red[0][0][0], part_dB,
-                                 part_dC, sc.abort);
+          sub_block<S, CPT, SP, true>(ln, cr, sb * kSB, nlive, has_z ? 1.f : 0.f, p.softplus != 0, &sm.x[st][0][0],
+                                      &sm.d[st][0][0], &sm.fB[0][0], &sm.fC[0][0], &sm.ds[0][0], &sm.gp[0][0], &sm.dF[0][0],
+                                      &sm.ck[st][sb][0][0], &sm.ox[0][0], &sm.od[0][0], &sm.oz[0][0], &sm.red[0][0][0],
+                                      part_dB, part_dC, sc.abort);
         else
-          sub_block<S, SP, false>(ln, cr, sb * kSB, nlive, has_z ? 1.f : 0.f, p.softplus != 0, &sm.x[st][0][0], &sm.d[st][0][0],
-                                  &sm.fB[0][0], &sm.fC[0][0], &sm.ds[0][0], &sm.gp[0][0], &sm.dF[0][0],
-                                  &sm.ck[st][sb][0][0], &sm.ox[0][0], &sm.od[0][0], &sm.oz[0][0], &sm.red[0][0][0], part_dB,
-                                  part_dC, sc.abort);
+          sub_block<S, CPT, SP, false>(ln, cr, sb * kSB, nlive, has_z ? 1.f : 0.f, p.softplus != 0, &sm.x[st][0][0],
+                                       &sm.d[st][0][0], &sm.fB[0][0], &sm.fC[0][0], &sm.ds[0][0], &sm.gp[0][0], &sm.dF[0][0],
+                                       &sm.ck[st][sb][0][0], &sm.ox[0][0], &sm.od[0][0], &sm.oz[0][0], &sm.red[0][0][0],
+                                       part_dB, part_dC, sc.abort);
       }
       __syncwarp();
       // ---- results of the tile: 16-byte stores of dx, ddelta, dz
 #pragma unroll
-      for (int k = 0; k < (kBT + 7) / 8; ++k) {
-        const int tt = xrow + 8 * k;
-        if (xcol_ok && tt < nlive) {
-          const size_t go = (row0 + tt) * D + d_w + xcc * 8;
-          *reinterpret_cast<uint4*>(gdx + go) = *reinterpret_cast<const uint4*>(&sm.ox[tt][xcc * 4]);
-          *reinterpret_cast<uint4*>(gdd + go) = *reinterpret_cast<const uint4*>(&sm.od[tt][xcc * 4]);
-          if (gdz != nullptr) *reinterpret_cast<uint4*>(gdz + go) = *reinterpret_cast<const uint4*>(&sm.oz[tt][xcc * 4]);
+      for (int k = 0; k < (XCH + 31) / 32; ++k) {
+        const int c = lane + 32 * k;
+        const int tt = c / CPR, cc = c % CPR;
+        if ((XCH % 32 == 0 || c < XCH) && d_w + cc * 8 < D && tt < nlive) {
+          const size_t go = (row0 + tt) * D + d_w + cc * 8;
+          *reinterpret_cast<uint4*>(gdx + go) = *reinterpret_cast<const uint4*>(&sm.ox[tt][cc * 4]);
+          *reinterpret_cast<uint4*>(gdd + go) = *reinterpret_cast<const uint4*>(&sm.od[tt][cc * 4]);
+          if (gdz != nullptr) *reinterpret_cast<uint4*>(gdz + go) = *reinterpret_cast<const uint4*>(&sm.oz[tt][cc * 4]);
         }
       }
     }
@@ -636,45 +694,55 @@ __global__ void __launch_bounds__(kBwdWarps * 32) ssm_bwd_warp_kernel(const BwdP
     if (gives_out) {
       // the earlier part of this chain (in time) belongs to the next worker
       float4* hb = sc.handoff + ((size_t)(worker + 1) * 32 + lane) * kBwdHandoffVec;
-      float f[32];
+      float f[8 * NV];
 #pragma unroll
       for (int q = 0; q < CPT; ++q)
 #pragma unroll
         for (int k = 0; k < H; ++k) {
           f[(q * H + k) * 2] = cr.mu[q][k].x;
           f[(q * H + k) * 2 + 1] = cr.mu[q][k].y;
-          f[16 + (q * H + k) * 2] = cr.dA[q][k].x;
-          f[16 + (q * H + k) * 2 + 1] = cr.dA[q][k].y;
+          f[4 * NV + (q * H + k) * 2] = cr.dA[q][k].x;
+          f[4 * NV + (q * H + k) * 2 + 1] = cr.dA[q][k].y;
         }
 #pragma unroll
-      for (int k = 0; k < 8; ++k) __stcg(hb + k, make_float4(f[4 * k], f[4 * k + 1], f[4 * k + 2], f[4 * k + 3]));
-      __stcg(hb + 8, make_float4(cr.dD, cr.dbias, 0.f, 0.f));
+      for (int k = 0; k < 2 * NV; ++k) __stcg(hb + k, make_float4(f[4 * k], f[4 * k + 1], f[4 * k + 2], f[4 * k + 3]));
+      __stcg(hb + 2 * NV, make_float4(cr.dD, cr.dbias, 0.f, 0.f));
       publish_handoff(sc, worker, lane);
-    } else if (valid) {
+    } else {
       // first step in time done: the chain is complete
-      const size_t part = (size_t)b * p.nseg + seg;
+      float dD_tot = cr.dD, dbias_tot = cr.dbias;
+      if constexpr (!OWN) {   // the two lanes of a group summed the steps of one parity each
+        dD_tot += __shfl_xor_sync(0xffffffffu, dD_tot, 1);
+        dbias_tot += __shfl_xor_sync(0xffffffffu, dbias_tot, 1);
+      }
+      if (valid) {
+        const size_t part = (size_t)b * p.nseg + seg;
 #pragma unroll
-      for (int q = 0; q < CPT; ++q)
+        for (int q = 0; q < CPT; ++q)
 #pragma unroll
-        for (int k = 0; k < S / 4; ++k) {
-          *reinterpret_cast<float4*>(p.dA_part + (part * D + chan(q)) * 16 + S * j + 4 * k) =
-              make_float4(cr.dA[q][2 * k].x, cr.dA[q][2 * k].y, cr.dA[q][2 * k + 1].x, cr.dA[q][2 * k + 1].y);
-          if (seg == 0 && p.dh0 != nullptr)   // the adjoint that leaves the first step is the gradient of the initial state
-            *reinterpret_cast<float4*>(p.dh0 + ((size_t)b * D + chan(q)) * 16 + S * j + 4 * k) =
-                make_float4(cr.mu[q][2 * k].x, cr.mu[q][2 * k].y, cr.mu[q][2 * k + 1].x, cr.mu[q][2 * k + 1].y);
+          for (int k = 0; k < S / 4; ++k) {
+            *reinterpret_cast<float4*>(p.dA_part + (part * D + chan(q)) * 16 + S * j + 4 * k) =
+                make_float4(cr.dA[q][2 * k].x, cr.dA[q][2 * k].y, cr.dA[q][2 * k + 1].x, cr.dA[q][2 * k + 1].y);
+            if (seg == 0 && p.dh0 != nullptr)   // the adjoint that leaves the first step is the gradient of the initial state
+              *reinterpret_cast<float4*>(p.dh0 + ((size_t)b * D + chan(q)) * 16 + S * j + 4 * k) =
+                  make_float4(cr.mu[q][2 * k].x, cr.mu[q][2 * k].y, cr.mu[q][2 * k + 1].x, cr.mu[q][2 * k + 1].y);
+          }
+        if (OWN || j == 0) {
+          p.dD_part[part * D + c_own] = dD_tot;
+          if (SP && p.dbias_part != nullptr) p.dbias_part[part * D + c_own] = dbias_tot;
         }
-      p.dD_part[part * D + c_own] = cr.dD;
-      if (SP && p.dbias_part != nullptr) p.dbias_part[part * D + c_own] = cr.dbias;
+      }
     }
   }
 }
 
 namespace {
 
-template <int S, bool SP>
+template <int S, int CPT, bool SP>
 cudaError_t launch_bwd_variant(const Plan& plan, const BwdParams& p, cudaStream_t s) {
-  const size_t smem = sizeof(BwdWarpSmem<S, SP>) * kBwdWarps;
-  auto kern = ssm_bwd_warp_kernel<S, SP>;
+  constexpr int CW = Lane<S, CPT>::CW;
+  const size_t smem = sizeof(BwdWarpSmem<S, CPT, SP>) * kBwdWarps;
+  auto kern = ssm_bwd_warp_kernel<S, CPT, SP>;
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
   int dev = 0, sms = 0, per_sm = 0;
@@ -683,7 +751,7 @@ cudaError_t launch_bwd_variant(const Plan& plan, const BwdParams& p, cudaStream_
   if ((e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, kBwdWarps * 32, smem)) != cudaSuccess) return e;
   if (per_sm < 1) return cudaErrorLaunchOutOfResources;
   WarpSched sc{};
-  sc.chains = p.batch * plan.nseg * ((p.D + 31) / 32);
+  sc.chains = p.batch * plan.nseg * ((p.D + CW - 1) / CW);
   sc.tiles = (plan.seg_steps + kBT - 1) / kBT;
   const bool can_share = p.abort != nullptr && p.flags != nullptr && p.handoff != nullptr && p.max_workers > 0;
   sc.workers = warp_workers(sc.chains, sms, per_sm * kBwdWarps, can_share ? p.max_workers : 0);
@@ -711,14 +779,18 @@ bool bwd_fast_applicable(const ssm_problem_t& prob, const BwdParams& p) {
   return prob.io_dtype == SSM_BF16 && prob.N == 16 && prob.D % 8 == 0 && p.seg_steps % kBT == 0 && al16(p.x) &&
          al16(p.delta) && al16(p.z) && al16(p.B) && al16(p.C) && al16(p.dout) && al16(p.dx) && al16(p.ddelta) &&
          al16(p.dz) && al16(p.A) && al16(p.ckpt) && al16(p.mu_in) && al16(p.dh0) && al16(p.dBC_part) && al16(p.dA_part) &&
-         al16(p.handoff);
+         al16(p.handoff) && (p.groups == (p.D + 31) / 32 || p.groups == (p.D + 15) / 16);
 }
 
 size_t bwd_handoff_bytes_per_worker() { return sizeof(float4) * kBwdHandoffVec * 32; }
+// channels per warp of the tuned kernel = the channel-group size of the dB / dC partial sums
+int bwd_fast_channels_per_warp() { return kBwdFastChannels; }
 
 cudaError_t launch_bwd_fast(const Plan& plan, const BwdParams& p, cudaStream_t s) {
   const bool sp = p.softplus || p.delta_bias != nullptr;
-  return sp ? launch_bwd_variant<8, true>(plan, p, s) : launch_bwd_variant<8, false>(plan, p, s);
+  if (p.groups == (p.D + 15) / 16 && p.groups != (p.D + 31) / 32)
+    return sp ? launch_bwd_variant<8, 1, true>(plan, p, s) : launch_bwd_variant<8, 1, false>(plan, p, s);
+  return sp ? launch_bwd_variant<8, 2, true>(plan, p, s) : launch_bwd_variant<8, 2, false>(plan, p, s);
 }
 
 }  // namespace ssm

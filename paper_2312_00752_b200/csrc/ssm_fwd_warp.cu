@@ -585,17 +585,17 @@ bool fwd_fast_applicable(const ssm_problem_t& prob, const FwdParams& p) {
          al16(p.h_last) && al16(p.handoff);
 }
 
-int fwd_states_per_thread() { return 8; }
+int fwd_states_per_thread() { return 16; }
 size_t fwd_handoff_bytes_per_worker() { return sizeof(float4) * kFwdHandoffVec * 32; }
 
 cudaError_t launch_fwd_fast(const Plan& plan, const FwdParams& p, int mode, cudaStream_t s) {
 #ifdef SSM_DEV_TUNING
   if (const char* e = getenv("SSM_FWD_S")) {
     if (e[0] == '4') return launch_s<4>(plan, p, mode, s);
-    if (e[0] == '1') return launch_s<16>(plan, p, mode, s);
+    if (e[0] == '8') return launch_s<8>(plan, p, mode, s);
   }
 #endif
-  return launch_s<8>(plan, p, mode, s);
+  return launch_s<16>(plan, p, mode, s);
 }
 
 }  // namespace ssm
