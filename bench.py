@@ -14,6 +14,7 @@ from __future__ import annotations
 
 import argparse
 import json
+import math
 import os
 import statistics
 import subprocess
@@ -27,9 +28,11 @@ if ROOT not in sys.path:
 
 METRIC = "selective-scan fwd+bwd elements/s (elements = batch*L*D); achieved HBM GB/s as % of measured B200 peak"
 FALLBACK_HBM_GBS = 6650.0
-# DRAM bytes (read + write) of one launch of the dominant kernel from an ncu capture at the bench workload itself
-# (profiles/ssm_bwd_fast_kernel_mamba2p8b_layer.md); None where no capture exists.
-NCU_TRAFFIC_BYTES = {3: 420.4e6 + 383.9e6}
+# DRAM bytes (read + write) of one launch of the dominant kernel of each direction from ncu captures at the bench
+# workload itself (profiles/ssm_bwd_warp_kernel_mamba2p8b_layer.md, profiles/ssm_fwd_warp_kernel_mamba2p8b_layer.md);
+# None where no capture exists.
+NCU_TRAFFIC_BYTES = {3: 703.1e6 + 395.5e6}
+NCU_TRAFFIC_BYTES_FWD = {3: 262.5e6 + 371.1e6}
 
 
 def parse_args():
@@ -146,41 +149,53 @@ def job_value(elements_per_rank: int, world: int, ms_per_step: float) -> float:
     return world * elements_per_rank / (ms_per_step * 1e-3)
 
 
-def kernels_per_step(plan_info: dict) -> int:
-    """Kernel launches of one fwd (saving states) + bwd (given saved states) pass."""
-    if plan_info["n_segments"] == 1:
-        return 1 + 2            # forward; backward + reduction
-    return 3 + 4                # summary, carry, forward; local adjoint, carry, backward, reduction
+def kernels_per_step(plan_info: dict, bwd_plan_info: dict) -> int:
+    """Kernel launches of one fwd (saving states) + bwd (given saved states) pass; each direction splits the sequence
+    in time on its own terms."""
+    fwd = 1 if plan_info["n_segments"] == 1 else 3        # [summary, carry,] forward
+    bwd = 2 if bwd_plan_info["n_segments"] == 1 else 4    # [adjoint pre-pass, carry,] backward, reduction
+    return fwd + bwd
+
+
+def workload_name(cfg) -> str:
+    return (f"{cfg.name} (config {cfg.cfg_id}): batch {cfg.batch}, L {cfg.L}, D {cfg.D}, N {cfg.N}, {cfg.io} io, "
+            f"fp32 state; one step = selective-scan forward (saving checkpoint states) + backward")
 
 
 # ------------------------------------------------------------------------------------------------ oracle timing
-def time_oracle(cfg, host, budget_core_s=25.0):
-    """Times the fp64 oracle (fwd and fwd+bwd) on a bounded sample of the workload: whole batch entries, all channels
-    or the first `dsel` channels, sized for roughly `budget_core_s` core-seconds."""
-    from oracle import ssm_oracle as O
-    cores = O.threads_available()
-    est_core_s = cfg.elements * cfg.N * 45e-9            # ~45 ns per state step for fwd+bwd on one core
-    frac = min(1.0, budget_core_s / est_core_s)
-    if frac * cfg.batch >= 1.0:
-        nb, dsel = int(frac * cfg.batch), cfg.D
-    else:
-        nb, dsel = 1, min(cfg.D, max(64, int(cfg.D * frac * cfg.batch) // 64 * 64))
-    sl = lambda a: a[:nb, :, :dsel]
-    x, dl, z, g = sl(host["x"]), sl(host["delta"]), sl(host["z"]), sl(host["dout"])
-    B, C = host["B"][:nb], host["C"][:nb]
-    A, Dk = host["A"][:dsel], host["D_skip"][:dsel]
+def time_oracle(cfg, host, nthreads=0, batch_entries=None):
+    """Times the fp64 oracle, as it stands, forward then backward, on the first `batch_entries` batch entries of the
+    workload (all of them by default: every channel and every step) with `nthreads` threads (0: all cores)."""
     import numpy as np
-    x, dl, z, g = (np.ascontiguousarray(v) for v in (x, dl, z, g))
+    from oracle import ssm_oracle as O
+    nb = cfg.batch if batch_entries is None else max(1, min(cfg.batch, batch_entries))
+    x, dl, z, g = (np.ascontiguousarray(host[k][:nb]) for k in ("x", "delta", "z", "dout"))
+    B, C = host["B"][:nb], host["C"][:nb]
+    A, Dk = host["A"], host["D_skip"]
     t0 = time.perf_counter()
-    O.scan_fwd(x, dl, A, B, C, D_skip=Dk, z=z)
+    O.scan_fwd(x, dl, A, B, C, D_skip=Dk, z=z, nthreads=nthreads)
     t1 = time.perf_counter()
-    O.scan_bwd(x, dl, A, B, C, Dk, z, g)
+    O.scan_bwd(x, dl, A, B, C, Dk, z, g, nthreads=nthreads)
     t2 = time.perf_counter()
-    el = nb * cfg.L * dsel
-    return {"value": el / (t2 - t0), "unit": "elements/s", "cores": cores, "kind": "oracle",
-            "sample": f"batch entries 0..{nb - 1}, channels 0..{dsel - 1} of the workload ({el} elements), "
-                      f"fwd {t1 - t0:.2f} s + bwd {t2 - t1:.2f} s wall",
+    el = nb * cfg.L * cfg.D
+    return {"value": el / (t2 - t0), "unit": "elements/s", "cores": nthreads if nthreads else O.threads_available(),
+            "kind": "oracle",
+            "sample": ("the whole workload" if nb == cfg.batch else f"batch entries 0..{nb - 1} of {cfg.batch}") +
+                      f" ({el} elements), fwd {t1 - t0:.2f} s + bwd {t2 - t1:.2f} s wall",
             "fwd_elements_per_s": el / (t1 - t0)}
+
+
+def cpu_baseline(cfg, host):
+    """The oracle on the host cores: all cores on the whole workload, one thread on a bounded part of it (about 30
+    core-seconds in total for the 2.8B layer shape; longer workloads are cut to whole batch entries / fewer steps)."""
+    est_core_s = cfg.elements * cfg.N * 45e-9            # ~45 ns per state step for fwd+bwd on one core
+    if est_core_s > 120:                                 # the long-sequence workload: not timed in full
+        return {"skipped": f"about {est_core_s:.0f} core-seconds"}
+    res = time_oracle(cfg, host, nthreads=0)
+    one = time_oracle(cfg, host, nthreads=1, batch_entries=max(1, int(cfg.batch * 8.0 / est_core_s)))
+    res["single_thread"] = {"value": one["value"], "unit": "elements/s", "cores": 1, "sample": one["sample"],
+                            "fwd_elements_per_s": one["fwd_elements_per_s"]}
+    return res
 
 
 def run_reference(args, cfg):
@@ -193,7 +208,7 @@ def run_reference(args, cfg):
     info = None
     for i in range(args.warmup + args.steps):
         t0 = time.perf_counter()
-        info = time_oracle(cfg, host, budget_core_s=8.0)
+        info = time_oracle(cfg, host)          # the whole workload, all cores
         if i >= args.warmup:
             per_step.append(info["value"])
             per_ms.append((time.perf_counter() - t0) * 1e3)
@@ -203,9 +218,8 @@ def run_reference(args, cfg):
     line = {"impl": "reference", "metric": METRIC, "value": v, "unit": "elements/s", "n_gpus": args.gpus,
             "steps": len(per_step), "warmup": args.warmup, "ms_per_step": statistics.median(per_ms),
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": {"workload": f"{cfg.name} (config {cfg.cfg_id}): batch {cfg.batch}, L {cfg.L}, D {cfg.D}, N {cfg.N}, "
-                                   f"{cfg.io} io; one step = oracle forward + backward on a bounded sample of this workload",
-                       "batch": cfg.batch, "L": cfg.L, "D": cfg.D, "N": cfg.N, "io": cfg.io},
+            "config": {"workload": workload_name(cfg), "batch": cfg.batch, "L": cfg.L, "D": cfg.D, "N": cfg.N,
+                       "io": cfg.io, "step": "fp64 oracle forward + backward over the whole workload, all host cores"},
             "cpu_baseline": {"value": v, "unit": "elements/s", "cores": info["cores"], "kind": "oracle",
                              "sample": info["sample"]},
             "e2e": {"value": v, "unit": "elements/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
@@ -214,6 +228,58 @@ def run_reference(args, cfg):
 
 
 # ------------------------------------------------------------------------------------------------ our arm
+def time_shape(K, torch, dev, stream, cfg, peak, general_A=False, reps=None):
+    """Forward (saving states) and backward times of one more workload, with timing-only inputs drawn on the device
+    (same shapes and value ranges as the seeded host recipe); every repetition is timed on its own with CUDA events and
+    a buffer larger than L2 is overwritten in between."""
+    io_t = torch.bfloat16 if cfg.io == "bf16" else torch.float32
+    g = torch.Generator(device=dev)
+    g.manual_seed(1234 + cfg.cfg_id)
+    shp, bshp = (cfg.batch, cfg.L, cfg.D), (cfg.batch, cfg.L, cfg.N)
+    rn = lambda shape: torch.randn(shape, generator=g, device=dev, dtype=torch.float32)
+    t = {k: rn(shp).to(io_t) for k in ("x", "z", "dout")}
+    t["B"], t["C"] = rn(bshp).to(io_t), rn(bshp).to(io_t)
+    tau = torch.exp(torch.empty(cfg.D, device=dev).uniform_(math.log(cfg.dt_min), math.log(cfg.dt_max), generator=g))
+    bias = tau + torch.log(-torch.expm1(-tau))
+    t["delta"] = torch.nn.functional.softplus(0.1 * rn(shp) + bias).to(io_t)
+    A = -(torch.arange(cfg.N, device=dev, dtype=torch.float32) + 1.0).repeat(cfg.D, 1)
+    if general_A:
+        A = A * (1.0 + 0.01 * rn((cfg.D, cfg.N)))
+    Dk = torch.ones(cfg.D, device=dev)
+    prob = K.make_problem(t["x"], t["B"], True, True, save_states=True)
+    out = torch.empty_like(t["x"])
+    saved = torch.empty(K.saved_state_bytes(prob) // 4, dtype=torch.float32, device=dev)
+    grads = {"dx": torch.empty_like(t["x"]), "ddelta": torch.empty_like(t["x"]), "dz": torch.empty_like(t["x"]),
+             "dB": torch.empty_like(t["B"]), "dC": torch.empty_like(t["B"]), "dA": torch.empty_like(A),
+             "dD": torch.empty_like(Dk)}
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+    fwd = lambda: K.ssm_scan_fwd(t["x"], t["delta"], A, t["B"], t["C"], Dk, t["z"], save_states=True, out=out,
+                                 saved_states=saved, stream=stream, general_A=general_A)
+    bwd = lambda: K.ssm_scan_bwd(t["x"], t["delta"], A, t["B"], t["C"], Dk, t["z"], t["dout"], saved, outputs=grads,
+                                 stream=stream, general_A=general_A)
+    reps = reps or (5 if cfg.elements > 2e8 else 12)
+    f_ms, b_ms = [], []
+    for i in range(3 + reps):
+        flush.zero_()
+        e = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
+        e[0].record(stream); fwd(); e[1].record(stream); bwd(); e[2].record(stream)
+        torch.cuda.synchronize(dev)
+        if i >= 3:
+            f_ms.append(e[0].elapsed_time(e[1])); b_ms.append(e[1].elapsed_time(e[2]))
+    fb, bb = algorithmic_bytes(cfg)
+    f, b = statistics.median(f_ms), statistics.median(b_ms)
+    res = {"workload": f"config {cfg.cfg_id}: batch {cfg.batch}, L {cfg.L}, D {cfg.D}, N {cfg.N}, {cfg.io} io" +
+                       (", A perturbed (no arithmetic progression: one exponential per state)" if general_A else ""),
+           "fwd_ms": f, "bwd_ms": b, "fwd_elements_per_s": cfg.elements / (f * 1e-3),
+           "bwd_elements_per_s": cfg.elements / (b * 1e-3), "step_elements_per_s": cfg.elements / ((f + b) * 1e-3),
+           "fwd_frac_of_hbm_peak": fb / (f * 1e-3) / 1e9 / peak, "bwd_frac_of_hbm_peak": bb / (b * 1e-3) / 1e9 / peak,
+           "plan": K.plan(prob), "bwd_plan": K.bwd_plan(prob), "repetitions": reps,
+           "inputs": "drawn on the device (timing only); L2 flushed between repetitions"}
+    del t, out, saved, grads, flush
+    torch.cuda.empty_cache()
+    return res
+
+
 def run_ours(args, cfg):
     import numpy as np
     import torch
@@ -242,6 +308,7 @@ def run_ours(args, cfg):
     d0 = sets[0]
     prob = K.make_problem(d0["x"], d0["B"], True, True, save_states=True)
     plan_info = K.plan(prob)
+    bwd_plan_info = K.bwd_plan(prob)
     out = torch.empty_like(d0["x"])
     saved = torch.empty(K.saved_state_bytes(prob) // 4, dtype=torch.float32, device=dev)
     grads = {"dx": torch.empty_like(d0["x"]), "ddelta": torch.empty_like(d0["x"]), "dz": torch.empty_like(d0["x"]),
@@ -338,21 +405,25 @@ def run_ours(args, cfg):
     line = {
         "metric": METRIC, "value": job_value(cfg.elements, world, ms_per_step), "unit": "elements/s",
         "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step,
-        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-        "config": {"workload": f"{cfg.name} (config {cfg.cfg_id}): batch {cfg.batch}, L {cfg.L}, D {cfg.D}, N {cfg.N}, "
-                               f"{cfg.io} io, fp32 state; one step = ssm_scan_fwd (saving checkpoint states) + ssm_scan_bwd",
-                   "batch": cfg.batch, "L": cfg.L, "D": cfg.D, "N": cfg.N, "io": cfg.io,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "io_dtype": cfg.io,
+        "data": "synthetic",
+        "config": {"workload": workload_name(cfg), "batch": cfg.batch, "L": cfg.L, "D": cfg.D, "N": cfg.N, "io": cfg.io,
+                   "step": "ssm_scan_fwd (saving checkpoint states) + ssm_scan_bwd through the C ABI",
                    "A": "perturbed (general path)" if args.general_A else "S4D-Real -(n+1)",
                    "l2": f"inputs larger than L2 (4 x {cfg.elements * (2 if cfg.io == 'bf16' else 4) / 1e6:.0f} MB) and "
                          f"{NSETS} input sets rotated between steps",
-                   "plan": plan_info, "parallelism": "replicas" if world > 1 else "single"},
+                   "plan": plan_info, "bwd_plan": bwd_plan_info,
+                   "parallelism": "replicas" if world > 1 else "single"},
         "clocks": clocks,
-        "gpu_launches": kernels_per_step(plan_info) * args.steps,
+        "gpu_launches": kernels_per_step(plan_info, bwd_plan_info) * args.steps,
         "fwd": {"ms": f_ms, "elements_per_s": cfg.elements / (f_ms * 1e-3), "algorithmic_bytes": fwd_bytes,
-                "achieved_gbs": fwd_gbs, "frac_of_hbm_peak": fwd_gbs / peak, **alu_fracs("fwd", f_ms)},
+                "achieved_gbs": fwd_gbs, "frac_of_hbm_peak": fwd_gbs / peak, **alu_fracs("fwd", f_ms),
+                "traffic": NCU_TRAFFIC_BYTES_FWD.get(cfg.cfg_id) if not args.general_A else None},
         "bwd": {"ms": b_ms, "elements_per_s": cfg.elements / (b_ms * 1e-3), "algorithmic_bytes": bwd_bytes,
                 "achieved_gbs": bwd_gbs, "frac_of_hbm_peak": bwd_gbs / peak, **alu_fracs("bwd", b_ms)},
-        "roofline": {"bound": "hbm", "kernel": "ssm_scan_bwd call (backward kernel + its reduction kernel)",
+        "roofline": {"bound": "hbm", "binding_bound": "alu (FP32 lanes; see roofline_alu)",
+                     "kernel": "ssm_scan_bwd call (ssm_bwd_warp_kernel, the dominant kernel, with its adjoint pre-pass, "
+                               "carry and reduction kernels)",
                      "achieved": bwd_gbs, "peak": peak, "peak_kind": f"{peak_kind} copy bandwidth",
                      "unit": "GB/s", "frac": bwd_gbs / peak,
                      "traffic": NCU_TRAFFIC_BYTES.get(cfg.cfg_id) if not args.general_A else None,
@@ -447,8 +518,18 @@ def run_ours(args, cfg):
         line["conv1d"] = {"error": str(exc)}
     if e2e is not None:
         line["e2e"] = e2e
+    if not args.no_extras:
+        line["general_A"] = time_shape(K, torch, dev, stream, cfg, peak, general_A=True)
+        line["configs"] = {}
+        for ci in (1, 2, 4):
+            if ci == cfg.cfg_id:
+                continue
+            try:
+                line["configs"][str(ci)] = time_shape(K, torch, dev, stream, synth.CONFIGS[ci], peak)
+            except Exception as exc:
+                line["configs"][str(ci)] = {"error": str(exc)}
     if not args.no_cpu_baseline and world >= 1:
-        line["cpu_baseline"] = time_oracle(cfg, host)
+        line["cpu_baseline"] = cpu_baseline(cfg, host)
     print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()

@@ -78,8 +78,9 @@ enum {
                                  parameter [D][N] like A instead of io_dtype [batch][L][N], and dB is float32 [D][N],
                                  summed over batch and time.  Generic kernels.                                    */
   SSM_FLAG_STATIC_C = 512u,   /* the same for C and dC                                                            */
-  SSM_FLAG_TEST_WITHHOLD = 16u /* test hook for the bounded waits: the tuned backward kernel never publishes its
-                                 hand-off flags and polls only 1000 times, so every dependent tile gives up and
+  SSM_FLAG_TEST_WITHHOLD = 16u /* test hook for the bounded waits: the tuned backward kernel shares channel groups
+                                 between neighbouring warps whatever the shape, never publishes a hand-off flag and
+                                 polls only 1000 times, so every warp that continues a group gives up and
                                  ssm_scan_check_status reports SSM_ERR_TIMEOUT; the gradients are then undefined  */
 };
 
@@ -212,11 +213,13 @@ SSM_API ssm_status_t ssm_scan_bwd_state(const ssm_problem_t* p, const void* x, c
                                         void* stream /* cudaStream_t */);
 
 /*
- * Reads back whether the last ssm_scan_bwd on this workspace completed.  The tuned backward kernel passes the adjoint
- * from one tile of a channel group to the next through a hand-off buffer and waits (with a bounded number of polls)
- * for the tile it depends on; if such a wait ever gives up, every block stops and an abort word is left in the
- * workspace.  This call synchronises `stream`, copies that word to the host and returns SSM_ERR_TIMEOUT if it is set
- * (the gradients of that call are then incomplete), SSM_OK otherwise.  `p` and `workspace` must be those of the call.
+ * Reads back whether the last ssm_scan_fwd* / ssm_scan_bwd* call on this workspace completed.  The tuned kernels give
+ * every resident warp an equal share of the (channel group, time) work; where a share ends inside a channel group, the
+ * next warp continues that group and first waits (with a bounded number of polls) for the state or adjoint the warp
+ * before it hands over through the workspace.  If such a wait ever gives up, the waiting warps stop and a status word
+ * (the first word of every non-empty workspace) is set.  This call synchronises `stream`, copies that word to the host
+ * and returns SSM_ERR_TIMEOUT if it is set (the results of that call are then incomplete), SSM_OK otherwise.  `p` and
+ * `workspace` must be those of the call.
  */
 SSM_API ssm_status_t ssm_scan_check_status(const ssm_problem_t* p, const void* workspace, void* stream /* cudaStream_t */);
 
@@ -281,6 +284,15 @@ SSM_API const char* ssm_status_string(ssm_status_t s);
  */
 SSM_API ssm_status_t ssm_scan_plan(const ssm_problem_t* p, int32_t* n_segments, int32_t* segment_steps,
                            int32_t* channels_per_block, int32_t* states_per_thread);
+
+/*
+ * The same for the backward pass, which decides about its time split on its own terms (Appendix D, chunking; the
+ * checkpoint states do not depend on the split): number of time segments, steps per segment, and the number of
+ * channels whose dB / dC terms are summed before they leave a kernel as a partial sum.  Any output pointer may be NULL.
+ * Host-only; launches nothing.
+ */
+SSM_API ssm_status_t ssm_scan_bwd_plan(const ssm_problem_t* p, int32_t* n_segments, int32_t* segment_steps,
+                                       int32_t* channels_per_group);
 
 #ifdef __cplusplus
 }

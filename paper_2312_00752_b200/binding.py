@@ -22,7 +22,7 @@ SSM_FLAG_STATIC_B, SSM_FLAG_STATIC_C = 256, 512
 
 EXPORTED_SYMBOLS = (
     "ssm_scan_fwd_workspace_bytes", "ssm_scan_bwd_workspace_bytes", "ssm_scan_saved_state_bytes",
-    "ssm_scan_checkpoint_steps", "ssm_scan_fwd", "ssm_scan_bwd", "ssm_status_string", "ssm_scan_plan",
+    "ssm_scan_checkpoint_steps", "ssm_scan_fwd", "ssm_scan_bwd", "ssm_status_string", "ssm_scan_plan", "ssm_scan_bwd_plan",
     "ssm_scan_fwd_static", "ssm_scan_check_status", "ssm_scan_fwd_state", "ssm_step",
     "ssm_scan_fwd_fused_dt", "ssm_scan_bwd_fused_dt", "ssm_scan_host_arena_bytes", "ssm_scan_fwd_bwd_host",
     "ssm_scan_bwd_state", "ssm_scan_bwd_fused_dt_state", "ssm_conv1d_fwd", "ssm_conv1d_bwd_workspace_bytes", "ssm_conv1d_bwd",
@@ -77,6 +77,8 @@ def load_library() -> ctypes.CDLL:
     lib.ssm_status_string.argtypes = [ctypes.c_int]
     lib.ssm_scan_plan.restype = ctypes.c_int
     lib.ssm_scan_plan.argtypes = [P] + [ctypes.POINTER(ctypes.c_int32)] * 4
+    lib.ssm_scan_bwd_plan.restype = ctypes.c_int
+    lib.ssm_scan_bwd_plan.argtypes = [P] + [ctypes.POINTER(ctypes.c_int32)] * 3
     lib.ssm_scan_fwd.restype = ctypes.c_int
     lib.ssm_scan_fwd.argtypes = [P] + [vp] * 9 + [vp, sz, vp]
     lib.ssm_scan_bwd.restype = ctypes.c_int
@@ -176,6 +178,13 @@ def plan(problem: ssm_problem_t) -> dict:
     v = [ctypes.c_int32() for _ in range(4)]
     _check(lib.ssm_scan_plan(ctypes.byref(problem), *[ctypes.byref(c) for c in v]), "ssm_scan_plan")
     return dict(zip(("n_segments", "segment_steps", "channels_per_block", "states_per_thread"), [c.value for c in v]))
+
+
+def bwd_plan(problem: ssm_problem_t) -> dict:
+    lib = load_library()
+    v = [ctypes.c_int32() for _ in range(3)]
+    _check(lib.ssm_scan_bwd_plan(ctypes.byref(problem), *[ctypes.byref(c) for c in v]), "ssm_scan_bwd_plan")
+    return dict(zip(("n_segments", "segment_steps", "channels_per_group"), [c.value for c in v]))
 
 
 def checkpoint_steps() -> int:

@@ -289,6 +289,17 @@ ssm_status_t ssm_scan_plan(const ssm_problem_t* p, int32_t* n_segments, int32_t*
   return SSM_OK;
 }
 
+ssm_status_t ssm_scan_bwd_plan(const ssm_problem_t* p, int32_t* n_segments, int32_t* segment_steps,
+                               int32_t* channels_per_group) {
+  const ssm_status_t st = validate_problem(p);
+  if (st != SSM_OK) return st;
+  const Plan pl = make_bwd_plan(*p);
+  if (n_segments) *n_segments = pl.nseg;
+  if (segment_steps) *segment_steps = pl.seg_steps;
+  if (channels_per_group) *channels_per_group = pl.bwd_ch;
+  return SSM_OK;
+}
+
 static ssm_status_t fwd_impl(const ssm_problem_t* p, const void* x, const void* delta, const float* delta_bias,
                              const float* A, const void* B, const void* C, const float* D_skip, const void* z,
                              const float* h0, void* out, float* h_last, void* saved_states, void* workspace,
