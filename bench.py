@@ -31,8 +31,8 @@ FALLBACK_HBM_GBS = 6650.0
 # DRAM bytes (read + write) of one launch of the dominant kernel of each direction from ncu captures at the bench
 # workload itself (profiles/ssm_bwd_warp_kernel_mamba2p8b_layer.md, profiles/ssm_fwd_warp_kernel_mamba2p8b_layer.md);
 # None where no capture exists.
-NCU_TRAFFIC_BYTES = {3: 703.1e6 + 395.5e6}
-NCU_TRAFFIC_BYTES_FWD = {3: 262.5e6 + 371.1e6}
+NCU_TRAFFIC_BYTES = {3: 705.7e6 + 395.8e6}
+NCU_TRAFFIC_BYTES_FWD = {3: 264.0e6 + 369.8e6}
 
 
 def parse_args():
@@ -41,6 +41,9 @@ def parse_args():
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--config", type=int, default=3, help="index into the five synthetic workloads")
+    ap.add_argument("--L", type=int, default=0, help="override the sequence length of the workload (profiling captures "
+                                                     "of the long-sequence path on a shortened copy)")
+    ap.add_argument("--D", type=int, default=0, help="override the channel count of the workload")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--general-A", action="store_true", help="perturb A so that no row is an arithmetic progression")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -542,6 +545,8 @@ def main():
     args = parse_args()
     from paper_2312_00752_b200 import synth
     cfg = synth.CONFIGS[args.config]
+    if args.L or args.D:
+        cfg = cfg.scaled(L=args.L or cfg.L, D=args.D or cfg.D, name=cfg.name + " (resized)")
     if args.impl == "reference":
         run_reference(args, cfg)
     else:

@@ -60,7 +60,10 @@ typedef enum {
   SSM_ERR_UNSUPPORTED = 2,  /* N or dtype outside the supported set                                             */
   SSM_ERR_WORKSPACE = 3,    /* workspace null / misaligned / smaller than the query reports                     */
   SSM_ERR_CUDA = 4,         /* a CUDA runtime call or a kernel launch failed                                    */
-  SSM_ERR_TIMEOUT = 5       /* a bounded device-side wait gave up (reported by ssm_scan_check_status)           */
+  SSM_ERR_TIMEOUT = 5,      /* a bounded device-side wait gave up (reported by ssm_scan_check_status)           */
+  SSM_ERR_BOUNDS = 6        /* bounds-checking build only: a tuned kernel computed a tile row or a global row /
+                               channel outside its range; the access was clamped or skipped, nothing faulted
+                               (reported by ssm_scan_check_status)                                              */
 } ssm_status_t;
 
 typedef enum { SSM_F32 = 0, SSM_BF16 = 1 } ssm_dtype_t;
@@ -219,7 +222,9 @@ SSM_API ssm_status_t ssm_scan_bwd_state(const ssm_problem_t* p, const void* x, c
  * before it hands over through the workspace.  If such a wait ever gives up, the waiting warps stop and a status word
  * (the first word of every non-empty workspace) is set.  This call synchronises `stream`, copies that word to the host
  * and returns SSM_ERR_TIMEOUT if it is set (the results of that call are then incomplete), SSM_OK otherwise.  `p` and
- * `workspace` must be those of the call.
+ * `workspace` must be those of the call.  A library built with -DSSM_DEBUG_BOUNDS (the stand-in for a memory checker:
+ * every tile row index and every global row / channel offset of the tuned kernels is range-checked, a bad one is
+ * clamped or its access skipped, nothing traps) reports a violation here as SSM_ERR_BOUNDS.
  */
 SSM_API ssm_status_t ssm_scan_check_status(const ssm_problem_t* p, const void* workspace, void* stream /* cudaStream_t */);
 

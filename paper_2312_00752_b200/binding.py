@@ -59,12 +59,14 @@ def load_library() -> ctypes.CDLL:
     global _lib
     if _lib is not None:
         return _lib
-    if _build.is_stale() and shutil.which(os.environ.get("NVCC", "nvcc")):
-        _build.build_library()
-    if not os.path.exists(_build.LIB_PATH):
-        raise SsmScanError(f"{_build.LIB_PATH} is missing and nvcc is not available to build it; "
-                           "there is no fallback path")
-    lib = ctypes.CDLL(_build.LIB_PATH)
+    path = os.environ.get("SSM_SCAN_LIBRARY")    # e.g. the bounds-checking build (build.DEBUG_LIB_PATH)
+    if path is None:
+        if _build.is_stale() and shutil.which(os.environ.get("NVCC", "nvcc")):
+            _build.build_library()
+        path = _build.LIB_PATH
+    if not os.path.exists(path):
+        raise SsmScanError(f"{path} is missing and nvcc is not available to build it; there is no fallback path")
+    lib = ctypes.CDLL(path)
     P = ctypes.POINTER(ssm_problem_t)
     vp, sz = ctypes.c_void_p, ctypes.c_size_t
     for name in ("ssm_scan_fwd_workspace_bytes", "ssm_scan_bwd_workspace_bytes", "ssm_scan_saved_state_bytes",

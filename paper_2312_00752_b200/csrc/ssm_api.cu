@@ -261,6 +261,7 @@ const char* ssm_status_string(ssm_status_t s) {
     case SSM_ERR_WORKSPACE: return "SSM_ERR_WORKSPACE: workspace missing, misaligned or too small";
     case SSM_ERR_CUDA: return "SSM_ERR_CUDA: a CUDA call or kernel launch failed";
     case SSM_ERR_TIMEOUT: return "SSM_ERR_TIMEOUT: a bounded device-side wait gave up";
+    case SSM_ERR_BOUNDS: return "SSM_ERR_BOUNDS: an index left its range (bounds-checking build)";
     default: return "unknown ssm_status_t";
   }
 }
@@ -274,7 +275,7 @@ ssm_status_t ssm_scan_check_status(const ssm_problem_t* p, const void* workspace
   if (cudaMemcpyAsync(&word, workspace, sizeof(int), cudaMemcpyDeviceToHost, s) != cudaSuccess)
     return SSM_ERR_CUDA;
   if (cudaStreamSynchronize(s) != cudaSuccess) return SSM_ERR_CUDA;
-  return word != 0 ? SSM_ERR_TIMEOUT : SSM_OK;
+  return word == 0 ? SSM_OK : (word == 2 ? SSM_ERR_BOUNDS : SSM_ERR_TIMEOUT);
 }
 
 ssm_status_t ssm_scan_plan(const ssm_problem_t* p, int32_t* n_segments, int32_t* segment_steps,

@@ -65,12 +65,6 @@ struct BwdWarpSmem {
   float4 red[kRB][32][S / 2];    // dB / dC terms of 4 steps: [step][lane][dB float4s | dC float4s], swizzled
 };
 
-#ifdef SSM_DEBUG_BOUNDS
-#define SSM_BROW(r, abort_ptr) \
-  (((unsigned)(r) < (unsigned)kBT) ? (r) : (((abort_ptr) != nullptr ? atomicExch((abort_ptr), 2) : 0), 0))
-#else
-#define SSM_BROW(r, abort_ptr) (r)
-#endif
 
 template <int S, int CPT_>
 struct Lane {
@@ -217,14 +211,14 @@ __device__ __forceinline__ void sub_block(const Lane<S, CPT>& ln, ChainRegs<S, C
     float dt[kSB][CPT], u[kSB][CPT];
 #pragma unroll
     for (int t = 0; t < kSB; ++t) {
-      const int r = SSM_BROW(r0 + t, abort_word);
+      const int r = SSM_TILE_ROW(r0 + t, kBT, abort_word);
       if constexpr (SP) ln.pick_row(tdF + r * CW, dt[t]);
       else ln.unpack_row(td + r * WPR, dt[t]);
       ln.unpack_row(tx + r * WPR, u[t]);
     }
 #pragma unroll
     for (int t = 0; t < kSB; ++t) {
-      const int r = SSM_BROW(r0 + t, abort_word);
+      const int r = SSM_TILE_ROW(r0 + t, kBT, abort_word);
       float2 Bv[H];
       ln.load_states_f(tfB + r * 16, Bv);
 #pragma unroll
@@ -244,7 +238,7 @@ __device__ __forceinline__ void sub_block(const Lane<S, CPT>& ln, ChainRegs<S, C
 #pragma unroll
   for (int m = kSB / 2 - 1; m >= 0; --m) {
     // ======== odd step t1 = 2m + 1: its state is hist[m]; its w = mu h_{t-1} waits for the even step's state
-    const int r1 = SSM_BROW(r0 + 2 * m + 1, abort_word);
+    const int r1 = SSM_TILE_ROW(r0 + 2 * m + 1, kBT, abort_word);
     float dt1[CPT], u1[CPT], ds1[CPT];
     if constexpr (SP) ln.pick_row(tdF + r1 * CW, dt1);
     else ln.unpack_row(td + r1 * WPR, dt1);
@@ -308,7 +302,7 @@ __device__ __forceinline__ void sub_block(const Lane<S, CPT>& ln, ChainRegs<S, C
     }
 
     // ======== even step t0 = 2m: its state is rebuilt from the one before it
-    const int r0e = SSM_BROW(r0 + 2 * m, abort_word);
+    const int r0e = SSM_TILE_ROW(r0 + 2 * m, kBT, abort_word);
     float dt0[CPT], u0[CPT], ds0[CPT];
     if constexpr (SP) ln.pick_row(tdF + r0e * CW, dt0);
     else ln.unpack_row(td + r0e * WPR, dt0);
@@ -446,7 +440,8 @@ __device__ __forceinline__ void sub_block(const Lane<S, CPT>& ln, ChainRegs<S, C
         else { acc.x += t4.x; acc.y += t4.y; acc.z += t4.z; acc.w += t4.w; }
       }
       const int row = r0 + 2 * m + s;
-      if (row < nlive) *reinterpret_cast<float4*>((which ? part_dC : part_dB) + (size_t)row * 16 + n0) = acc;
+      if (row < nlive && SSM_IN_RANGE(row < kBT && n0 + 4 <= 16, abort_word))
+        *reinterpret_cast<float4*>((which ? part_dC : part_dB) + (size_t)row * 16 + n0) = acc;
       __syncwarp();
     }
   }
@@ -680,7 +675,8 @@ __global__ void __launch_bounds__(kBwdWarps * 32, (CPT == 16 / S) ? 2 : 3)
       for (int k = 0; k < (XCH + 31) / 32; ++k) {
         const int c = lane + 32 * k;
         const int tt = c / CPR, cc = c % CPR;
-        if ((XCH % 32 == 0 || c < XCH) && d_w + cc * 8 < D && tt < nlive) {
+        if ((XCH % 32 == 0 || c < XCH) && d_w + cc * 8 < D && tt < nlive &&
+            SSM_IN_RANGE(row0 + tt < (size_t)p.batch * p.L && d_w + cc * 8 + 8 <= D, sc.abort)) {
           const size_t go = (row0 + tt) * D + d_w + cc * 8;
           *reinterpret_cast<uint4*>(gdx + go) = *reinterpret_cast<const uint4*>(&sm.ox[tt][cc * 4]);
           *reinterpret_cast<uint4*>(gdd + go) = *reinterpret_cast<const uint4*>(&sm.od[tt][cc * 4]);

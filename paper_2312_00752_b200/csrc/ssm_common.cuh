@@ -169,6 +169,19 @@ enum BwdMode { kBwdFull = 0, kBwdLocal = 1 };
 
 // ---------------------------------------------------------------------------------------------- device helpers
 #ifdef __CUDACC__
+// Bounds-checking build (-DSSM_DEBUG_BOUNDS; a memory checker is not available on the GPUs this is developed on): the
+// tuned kernels range-check every tile row index (clamped to row 0 on violation) and every global row / channel offset
+// they store to (the store is skipped), and record a violation as the value 2 in the status word of the workspace.
+// Nothing traps or asserts, so a bad index can be found on a small case without losing the context.
+#ifdef SSM_DEBUG_BOUNDS
+#define SSM_TILE_ROW(r, limit, status) \
+  (((unsigned)(r) < (unsigned)(limit)) ? (r) : (((status) != nullptr ? atomicExch((status), 2) : 0), 0))
+#define SSM_IN_RANGE(cond, status) ((cond) ? true : (((status) != nullptr ? atomicExch((status), 2) : 0), false))
+#else
+#define SSM_TILE_ROW(r, limit, status) (r)
+#define SSM_IN_RANGE(cond, status) true
+#endif
+
 __device__ __forceinline__ float ex2_approx(float v) {
   float r;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(v));

@@ -55,13 +55,6 @@ struct FwdWarpSmem {
 
 __device__ __forceinline__ void cp_async_wait_but_one() { asm volatile("cp.async.wait_group 1;" ::: "memory"); }
 
-#ifdef SSM_DEBUG_BOUNDS
-// Debug build: every tile-row index is checked; a violation is clamped and recorded in the abort word (value 2).
-#define SSM_ROW(r, limit, abort_ptr) \
-  (((unsigned)(r) < (unsigned)(limit)) ? (r) : (((abort_ptr) != nullptr ? atomicExch((abort_ptr), 2) : 0), 0))
-#else
-#define SSM_ROW(r, limit, abort_ptr) (r)
-#endif
 
 }  // namespace
 
@@ -290,7 +283,7 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32) ssm_fwd_warp_kernel(const
         float2 af[AP ? 1 : GB][AP ? 1 : CPT][AP ? 1 : H];          // general A: all decays
 #pragma unroll
         for (int t = 0; t < GB; ++t) {
-          const int r = SSM_ROW(r0 + gb * GB + t, kWT, sc.abort);
+          const int r = SSM_TILE_ROW(r0 + gb * GB + t, kWT, sc.abort);
           if constexpr (SP) pick_row(sm.dF[r], dt[t]);
           else unpack_row(sm.d[st][r], dt[t]);
           unpack_row(sm.x[st][r], u[t]);
@@ -316,7 +309,7 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32) ssm_fwd_warp_kernel(const
         // prepared one step ahead of the recurrence that consumes it
         float2 aN[2][CPT][H], bxN[2][CPT][H], CvN[2][FULL ? H : 1];
         auto front = [&](int t, float2 (&aF)[CPT][H], float2 (&bxF)[CPT][H], float2 (&CvF)[FULL ? H : 1]) {
-          const int r = SSM_ROW(r0 + gb * GB + t, kWT, sc.abort);
+          const int r = SSM_TILE_ROW(r0 + gb * GB + t, kWT, sc.abort);
           float2 Bv[H];
           if constexpr (BCW) {
             load_states_f(sm.fB[r], Bv);
@@ -394,7 +387,7 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32) ssm_fwd_warp_kernel(const
         if constexpr (FULL) {
 #pragma unroll
           for (int t = 0; t < GB; ++t) {
-            const int r = SSM_ROW(r0 + gb * GB + t, kWT, sc.abort);
+            const int r = SSM_TILE_ROW(r0 + gb * GB + t, kWT, sc.abort);
             const float s = fmaf(Dk, u[t][0], ytot[t]);
             // without z its tile is zero-filled: silu(0) = 0, and gate_off = 1 takes its place
             const float hz = 0.5f * zf[t];
@@ -444,7 +437,7 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32) ssm_fwd_warp_kernel(const
       for (int sb = 0; sb < kWT / kSub; ++sb) {
         const int ts = t0 + sb * kSub;
         if (ts >= t_to) break;
-        if (!SUMMARY && p.ckpt != nullptr && valid) {
+        if (!SUMMARY && p.ckpt != nullptr && valid && SSM_IN_RANGE(ts / kCkptSteps < p.nck && ts < p.L, sc.abort)) {
 #pragma unroll
           for (int q = 0; q < CPT; ++q)
 #pragma unroll
@@ -461,7 +454,8 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32) ssm_fwd_warp_kernel(const
 #pragma unroll
         for (int k = 0; k < 4; ++k) {
           const int tt = xrow + 8 * k;
-          if (xcol_ok && t0 + tt < t_to)
+          if (xcol_ok && t0 + tt < t_to &&
+              SSM_IN_RANGE(xo + (size_t)k * 8 * D + 8 <= (size_t)p.batch * p.L * D && d_w + xcc * 8 + 8 <= D, sc.abort))
             *reinterpret_cast<uint4*>(gout + xo + (size_t)k * 8 * D) = *reinterpret_cast<const uint4*>(&sm.o[tt][xcc * 4]);
         }
       }
