@@ -175,10 +175,13 @@ __device__ __forceinline__ void decays(float dt, const float2 (&A2)[H], float a0
 }
 
 // Per-thread state that lives along a chain
-template <int S, int CPT>
+template <int S, int CPT, bool ZOH>
 struct ChainRegs {
   static constexpr int H = S / 2;
   float2 A2[CPT][H];    // A * log2(e)
+  // ZOH: B-bar = E B with the input gain E = (a - 1) / A (Eq. 4), and E = delta where A = 0: 1 / A (0 where A = 0) and
+  // the indicator of A = 0
+  float2 invA[ZOH ? CPT : 1][ZOH ? H : 1], zeroA[ZOH ? CPT : 1][ZOH ? H : 1];
   float a0s[CPT], rs[CPT];
   float2 mu[CPT][H];    // adjoint flowing backwards in time
   float2 dA[CPT][H];
@@ -186,8 +189,8 @@ struct ChainRegs {
 };
 
 // One sub-block of 8 steps: rows [r0, r0 + 8) of the tile; nlive = rows of the tile inside the segment.
-template <int S, int CPT, bool SP, bool AP>
-__device__ __forceinline__ void sub_block(const Lane<S, CPT>& ln, ChainRegs<S, CPT>& cr, int r0, int nlive, float gate_on,
+template <int S, int CPT, bool SP, bool AP, bool ZOH>
+__device__ __forceinline__ void sub_block(const Lane<S, CPT>& ln, ChainRegs<S, CPT, ZOH>& cr, int r0, int nlive, float gate_on,
                                           bool softplus, const uint32_t* tx, const uint32_t* td, const float* tfB,
                                           const float* tfC, const float* tds, const float* tgp, const float* tdF,
                                           const float4* tck, uint32_t* tox, uint32_t* tod, uint32_t* toz, float4* tred,
@@ -196,6 +199,16 @@ __device__ __forceinline__ void sub_block(const Lane<S, CPT>& ln, ChainRegs<S, C
   constexpr int LPC = LN::LPC, H = LN::H, V = LN::V, CW = LN::CW, WPR = CW / 2;
   constexpr bool OWN = LN::OWN;
   const int lane = ln.lane;
+  // ZOH input gain E = (a - 1) / A (delta where A = 0) and its derivative dE/dA = (delta a - E) / A (delta^2 / 2 where
+  // A = 0); dE/ddelta = a
+  auto gain = [&](int q, int k, float2 a, float dtq) {
+    return f2fma(f2fma(a, f2dup(1.f), f2dup(-1.f)), cr.invA[ZOH ? q : 0][ZOH ? k : 0],
+                 f2mul(cr.zeroA[ZOH ? q : 0][ZOH ? k : 0], f2dup(dtq)));
+  };
+  auto gain_dA = [&](int q, int k, float2 a, float2 E, float dtq) {
+    return f2fma(f2fma(f2dup(dtq), a, f2mul(E, f2dup(-1.f))), cr.invA[ZOH ? q : 0][ZOH ? k : 0],
+                 f2mul(cr.zeroA[ZOH ? q : 0][ZOH ? k : 0], f2dup(0.5f * dtq * dtq)));
+  };
   // ---- forward sweep from the checkpoint: the states after the odd steps stay in registers
   float2 hist[kSB / 2][CPT][H];
   {
@@ -228,7 +241,8 @@ __device__ __forceinline__ void sub_block(const Lane<S, CPT>& ln, ChainRegs<S, C
         const float2 du2 = f2dup(dt[t][q] * u[t][q]);
 #pragma unroll
         for (int k = 0; k < H; ++k) {
-          h[q][k] = f2fma(a[k], h[q][k], f2mul(du2, Bv[k]));
+          const float2 bx = ZOH ? f2mul(f2mul(gain(q, k, a[k], dt[t][q]), f2dup(u[t][q])), Bv[k]) : f2mul(du2, Bv[k]);
+          h[q][k] = f2fma(a[k], h[q][k], bx);
           if (t & 1) hist[t >> 1][q][k] = h[q][k];
         }
       }
@@ -247,7 +261,7 @@ __device__ __forceinline__ void sub_block(const Lane<S, CPT>& ln, ChainRegs<S, C
     const float gp1 = tgp[r1 * CW + ln.co];
     float raw1 = 0.f;
     if constexpr (SP) raw1 = __uint_as_float((uint32_t)reinterpret_cast<const uint16_t*>(td + r1 * WPR)[ln.co] << 16);
-    float y1[CPT], lb1[CPT];
+    float y1[CPT], lb1[CPT], mb1[ZOH ? CPT : 1];   // mb: sum mu B (ZOH: the step-size gradient through E)
     {
       float2 Bv[H], Cv[H];
       ln.load_states_f(tfB + r1 * 16, Bv);
@@ -257,25 +271,35 @@ __device__ __forceinline__ void sub_block(const Lane<S, CPT>& ln, ChainRegs<S, C
       for (int q = 0; q < CPT; ++q) {
         float2 a[H];
         decays<H, AP>(dt1[q], cr.A2[q], cr.a0s[q], cr.rs[q], a);
-        const float2 ds2 = f2dup(ds1[q]), du2 = f2dup(dt1[q] * u1[q]);
-        float2 yv = make_float2(0.f, 0.f), lb = yv;
+        // with ZOH the input weight of a state is E x instead of delta x: lw = lam E takes the place of lam below
+        const float2 ds2 = f2dup(ds1[q]), du2 = f2dup(ZOH ? u1[q] : dt1[q] * u1[q]);
+        float2 yv = make_float2(0.f, 0.f), lb = yv, mb = yv;
 #pragma unroll
         for (int k = 0; k < H; ++k) {
           const float2 hc = hist[m][q][k];
           const float2 lam = f2fma(Cv[k], ds2, cr.mu[q][k]);
+          float2 lw = lam;
+          if constexpr (ZOH) {
+            const float2 E = gain(q, k, a[k], dt1[q]);
+            lw = f2mul(lam, E);
+            // dE/dA adds lam (dE/dA) B x to dA
+            cr.dA[q][k] = f2fma(f2mul(lam, gain_dA(q, k, a[k], E, dt1[q])), f2mul(Bv[k], f2dup(u1[q])), cr.dA[q][k]);
+          }
           if (q == 0) {
             dCt[k] = f2mul(ds2, hc);
-            dBt[k] = f2mul(lam, du2);
+            dBt[k] = f2mul(lw, du2);
           } else {
             dCt[k] = f2fma(ds2, hc, dCt[k]);
-            dBt[k] = f2fma(lam, du2, dBt[k]);
+            dBt[k] = f2fma(lw, du2, dBt[k]);
           }
-          lb = f2fma(lam, Bv[k], lb);
+          lb = f2fma(lw, Bv[k], lb);
           yv = f2fma(Cv[k], hc, yv);
           cr.mu[q][k] = f2mul(a[k], lam);
+          if constexpr (ZOH) mb = f2fma(cr.mu[q][k], Bv[k], mb);
         }
         y1[q] = yv.x + yv.y;
         lb1[q] = lb.x + lb.y;
+        if constexpr (ZOH) mb1[q] = mb.x + mb.y;
       }
       // dB / dC terms of this step into the transposing buffer (swizzled: conflict-free 16-byte stores)
       float4* rrow = tred + ((2 * m + 1) & (kRB - 1)) * 32 * V + lane * V;
@@ -294,11 +318,13 @@ __device__ __forceinline__ void sub_block(const Lane<S, CPT>& ln, ChainRegs<S, C
           if ((q & (2 * mm - 1)) == 0) {
             y1[q] += __shfl_xor_sync(0xffffffffu, y1[q + mm], mm);
             lb1[q] += __shfl_xor_sync(0xffffffffu, lb1[q + mm], mm);
+            if constexpr (ZOH) mb1[q] += __shfl_xor_sync(0xffffffffu, mb1[q + mm], mm);
           }
       }
     } else {
       y1[0] += __shfl_xor_sync(0xffffffffu, y1[0], 1);
       lb1[0] += __shfl_xor_sync(0xffffffffu, lb1[0], 1);
+      if constexpr (ZOH) mb1[0] += __shfl_xor_sync(0xffffffffu, mb1[0], 1);
     }
 
     // ======== even step t0 = 2m: its state is rebuilt from the one before it
@@ -311,7 +337,7 @@ __device__ __forceinline__ void sub_block(const Lane<S, CPT>& ln, ChainRegs<S, C
     const float gp0 = tgp[r0e * CW + ln.co];
     float raw0 = 0.f;
     if constexpr (SP) raw0 = __uint_as_float((uint32_t)reinterpret_cast<const uint16_t*>(td + r0e * WPR)[ln.co] << 16);
-    float y0[CPT], lb0[CPT], wa0[CPT], wa1[CPT];
+    float y0[CPT], lb0[CPT], wa0[CPT], wa1[CPT], mb0[ZOH ? CPT : 1];
     {
       float2 Bv[H], Cv[H];
       ln.load_states_f(tfB + r0e * 16, Bv);
@@ -321,8 +347,8 @@ __device__ __forceinline__ void sub_block(const Lane<S, CPT>& ln, ChainRegs<S, C
       for (int q = 0; q < CPT; ++q) {
         float2 a[H];
         decays<H, AP>(dt0[q], cr.A2[q], cr.a0s[q], cr.rs[q], a);
-        const float2 ds2 = f2dup(ds0[q]), du2 = f2dup(dt0[q] * u0[q]), dt02 = f2dup(dt0[q]), dt12 = f2dup(dt1[q]);
-        float2 yv = make_float2(0.f, 0.f), lb = yv, w0a = yv, w1a = yv;
+        const float2 ds2 = f2dup(ds0[q]), du2 = f2dup(ZOH ? u0[q] : dt0[q] * u0[q]), dt02 = f2dup(dt0[q]), dt12 = f2dup(dt1[q]);
+        float2 yv = make_float2(0.f, 0.f), lb = yv, w0a = yv, w1a = yv, mb = yv;
 #pragma unroll
         for (int k = 0; k < H; ++k) {
           float2 hpp;   // the state before the even step: the history entry before, or the checkpoint
@@ -332,21 +358,29 @@ __device__ __forceinline__ void sub_block(const Lane<S, CPT>& ln, ChainRegs<S, C
             const float4 v = tck[(q * (S / 4) + (k >> 1)) * 32 + lane];
             hpp = (k & 1) ? make_float2(v.z, v.w) : make_float2(v.x, v.y);
           }
-          const float2 he = f2fma(a[k], hpp, f2mul(du2, Bv[k]));      // h after the even step
+          float2 E = make_float2(0.f, 0.f);
+          if constexpr (ZOH) E = gain(q, k, a[k], dt0[q]);
+          const float2 he = f2fma(a[k], hpp, f2mul(ZOH ? f2mul(E, du2) : du2, Bv[k]));      // h after the even step
           const float2 w1 = f2mul(cr.mu[q][k], he);                   // the odd step's w = mu_{t1} h_{t1 - 1}
           w1a = f2fma(w1, cr.A2[q][k], w1a);
           cr.dA[q][k] = f2fma(w1, dt12, cr.dA[q][k]);
           const float2 lam = f2fma(Cv[k], ds2, cr.mu[q][k]);
+          float2 lw = lam;
+          if constexpr (ZOH) {
+            lw = f2mul(lam, E);
+            cr.dA[q][k] = f2fma(f2mul(lam, gain_dA(q, k, a[k], E, dt0[q])), f2mul(Bv[k], f2dup(u0[q])), cr.dA[q][k]);
+          }
           if (q == 0) {
             dCt[k] = f2mul(ds2, he);
-            dBt[k] = f2mul(lam, du2);
+            dBt[k] = f2mul(lw, du2);
           } else {
             dCt[k] = f2fma(ds2, he, dCt[k]);
-            dBt[k] = f2fma(lam, du2, dBt[k]);
+            dBt[k] = f2fma(lw, du2, dBt[k]);
           }
-          lb = f2fma(lam, Bv[k], lb);
+          lb = f2fma(lw, Bv[k], lb);
           yv = f2fma(Cv[k], he, yv);
           cr.mu[q][k] = f2mul(a[k], lam);
+          if constexpr (ZOH) mb = f2fma(cr.mu[q][k], Bv[k], mb);
           const float2 w0 = f2mul(cr.mu[q][k], hpp);
           w0a = f2fma(w0, cr.A2[q][k], w0a);
           cr.dA[q][k] = f2fma(w0, dt02, cr.dA[q][k]);
@@ -355,6 +389,7 @@ __device__ __forceinline__ void sub_block(const Lane<S, CPT>& ln, ChainRegs<S, C
         lb0[q] = lb.x + lb.y;
         wa0[q] = w0a.x + w0a.y;
         wa1[q] = w1a.x + w1a.y;
+        if constexpr (ZOH) mb0[q] = mb.x + mb.y;
       }
       float4* rrow = tred + ((2 * m) & (kRB - 1)) * 32 * V + lane * V;
       const int swz = (lane / (8 / V)) & (V - 1);
@@ -374,17 +409,19 @@ __device__ __forceinline__ void sub_block(const Lane<S, CPT>& ln, ChainRegs<S, C
             lb0[q] += __shfl_xor_sync(0xffffffffu, lb0[q + mm], mm);
             wa0[q] += __shfl_xor_sync(0xffffffffu, wa0[q + mm], mm);
             wa1[q] += __shfl_xor_sync(0xffffffffu, wa1[q + mm], mm);
+            if constexpr (ZOH) mb0[q] += __shfl_xor_sync(0xffffffffu, mb0[q + mm], mm);
           }
       }
       // ---- finish both steps of the pair for this lane's own channel
       const float dz1 = gp1 * fmaf(cr.Dk, u1[0], y1[0]);
-      const float dx1 = fmaf(dt1[0], lb1[0], ds1[0] * cr.Dk);
+      // default rule: dx = delta sum lam B, ddelta = x sum lam B + sum w A; ZOH: dx = sum lam E B, ddelta = x sum mu B + sum w A
+      const float dx1 = ZOH ? fmaf(ds1[0], cr.Dk, lb1[0]) : fmaf(dt1[0], lb1[0], ds1[0] * cr.Dk);
       const float dz0 = gp0 * fmaf(cr.Dk, u0[0], y0[0]);
-      const float dx0 = fmaf(dt0[0], lb0[0], ds0[0] * cr.Dk);
+      const float dx0 = ZOH ? fmaf(ds0[0], cr.Dk, lb0[0]) : fmaf(dt0[0], lb0[0], ds0[0] * cr.Dk);
       cr.dD = fmaf(ds1[0], u1[0], cr.dD);
       cr.dD = fmaf(ds0[0], u0[0], cr.dD);
-      float dd1 = fmaf(u1[0], lb1[0], wa1[0] * kInvLog2e);
-      float dd0 = fmaf(u0[0], lb0[0], wa0[0] * kInvLog2e);
+      float dd1 = fmaf(u1[0], ZOH ? mb1[0] : lb1[0], wa1[0] * kInvLog2e);
+      float dd0 = fmaf(u0[0], ZOH ? mb0[0] : lb0[0], wa0[0] * kInvLog2e);
       if constexpr (SP) {
         // the gradient goes to the pre-activation v: d softplus(v) / dv = sigmoid(v); the bias gets the sum over time
         if (softplus) {
@@ -406,15 +443,16 @@ __device__ __forceinline__ void sub_block(const Lane<S, CPT>& ln, ChainRegs<S, C
       lb0[0] += __shfl_xor_sync(0xffffffffu, lb0[0], 1);
       wa0[0] += __shfl_xor_sync(0xffffffffu, wa0[0], 1);
       wa1[0] += __shfl_xor_sync(0xffffffffu, wa1[0], 1);
+      if constexpr (ZOH) mb0[0] += __shfl_xor_sync(0xffffffffu, mb0[0], 1);
       const bool odd = ln.j != 0;
       const float ym = odd ? y1[0] : y0[0], lbm = odd ? lb1[0] : lb0[0], wam = odd ? wa1[0] : wa0[0];
       const float um = odd ? u1[0] : u0[0], dtm = odd ? dt1[0] : dt0[0], dsm = odd ? ds1[0] : ds0[0];
       const float gpm = odd ? gp1 : gp0;
       const int rm = odd ? r1 : r0e;
       const float dzm = gpm * fmaf(cr.Dk, um, ym);
-      const float dxm = fmaf(dtm, lbm, dsm * cr.Dk);
+      const float dxm = ZOH ? fmaf(dsm, cr.Dk, lbm) : fmaf(dtm, lbm, dsm * cr.Dk);
       cr.dD = fmaf(dsm, um, cr.dD);
-      float ddm = fmaf(um, lbm, wam * kInvLog2e);
+      float ddm = fmaf(um, ZOH ? (odd ? mb1[0] : mb0[0]) : lbm, wam * kInvLog2e);
       if constexpr (SP) {
         if (softplus) ddm *= sigmoid_fast((odd ? raw1 : raw0) + cr.bias_own);
         if (r0 + 2 * m + (odd ? 1 : 0) < nlive) cr.dbias += ddm;
@@ -449,7 +487,7 @@ __device__ __forceinline__ void sub_block(const Lane<S, CPT>& ln, ChainRegs<S, C
 
 }  // namespace
 
-template <int S, int CPT, bool SP>
+template <int S, int CPT, bool SP, bool ZOH>
 __global__ void __launch_bounds__(kBwdWarps * 32, (CPT == 16 / S) ? 2 : 3)
     ssm_bwd_warp_kernel(const BwdParams p, const WarpSched sc) {
   using LN = Lane<S, CPT>;
@@ -541,7 +579,7 @@ __global__ void __launch_bounds__(kBwdWarps * 32, (CPT == 16 / S) ? 2 : 3)
     issue_tile(tile_hi, 0);
 
     // ---- per-thread constants and carried values
-    ChainRegs<S, CPT> cr;
+    ChainRegs<S, CPT, ZOH> cr;
     bool ap = !p.general_A;
 #pragma unroll
     for (int q = 0; q < CPT; ++q) {
@@ -557,7 +595,15 @@ __global__ void __launch_bounds__(kBwdWarps * 32, (CPT == 16 / S) ? 2 : 3)
 #pragma unroll
       for (int k = 2; k < S; ++k) ap = ap && fabsf(av[k] - (av[0] + (float)k * step)) <= tol;
 #pragma unroll
-      for (int k = 0; k < H; ++k) cr.A2[q][k] = make_float2(av[2 * k] * kLog2e, av[2 * k + 1] * kLog2e);
+      for (int k = 0; k < H; ++k) {
+        cr.A2[q][k] = make_float2(av[2 * k] * kLog2e, av[2 * k + 1] * kLog2e);
+        if constexpr (ZOH) {
+          auto inv = [](float v) { return v != 0.f ? 1.f / v : 0.f; };
+          auto isz = [](float v) { return v != 0.f ? 0.f : 1.f; };
+          cr.invA[q][k] = make_float2(inv(av[2 * k]), inv(av[2 * k + 1]));
+          cr.zeroA[q][k] = make_float2(isz(av[2 * k]), isz(av[2 * k + 1]));
+        }
+      }
       cr.a0s[q] = cr.A2[q][0].x;
       cr.rs[q] = cr.A2[q][0].y - cr.A2[q][0].x;
     }
@@ -659,12 +705,12 @@ __global__ void __launch_bounds__(kBwdWarps * 32, (CPT == 16 / S) ? 2 : 3)
       for (int sb = kBT / kSB - 1; sb >= 0; --sb) {
         if (sb * kSB >= nlive) continue;   // a sub-block of identity steps
         if (ap)
-          sub_block<S, CPT, SP, true>(ln, cr, sb * kSB, nlive, has_z ? 1.f : 0.f, p.softplus != 0, &sm.x[st][0][0],
+          sub_block<S, CPT, SP, true, ZOH>(ln, cr, sb * kSB, nlive, has_z ? 1.f : 0.f, p.softplus != 0, &sm.x[st][0][0],
                                       &sm.d[st][0][0], &sm.fB[0][0], &sm.fC[0][0], &sm.ds[0][0], &sm.gp[0][0], &sm.dF[0][0],
                                       &sm.ck[st][sb][0][0], &sm.ox[0][0], &sm.od[0][0], &sm.oz[0][0], &sm.red[0][0][0],
                                       part_dB, part_dC, sc.abort);
         else
-          sub_block<S, CPT, SP, false>(ln, cr, sb * kSB, nlive, has_z ? 1.f : 0.f, p.softplus != 0, &sm.x[st][0][0],
+          sub_block<S, CPT, SP, false, ZOH>(ln, cr, sb * kSB, nlive, has_z ? 1.f : 0.f, p.softplus != 0, &sm.x[st][0][0],
                                        &sm.d[st][0][0], &sm.fB[0][0], &sm.fC[0][0], &sm.ds[0][0], &sm.gp[0][0], &sm.dF[0][0],
                                        &sm.ck[st][sb][0][0], &sm.ox[0][0], &sm.od[0][0], &sm.oz[0][0], &sm.red[0][0][0],
                                        part_dB, part_dC, sc.abort);
@@ -734,11 +780,11 @@ __global__ void __launch_bounds__(kBwdWarps * 32, (CPT == 16 / S) ? 2 : 3)
 
 namespace {
 
-template <int S, int CPT, bool SP>
+template <int S, int CPT, bool SP, bool ZOH>
 cudaError_t launch_bwd_variant(const Plan& plan, const BwdParams& p, cudaStream_t s) {
   constexpr int CW = Lane<S, CPT>::CW;
   const size_t smem = sizeof(BwdWarpSmem<S, CPT, SP>) * kBwdWarps;
-  auto kern = ssm_bwd_warp_kernel<S, CPT, SP>;
+  auto kern = ssm_bwd_warp_kernel<S, CPT, SP, ZOH>;
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
   int dev = 0, sms = 0, per_sm = 0;
@@ -771,7 +817,7 @@ cudaError_t launch_bwd_variant(const Plan& plan, const BwdParams& p, cudaStream_
 
 bool bwd_fast_applicable(const ssm_problem_t& prob, const BwdParams& p) {
   auto al16 = [](const void* q) { return q == nullptr || (reinterpret_cast<uintptr_t>(q) & 15) == 0; };
-  if (p.static_B || p.static_C || p.zoh) return false;  // input-dependent B, C and the default B-bar only
+  if (p.static_B || p.static_C) return false;  // input-dependent B, C only
   return prob.io_dtype == SSM_BF16 && prob.N == 16 && prob.D % 8 == 0 && p.seg_steps % kBT == 0 && al16(p.x) &&
          al16(p.delta) && al16(p.z) && al16(p.B) && al16(p.C) && al16(p.dout) && al16(p.dx) && al16(p.ddelta) &&
          al16(p.dz) && al16(p.A) && al16(p.ckpt) && al16(p.mu_in) && al16(p.dh0) && al16(p.dBC_part) && al16(p.dA_part) &&
@@ -784,9 +830,8 @@ int bwd_fast_channels_per_warp() { return kBwdFastChannels; }
 
 cudaError_t launch_bwd_fast(const Plan& plan, const BwdParams& p, cudaStream_t s) {
   const bool sp = p.softplus || p.delta_bias != nullptr;
-  if (p.groups == (p.D + 15) / 16 && p.groups != (p.D + 31) / 32)
-    return sp ? launch_bwd_variant<8, 1, true>(plan, p, s) : launch_bwd_variant<8, 1, false>(plan, p, s);
-  return sp ? launch_bwd_variant<8, 2, true>(plan, p, s) : launch_bwd_variant<8, 2, false>(plan, p, s);
+  if (p.zoh) return sp ? launch_bwd_variant<8, 2, true, true>(plan, p, s) : launch_bwd_variant<8, 2, false, true>(plan, p, s);
+  return sp ? launch_bwd_variant<8, 2, true, false>(plan, p, s) : launch_bwd_variant<8, 2, false, false>(plan, p, s);
 }
 
 }  // namespace ssm
