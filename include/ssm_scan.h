@@ -12,14 +12,14 @@
  *     out[b,t,d] = s[t] * z[b,t,d] / (1 + exp(-z[b,t,d]))                    SiLU gate
  *
  * B-bar is delta*B unless SSM_FLAG_ZOH_BBAR asks for the zero-order-hold expression of Eq. 4.  delta is the positive
- * step size, i.e. the value AFTER the softplus of Algorithm 2 step 4 (the *_fused_dt calls take the pre-activation).  The (batch, L, D, N) tensors a, B-bar and h never exist in device
- * memory (Section 3.3); long sequences are split in time and the state is carried between the pieces
- * (Appendix D, "we split the sequences into chunks").  The backward pass recomputes the states from saved or
+ * step size, i.e. the value AFTER the softplus of Algorithm 2 step 4 (the *_fused_dt calls take the pre-activation).
+ * The (batch, L, D, N) tensors a, B-bar and h never exist in device memory (Section 3.3); long sequences are split in
+ * time and the state is carried between the pieces (the chunked scan of Appendix D).  The backward pass recomputes the states from saved or
  * rebuilt checkpoint states instead of reading them (Section 3.3 and Appendix D, recomputation).
  *
  * Conventions common to all entry points
- *   - Every pointer except `p` is DEVICE memory owned by the caller (ssm_scan_fwd_bwd_host alone takes host buffers); the library never allocates, frees or keeps a
- *     pointer after the call returns.  Scratch memory is the caller's `workspace` (size from the *_workspace_bytes
+ *   - Every pointer except `p` is DEVICE memory owned by the caller (ssm_scan_fwd_bwd_host alone takes host
+ *     buffers); the library never allocates, frees or keeps a pointer after the call returns.  Scratch memory is the caller's `workspace` (size from the *_workspace_bytes
  *     queries; at least 256-byte aligned; contents undefined between calls; calls that overlap on the GPU must not
  *     share a workspace).
  *   - Layouts are dense row-major: x, delta, z, out, dout, dx, ddelta, dz are [batch][L][D]; B, C, dB, dC are
@@ -72,7 +72,7 @@ enum {
   SSM_FLAG_HAS_Z = 1u,        /* z is given: out = s * silu(z); otherwise out = s and dz is not produced        */
   SSM_FLAG_HAS_DSKIP = 2u,    /* D_skip is given; otherwise the skip term is absent and dD is not produced      */
   SSM_FLAG_SAVE_STATES = 4u,  /* forward: also write the checkpoint states that backward starts its recomputation
-                                 from (Appendix D keeps "intermediate scan states" between chunks)             */
+                                 from (the scan states Appendix D keeps between chunks)                          */
   SSM_FLAG_GENERAL_A = 8u,    /* do not use the fast path for rows of A that are arithmetic progressions in n   */
   SSM_FLAG_DELTA_SOFTPLUS = 32u, /* ssm_scan_*_fused_dt: the step size is softplus(delta_pre + delta_bias[d])         */
   SSM_FLAG_ZOH_BBAR = 64u,    /* B-bar = (exp(delta A) - 1) / A * B, the zero-order hold of Eq. 4 (delta * B at A = 0),
@@ -179,7 +179,7 @@ SSM_API ssm_status_t ssm_step(const ssm_problem_t* p, const void* x, const void*
 
 /*
  * Backward: gradients of loss = sum(dout * out) with respect to every input (the adjoint of the four lines at
- * the top; the states are recomputed on chip from checkpoint states, Section 3.3 "recomputation").
+ * the top; the states are recomputed on chip from checkpoint states, Section 3.3, recomputation).
  *   x, delta, A, B, C, D_skip, z   the forward inputs, same rules as above
  *   dout                  in, io_dtype [batch][L][D], required
  *   saved_states          in, float32, as written by ssm_scan_fwd with SSM_FLAG_SAVE_STATES for the same problem and

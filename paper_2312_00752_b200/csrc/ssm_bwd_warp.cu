@@ -179,9 +179,8 @@ template <int S, int CPT, bool ZOH>
 struct ChainRegs {
   static constexpr int H = S / 2;
   float2 A2[CPT][H];    // A * log2(e)
-  // ZOH: B-bar = E B with the input gain E = (a - 1) / A (Eq. 4), and E = delta where A = 0: 1 / A (0 where A = 0) and
-  // the indicator of A = 0
-  float2 invA[ZOH ? CPT : 1][ZOH ? H : 1], zeroA[ZOH ? CPT : 1][ZOH ? H : 1];
+  // ZOH: B-bar = E B with the input gain E = (a - 1) / A (Eq. 4): 1 / A (0 where A = 0)
+  float2 invA[ZOH ? CPT : 1][ZOH ? H : 1];
   float a0s[CPT], rs[CPT];
   float2 mu[CPT][H];    // adjoint flowing backwards in time
   float2 dA[CPT][H];
@@ -199,15 +198,13 @@ __device__ __forceinline__ void sub_block(const Lane<S, CPT>& ln, ChainRegs<S, C
   constexpr int LPC = LN::LPC, H = LN::H, V = LN::V, CW = LN::CW, WPR = CW / 2;
   constexpr bool OWN = LN::OWN;
   const int lane = ln.lane;
-  // ZOH input gain E = (a - 1) / A (delta where A = 0) and its derivative dE/dA = (delta a - E) / A (delta^2 / 2 where
-  // A = 0); dE/ddelta = a
+  // ZOH input gain E = (a - 1) / A and its derivative dE/dA = (delta a - E) / A, each with its series for small
+  // delta A (which covers A = 0); dE/ddelta = a
   auto gain = [&](int q, int k, float2 a, float dtq) {
-    return f2fma(f2fma(a, f2dup(1.f), f2dup(-1.f)), cr.invA[ZOH ? q : 0][ZOH ? k : 0],
-                 f2mul(cr.zeroA[ZOH ? q : 0][ZOH ? k : 0], f2dup(dtq)));
+    return zoh_gain_pair(a, f2mul(f2dup(dtq), cr.A2[q][k]), dtq, cr.invA[ZOH ? q : 0][ZOH ? k : 0]);
   };
   auto gain_dA = [&](int q, int k, float2 a, float2 E, float dtq) {
-    return f2fma(f2fma(f2dup(dtq), a, f2mul(E, f2dup(-1.f))), cr.invA[ZOH ? q : 0][ZOH ? k : 0],
-                 f2mul(cr.zeroA[ZOH ? q : 0][ZOH ? k : 0], f2dup(0.5f * dtq * dtq)));
+    return zoh_gain_dA_pair(a, E, f2mul(f2dup(dtq), cr.A2[q][k]), dtq, cr.invA[ZOH ? q : 0][ZOH ? k : 0]);
   };
   // ---- forward sweep from the checkpoint: the states after the odd steps stay in registers
   float2 hist[kSB / 2][CPT][H];
@@ -599,9 +596,7 @@ __global__ void __launch_bounds__(kBwdWarps * 32, (CPT == 16 / S) ? 2 : 3)
         cr.A2[q][k] = make_float2(av[2 * k] * kLog2e, av[2 * k + 1] * kLog2e);
         if constexpr (ZOH) {
           auto inv = [](float v) { return v != 0.f ? 1.f / v : 0.f; };
-          auto isz = [](float v) { return v != 0.f ? 0.f : 1.f; };
           cr.invA[q][k] = make_float2(inv(av[2 * k]), inv(av[2 * k + 1]));
-          cr.zeroA[q][k] = make_float2(isz(av[2 * k]), isz(av[2 * k + 1]));
         }
       }
       cr.a0s[q] = cr.A2[q][0].x;

@@ -1,5 +1,5 @@
-// Carrying the state across time segments (Appendix D: "we split the sequences into chunks ... as long as we have
-// the intermediate scan states, we can continue the scan with the next chunk").
+// Carrying the state across time segments (Appendix D: a sequence too long for on-chip memory is scanned chunk by
+// chunk, each chunk continuing from the scan state the previous one ended in).
 //
 // A segment g that starts from a zero state ends in a local state e_g, and multiplies whatever state it was given by
 // P_g = prod_t a_t = exp(A_n * sum_{t in g} delta_t).  The true state before segment g+1 is therefore

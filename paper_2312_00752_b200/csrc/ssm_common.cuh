@@ -342,6 +342,37 @@ __device__ __forceinline__ float zoh_gain_dA(float dt, float A, float a, float E
   return __fdividef(fmaf(dt, a, -E), A);
 }
 
+// The same two quantities for a pair of states in the tuned kernels (bf16 io), without a branch.  `a` are the decays
+// the kernel has anyway, y2 = dt * A * log2(e), invA = 1 / A (0 where A = 0).  The closed forms (a - 1) / A and
+// (dt a - E) / A lose all their digits as dt A -> 0 (a is rounded to 2^-24 next to 1), so for |dt A| < 1/4 the series
+// in y = dt A take over; they also cover A = 0 (E = dt, dE/dA = dt^2 / 2).
+__device__ __forceinline__ float2 zoh_gain_pair(float2 a, float2 y2, float dt, float2 invA) {
+  constexpr float kLn2 = 0.6931471805599453f;
+  constexpr float c1 = kLn2 / 2.f, c2 = kLn2 * kLn2 / 6.f, c3 = kLn2 * kLn2 * kLn2 / 24.f,
+                  c4 = kLn2 * kLn2 * kLn2 * kLn2 / 120.f;
+  float2 g = f2fma(y2, f2dup(c4), f2dup(c3));
+  g = f2fma(y2, g, f2dup(c2));
+  g = f2fma(y2, g, f2dup(c1));
+  g = f2fma(y2, g, f2dup(1.f));
+  const float2 Es = f2mul(f2dup(dt), g);
+  const float2 Ec = f2mul(f2fma(a, f2dup(1.f), f2dup(-1.f)), invA);
+  constexpr float kSmall = 0.25f * kLog2e;
+  return make_float2(fabsf(y2.x) < kSmall ? Es.x : Ec.x, fabsf(y2.y) < kSmall ? Es.y : Ec.y);
+}
+__device__ __forceinline__ float2 zoh_gain_dA_pair(float2 a, float2 E, float2 y2, float dt, float2 invA) {
+  constexpr float kLn2 = 0.6931471805599453f;
+  constexpr float c1 = kLn2 / 3.f, c2 = kLn2 * kLn2 / 8.f, c3 = kLn2 * kLn2 * kLn2 / 30.f,
+                  c4 = kLn2 * kLn2 * kLn2 * kLn2 / 144.f;
+  float2 g = f2fma(y2, f2dup(c4), f2dup(c3));
+  g = f2fma(y2, g, f2dup(c2));
+  g = f2fma(y2, g, f2dup(c1));
+  g = f2fma(y2, g, f2dup(0.5f));
+  const float2 Gs = f2mul(f2dup(dt * dt), g);
+  const float2 Gc = f2mul(f2fma(f2dup(dt), a, f2mul(E, f2dup(-1.f))), invA);
+  constexpr float kSmall = 0.25f * kLog2e;
+  return make_float2(fabsf(y2.x) < kSmall ? Gs.x : Gc.x, fabsf(y2.y) < kSmall ? Gs.y : Gc.y);
+}
+
 // tanh through the hardware unit (one special-function operation; relative error about 2^-11: bf16 io only)
 __device__ __forceinline__ float tanh_approx(float v) {
   float r;

@@ -24,7 +24,6 @@
 // Discretization.  a = 2^(delta * A * log2 e) with the hardware ex2.  When the S values of A a thread owns form an
 // arithmetic progression (as in the S4D-Real initialisation A_n = -(n+1)) the S decays come from two exponentials,
 // a_k = a_0 r^k; the test is made per warp at run time and can be disabled by SSM_FLAG_GENERAL_A.
-#include <cstdlib>
 #include <type_traits>
 
 #include "ssm_common.cuh"
@@ -201,7 +200,7 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32) ssm_fwd_warp_kernel(const
     auto chan = [&](int q) { return c_grp + (j ^ q); };
     float2 A2[CPT][H];    // A * log2(e)
     float2 h[CPT][H];
-    float2 invA[ZOH ? CPT : 1][ZOH ? H : 1], zeroA[ZOH ? CPT : 1][ZOH ? H : 1];
+    float2 invA[ZOH ? CPT : 1][ZOH ? H : 1];   // ZOH: 1 / A (0 where A = 0)
     float a0s[CPT], rs[CPT];
     bool ap = !p.general_A;
 #pragma unroll
@@ -222,9 +221,7 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32) ssm_fwd_warp_kernel(const
         A2[q][k] = make_float2(av[2 * k] * kLog2e, av[2 * k + 1] * kLog2e);
         if (ZOH) {
           auto inv = [](float v) { return v != 0.f ? 1.f / v : 0.f; };
-          auto isz = [](float v) { return v != 0.f ? 0.f : 1.f; };
           invA[q][k] = make_float2(inv(av[2 * k]), inv(av[2 * k + 1]));
-          zeroA[q][k] = make_float2(isz(av[2 * k]), isz(av[2 * k + 1]));
         }
       }
       a0s[q] = A2[q][0].x;
@@ -344,9 +341,8 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32) ssm_fwd_warp_kernel(const
 #pragma unroll
             for (int k = 0; k < H; ++k) {
               if constexpr (ZOH) {
-                // B-bar = E B with the input gain E = (a - 1) / A (Eq. 4), and E = delta where A = 0
-                const float2 E =
-                    f2fma(f2fma(a[k], f2dup(1.f), f2dup(-1.f)), invA[q][k], f2mul(zeroA[q][k], f2dup(dt[t][q])));
+                // B-bar = E B with the input gain E = (a - 1) / A (Eq. 4; E = delta at A = 0, a series for small delta A)
+                const float2 E = zoh_gain_pair(a[k], f2mul(f2dup(dt[t][q]), A2[q][k]), dt[t][q], invA[q][k]);
                 bxF[q][k] = f2mul(f2mul(E, f2dup(u[t][q])), Bv[k]);
               } else {
                 bxF[q][k] = f2mul(du2, Bv[k]);
@@ -501,10 +497,7 @@ namespace {
 
 template <int S, int MODE, bool SP, bool ZOH, bool BCW>
 cudaError_t launch_variant_w(const Plan& plan, const FwdParams& p, cudaStream_t s) {
-  size_t smem = sizeof(FwdWarpSmem<MODE == kFwdFull, SP, BCW>) * kWarpsPerBlock;
-#ifdef SSM_DEV_TUNING
-  if (const char* e = getenv("SSM_FWD_SMEM")) smem = (size_t)atoi(e);
-#endif
+  const size_t smem = sizeof(FwdWarpSmem<MODE == kFwdFull, SP, BCW>) * kWarpsPerBlock;
   auto kern = ssm_fwd_warp_kernel<S, MODE, SP, ZOH, BCW>;
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
@@ -531,9 +524,8 @@ cudaError_t launch_variant_w(const Plan& plan, const FwdParams& p, cudaStream_t 
 
 template <int S, int MODE, bool SP, bool ZOH>
 cudaError_t launch_variant(const Plan& plan, const FwdParams& p, cudaStream_t s) {
-#ifdef SSM_DEV_TUNING
-  if (getenv("SSM_FWD_PACKED")) return launch_variant_w<S, MODE, SP, ZOH, false>(plan, p, s);
-#endif
+  // B and C widened to float once per tile (BCW): measured faster than unpacking bf16 in the step loop at 16 states
+  // per thread.
   return launch_variant_w<S, MODE, SP, ZOH, true>(plan, p, s);
 }
 
@@ -583,12 +575,6 @@ int fwd_states_per_thread() { return 16; }
 size_t fwd_handoff_bytes_per_worker() { return sizeof(float4) * kFwdHandoffVec * 32; }
 
 cudaError_t launch_fwd_fast(const Plan& plan, const FwdParams& p, int mode, cudaStream_t s) {
-#ifdef SSM_DEV_TUNING
-  if (const char* e = getenv("SSM_FWD_S")) {
-    if (e[0] == '4') return launch_s<4>(plan, p, mode, s);
-    if (e[0] == '8') return launch_s<8>(plan, p, mode, s);
-  }
-#endif
   return launch_s<16>(plan, p, mode, s);
 }
 

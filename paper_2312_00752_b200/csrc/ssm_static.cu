@@ -53,7 +53,8 @@ extern "C" ssm_status_t ssm_scan_fwd_static(const ssm_problem_t* p, const void* 
   if (need > (size_t)SSM_STATIC_SCRATCH_BYTES) return SSM_ERR_WORKSPACE;
   void* scratch = nullptr;
   if (static_scratch_on_current_device(&scratch) != cudaSuccess) return SSM_ERR_CUDA;
-  // Nothing in the scratch has to start at zero: the summary pass writes every segment end state and step-size sum,
+  // The scratch needs no preparation here: ssm_scan_fwd clears the status word and the hand-off flags at its head on
+  // the caller's stream (memsets, no allocation), the summary pass writes every segment end state and step-size sum,
   // and the carry pass writes every segment start state, before any of them is read.
   return ssm_scan_fwd(p, x, delta, A, B, C, D_skip, z, out, saved_states, scratch, (size_t)SSM_STATIC_SCRATCH_BYTES,
                       stream);

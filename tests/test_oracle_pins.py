@@ -72,8 +72,8 @@ def test_matrix_form(L, N):
 # --------------------------------------------------------------------------------------------------------------
 # Gate (Section 3.4, Figure 3: the SiLU branch multiplies the SSM output): the gated output equals the pre-gate readout
 # times z * sigmoid(z), with the sigmoid taken from a library (scipy's expit) rather than retyped; and, for the
-# backward pass, dz equals dout * s * d/dz [z expit(z)] with the derivative of the library function taken by complex-step
-# free central differences of expit itself.
+# backward pass, dz equals dout * s * d/dz [z expit(z)], the derivative written with the library function alone
+# (expit'(z) = expit(z) expit(-z)).
 def test_gate_is_library_silu():
     from scipy.special import expit
     p = _rand_problem(2, 40, 6, 4)
