@@ -9,6 +9,7 @@ namespace ssm {
 int fwd_channels_per_block(int N);
 int bwd_channels_per_block(int N);
 int fwd_states_per_thread();
+int fwd_fast_channels_per_warp();
 int bwd_fast_channels_per_warp();
 bool bwd_fast_applicable(const ssm_problem_t& prob, const BwdParams& p);
 size_t fwd_handoff_bytes_per_worker();
@@ -55,9 +56,10 @@ Plan make_plan(const ssm_problem_t& p) {
   const long long sub_partitions = 4LL * kNumSMs;
   int nseg = 1;
   if (tuned_shape(p)) {
-    // one warp per 32 channels; a split doubles the forward arithmetic, so only when fewer than half of the
-    // sub-partitions would have a warp, and then into two rounds of chains
-    const long long chains = (long long)p.batch * ((p.D + 31) / 32);
+    // one warp per chain of fwd_fast_channels_per_warp() channels; a split costs half a forward sweep more, so only
+    // when fewer than half of the sub-partitions would have a warp, and then into two rounds of chains
+    const int cw = fwd_fast_channels_per_warp();
+    const long long chains = (long long)p.batch * ((p.D + cw - 1) / cw);
     if (2 * chains < sub_partitions) {
       const long long want = (2 * sub_partitions + chains - 1) / chains;
       const long long max_by_len = std::max(1, p.L / 256);
@@ -114,7 +116,8 @@ struct FwdWorkspace {
 };
 static FwdWorkspace fwd_layout(const ssm_problem_t& p, const Plan& pl) {
   FwdWorkspace w{};
-  w.max_workers = tuned_shape(p) ? shared_workers((long long)p.batch * pl.nseg * ((p.D + 31) / 32)) : 0;
+  const int cw = fwd_fast_channels_per_warp();
+  w.max_workers = tuned_shape(p) ? shared_workers((long long)p.batch * pl.nseg * ((p.D + cw - 1) / cw)) : 0;
   if (pl.nseg == 1 && w.max_workers == 0) return w;
   size_t off = kStatusBytes;
   auto take = [&](size_t bytes) {

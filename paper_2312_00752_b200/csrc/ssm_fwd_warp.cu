@@ -1,25 +1,29 @@
 // Forward selective scan, tuned path: bf16 io, N = 16, D % 8 == 0, 16-byte aligned pointers.
 // Same mathematics and modes as ssm_fwd.cu (Algorithm 2 steps 5-6; Eq. 2a/2b; Eq. 4's A-bar; fused skip and gate).
 //
-// One warp is one worker: it owns 32 adjacent channels of one batch entry and sweeps time sequentially (the path is
-// bound by arithmetic issue, not by memory, so a time-parallel scan inside a block would only add arithmetic); it
-// stages its own tiles and shares nothing with the other warps of its block, so there is no block-wide barrier.
+// One warp is one worker: it owns CW adjacent channels of one batch entry (a chain) and sweeps time sequentially (the
+// path is bound by arithmetic issue, not by memory, so a time-parallel scan inside a block would only add arithmetic);
+// it stages its own tiles and shares nothing with the other warps of its block, so there is no block-wide barrier.
 //
-// Mapping.  A thread holds 16 recurrences as packed float2 pairs (two-wide FP32 instructions): S states of CPT = 16 / S
-// channels, S = 16, 8 or 4.  The LPC = 16 / S lanes of a group cover the 16 states of the group's CPT channels.  Local
-// channel q of lane j (j = lane % LPC) is channel j ^ q of the group, so that the partial readout sums can be exchanged
-// with xor-shuffles without a select, after which lane j holds the total of local channel 0: every lane finishes (skip
-// term, gate, rounding) exactly one channel per step, channel `lane` of the warp's 32.  Larger S means less
-// per-(step, channel) work per recurrence (decays, unpacking, exchanges) and more B / C operands per thread.
+// Mapping.  A thread holds S states of one channel as packed float2 pairs (two-wide FP32 instructions); LPC = 16 / S
+// lanes cover a channel, so a warp covers CW = 32 / LPC channels.
+//   S = 16: one lane per channel, 32 channels per warp; the readout sum over n stays inside the thread.
+//           This is the mapping the library uses.
+//   S = 8:  a lane pair per channel, 16 channels per warp, i.e. twice as many chains of half the arithmetic each, which
+//           puts two warps on every SM sub-partition at the layer shapes.  The two partial readout sums of a channel
+//           are exchanged with one xor-shuffle per PAIR of steps: lane j of the pair ends up with the total of the step
+//           of parity j and finishes (skip term, gate, rounding) that step alone, so nothing of the epilogue is computed
+//           twice.  Measured slower than S = 16 at the layer shapes for arithmetic-progression A (the per-channel work
+//           and the B / C staging are spread over half as many states) and 3 % faster for general A; it is compiled
+//           only with -DSSM_FWD_LANE_PAIR.
 //
 // Staging.  16-byte cp.async copies of x, delta, z, B, C into a three-stage ring of 32-step tiles private to the warp;
-// the output tile is collected in shared memory and written with 16-byte stores.  B and C stay packed bf16 in shared
-// memory and are widened in registers (an ALU-pipe operation per value, next to a saturated FMA pipe), which halves
-// the shared-memory words a thread has to fetch per step.
+// the output tile is collected in shared memory and written with 16-byte stores.  B and C are widened to float once
+// per tile (one row per lane), so the step loop fetches them with 16-byte loads and no conversion.
 //
 // Schedule.  The grid is sized to the warps the GPU holds at once; the linear (chain, tile) space is cut into equal
 // ranges (WarpSched in ssm_common.cuh), so every SM sub-partition gets the same amount of work whatever the ratio of
-// channel groups to warps, at the price of one state hand-off through L2 per worker.
+// chains to warps, at the price of one state hand-off through L2 per worker.
 //
 // Discretization.  a = 2^(delta * A * log2 e) with the hardware ex2.  When the S values of A a thread owns form an
 // arithmetic progression (as in the S4D-Real initialisation A_n = -(n+1)) the S decays come from two exponentials,
@@ -36,37 +40,45 @@ constexpr int kWT = 32;          // steps per tile
 constexpr int kWStages = 3;      // ring stages
 constexpr int kSub = kCkptSteps; // steps per unrolled sub-block: a checkpoint is written at the start of each
 constexpr int kWarpsPerBlock = 4;
-constexpr int kFwdHandoffVec = 5;   // float4 per lane: 16 states, sum of delta
 static_assert(kWT % kSub == 0, "tiles are whole sub-blocks");
 
-template <bool FULL, bool SP, bool BCW>
+template <int CW, bool FULL, bool SP, bool BCW>
 struct FwdWarpSmem {
-  uint32_t x[kWStages][kWT][16];   // bf16 pairs, 32 channels
-  uint32_t d[kWStages][kWT][16];
-  uint32_t z[FULL ? kWStages : 1][FULL ? kWT : 1][16];
-  uint32_t rB[kWStages][kWT][8];   // bf16 pairs, 16 states
-  uint32_t rC[FULL ? kWStages : 1][FULL ? kWT : 1][8];
-  float fB[BCW ? kWT : 1][16];     // BCW: B and C of the current tile widened to float
-  float fC[(BCW && FULL) ? kWT : 1][16];
-  float dF[SP ? kWT : 1][32];      // SP: step sizes after bias and softplus
-  uint32_t o[FULL ? kWT : 1][16];  // output tile (bf16 pairs)
+  uint32_t x[kWStages][kWT][CW / 2];   // bf16 pairs, CW channels
+  uint32_t d[kWStages][kWT][CW / 2];
+  uint32_t z[FULL ? kWStages : 1][FULL ? kWT : 1][CW / 2];
+  // B and C rows are padded (12 and 20 words instead of 8 and 16) so that the one-row-per-lane widening pass of a
+  // tile reads and writes them without bank conflicts
+  uint32_t rB[kWStages][kWT][12];  // bf16 pairs, 16 states
+  uint32_t rC[FULL ? kWStages : 1][FULL ? kWT : 1][12];
+  float fB[BCW ? kWT : 1][20];     // BCW: B and C of the current tile widened to float
+  float fC[(BCW && FULL) ? kWT : 1][20];
+  float dF[SP ? kWT : 1][CW];      // SP: step sizes after bias and softplus
+  uint32_t o[FULL ? kWT : 1][CW / 2];  // output tile (bf16 pairs)
 };
 
 __device__ __forceinline__ void cp_async_wait_but_one() { asm volatile("cp.async.wait_group 1;" ::: "memory"); }
 
+__device__ __forceinline__ float bf16at(const uint32_t* row, int c) {
+  return __uint_as_float((uint32_t)reinterpret_cast<const uint16_t*>(row)[c] << 16);
+}
 
 }  // namespace
 
 template <int S, int MODE, bool SP, bool ZOH, bool BCW>
 __global__ void __launch_bounds__(kWarpsPerBlock * 32) ssm_fwd_warp_kernel(const FwdParams p, const WarpSched sc) {
+  static_assert(S == 16 || S == 8, "one lane or a lane pair per channel");
   constexpr bool FULL = (MODE == kFwdFull);
   constexpr bool SUMMARY = (MODE == kFwdSummary);
-  constexpr int LPC = 16 / S, CPT = LPC, H = S / 2;
-  using Smem = FwdWarpSmem<FULL, SP, BCW>;
+  constexpr int LPC = 16 / S, H = S / 2, CW = 32 / LPC;
+  constexpr int CH = CW / 8;        // 16-byte chunks per tile row of x, delta, z, out
+  constexpr int RP = 32 / CH;       // tile rows a warp covers with one chunk per lane
+  constexpr int HV = S / 4 + 1;     // float4 per lane of a hand-off: S states, sum of delta
+  using Smem = FwdWarpSmem<CW, FULL, SP, BCW>;
   extern __shared__ __align__(16) unsigned char smem_raw[];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   Smem& sm = reinterpret_cast<Smem*>(smem_raw)[warp];
-  const int j = lane % LPC, g = lane / LPC;
+  const int j = lane % LPC, g = lane / LPC;   // g: this lane's channel of the chain, j: which S states of it
   const int D = p.D;
   const bool has_z = FULL && p.z != nullptr;
   const int worker = blockIdx.x * kWarpsPerBlock + warp;
@@ -78,61 +90,16 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32) ssm_fwd_warp_kernel(const
   const __nv_bfloat16* __restrict__ gC = static_cast<const __nv_bfloat16*>(p.C);
   __nv_bfloat16* __restrict__ gout = static_cast<__nv_bfloat16*>(p.out);
 
-  // byte-permute selectors that widen one half of a packed bf16 pair: local channel q of lane j is channel j ^ q
-  const uint32_t sel0 = (j & 1) ? 0x3244u : 0x1044u, sel1 = (j & 1) ? 0x1044u : 0x3244u;
-  // the CPT values of a tile row (32 channels as 16 bf16 pairs) that belong to this thread, by local channel
-  auto unpack_row = [&](const uint32_t* row, float (&v)[CPT]) {
-    if constexpr (CPT == 1) {
-      v[0] = __uint_as_float((uint32_t)reinterpret_cast<const uint16_t*>(row)[lane] << 16);
-    } else if constexpr (CPT == 2) {
-      const uint32_t w = row[g];
-      v[0] = bf16sel(w, sel0);
-      v[1] = bf16sel(w, sel1);
-    } else {
-      const uint2 w = *reinterpret_cast<const uint2*>(row + 2 * g);
-      const uint32_t wa = (j & 2) ? w.y : w.x, wb = (j & 2) ? w.x : w.y;
-      v[0] = bf16sel(wa, sel0);
-      v[1] = bf16sel(wa, sel1);
-      v[2] = bf16sel(wb, sel0);
-      v[3] = bf16sel(wb, sel1);
-    }
-  };
-  // the same from a row of 32 floats
-  auto pick_row = [&](const float* row, float (&v)[CPT]) {
-    if constexpr (CPT == 1) {
-      v[0] = row[lane];
-    } else if constexpr (CPT == 2) {
-      const float2 f = *reinterpret_cast<const float2*>(row + 2 * g);
-      v[0] = (j & 1) ? f.y : f.x;
-      v[1] = (j & 1) ? f.x : f.y;
-    } else {
-      const float4 f = *reinterpret_cast<const float4*>(row + 4 * g);
-      const float a0 = (j & 2) ? f.z : f.x, a1 = (j & 2) ? f.w : f.y, b0 = (j & 2) ? f.x : f.z, b1 = (j & 2) ? f.y : f.w;
-      v[0] = (j & 1) ? a1 : a0;
-      v[1] = (j & 1) ? a0 : a1;
-      v[2] = (j & 1) ? b1 : b0;
-      v[3] = (j & 1) ? b0 : b1;
-    }
-  };
   // this thread's S states of a packed B or C row (16 states as 8 bf16 pairs), widened
   auto load_states = [&](const uint32_t* row, float2 (&v)[H]) {
-    if constexpr (H == 8) {
-      const uint4 a = *reinterpret_cast<const uint4*>(row), b = *reinterpret_cast<const uint4*>(row + 4);
-      const uint32_t w[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
 #pragma unroll
-      for (int k = 0; k < 8; ++k) v[k] = make_float2(bf16lo(w[k]), bf16hi(w[k]));
-    } else if constexpr (H == 4) {
-      const uint4 a = *reinterpret_cast<const uint4*>(row + 4 * j);
+    for (int k = 0; k < H / 4; ++k) {
+      const uint4 a = *reinterpret_cast<const uint4*>(row + H * j + 4 * k);
       const uint32_t w[4] = {a.x, a.y, a.z, a.w};
 #pragma unroll
-      for (int k = 0; k < 4; ++k) v[k] = make_float2(bf16lo(w[k]), bf16hi(w[k]));
-    } else {
-      const uint2 a = *reinterpret_cast<const uint2*>(row + 2 * j);
-      v[0] = make_float2(bf16lo(a.x), bf16hi(a.x));
-      v[1] = make_float2(bf16lo(a.y), bf16hi(a.y));
+      for (int i = 0; i < 4; ++i) v[4 * k + i] = make_float2(bf16lo(w[i]), bf16hi(w[i]));
     }
   };
-
   // the same from a row of 16 floats
   auto load_states_f = [&](const float* row, float2 (&v)[H]) {
 #pragma unroll
@@ -147,11 +114,11 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32) ssm_fwd_warp_kernel(const
   for (int pi = 0; pi < wl.count; ++pi) {
     int chain, from, to;
     get_piece(wl, sc.tiles, pi, chain, from, to);
-    const int groups = (D + 31) / 32;
+    const int groups = (D + CW - 1) / CW;
     const int grp = chain % groups;
     const int bs = chain / groups;
     const int seg = bs % p.nseg, b = bs / p.nseg;
-    const int d_w = grp * 32;
+    const int d_w = grp * CW;
     const int t_seg0 = seg * p.seg_steps;
     const int t_seg_end = min(p.L, t_seg0 + p.seg_steps);
     const int t_from = t_seg0 + from * kWT;
@@ -160,8 +127,8 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32) ssm_fwd_warp_kernel(const
     const bool gives_out = to < sc.tiles;
     const size_t row_from = (size_t)b * p.L + t_from;
 
-    // ---- staging (this lane's chunks of a tile: rows lane / 4 + 8 k of x, delta, z; rows lane / 2 + 16 k of B, C)
-    const int xrow = lane >> 2, xcc = lane & 3;
+    // ---- staging (this lane's chunks of a tile: rows lane / CH + RP k of x, delta, z; rows lane / 2 + 16 k of B, C)
+    const int xrow = lane / CH, xcc = lane % CH;
     const bool xcol_ok = d_w + xcc * 8 < D;
     const size_t xoff = (row_from + xrow) * D + d_w + xcc * 8;
     const int brow = lane >> 1, bhc = lane & 1;
@@ -172,10 +139,10 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32) ssm_fwd_warp_kernel(const
         const int t0 = t_from + i * kWT;
         const size_t xo = xoff + (size_t)i * kWT * D, bo = boff + (size_t)i * kWT * 16;
 #pragma unroll
-        for (int k = 0; k < 4; ++k) {
-          const int tt = xrow + 8 * k;
+        for (int k = 0; k < kWT / RP; ++k) {
+          const int tt = xrow + RP * k;
           const bool ok = xcol_ok && (t0 + tt < t_to);
-          const size_t go = ok ? xo + (size_t)k * 8 * D : 0;
+          const size_t go = ok ? xo + (size_t)k * RP * D : 0;
           cp_async16(&sm.x[st][tt][xcc * 4], gx + go, ok);
           cp_async16(&sm.d[st][tt][xcc * 4], gd + go, ok);
           if (FULL) cp_async16(&sm.z[st][tt][xcc * 4], (has_z ? gz : gx) + go, ok && has_z);
@@ -195,21 +162,19 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32) ssm_fwd_warp_kernel(const
     issue_tile(1);
 
     // ---- per-thread constants and state
-    const int c_grp = d_w + g * CPT;                      // first channel of this lane group (all valid or none)
-    const bool valid = c_grp < D;
-    auto chan = [&](int q) { return c_grp + (j ^ q); };
-    float2 A2[CPT][H];    // A * log2(e)
-    float2 h[CPT][H];
-    float2 invA[ZOH ? CPT : 1][ZOH ? H : 1];   // ZOH: 1 / A (0 where A = 0)
-    float a0s[CPT], rs[CPT];
+    const int c_own = d_w + g;            // this lane's channel
+    const bool valid = c_own < D;
+    float2 A2[H];    // A * log2(e)
+    float2 h[H];
+    float2 invA[ZOH ? H : 1];   // ZOH: 1 / A (0 where A = 0)
+    float a0s, rs;
     bool ap = !p.general_A;
-#pragma unroll
-    for (int q = 0; q < CPT; ++q) {
+    {
       float av[S];
 #pragma unroll
       for (int k = 0; k < S / 4; ++k) {
         float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (valid) a = *reinterpret_cast<const float4*>(p.A + (size_t)chan(q) * 16 + S * j + 4 * k);
+        if (valid) a = *reinterpret_cast<const float4*>(p.A + (size_t)c_own * 16 + S * j + 4 * k);
         av[4 * k] = a.x; av[4 * k + 1] = a.y; av[4 * k + 2] = a.z; av[4 * k + 3] = a.w;
       }
       const float step = av[1] - av[0];
@@ -218,19 +183,20 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32) ssm_fwd_warp_kernel(const
       for (int k = 2; k < S; ++k) ap = ap && fabsf(av[k] - (av[0] + (float)k * step)) <= tol;
 #pragma unroll
       for (int k = 0; k < H; ++k) {
-        A2[q][k] = make_float2(av[2 * k] * kLog2e, av[2 * k + 1] * kLog2e);
+        A2[k] = make_float2(av[2 * k] * kLog2e, av[2 * k + 1] * kLog2e);
         if (ZOH) {
           auto inv = [](float v) { return v != 0.f ? 1.f / v : 0.f; };
-          invA[q][k] = make_float2(inv(av[2 * k]), inv(av[2 * k + 1]));
+          invA[k] = make_float2(inv(av[2 * k]), inv(av[2 * k + 1]));
         }
       }
-      a0s[q] = A2[q][0].x;
-      rs[q] = A2[q][0].y - A2[q][0].x;
+      a0s = A2[0].x;
+      rs = A2[0].y - A2[0].x;
     }
     ap = __all_sync(0xffffffffu, ap);
-    const int c_own = d_w + lane;   // the channel this lane finishes
-    const float Dk = (FULL && p.Dskip != nullptr && c_own < D) ? p.Dskip[c_own] : 0.f;
-    const float bias_own = (SP && p.delta_bias != nullptr && c_own < D) ? p.delta_bias[c_own] : 0.f;
+    const float Dk = (FULL && p.Dskip != nullptr && valid) ? p.Dskip[c_own] : 0.f;
+    // the softplus pass walks the tile with one (row, channel) element per lane: channel lane % CW
+    const int c_prep = d_w + (lane % CW);
+    const float bias_prep = (SP && p.delta_bias != nullptr && c_prep < D) ? p.delta_bias[c_prep] : 0.f;
     float dsum = 0.f;
 
     if (from > 0) {
@@ -239,73 +205,74 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32) ssm_fwd_warp_kernel(const
         cp_async_wait_all();
         return;
       }
-      const float4* hb = sc.handoff + ((size_t)worker * 32 + lane) * kFwdHandoffVec;
-      float4 v[4];
+      const float4* hb = sc.handoff + ((size_t)worker * 32 + lane) * HV;
+      float4 v[S / 4];
 #pragma unroll
-      for (int k = 0; k < 4; ++k) v[k] = __ldcg(hb + k);
-      const float4 dv = __ldcg(hb + 4);
+      for (int k = 0; k < S / 4; ++k) v[k] = __ldcg(hb + k);
+      const float4 dv = __ldcg(hb + S / 4);
       dsum = dv.x;
-      const float* f = reinterpret_cast<const float*>(v);
 #pragma unroll
-      for (int q = 0; q < CPT; ++q)
-#pragma unroll
-        for (int k = 0; k < H; ++k) h[q][k] = make_float2(f[(q * H + k) * 2], f[(q * H + k) * 2 + 1]);
+      for (int k = 0; k < S / 4; ++k) {
+        h[2 * k] = make_float2(v[k].x, v[k].y);
+        h[2 * k + 1] = make_float2(v[k].z, v[k].w);
+      }
     } else {
 #pragma unroll
-      for (int q = 0; q < CPT; ++q) {
-#pragma unroll
-        for (int k = 0; k < S / 4; ++k) {
-          float4 hs = make_float4(0.f, 0.f, 0.f, 0.f);
-          if (valid && p.h_start != nullptr)
-            hs = *reinterpret_cast<const float4*>(p.h_start + (((size_t)b * p.nseg + seg) * D + chan(q)) * 16 + S * j + 4 * k);
-          h[q][2 * k] = make_float2(hs.x, hs.y);
-          h[q][2 * k + 1] = make_float2(hs.z, hs.w);
-        }
+      for (int k = 0; k < S / 4; ++k) {
+        float4 hs = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (valid && p.h_start != nullptr)
+          hs = *reinterpret_cast<const float4*>(p.h_start + (((size_t)b * p.nseg + seg) * D + c_own) * 16 + S * j + 4 * k);
+        h[2 * k] = make_float2(hs.x, hs.y);
+        h[2 * k + 1] = make_float2(hs.z, hs.w);
       }
     }
 
     // ---- one sub-block of kSub steps of tile stage st, rows [r0, r0 + kSub), in batches of GB steps.  A batch runs in
-    // three phases so that a lone warp has independent long-latency work in flight: (1) the step sizes, inputs and
-    // exponentials of all GB steps, (2) the recurrences and readouts, (3) skip term, gate and rounding of the GB
-    // results.  There is no branch inside a batch.
+    // three phases so that a warp has independent long-latency work in flight and no load has to pass an earlier
+    // store: (1) the step sizes, inputs and exponentials of all GB steps, (2) the recurrences and readouts, (3) skip
+    // term, gate and rounding of the results.  There is no branch inside a batch.
     auto compute_sub = [&](int st, int r0, auto ap_tag) {
       constexpr bool AP = decltype(ap_tag)::value;
-      constexpr int GB = AP ? (8 / CPT) : 2;
+      constexpr int GB = AP ? 8 : (S == 16 ? 2 : 4);
+      constexpr int NE = GB / LPC;        // results this lane finishes per batch
       const float gate_off = has_z ? 0.f : 1.f;
 #pragma unroll
       for (int gb = 0; gb < kSub / GB; ++gb) {
-        float dt[GB][CPT], u[GB][CPT], du[GB][CPT];
-        float zf[FULL ? GB : 1];   // loaded before the batch stores anything: a load may not pass an earlier store
-        float e0[AP ? GB : 1][CPT], e1[AP ? GB : 1][CPT];          // AP: first decay and ratio
-        float2 af[AP ? 1 : GB][AP ? 1 : CPT][AP ? 1 : H];          // general A: all decays
+        float dt[GB], u[GB], du[GB];
+        float zf[FULL ? NE : 1];   // loaded before the batch stores anything: a load may not pass an earlier store
+        float e0[AP ? GB : 1], e1[AP ? GB : 1];          // AP: first decay and ratio
+        float2 af[AP ? 1 : GB][AP ? 1 : H];              // general A: all decays
 #pragma unroll
         for (int t = 0; t < GB; ++t) {
           const int r = SSM_TILE_ROW(r0 + gb * GB + t, kWT, sc.abort);
-          if constexpr (SP) pick_row(sm.dF[r], dt[t]);
-          else unpack_row(sm.d[st][r], dt[t]);
-          unpack_row(sm.x[st][r], u[t]);
-          if constexpr (FULL)
-            zf[t] = __uint_as_float((uint32_t)reinterpret_cast<const uint16_t*>(sm.z[st][r])[lane] << 16);
+          if constexpr (SP) dt[t] = sm.dF[r][g];
+          else dt[t] = bf16at(sm.d[st][r], g);
+          u[t] = bf16at(sm.x[st][r], g);
+          du[t] = dt[t] * u[t];
+          if constexpr (AP) {
+            e0[t] = ex2_approx(dt[t] * a0s);
+            e1[t] = ex2_approx(dt[t] * rs);
+          } else {
 #pragma unroll
-          for (int q = 0; q < CPT; ++q) {
-            du[t][q] = dt[t][q] * u[t][q];
-            if constexpr (AP) {
-              e0[t][q] = ex2_approx(dt[t][q] * a0s[q]);
-              e1[t][q] = ex2_approx(dt[t][q] * rs[q]);
-            } else {
-#pragma unroll
-              for (int k = 0; k < H; ++k) {
-                const float2 e = f2mul(f2dup(dt[t][q]), A2[q][k]);
-                af[t][q][k] = make_float2(ex2_approx(e.x), ex2_approx(e.y));
-              }
+            for (int k = 0; k < H; ++k) {
+              const float2 e = f2mul(f2dup(dt[t]), A2[k]);
+              af[t][k] = make_float2(ex2_approx(e.x), ex2_approx(e.y));
             }
           }
-          if constexpr (SUMMARY) dsum += dt[t][0];
+          if constexpr (SUMMARY) dsum += dt[t];
+        }
+        if constexpr (FULL) {
+          // lane j of a channel's LPC lanes finishes the steps t with t % LPC == j
+#pragma unroll
+          for (int m = 0; m < NE; ++m) {
+            const int r = SSM_TILE_ROW(r0 + gb * GB + m * LPC + j, kWT, sc.abort);
+            zf[m] = bf16at(sm.z[st][r], g);
+          }
         }
         // everything of a step that does not depend on the state (B and C of the step, decays, input terms) is
         // prepared one step ahead of the recurrence that consumes it
-        float2 aN[2][CPT][H], bxN[2][CPT][H], CvN[2][FULL ? H : 1];
-        auto front = [&](int t, float2 (&aF)[CPT][H], float2 (&bxF)[CPT][H], float2 (&CvF)[FULL ? H : 1]) {
+        float2 aN[2][H], bxN[2][H], CvN[2][FULL ? H : 1];
+        auto front = [&](int t, float2 (&a)[H], float2 (&bxF)[H], float2 (&CvF)[FULL ? H : 1]) {
           const int r = SSM_TILE_ROW(r0 + gb * GB + t, kWT, sc.abort);
           float2 Bv[H];
           if constexpr (BCW) {
@@ -315,80 +282,71 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32) ssm_fwd_warp_kernel(const
             load_states(sm.rB[st][r], Bv);
             if constexpr (FULL) load_states(sm.rC[st][r], CvF);
           }
+          if constexpr (AP) {
+            const float a0 = e0[t], rr = e1[t];
+            const float r2 = rr * rr;
+            a[0] = make_float2(a0, a0 * rr);
+            a[1] = f2mul(a[0], f2dup(r2));
+            const float r4 = r2 * r2;
+            a[2] = f2mul(a[0], f2dup(r4));
+            a[3] = f2mul(a[1], f2dup(r4));
+            if constexpr (H > 4) {
+              const float r8 = r4 * r4;
 #pragma unroll
-          for (int q = 0; q < CPT; ++q) {
-            float2 (&a)[H] = aF[q];
-            if constexpr (AP) {
-              const float a0 = e0[t][q], rr = e1[t][q];
-              const float r2 = rr * rr;
-              a[0] = make_float2(a0, a0 * rr);
-              if constexpr (H > 1) a[1] = f2mul(a[0], f2dup(r2));
-              if constexpr (H > 2) {
-                const float r4 = r2 * r2;
-                a[2] = f2mul(a[0], f2dup(r4));
-                a[3] = f2mul(a[1], f2dup(r4));
-                if constexpr (H > 4) {
-                  const float r8 = r4 * r4;
-#pragma unroll
-                  for (int k = 0; k < 4; ++k) a[4 + k] = f2mul(a[k], f2dup(r8));
-                }
-              }
-            } else {
-#pragma unroll
-              for (int k = 0; k < H; ++k) a[k] = af[t][q][k];
+              for (int k = 0; k < 4; ++k) a[4 + k] = f2mul(a[k], f2dup(r8));
             }
-            const float2 du2 = f2dup(du[t][q]);
+          } else {
 #pragma unroll
-            for (int k = 0; k < H; ++k) {
-              if constexpr (ZOH) {
-                // B-bar = E B with the input gain E = (a - 1) / A (Eq. 4; E = delta at A = 0, a series for small delta A)
-                const float2 E = zoh_gain_pair(a[k], f2mul(f2dup(dt[t][q]), A2[q][k]), dt[t][q], invA[q][k]);
-                bxF[q][k] = f2mul(f2mul(E, f2dup(u[t][q])), Bv[k]);
-              } else {
-                bxF[q][k] = f2mul(du2, Bv[k]);
-              }
+            for (int k = 0; k < H; ++k) a[k] = af[t][k];
+          }
+          const float2 du2 = f2dup(du[t]);
+#pragma unroll
+          for (int k = 0; k < H; ++k) {
+            if constexpr (ZOH) {
+              // B-bar = E B with the input gain E = (a - 1) / A (Eq. 4; E = delta at A = 0, a series for small delta A)
+              const float2 E = zoh_gain_pair(a[k], f2mul(f2dup(dt[t]), A2[k]), dt[t], invA[k]);
+              bxF[k] = f2mul(f2mul(E, f2dup(u[t])), Bv[k]);
+            } else {
+              bxF[k] = f2mul(du2, Bv[k]);
             }
           }
         };
-        float ytot[GB];
+        float ypart[FULL ? GB : 1];
         front(0, aN[0], bxN[0], CvN[0]);
 #pragma unroll
         for (int t = 0; t < GB; ++t) {
           if (t + 1 < GB) front(t + 1, aN[(t + 1) & 1], bxN[(t + 1) & 1], CvN[(t + 1) & 1]);
-          float y[CPT];
+          float2 yv = make_float2(0.f, 0.f), yw = make_float2(0.f, 0.f);
 #pragma unroll
-          for (int q = 0; q < CPT; ++q) {
-            float2 yv = make_float2(0.f, 0.f), yw = make_float2(0.f, 0.f);
-#pragma unroll
-            for (int k = 0; k < H; ++k) {
-              h[q][k] = f2fma(aN[t & 1][q][k], h[q][k], bxN[t & 1][q][k]);
-              if constexpr (FULL) {
-                if (k & 1) yw = f2fma(CvN[t & 1][k], h[q][k], yw);
-                else yv = f2fma(CvN[t & 1][k], h[q][k], yv);
-              }
+          for (int k = 0; k < H; ++k) {
+            h[k] = f2fma(aN[t & 1][k], h[k], bxN[t & 1][k]);
+            if constexpr (FULL) {
+              if (k & 1) yw = f2fma(CvN[t & 1][k], h[k], yw);
+              else yv = f2fma(CvN[t & 1][k], h[k], yv);
             }
-            if constexpr (FULL) y[q] = (yv.x + yw.x) + (yv.y + yw.y);
           }
-          if constexpr (FULL) {
-            // reduce-scatter over the lane group: afterwards y[0] is the total of this lane's own channel
-#pragma unroll
-            for (int m = 1; m < LPC; m <<= 1) {
-#pragma unroll
-              for (int q = 0; q < CPT; ++q)
-                if ((q & (2 * m - 1)) == 0) y[q] += __shfl_xor_sync(0xffffffffu, y[q + m], m);
-            }
-            ytot[t] = y[0];
-          }
+          if constexpr (FULL) ypart[t] = (yv.x + yw.x) + (yv.y + yw.y);
         }
         if constexpr (FULL) {
 #pragma unroll
-          for (int t = 0; t < GB; ++t) {
-            const int r = SSM_TILE_ROW(r0 + gb * GB + t, kWT, sc.abort);
-            const float s = fmaf(Dk, u[t][0], ytot[t]);
+          for (int m = 0; m < NE; ++m) {
+            float ytot, um;
+            if constexpr (LPC == 1) {
+              ytot = ypart[m];
+              um = u[m];
+            } else {
+              // the pair's partial sums of steps 2m and 2m + 1 cross over: lane j keeps the step of parity j
+              const float keep = j ? ypart[2 * m + 1] : ypart[2 * m];
+              const float send = j ? ypart[2 * m] : ypart[2 * m + 1];
+              ytot = keep + __shfl_xor_sync(0xffffffffu, send, 1);
+              um = j ? u[2 * m + 1] : u[2 * m];
+            }
+            const int r = SSM_TILE_ROW(r0 + gb * GB + m * LPC + j, kWT, sc.abort);
+            const float s = fmaf(Dk, um, ytot);
             // without z its tile is zero-filled: silu(0) = 0, and gate_off = 1 takes its place
-            const float hz = 0.5f * zf[t];
+            const float hz = 0.5f * zf[m];
             const float gate = fmaf(hz, tanh_approx(hz), hz) + gate_off;
-            reinterpret_cast<__nv_bfloat16*>(sm.o[r])[lane] = __float2bfloat16_rn(s * gate);
+            reinterpret_cast<__nv_bfloat16*>(sm.o[r])[g] = __float2bfloat16_rn(s * gate);
           }
         }
       }
@@ -422,10 +380,11 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32) ssm_fwd_warp_kernel(const
         // step sizes of the tile, once per element: pre-activation + bias, softplus; rows past the end stay identity
         // steps (delta = 0)
 #pragma unroll 4
-        for (int r = 0; r < kWT; ++r) {
-          float v = __uint_as_float((uint32_t)reinterpret_cast<const uint16_t*>(sm.d[st][r])[lane] << 16) + bias_own;
+        for (int rr = 0; rr < kWT; rr += 32 / CW) {
+          const int r = rr + lane / CW, c = lane % CW;
+          float v = bf16at(sm.d[st][r], c) + bias_prep;
           if (p.softplus) v = softplus_fast(v);
-          sm.dF[r][lane] = (t0 + r < t_to) ? v : 0.f;
+          sm.dF[r][c] = (t0 + r < t_to) ? v : 0.f;
         }
         __syncwarp();
       }
@@ -435,11 +394,9 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32) ssm_fwd_warp_kernel(const
         if (ts >= t_to) break;
         if (!SUMMARY && p.ckpt != nullptr && valid && SSM_IN_RANGE(ts / kCkptSteps < p.nck && ts < p.L, sc.abort)) {
 #pragma unroll
-          for (int q = 0; q < CPT; ++q)
-#pragma unroll
-            for (int k = 0; k < S / 4; ++k)
-              *reinterpret_cast<float4*>(p.ckpt + (((size_t)b * p.nck + ts / kCkptSteps) * D + chan(q)) * 16 + S * j + 4 * k) =
-                  make_float4(h[q][2 * k].x, h[q][2 * k].y, h[q][2 * k + 1].x, h[q][2 * k + 1].y);
+          for (int k = 0; k < S / 4; ++k)
+            *reinterpret_cast<float4*>(p.ckpt + (((size_t)b * p.nck + ts / kCkptSteps) * D + c_own) * 16 + S * j + 4 * k) =
+                make_float4(h[2 * k].x, h[2 * k].y, h[2 * k + 1].x, h[2 * k + 1].y);
         }
         if (ap) compute_sub(st, sb * kSub, std::true_type{});
         else compute_sub(st, sb * kSub, std::false_type{});
@@ -448,11 +405,11 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32) ssm_fwd_warp_kernel(const
         __syncwarp();
         const size_t xo = xoff + (size_t)i * kWT * D;
 #pragma unroll
-        for (int k = 0; k < 4; ++k) {
-          const int tt = xrow + 8 * k;
+        for (int k = 0; k < kWT / RP; ++k) {
+          const int tt = xrow + RP * k;
           if (xcol_ok && t0 + tt < t_to &&
-              SSM_IN_RANGE(xo + (size_t)k * 8 * D + 8 <= (size_t)p.batch * p.L * D && d_w + xcc * 8 + 8 <= D, sc.abort))
-            *reinterpret_cast<uint4*>(gout + xo + (size_t)k * 8 * D) = *reinterpret_cast<const uint4*>(&sm.o[tt][xcc * 4]);
+              SSM_IN_RANGE(xo + (size_t)k * RP * D + 8 <= (size_t)p.batch * p.L * D && d_w + xcc * 8 + 8 <= D, sc.abort))
+            *reinterpret_cast<uint4*>(gout + xo + (size_t)k * RP * D) = *reinterpret_cast<const uint4*>(&sm.o[tt][xcc * 4]);
         }
       }
     }
@@ -461,18 +418,11 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32) ssm_fwd_warp_kernel(const
 
     if (gives_out) {
       // the rest of this chain belongs to the next worker
-      float4* hb = sc.handoff + ((size_t)(worker + 1) * 32 + lane) * kFwdHandoffVec;
-      float f[16];
+      float4* hb = sc.handoff + ((size_t)(worker + 1) * 32 + lane) * HV;
 #pragma unroll
-      for (int q = 0; q < CPT; ++q)
-#pragma unroll
-        for (int k = 0; k < H; ++k) {
-          f[(q * H + k) * 2] = h[q][k].x;
-          f[(q * H + k) * 2 + 1] = h[q][k].y;
-        }
-#pragma unroll
-      for (int k = 0; k < 4; ++k) __stcg(hb + k, make_float4(f[4 * k], f[4 * k + 1], f[4 * k + 2], f[4 * k + 3]));
-      __stcg(hb + 4, make_float4(dsum, 0.f, 0.f, 0.f));
+      for (int k = 0; k < S / 4; ++k)
+        __stcg(hb + k, make_float4(h[2 * k].x, h[2 * k].y, h[2 * k + 1].x, h[2 * k + 1].y));
+      __stcg(hb + S / 4, make_float4(dsum, 0.f, 0.f, 0.f));
       publish_handoff(sc, worker, lane);
     } else if (valid) {
       float* dst = nullptr;
@@ -480,24 +430,29 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32) ssm_fwd_warp_kernel(const
       if (SUMMARY) dst = p.seg_end + ((size_t)b * p.nseg + seg) * D * 16;
       if (dst != nullptr) {
 #pragma unroll
-        for (int q = 0; q < CPT; ++q)
-#pragma unroll
-          for (int k = 0; k < S / 4; ++k)
-            *reinterpret_cast<float4*>(dst + (size_t)chan(q) * 16 + S * j + 4 * k) =
-                make_float4(h[q][2 * k].x, h[q][2 * k].y, h[q][2 * k + 1].x, h[q][2 * k + 1].y);
+        for (int k = 0; k < S / 4; ++k)
+          *reinterpret_cast<float4*>(dst + (size_t)c_own * 16 + S * j + 4 * k) =
+              make_float4(h[2 * k].x, h[2 * k].y, h[2 * k + 1].x, h[2 * k + 1].y);
       }
-      if (SUMMARY) p.seg_dsum[((size_t)b * p.nseg + seg) * D + c_own] = dsum;
+      if (SUMMARY && j == 0) p.seg_dsum[((size_t)b * p.nseg + seg) * D + c_own] = dsum;
     }
   }
 }
 
 int warp_workers(int chains, int sms, int per_sm, int max_workers);
 
+#ifdef SSM_FWD_LANE_PAIR
+constexpr int kFwdS = 8;   // a lane pair per channel, 16-channel chains
+#else
+constexpr int kFwdS = 16;  // a lane per channel, 32-channel chains
+#endif
+
 namespace {
 
 template <int S, int MODE, bool SP, bool ZOH, bool BCW>
 cudaError_t launch_variant_w(const Plan& plan, const FwdParams& p, cudaStream_t s) {
-  const size_t smem = sizeof(FwdWarpSmem<MODE == kFwdFull, SP, BCW>) * kWarpsPerBlock;
+  constexpr int CW = 2 * S;   // channels per chain
+  const size_t smem = sizeof(FwdWarpSmem<CW, MODE == kFwdFull, SP, BCW>) * kWarpsPerBlock;
   auto kern = ssm_fwd_warp_kernel<S, MODE, SP, ZOH, BCW>;
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
@@ -507,7 +462,7 @@ cudaError_t launch_variant_w(const Plan& plan, const FwdParams& p, cudaStream_t 
   if ((e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, kWarpsPerBlock * 32, smem)) != cudaSuccess) return e;
   if (per_sm < 1) return cudaErrorLaunchOutOfResources;
   WarpSched sc{};
-  sc.chains = p.batch * plan.nseg * ((p.D + 31) / 32);
+  sc.chains = p.batch * plan.nseg * ((p.D + CW - 1) / CW);
   sc.tiles = (plan.seg_steps + kWT - 1) / kWT;
   const bool can_share = p.abort != nullptr && p.flags != nullptr && p.handoff != nullptr;
   sc.workers = warp_workers(sc.chains, sms, per_sm * kWarpsPerBlock, can_share ? p.max_workers : 0);
@@ -571,11 +526,12 @@ bool fwd_fast_applicable(const ssm_problem_t& prob, const FwdParams& p) {
          al16(p.h_last) && al16(p.handoff);
 }
 
-int fwd_states_per_thread() { return 16; }
-size_t fwd_handoff_bytes_per_worker() { return sizeof(float4) * kFwdHandoffVec * 32; }
+int fwd_states_per_thread() { return kFwdS; }
+int fwd_fast_channels_per_warp() { return 2 * kFwdS; }
+size_t fwd_handoff_bytes_per_worker() { return sizeof(float4) * (kFwdS / 4 + 1) * 32; }
 
 cudaError_t launch_fwd_fast(const Plan& plan, const FwdParams& p, int mode, cudaStream_t s) {
-  return launch_s<16>(plan, p, mode, s);
+  return launch_s<kFwdS>(plan, p, mode, s);
 }
 
 }  // namespace ssm
