@@ -36,7 +36,7 @@ static ssm_status_t validate_problem(const ssm_problem_t* p) {
                              SSM_FLAG_DELTA_SOFTPLUS | SSM_FLAG_ZOH_BBAR | SSM_FLAG_STATIC_B | SSM_FLAG_STATIC_C))
     return SSM_ERR_INVALID_ARG;
   if (p->io_dtype != SSM_F32 && p->io_dtype != SSM_BF16) return SSM_ERR_UNSUPPORTED;
-  if (p->N != 1 && p->N != 2 && p->N != 4 && p->N != 8 && p->N != 16) return SSM_ERR_UNSUPPORTED;
+  if (p->N != 1 && p->N != 2 && p->N != 4 && p->N != 8 && p->N != 16 && p->N != 32 && p->N != 64) return SSM_ERR_UNSUPPORTED;
   if (p->batch > 65535) return SSM_ERR_UNSUPPORTED;  // batch is a grid z dimension
   return SSM_OK;
 }
@@ -260,7 +260,7 @@ const char* ssm_status_string(ssm_status_t s) {
   switch (s) {
     case SSM_OK: return "SSM_OK";
     case SSM_ERR_INVALID_ARG: return "SSM_ERR_INVALID_ARG: null or misaligned pointer, bad dimension or flag";
-    case SSM_ERR_UNSUPPORTED: return "SSM_ERR_UNSUPPORTED: N must be 1, 2, 4, 8 or 16 and io_dtype f32 or bf16";
+    case SSM_ERR_UNSUPPORTED: return "SSM_ERR_UNSUPPORTED: N must be a power of two up to 64 and io_dtype f32 or bf16";
     case SSM_ERR_WORKSPACE: return "SSM_ERR_WORKSPACE: workspace missing, misaligned or too small";
     case SSM_ERR_CUDA: return "SSM_ERR_CUDA: a CUDA call or kernel launch failed";
     case SSM_ERR_TIMEOUT: return "SSM_ERR_TIMEOUT: a bounded device-side wait gave up";

@@ -26,7 +26,8 @@ template <int N>
 struct BwdGeom {
   static constexpr int S = N < 4 ? N : 4;
   static constexpr int LPC = N / S;             // lanes per channel
-  static constexpr int CH = 32;                 // channels per block (one per thread group)
+  // channels per block (one per thread group); fewer for N > 16 so that the recomputed states of a tile fit
+  static constexpr int CH = N <= 16 ? 32 : (N == 32 ? 16 : 8);
   static constexpr int THREADS = CH * LPC;
   static constexpr int WARPS = THREADS / 32;
 };
@@ -410,6 +411,8 @@ template <typename IO>
 static cudaError_t launch_bwd_io(const ssm_problem_t& prob, const Plan& plan, const BwdParams& p, int mode,
                                  cudaStream_t s) {
   switch (prob.N) {
+    case 64: return launch_bwd_n<IO, 64>(plan, p, mode, s);
+    case 32: return launch_bwd_n<IO, 32>(plan, p, mode, s);
     case 16: return launch_bwd_n<IO, 16>(plan, p, mode, s);
     case 8: return launch_bwd_n<IO, 8>(plan, p, mode, s);
     case 4: return launch_bwd_n<IO, 4>(plan, p, mode, s);
@@ -419,7 +422,7 @@ static cudaError_t launch_bwd_io(const ssm_problem_t& prob, const Plan& plan, co
   }
 }
 
-int bwd_channels_per_block(int) { return 32; }
+int bwd_channels_per_block(int N) { return N <= 16 ? 32 : (N == 32 ? 16 : 8); }
 
 bool bwd_fast_applicable(const ssm_problem_t& prob, const BwdParams& p);
 cudaError_t launch_bwd_fast(const Plan& plan, const BwdParams& p, cudaStream_t s);

@@ -15,8 +15,9 @@
 
 namespace ssm {
 
-// threads per block: 16 thread groups for N = 16, 32 groups otherwise (keeps the staged tiles below 48 KB)
-__host__ __device__ constexpr int fwd_threads(int N) { return N == 16 ? 64 : 32; }
+// threads per block: 16 thread groups (of N / 4 lanes each) for N >= 16, 32 groups otherwise (keeps the staged tiles
+// below 48 KB)
+__host__ __device__ constexpr int fwd_threads(int N) { return N >= 16 ? 4 * N : 32; }
 constexpr int kFwdTile = 32;  // time steps staged in shared memory at a time
 
 template <typename IO, int N, int CPT, int MODE>
@@ -231,6 +232,8 @@ template <typename IO>
 static cudaError_t launch_fwd_io(const ssm_problem_t& prob, const Plan& plan, const FwdParams& p, int mode,
                                  cudaStream_t s) {
   switch (prob.N) {
+    case 64: return launch_fwd_mode<IO, 64, 2>(plan, p, mode, s);
+    case 32: return launch_fwd_mode<IO, 32, 2>(plan, p, mode, s);
     case 16: return launch_fwd_mode<IO, 16, 2>(plan, p, mode, s);
     case 8: return launch_fwd_mode<IO, 8, 2>(plan, p, mode, s);
     case 4: return launch_fwd_mode<IO, 4, 2>(plan, p, mode, s);

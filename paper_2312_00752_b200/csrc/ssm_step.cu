@@ -77,6 +77,8 @@ template <typename IO>
 static cudaError_t launch_step_io(const StepParams& p, cudaStream_t s) {
   dim3 grid((p.D + 127) / 128, p.batch);
   switch (p.N) {
+    case 64: ssm_step_kernel<IO, 64><<<grid, 128, 0, s>>>(p); break;
+    case 32: ssm_step_kernel<IO, 32><<<grid, 128, 0, s>>>(p); break;
     case 16: ssm_step_kernel<IO, 16><<<grid, 128, 0, s>>>(p); break;
     case 8: ssm_step_kernel<IO, 8><<<grid, 128, 0, s>>>(p); break;
     case 4: ssm_step_kernel<IO, 4><<<grid, 128, 0, s>>>(p); break;

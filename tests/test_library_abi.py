@@ -48,7 +48,7 @@ def test_queries_and_plan():
 
 
 @pytest.mark.parametrize("bad,code", [
-    (dict(N=3), 2), (dict(N=32), 2), (dict(io=5), 2), (dict(L=0), 1), (dict(batch=-1), 1), (dict(flags=1 << 12), 1),
+    (dict(N=3), 2), (dict(N=128), 2), (dict(io=5), 2), (dict(L=0), 1), (dict(batch=-1), 1), (dict(flags=1 << 12), 1),
 ])
 def test_invalid_problems_are_rejected(bad, code):
     lib = K.load_library()
