@@ -231,14 +231,15 @@ def run_reference(args, cfg):
 
 
 # ------------------------------------------------------------------------------------------------ our arm
-def time_shape(K, torch, dev, stream, cfg, peak, general_A=False, reps=None):
+def time_shape(K, torch, dev, stream, cfg, peak, general_A=False, reps=None, zoh=False, complex_state=False):
     """Forward (saving states) and backward times of one more workload, with timing-only inputs drawn on the device
     (same shapes and value ranges as the seeded host recipe); every repetition is timed on its own with CUDA events and
     a buffer larger than L2 is overwritten in between."""
     io_t = torch.bfloat16 if cfg.io == "bf16" else torch.float32
     g = torch.Generator(device=dev)
     g.manual_seed(1234 + cfg.cfg_id)
-    shp, bshp = (cfg.batch, cfg.L, cfg.D), (cfg.batch, cfg.L, cfg.N)
+    shp = (cfg.batch, cfg.L, cfg.D)
+    bshp = (cfg.batch, cfg.L, cfg.N, 2) if complex_state else (cfg.batch, cfg.L, cfg.N)
     rn = lambda shape: torch.randn(shape, generator=g, device=dev, dtype=torch.float32)
     t = {k: rn(shp).to(io_t) for k in ("x", "z", "dout")}
     t["B"], t["C"] = rn(bshp).to(io_t), rn(bshp).to(io_t)
@@ -248,8 +249,12 @@ def time_shape(K, torch, dev, stream, cfg, peak, general_A=False, reps=None):
     A = -(torch.arange(cfg.N, device=dev, dtype=torch.float32) + 1.0).repeat(cfg.D, 1)
     if general_A:
         A = A * (1.0 + 0.01 * rn((cfg.D, cfg.N)))
+    if complex_state:   # S4D-Lin (Section 3.6): A_n = -1/2 + n i as (re, im) pairs
+        A = torch.stack([torch.full((cfg.D, cfg.N), -0.5, device=dev),
+                         torch.arange(cfg.N, device=dev, dtype=torch.float32).repeat(cfg.D, 1)], dim=-1).contiguous()
     Dk = torch.ones(cfg.D, device=dev)
-    prob = K.make_problem(t["x"], t["B"], True, True, save_states=True)
+    opts = dict(zoh=zoh, complex_state=complex_state) if (zoh or complex_state) else {}
+    prob = K.make_problem(t["x"], t["B"], True, True, save_states=True, zoh=zoh, complex_state=complex_state)
     out = torch.empty_like(t["x"])
     saved = torch.empty(K.saved_state_bytes(prob) // 4, dtype=torch.float32, device=dev)
     grads = {"dx": torch.empty_like(t["x"]), "ddelta": torch.empty_like(t["x"]), "dz": torch.empty_like(t["x"]),
@@ -257,9 +262,9 @@ def time_shape(K, torch, dev, stream, cfg, peak, general_A=False, reps=None):
              "dD": torch.empty_like(Dk)}
     flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
     fwd = lambda: K.ssm_scan_fwd(t["x"], t["delta"], A, t["B"], t["C"], Dk, t["z"], save_states=True, out=out,
-                                 saved_states=saved, stream=stream, general_A=general_A)
+                                 saved_states=saved, stream=stream, general_A=general_A, **opts)
     bwd = lambda: K.ssm_scan_bwd(t["x"], t["delta"], A, t["B"], t["C"], Dk, t["z"], t["dout"], saved, outputs=grads,
-                                 stream=stream, general_A=general_A)
+                                 stream=stream, general_A=general_A, **opts)
     reps = reps or (5 if cfg.elements > 2e8 else 12)
     f_ms, b_ms = [], []
     for i in range(3 + reps):
@@ -270,9 +275,15 @@ def time_shape(K, torch, dev, stream, cfg, peak, general_A=False, reps=None):
         if i >= 3:
             f_ms.append(e[0].elapsed_time(e[1])); b_ms.append(e[1].elapsed_time(e[2]))
     fb, bb = algorithmic_bytes(cfg)
+    if complex_state:   # B, C, dB, dC are twice as wide
+        esz = 2 if cfg.io == "bf16" else 4
+        fb += 2 * cfg.batch * cfg.L * cfg.N * esz
+        bb += 4 * cfg.batch * cfg.L * cfg.N * esz
     f, b = statistics.median(f_ms), statistics.median(b_ms)
     res = {"workload": f"config {cfg.cfg_id}: batch {cfg.batch}, L {cfg.L}, D {cfg.D}, N {cfg.N}, {cfg.io} io" +
-                       (", A perturbed (no arithmetic progression: one exponential per state)" if general_A else ""),
+                       (", A perturbed (no arithmetic progression: one exponential per state)" if general_A else "") +
+                       (", zero-order-hold B-bar (SSM_FLAG_ZOH_BBAR)" if zoh else "") +
+                       (", complex state with S4D-Lin A (SSM_FLAG_COMPLEX; plain kernels)" if complex_state else ""),
            "fwd_ms": f, "bwd_ms": b, "fwd_elements_per_s": cfg.elements / (f * 1e-3),
            "bwd_elements_per_s": cfg.elements / (b * 1e-3), "step_elements_per_s": cfg.elements / ((f + b) * 1e-3),
            "fwd_frac_of_hbm_peak": fb / (f * 1e-3) / 1e9 / peak, "bwd_frac_of_hbm_peak": bb / (b * 1e-3) / 1e9 / peak,
@@ -523,6 +534,12 @@ def run_ours(args, cfg):
         line["e2e"] = e2e
     if not args.no_extras:
         line["general_A"] = time_shape(K, torch, dev, stream, cfg, peak, general_A=True)
+        line["variants"] = {}
+        for name, kw in (("zoh", dict(zoh=True)), ("complex_state", dict(complex_state=True))):
+            try:
+                line["variants"][name] = time_shape(K, torch, dev, stream, cfg, peak, reps=5, **kw)
+            except Exception as exc:
+                line["variants"][name] = {"error": str(exc)}
         line["configs"] = {}
         for ci in (1, 2, 4):
             if ci == cfg.cfg_id:

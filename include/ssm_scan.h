@@ -82,6 +82,13 @@ enum {
                                  parameter [D][N] like A instead of io_dtype [batch][L][N], and dB is float32 [D][N],
                                  summed over batch and time.  Generic kernels.                                    */
   SSM_FLAG_STATIC_C = 512u,   /* the same for C and dC                                                            */
+  SSM_FLAG_COMPLEX = 1024u,   /* complex-valued state (Section 3.6): A and dA are float32 [D][N][2], B, C, dB, dC io_dtype
+                                 [batch][L][N][2], every state array (saved_states, h0, h_last, dh_last, dh0, the h of
+                                 ssm_step) float32 [..][N][2], all as interleaved (re, im) pairs; the readout is
+                                 s = 2 Re(sum_n C h) + D_skip x (the N states stand for N conjugate pairs); a gradient
+                                 of a complex quantity holds (dL/dRe, dL/dIm).  N <= 32.  Not combined with
+                                 SSM_FLAG_ZOH_BBAR, SSM_FLAG_STATIC_B / _C, the *_fused_dt calls or
+                                 ssm_scan_fwd_bwd_host (SSM_ERR_UNSUPPORTED).  Plain kernels, no time split.      */
   SSM_FLAG_TEST_WITHHOLD = 16u /* test hook for the bounded waits: the tuned backward kernel shares channel groups
                                  between neighbouring warps whatever the shape, never publishes a hand-off flag and
                                  polls only 1000 times, so every warp that continues a group gives up and

@@ -19,6 +19,7 @@ SSM_FLAG_HAS_Z, SSM_FLAG_HAS_DSKIP, SSM_FLAG_SAVE_STATES, SSM_FLAG_GENERAL_A, SS
 SSM_FLAG_DELTA_SOFTPLUS = 32
 SSM_FLAG_ZOH_BBAR = 64
 SSM_FLAG_STATIC_B, SSM_FLAG_STATIC_C = 256, 512
+SSM_FLAG_COMPLEX = 1024
 
 EXPORTED_SYMBOLS = (
     "ssm_scan_fwd_workspace_bytes", "ssm_scan_bwd_workspace_bytes", "ssm_scan_saved_state_bytes",
@@ -133,13 +134,14 @@ def _io_dtype(t: torch.Tensor) -> int:
 
 def make_problem(x: torch.Tensor, B: torch.Tensor, has_z: bool, has_dskip: bool, save_states: bool = False,
                  general_A: bool = False, zoh: bool = False, static_B: bool = False,
-                 static_C: bool = False) -> ssm_problem_t:
+                 static_C: bool = False, complex_state: bool = False) -> ssm_problem_t:
+    """complex_state: B is (batch, L, N, 2), interleaved (re, im) pairs (SSM_FLAG_COMPLEX)."""
     batch, L, D = x.shape
     flags = (SSM_FLAG_HAS_Z if has_z else 0) | (SSM_FLAG_HAS_DSKIP if has_dskip else 0) \
         | (SSM_FLAG_SAVE_STATES if save_states else 0) | (SSM_FLAG_GENERAL_A if general_A else 0) \
         | (SSM_FLAG_ZOH_BBAR if zoh else 0) | (SSM_FLAG_STATIC_B if static_B else 0) \
-        | (SSM_FLAG_STATIC_C if static_C else 0)
-    return ssm_problem_t(batch, L, D, B.shape[-1], _io_dtype(x), flags)
+        | (SSM_FLAG_STATIC_C if static_C else 0) | (SSM_FLAG_COMPLEX if complex_state else 0)
+    return ssm_problem_t(batch, L, D, B.shape[-2] if complex_state else B.shape[-1], _io_dtype(x), flags)
 
 
 def _dev_ptr(t, name, shape=None, dtype=None):
@@ -206,8 +208,12 @@ def saved_state_bytes(problem: ssm_problem_t) -> int:
 
 
 def ssm_scan_fwd(x, delta, A, B, C, D_skip=None, z=None, *, save_states=False, general_A=False, zoh=False, out=None,
-                 saved_states=None, workspace=None, stream=None, h0=None, h_last=None, static_B=False, static_C=False):
+                 saved_states=None, workspace=None, stream=None, h0=None, h_last=None, static_B=False, static_C=False,
+                 complex_state=False):
     """out = selective_scan(x, delta, A, B, C) (+ D_skip * x) (* silu(z)); see include/ssm_scan.h.
+
+    complex_state=True (SSM_FLAG_COMPLEX): A is float32 (D, N, 2), B and C are io dtype (batch, L, N, 2), h0 / h_last
+    float32 (batch, D, N, 2), all interleaved (re, im) pairs (torch.view_as_real of a complex tensor).
 
     x, delta, z: (batch, L, D) io dtype; B, C: (batch, L, N) io dtype; A: (D, N) float32; D_skip: (D) float32.
     Returns `out`, or `(out, saved_states)` with save_states=True.  Enqueues on `stream` (default: torch's current
@@ -216,11 +222,13 @@ def ssm_scan_fwd(x, delta, A, B, C, D_skip=None, z=None, *, save_states=False, g
     (ssm_scan_fwd_state).
     """
     lib = load_library()
-    prob = make_problem(x, B, z is not None, D_skip is not None, save_states, general_A, zoh, static_B, static_C)
+    prob = make_problem(x, B, z is not None, D_skip is not None, save_states, general_A, zoh, static_B, static_C,
+                        complex_state)
     batch, L, D, N = prob.batch, prob.L, prob.D, prob.N
     io = x.dtype
-    bshape, bdt = ((D, N), torch.float32) if static_B else ((batch, L, N), io)   # static: a parameter like A
-    cshape, cdt = ((D, N), torch.float32) if static_C else ((batch, L, N), io)
+    c2 = (2,) if complex_state else ()
+    bshape, bdt = ((D, N), torch.float32) if static_B else ((batch, L, N) + c2, io)   # static: a parameter like A
+    cshape, cdt = ((D, N), torch.float32) if static_C else ((batch, L, N) + c2, io)
     if out is None:
         out = torch.empty_like(x)
     if save_states and saved_states is None:
@@ -230,10 +238,10 @@ def ssm_scan_fwd(x, delta, A, B, C, D_skip=None, z=None, *, save_states=False, g
     ws = workspace if workspace is not None else _workspace(need, x.device, stream_ptr)
     code = lib.ssm_scan_fwd_state(
         ctypes.byref(prob), _dev_ptr(x, "x", (batch, L, D), io), _dev_ptr(delta, "delta", (batch, L, D), io),
-        _dev_ptr(A, "A", (D, N), torch.float32), _dev_ptr(B, "B", bshape, bdt),
+        _dev_ptr(A, "A", (D, N) + c2, torch.float32), _dev_ptr(B, "B", bshape, bdt),
         _dev_ptr(C, "C", cshape, cdt), _dev_ptr(D_skip, "D_skip", (D,), torch.float32),
-        _dev_ptr(z, "z", (batch, L, D), io), _dev_ptr(h0, "h0", (batch, D, N), torch.float32),
-        _dev_ptr(out, "out", (batch, L, D), io), _dev_ptr(h_last, "h_last", (batch, D, N), torch.float32),
+        _dev_ptr(z, "z", (batch, L, D), io), _dev_ptr(h0, "h0", (batch, D, N) + c2, torch.float32),
+        _dev_ptr(out, "out", (batch, L, D), io), _dev_ptr(h_last, "h_last", (batch, D, N) + c2, torch.float32),
         _dev_ptr(saved_states if save_states else None, "saved_states"),
         _dev_ptr(ws, "workspace"), ctypes.c_size_t(0 if ws is None else ws.numel() * ws.element_size()),
         ctypes.c_void_p(stream_ptr))
@@ -321,27 +329,29 @@ def ssm_scan_bwd_fused_dt(x, delta_pre, delta_bias, A, B, C, D_skip, z, dout, sa
     return o
 
 
-def ssm_step(x, delta, A, B, C, D_skip, z, h, *, zoh=False, out=None, stream=None, static_B=False, static_C=False):
+def ssm_step(x, delta, A, B, C, D_skip, z, h, *, zoh=False, out=None, stream=None, static_B=False, static_C=False,
+             complex_state=False):
     """One recurrent step: x, delta, z (batch, D), B, C (batch, N) io dtype; h (batch, D, N) float32 is updated in
-    place.  Returns out (batch, D)."""
+    place.  Returns out (batch, D).  complex_state: A (D, N, 2), B, C (batch, N, 2), h (batch, D, N, 2)."""
     lib = load_library()
     batch, D = x.shape
-    N = B.shape[-1]
+    N = B.shape[-2] if complex_state else B.shape[-1]
+    c2 = (2,) if complex_state else ()
     prob = ssm_problem_t(batch, 1, D, N, _io_dtype(x),
                          (SSM_FLAG_HAS_Z if z is not None else 0) | (SSM_FLAG_HAS_DSKIP if D_skip is not None else 0)
                          | (SSM_FLAG_ZOH_BBAR if zoh else 0) | (SSM_FLAG_STATIC_B if static_B else 0)
-                         | (SSM_FLAG_STATIC_C if static_C else 0))
+                         | (SSM_FLAG_STATIC_C if static_C else 0) | (SSM_FLAG_COMPLEX if complex_state else 0))
     io = x.dtype
     if out is None:
         out = torch.empty_like(x)
     stream_ptr = (stream if stream is not None else torch.cuda.current_stream(x.device)).cuda_stream
     code = lib.ssm_step(
         ctypes.byref(prob), _dev_ptr(x, "x", (batch, D), io), _dev_ptr(delta, "delta", (batch, D), io),
-        _dev_ptr(A, "A", (D, N), torch.float32),
-        _dev_ptr(B, "B", (D, N) if static_B else (batch, N), torch.float32 if static_B else io),
-        _dev_ptr(C, "C", (D, N) if static_C else (batch, N), torch.float32 if static_C else io),
+        _dev_ptr(A, "A", (D, N) + c2, torch.float32),
+        _dev_ptr(B, "B", (D, N) if static_B else (batch, N) + c2, torch.float32 if static_B else io),
+        _dev_ptr(C, "C", (D, N) if static_C else (batch, N) + c2, torch.float32 if static_C else io),
         _dev_ptr(D_skip, "D_skip", (D,), torch.float32), _dev_ptr(z, "z", (batch, D), io),
-        _dev_ptr(h, "h", (batch, D, N), torch.float32), _dev_ptr(out, "out", (batch, D), io),
+        _dev_ptr(h, "h", (batch, D, N) + c2, torch.float32), _dev_ptr(out, "out", (batch, D), io),
         ctypes.c_void_p(stream_ptr))
     _check(code, "ssm_step")
     return out
@@ -387,7 +397,7 @@ def ssm_scan_fwd_static(x, delta, A, B, C, D_skip=None, z=None, *, save_states=F
 
 def ssm_scan_bwd(x, delta, A, B, C, D_skip, z, dout, saved_states=None, *, general_A=False, zoh=False, workspace=None,
                  stream=None, outputs=None, extra_flags=0, h0=None, dh_last=None, want_dh0=False, static_B=False,
-                 static_C=False):
+                 static_C=False, complex_state=False):
     """Gradients of sum(dout * out) w.r.t. x, delta, A, B, C, D_skip, z; see include/ssm_scan.h.
 
     Returns a dict with dx, ddelta, dz (io dtype, (batch, L, D)); dB, dC (io dtype, (batch, L, N)); dA (float32, (D, N));
@@ -395,19 +405,21 @@ def ssm_scan_bwd(x, delta, A, B, C, D_skip, z, dout, saved_states=None, *, gener
     With h0, dh_last or want_dh0 the call goes through ssm_scan_bwd_state: h0 / dh_last (batch, D, N) float32 are the
     state before the first step and the gradient arriving at the state after the last step, and the dict also holds
     dh0 (batch, D, N) float32.  With static_B / static_C, B / C is a float32 (D, N) parameter and dB / dC is its
-    float32 (D, N) gradient.
+    float32 (D, N) gradient.  With complex_state every complex array (A, B, C, their gradients, h0, dh_last, dh0) has a
+    trailing dimension 2 of (re, im) pairs, and a gradient pair is (dL/dRe, dL/dIm).
     """
     lib = load_library()
-    prob = make_problem(x, B, z is not None, D_skip is not None, False, general_A, zoh, static_B, static_C)
+    prob = make_problem(x, B, z is not None, D_skip is not None, False, general_A, zoh, static_B, static_C, complex_state)
     prob.flags |= int(extra_flags)
     batch, L, D, N = prob.batch, prob.L, prob.D, prob.N
     io = x.dtype
-    bshape, bdt = ((D, N), torch.float32) if static_B else ((batch, L, N), io)
-    cshape, cdt = ((D, N), torch.float32) if static_C else ((batch, L, N), io)
+    c2 = (2,) if complex_state else ()
+    bshape, bdt = ((D, N), torch.float32) if static_B else ((batch, L, N) + c2, io)
+    cshape, cdt = ((D, N), torch.float32) if static_C else ((batch, L, N) + c2, io)
     o = dict(outputs or {})
     o.setdefault("dx", torch.empty_like(x))
     o.setdefault("ddelta", torch.empty_like(x))
-    o.setdefault("dA", torch.empty((D, N), dtype=torch.float32, device=x.device))
+    o.setdefault("dA", torch.empty((D, N) + c2, dtype=torch.float32, device=x.device))
     o.setdefault("dB", torch.empty_like(B))
     o.setdefault("dC", torch.empty_like(C))
     if D_skip is not None:
@@ -424,29 +436,29 @@ def ssm_scan_bwd(x, delta, A, B, C, D_skip, z, dout, saved_states=None, *, gener
     if h0 is not None or dh_last is not None or want_dh0:
         f32 = torch.float32
         if want_dh0:
-            o.setdefault("dh0", torch.empty((batch, D, N), dtype=f32, device=x.device))
+            o.setdefault("dh0", torch.empty((batch, D, N) + c2, dtype=f32, device=x.device))
         code = lib.ssm_scan_bwd_state(
             ctypes.byref(prob), _dev_ptr(x, "x", (batch, L, D), io), _dev_ptr(delta, "delta", (batch, L, D), io),
-            _dev_ptr(A, "A", (D, N), f32), _dev_ptr(B, "B", bshape, bdt), _dev_ptr(C, "C", cshape, cdt),
+            _dev_ptr(A, "A", (D, N) + c2, f32), _dev_ptr(B, "B", bshape, bdt), _dev_ptr(C, "C", cshape, cdt),
             _dev_ptr(D_skip, "D_skip", (D,), f32), _dev_ptr(z, "z", (batch, L, D), io),
-            _dev_ptr(dout, "dout", (batch, L, D), io), _dev_ptr(h0, "h0", (batch, D, N), f32),
-            _dev_ptr(dh_last, "dh_last", (batch, D, N), f32), _dev_ptr(saved_states, "saved_states"),
+            _dev_ptr(dout, "dout", (batch, L, D), io), _dev_ptr(h0, "h0", (batch, D, N) + c2, f32),
+            _dev_ptr(dh_last, "dh_last", (batch, D, N) + c2, f32), _dev_ptr(saved_states, "saved_states"),
             _dev_ptr(o["dx"], "dx", (batch, L, D), io), _dev_ptr(o["ddelta"], "ddelta", (batch, L, D), io),
-            _dev_ptr(o["dA"], "dA", (D, N), f32), _dev_ptr(o["dB"], "dB", bshape, bdt),
+            _dev_ptr(o["dA"], "dA", (D, N) + c2, f32), _dev_ptr(o["dB"], "dB", bshape, bdt),
             _dev_ptr(o["dC"], "dC", cshape, cdt), _dev_ptr(o["dD"], "dD", (D,), f32),
-            _dev_ptr(o["dz"], "dz", (batch, L, D), io), _dev_ptr(o.get("dh0"), "dh0", (batch, D, N), f32),
+            _dev_ptr(o["dz"], "dz", (batch, L, D), io), _dev_ptr(o.get("dh0"), "dh0", (batch, D, N) + c2, f32),
             _dev_ptr(ws, "workspace"), ctypes.c_size_t(0 if ws is None else ws.numel() * ws.element_size()),
             ctypes.c_void_p(stream_ptr))
         _check(code, "ssm_scan_bwd_state")
         return o
     code = lib.ssm_scan_bwd(
         ctypes.byref(prob), _dev_ptr(x, "x", (batch, L, D), io), _dev_ptr(delta, "delta", (batch, L, D), io),
-        _dev_ptr(A, "A", (D, N), torch.float32), _dev_ptr(B, "B", bshape, bdt),
+        _dev_ptr(A, "A", (D, N) + c2, torch.float32), _dev_ptr(B, "B", bshape, bdt),
         _dev_ptr(C, "C", cshape, cdt), _dev_ptr(D_skip, "D_skip", (D,), torch.float32),
         _dev_ptr(z, "z", (batch, L, D), io), _dev_ptr(dout, "dout", (batch, L, D), io),
         _dev_ptr(saved_states, "saved_states"),
         _dev_ptr(o["dx"], "dx", (batch, L, D), io), _dev_ptr(o["ddelta"], "ddelta", (batch, L, D), io),
-        _dev_ptr(o["dA"], "dA", (D, N), torch.float32), _dev_ptr(o["dB"], "dB", bshape, bdt),
+        _dev_ptr(o["dA"], "dA", (D, N) + c2, torch.float32), _dev_ptr(o["dB"], "dB", bshape, bdt),
         _dev_ptr(o["dC"], "dC", cshape, cdt), _dev_ptr(o["dD"], "dD", (D,), torch.float32),
         _dev_ptr(o["dz"], "dz", (batch, L, D), io),
         _dev_ptr(ws, "workspace"), ctypes.c_size_t(0 if ws is None else ws.numel() * ws.element_size()),

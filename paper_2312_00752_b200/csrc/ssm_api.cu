@@ -8,6 +8,18 @@ namespace ssm {
 
 int fwd_channels_per_block(int N);
 int bwd_channels_per_block(int N);
+bool complex_supported(const ssm_problem_t& p);
+size_t complex_bwd_workspace_bytes(const ssm_problem_t& p);
+size_t complex_saved_state_bytes(const ssm_problem_t& p);
+cudaError_t complex_fwd(const ssm_problem_t& prob, const void* x, const void* delta, const float* A, const void* B,
+                        const void* C, const float* D_skip, const void* z, const float* h0, void* out, float* h_last,
+                        void* saved_states, cudaStream_t s);
+cudaError_t complex_bwd(const ssm_problem_t& prob, const void* x, const void* delta, const float* A, const void* B,
+                        const void* C, const float* D_skip, const void* z, const void* dout, const float* h0,
+                        const float* dh_last, const void* saved_states, void* dx, void* ddelta, float* dA, void* dB,
+                        void* dC, float* dD, void* dz, float* dh0, void* workspace, cudaStream_t s);
+cudaError_t complex_step(const ssm_problem_t& prob, const void* x, const void* delta, const float* A, const void* B,
+                         const void* C, const float* D_skip, const void* z, float* h, void* out, cudaStream_t s);
 int fwd_states_per_thread();
 int fwd_fast_channels_per_warp();
 int bwd_fast_channels_per_warp();
@@ -17,7 +29,8 @@ size_t bwd_handoff_bytes_per_worker();
 
 // Shapes the tuned warp-per-worker kernels take (they also want 16-byte aligned pointers, checked per call).
 static bool tuned_shape(const ssm_problem_t& p) {
-  return p.io_dtype == SSM_BF16 && p.N == 16 && p.D % 8 == 0 && !(p.flags & (SSM_FLAG_STATIC_B | SSM_FLAG_STATIC_C));
+  return p.io_dtype == SSM_BF16 && p.N == 16 && p.D % 8 == 0 &&
+         !(p.flags & (SSM_FLAG_STATIC_B | SSM_FLAG_STATIC_C | SSM_FLAG_COMPLEX));
 }
 // Workers the hand-off slots of a workspace allow for `chains` chains of 32 channels: none while every chain can have
 // a warp of its own in the first round (one warp per SM sub-partition), else up to 12 resident warps per SM.
@@ -33,11 +46,12 @@ static ssm_status_t validate_problem(const ssm_problem_t* p) {
   if (p == nullptr) return SSM_ERR_INVALID_ARG;
   if (p->batch < 1 || p->L < 1 || p->D < 1 || p->N < 1) return SSM_ERR_INVALID_ARG;
   if (p->flags & ~(uint32_t)(SSM_FLAG_HAS_Z | SSM_FLAG_HAS_DSKIP | SSM_FLAG_SAVE_STATES | SSM_FLAG_GENERAL_A | SSM_FLAG_TEST_WITHHOLD |
-                             SSM_FLAG_DELTA_SOFTPLUS | SSM_FLAG_ZOH_BBAR | SSM_FLAG_STATIC_B | SSM_FLAG_STATIC_C))
+                             SSM_FLAG_DELTA_SOFTPLUS | SSM_FLAG_ZOH_BBAR | SSM_FLAG_STATIC_B | SSM_FLAG_STATIC_C | SSM_FLAG_COMPLEX))
     return SSM_ERR_INVALID_ARG;
   if (p->io_dtype != SSM_F32 && p->io_dtype != SSM_BF16) return SSM_ERR_UNSUPPORTED;
   if (p->N != 1 && p->N != 2 && p->N != 4 && p->N != 8 && p->N != 16 && p->N != 32 && p->N != 64) return SSM_ERR_UNSUPPORTED;
   if (p->batch > 65535) return SSM_ERR_UNSUPPORTED;  // batch is a grid z dimension
+  if ((p->flags & SSM_FLAG_COMPLEX) && !complex_supported(*p)) return SSM_ERR_UNSUPPORTED;
   return SSM_OK;
 }
 
@@ -55,7 +69,9 @@ Plan make_plan(const ssm_problem_t& p) {
   const long long warps = std::max<long long>(1, groups * (p.N / S) / 32);
   const long long sub_partitions = 4LL * kNumSMs;
   int nseg = 1;
-  if (tuned_shape(p)) {
+  if (p.flags & SSM_FLAG_COMPLEX) {
+    // the complex path does not split time
+  } else if (tuned_shape(p)) {
     // one warp per chain of fwd_fast_channels_per_warp() channels; a split costs half a forward sweep more, so only
     // when fewer than half of the sub-partitions would have a warp, and then into two rounds of chains
     const int cw = fwd_fast_channels_per_warp();
@@ -93,7 +109,9 @@ Plan make_bwd_plan(const ssm_problem_t& p) {
   const long long chains = (long long)p.batch * pl.bwd_groups;
   const long long resident = 4LL * kNumSMs;
   int nseg = 1;
-  if (tuned_shape(p) ? chains < 2 * resident : chains * 4 < resident * 3) {
+  if (p.flags & SSM_FLAG_COMPLEX) {
+    // the complex path does not split time
+  } else if (tuned_shape(p) ? chains < 2 * resident : chains * 4 < resident * 3) {
     // the tuned kernel wants two warps per SM sub-partition (a lone warp cannot cover its own latencies), i.e. two
     // rounds of chains; the adjoint pre-pass that a split costs is about a tenth of the backward work
     const long long want = (2 * resident + chains - 1) / chains;
@@ -245,11 +263,13 @@ size_t ssm_scan_fwd_workspace_bytes(const ssm_problem_t* p) {
 
 size_t ssm_scan_bwd_workspace_bytes(const ssm_problem_t* p) {
   if (validate_problem(p) != SSM_OK) return 0;
+  if (p->flags & SSM_FLAG_COMPLEX) return complex_bwd_workspace_bytes(*p);
   return bwd_layout(*p, make_bwd_plan(*p), make_plan(*p)).total;
 }
 
 size_t ssm_scan_saved_state_bytes(const ssm_problem_t* p) {
   if (validate_problem(p) != SSM_OK) return 0;
+  if (p->flags & SSM_FLAG_COMPLEX) return complex_saved_state_bytes(*p);
   const size_t nck = (size_t)(p->L + kCkptSteps - 1) / kCkptSteps;
   return (size_t)p->batch * nck * p->D * p->N * sizeof(float);
 }
@@ -321,6 +341,13 @@ static ssm_status_t fwd_impl(const ssm_problem_t* p, const void* x, const void* 
   for (const void* q : {(const void*)A, (const void*)D_skip, (const void*)saved_states, (const void*)h0, (const void*)h_last,
                         (const void*)delta_bias})
     if (q && !aligned_to(q, 4)) return SSM_ERR_INVALID_ARG;
+  if (p->flags & SSM_FLAG_COMPLEX) {
+    if (delta_bias != nullptr) return SSM_ERR_UNSUPPORTED;
+    return complex_fwd(*p, x, delta, A, B, C, has_d ? D_skip : nullptr, has_z ? z : nullptr, h0, out, h_last,
+                       save ? saved_states : nullptr, static_cast<cudaStream_t>(stream)) == cudaSuccess
+               ? SSM_OK
+               : SSM_ERR_CUDA;
+  }
   const Plan pl = make_plan(*p);
   st = check_ws(workspace, workspace_bytes, fwd_layout(*p, pl).total);
   if (st != SSM_OK) return st;
@@ -403,6 +430,11 @@ ssm_status_t ssm_step(const ssm_problem_t* p, const void* x, const void* delta, 
   if (!static_bc_aligned(*p, B, C, nullptr, nullptr)) return SSM_ERR_INVALID_ARG;
   for (const void* q : {(const void*)A, (const void*)D_skip, (const void*)h})
     if (q && !aligned_to(q, 4)) return SSM_ERR_INVALID_ARG;
+  if (p->flags & SSM_FLAG_COMPLEX)
+    return complex_step(*p, x, delta, A, B, C, has_d ? D_skip : nullptr, has_z ? z : nullptr, h, out,
+                        static_cast<cudaStream_t>(stream)) == cudaSuccess
+               ? SSM_OK
+               : SSM_ERR_CUDA;
   StepParams sp{};
   sp.x = x;
   sp.delta = delta;
@@ -442,6 +474,16 @@ static ssm_status_t bwd_impl(const ssm_problem_t* p, const void* x, const void* 
                         (const void*)delta_bias, (const void*)ddelta_bias, (const void*)h0, (const void*)dh_last,
                         (const void*)dh0})
     if (q && !aligned_to(q, 4)) return SSM_ERR_INVALID_ARG;
+  if (p->flags & SSM_FLAG_COMPLEX) {
+    if (delta_bias != nullptr || ddelta_bias != nullptr) return SSM_ERR_UNSUPPORTED;
+    st = check_ws(workspace, workspace_bytes, complex_bwd_workspace_bytes(*p));
+    if (st != SSM_OK) return st;
+    return complex_bwd(*p, x, delta, A, B, C, has_d ? D_skip : nullptr, has_z ? z : nullptr, dout, h0, dh_last,
+                       saved_states, dx, ddelta, dA, dB, dC, has_d ? dD : nullptr, has_z ? dz : nullptr, dh0, workspace,
+                       static_cast<cudaStream_t>(stream)) == cudaSuccess
+               ? SSM_OK
+               : SSM_ERR_CUDA;
+  }
   const Plan pl = make_bwd_plan(*p), pl_fwd = make_plan(*p);
   const BwdWorkspace w = bwd_layout(*p, pl, pl_fwd);
   st = check_ws(workspace, workspace_bytes, w.total);

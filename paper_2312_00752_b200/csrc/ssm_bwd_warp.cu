@@ -181,6 +181,7 @@ struct ChainRegs {
   float2 A2[CPT][H];    // A * log2(e)
   // ZOH: B-bar = E B with the input gain E = (a - 1) / A (Eq. 4): 1 / A (0 where A = 0)
   float2 invA[ZOH ? CPT : 1][ZOH ? H : 1];
+  float minA;           // ZOH: smallest |A| among this thread's states
   float a0s[CPT], rs[CPT];
   float2 mu[CPT][H];    // adjoint flowing backwards in time
   float2 dA[CPT][H];
@@ -188,7 +189,8 @@ struct ChainRegs {
 };
 
 // One sub-block of 8 steps: rows [r0, r0 + 8) of the tile; nlive = rows of the tile inside the segment.
-template <int S, int CPT, bool SP, bool AP, bool ZOH>
+// ZS (ZOH only): some |delta A| of the sub-block is too small for the closed form of the input gain.
+template <int S, int CPT, bool SP, bool AP, bool ZOH, bool ZS>
 __device__ __forceinline__ void sub_block(const Lane<S, CPT>& ln, ChainRegs<S, CPT, ZOH>& cr, int r0, int nlive, float gate_on,
                                           bool softplus, const uint32_t* tx, const uint32_t* td, const float* tfB,
                                           const float* tfC, const float* tds, const float* tgp, const float* tdF,
@@ -201,10 +203,14 @@ __device__ __forceinline__ void sub_block(const Lane<S, CPT>& ln, ChainRegs<S, C
   // ZOH input gain E = (a - 1) / A and its derivative dE/dA = (delta a - E) / A, each with its series for small
   // delta A (which covers A = 0); dE/ddelta = a
   auto gain = [&](int q, int k, float2 a, float dtq) {
-    return zoh_gain_pair(a, f2mul(f2dup(dtq), cr.A2[q][k]), dtq, cr.invA[ZOH ? q : 0][ZOH ? k : 0]);
+    const float2 invA = cr.invA[ZOH ? q : 0][ZOH ? k : 0];
+    if constexpr (ZS) return zoh_gain_pair(a, f2mul(f2dup(dtq), cr.A2[q][k]), dtq, invA);
+    else return zoh_gain_closed(a, invA);
   };
   auto gain_dA = [&](int q, int k, float2 a, float2 E, float dtq) {
-    return zoh_gain_dA_pair(a, E, f2mul(f2dup(dtq), cr.A2[q][k]), dtq, cr.invA[ZOH ? q : 0][ZOH ? k : 0]);
+    const float2 invA = cr.invA[ZOH ? q : 0][ZOH ? k : 0];
+    if constexpr (ZS) return zoh_gain_dA_pair(a, E, f2mul(f2dup(dtq), cr.A2[q][k]), dtq, invA);
+    else return zoh_gain_dA_closed(a, E, dtq, invA);
   };
   // ---- forward sweep from the checkpoint: the states after the odd steps stay in registers
   float2 hist[kSB / 2][CPT][H];
@@ -578,6 +584,7 @@ __global__ void __launch_bounds__(kBwdWarps * 32, (CPT == 16 / S) ? 2 : 3)
     // ---- per-thread constants and carried values
     ChainRegs<S, CPT, ZOH> cr;
     bool ap = !p.general_A;
+    cr.minA = 3.0e38f;
 #pragma unroll
     for (int q = 0; q < CPT; ++q) {
       float av[S];
@@ -591,6 +598,10 @@ __global__ void __launch_bounds__(kBwdWarps * 32, (CPT == 16 / S) ? 2 : 3)
       const float tol = 1e-6f * fabsf(av[S - 1]);
 #pragma unroll
       for (int k = 2; k < S; ++k) ap = ap && fabsf(av[k] - (av[0] + (float)k * step)) <= tol;
+      if (ZOH && valid) {
+#pragma unroll
+        for (int k = 0; k < S; ++k) cr.minA = fminf(cr.minA, fabsf(av[k]));
+      }
 #pragma unroll
       for (int k = 0; k < H; ++k) {
         cr.A2[q][k] = make_float2(av[2 * k] * kLog2e, av[2 * k + 1] * kLog2e);
@@ -699,16 +710,37 @@ __global__ void __launch_bounds__(kBwdWarps * 32, (CPT == 16 / S) ? 2 : 3)
 #pragma unroll 1
       for (int sb = kBT / kSB - 1; sb >= 0; --sb) {
         if (sb * kSB >= nlive) continue;   // a sub-block of identity steps
-        if (ap)
-          sub_block<S, CPT, SP, true, ZOH>(ln, cr, sb * kSB, nlive, has_z ? 1.f : 0.f, p.softplus != 0, &sm.x[st][0][0],
-                                      &sm.d[st][0][0], &sm.fB[0][0], &sm.fC[0][0], &sm.ds[0][0], &sm.gp[0][0], &sm.dF[0][0],
-                                      &sm.ck[st][sb][0][0], &sm.ox[0][0], &sm.od[0][0], &sm.oz[0][0], &sm.red[0][0][0],
-                                      part_dB, part_dC, sc.abort);
-        else
-          sub_block<S, CPT, SP, false, ZOH>(ln, cr, sb * kSB, nlive, has_z ? 1.f : 0.f, p.softplus != 0, &sm.x[st][0][0],
-                                       &sm.d[st][0][0], &sm.fB[0][0], &sm.fC[0][0], &sm.ds[0][0], &sm.gp[0][0], &sm.dF[0][0],
-                                       &sm.ck[st][sb][0][0], &sm.ox[0][0], &sm.od[0][0], &sm.oz[0][0], &sm.red[0][0][0],
-                                       part_dB, part_dC, sc.abort);
+        bool zs = false;
+        if constexpr (ZOH) {
+          // smallest step size of the live rows of the sub-block among this thread's channels
+          float dmin = 3.0e38f;
+          for (int t = 0; t < kSB && sb * kSB + t < nlive; ++t) {
+            float dv[CPT];
+            if constexpr (SP) ln.pick_row(&sm.dF[0][0] + (sb * kSB + t) * LN::CW, dv);
+            else ln.unpack_row(&sm.d[st][0][0] + (sb * kSB + t) * (LN::CW / 2), dv);
+#pragma unroll
+            for (int q = 0; q < CPT; ++q) dmin = fminf(dmin, fabsf(dv[q]));
+          }
+          zs = __any_sync(0xffffffffu, dmin * cr.minA < kZohSmall);
+        }
+#define SSM_SUB_BLOCK(AP_, ZS_)                                                                                     \
+  sub_block<S, CPT, SP, AP_, ZOH, ZS_>(ln, cr, sb * kSB, nlive, has_z ? 1.f : 0.f, p.softplus != 0, &sm.x[st][0][0], \
+                                       &sm.d[st][0][0], &sm.fB[0][0], &sm.fC[0][0], &sm.ds[0][0], &sm.gp[0][0],      \
+                                       &sm.dF[0][0], &sm.ck[st][sb][0][0], &sm.ox[0][0], &sm.od[0][0], &sm.oz[0][0], \
+                                       &sm.red[0][0][0], part_dB, part_dC, sc.abort)
+        if constexpr (ZOH) {
+          if (zs) {
+            if (ap) SSM_SUB_BLOCK(true, true);
+            else SSM_SUB_BLOCK(false, true);
+          } else {
+            if (ap) SSM_SUB_BLOCK(true, false);
+            else SSM_SUB_BLOCK(false, false);
+          }
+        } else {
+          if (ap) SSM_SUB_BLOCK(true, false);
+          else SSM_SUB_BLOCK(false, false);
+        }
+#undef SSM_SUB_BLOCK
       }
       __syncwarp();
       // ---- results of the tile: 16-byte stores of dx, ddelta, dz

@@ -342,7 +342,20 @@ __device__ __forceinline__ float zoh_gain_dA(float dt, float A, float a, float E
   return __fdividef(fmaf(dt, a, -E), A);
 }
 
-// The same two quantities for a pair of states in the tuned kernels (bf16 io), without a branch.  `a` are the decays
+// The tuned kernels (bf16 io) take the closed forms E = (a - 1) / A, dE/dA = (dt a - E) / A from the decays they have
+// anyway while every |dt A| of a sub-block of steps is at least kZohSmall: the relative error of E is then that of a
+// (about 2.4e-7) divided by |dt A|, at most 5e-4 (a quarter of the bf16 rounding of the results), and the dE/dA term
+// carries the same relative error into dA.  A sub-block with a smaller |dt A| anywhere in the warp (A = 0 included)
+// runs the variant with the selects below.  The threshold sits below the step sizes of the layer workloads
+// (delta >= 1e-3 with |A| >= 1), which therefore take the closed forms.
+constexpr float kZohSmall = 0.00048828125f;   // 2^-11
+__device__ __forceinline__ float2 zoh_gain_closed(float2 a, float2 invA) {
+  return f2mul(f2fma(a, f2dup(1.f), f2dup(-1.f)), invA);
+}
+__device__ __forceinline__ float2 zoh_gain_dA_closed(float2 a, float2 E, float dt, float2 invA) {
+  return f2mul(f2fma(f2dup(dt), a, f2mul(E, f2dup(-1.f))), invA);
+}
+// The same two quantities for a pair of states, without a branch, accurate for every dt A.  `a` are the decays
 // the kernel has anyway, y2 = dt * A * log2(e), invA = 1 / A (0 where A = 0).  The closed forms (a - 1) / A and
 // (dt a - E) / A lose all their digits as dt A -> 0 (a is rounded to 2^-24 next to 1), so for |dt A| < 1/4 the series
 // in y = dt A take over; they also cover A = 0 (E = dt, dE/dA = dt^2 / 2).

@@ -1,0 +1,604 @@
+// Selective scan with a complex-valued state (Section 3.6, "Real vs. Complex"; S4D-Lin A_n = -1/2 + n i is the
+// paper's initialisation for it), selected by SSM_FLAG_COMPLEX: forward, backward and the single recurrent step.
+//
+//   a[t,n] = exp(delta[t] A[d,n])   (complex)        h[t,n] = a[t,n] h[t-1,n] + delta[t] B[t,n] x[t]   (complex)
+//   s[t]   = 2 Re(sum_n C[t,n] h[t,n]) + D_skip[d] x[t]                    out[t] = s[t] silu(z[t])
+//
+// The N complex states stand for N conjugate pairs of a real system, hence twice the real part (the paper does not
+// say how a complex state gives a real output; this is the convention of the parameterisation it cites).  Complex
+// arrays are interleaved (re, im) pairs: A, dA float32 [D][N][2]; B, C, dB, dC io dtype [batch][L][N][2]; states
+// float32 [..][N][2].  A gradient of a complex quantity holds (dL/dRe, dL/dIm).
+//
+// Backward (adjoint for the real loss sum(dout out); for a product p = u v the gradient of u is conj(v) times the
+// gradient of p, for a real u its real part):
+//   lam[t] = 2 ds[t] conj(C[t]) + mu[t+1],   mu[t] = conj(a[t]) lam[t]
+//   dC[t] = sum_d 2 ds conj(h[t]);  dB[t] = sum_d delta x lam[t];  dx = ds D + delta sum_n Re(conj(B) lam)
+//   w = conj(h[t-1]) mu[t];  ddelta = sum_n Re(conj(A) w) + x sum_n Re(conj(B) lam);  dA = sum_t delta w;  dh0 = mu[1]
+//
+// These are plain kernels in the style of the generic real ones (ssm_fwd.cu, ssm_bwd.cu): a thread owns S = min(4, N)
+// complex states of one channel, N / S lanes share a channel, time is swept sequentially in tiles of 32 steps staged
+// in shared memory, the backward rebuilds the states of a tile from a checkpoint (one per 8 steps) into shared memory
+// and walks it in reverse.  The sequence is not split in time on this path.  The magnitude of a comes from the
+// hardware ex2, its phase from sincos after an explicit reduction of the angle to [-pi, pi].
+#include "ssm_common.cuh"
+
+namespace ssm {
+
+namespace {
+
+constexpr int kCT = 32;   // steps per tile
+static_assert(kCT % kCkptSteps == 0, "a tile starts on a checkpoint");
+
+struct CplxParams {
+  const void *x, *delta, *z, *B, *C, *dout;
+  const float2* A;       // [D][N]
+  const float* Dskip;    // null: no skip term
+  const float2* h0;      // [batch][D][N]; null: zero
+  void* out;
+  float2* h_last;        // [batch][D][N]; null: not wanted
+  float2* ckpt;          // [batch][nck][D][N] (forward: written if not null; backward: read)
+  const float2* dh_last; // backward: adjoint entering the last state; null: zero
+  void *dx, *ddelta, *dz;
+  float* dBC_part;       // [groups][2][batch*L*N*2]
+  float2* dA_part;       // [batch][D][N]
+  float* dD_part;        // [batch][D]
+  float2* dh0;           // null: not wanted
+  int batch, L, D, nck;
+};
+
+__device__ __forceinline__ float2 cmul(float2 a, float2 b) {
+  return make_float2(a.x * b.x - a.y * b.y, a.x * b.y + a.y * b.x);
+}
+// conj(a) * b
+__device__ __forceinline__ float2 cmulc(float2 a, float2 b) {
+  return make_float2(a.x * b.x + a.y * b.y, a.x * b.y - a.y * b.x);
+}
+// exp(dt * A) for A = (re, im)
+__device__ __forceinline__ float2 cexp_step(float dt, float2 A) {
+  const float mag = ex2_approx(dt * A.x * kLog2e);
+  const float ang = dt * A.y;
+  const float k = rintf(ang * 0.15915494309189535f);
+  float r = fmaf(-k, 6.2831854820251465f, ang);     // 2 pi split in two floats
+  r = fmaf(-k, -1.7484555e-7f, r);
+  float sn, cs;
+  __sincosf(r, &sn, &cs);
+  return make_float2(mag * cs, mag * sn);
+}
+
+template <typename IO>
+__device__ __forceinline__ float2 io2_to_float2(const IO* p) {
+  return make_float2(io_to_float<IO>(p[0]), io_to_float<IO>(p[1]));
+}
+
+template <int N>
+struct CGeom {
+  static constexpr int S = N < 4 ? N : 4;        // complex states per thread
+  static constexpr int LPC = N / S;              // lanes per channel
+  static constexpr int CH = N <= 16 ? 32 : 16;   // channels per block
+  static constexpr int THREADS = CH * LPC;
+  static constexpr int WARPS = (THREADS + 31) / 32;
+};
+
+// ---------------------------------------------------------------------------------------------------- forward
+// WRITE_OUT false: only the checkpoint states are produced (backward without saved states).
+template <typename IO, int N, bool WRITE_OUT>
+__global__ void __launch_bounds__(CGeom<N>::THREADS) ssm_cfwd_kernel(const CplxParams p) {
+  using G = CGeom<N>;
+  constexpr int S = G::S, LPC = G::LPC, CH = G::CH, T = kCT, THREADS = G::THREADS;
+  __shared__ __align__(16) IO s_x[T][CH];
+  __shared__ __align__(16) IO s_d[T][CH];
+  __shared__ __align__(16) IO s_z[WRITE_OUT ? T : 1][CH];
+  __shared__ __align__(16) IO s_o[WRITE_OUT ? T : 1][CH];
+  __shared__ __align__(16) float2 s_B[T][N];
+  __shared__ __align__(16) float2 s_C[WRITE_OUT ? T : 1][N];
+
+  const IO* __restrict__ gx = static_cast<const IO*>(p.x);
+  const IO* __restrict__ gd = static_cast<const IO*>(p.delta);
+  const IO* __restrict__ gz = static_cast<const IO*>(p.z);
+  const IO* __restrict__ gB = static_cast<const IO*>(p.B);
+  const IO* __restrict__ gC = static_cast<const IO*>(p.C);
+  IO* __restrict__ gout = static_cast<IO*>(p.out);
+
+  const int tid = threadIdx.x;
+  const int j = tid % LPC, slot = tid / LPC;
+  const int d_cta = blockIdx.x * CH, b = blockIdx.y;
+  const int D = p.D, d = d_cta + slot;
+  const bool valid = d < D;
+
+  float2 Ar[S], h[S];
+#pragma unroll
+  for (int k = 0; k < S; ++k) {
+    Ar[k] = valid ? p.A[(size_t)d * N + j * S + k] : make_float2(0.f, 0.f);
+    h[k] = (valid && p.h0 != nullptr) ? p.h0[((size_t)b * D + d) * N + j * S + k] : make_float2(0.f, 0.f);
+  }
+  const float Dk = (valid && p.Dskip != nullptr) ? p.Dskip[d] : 0.f;
+
+  for (int t0 = 0; t0 < p.L; t0 += T) {
+    const int nt = min(T, p.L - t0);
+    const size_t row0 = (size_t)b * p.L + t0;
+    __syncthreads();
+    for (int i = tid; i < T * CH; i += THREADS) {
+      const int tt = i / CH, c = i % CH;
+      const bool ok = tt < nt && d_cta + c < D;
+      const size_t g = (row0 + tt) * D + d_cta + c;
+      const IO zero = float_to_io<IO>(0.f);
+      s_x[tt][c] = ok ? gx[g] : zero;
+      s_d[tt][c] = ok ? gd[g] : zero;
+      if constexpr (WRITE_OUT) s_z[tt][c] = (ok && gz != nullptr) ? gz[g] : zero;
+    }
+    for (int i = tid; i < T * N; i += THREADS) {
+      const int tt = i / N;
+      const bool ok = tt < nt;
+      s_B[tt][i % N] = ok ? io2_to_float2<IO>(gB + (row0 * N + i) * 2) : make_float2(0.f, 0.f);
+      if constexpr (WRITE_OUT) s_C[tt][i % N] = ok ? io2_to_float2<IO>(gC + (row0 * N + i) * 2) : make_float2(0.f, 0.f);
+    }
+    __syncthreads();
+
+    for (int tt = 0; tt < nt; ++tt) {
+      if (p.ckpt != nullptr && valid && ((t0 + tt) % kCkptSteps) == 0) {
+        float2* dst = p.ckpt + (((size_t)b * p.nck + (t0 + tt) / kCkptSteps) * D + d) * N + j * S;
+#pragma unroll
+        for (int k = 0; k < S; ++k) dst[k] = h[k];
+      }
+      const float dt = io_to_float<IO>(s_d[tt][slot]);
+      const float u = io_to_float<IO>(s_x[tt][slot]);
+      const float du = dt * u;
+      float y = 0.f;
+#pragma unroll
+      for (int k = 0; k < S; ++k) {
+        const float2 a = cexp_step(dt, Ar[k]);
+        const float2 Bk = s_B[tt][j * S + k];
+        const float2 ah = cmul(a, h[k]);
+        h[k] = make_float2(fmaf(du, Bk.x, ah.x), fmaf(du, Bk.y, ah.y));
+        if constexpr (WRITE_OUT) {
+          const float2 Ck = s_C[tt][j * S + k];
+          y += Ck.x * h[k].x - Ck.y * h[k].y;
+        }
+      }
+      if constexpr (WRITE_OUT) {
+#pragma unroll
+        for (int m = LPC / 2; m >= 1; m >>= 1) y += __shfl_xor_sync(0xffffffffu, y, m);
+        if (j == 0) {
+          float s = fmaf(Dk, u, 2.f * y);
+          if (gz != nullptr) {
+            const float zz = io_to_float<IO>(s_z[tt][slot]);
+            s = s * zz * sigmoid_fast(zz);
+          }
+          s_o[tt][slot] = float_to_io<IO>(s);
+        }
+      }
+    }
+    if constexpr (WRITE_OUT) {
+      __syncthreads();
+      for (int i = tid; i < nt * CH; i += THREADS) {
+        const int tt = i / CH, c = i % CH;
+        if (d_cta + c < D) gout[(row0 + tt) * D + d_cta + c] = s_o[tt][c];
+      }
+    }
+  }
+  if (valid && p.h_last != nullptr) {
+#pragma unroll
+    for (int k = 0; k < S; ++k) p.h_last[((size_t)b * D + d) * N + j * S + k] = h[k];
+  }
+}
+
+// ---------------------------------------------------------------------------------------------------- backward
+template <typename IO, int N>
+constexpr size_t cbwd_smem_bytes() {
+  using G = CGeom<N>;
+  return sizeof(float2) * ((size_t)(kCT + 1) * G::CH * N      // h_0 .. h_T
+                           + 2 * (size_t)kCT * N               // B, C
+                           + (size_t)G::WARPS * kCT * 2 * N)   // per-warp dB/dC sums
+         + sizeof(float) * (size_t)kCT * G::CH                 // s (pre-gate readout)
+         + sizeof(IO) * 4 * (size_t)kCT * G::CH;               // x, delta, z, dout (reused for dx, ddelta, dz)
+}
+
+template <typename IO, int N>
+__global__ void __launch_bounds__(CGeom<N>::THREADS) ssm_cbwd_kernel(const CplxParams p) {
+  using G = CGeom<N>;
+  constexpr int S = G::S, LPC = G::LPC, CH = G::CH, WARPS = G::WARPS, T = kCT, THREADS = G::THREADS;
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  float2* s_h = reinterpret_cast<float2*>(smem_raw);         // [T+1][CH][N]
+  float2* s_B = s_h + (size_t)(T + 1) * CH * N;              // [T][N]
+  float2* s_C = s_B + T * N;                                 // [T][N]
+  float2* s_part = s_C + T * N;                              // [WARPS][T][2][N]
+  float* s_s = reinterpret_cast<float*>(s_part + (size_t)WARPS * T * 2 * N);   // [T][CH]
+  IO* s_x = reinterpret_cast<IO*>(s_s + T * CH);             // [T][CH] (becomes dx)
+  IO* s_d = s_x + T * CH;                                    // (becomes ddelta)
+  IO* s_z = s_d + T * CH;                                    // (becomes dz)
+  IO* s_g = s_z + T * CH;
+
+  const IO* __restrict__ gx = static_cast<const IO*>(p.x);
+  const IO* __restrict__ gd = static_cast<const IO*>(p.delta);
+  const IO* __restrict__ gz = static_cast<const IO*>(p.z);
+  const IO* __restrict__ gg = static_cast<const IO*>(p.dout);
+  const IO* __restrict__ gB = static_cast<const IO*>(p.B);
+  const IO* __restrict__ gC = static_cast<const IO*>(p.C);
+  IO* __restrict__ gdx = static_cast<IO*>(p.dx);
+  IO* __restrict__ gdd = static_cast<IO*>(p.ddelta);
+  IO* __restrict__ gdz = static_cast<IO*>(p.dz);
+
+  const int tid = threadIdx.x;
+  const int lane = tid & 31, warp = tid >> 5;
+  const int j = tid % LPC, slot = tid / LPC;
+  const int d_cta = blockIdx.x * CH, b = blockIdx.y;
+  const int D = p.D, d = d_cta + slot;
+  const bool valid = d < D;
+  const bool has_z = gz != nullptr;
+
+  float2 Ar[S], mu[S], dA[S];
+  float dD_acc = 0.f;
+  const float Dk = (valid && p.Dskip != nullptr) ? p.Dskip[d] : 0.f;
+#pragma unroll
+  for (int k = 0; k < S; ++k) {
+    Ar[k] = valid ? p.A[(size_t)d * N + j * S + k] : make_float2(0.f, 0.f);
+    mu[k] = (valid && p.dh_last != nullptr) ? p.dh_last[((size_t)b * D + d) * N + j * S + k] : make_float2(0.f, 0.f);
+    dA[k] = make_float2(0.f, 0.f);
+  }
+
+  for (int kb = (p.L - 1) / T; kb >= 0; --kb) {
+    const int t0 = kb * T;
+    const int nt = min(T, p.L - t0);
+    const size_t row0 = (size_t)b * p.L + t0;
+    __syncthreads();
+    for (int i = tid; i < T * CH; i += THREADS) {
+      const int tt = i / CH, c = i % CH;
+      const bool ok = tt < nt && d_cta + c < D;
+      const size_t g = (row0 + tt) * D + d_cta + c;
+      const IO zero = float_to_io<IO>(0.f);
+      s_x[i] = ok ? gx[g] : zero;
+      s_d[i] = ok ? gd[g] : zero;
+      s_z[i] = (ok && has_z) ? gz[g] : zero;
+      s_g[i] = ok ? gg[g] : zero;
+    }
+    for (int i = tid; i < T * N; i += THREADS) {
+      const bool ok = i / N < nt;
+      s_B[i] = ok ? io2_to_float2<IO>(gB + (row0 * N + i) * 2) : make_float2(0.f, 0.f);
+      s_C[i] = ok ? io2_to_float2<IO>(gC + (row0 * N + i) * 2) : make_float2(0.f, 0.f);
+    }
+    float2 h[S];
+#pragma unroll
+    for (int k = 0; k < S; ++k) {
+      h[k] = valid ? p.ckpt[(((size_t)b * p.nck + (size_t)kb * (T / kCkptSteps)) * D + d) * N + j * S + k]
+                   : make_float2(0.f, 0.f);
+      s_h[(size_t)slot * N + j * S + k] = h[k];
+    }
+    __syncthreads();
+
+    // ---- recompute h_1 .. h_nt of this tile and the pre-gate readout
+    for (int tt = 0; tt < nt; ++tt) {
+      const float dt = io_to_float<IO>(s_d[tt * CH + slot]);
+      const float u = io_to_float<IO>(s_x[tt * CH + slot]);
+      const float du = dt * u;
+      float y = 0.f;
+#pragma unroll
+      for (int k = 0; k < S; ++k) {
+        const float2 a = cexp_step(dt, Ar[k]);
+        const float2 Bk = s_B[tt * N + j * S + k], Ck = s_C[tt * N + j * S + k];
+        const float2 ah = cmul(a, h[k]);
+        h[k] = make_float2(fmaf(du, Bk.x, ah.x), fmaf(du, Bk.y, ah.y));
+        y += Ck.x * h[k].x - Ck.y * h[k].y;
+        s_h[((size_t)(tt + 1) * CH + slot) * N + j * S + k] = h[k];
+      }
+#pragma unroll
+      for (int m = LPC / 2; m >= 1; m >>= 1) y += __shfl_xor_sync(0xffffffffu, y, m);
+      if (j == 0) s_s[tt * CH + slot] = fmaf(Dk, u, 2.f * y);
+    }
+    __syncwarp();
+
+    // ---- reverse recurrence over the tile
+    for (int tt = nt - 1; tt >= 0; --tt) {
+      const float dt = io_to_float<IO>(s_d[tt * CH + slot]);
+      const float u = io_to_float<IO>(s_x[tt * CH + slot]);
+      const float g = io_to_float<IO>(s_g[tt * CH + slot]);
+      const float du = dt * u;
+      float ds = g, dzv = 0.f;
+      if (has_z) {
+        const float zz = io_to_float<IO>(s_z[tt * CH + slot]);
+        const float sg = sigmoid_fast(zz);
+        ds = g * zz * sg;
+        dzv = g * s_s[tt * CH + slot] * sg * fmaf(zz, 1.f - sg, 1.f);
+      }
+      const float ds2 = 2.f * ds;
+      float lamB = 0.f, wA = 0.f;
+      float2 dBp[S], dCp[S];
+#pragma unroll
+      for (int k = 0; k < S; ++k) {
+        const float2 ht = s_h[((size_t)(tt + 1) * CH + slot) * N + j * S + k];
+        const float2 hp = s_h[((size_t)tt * CH + slot) * N + j * S + k];
+        const float2 Bk = s_B[tt * N + j * S + k], Ck = s_C[tt * N + j * S + k];
+        const float2 lam = make_float2(fmaf(ds2, Ck.x, mu[k].x), fmaf(-ds2, Ck.y, mu[k].y));
+        dCp[k] = make_float2(ds2 * ht.x, -ds2 * ht.y);
+        dBp[k] = make_float2(du * lam.x, du * lam.y);
+        lamB += Bk.x * lam.x + Bk.y * lam.y;
+        mu[k] = cmulc(cexp_step(dt, Ar[k]), lam);
+        const float2 w = cmulc(hp, mu[k]);
+        wA += Ar[k].x * w.x + Ar[k].y * w.y;
+        dA[k].x = fmaf(dt, w.x, dA[k].x);
+        dA[k].y = fmaf(dt, w.y, dA[k].y);
+      }
+#pragma unroll
+      for (int m = LPC / 2; m >= 1; m >>= 1) {
+        lamB += __shfl_xor_sync(0xffffffffu, lamB, m);
+        wA += __shfl_xor_sync(0xffffffffu, wA, m);
+      }
+      // sum dB/dC over the channels held by this warp (lanes that share j), in a fixed xor tree
+#pragma unroll
+      for (int k = 0; k < S; ++k) {
+#pragma unroll
+        for (int m = 16; m >= LPC; m >>= 1) {
+          dBp[k].x += __shfl_xor_sync(0xffffffffu, dBp[k].x, m);
+          dBp[k].y += __shfl_xor_sync(0xffffffffu, dBp[k].y, m);
+          dCp[k].x += __shfl_xor_sync(0xffffffffu, dCp[k].x, m);
+          dCp[k].y += __shfl_xor_sync(0xffffffffu, dCp[k].y, m);
+        }
+      }
+      if (lane < LPC) {
+#pragma unroll
+        for (int k = 0; k < S; ++k) {
+          s_part[(((size_t)warp * T + tt) * 2 + 0) * N + j * S + k] = dBp[k];
+          s_part[(((size_t)warp * T + tt) * 2 + 1) * N + j * S + k] = dCp[k];
+        }
+      }
+      if (j == 0) {
+        dD_acc = fmaf(ds, u, dD_acc);
+        s_x[tt * CH + slot] = float_to_io<IO>(fmaf(ds, Dk, dt * lamB));
+        s_d[tt * CH + slot] = float_to_io<IO>(fmaf(u, lamB, wA));
+        s_z[tt * CH + slot] = float_to_io<IO>(dzv);
+      }
+    }
+    __syncthreads();
+
+    for (int i = tid; i < nt * CH; i += THREADS) {
+      const int tt = i / CH, c = i % CH;
+      if (d_cta + c < D) {
+        const size_t g = (row0 + tt) * D + d_cta + c;
+        gdx[g] = s_x[i];
+        gdd[g] = s_d[i];
+        if (gdz != nullptr) gdz[g] = s_z[i];
+      }
+    }
+    // partial sums of this channel block: [block][2][batch*L*N] complex, warps added in ascending order
+    const size_t bln = (size_t)p.batch * p.L * N;
+    float2* part = reinterpret_cast<float2*>(p.dBC_part);
+    for (int i = tid; i < nt * 2 * N; i += THREADS) {
+      const int tt = i / (2 * N), which = (i / N) & 1, n = i % N;
+      float2 acc = make_float2(0.f, 0.f);
+#pragma unroll
+      for (int w = 0; w < WARPS; ++w) {
+        const float2 v = s_part[(((size_t)w * T + tt) * 2 + which) * N + n];
+        acc.x += v.x;
+        acc.y += v.y;
+      }
+      part[((size_t)blockIdx.x * 2 + which) * bln + (row0 + tt) * N + n] = acc;
+    }
+  }
+
+  if (valid) {
+#pragma unroll
+    for (int k = 0; k < S; ++k) p.dA_part[((size_t)b * D + d) * N + j * S + k] = dA[k];
+    if (j == 0) p.dD_part[(size_t)b * D + d] = dD_acc;
+    if (p.dh0 != nullptr) {
+#pragma unroll
+      for (int k = 0; k < S; ++k) p.dh0[((size_t)b * D + d) * N + j * S + k] = mu[k];
+    }
+  }
+}
+
+// ---------------------------------------------------------------------------------------------------- one step
+template <typename IO>
+__global__ void __launch_bounds__(128) ssm_cstep_kernel(const CplxParams p, int N) {
+  const long long e = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (e >= (long long)p.batch * p.D) return;
+  const int b = (int)(e / p.D), d = (int)(e % p.D);
+  const float dt = io_to_float<IO>(static_cast<const IO*>(p.delta)[e]);
+  const float u = io_to_float<IO>(static_cast<const IO*>(p.x)[e]);
+  const IO* gB = static_cast<const IO*>(p.B) + (size_t)b * N * 2;
+  const IO* gC = static_cast<const IO*>(p.C) + (size_t)b * N * 2;
+  float2* hrow = p.h_last + e * N;     // the state, updated in place
+  const float du = dt * u;
+  float y = 0.f;
+  for (int n = 0; n < N; ++n) {
+    const float2 a = cexp_step(dt, p.A[(size_t)d * N + n]);
+    const float2 Bn = io2_to_float2<IO>(gB + 2 * n), Cn = io2_to_float2<IO>(gC + 2 * n);
+    const float2 ah = cmul(a, hrow[n]);
+    const float2 hn = make_float2(fmaf(du, Bn.x, ah.x), fmaf(du, Bn.y, ah.y));
+    hrow[n] = hn;
+    y += Cn.x * hn.x - Cn.y * hn.y;
+  }
+  float s = 2.f * y + (p.Dskip != nullptr ? p.Dskip[d] * u : 0.f);
+  if (p.z != nullptr) {
+    const float zz = io_to_float<IO>(static_cast<const IO*>(p.z)[e]);
+    s = s * zz * sigmoid_fast(zz);
+  }
+  static_cast<IO*>(p.out)[e] = float_to_io<IO>(s);
+}
+
+template <typename IO, int N>
+cudaError_t launch_cfwd_n(const CplxParams& p, bool write_out, cudaStream_t s) {
+  using G = CGeom<N>;
+  const dim3 grid((p.D + G::CH - 1) / G::CH, p.batch);
+  if (write_out) ssm_cfwd_kernel<IO, N, true><<<grid, G::THREADS, 0, s>>>(p);
+  else ssm_cfwd_kernel<IO, N, false><<<grid, G::THREADS, 0, s>>>(p);
+  return cudaGetLastError();
+}
+
+template <typename IO, int N>
+cudaError_t launch_cbwd_n(const CplxParams& p, cudaStream_t s) {
+  using G = CGeom<N>;
+  const dim3 grid((p.D + G::CH - 1) / G::CH, p.batch);
+  constexpr size_t smem = cbwd_smem_bytes<IO, N>();
+  cudaError_t e = cudaFuncSetAttribute(ssm_cbwd_kernel<IO, N>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (e != cudaSuccess) return e;
+  ssm_cbwd_kernel<IO, N><<<grid, G::THREADS, smem, s>>>(p);
+  return cudaGetLastError();
+}
+
+template <typename IO>
+cudaError_t launch_cfwd_io(int N, const CplxParams& p, bool write_out, cudaStream_t s) {
+  switch (N) {
+    case 32: return launch_cfwd_n<IO, 32>(p, write_out, s);
+    case 16: return launch_cfwd_n<IO, 16>(p, write_out, s);
+    case 8: return launch_cfwd_n<IO, 8>(p, write_out, s);
+    case 4: return launch_cfwd_n<IO, 4>(p, write_out, s);
+    case 2: return launch_cfwd_n<IO, 2>(p, write_out, s);
+    case 1: return launch_cfwd_n<IO, 1>(p, write_out, s);
+    default: return cudaErrorInvalidValue;
+  }
+}
+template <typename IO>
+cudaError_t launch_cbwd_io(int N, const CplxParams& p, cudaStream_t s) {
+  switch (N) {
+    case 32: return launch_cbwd_n<IO, 32>(p, s);
+    case 16: return launch_cbwd_n<IO, 16>(p, s);
+    case 8: return launch_cbwd_n<IO, 8>(p, s);
+    case 4: return launch_cbwd_n<IO, 4>(p, s);
+    case 2: return launch_cbwd_n<IO, 2>(p, s);
+    case 1: return launch_cbwd_n<IO, 1>(p, s);
+    default: return cudaErrorInvalidValue;
+  }
+}
+
+inline size_t align256(size_t v) { return (v + 255) & ~(size_t)255; }
+
+struct CplxWorkspace {
+  size_t dBC_part, dA_part, dD_part, ckpt, total;
+  int groups, nck;
+};
+CplxWorkspace cplx_layout(const ssm_problem_t& p) {
+  CplxWorkspace w{};
+  const int ch = p.N <= 16 ? 32 : 16;
+  w.groups = (p.D + ch - 1) / ch;
+  w.nck = (p.L + kCkptSteps - 1) / kCkptSteps;
+  size_t off = 256;   // status block (this path has no device-side wait: the word stays zero)
+  auto take = [&](size_t bytes) {
+    const size_t at = off;
+    off += align256(bytes);
+    return at;
+  };
+  w.dBC_part = take((size_t)w.groups * 2 * p.batch * p.L * p.N * sizeof(float2));
+  w.dA_part = take((size_t)p.batch * p.D * p.N * sizeof(float2));
+  w.dD_part = take((size_t)p.batch * p.D * sizeof(float));
+  w.ckpt = take((size_t)p.batch * w.nck * p.D * p.N * sizeof(float2));
+  w.total = off;
+  return w;
+}
+
+}  // namespace
+
+// Which problems the complex path takes, beyond the checks every problem gets.
+bool complex_supported(const ssm_problem_t& p) {
+  const uint32_t not_with = SSM_FLAG_ZOH_BBAR | SSM_FLAG_STATIC_B | SSM_FLAG_STATIC_C | SSM_FLAG_DELTA_SOFTPLUS;
+  return p.N <= 32 && (p.flags & not_with) == 0;
+}
+
+size_t complex_bwd_workspace_bytes(const ssm_problem_t& p) { return cplx_layout(p).total; }
+
+size_t complex_saved_state_bytes(const ssm_problem_t& p) {
+  return (size_t)p.batch * ((p.L + kCkptSteps - 1) / kCkptSteps) * p.D * p.N * sizeof(float2);
+}
+
+cudaError_t complex_fwd(const ssm_problem_t& prob, const void* x, const void* delta, const float* A, const void* B,
+                        const void* C, const float* D_skip, const void* z, const float* h0, void* out, float* h_last,
+                        void* saved_states, cudaStream_t s) {
+  CplxParams p{};
+  p.x = x;
+  p.delta = delta;
+  p.z = z;
+  p.B = B;
+  p.C = C;
+  p.A = reinterpret_cast<const float2*>(A);
+  p.Dskip = D_skip;
+  p.h0 = reinterpret_cast<const float2*>(h0);
+  p.out = out;
+  p.h_last = reinterpret_cast<float2*>(h_last);
+  p.ckpt = static_cast<float2*>(saved_states);
+  p.batch = prob.batch;
+  p.L = prob.L;
+  p.D = prob.D;
+  p.nck = (prob.L + kCkptSteps - 1) / kCkptSteps;
+  return prob.io_dtype == SSM_BF16 ? launch_cfwd_io<__nv_bfloat16>(prob.N, p, true, s)
+                                   : launch_cfwd_io<float>(prob.N, p, true, s);
+}
+
+cudaError_t complex_bwd(const ssm_problem_t& prob, const void* x, const void* delta, const float* A, const void* B,
+                        const void* C, const float* D_skip, const void* z, const void* dout, const float* h0,
+                        const float* dh_last, const void* saved_states, void* dx, void* ddelta, float* dA, void* dB,
+                        void* dC, float* dD, void* dz, float* dh0, void* workspace, cudaStream_t s) {
+  const CplxWorkspace w = cplx_layout(prob);
+  char* ws = static_cast<char*>(workspace);
+  cudaError_t e = cudaMemsetAsync(ws, 0, 256, s);
+  if (e != cudaSuccess) return e;
+  CplxParams p{};
+  p.x = x;
+  p.delta = delta;
+  p.z = z;
+  p.B = B;
+  p.C = C;
+  p.dout = dout;
+  p.A = reinterpret_cast<const float2*>(A);
+  p.Dskip = D_skip;
+  p.h0 = reinterpret_cast<const float2*>(h0);
+  p.batch = prob.batch;
+  p.L = prob.L;
+  p.D = prob.D;
+  p.nck = w.nck;
+  const bool bf = prob.io_dtype == SSM_BF16;
+  const float2* ckpt = static_cast<const float2*>(saved_states);
+  if (ckpt == nullptr) {
+    // rebuild the checkpoint states with one more forward sweep
+    CplxParams f = p;
+    f.ckpt = reinterpret_cast<float2*>(ws + w.ckpt);
+    e = bf ? launch_cfwd_io<__nv_bfloat16>(prob.N, f, false, s) : launch_cfwd_io<float>(prob.N, f, false, s);
+    if (e != cudaSuccess) return e;
+    ckpt = f.ckpt;
+  }
+  p.ckpt = const_cast<float2*>(ckpt);
+  p.dh_last = reinterpret_cast<const float2*>(dh_last);
+  p.dx = dx;
+  p.ddelta = ddelta;
+  p.dz = dz;
+  p.dBC_part = reinterpret_cast<float*>(ws + w.dBC_part);
+  p.dA_part = reinterpret_cast<float2*>(ws + w.dA_part);
+  p.dD_part = reinterpret_cast<float*>(ws + w.dD_part);
+  p.dh0 = reinterpret_cast<float2*>(dh0);
+  e = bf ? launch_cbwd_io<__nv_bfloat16>(prob.N, p, s) : launch_cbwd_io<float>(prob.N, p, s);
+  if (e != cudaSuccess) return e;
+  // the fixed-order second stage is the real path's, on arrays of 2 N floats per complex row
+  ReduceParams rp{};
+  rp.dBC_part = p.dBC_part;
+  rp.dB = dB;
+  rp.dC = dC;
+  rp.dA_part = reinterpret_cast<const float*>(p.dA_part);
+  rp.dD_part = p.dD_part;
+  rp.dA = dA;
+  rp.dD = dD;
+  rp.bln = (long long)prob.batch * prob.L * prob.N * 2;
+  rp.groups = w.groups;
+  rp.parts = prob.batch;
+  rp.D = prob.D;
+  rp.N = prob.N * 2;
+  return launch_bwd_reduce(prob, rp, s);
+}
+
+cudaError_t complex_step(const ssm_problem_t& prob, const void* x, const void* delta, const float* A, const void* B,
+                         const void* C, const float* D_skip, const void* z, float* h, void* out, cudaStream_t s) {
+  CplxParams p{};
+  p.x = x;
+  p.delta = delta;
+  p.z = z;
+  p.B = B;
+  p.C = C;
+  p.A = reinterpret_cast<const float2*>(A);
+  p.Dskip = D_skip;
+  p.h_last = reinterpret_cast<float2*>(h);
+  p.out = out;
+  p.batch = prob.batch;
+  p.D = prob.D;
+  const unsigned grid = (unsigned)(((long long)prob.batch * prob.D + 127) / 128);
+  if (prob.io_dtype == SSM_BF16) ssm_cstep_kernel<__nv_bfloat16><<<grid, 128, 0, s>>>(p, prob.N);
+  else ssm_cstep_kernel<float><<<grid, 128, 0, s>>>(p, prob.N);
+  return cudaGetLastError();
+}
+
+}  // namespace ssm

@@ -168,6 +168,7 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32) ssm_fwd_warp_kernel(const
     float2 h[H];
     float2 invA[ZOH ? H : 1];   // ZOH: 1 / A (0 where A = 0)
     float a0s, rs;
+    float minA = 3.0e38f;       // ZOH: smallest |A| among this thread's states
     bool ap = !p.general_A;
     {
       float av[S];
@@ -181,6 +182,10 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32) ssm_fwd_warp_kernel(const
       const float tol = 1e-6f * fabsf(av[S - 1]);
 #pragma unroll
       for (int k = 2; k < S; ++k) ap = ap && fabsf(av[k] - (av[0] + (float)k * step)) <= tol;
+      if (ZOH && valid) {
+#pragma unroll
+        for (int k = 0; k < S; ++k) minA = fminf(minA, fabsf(av[k]));
+      }
 #pragma unroll
       for (int k = 0; k < H; ++k) {
         A2[k] = make_float2(av[2 * k] * kLog2e, av[2 * k + 1] * kLog2e);
@@ -231,8 +236,10 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32) ssm_fwd_warp_kernel(const
     // three phases so that a warp has independent long-latency work in flight and no load has to pass an earlier
     // store: (1) the step sizes, inputs and exponentials of all GB steps, (2) the recurrences and readouts, (3) skip
     // term, gate and rounding of the results.  There is no branch inside a batch.
-    auto compute_sub = [&](int st, int r0, auto ap_tag) {
+    // zs_tag (ZOH only): some |delta A| of the sub-block is too small for the closed form of the input gain.
+    auto compute_sub = [&](int st, int r0, auto ap_tag, auto zs_tag) {
       constexpr bool AP = decltype(ap_tag)::value;
+      constexpr bool ZS = decltype(zs_tag)::value;
       constexpr int GB = AP ? 8 : (S == 16 ? 2 : 4);
       constexpr int NE = GB / LPC;        // results this lane finishes per batch
       const float gate_off = has_z ? 0.f : 1.f;
@@ -304,7 +311,9 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32) ssm_fwd_warp_kernel(const
           for (int k = 0; k < H; ++k) {
             if constexpr (ZOH) {
               // B-bar = E B with the input gain E = (a - 1) / A (Eq. 4; E = delta at A = 0, a series for small delta A)
-              const float2 E = zoh_gain_pair(a[k], f2mul(f2dup(dt[t]), A2[k]), dt[t], invA[k]);
+              float2 E;
+              if constexpr (ZS) E = zoh_gain_pair(a[k], f2mul(f2dup(dt[t]), A2[k]), dt[t], invA[k]);
+              else E = zoh_gain_closed(a[k], invA[k]);
               bxF[k] = f2mul(f2mul(E, f2dup(u[t])), Bv[k]);
             } else {
               bxF[k] = f2mul(du2, Bv[k]);
@@ -398,8 +407,22 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32) ssm_fwd_warp_kernel(const
             *reinterpret_cast<float4*>(p.ckpt + (((size_t)b * p.nck + ts / kCkptSteps) * D + c_own) * 16 + S * j + 4 * k) =
                 make_float4(h[2 * k].x, h[2 * k].y, h[2 * k + 1].x, h[2 * k + 1].y);
         }
-        if (ap) compute_sub(st, sb * kSub, std::true_type{});
-        else compute_sub(st, sb * kSub, std::false_type{});
+        if constexpr (ZOH) {
+          // smallest step size of the live rows of the sub-block for this lane's channel
+          float dmin = 3.0e38f;
+          for (int t = 0; t < kSub && ts + t < t_to; ++t)
+            dmin = fminf(dmin, fabsf(SP ? sm.dF[SP ? sb * kSub + t : 0][g] : bf16at(sm.d[st][sb * kSub + t], g)));
+          if (__any_sync(0xffffffffu, dmin * minA < kZohSmall)) {
+            if (ap) compute_sub(st, sb * kSub, std::true_type{}, std::true_type{});
+            else compute_sub(st, sb * kSub, std::false_type{}, std::true_type{});
+          } else {
+            if (ap) compute_sub(st, sb * kSub, std::true_type{}, std::false_type{});
+            else compute_sub(st, sb * kSub, std::false_type{}, std::false_type{});
+          }
+        } else {
+          if (ap) compute_sub(st, sb * kSub, std::true_type{}, std::false_type{});
+          else compute_sub(st, sb * kSub, std::false_type{}, std::false_type{});
+        }
       }
       if constexpr (FULL) {
         __syncwarp();

@@ -117,6 +117,7 @@ extern "C" ssm_status_t ssm_scan_fwd_bwd_host(const ssm_problem_t* p, const void
                                               void* stream) {
   HostPlan h;
   if (!make_host_plan(p, &h)) return SSM_ERR_INVALID_ARG;
+  if (p->flags & SSM_FLAG_COMPLEX) return SSM_ERR_UNSUPPORTED;   // this entry point moves real-state buffers only
   const bool has_z = p->flags & SSM_FLAG_HAS_Z, has_d = p->flags & SSM_FLAG_HAS_DSKIP;
   if (!x || !delta || !A || !B || !C || !dout || !out || !dx || !ddelta || !dA || !dB || !dC) return SSM_ERR_INVALID_ARG;
   if ((has_z && (!z || !dz)) || (has_d && (!D_skip || !dD))) return SSM_ERR_INVALID_ARG;

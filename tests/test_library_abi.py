@@ -59,6 +59,19 @@ def test_invalid_problems_are_rejected(bad, code):
     assert lib.ssm_scan_fwd(ctypes.byref(p), one, one, one, one, one, one, one, one, None, None, 0, None) == code
 
 
+def test_complex_state_queries_and_refused_combinations():
+    lib = K.load_library()
+    real = _prob(2, 100, 64, N=8, io=K.SSM_F32, flags=3)
+    cplx = _prob(2, 100, 64, N=8, io=K.SSM_F32, flags=3 | K.SSM_FLAG_COMPLEX)
+    assert K.saved_state_bytes(cplx) == 2 * K.saved_state_bytes(real)        # (re, im) pairs
+    assert K.fwd_workspace_bytes(cplx) == 0 and K.bwd_workspace_bytes(cplx) > 0
+    assert K.plan(_prob(1, 524288, 64, N=8, flags=3 | K.SSM_FLAG_COMPLEX))["n_segments"] == 1   # no time split
+    for extra in (K.SSM_FLAG_ZOH_BBAR, K.SSM_FLAG_STATIC_B, K.SSM_FLAG_STATIC_C, K.SSM_FLAG_DELTA_SOFTPLUS):
+        bad = _prob(2, 100, 64, N=8, flags=3 | K.SSM_FLAG_COMPLEX | extra)
+        assert lib.ssm_scan_plan(ctypes.byref(bad), None, None, None, None) == 2
+    assert lib.ssm_scan_plan(ctypes.byref(_prob(2, 100, 64, N=64, flags=3 | K.SSM_FLAG_COMPLEX)), None, None, None, None) == 2
+
+
 def test_null_misaligned_and_workspace_errors_before_launch():
     lib = K.load_library()
     p = _prob()
