@@ -20,6 +20,7 @@ cudaError_t complex_bwd(const ssm_problem_t& prob, const void* x, const void* de
                         void* dC, float* dD, void* dz, float* dh0, void* workspace, cudaStream_t s);
 cudaError_t complex_step(const ssm_problem_t& prob, const void* x, const void* delta, const float* A, const void* B,
                          const void* C, const float* D_skip, const void* z, float* h, void* out, cudaStream_t s);
+bool bwd_local_fast_applicable(const ssm_problem_t& prob, const BwdParams& p);
 int fwd_states_per_thread();
 int fwd_fast_channels_per_warp();
 int bwd_fast_channels_per_warp();
@@ -199,7 +200,7 @@ static BwdWorkspace bwd_layout(const ssm_problem_t& p, const Plan& pl, const Pla
   const long long chains = (long long)parts * pl.bwd_groups;
   w.max_workers = !tuned_shape(p) ? 0 : (p.flags & SSM_FLAG_TEST_WITHHOLD) ? (int)std::max<long long>(1, (2 * chains + 2) / 3)
                                                                             : shared_workers(chains);
-  w.flags = take((size_t)(w.max_workers + 1) * sizeof(int));
+  w.flags = take((size_t)2 * (w.max_workers + 1) * sizeof(int));   // backward kernel | adjoint pre-pass
   w.handoff = take((size_t)(w.max_workers + 1) * bwd_handoff_bytes_per_worker());
   if (p.flags & SSM_FLAG_STATIC_B) w.dBs_part = take(parts * p.D * p.N * sizeof(float));
   if (p.flags & SSM_FLAG_STATIC_C) w.dCs_part = take(parts * p.D * p.N * sizeof(float));
@@ -568,7 +569,15 @@ static ssm_status_t bwd_impl(const ssm_problem_t* p, const void* x, const void* 
   // the hand-off flags of the tuned kernel start at zero (the status word was cleared above)
   if (cudaMemsetAsync(ws + w.flags, 0, w.handoff - w.flags, s) != cudaSuccess) return SSM_ERR_CUDA;
 
-  if (pl.nseg > 1) {
+  if (pl.nseg == 2 && dh_last == nullptr && (bp.seg_local = reinterpret_cast<float*>(ws + w.mu_in),
+                                              bp.seg_dsum = reinterpret_cast<float*>(ws + w.seg_dsum),
+                                              bwd_local_fast_applicable(*p, bp))) {
+    // two segments and nothing flowing in from outside: the adjoint leaving segment 1 IS the inflow of segment 0, so
+    // the tuned pre-pass writes it there and the carry scan is skipped
+    bp.local_as_inflow = 1;
+    if (launch_bwd(*p, pl, bp, kBwdLocal, s) != cudaSuccess) return SSM_ERR_CUDA;
+    bp.mu_in = bp.seg_local;
+  } else if (pl.nseg > 1) {
     bp.seg_local = reinterpret_cast<float*>(ws + w.seg_local);
     bp.seg_dsum = reinterpret_cast<float*>(ws + w.seg_dsum);
     if (launch_bwd(*p, pl, bp, kBwdLocal, s) != cudaSuccess) return SSM_ERR_CUDA;

@@ -100,6 +100,9 @@ struct BwdParams {
   const float* ckpt;      // [batch][nck][D][N]
   const float* mu_in;     // [batch][nseg][D][N] adjoint inflow of each segment; null: zero
   float* seg_local;       // LOCAL mode: [batch][nseg][D][N] adjoint leaving each segment with zero inflow
+  int local_as_inflow;    // tuned LOCAL kernel, two segments, no outside adjoint: write the result of segment 1 as the
+                          // inflow of segment 0 and zero as the inflow of segment 1 (the layout of mu_in), so that the
+                          // carry scan over two segments is not needed
   float* seg_dsum;        // LOCAL mode: [batch][nseg][D]
   void* dx;
   void* ddelta;
