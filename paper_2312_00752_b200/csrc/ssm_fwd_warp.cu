@@ -526,17 +526,28 @@ cudaError_t launch_s(const Plan& plan, const FwdParams& p, int mode, cudaStream_
 }  // namespace
 
 // Workers for `chains` chains on a GPU that holds `per_sm` warps of the kernel on each of `sms` SMs.  With more
-// chains than one warp per SM sub-partition the worker count is a whole number of such rounds (as many as are
-// resident), so that every sub-partition carries the same load and chains are shared between neighbouring workers;
-// with fewer chains, or without hand-off slots in the workspace (`max_workers` 0), every chain is a worker of its own
-// and nothing is shared (then the grid may also exceed what is resident, since nobody waits).
+// chains than one warp per SM sub-partition the worker count is a whole number r of such rounds (so that every
+// sub-partition carries the same load and chains are shared between neighbouring workers).  r is the one with the
+// shortest estimated run: a worker's share is chains / workers chains but never finishes before one whole chain has
+// been walked (a chain is sequential), and r warps on a sub-partition each run slower than one alone, by the factors
+// measured on these kernels (two warps: 1.4 times slower each, i.e. 1.43 times the throughput).  With fewer chains, or
+// without hand-off slots in the workspace (`max_workers` 0), every chain is a worker of its own and nothing is shared
+// (then the grid may also exceed what is resident, since nobody waits).
 int warp_workers(int chains, int sms, int per_sm, int max_workers) {
   const int round = 4 * sms;
   if (max_workers <= 0 || chains <= round) return chains;
-  int rounds = chains / round;
-  if (rounds > per_sm / 4) rounds = per_sm / 4;
-  if (rounds < 1) rounds = 1;
-  int workers = rounds * round;
+  static const float slow[5] = {0.f, 1.0f, 1.4f, 1.95f, 2.5f};
+  int best = 1;
+  float best_t = 0.f;
+  for (int r = 1; r <= 4 && r <= per_sm / 4 && r * round <= max_workers; ++r) {
+    const float share = (float)chains / (float)(r * round);
+    const float t = (share > 1.f ? share : 1.f) * slow[r];
+    if (r == 1 || t < best_t) {
+      best = r;
+      best_t = t;
+    }
+  }
+  int workers = best * round;
   if (workers > max_workers) workers = max_workers;
   return workers;
 }
