@@ -33,12 +33,13 @@ static bool tuned_shape(const ssm_problem_t& p) {
   return p.io_dtype == SSM_BF16 && p.N == 16 && p.D % 8 == 0 &&
          !(p.flags & (SSM_FLAG_STATIC_B | SSM_FLAG_STATIC_C | SSM_FLAG_COMPLEX));
 }
-// Workers the hand-off slots of a workspace allow for `chains` chains of 32 channels: none while every chain can have
-// a warp of its own in the first round (one warp per SM sub-partition), else up to 12 resident warps per SM.
+// Workers the hand-off slots of a workspace allow for `chains` chains: none while every chain can have a warp of its
+// own in the first round (one warp per SM sub-partition); else at least two rounds (a kernel may share chains between
+// more warps than there are chains) and at most 12 resident warps per SM.
 constexpr int kMaxWarpsPerSM = 12;
 static int shared_workers(long long chains) {
   if (chains <= 4LL * kNumSMs) return 0;
-  return (int)std::min<long long>(chains, (long long)kMaxWarpsPerSM * kNumSMs);
+  return (int)std::min<long long>(std::max<long long>(chains, 8LL * kNumSMs), (long long)kMaxWarpsPerSM * kNumSMs);
 }
 
 static inline size_t align_up(size_t v) { return (v + 255) & ~(size_t)255; }

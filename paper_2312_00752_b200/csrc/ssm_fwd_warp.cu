@@ -37,20 +37,20 @@ namespace ssm {
 namespace {
 
 constexpr int kWT = 32;          // steps per tile
-constexpr int kWStages = 3;      // ring stages
 constexpr int kSub = kCkptSteps; // steps per unrolled sub-block: a checkpoint is written at the start of each
 constexpr int kWarpsPerBlock = 4;
 static_assert(kWT % kSub == 0, "tiles are whole sub-blocks");
 
-template <int CW, bool FULL, bool SP, bool BCW>
+// NST ring stages: 3 (two tiles in flight) or 2 (one tile in flight; small enough for two blocks per SM in FULL mode)
+template <int CW, bool FULL, bool SP, bool BCW, int NST>
 struct FwdWarpSmem {
-  uint32_t x[kWStages][kWT][CW / 2];   // bf16 pairs, CW channels
-  uint32_t d[kWStages][kWT][CW / 2];
-  uint32_t z[FULL ? kWStages : 1][FULL ? kWT : 1][CW / 2];
+  uint32_t x[NST][kWT][CW / 2];   // bf16 pairs, CW channels
+  uint32_t d[NST][kWT][CW / 2];
+  uint32_t z[FULL ? NST : 1][FULL ? kWT : 1][CW / 2];
   // B and C rows are padded (12 and 20 words instead of 8 and 16) so that the one-row-per-lane widening pass of a
   // tile reads and writes them without bank conflicts
-  uint32_t rB[kWStages][kWT][12];  // bf16 pairs, 16 states
-  uint32_t rC[FULL ? kWStages : 1][FULL ? kWT : 1][12];
+  uint32_t rB[NST][kWT][12];  // bf16 pairs, 16 states
+  uint32_t rC[FULL ? NST : 1][FULL ? kWT : 1][12];
   float fB[BCW ? kWT : 1][20];     // BCW: B and C of the current tile widened to float
   float fC[(BCW && FULL) ? kWT : 1][20];
   float dF[SP ? kWT : 1][CW];      // SP: step sizes after bias and softplus
@@ -65,8 +65,9 @@ __device__ __forceinline__ float bf16at(const uint32_t* row, int c) {
 
 }  // namespace
 
-template <int S, int MODE, bool SP, bool ZOH, bool BCW>
+template <int S, int MODE, bool SP, bool ZOH, bool BCW, int NST>
 __global__ void __launch_bounds__(kWarpsPerBlock * 32) ssm_fwd_warp_kernel(const FwdParams p, const WarpSched sc) {
+  static_assert(NST == 2 || NST == 3, "ring stages");
   static_assert(S == 16 || S == 8, "one lane or a lane pair per channel");
   constexpr bool FULL = (MODE == kFwdFull);
   constexpr bool SUMMARY = (MODE == kFwdSummary);
@@ -74,7 +75,7 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32) ssm_fwd_warp_kernel(const
   constexpr int CH = CW / 8;        // 16-byte chunks per tile row of x, delta, z, out
   constexpr int RP = 32 / CH;       // tile rows a warp covers with one chunk per lane
   constexpr int HV = S / 4 + 1;     // float4 per lane of a hand-off: S states, sum of delta
-  using Smem = FwdWarpSmem<CW, FULL, SP, BCW>;
+  using Smem = FwdWarpSmem<CW, FULL, SP, BCW, NST>;
   extern __shared__ __align__(16) unsigned char smem_raw[];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   Smem& sm = reinterpret_cast<Smem*>(smem_raw)[warp];
@@ -135,7 +136,7 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32) ssm_fwd_warp_kernel(const
     const size_t boff = (row_from + brow) * 16 + bhc * 8;
     auto issue_tile = [&](int i) {
       if (i < ntiles) {
-        const int st = i % kWStages;
+        const int st = i % NST;
         const int t0 = t_from + i * kWT;
         const size_t xo = xoff + (size_t)i * kWT * D, bo = boff + (size_t)i * kWT * 16;
 #pragma unroll
@@ -159,7 +160,7 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32) ssm_fwd_warp_kernel(const
       cp_async_commit();
     };
     issue_tile(0);
-    issue_tile(1);
+    if constexpr (NST == 3) issue_tile(1);
 
     // ---- per-thread constants and state
     const int c_own = d_w + g;            // this lane's channel
@@ -362,10 +363,11 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32) ssm_fwd_warp_kernel(const
     };
 
     for (int i = 0; i < ntiles; ++i) {
-      cp_async_wait_but_one();
+      if constexpr (NST == 3) cp_async_wait_but_one();
+      else cp_async_wait_all();
       __syncwarp();             // tile i landed for all lanes; all lanes are done with tile i - 1
-      issue_tile(i + 2);        // into the stage tile i - 1 used
-      const int st = i % kWStages;
+      issue_tile(i + NST - 1);  // into the stage tile i - 1 used
+      const int st = i % NST;
       const int t0 = t_from + i * kWT;
       if constexpr (BCW) {
         // B and C of the tile to float, one row per lane
@@ -463,6 +465,7 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32) ssm_fwd_warp_kernel(const
 }
 
 int warp_workers(int chains, int sms, int per_sm, int max_workers);
+float warp_run_estimate(int chains, int sms, int per_sm, int max_workers);
 
 #ifdef SSM_FWD_LANE_PAIR
 constexpr int kFwdS = 8;   // a lane pair per channel, 16-channel chains
@@ -472,23 +475,47 @@ constexpr int kFwdS = 16;  // a lane per channel, 32-channel chains
 
 namespace {
 
+template <int S, int MODE, bool SP, bool ZOH, bool BCW, int NST>
+cudaError_t fwd_occupancy(int* per_sm, size_t* smem_bytes) {
+  constexpr int CW = 2 * S;   // channels per chain
+  const size_t smem = sizeof(FwdWarpSmem<CW, MODE == kFwdFull, SP, BCW, NST>) * kWarpsPerBlock;
+  auto kern = ssm_fwd_warp_kernel<S, MODE, SP, ZOH, BCW, NST>;
+  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (e != cudaSuccess) return e;
+  *smem_bytes = smem;
+  return cudaOccupancyMaxActiveBlocksPerMultiprocessor(per_sm, kern, kWarpsPerBlock * 32, smem);
+}
+
 template <int S, int MODE, bool SP, bool ZOH, bool BCW>
 cudaError_t launch_variant_w(const Plan& plan, const FwdParams& p, cudaStream_t s) {
   constexpr int CW = 2 * S;   // channels per chain
-  const size_t smem = sizeof(FwdWarpSmem<CW, MODE == kFwdFull, SP, BCW>) * kWarpsPerBlock;
-  auto kern = ssm_fwd_warp_kernel<S, MODE, SP, ZOH, BCW>;
-  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-  if (e != cudaSuccess) return e;
   int dev = 0, sms = 0, per_sm = 0;
+  size_t smem = 0;
+  cudaError_t e;
   if ((e = cudaGetDevice(&dev)) != cudaSuccess) return e;
   if ((e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
-  if ((e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, kWarpsPerBlock * 32, smem)) != cudaSuccess) return e;
+  if ((e = fwd_occupancy<S, MODE, SP, ZOH, BCW, 3>(&per_sm, &smem)) != cudaSuccess) return e;
   if (per_sm < 1) return cudaErrorLaunchOutOfResources;
   WarpSched sc{};
   sc.chains = p.batch * plan.nseg * ((p.D + CW - 1) / CW);
   sc.tiles = (plan.seg_steps + kWT - 1) / kWT;
   const bool can_share = p.abort != nullptr && p.flags != nullptr && p.handoff != nullptr;
-  sc.workers = warp_workers(sc.chains, sms, per_sm * kWarpsPerBlock, can_share ? p.max_workers : 0);
+  const int max_workers = can_share ? p.max_workers : 0;
+  // The two-stage ring (one tile in flight instead of two) lets more warps share an SM: taken when that shortens the
+  // estimated run by more than the shorter prefetch distance may cost.
+  bool two_stage = false;
+  if constexpr (!ZOH && MODE != kFwdSummary) {
+    int per_sm2 = 0;
+    size_t smem2 = 0;
+    if ((e = fwd_occupancy<S, MODE, SP, ZOH, BCW, 2>(&per_sm2, &smem2)) != cudaSuccess) return e;
+    if (per_sm2 > per_sm && warp_run_estimate(sc.chains, sms, per_sm2 * kWarpsPerBlock, max_workers) <
+                                0.93f * warp_run_estimate(sc.chains, sms, per_sm * kWarpsPerBlock, max_workers)) {
+      two_stage = true;
+      per_sm = per_sm2;
+      smem = smem2;
+    }
+  }
+  sc.workers = warp_workers(sc.chains, sms, per_sm * kWarpsPerBlock, max_workers);
   const long long total = (long long)sc.chains * sc.tiles;
   sc.quota = (int)((total + sc.workers - 1) / sc.workers);
   sc.spin_limit = 1 << 22;
@@ -496,7 +523,13 @@ cudaError_t launch_variant_w(const Plan& plan, const FwdParams& p, cudaStream_t 
   sc.abort = p.abort;
   sc.handoff = p.handoff;
   const unsigned grid = (unsigned)((sc.workers + kWarpsPerBlock - 1) / kWarpsPerBlock);
-  kern<<<grid, kWarpsPerBlock * 32, smem, s>>>(p, sc);
+  if constexpr (!ZOH && MODE != kFwdSummary) {
+    if (two_stage) {
+      ssm_fwd_warp_kernel<S, MODE, SP, ZOH, BCW, 2><<<grid, kWarpsPerBlock * 32, smem, s>>>(p, sc);
+      return cudaGetLastError();
+    }
+  }
+  ssm_fwd_warp_kernel<S, MODE, SP, ZOH, BCW, 3><<<grid, kWarpsPerBlock * 32, smem, s>>>(p, sc);
   return cudaGetLastError();
 }
 
@@ -533,9 +566,8 @@ cudaError_t launch_s(const Plan& plan, const FwdParams& p, int mode, cudaStream_
 // measured on these kernels (two warps: 1.4 times slower each, i.e. 1.43 times the throughput).  With fewer chains, or
 // without hand-off slots in the workspace (`max_workers` 0), every chain is a worker of its own and nothing is shared
 // (then the grid may also exceed what is resident, since nobody waits).
-int warp_workers(int chains, int sms, int per_sm, int max_workers) {
+static int warp_rounds(int chains, int sms, int per_sm, int max_workers, float* estimate) {
   const int round = 4 * sms;
-  if (max_workers <= 0 || chains <= round) return chains;
   static const float slow[5] = {0.f, 1.0f, 1.4f, 1.95f, 2.5f};
   int best = 1;
   float best_t = 0.f;
@@ -547,9 +579,28 @@ int warp_workers(int chains, int sms, int per_sm, int max_workers) {
       best_t = t;
     }
   }
-  int workers = best * round;
+  if (best_t == 0.f) best_t = (float)chains / (float)round;   // no sharing possible: whole chains in waves
+  *estimate = best_t;
+  return best;
+}
+
+int warp_workers(int chains, int sms, int per_sm, int max_workers) {
+  const int round = 4 * sms;
+  if (max_workers <= 0 || chains <= round) return chains;
+  float t;
+  int workers = warp_rounds(chains, sms, per_sm, max_workers, &t) * round;
   if (workers > max_workers) workers = max_workers;
   return workers;
+}
+
+// The estimate behind warp_workers, in units of the time one warp alone on its sub-partition needs for one chain.
+float warp_run_estimate(int chains, int sms, int per_sm, int max_workers) {
+  const int round = 4 * sms;
+  if (chains <= round) return 1.f;
+  float t;
+  if (max_workers <= 0) return (float)((chains + round - 1) / round);
+  warp_rounds(chains, sms, per_sm, max_workers, &t);
+  return t;
 }
 
 bool fwd_fast_applicable(const ssm_problem_t& prob, const FwdParams& p) {
