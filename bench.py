@@ -31,8 +31,8 @@ FALLBACK_HBM_GBS = 6650.0
 # DRAM bytes (read + write) of one launch of the dominant kernel of each direction from ncu captures at the bench
 # workload itself (profiles/ssm_bwd_warp_kernel_mamba2p8b_layer.md, profiles/ssm_fwd_warp_kernel_mamba2p8b_layer.md);
 # None where no capture exists.
-NCU_TRAFFIC_BYTES = {3: 705.7e6 + 395.8e6}
-NCU_TRAFFIC_BYTES_FWD = {3: 264.0e6 + 369.8e6}
+NCU_TRAFFIC_BYTES = {3: 705.3e6 + 396.0e6}
+NCU_TRAFFIC_BYTES_FWD = {3: 263.8e6 + 368.5e6}
 
 
 def parse_args():
@@ -156,7 +156,8 @@ def kernels_per_step(plan_info: dict, bwd_plan_info: dict) -> int:
     """Kernel launches of one fwd (saving states) + bwd (given saved states) pass; each direction splits the sequence
     in time on its own terms."""
     fwd = 1 if plan_info["n_segments"] == 1 else 3        # [summary, carry,] forward
-    bwd = 2 if bwd_plan_info["n_segments"] == 1 else 4    # [adjoint pre-pass, carry,] backward, reduction
+    # [adjoint pre-pass, carry (not with two segments: the pre-pass writes the inflow itself),] backward, reduction
+    bwd = {1: 2, 2: 3}.get(bwd_plan_info["n_segments"], 4)
     return fwd + bwd
 
 

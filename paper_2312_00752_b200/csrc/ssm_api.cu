@@ -30,8 +30,9 @@ size_t bwd_handoff_bytes_per_worker();
 
 // Shapes the tuned warp-per-worker kernels take (they also want 16-byte aligned pointers, checked per call).
 static bool tuned_shape(const ssm_problem_t& p) {
-  return p.io_dtype == SSM_BF16 && p.N == 16 && p.D % 8 == 0 &&
-         !(p.flags & (SSM_FLAG_STATIC_B | SSM_FLAG_STATIC_C | SSM_FLAG_COMPLEX));
+  const bool static_bc = p.flags & (SSM_FLAG_STATIC_B | SSM_FLAG_STATIC_C);
+  return p.io_dtype == SSM_BF16 && p.N == 16 && p.D % 8 == 0 && !(p.flags & SSM_FLAG_COMPLEX) &&
+         !(static_bc && (p.flags & SSM_FLAG_ZOH_BBAR));   // non-selective B / C: tuned with the default B-bar rule only
 }
 // Workers the hand-off slots of a workspace allow for `chains` chains: none while every chain can have a warp of its
 // own in the first round (one warp per SM sub-partition); else at least two rounds (a kernel may share chains between

@@ -42,17 +42,19 @@ constexpr int kWarpsPerBlock = 4;
 static_assert(kWT % kSub == 0, "tiles are whole sub-blocks");
 
 // NST ring stages: 3 (two tiles in flight) or 2 (one tile in flight; small enough for two blocks per SM in FULL mode)
-template <int CW, bool FULL, bool SP, bool BCW, int NST>
+// BC: bit 0 = B is a per-channel parameter (no B tile), bit 1 = the same for C (Algorithm 1's non-selective B / C)
+template <int CW, bool FULL, bool SP, int BC, int NST>
 struct FwdWarpSmem {
+  static constexpr bool TB = !(BC & 1), TC = FULL && !(BC & 2);   // tiles of B / C are staged
   uint32_t x[NST][kWT][CW / 2];   // bf16 pairs, CW channels
   uint32_t d[NST][kWT][CW / 2];
   uint32_t z[FULL ? NST : 1][FULL ? kWT : 1][CW / 2];
   // B and C rows are padded (12 and 20 words instead of 8 and 16) so that the one-row-per-lane widening pass of a
   // tile reads and writes them without bank conflicts
-  uint32_t rB[NST][kWT][12];  // bf16 pairs, 16 states
-  uint32_t rC[FULL ? NST : 1][FULL ? kWT : 1][12];
-  float fB[BCW ? kWT : 1][20];     // BCW: B and C of the current tile widened to float
-  float fC[(BCW && FULL) ? kWT : 1][20];
+  uint32_t rB[TB ? NST : 1][TB ? kWT : 1][12];  // bf16 pairs, 16 states
+  uint32_t rC[TC ? NST : 1][TC ? kWT : 1][12];
+  float fB[TB ? kWT : 1][20];      // B and C of the current tile widened to float
+  float fC[TC ? kWT : 1][20];
   float dF[SP ? kWT : 1][CW];      // SP: step sizes after bias and softplus
   uint32_t o[FULL ? kWT : 1][CW / 2];  // output tile (bf16 pairs)
 };
@@ -65,7 +67,7 @@ __device__ __forceinline__ float bf16at(const uint32_t* row, int c) {
 
 }  // namespace
 
-template <int S, int MODE, bool SP, bool ZOH, bool BCW, int NST>
+template <int S, int MODE, bool SP, bool ZOH, int BC, int NST>
 __global__ void __launch_bounds__(kWarpsPerBlock * 32) ssm_fwd_warp_kernel(const FwdParams p, const WarpSched sc) {
   static_assert(NST == 2 || NST == 3, "ring stages");
   static_assert(S == 16 || S == 8, "one lane or a lane pair per channel");
@@ -75,7 +77,8 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32) ssm_fwd_warp_kernel(const
   constexpr int CH = CW / 8;        // 16-byte chunks per tile row of x, delta, z, out
   constexpr int RP = 32 / CH;       // tile rows a warp covers with one chunk per lane
   constexpr int HV = S / 4 + 1;     // float4 per lane of a hand-off: S states, sum of delta
-  using Smem = FwdWarpSmem<CW, FULL, SP, BCW, NST>;
+  using Smem = FwdWarpSmem<CW, FULL, SP, BC, NST>;
+  constexpr bool TB = Smem::TB, TC = Smem::TC;   // B / C are inputs [batch][L][16] staged in tiles (else parameters)
   extern __shared__ __align__(16) unsigned char smem_raw[];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   Smem& sm = reinterpret_cast<Smem*>(smem_raw)[warp];
@@ -91,17 +94,7 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32) ssm_fwd_warp_kernel(const
   const __nv_bfloat16* __restrict__ gC = static_cast<const __nv_bfloat16*>(p.C);
   __nv_bfloat16* __restrict__ gout = static_cast<__nv_bfloat16*>(p.out);
 
-  // this thread's S states of a packed B or C row (16 states as 8 bf16 pairs), widened
-  auto load_states = [&](const uint32_t* row, float2 (&v)[H]) {
-#pragma unroll
-    for (int k = 0; k < H / 4; ++k) {
-      const uint4 a = *reinterpret_cast<const uint4*>(row + H * j + 4 * k);
-      const uint32_t w[4] = {a.x, a.y, a.z, a.w};
-#pragma unroll
-      for (int i = 0; i < 4; ++i) v[4 * k + i] = make_float2(bf16lo(w[i]), bf16hi(w[i]));
-    }
-  };
-  // the same from a row of 16 floats
+  // this thread's S states of a row of 16 floats
   auto load_states_f = [&](const float* row, float2 (&v)[H]) {
 #pragma unroll
     for (int k = 0; k < H / 2; ++k) {
@@ -153,8 +146,8 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32) ssm_fwd_warp_kernel(const
           const int tt = brow + 16 * k;
           const bool ok = t0 + tt < t_to;
           const size_t go = ok ? bo + (size_t)k * 16 * 16 : 0;
-          cp_async16(&sm.rB[st][tt][bhc * 4], gB + go, ok);
-          if (FULL) cp_async16(&sm.rC[st][tt][bhc * 4], gC + go, ok);
+          if constexpr (TB) cp_async16(&sm.rB[st][tt][bhc * 4], gB + go, ok);
+          if constexpr (TC) cp_async16(&sm.rC[st][tt][bhc * 4], gC + go, ok);
         }
       }
       cp_async_commit();
@@ -168,6 +161,24 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32) ssm_fwd_warp_kernel(const
     float2 A2[H];    // A * log2(e)
     float2 h[H];
     float2 invA[ZOH ? H : 1];   // ZOH: 1 / A (0 where A = 0)
+    float2 Bst[TB ? 1 : H], Cst[(TC || !FULL) ? 1 : H];   // B / C as parameters: this thread's entries
+    if constexpr (!TB || (FULL && !TC)) {
+#pragma unroll
+      for (int k = 0; k < S / 4; ++k) {
+        if constexpr (!TB) {
+          float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+          if (valid) v = *reinterpret_cast<const float4*>(static_cast<const float*>(p.B) + (size_t)c_own * 16 + S * j + 4 * k);
+          Bst[2 * k] = make_float2(v.x, v.y);
+          Bst[2 * k + 1] = make_float2(v.z, v.w);
+        }
+        if constexpr (FULL && !TC) {
+          float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+          if (valid) v = *reinterpret_cast<const float4*>(static_cast<const float*>(p.C) + (size_t)c_own * 16 + S * j + 4 * k);
+          Cst[2 * k] = make_float2(v.x, v.y);
+          Cst[2 * k + 1] = make_float2(v.z, v.w);
+        }
+      }
+    }
     float a0s, rs;
     float minA = 3.0e38f;       // ZOH: smallest |A| among this thread's states
     bool ap = !p.general_A;
@@ -283,12 +294,17 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32) ssm_fwd_warp_kernel(const
         auto front = [&](int t, float2 (&a)[H], float2 (&bxF)[H], float2 (&CvF)[FULL ? H : 1]) {
           const int r = SSM_TILE_ROW(r0 + gb * GB + t, kWT, sc.abort);
           float2 Bv[H];
-          if constexpr (BCW) {
+          if constexpr (TB) {
             load_states_f(sm.fB[r], Bv);
-            if constexpr (FULL) load_states_f(sm.fC[r], CvF);
           } else {
-            load_states(sm.rB[st][r], Bv);
-            if constexpr (FULL) load_states(sm.rC[st][r], CvF);
+#pragma unroll
+            for (int k = 0; k < H; ++k) Bv[k] = Bst[k];
+          }
+          if constexpr (TC) {
+            load_states_f(sm.fC[r], CvF);
+          } else if constexpr (FULL) {
+#pragma unroll
+            for (int k = 0; k < H; ++k) CvF[k] = Cst[k];
           }
           if constexpr (AP) {
             const float a0 = e0[t], rr = e1[t];
@@ -369,7 +385,7 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32) ssm_fwd_warp_kernel(const
       issue_tile(i + NST - 1);  // into the stage tile i - 1 used
       const int st = i % NST;
       const int t0 = t_from + i * kWT;
-      if constexpr (BCW) {
+      if constexpr (TB) {
         // B and C of the tile to float, one row per lane
         const uint4 b0 = *reinterpret_cast<const uint4*>(&sm.rB[st][lane][0]), b1 = *reinterpret_cast<const uint4*>(&sm.rB[st][lane][4]);
         const uint32_t wb[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
@@ -377,7 +393,9 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32) ssm_fwd_warp_kernel(const
         for (int k = 0; k < 4; ++k)
           *reinterpret_cast<float4*>(&sm.fB[lane][4 * k]) =
               make_float4(bf16lo(wb[2 * k]), bf16hi(wb[2 * k]), bf16lo(wb[2 * k + 1]), bf16hi(wb[2 * k + 1]));
-        if constexpr (FULL) {
+      }
+      if constexpr (TC) {
+        {
           const uint4 c0 = *reinterpret_cast<const uint4*>(&sm.rC[st][lane][0]), c1 = *reinterpret_cast<const uint4*>(&sm.rC[st][lane][4]);
           const uint32_t wc[8] = {c0.x, c0.y, c0.z, c0.w, c1.x, c1.y, c1.z, c1.w};
 #pragma unroll
@@ -385,8 +403,8 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32) ssm_fwd_warp_kernel(const
             *reinterpret_cast<float4*>(&sm.fC[lane][4 * k]) =
                 make_float4(bf16lo(wc[2 * k]), bf16hi(wc[2 * k]), bf16lo(wc[2 * k + 1]), bf16hi(wc[2 * k + 1]));
         }
-        if constexpr (!SP) __syncwarp();
       }
+      if constexpr ((TB || TC) && !SP) __syncwarp();
       if constexpr (SP) {
         // step sizes of the tile, once per element: pre-activation + bias, softplus; rows past the end stay identity
         // steps (delta = 0)
@@ -475,18 +493,18 @@ constexpr int kFwdS = 16;  // a lane per channel, 32-channel chains
 
 namespace {
 
-template <int S, int MODE, bool SP, bool ZOH, bool BCW, int NST>
+template <int S, int MODE, bool SP, bool ZOH, int BC, int NST>
 cudaError_t fwd_occupancy(int* per_sm, size_t* smem_bytes) {
   constexpr int CW = 2 * S;   // channels per chain
-  const size_t smem = sizeof(FwdWarpSmem<CW, MODE == kFwdFull, SP, BCW, NST>) * kWarpsPerBlock;
-  auto kern = ssm_fwd_warp_kernel<S, MODE, SP, ZOH, BCW, NST>;
+  const size_t smem = sizeof(FwdWarpSmem<CW, MODE == kFwdFull, SP, BC, NST>) * kWarpsPerBlock;
+  auto kern = ssm_fwd_warp_kernel<S, MODE, SP, ZOH, BC, NST>;
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
   *smem_bytes = smem;
   return cudaOccupancyMaxActiveBlocksPerMultiprocessor(per_sm, kern, kWarpsPerBlock * 32, smem);
 }
 
-template <int S, int MODE, bool SP, bool ZOH, bool BCW>
+template <int S, int MODE, bool SP, bool ZOH, int BC>
 cudaError_t launch_variant_w(const Plan& plan, const FwdParams& p, cudaStream_t s) {
   constexpr int CW = 2 * S;   // channels per chain
   int dev = 0, sms = 0, per_sm = 0;
@@ -494,7 +512,7 @@ cudaError_t launch_variant_w(const Plan& plan, const FwdParams& p, cudaStream_t 
   cudaError_t e;
   if ((e = cudaGetDevice(&dev)) != cudaSuccess) return e;
   if ((e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
-  if ((e = fwd_occupancy<S, MODE, SP, ZOH, BCW, 3>(&per_sm, &smem)) != cudaSuccess) return e;
+  if ((e = fwd_occupancy<S, MODE, SP, ZOH, BC, 3>(&per_sm, &smem)) != cudaSuccess) return e;
   if (per_sm < 1) return cudaErrorLaunchOutOfResources;
   WarpSched sc{};
   sc.chains = p.batch * plan.nseg * ((p.D + CW - 1) / CW);
@@ -504,10 +522,10 @@ cudaError_t launch_variant_w(const Plan& plan, const FwdParams& p, cudaStream_t 
   // The two-stage ring (one tile in flight instead of two) lets more warps share an SM: taken when that shortens the
   // estimated run by more than the shorter prefetch distance may cost.
   bool two_stage = false;
-  if constexpr (!ZOH && MODE != kFwdSummary) {
+  if constexpr (!ZOH && MODE != kFwdSummary && BC == 0) {
     int per_sm2 = 0;
     size_t smem2 = 0;
-    if ((e = fwd_occupancy<S, MODE, SP, ZOH, BCW, 2>(&per_sm2, &smem2)) != cudaSuccess) return e;
+    if ((e = fwd_occupancy<S, MODE, SP, ZOH, BC, 2>(&per_sm2, &smem2)) != cudaSuccess) return e;
     if (per_sm2 > per_sm && warp_run_estimate(sc.chains, sms, per_sm2 * kWarpsPerBlock, max_workers) <
                                 0.93f * warp_run_estimate(sc.chains, sms, per_sm * kWarpsPerBlock, max_workers)) {
       two_stage = true;
@@ -523,21 +541,25 @@ cudaError_t launch_variant_w(const Plan& plan, const FwdParams& p, cudaStream_t 
   sc.abort = p.abort;
   sc.handoff = p.handoff;
   const unsigned grid = (unsigned)((sc.workers + kWarpsPerBlock - 1) / kWarpsPerBlock);
-  if constexpr (!ZOH && MODE != kFwdSummary) {
+  if constexpr (!ZOH && MODE != kFwdSummary && BC == 0) {
     if (two_stage) {
-      ssm_fwd_warp_kernel<S, MODE, SP, ZOH, BCW, 2><<<grid, kWarpsPerBlock * 32, smem, s>>>(p, sc);
+      ssm_fwd_warp_kernel<S, MODE, SP, ZOH, BC, 2><<<grid, kWarpsPerBlock * 32, smem, s>>>(p, sc);
       return cudaGetLastError();
     }
   }
-  ssm_fwd_warp_kernel<S, MODE, SP, ZOH, BCW, 3><<<grid, kWarpsPerBlock * 32, smem, s>>>(p, sc);
+  ssm_fwd_warp_kernel<S, MODE, SP, ZOH, BC, 3><<<grid, kWarpsPerBlock * 32, smem, s>>>(p, sc);
   return cudaGetLastError();
 }
 
 template <int S, int MODE, bool SP, bool ZOH>
 cudaError_t launch_variant(const Plan& plan, const FwdParams& p, cudaStream_t s) {
-  // B and C widened to float once per tile (BCW): measured faster than unpacking bf16 in the step loop at 16 states
-  // per thread.
-  return launch_variant_w<S, MODE, SP, ZOH, true>(plan, p, s);
+  // non-selective B / C (parameters [D][16]): variants without the ZOH rule only (fwd_fast_applicable)
+  if constexpr (!ZOH) {
+    if (p.static_B && p.static_C) return launch_variant_w<S, MODE, SP, ZOH, 3>(plan, p, s);
+    if (p.static_B) return launch_variant_w<S, MODE, SP, ZOH, 1>(plan, p, s);
+    if (p.static_C) return launch_variant_w<S, MODE, SP, ZOH, 2>(plan, p, s);
+  }
+  return launch_variant_w<S, MODE, SP, ZOH, 0>(plan, p, s);
 }
 
 template <int S, int MODE>
@@ -605,7 +627,7 @@ float warp_run_estimate(int chains, int sms, int per_sm, int max_workers) {
 
 bool fwd_fast_applicable(const ssm_problem_t& prob, const FwdParams& p) {
   auto al16 = [](const void* q) { return q == nullptr || (reinterpret_cast<uintptr_t>(q) & 15) == 0; };
-  if (p.static_B || p.static_C) return false;  // input-dependent B, C only
+  if ((p.static_B || p.static_C) && p.zoh) return false;  // non-selective B / C: default B-bar rule only
   return prob.io_dtype == SSM_BF16 && prob.N == 16 && prob.D % 8 == 0 && al16(p.x) && al16(p.delta) && al16(p.z) &&
          al16(p.B) && al16(p.C) && al16(p.out) && al16(p.A) && al16(p.h_start) && al16(p.ckpt) && al16(p.seg_end) &&
          al16(p.h_last) && al16(p.handoff);

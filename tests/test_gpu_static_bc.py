@@ -48,6 +48,10 @@ def _oracle_static(inp, Bs, Cs, zoh=False):
     (2, 70, 12, 8, "f32", True, False, False),       # selective C only
     (1, 90, 16, 4, "f32", False, True, True),        # selective B only, ZOH rule
     (1, 1200, 16, 16, "f32", True, True, False),     # time split: the adjoint pre-pass with static C
+    (2, 130, 40, 16, "bf16", True, False, False),    # tuned kernels (bf16, N = 16, default B-bar rule): selective C only
+    (1, 97, 72, 16, "bf16", False, True, False),     # tuned kernels: selective B only, channel blocks 32 + 32 + 8
+    (1, 4200, 48, 16, "bf16", True, True, False),    # tuned kernels with a time split in both directions
+    (2, 64, 32, 16, "bf16", True, True, True),       # ZOH with non-selective B / C stays on the generic kernels
 ])
 def test_static_b_and_c(batch, L, D, N, io, sB, sC, zoh):
     import torch
