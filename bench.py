@@ -232,7 +232,8 @@ def run_reference(args, cfg):
 
 
 # ------------------------------------------------------------------------------------------------ our arm
-def time_shape(K, torch, dev, stream, cfg, peak, general_A=False, reps=None, zoh=False, complex_state=False):
+def time_shape(K, torch, dev, stream, cfg, peak, general_A=False, reps=None, zoh=False, complex_state=False,
+               static_bc=False):
     """Forward (saving states) and backward times of one more workload, with timing-only inputs drawn on the device
     (same shapes and value ranges as the seeded host recipe); every repetition is timed on its own with CUDA events and
     a buffer larger than L2 is overwritten in between."""
@@ -244,6 +245,8 @@ def time_shape(K, torch, dev, stream, cfg, peak, general_A=False, reps=None, zoh
     rn = lambda shape: torch.randn(shape, generator=g, device=dev, dtype=torch.float32)
     t = {k: rn(shp).to(io_t) for k in ("x", "z", "dout")}
     t["B"], t["C"] = rn(bshp).to(io_t), rn(bshp).to(io_t)
+    if static_bc:   # B and C as float32 parameters [D][N] (Algorithm 1)
+        t["B"], t["C"] = rn((cfg.D, cfg.N)), rn((cfg.D, cfg.N))
     tau = torch.exp(torch.empty(cfg.D, device=dev).uniform_(math.log(cfg.dt_min), math.log(cfg.dt_max), generator=g))
     bias = tau + torch.log(-torch.expm1(-tau))
     t["delta"] = torch.nn.functional.softplus(0.1 * rn(shp) + bias).to(io_t)
@@ -255,7 +258,10 @@ def time_shape(K, torch, dev, stream, cfg, peak, general_A=False, reps=None, zoh
                          torch.arange(cfg.N, device=dev, dtype=torch.float32).repeat(cfg.D, 1)], dim=-1).contiguous()
     Dk = torch.ones(cfg.D, device=dev)
     opts = dict(zoh=zoh, complex_state=complex_state) if (zoh or complex_state) else {}
-    prob = K.make_problem(t["x"], t["B"], True, True, save_states=True, zoh=zoh, complex_state=complex_state)
+    if static_bc:
+        opts = dict(static_B=True, static_C=True)
+    prob = K.make_problem(t["x"], t["B"], True, True, save_states=True, zoh=zoh, complex_state=complex_state,
+                          static_B=static_bc, static_C=static_bc)
     out = torch.empty_like(t["x"])
     saved = torch.empty(K.saved_state_bytes(prob) // 4, dtype=torch.float32, device=dev)
     grads = {"dx": torch.empty_like(t["x"]), "ddelta": torch.empty_like(t["x"]), "dz": torch.empty_like(t["x"]),
@@ -284,7 +290,8 @@ def time_shape(K, torch, dev, stream, cfg, peak, general_A=False, reps=None, zoh
     res = {"workload": f"config {cfg.cfg_id}: batch {cfg.batch}, L {cfg.L}, D {cfg.D}, N {cfg.N}, {cfg.io} io" +
                        (", A perturbed (no arithmetic progression: one exponential per state)" if general_A else "") +
                        (", zero-order-hold B-bar (SSM_FLAG_ZOH_BBAR)" if zoh else "") +
-                       (", complex state with S4D-Lin A (SSM_FLAG_COMPLEX; plain kernels)" if complex_state else ""),
+                       (", complex state with S4D-Lin A (SSM_FLAG_COMPLEX; plain kernels)" if complex_state else "") +
+                       (", B and C as parameters (SSM_FLAG_STATIC_B | SSM_FLAG_STATIC_C)" if static_bc else ""),
            "fwd_ms": f, "bwd_ms": b, "fwd_elements_per_s": cfg.elements / (f * 1e-3),
            "bwd_elements_per_s": cfg.elements / (b * 1e-3), "step_elements_per_s": cfg.elements / ((f + b) * 1e-3),
            "fwd_frac_of_hbm_peak": fb / (f * 1e-3) / 1e9 / peak, "bwd_frac_of_hbm_peak": bb / (b * 1e-3) / 1e9 / peak,
@@ -536,7 +543,8 @@ def run_ours(args, cfg):
     if not args.no_extras:
         line["general_A"] = time_shape(K, torch, dev, stream, cfg, peak, general_A=True)
         line["variants"] = {}
-        for name, kw in (("zoh", dict(zoh=True)), ("complex_state", dict(complex_state=True))):
+        for name, kw in (("zoh", dict(zoh=True)), ("static_bc", dict(static_bc=True)),
+                         ("complex_state", dict(complex_state=True))):
             try:
                 line["variants"][name] = time_shape(K, torch, dev, stream, cfg, peak, reps=5, **kw)
             except Exception as exc:

@@ -80,7 +80,8 @@ enum {
                                  instead of the default delta * B; honoured by every call                        */
   SSM_FLAG_STATIC_B = 256u,   /* B is not input-dependent (Algorithm 1; the selective-parameter ablation, Table 7): B is a float32
                                  parameter [D][N] like A instead of io_dtype [batch][L][N], and dB is float32 [D][N],
-                                 summed over batch and time.  Generic kernels.                                    */
+                                 summed over batch and time.  Tuned kernels for bf16 / N = 16 with the default B-bar
+                                 rule, generic kernels otherwise.                                                */
   SSM_FLAG_STATIC_C = 512u,   /* the same for C and dC                                                            */
   SSM_FLAG_COMPLEX = 1024u,   /* complex-valued state (Section 3.6): A and dA are float32 [D][N][2], B, C, dB, dC io_dtype
                                  [batch][L][N][2], every state array (saved_states, h0, h_last, dh_last, dh0, the h of

@@ -250,15 +250,18 @@ def ssm_scan_fwd(x, delta, A, B, C, D_skip=None, z=None, *, save_states=False, g
 
 
 def ssm_scan_fwd_fused_dt(x, delta_pre, delta_bias, A, B, C, D_skip=None, z=None, *, softplus=True, save_states=False,
-                          out=None, saved_states=None, stream=None, h0=None, h_last=None, zoh=False):
+                          out=None, saved_states=None, stream=None, h0=None, h_last=None, zoh=False, static_B=False,
+                          static_C=False):
     """Forward with the step-size activation fused: delta = softplus(delta_pre + delta_bias) (or the plain sum with
-    softplus=False), in float32.  Otherwise as ssm_scan_fwd."""
+    softplus=False), in float32.  Otherwise as ssm_scan_fwd (static_B / static_C: B / C float32 (D, N))."""
     lib = load_library()
-    prob = make_problem(x, B, z is not None, D_skip is not None, save_states, False, zoh)
+    prob = make_problem(x, B, z is not None, D_skip is not None, save_states, False, zoh, static_B, static_C)
     if softplus:
         prob.flags |= SSM_FLAG_DELTA_SOFTPLUS
     batch, L, D, N = prob.batch, prob.L, prob.D, prob.N
     io = x.dtype
+    bshape, bdt = ((D, N), torch.float32) if static_B else ((batch, L, N), io)
+    cshape, cdt = ((D, N), torch.float32) if static_C else ((batch, L, N), io)
     if out is None:
         out = torch.empty_like(x)
     if save_states and saved_states is None:
@@ -268,7 +271,7 @@ def ssm_scan_fwd_fused_dt(x, delta_pre, delta_bias, A, B, C, D_skip=None, z=None
     code = lib.ssm_scan_fwd_fused_dt(
         ctypes.byref(prob), _dev_ptr(x, "x", (batch, L, D), io), _dev_ptr(delta_pre, "delta_pre", (batch, L, D), io),
         _dev_ptr(delta_bias, "delta_bias", (D,), torch.float32), _dev_ptr(A, "A", (D, N), torch.float32),
-        _dev_ptr(B, "B", (batch, L, N), io), _dev_ptr(C, "C", (batch, L, N), io),
+        _dev_ptr(B, "B", bshape, bdt), _dev_ptr(C, "C", cshape, cdt),
         _dev_ptr(D_skip, "D_skip", (D,), torch.float32), _dev_ptr(z, "z", (batch, L, D), io),
         _dev_ptr(h0, "h0", (batch, D, N), torch.float32), _dev_ptr(out, "out", (batch, L, D), io),
         _dev_ptr(h_last, "h_last", (batch, D, N), torch.float32),
@@ -280,19 +283,22 @@ def ssm_scan_fwd_fused_dt(x, delta_pre, delta_bias, A, B, C, D_skip=None, z=None
 
 
 def ssm_scan_bwd_fused_dt(x, delta_pre, delta_bias, A, B, C, D_skip, z, dout, saved_states=None, *, softplus=True,
-                          stream=None, zoh=False, h0=None, dh_last=None, want_dh0=False):
+                          stream=None, zoh=False, h0=None, dh_last=None, want_dh0=False, static_B=False,
+                          static_C=False):
     """Backward of ssm_scan_fwd_fused_dt.  Returns the dict of ssm_scan_bwd with `ddelta` the gradient of delta_pre
     and an extra `ddelta_bias` (D,) float32.  h0, dh_last, want_dh0 as in ssm_scan_bwd (ssm_scan_bwd_fused_dt_state)."""
     lib = load_library()
-    prob = make_problem(x, B, z is not None, D_skip is not None, False, False, zoh)
+    prob = make_problem(x, B, z is not None, D_skip is not None, False, False, zoh, static_B, static_C)
     if softplus:
         prob.flags |= SSM_FLAG_DELTA_SOFTPLUS
     batch, L, D, N = prob.batch, prob.L, prob.D, prob.N
     io = x.dtype
+    bshape, bdt = ((D, N), torch.float32) if static_B else ((batch, L, N), io)
+    cshape, cdt = ((D, N), torch.float32) if static_C else ((batch, L, N), io)
     o = {"dx": torch.empty_like(x), "ddelta": torch.empty_like(x),
          "ddelta_bias": torch.empty((D,), dtype=torch.float32, device=x.device),
          "dA": torch.empty((D, N), dtype=torch.float32, device=x.device), "dB": torch.empty_like(B),
-         "dC": torch.empty_like(B),
+         "dC": torch.empty_like(C),
          "dD": torch.empty((D,), dtype=torch.float32, device=x.device) if D_skip is not None else None,
          "dz": torch.empty_like(x) if z is not None else None}
     stream_ptr = (stream if stream is not None else torch.cuda.current_stream(x.device)).cuda_stream
@@ -304,7 +310,7 @@ def ssm_scan_bwd_fused_dt(x, delta_pre, delta_bias, A, B, C, D_skip, z, dout, sa
         code = lib.ssm_scan_bwd_fused_dt_state(
             ctypes.byref(prob), _dev_ptr(x, "x", (batch, L, D), io), _dev_ptr(delta_pre, "delta_pre", (batch, L, D), io),
             _dev_ptr(delta_bias, "delta_bias", (D,), f32), _dev_ptr(A, "A", (D, N), f32),
-            _dev_ptr(B, "B", (batch, L, N), io), _dev_ptr(C, "C", (batch, L, N), io), _dev_ptr(D_skip, "D_skip", (D,), f32),
+            _dev_ptr(B, "B", bshape, bdt), _dev_ptr(C, "C", cshape, cdt), _dev_ptr(D_skip, "D_skip", (D,), f32),
             _dev_ptr(z, "z", (batch, L, D), io), _dev_ptr(dout, "dout", (batch, L, D), io),
             _dev_ptr(h0, "h0", (batch, D, N), f32), _dev_ptr(dh_last, "dh_last", (batch, D, N), f32),
             _dev_ptr(saved_states, "saved_states"), _dev_ptr(o["dx"], "dx"), _dev_ptr(o["ddelta"], "ddelta"),
@@ -317,7 +323,7 @@ def ssm_scan_bwd_fused_dt(x, delta_pre, delta_bias, A, B, C, D_skip, z, dout, sa
     code = lib.ssm_scan_bwd_fused_dt(
         ctypes.byref(prob), _dev_ptr(x, "x", (batch, L, D), io), _dev_ptr(delta_pre, "delta_pre", (batch, L, D), io),
         _dev_ptr(delta_bias, "delta_bias", (D,), torch.float32), _dev_ptr(A, "A", (D, N), torch.float32),
-        _dev_ptr(B, "B", (batch, L, N), io), _dev_ptr(C, "C", (batch, L, N), io),
+        _dev_ptr(B, "B", bshape, bdt), _dev_ptr(C, "C", cshape, cdt),
         _dev_ptr(D_skip, "D_skip", (D,), torch.float32), _dev_ptr(z, "z", (batch, L, D), io),
         _dev_ptr(dout, "dout", (batch, L, D), io), _dev_ptr(saved_states, "saved_states"),
         _dev_ptr(o["dx"], "dx"), _dev_ptr(o["ddelta"], "ddelta"), _dev_ptr(o["ddelta_bias"], "ddelta_bias"),

@@ -26,7 +26,7 @@ int fwd_fast_channels_per_warp();
 int bwd_fast_channels_per_warp();
 bool bwd_fast_applicable(const ssm_problem_t& prob, const BwdParams& p);
 size_t fwd_handoff_bytes_per_worker();
-size_t bwd_handoff_bytes_per_worker();
+size_t bwd_handoff_bytes_per_worker(bool static_B, bool static_C);
 
 // Shapes the tuned warp-per-worker kernels take (they also want 16-byte aligned pointers, checked per call).
 static bool tuned_shape(const ssm_problem_t& p) {
@@ -203,7 +203,8 @@ static BwdWorkspace bwd_layout(const ssm_problem_t& p, const Plan& pl, const Pla
   w.max_workers = !tuned_shape(p) ? 0 : (p.flags & SSM_FLAG_TEST_WITHHOLD) ? (int)std::max<long long>(1, (2 * chains + 2) / 3)
                                                                             : shared_workers(chains);
   w.flags = take((size_t)2 * (w.max_workers + 1) * sizeof(int));   // backward kernel | adjoint pre-pass
-  w.handoff = take((size_t)(w.max_workers + 1) * bwd_handoff_bytes_per_worker());
+  w.handoff = take((size_t)(w.max_workers + 1) *
+                   bwd_handoff_bytes_per_worker(p.flags & SSM_FLAG_STATIC_B, p.flags & SSM_FLAG_STATIC_C));
   if (p.flags & SSM_FLAG_STATIC_B) w.dBs_part = take(parts * p.D * p.N * sizeof(float));
   if (p.flags & SSM_FLAG_STATIC_C) w.dCs_part = take(parts * p.D * p.N * sizeof(float));
   w.total = off;

@@ -28,13 +28,14 @@ constexpr int kLStages = 3;      // ring stages
 constexpr int kLWarps = 4;       // warps per block
 constexpr int kLocalHandoffVec = 5;   // float4 per lane: 16 adjoint values, sum of delta
 
-template <bool SP>
+// SC: C is a per-channel parameter [D][16] (no C tile)
+template <bool SP, bool SC>
 struct LocalWarpSmem {
   uint32_t d[kLStages][kLT][16];   // bf16 pairs, 32 channels
   uint32_t z[kLStages][kLT][16];
   uint32_t g[kLStages][kLT][16];
-  uint32_t rC[kLStages][kLT][12];  // bf16 pairs, 16 states; rows padded against bank conflicts of the widening pass
-  float fC[kLT][20];               // C of the current tile widened to float (padded likewise)
+  uint32_t rC[SC ? 1 : kLStages][SC ? 1 : kLT][12];  // bf16 pairs, 16 states; rows padded against bank conflicts of the widening pass
+  float fC[SC ? 1 : kLT][20];               // C of the current tile widened to float (padded likewise)
   float dF[SP ? kLT : 1][32];      // SP: step sizes after bias and softplus
 };
 
@@ -43,10 +44,10 @@ __device__ __forceinline__ void cp_async_wait_but_one() { asm volatile("cp.async
 }  // namespace
 
 // SP: `delta` holds the pre-activation and the step size is delta + bias, through the softplus if asked (Algorithm 2 step 4)
-template <bool SP>
+template <bool SP, bool SC>
 __global__ void __launch_bounds__(kLWarps * 32) ssm_bwd_local_warp_kernel(const BwdParams p, const WarpSched sc) {
   constexpr int H = 8;   // float2 pairs of states per thread
-  using Smem = LocalWarpSmem<SP>;
+  using Smem = LocalWarpSmem<SP, SC>;
   extern __shared__ __align__(16) unsigned char smem_raw[];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   Smem& sm = reinterpret_cast<Smem*>(smem_raw)[warp];
@@ -106,7 +107,7 @@ __global__ void __launch_bounds__(kLWarps * 32) ssm_bwd_local_warp_kernel(const 
           const int tt = brow + 16 * k;
           const bool ok = t0 + tt < t_seg_end;
           const size_t go = ok ? (row0 + tt) * 16 + bhc * 8 : 0;
-          cp_async16(&sm.rC[st][tt][bhc * 4], gC + go, ok);
+          if constexpr (!SC) cp_async16(&sm.rC[st][tt][bhc * 4], gC + go, ok);
         }
       }
       cp_async_commit();
@@ -135,6 +136,16 @@ __global__ void __launch_bounds__(kLWarps * 32) ssm_bwd_local_warp_kernel(const 
       for (int k = 0; k < H; ++k) A2[k] = make_float2(av[2 * k] * kLog2e, av[2 * k + 1] * kLog2e);
     }
     ap = __all_sync(0xffffffffu, ap);
+    float2 Cst[SC ? H : 1];   // C as a parameter: this channel's row
+    if constexpr (SC) {
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (valid) v = *reinterpret_cast<const float4*>(static_cast<const float*>(p.C) + (size_t)c_own * 16 + 4 * k);
+        Cst[2 * k] = make_float2(v.x, v.y);
+        Cst[2 * k + 1] = make_float2(v.z, v.w);
+      }
+    }
     const float a0s = A2[0].x, rs = A2[0].y - A2[0].x;
     const float bias_own = (SP && p.delta_bias != nullptr && valid) ? p.delta_bias[c_own] : 0.f;
     float dsum = 0.f;
@@ -199,7 +210,9 @@ __global__ void __launch_bounds__(kLWarps * 32) ssm_bwd_local_warp_kernel(const 
         const float2 ds2 = f2dup(dsv[t]);
 #pragma unroll
         for (int k = 0; k < 4; ++k) {
-          const float4 c = *reinterpret_cast<const float4*>(&sm.fC[r][4 * k]);
+          float4 c;
+          if constexpr (SC) c = make_float4(Cst[2 * k].x, Cst[2 * k].y, Cst[2 * k + 1].x, Cst[2 * k + 1].y);
+          else c = *reinterpret_cast<const float4*>(&sm.fC[r][4 * k]);
           mu[2 * k] = f2mul(a[2 * k], f2fma(make_float2(c.x, c.y), ds2, mu[2 * k]));
           mu[2 * k + 1] = f2mul(a[2 * k + 1], f2fma(make_float2(c.z, c.w), ds2, mu[2 * k + 1]));
         }
@@ -213,13 +226,15 @@ __global__ void __launch_bounds__(kLWarps * 32) ssm_bwd_local_warp_kernel(const 
       const int st = i % kLStages;
       const int t0 = t_seg0 + (tile_hi - i) * kLT;
       {
-        // C of the tile to float, one row per lane
-        const uint4 c0 = *reinterpret_cast<const uint4*>(&sm.rC[st][lane][0]), c1 = *reinterpret_cast<const uint4*>(&sm.rC[st][lane][4]);
-        const uint32_t wc[8] = {c0.x, c0.y, c0.z, c0.w, c1.x, c1.y, c1.z, c1.w};
+        if constexpr (!SC) {
+          // C of the tile to float, one row per lane
+          const uint4 c0 = *reinterpret_cast<const uint4*>(&sm.rC[st][lane][0]), c1 = *reinterpret_cast<const uint4*>(&sm.rC[st][lane][4]);
+          const uint32_t wc[8] = {c0.x, c0.y, c0.z, c0.w, c1.x, c1.y, c1.z, c1.w};
 #pragma unroll
-        for (int k = 0; k < 4; ++k)
-          *reinterpret_cast<float4*>(&sm.fC[lane][4 * k]) =
-              make_float4(bf16lo(wc[2 * k]), bf16hi(wc[2 * k]), bf16lo(wc[2 * k + 1]), bf16hi(wc[2 * k + 1]));
+          for (int k = 0; k < 4; ++k)
+            *reinterpret_cast<float4*>(&sm.fC[lane][4 * k]) =
+                make_float4(bf16lo(wc[2 * k]), bf16hi(wc[2 * k]), bf16lo(wc[2 * k + 1]), bf16hi(wc[2 * k + 1]));
+        }
         if constexpr (SP) {
           // step sizes of the tile, once per element; rows past the end of the segment stay identity steps
 #pragma unroll 8
@@ -266,17 +281,16 @@ __global__ void __launch_bounds__(kLWarps * 32) ssm_bwd_local_warp_kernel(const 
 
 bool bwd_local_fast_applicable(const ssm_problem_t& prob, const BwdParams& p) {
   auto al16 = [](const void* q) { return q == nullptr || (reinterpret_cast<uintptr_t>(q) & 15) == 0; };
-  if (p.static_C) return false;
   return prob.io_dtype == SSM_BF16 && prob.N == 16 && prob.D % 8 == 0 && p.seg_steps % kLT == 0 && al16(p.delta) &&
          al16(p.z) && al16(p.dout) && al16(p.C) && al16(p.A) && al16(p.seg_local) && al16(p.handoff);
 }
 
 namespace {
 
-template <bool SP>
+template <bool SP, bool SC>
 cudaError_t launch_local(const Plan& plan, const BwdParams& p, cudaStream_t s) {
-  const size_t smem = sizeof(LocalWarpSmem<SP>) * kLWarps;
-  auto kern = ssm_bwd_local_warp_kernel<SP>;
+  const size_t smem = sizeof(LocalWarpSmem<SP, SC>) * kLWarps;
+  auto kern = ssm_bwd_local_warp_kernel<SP, SC>;
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
   int dev = 0, sms = 0, per_sm = 0;
@@ -304,7 +318,9 @@ cudaError_t launch_local(const Plan& plan, const BwdParams& p, cudaStream_t s) {
 
 cudaError_t launch_bwd_local_fast(const Plan& plan, const BwdParams& p, cudaStream_t s) {
   if (plan.nseg < 2) return cudaSuccess;
-  return (p.softplus || p.delta_bias != nullptr) ? launch_local<true>(plan, p, s) : launch_local<false>(plan, p, s);
+  const bool sp = p.softplus || p.delta_bias != nullptr;
+  if (p.static_C) return sp ? launch_local<true, true>(plan, p, s) : launch_local<false, true>(plan, p, s);
+  return sp ? launch_local<true, false>(plan, p, s) : launch_local<false, false>(plan, p, s);
 }
 
 }  // namespace ssm

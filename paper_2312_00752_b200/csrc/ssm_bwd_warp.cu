@@ -40,7 +40,8 @@ constexpr int kSB = kCkptSteps;    // steps per sub-block = checkpoint spacing
 constexpr int kRB = 4;             // steps between two dB / dC transposes
 constexpr int kBwdWarps = 4;       // warps per block
 constexpr int kBwdFastChannels = 32;   // channels per warp of the mapping the launcher picks
-constexpr int kBwdHandoffVec = 9;  // float4 per lane: mu (4), dA (4), dD and dbias (1)
+// float4 per lane of a hand-off: mu (4), dA (4), dD and dbias (1), and 4 more for each of dB / dC that is a parameter
+__host__ __device__ constexpr int bwd_handoff_vec(int bc) { return 9 + 4 * ((bc & 1) + ((bc >> 1) & 1)); }
 constexpr float kInvLog2e = 0.6931471805599453f;
 static_assert(kSB == 8 && kBT % kSB == 0, "sub-blocks of 8 steps, whole sub-blocks per tile");
 
@@ -175,9 +176,13 @@ __device__ __forceinline__ void decays(float dt, const float2 (&A2)[H], float a0
 }
 
 // Per-thread state that lives along a chain
-template <int S, int CPT, bool ZOH>
+// BC: bit 0 = B is a per-channel parameter [D][16] (Algorithm 1's non-selective B), bit 1 = the same for C
+template <int S, int CPT, bool ZOH, int BC>
 struct ChainRegs {
   static constexpr int H = S / 2;
+  static constexpr bool SB = BC & 1, SC = BC & 2;
+  float2 Bst[SB ? CPT : 1][SB ? H : 1], dBs[SB ? CPT : 1][SB ? H : 1];   // the parameter and its gradient over time
+  float2 Cst[SC ? CPT : 1][SC ? H : 1], dCs[SC ? CPT : 1][SC ? H : 1];
   float2 A2[CPT][H];    // A * log2(e)
   // ZOH: B-bar = E B with the input gain E = (a - 1) / A (Eq. 4): 1 / A (0 where A = 0)
   float2 invA[ZOH ? CPT : 1][ZOH ? H : 1];
@@ -190,8 +195,8 @@ struct ChainRegs {
 
 // One sub-block of 8 steps: rows [r0, r0 + 8) of the tile; nlive = rows of the tile inside the segment.
 // ZS (ZOH only): some |delta A| of the sub-block is too small for the closed form of the input gain.
-template <int S, int CPT, bool SP, bool AP, bool ZOH, bool ZS>
-__device__ __forceinline__ void sub_block(const Lane<S, CPT>& ln, ChainRegs<S, CPT, ZOH>& cr, int r0, int nlive, float gate_on,
+template <int S, int CPT, bool SP, bool AP, bool ZOH, bool ZS, int BC>
+__device__ __forceinline__ void sub_block(const Lane<S, CPT>& ln, ChainRegs<S, CPT, ZOH, BC>& cr, int r0, int nlive, float gate_on,
                                           bool softplus, const uint32_t* tx, const uint32_t* td, const float* tfB,
                                           const float* tfC, const float* tds, const float* tgp, const float* tdF,
                                           const float4* tck, uint32_t* tox, uint32_t* tod, uint32_t* toz, float4* tred,
@@ -199,7 +204,11 @@ __device__ __forceinline__ void sub_block(const Lane<S, CPT>& ln, ChainRegs<S, C
   using LN = Lane<S, CPT>;
   constexpr int LPC = LN::LPC, H = LN::H, V = LN::V, CW = LN::CW, WPR = CW / 2;
   constexpr bool OWN = LN::OWN;
+  constexpr bool SB = BC & 1, SC = BC & 2;
   const int lane = ln.lane;
+  // B / C of a (step, channel, state pair): the staged row, or the channel's parameter
+  auto Bof = [&](const float2 (&Bv)[H], int q, int k) { return SB ? cr.Bst[SB ? q : 0][SB ? k : 0] : Bv[k]; };
+  auto Cof = [&](const float2 (&Cv)[H], int q, int k) { return SC ? cr.Cst[SC ? q : 0][SC ? k : 0] : Cv[k]; };
   // ZOH input gain E = (a - 1) / A and its derivative dE/dA = (delta a - E) / A, each with its series for small
   // delta A (which covers A = 0); dE/ddelta = a
   auto gain = [&](int q, int k, float2 a, float dtq) {
@@ -236,7 +245,7 @@ __device__ __forceinline__ void sub_block(const Lane<S, CPT>& ln, ChainRegs<S, C
     for (int t = 0; t < kSB; ++t) {
       const int r = SSM_TILE_ROW(r0 + t, kBT, abort_word);
       float2 Bv[H];
-      ln.load_states_f(tfB + r * 16, Bv);
+      if constexpr (!SB) ln.load_states_f(tfB + r * 16, Bv);
 #pragma unroll
       for (int q = 0; q < CPT; ++q) {
         float2 a[H];
@@ -244,7 +253,8 @@ __device__ __forceinline__ void sub_block(const Lane<S, CPT>& ln, ChainRegs<S, C
         const float2 du2 = f2dup(dt[t][q] * u[t][q]);
 #pragma unroll
         for (int k = 0; k < H; ++k) {
-          const float2 bx = ZOH ? f2mul(f2mul(gain(q, k, a[k], dt[t][q]), f2dup(u[t][q])), Bv[k]) : f2mul(du2, Bv[k]);
+          const float2 Bk = Bof(Bv, q, k);
+          const float2 bx = ZOH ? f2mul(f2mul(gain(q, k, a[k], dt[t][q]), f2dup(u[t][q])), Bk) : f2mul(du2, Bk);
           h[q][k] = f2fma(a[k], h[q][k], bx);
           if (t & 1) hist[t >> 1][q][k] = h[q][k];
         }
@@ -267,8 +277,8 @@ __device__ __forceinline__ void sub_block(const Lane<S, CPT>& ln, ChainRegs<S, C
     float y1[CPT], lb1[CPT], mb1[ZOH ? CPT : 1];   // mb: sum mu B (ZOH: the step-size gradient through E)
     {
       float2 Bv[H], Cv[H];
-      ln.load_states_f(tfB + r1 * 16, Bv);
-      ln.load_states_f(tfC + r1 * 16, Cv);
+      if constexpr (!SB) ln.load_states_f(tfB + r1 * 16, Bv);
+      if constexpr (!SC) ln.load_states_f(tfC + r1 * 16, Cv);
       float2 dBt[H], dCt[H];
 #pragma unroll
       for (int q = 0; q < CPT; ++q) {
@@ -280,25 +290,26 @@ __device__ __forceinline__ void sub_block(const Lane<S, CPT>& ln, ChainRegs<S, C
 #pragma unroll
         for (int k = 0; k < H; ++k) {
           const float2 hc = hist[m][q][k];
-          const float2 lam = f2fma(Cv[k], ds2, cr.mu[q][k]);
+          const float2 Bk = Bof(Bv, q, k), Ck = Cof(Cv, q, k);
+          const float2 lam = f2fma(Ck, ds2, cr.mu[q][k]);
           float2 lw = lam;
           if constexpr (ZOH) {
             const float2 E = gain(q, k, a[k], dt1[q]);
             lw = f2mul(lam, E);
             // dE/dA adds lam (dE/dA) B x to dA
-            cr.dA[q][k] = f2fma(f2mul(lam, gain_dA(q, k, a[k], E, dt1[q])), f2mul(Bv[k], f2dup(u1[q])), cr.dA[q][k]);
+            cr.dA[q][k] = f2fma(f2mul(lam, gain_dA(q, k, a[k], E, dt1[q])), f2mul(Bk, f2dup(u1[q])), cr.dA[q][k]);
           }
-          if (q == 0) {
-            dCt[k] = f2mul(ds2, hc);
-            dBt[k] = f2mul(lw, du2);
-          } else {
-            dCt[k] = f2fma(ds2, hc, dCt[k]);
-            dBt[k] = f2fma(lw, du2, dBt[k]);
-          }
-          lb = f2fma(lw, Bv[k], lb);
-          yv = f2fma(Cv[k], hc, yv);
+          // dB / dC terms: summed over the thread's channels for the cross-lane sum, or over time per channel
+          if constexpr (SC) cr.dCs[SC ? q : 0][SC ? k : 0] = f2fma(ds2, hc, cr.dCs[SC ? q : 0][SC ? k : 0]);
+          else if (q == 0) dCt[k] = f2mul(ds2, hc);
+          else dCt[k] = f2fma(ds2, hc, dCt[k]);
+          if constexpr (SB) cr.dBs[SB ? q : 0][SB ? k : 0] = f2fma(lw, du2, cr.dBs[SB ? q : 0][SB ? k : 0]);
+          else if (q == 0) dBt[k] = f2mul(lw, du2);
+          else dBt[k] = f2fma(lw, du2, dBt[k]);
+          lb = f2fma(lw, Bk, lb);
+          yv = f2fma(Ck, hc, yv);
           cr.mu[q][k] = f2mul(a[k], lam);
-          if constexpr (ZOH) mb = f2fma(cr.mu[q][k], Bv[k], mb);
+          if constexpr (ZOH) mb = f2fma(cr.mu[q][k], Bk, mb);
         }
         y1[q] = yv.x + yv.y;
         lb1[q] = lb.x + lb.y;
@@ -309,8 +320,9 @@ __device__ __forceinline__ void sub_block(const Lane<S, CPT>& ln, ChainRegs<S, C
       const int swz = (lane / (8 / V)) & (V - 1);
 #pragma unroll
       for (int v = 0; v < V / 2; ++v) {
-        rrow[v ^ swz] = make_float4(dBt[2 * v].x, dBt[2 * v].y, dBt[2 * v + 1].x, dBt[2 * v + 1].y);
-        rrow[(V / 2 + v) ^ swz] = make_float4(dCt[2 * v].x, dCt[2 * v].y, dCt[2 * v + 1].x, dCt[2 * v + 1].y);
+        if constexpr (!SB) rrow[v ^ swz] = make_float4(dBt[2 * v].x, dBt[2 * v].y, dBt[2 * v + 1].x, dBt[2 * v + 1].y);
+        if constexpr (!SC)
+          rrow[(V / 2 + v) ^ swz] = make_float4(dCt[2 * v].x, dCt[2 * v].y, dCt[2 * v + 1].x, dCt[2 * v + 1].y);
       }
     }
     if constexpr (OWN) {
@@ -343,8 +355,8 @@ __device__ __forceinline__ void sub_block(const Lane<S, CPT>& ln, ChainRegs<S, C
     float y0[CPT], lb0[CPT], wa0[CPT], wa1[CPT], mb0[ZOH ? CPT : 1];
     {
       float2 Bv[H], Cv[H];
-      ln.load_states_f(tfB + r0e * 16, Bv);
-      ln.load_states_f(tfC + r0e * 16, Cv);
+      if constexpr (!SB) ln.load_states_f(tfB + r0e * 16, Bv);
+      if constexpr (!SC) ln.load_states_f(tfC + r0e * 16, Cv);
       float2 dBt[H], dCt[H];
 #pragma unroll
       for (int q = 0; q < CPT; ++q) {
@@ -363,27 +375,27 @@ __device__ __forceinline__ void sub_block(const Lane<S, CPT>& ln, ChainRegs<S, C
           }
           float2 E = make_float2(0.f, 0.f);
           if constexpr (ZOH) E = gain(q, k, a[k], dt0[q]);
-          const float2 he = f2fma(a[k], hpp, f2mul(ZOH ? f2mul(E, du2) : du2, Bv[k]));      // h after the even step
+          const float2 Bk = Bof(Bv, q, k), Ck = Cof(Cv, q, k);
+          const float2 he = f2fma(a[k], hpp, f2mul(ZOH ? f2mul(E, du2) : du2, Bk));      // h after the even step
           const float2 w1 = f2mul(cr.mu[q][k], he);                   // the odd step's w = mu_{t1} h_{t1 - 1}
           w1a = f2fma(w1, cr.A2[q][k], w1a);
           cr.dA[q][k] = f2fma(w1, dt12, cr.dA[q][k]);
-          const float2 lam = f2fma(Cv[k], ds2, cr.mu[q][k]);
+          const float2 lam = f2fma(Ck, ds2, cr.mu[q][k]);
           float2 lw = lam;
           if constexpr (ZOH) {
             lw = f2mul(lam, E);
-            cr.dA[q][k] = f2fma(f2mul(lam, gain_dA(q, k, a[k], E, dt0[q])), f2mul(Bv[k], f2dup(u0[q])), cr.dA[q][k]);
+            cr.dA[q][k] = f2fma(f2mul(lam, gain_dA(q, k, a[k], E, dt0[q])), f2mul(Bk, f2dup(u0[q])), cr.dA[q][k]);
           }
-          if (q == 0) {
-            dCt[k] = f2mul(ds2, he);
-            dBt[k] = f2mul(lw, du2);
-          } else {
-            dCt[k] = f2fma(ds2, he, dCt[k]);
-            dBt[k] = f2fma(lw, du2, dBt[k]);
-          }
-          lb = f2fma(lw, Bv[k], lb);
-          yv = f2fma(Cv[k], he, yv);
+          if constexpr (SC) cr.dCs[SC ? q : 0][SC ? k : 0] = f2fma(ds2, he, cr.dCs[SC ? q : 0][SC ? k : 0]);
+          else if (q == 0) dCt[k] = f2mul(ds2, he);
+          else dCt[k] = f2fma(ds2, he, dCt[k]);
+          if constexpr (SB) cr.dBs[SB ? q : 0][SB ? k : 0] = f2fma(lw, du2, cr.dBs[SB ? q : 0][SB ? k : 0]);
+          else if (q == 0) dBt[k] = f2mul(lw, du2);
+          else dBt[k] = f2fma(lw, du2, dBt[k]);
+          lb = f2fma(lw, Bk, lb);
+          yv = f2fma(Ck, he, yv);
           cr.mu[q][k] = f2mul(a[k], lam);
-          if constexpr (ZOH) mb = f2fma(cr.mu[q][k], Bv[k], mb);
+          if constexpr (ZOH) mb = f2fma(cr.mu[q][k], Bk, mb);
           const float2 w0 = f2mul(cr.mu[q][k], hpp);
           w0a = f2fma(w0, cr.A2[q][k], w0a);
           cr.dA[q][k] = f2fma(w0, dt02, cr.dA[q][k]);
@@ -398,8 +410,9 @@ __device__ __forceinline__ void sub_block(const Lane<S, CPT>& ln, ChainRegs<S, C
       const int swz = (lane / (8 / V)) & (V - 1);
 #pragma unroll
       for (int v = 0; v < V / 2; ++v) {
-        rrow[v ^ swz] = make_float4(dBt[2 * v].x, dBt[2 * v].y, dBt[2 * v + 1].x, dBt[2 * v + 1].y);
-        rrow[(V / 2 + v) ^ swz] = make_float4(dCt[2 * v].x, dCt[2 * v].y, dCt[2 * v + 1].x, dCt[2 * v + 1].y);
+        if constexpr (!SB) rrow[v ^ swz] = make_float4(dBt[2 * v].x, dBt[2 * v].y, dBt[2 * v + 1].x, dBt[2 * v + 1].y);
+        if constexpr (!SC)
+          rrow[(V / 2 + v) ^ swz] = make_float4(dCt[2 * v].x, dCt[2 * v].y, dCt[2 * v + 1].x, dCt[2 * v + 1].y);
       }
     }
     if constexpr (OWN) {
@@ -465,24 +478,27 @@ __device__ __forceinline__ void sub_block(const Lane<S, CPT>& ln, ChainRegs<S, C
       reinterpret_cast<__nv_bfloat16*>(toz + rm * WPR)[ln.co] = __float2bfloat16_rn(dzm * gate_on);
     }
 
-    if ((2 * m) % kRB == 0) {
+    if (BC != 3 && (2 * m) % kRB == 0) {
       // dB / dC of steps 2m .. 2m + 3: every lane sums one float4 of one step over the lane groups, ascending
+      // (a half that is a parameter has nothing in the buffer: its lanes idle)
       __syncwarp();
       const int s = lane >> 3, o = lane & 7;
       const int which = o >> 2, n0 = 4 * (o & 3);
-      const int jo = n0 / S, v = which * (S / 4) + (n0 % S) / 4;
-      const float4* rs_ = tred + s * 32 * V;
-      float4 acc;
+      if (!(which ? SC : SB)) {
+        const int jo = n0 / S, v = which * (S / 4) + (n0 % S) / 4;
+        const float4* rs_ = tred + s * 32 * V;
+        float4 acc;
 #pragma unroll
-      for (int gg = 0; gg < 32 / LPC; ++gg) {
-        const int l = gg * LPC + jo;
-        const float4 t4 = rs_[l * V + (v ^ ((l / (8 / V)) & (V - 1)))];
-        if (gg == 0) acc = t4;
-        else { acc.x += t4.x; acc.y += t4.y; acc.z += t4.z; acc.w += t4.w; }
+        for (int gg = 0; gg < 32 / LPC; ++gg) {
+          const int l = gg * LPC + jo;
+          const float4 t4 = rs_[l * V + (v ^ ((l / (8 / V)) & (V - 1)))];
+          if (gg == 0) acc = t4;
+          else { acc.x += t4.x; acc.y += t4.y; acc.z += t4.z; acc.w += t4.w; }
+        }
+        const int row = r0 + 2 * m + s;
+        if (row < nlive && SSM_IN_RANGE(row < kBT && n0 + 4 <= 16, abort_word))
+          *reinterpret_cast<float4*>((which ? part_dC : part_dB) + (size_t)row * 16 + n0) = acc;
       }
-      const int row = r0 + 2 * m + s;
-      if (row < nlive && SSM_IN_RANGE(row < kBT && n0 + 4 <= 16, abort_word))
-        *reinterpret_cast<float4*>((which ? part_dC : part_dB) + (size_t)row * 16 + n0) = acc;
       __syncwarp();
     }
   }
@@ -490,9 +506,11 @@ __device__ __forceinline__ void sub_block(const Lane<S, CPT>& ln, ChainRegs<S, C
 
 }  // namespace
 
-template <int S, int CPT, bool SP, bool ZOH>
+template <int S, int CPT, bool SP, bool ZOH, int BC>
 __global__ void __launch_bounds__(kBwdWarps * 32, (CPT == 16 / S) ? 2 : 3)
     ssm_bwd_warp_kernel(const BwdParams p, const WarpSched sc) {
+  constexpr bool SB = BC & 1, SC = BC & 2;
+  constexpr int HV = bwd_handoff_vec(BC);
   using LN = Lane<S, CPT>;
   constexpr int H = S / 2, CW = LN::CW, WPR = CW / 2, NV = CPT * S / 4;   // NV: float4 of a thread's states
   constexpr bool OWN = LN::OWN;
@@ -562,8 +580,8 @@ __global__ void __launch_bounds__(kBwdWarps * 32, (CPT == 16 / S) ? 2 : 3)
           const int tt = lane >> 1, hc = lane & 1;
           const bool ok = t0 + tt < t_seg_end;
           const size_t go = ok ? (row0 + tt) * 16 + hc * 8 : 0;
-          cp_async16(&sm.rB[st][tt][hc * 4], gB + go, ok);
-          cp_async16(&sm.rC[st][tt][hc * 4], gC + go, ok);
+          if constexpr (!SB) cp_async16(&sm.rB[st][tt][hc * 4], gB + go, ok);
+          if constexpr (!SC) cp_async16(&sm.rC[st][tt][hc * 4], gC + go, ok);
         }
 #pragma unroll
         for (int sb = 0; sb < kBT / kSB; ++sb) {
@@ -582,7 +600,7 @@ __global__ void __launch_bounds__(kBwdWarps * 32, (CPT == 16 / S) ? 2 : 3)
     issue_tile(tile_hi, 0);
 
     // ---- per-thread constants and carried values
-    ChainRegs<S, CPT, ZOH> cr;
+    ChainRegs<S, CPT, ZOH, BC> cr;
     bool ap = !p.general_A;
     cr.minA = 3.0e38f;
 #pragma unroll
@@ -612,6 +630,26 @@ __global__ void __launch_bounds__(kBwdWarps * 32, (CPT == 16 / S) ? 2 : 3)
       }
       cr.a0s[q] = cr.A2[q][0].x;
       cr.rs[q] = cr.A2[q][0].y - cr.A2[q][0].x;
+      if constexpr (SB || SC) {
+#pragma unroll
+        for (int k = 0; k < S / 4; ++k) {
+          const size_t at = (size_t)chan(q) * 16 + S * j + 4 * k;
+          if constexpr (SB) {
+            float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (valid) v = *reinterpret_cast<const float4*>(static_cast<const float*>(p.B) + at);
+            cr.Bst[q][2 * k] = make_float2(v.x, v.y);
+            cr.Bst[q][2 * k + 1] = make_float2(v.z, v.w);
+            cr.dBs[q][2 * k] = cr.dBs[q][2 * k + 1] = make_float2(0.f, 0.f);
+          }
+          if constexpr (SC) {
+            float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (valid) v = *reinterpret_cast<const float4*>(static_cast<const float*>(p.C) + at);
+            cr.Cst[q][2 * k] = make_float2(v.x, v.y);
+            cr.Cst[q][2 * k + 1] = make_float2(v.z, v.w);
+            cr.dCs[q][2 * k] = cr.dCs[q][2 * k + 1] = make_float2(0.f, 0.f);
+          }
+        }
+      }
     }
     ap = __all_sync(0xffffffffu, ap);
     const int c_own = d_w + ln.co;
@@ -624,11 +662,29 @@ __global__ void __launch_bounds__(kBwdWarps * 32, (CPT == 16 / S) ? 2 : 3)
         cp_async_wait_all();
         return;
       }
-      const float4* hb = sc.handoff + ((size_t)worker * 32 + lane) * kBwdHandoffVec;
+      const float4* hb = sc.handoff + ((size_t)worker * 32 + lane) * HV;
       float4 v[2 * NV];
 #pragma unroll
       for (int k = 0; k < 2 * NV; ++k) v[k] = __ldcg(hb + k);
       const float4 dv = __ldcg(hb + 2 * NV);
+      if constexpr (SB || SC) {
+        // the gradient sums of the parameters B / C ride along like dA
+#pragma unroll
+        for (int q = 0; q < CPT; ++q)
+#pragma unroll
+          for (int k = 0; k < S / 4; ++k) {
+            if constexpr (SB) {
+              const float4 w = __ldcg(hb + 2 * NV + 1 + q * (S / 4) + k);
+              cr.dBs[q][2 * k] = make_float2(w.x, w.y);
+              cr.dBs[q][2 * k + 1] = make_float2(w.z, w.w);
+            }
+            if constexpr (SC) {
+              const float4 w = __ldcg(hb + 2 * NV + 1 + (SB ? NV : 0) + q * (S / 4) + k);
+              cr.dCs[q][2 * k] = make_float2(w.x, w.y);
+              cr.dCs[q][2 * k + 1] = make_float2(w.z, w.w);
+            }
+          }
+      }
       const float* f = reinterpret_cast<const float*>(v);
 #pragma unroll
       for (int q = 0; q < CPT; ++q)
@@ -666,10 +722,14 @@ __global__ void __launch_bounds__(kBwdWarps * 32, (CPT == 16 / S) ? 2 : 3)
         for (int k = 0; k < (kBT * 4 + 31) / 32; ++k) {
           const int c = lane + 32 * k, rr = c >> 2, qq = c & 3;
           if (kBT * 4 % 32 == 0 || rr < kBT) {
-            const uint2 wb = *reinterpret_cast<const uint2*>(&sm.rB[st][rr][2 * qq]);
-            const uint2 wc = *reinterpret_cast<const uint2*>(&sm.rC[st][rr][2 * qq]);
-            *reinterpret_cast<float4*>(&sm.fB[rr][4 * qq]) = make_float4(bf16lo(wb.x), bf16hi(wb.x), bf16lo(wb.y), bf16hi(wb.y));
-            *reinterpret_cast<float4*>(&sm.fC[rr][4 * qq]) = make_float4(bf16lo(wc.x), bf16hi(wc.x), bf16lo(wc.y), bf16hi(wc.y));
+            if constexpr (!SB) {
+              const uint2 wb = *reinterpret_cast<const uint2*>(&sm.rB[st][rr][2 * qq]);
+              *reinterpret_cast<float4*>(&sm.fB[rr][4 * qq]) = make_float4(bf16lo(wb.x), bf16hi(wb.x), bf16lo(wb.y), bf16hi(wb.y));
+            }
+            if constexpr (!SC) {
+              const uint2 wc = *reinterpret_cast<const uint2*>(&sm.rC[st][rr][2 * qq]);
+              *reinterpret_cast<float4*>(&sm.fC[rr][4 * qq]) = make_float4(bf16lo(wc.x), bf16hi(wc.x), bf16lo(wc.y), bf16hi(wc.y));
+            }
           }
         }
         // per-element gate terms of the tile: ds = dout silu(z), gp = dout silu'(z); element e = lane + 32 i
@@ -724,7 +784,7 @@ __global__ void __launch_bounds__(kBwdWarps * 32, (CPT == 16 / S) ? 2 : 3)
           zs = __any_sync(0xffffffffu, dmin * cr.minA < kZohSmall);
         }
 #define SSM_SUB_BLOCK(AP_, ZS_)                                                                                     \
-  sub_block<S, CPT, SP, AP_, ZOH, ZS_>(ln, cr, sb * kSB, nlive, has_z ? 1.f : 0.f, p.softplus != 0, &sm.x[st][0][0], \
+  sub_block<S, CPT, SP, AP_, ZOH, ZS_, BC>(ln, cr, sb * kSB, nlive, has_z ? 1.f : 0.f, p.softplus != 0, &sm.x[st][0][0], \
                                        &sm.d[st][0][0], &sm.fB[0][0], &sm.fC[0][0], &sm.ds[0][0], &sm.gp[0][0],      \
                                        &sm.dF[0][0], &sm.ck[st][sb][0][0], &sm.ox[0][0], &sm.od[0][0], &sm.oz[0][0], \
                                        &sm.red[0][0][0], part_dB, part_dC, sc.abort)
@@ -762,7 +822,20 @@ __global__ void __launch_bounds__(kBwdWarps * 32, (CPT == 16 / S) ? 2 : 3)
 
     if (gives_out) {
       // the earlier part of this chain (in time) belongs to the next worker
-      float4* hb = sc.handoff + ((size_t)(worker + 1) * 32 + lane) * kBwdHandoffVec;
+      float4* hb = sc.handoff + ((size_t)(worker + 1) * 32 + lane) * HV;
+      if constexpr (SB || SC) {
+#pragma unroll
+        for (int q = 0; q < CPT; ++q)
+#pragma unroll
+          for (int k = 0; k < S / 4; ++k) {
+            if constexpr (SB)
+              __stcg(hb + 2 * NV + 1 + q * (S / 4) + k, make_float4(cr.dBs[q][2 * k].x, cr.dBs[q][2 * k].y,
+                                                                    cr.dBs[q][2 * k + 1].x, cr.dBs[q][2 * k + 1].y));
+            if constexpr (SC)
+              __stcg(hb + 2 * NV + 1 + (SB ? NV : 0) + q * (S / 4) + k,
+                     make_float4(cr.dCs[q][2 * k].x, cr.dCs[q][2 * k].y, cr.dCs[q][2 * k + 1].x, cr.dCs[q][2 * k + 1].y));
+          }
+      }
       float f[8 * NV];
 #pragma unroll
       for (int q = 0; q < CPT; ++q)
@@ -792,6 +865,12 @@ __global__ void __launch_bounds__(kBwdWarps * 32, (CPT == 16 / S) ? 2 : 3)
           for (int k = 0; k < S / 4; ++k) {
             *reinterpret_cast<float4*>(p.dA_part + (part * D + chan(q)) * 16 + S * j + 4 * k) =
                 make_float4(cr.dA[q][2 * k].x, cr.dA[q][2 * k].y, cr.dA[q][2 * k + 1].x, cr.dA[q][2 * k + 1].y);
+            if constexpr (SB)
+              *reinterpret_cast<float4*>(p.dBs_part + (part * D + chan(q)) * 16 + S * j + 4 * k) =
+                  make_float4(cr.dBs[q][2 * k].x, cr.dBs[q][2 * k].y, cr.dBs[q][2 * k + 1].x, cr.dBs[q][2 * k + 1].y);
+            if constexpr (SC)
+              *reinterpret_cast<float4*>(p.dCs_part + (part * D + chan(q)) * 16 + S * j + 4 * k) =
+                  make_float4(cr.dCs[q][2 * k].x, cr.dCs[q][2 * k].y, cr.dCs[q][2 * k + 1].x, cr.dCs[q][2 * k + 1].y);
             if (seg == 0 && p.dh0 != nullptr)   // the adjoint that leaves the first step is the gradient of the initial state
               *reinterpret_cast<float4*>(p.dh0 + ((size_t)b * D + chan(q)) * 16 + S * j + 4 * k) =
                   make_float4(cr.mu[q][2 * k].x, cr.mu[q][2 * k].y, cr.mu[q][2 * k + 1].x, cr.mu[q][2 * k + 1].y);
@@ -807,11 +886,11 @@ __global__ void __launch_bounds__(kBwdWarps * 32, (CPT == 16 / S) ? 2 : 3)
 
 namespace {
 
-template <int S, int CPT, bool SP, bool ZOH>
+template <int S, int CPT, bool SP, bool ZOH, int BC = 0>
 cudaError_t launch_bwd_variant(const Plan& plan, const BwdParams& p, cudaStream_t s) {
   constexpr int CW = Lane<S, CPT>::CW;
   const size_t smem = sizeof(BwdWarpSmem<S, CPT, SP>) * kBwdWarps;
-  auto kern = ssm_bwd_warp_kernel<S, CPT, SP, ZOH>;
+  auto kern = ssm_bwd_warp_kernel<S, CPT, SP, ZOH, BC>;
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
   int dev = 0, sms = 0, per_sm = 0;
@@ -844,19 +923,28 @@ cudaError_t launch_bwd_variant(const Plan& plan, const BwdParams& p, cudaStream_
 
 bool bwd_fast_applicable(const ssm_problem_t& prob, const BwdParams& p) {
   auto al16 = [](const void* q) { return q == nullptr || (reinterpret_cast<uintptr_t>(q) & 15) == 0; };
-  if (p.static_B || p.static_C) return false;  // input-dependent B, C only
+  if ((p.static_B || p.static_C) && p.zoh) return false;  // non-selective B / C: default B-bar rule only
+  if ((p.static_B && !al16(p.dBs_part)) || (p.static_C && !al16(p.dCs_part))) return false;
   return prob.io_dtype == SSM_BF16 && prob.N == 16 && prob.D % 8 == 0 && p.seg_steps % kBT == 0 && al16(p.x) &&
          al16(p.delta) && al16(p.z) && al16(p.B) && al16(p.C) && al16(p.dout) && al16(p.dx) && al16(p.ddelta) &&
          al16(p.dz) && al16(p.A) && al16(p.ckpt) && al16(p.mu_in) && al16(p.dh0) && al16(p.dBC_part) && al16(p.dA_part) &&
          al16(p.handoff) && (p.groups == (p.D + 31) / 32 || p.groups == (p.D + 15) / 16);
 }
 
-size_t bwd_handoff_bytes_per_worker() { return sizeof(float4) * kBwdHandoffVec * 32; }
+size_t bwd_handoff_bytes_per_worker(bool static_B, bool static_C) {
+  return sizeof(float4) * bwd_handoff_vec((static_B ? 1 : 0) | (static_C ? 2 : 0)) * 32;
+}
 // channels per warp of the tuned kernel = the channel-group size of the dB / dC partial sums
 int bwd_fast_channels_per_warp() { return kBwdFastChannels; }
 
 cudaError_t launch_bwd_fast(const Plan& plan, const BwdParams& p, cudaStream_t s) {
   const bool sp = p.softplus || p.delta_bias != nullptr;
+  if (p.static_B || p.static_C) {   // (never with ZOH: bwd_fast_applicable)
+    const int bc = (p.static_B ? 1 : 0) | (p.static_C ? 2 : 0);
+    if (bc == 3) return sp ? launch_bwd_variant<8, 2, true, false, 3>(plan, p, s) : launch_bwd_variant<8, 2, false, false, 3>(plan, p, s);
+    if (bc == 1) return sp ? launch_bwd_variant<8, 2, true, false, 1>(plan, p, s) : launch_bwd_variant<8, 2, false, false, 1>(plan, p, s);
+    return sp ? launch_bwd_variant<8, 2, true, false, 2>(plan, p, s) : launch_bwd_variant<8, 2, false, false, 2>(plan, p, s);
+  }
   if (p.zoh) return sp ? launch_bwd_variant<8, 2, true, true>(plan, p, s) : launch_bwd_variant<8, 2, false, true>(plan, p, s);
   return sp ? launch_bwd_variant<8, 2, true, false>(plan, p, s) : launch_bwd_variant<8, 2, false, false>(plan, p, s);
 }

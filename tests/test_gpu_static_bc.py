@@ -83,3 +83,58 @@ def test_static_b_and_c(batch, L, D, N, io, sB, sC, zoh):
                                dev["D_skip"], dev["z"][:, t].contiguous(), h, zoh=zoh, static_B=sB, static_C=sC))
     got = np.stack([U.to_host(o) for o in outs], axis=1)
     assert U.rel_err(got, ref["out"][:, :3]) <= tol["out"] * max(1.0, np.abs(ref["out"]).max() / np.abs(ref["out"][:, :3]).max())
+
+
+@pytest.mark.parametrize("fused_dt", [False, True])
+def test_static_tuned_kernels_with_shared_chains(fused_dt):
+    """The 2.8B layer width on a short sequence: 640 chains for 592 resident warps, so neighbouring warps share chains and
+    the gradient sums of the parameters B / C cross the hand-off.  Checked on sampled channels (the oracle is driven one
+    channel at a time)."""
+    import torch
+    from oracle import ssm_oracle as O
+    from paper_2312_00752_b200 import binding as K
+    batch, L, D, N, io = 4, 64, 5120, 16, "bf16"
+    cfg = synth.ScanConfig("static_bc_wide", 18, batch, L, D, N, io, 1e-3, 1e-1)
+    inp = synth.make_inputs(cfg, seed=0)
+    rng = np.random.default_rng(11)
+    Bs = rng.standard_normal((D, N)).astype(np.float32)
+    Cs = rng.standard_normal((D, N)).astype(np.float32)
+    bias = (0.1 * rng.standard_normal(D)).astype(np.float32)
+    dev = U.to_device(inp, io)
+    B, C = torch.from_numpy(Bs).cuda(), torch.from_numpy(Cs).cuda()
+    if fused_dt:
+        # `delta` is taken as the pre-activation: step size = softplus(delta + bias)
+        tb = torch.from_numpy(bias).cuda()
+        out, saved = K.ssm_scan_fwd_fused_dt(dev["x"], dev["delta"], tb, dev["A"], B, C, dev["D_skip"], dev["z"],
+                                             save_states=True, static_B=True, static_C=True)
+        g = K.ssm_scan_bwd_fused_dt(dev["x"], dev["delta"], tb, dev["A"], B, C, dev["D_skip"], dev["z"], dev["dout"],
+                                    saved, static_B=True, static_C=True)
+    else:
+        args = (dev["x"], dev["delta"], dev["A"], B, C, dev["D_skip"], dev["z"])
+        out, saved = K.ssm_scan_fwd(*args, save_states=True, static_B=True, static_C=True)
+        g = K.ssm_scan_bwd(*args, dev["dout"], saved, static_B=True, static_C=True)
+    got = {k: U.to_host(v) for k, v in g.items() if v is not None}
+    got["out"] = U.to_host(out)
+    chans = sorted(set([0, 1, 31, 32, 33, 2559, 2560, 5119] + [int(c) for c in rng.integers(0, D, 16)]))
+    tol = U.TOL[io]
+    ref_scale = {}
+    errs = {}
+    for d in chans:
+        sl = lambda a: a[:, :, d:d + 1]
+        Bd, Cd = np.broadcast_to(Bs[d], (batch, L, N)), np.broadcast_to(Cs[d], (batch, L, N))
+        kw = dict(delta_softplus=True, delta_bias=bias[d:d + 1]) if fused_dt else {}
+        o = O.scan_fwd(sl(inp["x"]), sl(inp["delta"]), inp["A"][d:d + 1], Bd, Cd, D_skip=inp["D_skip"][d:d + 1],
+                       z=sl(inp["z"]), **kw)
+        r = O.scan_bwd(sl(inp["x"]), sl(inp["delta"]), inp["A"][d:d + 1], Bd, Cd, inp["D_skip"][d:d + 1], sl(inp["z"]),
+                       sl(inp["dout"]), **kw)
+        pairs = {"out": (got["out"][:, :, d], o[:, :, 0]), "dx": (got["dx"][:, :, d], r["dx"][:, :, 0]),
+                 "ddelta": (got["ddelta"][:, :, d], r["ddelta"][:, :, 0]), "dz": (got["dz"][:, :, d], r["dz"][:, :, 0]),
+                 "dB": (got["dB"][d], r["dB"].sum(axis=(0, 1))), "dC": (got["dC"][d], r["dC"].sum(axis=(0, 1))),
+                 "dA": (got["dA"][d], r["dA"][0]), "dD": (got["dD"][d:d + 1], r["dD"])}
+        if fused_dt:
+            pairs["ddelta_bias"] = (got["ddelta_bias"][d:d + 1], r["ddelta_bias"])
+        for k, (a, b) in pairs.items():
+            ref_scale[k] = max(ref_scale.get(k, 0.0), float(np.abs(b).max()))
+            errs[k] = max(errs.get(k, 0.0), float(np.abs(a - b).max()))
+    for k in errs:
+        assert errs[k] <= (tol["out"] if k == "out" else tol["grad"]) * ref_scale[k], (k, errs[k], ref_scale[k])
