@@ -444,8 +444,8 @@ def run_ours(args, cfg):
         "bwd": {"ms": b_ms, "elements_per_s": cfg.elements / (b_ms * 1e-3), "algorithmic_bytes": bwd_bytes,
                 "achieved_gbs": bwd_gbs, "frac_of_hbm_peak": bwd_gbs / peak, **alu_fracs("bwd", b_ms)},
         "roofline": {"bound": "hbm", "binding_bound": "alu (FP32 lanes; see roofline_alu)",
-                     "kernel": "ssm_scan_bwd call (ssm_bwd_warp_kernel, the dominant kernel, with its adjoint pre-pass, "
-                               "carry and reduction kernels)",
+                     "kernel": "ssm_scan_bwd call (ssm_bwd_warp_kernel, the dominant kernel, timed together with the "
+                               "adjoint pre-pass and reduction kernels of the same call)",
                      "achieved": bwd_gbs, "peak": peak, "peak_kind": f"{peak_kind} copy bandwidth",
                      "unit": "GB/s", "frac": bwd_gbs / peak,
                      "traffic": NCU_TRAFFIC_BYTES.get(cfg.cfg_id) if not args.general_A else None,
