@@ -43,7 +43,7 @@ static_assert(kWT % kSub == 0, "tiles are whole sub-blocks");
 
 // NST ring stages: 3 (two tiles in flight) or 2 (one tile in flight; small enough for two blocks per SM in FULL mode)
 // BC: bit 0 = B is a per-channel parameter (no B tile), bit 1 = the same for C (Algorithm 1's non-selective B / C)
-template <int CW, bool FULL, bool SP, int BC, int NST>
+template <int CW, bool FULL, bool SPF, int BC, int NST>
 struct FwdWarpSmem {
   static constexpr bool TB = !(BC & 1), TC = FULL && !(BC & 2);   // tiles of B / C are staged
   uint32_t x[NST][kWT][CW / 2];   // bf16 pairs, CW channels
@@ -55,7 +55,7 @@ struct FwdWarpSmem {
   uint32_t rC[TC ? NST : 1][TC ? kWT : 1][12];
   float fB[TB ? kWT : 1][20];      // B and C of the current tile widened to float
   float fC[TC ? kWT : 1][20];
-  float dF[SP ? kWT : 1][CW];      // SP: step sizes after bias and softplus
+  float dF[SPF ? kWT : 1][CW];     // SPF: step sizes after bias and softplus, prepared per tile
   uint32_t o[FULL ? kWT : 1][CW / 2];  // output tile (bf16 pairs)
 };
 
@@ -77,7 +77,10 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32) ssm_fwd_warp_kernel(const
   constexpr int CH = CW / 8;        // 16-byte chunks per tile row of x, delta, z, out
   constexpr int RP = 32 / CH;       // tile rows a warp covers with one chunk per lane
   constexpr int HV = S / 4 + 1;     // float4 per lane of a hand-off: S states, sum of delta
-  using Smem = FwdWarpSmem<CW, FULL, SP, BC, NST>;
+  // fused step size: evaluated inside the step batches (each lane for its own channel), except with the ZOH rule, whose
+  // choice of variant needs the step sizes of a sub-block before it starts: then they are prepared per tile
+  constexpr bool SPF = SP && ZOH;
+  using Smem = FwdWarpSmem<CW, FULL, SPF, BC, NST>;
   constexpr bool TB = Smem::TB, TC = Smem::TC;   // B / C are inputs [batch][L][16] staged in tiles (else parameters)
   extern __shared__ __align__(16) unsigned char smem_raw[];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -213,7 +216,9 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32) ssm_fwd_warp_kernel(const
     const float Dk = (FULL && p.Dskip != nullptr && valid) ? p.Dskip[c_own] : 0.f;
     // the softplus pass walks the tile with one (row, channel) element per lane: channel lane % CW
     const int c_prep = d_w + (lane % CW);
-    const float bias_prep = (SP && p.delta_bias != nullptr && c_prep < D) ? p.delta_bias[c_prep] : 0.f;
+    const float bias_prep = (SPF && p.delta_bias != nullptr && c_prep < D) ? p.delta_bias[c_prep] : 0.f;
+    const float bias_own = (SP && !SPF && p.delta_bias != nullptr && valid) ? p.delta_bias[c_own] : 0.f;
+    int rows_live = 0;   // rows of the current tile inside the piece (the rest are identity steps)
     float dsum = 0.f;
 
     if (from > 0) {
@@ -264,8 +269,16 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32) ssm_fwd_warp_kernel(const
 #pragma unroll
         for (int t = 0; t < GB; ++t) {
           const int r = SSM_TILE_ROW(r0 + gb * GB + t, kWT, sc.abort);
-          if constexpr (SP) dt[t] = sm.dF[r][g];
-          else dt[t] = bf16at(sm.d[st][r], g);
+          if constexpr (SPF) {
+            dt[t] = sm.dF[r][g];
+          } else if constexpr (SP) {
+            // pre-activation + bias, through the softplus if asked; rows past the end stay identity steps (delta = 0)
+            float v = bf16at(sm.d[st][r], g) + bias_own;
+            if (p.softplus) v = softplus_fast(v);
+            dt[t] = (r0 + gb * GB + t < rows_live) ? v : 0.f;
+          } else {
+            dt[t] = bf16at(sm.d[st][r], g);
+          }
           u[t] = bf16at(sm.x[st][r], g);
           du[t] = dt[t] * u[t];
           if constexpr (AP) {
@@ -404,8 +417,9 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32) ssm_fwd_warp_kernel(const
                 make_float4(bf16lo(wc[2 * k]), bf16hi(wc[2 * k]), bf16lo(wc[2 * k + 1]), bf16hi(wc[2 * k + 1]));
         }
       }
-      if constexpr ((TB || TC) && !SP) __syncwarp();
-      if constexpr (SP) {
+      rows_live = t_to - t0;
+      if constexpr ((TB || TC) && !SPF) __syncwarp();
+      if constexpr (SPF) {
         // step sizes of the tile, once per element: pre-activation + bias, softplus; rows past the end stay identity
         // steps (delta = 0)
 #pragma unroll 4
@@ -431,7 +445,7 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32) ssm_fwd_warp_kernel(const
           // smallest step size of the live rows of the sub-block for this lane's channel
           float dmin = 3.0e38f;
           for (int t = 0; t < kSub && ts + t < t_to; ++t)
-            dmin = fminf(dmin, fabsf(SP ? sm.dF[SP ? sb * kSub + t : 0][g] : bf16at(sm.d[st][sb * kSub + t], g)));
+            dmin = fminf(dmin, fabsf(SPF ? sm.dF[SPF ? sb * kSub + t : 0][g] : bf16at(sm.d[st][sb * kSub + t], g)));
           if (__any_sync(0xffffffffu, dmin * minA < kZohSmall)) {
             if (ap) compute_sub(st, sb * kSub, std::true_type{}, std::true_type{});
             else compute_sub(st, sb * kSub, std::false_type{}, std::true_type{});
@@ -496,7 +510,7 @@ namespace {
 template <int S, int MODE, bool SP, bool ZOH, int BC, int NST>
 cudaError_t fwd_occupancy(int* per_sm, size_t* smem_bytes) {
   constexpr int CW = 2 * S;   // channels per chain
-  const size_t smem = sizeof(FwdWarpSmem<CW, MODE == kFwdFull, SP, BC, NST>) * kWarpsPerBlock;
+  const size_t smem = sizeof(FwdWarpSmem<CW, MODE == kFwdFull, SP && ZOH, BC, NST>) * kWarpsPerBlock;
   auto kern = ssm_fwd_warp_kernel<S, MODE, SP, ZOH, BC, NST>;
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
