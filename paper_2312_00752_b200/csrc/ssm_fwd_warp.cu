@@ -257,7 +257,7 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32) ssm_fwd_warp_kernel(const
     auto compute_sub = [&](int st, int r0, auto ap_tag, auto zs_tag) {
       constexpr bool AP = decltype(ap_tag)::value;
       constexpr bool ZS = decltype(zs_tag)::value;
-      constexpr int GB = AP ? 8 : (S == 16 ? 2 : 4);
+      constexpr int GB = AP ? 8 : 4;   // general A: 4 steps of exponentials in flight (2 were measured slower, 8 cost the arithmetic-progression body registers)
       constexpr int NE = GB / LPC;        // results this lane finishes per batch
       const float gate_off = has_z ? 0.f : 1.f;
 #pragma unroll
