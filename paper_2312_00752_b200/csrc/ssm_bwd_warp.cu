@@ -272,8 +272,6 @@ __device__ __forceinline__ void sub_block(const Lane<S, CPT>& ln, ChainRegs<S, C
     ln.unpack_row(tx + r1 * WPR, u1);
     ln.pick_row(tds + r1 * CW, ds1);
     const float gp1 = tgp[r1 * CW + ln.co];
-    float raw1 = 0.f;
-    if constexpr (SP) raw1 = __uint_as_float((uint32_t)reinterpret_cast<const uint16_t*>(td + r1 * WPR)[ln.co] << 16);
     float y1[CPT], lb1[CPT], mb1[ZOH ? CPT : 1];   // mb: sum mu B (ZOH: the step-size gradient through E)
     {
       float2 Bv[H], Cv[H];
@@ -350,8 +348,6 @@ __device__ __forceinline__ void sub_block(const Lane<S, CPT>& ln, ChainRegs<S, C
     ln.unpack_row(tx + r0e * WPR, u0);
     ln.pick_row(tds + r0e * CW, ds0);
     const float gp0 = tgp[r0e * CW + ln.co];
-    float raw0 = 0.f;
-    if constexpr (SP) raw0 = __uint_as_float((uint32_t)reinterpret_cast<const uint16_t*>(td + r0e * WPR)[ln.co] << 16);
     float y0[CPT], lb0[CPT], wa0[CPT], wa1[CPT], mb0[ZOH ? CPT : 1];
     {
       float2 Bv[H], Cv[H];
@@ -441,8 +437,8 @@ __device__ __forceinline__ void sub_block(const Lane<S, CPT>& ln, ChainRegs<S, C
       if constexpr (SP) {
         // the gradient goes to the pre-activation v: d softplus(v) / dv = sigmoid(v); the bias gets the sum over time
         if (softplus) {
-          dd1 *= sigmoid_fast(raw1 + cr.bias_own);
-          dd0 *= sigmoid_fast(raw0 + cr.bias_own);
+          dd1 *= sigmoid_from_softplus(dt1[0]);
+          dd0 *= sigmoid_from_softplus(dt0[0]);
         }
         if (r0 + 2 * m + 1 < nlive) cr.dbias += dd1;
         if (r0 + 2 * m < nlive) cr.dbias += dd0;
@@ -470,7 +466,7 @@ __device__ __forceinline__ void sub_block(const Lane<S, CPT>& ln, ChainRegs<S, C
       cr.dD = fmaf(dsm, um, cr.dD);
       float ddm = fmaf(um, ZOH ? (odd ? mb1[0] : mb0[0]) : lbm, wam * kInvLog2e);
       if constexpr (SP) {
-        if (softplus) ddm *= sigmoid_fast((odd ? raw1 : raw0) + cr.bias_own);
+        if (softplus) ddm *= sigmoid_from_softplus(dtm);
         if (r0 + 2 * m + (odd ? 1 : 0) < nlive) cr.dbias += ddm;
       }
       reinterpret_cast<__nv_bfloat16*>(tox + rm * WPR)[ln.co] = __float2bfloat16_rn(dxm);

@@ -313,6 +313,14 @@ __device__ __forceinline__ float softplus_fast(float v) {
   return fmaxf(v, 0.f) + (e < 0.0625f ? series : lg * 0.6931471805599453f);
 }
 
+// sigmoid(v) from dt = softplus(v): sigmoid(v) = 1 - e^-dt (the derivative of the softplus, for the backward of the fused
+// step size); a short series below dt = 1/32, where the difference would cancel
+__device__ __forceinline__ float sigmoid_from_softplus(float dt) {
+  const float closed = 1.f - ex2_approx(-dt * kLog2e);
+  const float series = dt * fmaf(dt, fmaf(dt, 0.16666667f, -0.5f), 1.f);
+  return dt < 0.03125f ? series : closed;
+}
+
 // softplus(v) = log(1 + e^v) = max(v, 0) + log1p(e^-|v|) with the precise library log1p (generic kernels)
 __device__ __forceinline__ float softplus_precise(float v) { return fmaxf(v, 0.f) + log1pf(__expf(-fabsf(v))); }
 
