@@ -190,7 +190,7 @@ struct ChainRegs {
   float a0s[CPT], rs[CPT];
   float2 mu[CPT][H];    // adjoint flowing backwards in time
   float2 dA[CPT][H];
-  float Dk, bias_own, dD, dbias;
+  float Dk, dD, dbias;
 };
 
 // One sub-block of 8 steps: rows [r0, r0 + 8) of the tile; nlive = rows of the tile inside the segment.
@@ -650,7 +650,6 @@ __global__ void __launch_bounds__(kBwdWarps * 32, (CPT == 16 / S) ? 2 : 3)
     ap = __all_sync(0xffffffffu, ap);
     const int c_own = d_w + ln.co;
     cr.Dk = (p.Dskip != nullptr && c_own < D) ? p.Dskip[c_own] : 0.f;
-    cr.bias_own = (SP && p.delta_bias != nullptr && c_own < D) ? p.delta_bias[c_own] : 0.f;
     cr.dD = 0.f;
     cr.dbias = 0.f;
     if (from > 0) {
