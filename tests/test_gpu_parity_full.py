@@ -110,3 +110,35 @@ def test_long_sequence_full_size():
     assert np.abs(lhs_C - rhs_C).max() <= 3e-2 * np.abs(rhs_C).max()
     del dev
     torch.cuda.empty_cache()
+
+
+@pytest.mark.parametrize("general_A", [False, True])
+def test_wide_ragged_shape_on_sampled_channels(general_A):
+    """Batch 8, 70 steps (two tiles and a ragged one), 5000 channels (156 full groups of 32 and one of 8): 1256 chains,
+    so the forward takes the two-stage ring with two warps per sub-partition and neighbouring warps share chains in
+    both directions.  The oracle runs on sampled channels, the partial group included (dB / dC are sums over all
+    channels and are checked by the other tests of this file)."""
+    from oracle import ssm_oracle as O
+    from paper_2312_00752_b200 import binding as K
+    cfg = synth.ScanConfig("wide_ragged", 19, 8, 70, 5000, 16, "bf16", 1e-3, 1e-1)
+    inp = synth.make_inputs(cfg, seed=0)
+    if general_A:
+        rng = np.random.default_rng(5)
+        inp["A"] = (inp["A"] * (1 + 0.05 * rng.standard_normal(inp["A"].shape))).astype(np.float32)
+    dev = U.to_device(inp, "bf16")
+    got = U.gpu_fwd_bwd(dev, general_A=general_A)
+    rng = np.random.default_rng(9)
+    ch = np.array(sorted(set([0, 31, 32, 4991, 4992, 4995, 4999] + [int(c) for c in rng.integers(0, 5000, 40)])))
+    sub = lambda k: np.ascontiguousarray(inp[k][:, :, ch])
+    ref_out = O.scan_fwd(sub("x"), sub("delta"), inp["A"][ch], inp["B"], inp["C"], D_skip=inp["D_skip"][ch], z=sub("z"))
+    ref = O.scan_bwd(sub("x"), sub("delta"), inp["A"][ch], inp["B"], inp["C"], inp["D_skip"][ch], sub("z"), sub("dout"))
+    tol = U.TOL["bf16"]
+    assert U.rel_err(got["out"][:, :, ch], ref_out) <= tol["out"]
+    for k in ("dx", "ddelta", "dz"):
+        assert U.rel_err(got[k][:, :, ch], ref[k]) <= tol["grad"], k
+    for k in ("dA", "dD"):
+        assert U.rel_err(got[k][ch], ref[k]) <= tol["grad"], k
+    # run-to-run bit equality with shared chains
+    again = U.gpu_fwd_bwd(dev, general_A=general_A)
+    for k in ("out", "dx", "ddelta", "dz", "dB", "dC", "dA", "dD"):
+        assert np.array_equal(got[k], again[k]), k
