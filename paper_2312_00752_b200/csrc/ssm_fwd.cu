@@ -17,7 +17,7 @@ namespace ssm {
 
 // threads per block: 16 thread groups (of N / 4 lanes each) for N >= 16, 32 groups otherwise (keeps the staged tiles
 // below 48 KB)
-__host__ __device__ constexpr int fwd_threads(int N) { return N >= 16 ? 4 * N : 32; }
+__host__ __device__ constexpr int fwd_threads(int N) { return N >= 16 ? 4 * N : (N == 8 ? 64 : 32); }
 constexpr int kFwdTile = 32;  // time steps staged in shared memory at a time
 
 template <typename IO, int N, int CPT, int MODE>
