@@ -84,7 +84,9 @@ Plan make_plan(const ssm_problem_t& p) {
       const long long max_by_len = std::max(1, p.L / 256);
       nseg = (int)std::min<long long>(std::min(want, max_by_len), 65535);
     }
-  } else if (warps < sub_partitions * 3 / 4) {
+  } else if (warps < sub_partitions * 3) {
+    // generic kernels: a warp is latency-bound, so aim for 6 warps per sub-partition although a split costs half a
+    // sweep more (measured 2 to 2.5 times faster than one or two warps per sub-partition)
     const long long want = (6 * sub_partitions + warps - 1) / warps;
     const long long max_by_len = std::max(1, p.L / 256);
     nseg = (int)std::min<long long>(std::min(want, max_by_len), 65535);
@@ -96,12 +98,14 @@ Plan make_plan(const ssm_problem_t& p) {
   return pl;
 }
 
-// The backward pass splits time on its own terms.  Its unit of work is a chain (batch entry, segment, group of 32
-// channels) walked by one block of the persistent kernel, 4 blocks per SM; a problem with fewer chains than resident
-// blocks (the 130M layer shape: 384 for 592) leaves SMs idle and every chain sequential, and the extra adjoint pre-pass
-// that a split needs costs about a third of a forward sweep.  So: no split while the chains nearly fill the GPU,
-// otherwise enough segments for about 3 chains per resident block (segments of at least 256 steps).  The checkpoint
-// states do not depend on the split, so forward and backward may disagree about it.
+static long long generic_bwd_warps(int N) {   // warps of a block of the generic backward kernel
+  const int lpc = N / (N < 4 ? N : 4);
+  return std::max(1, bwd_channels_per_block(N) * lpc / 32);
+}
+
+// The backward pass splits time on its own terms (the checkpoint states do not depend on the split, so forward and
+// backward may disagree about it).  A split costs an adjoint pre-pass over all segments but the first and a carry scan;
+// it pays when the chains alone leave the SM sub-partitions with too few warps.  Segments are at least 256 steps.
 Plan make_bwd_plan(const ssm_problem_t& p) {
   Plan pl = make_plan(p);
   if (tuned_shape(p)) {
@@ -114,10 +118,17 @@ Plan make_bwd_plan(const ssm_problem_t& p) {
   int nseg = 1;
   if (p.flags & SSM_FLAG_COMPLEX) {
     // the complex path does not split time
-  } else if (tuned_shape(p) ? chains < 2 * resident : chains * 4 < resident * 3) {
+  } else if (tuned_shape(p)) {
     // the tuned kernel wants two warps per SM sub-partition (a lone warp cannot cover its own latencies), i.e. two
     // rounds of chains; the adjoint pre-pass that a split costs is about a tenth of the backward work
-    const long long want = (2 * resident + chains - 1) / chains;
+    if (chains < 2 * resident) {
+      const long long want = (2 * resident + chains - 1) / chains;
+      const long long max_by_len = std::max(1, p.L / 256);
+      nseg = (int)std::min<long long>(std::min(want, max_by_len), 65535);
+    }
+  } else if (chains * generic_bwd_warps(p.N) < 4 * resident) {
+    // generic kernel: latency-bound warps, so aim for 8 per sub-partition (measured against 2: 1.1 to 1.5 times faster)
+    const long long want = (8 * resident + chains * generic_bwd_warps(p.N) - 1) / (chains * generic_bwd_warps(p.N));
     const long long max_by_len = std::max(1, p.L / 256);
     nseg = (int)std::min<long long>(std::min(want, max_by_len), 65535);
   }
