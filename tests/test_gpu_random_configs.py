@@ -59,6 +59,12 @@ def test_random_problem(case):
             continue
         state_tol = 1e-4 if k == "dh0" and c["io"] == "bf16" else tol["grad"]   # dh0 is float32 on both paths
         assert U.rel_err(U.to_host(g[k]), ref[k]) <= max(state_tol, 0.0), (k, c)
+    if c["io"] == "bf16":
+        # beside the tolerances relative to the largest element: every element within its own rounding
+        got = {k: U.to_host(v) for k, v in g.items() if v is not None}
+        got["out"] = U.to_host(out)
+        ref_all = dict(ref, out=ref_out)
+        U.assert_elementwise(got, ref_all, "bf16", f"random case {c}")
 
 
 FUSED_CASES = [_draw(np.random.default_rng([2312, 753, i])) for i in range(40)]
