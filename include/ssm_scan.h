@@ -108,7 +108,10 @@ SSM_API size_t ssm_scan_fwd_workspace_bytes(const ssm_problem_t* p);
 SSM_API size_t ssm_scan_bwd_workspace_bytes(const ssm_problem_t* p);
 
 /* Bytes of the `saved_states` buffer: float32 states h at the start of every block of ssm_scan_checkpoint_steps()
- * time steps, laid out [batch][ceil(L / steps)][D][N].  Independent of flags. */
+ * time steps.  The buffer is opaque: its layout is the library's ([batch][ceil(L / steps)][D][N], or for bf16 io with
+ * N = 16 and D % 8 == 0 a layout tiled by groups of 32 channels, D rounded up to a multiple of 32) and depends on the
+ * problem (dimensions, dtype, SSM_FLAG_COMPLEX, the STATIC / ZOH flags); a buffer written by a forward call is valid
+ * for backward calls with the same ssm_problem_t only. */
 SSM_API size_t ssm_scan_saved_state_bytes(const ssm_problem_t* p);
 SSM_API int32_t ssm_scan_checkpoint_steps(void);
 

@@ -201,7 +201,7 @@ static BwdWorkspace bwd_layout(const ssm_problem_t& p, const Plan& pl, const Pla
   w.dA_part = take(parts * p.D * p.N * sizeof(float));
   w.dD_part = take(parts * p.D * sizeof(float));
   w.dbias_part = take(parts * p.D * sizeof(float));
-  w.ckpt = take((size_t)p.batch * pl.nck * p.D * p.N * sizeof(float));
+  w.ckpt = take((size_t)p.batch * pl.nck * ckpt_floats_per_step(tuned_shape(p), p.D, p.N) * sizeof(float));
   if (pl.nseg > 1) {
     const size_t st = parts * p.D * p.N * sizeof(float);
     w.seg_local = take(st);
@@ -286,7 +286,7 @@ size_t ssm_scan_saved_state_bytes(const ssm_problem_t* p) {
   if (validate_problem(p) != SSM_OK) return 0;
   if (p->flags & SSM_FLAG_COMPLEX) return complex_saved_state_bytes(*p);
   const size_t nck = (size_t)(p->L + kCkptSteps - 1) / kCkptSteps;
-  return (size_t)p->batch * nck * p->D * p->N * sizeof(float);
+  return (size_t)p->batch * nck * ckpt_floats_per_step(tuned_shape(*p), p->D, p->N) * sizeof(float);
 }
 
 int32_t ssm_scan_checkpoint_steps(void) { return kCkptSteps; }
@@ -404,6 +404,7 @@ static ssm_status_t fwd_impl(const ssm_problem_t* p, const void* x, const void* 
   fp.h_start = h_start;
   fp.h_last = h_last;
   fp.ckpt = save ? static_cast<float*>(saved_states) : nullptr;
+  fp.ckpt_tiled = tuned_shape(*p) ? 1 : 0;
   if (launch_fwd(*p, pl, fp, kFwdFull, s) != cudaSuccess) return SSM_ERR_CUDA;
   return SSM_OK;
 }
@@ -539,6 +540,7 @@ static ssm_status_t bwd_impl(const ssm_problem_t* p, const void* x, const void* 
       return SSM_ERR_CUDA;
     fp.h_start = h_start;
     fp.ckpt = reinterpret_cast<float*>(ws + w.ckpt);
+    fp.ckpt_tiled = tuned_shape(*p) ? 1 : 0;
     if (launch_fwd(*p, pl_fwd, fp, kFwdCkptOnly, s) != cudaSuccess) return SSM_ERR_CUDA;
     ckpt = fp.ckpt;
   }
@@ -553,6 +555,7 @@ static ssm_status_t bwd_impl(const ssm_problem_t* p, const void* x, const void* 
   bp.Dskip = has_d ? D_skip : nullptr;
   bp.dout = dout;
   bp.ckpt = ckpt;
+  bp.ckpt_tiled = tuned_shape(*p) ? 1 : 0;
   bp.dx = dx;
   bp.ddelta = ddelta;
   bp.dz = has_z ? dz : nullptr;

@@ -126,7 +126,7 @@ __global__ void __launch_bounds__(BwdGeom<N>::THREADS) ssm_bwd_kernel(const BwdP
     float h[S];
 #pragma unroll
     for (int k = 0; k < S; ++k) {
-      h[k] = valid ? p.ckpt[(((size_t)b * p.nck + (size_t)kb * (T / kCkptSteps)) * D + d) * N + j * S + k] : 0.f;
+      h[k] = valid ? p.ckpt[ckpt_offset(p.ckpt_tiled, b, p.nck, kb * (T / kCkptSteps), D, N, d, j * S + k)] : 0.f;
       s_h[(size_t)slot * N + j * S + k] = h[k];
     }
     __syncthreads();

@@ -586,7 +586,7 @@ __global__ void __launch_bounds__(kBwdWarps * 32, (CPT == 16 / S) ? 2 : 3)
           for (int q = 0; q < CPT; ++q)
 #pragma unroll
             for (int k = 0; k < S / 4; ++k) {
-              const size_t go = ok ? (((size_t)b * p.nck + (t0 + sb * kSB) / kCkptSteps) * D + chan(q)) * 16 + S * j + 4 * k : 0;
+              const size_t go = ok ? ckpt_offset(1, b, p.nck, (t0 + sb * kSB) / kCkptSteps, D, 16, chan(q), S * j + 4 * k) : 0;
               cp_async16(&sm.ck[st][sb][q * (S / 4) + k][lane], p.ckpt + go, ok);
             }
         }

@@ -34,6 +34,20 @@ struct Plan {
 Plan make_plan(const ssm_problem_t& p);
 
 // ---------------------------------------------------------------------------------------------- kernel params
+// Offset (in floats) of state n of channel d in checkpoint kc of batch entry b.
+//   plain: [batch][nck][D][N].
+//   tiled (N = 16 only): [batch][nck][ceil(D / 32)][4][32][4] -- within a group of 32 channels the four 16-byte quarters
+//   of a channel's 16 states are split over four planes, so that the 32 lanes of a warp that own one channel each write
+//   (and read) 512 contiguous bytes per instruction instead of 16 bytes every 64.
+__host__ __device__ __forceinline__ size_t ckpt_offset(int tiled, int b, int nck, int kc, int D, int N, int d, int n) {
+  if (tiled) return ((((size_t)b * nck + kc) * ((D + 31) / 32) + (d >> 5)) * 4 + (n >> 2)) * 128 + (size_t)(d & 31) * 4 + (n & 3);
+  return (((size_t)b * nck + kc) * D + d) * N + n;
+}
+// floats of the checkpoint states of one batch entry and checkpoint
+__host__ __device__ __forceinline__ size_t ckpt_floats_per_step(int tiled, int D, int N) {
+  return tiled ? (size_t)((D + 31) / 32) * 512 : (size_t)D * N;
+}
+
 struct FwdParams {
   const void* x;
   const void* delta;
@@ -44,7 +58,8 @@ struct FwdParams {
   const float* Dskip;  // null: no skip term
   void* out;           // FULL mode
   const float* h_start;  // [batch][nseg][D][N] start state of each segment; null: zero
-  float* ckpt;           // [batch][nck][D][N] checkpoint states to write; null: none
+  float* ckpt;           // checkpoint states to write (layout: ckpt_offset below); null: none
+  int ckpt_tiled;        // 1: the layout of the tuned bf16 / N = 16 kernels
   float* seg_end;        // SUMMARY mode: [batch][nseg][D][N] end state of each segment started from zero
   float* seg_dsum;       // SUMMARY mode: [batch][nseg][D] sum of delta over the segment
   float* h_last;         // FULL mode: [batch][D][N] state after the last step; null: not wanted
@@ -97,7 +112,8 @@ struct BwdParams {
   const float* A;
   const float* Dskip;
   const void* dout;
-  const float* ckpt;      // [batch][nck][D][N]
+  const float* ckpt;      // checkpoint states (layout: ckpt_offset below)
+  int ckpt_tiled;         // 1: the layout of the tuned bf16 / N = 16 kernels
   const float* mu_in;     // [batch][nseg][D][N] adjoint inflow of each segment; null: zero
   float* seg_local;       // LOCAL mode: [batch][nseg][D][N] adjoint leaving each segment with zero inflow
   int local_as_inflow;    // tuned LOCAL kernel, two segments, no outside adjoint: write the result of segment 1 as the

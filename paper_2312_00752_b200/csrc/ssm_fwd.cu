@@ -118,7 +118,7 @@ __global__ void __launch_bounds__(fwd_threads(N)) ssm_fwd_kernel(const FwdParams
         for (int q = 0; q < CPT; ++q) {
           const int d = d_thr + q;
           if (d < D) {
-            float* dst = p.ckpt + (((size_t)b * p.nck + kc) * D + d) * N + j * S;
+            float* dst = p.ckpt + ckpt_offset(p.ckpt_tiled, b, p.nck, kc, D, N, d, j * S);
 #pragma unroll
             for (int k = 0; k < S; ++k) dst[k] = h[q][k];
           }

@@ -218,6 +218,10 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32) ssm_fwd_warp_kernel(const
     const int c_prep = d_w + (lane % CW);
     const float bias_prep = (SPF && p.delta_bias != nullptr && c_prep < D) ? p.delta_bias[c_prep] : 0.f;
     const float bias_own = (SP && !SPF && p.delta_bias != nullptr && valid) ? p.delta_bias[c_own] : 0.f;
+    // this lane's first 16 bytes of checkpoint 0 of the batch entry (tiled layout, ckpt_offset) and the floats from one
+    // checkpoint to the next; the lane's S / 4 quarters are 128 floats apart
+    const size_t ck_stride = ckpt_floats_per_step(1, D, 16);
+    float* const ck_lane = (!SUMMARY && p.ckpt != nullptr && valid) ? p.ckpt + ckpt_offset(1, b, p.nck, 0, D, 16, c_own, S * j) : nullptr;
     int rows_live = 0;   // rows of the current tile inside the piece (the rest are identity steps)
     float dsum = 0.f;
 
@@ -435,11 +439,11 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32) ssm_fwd_warp_kernel(const
       for (int sb = 0; sb < kWT / kSub; ++sb) {
         const int ts = t0 + sb * kSub;
         if (ts >= t_to) break;
-        if (!SUMMARY && p.ckpt != nullptr && valid && SSM_IN_RANGE(ts / kCkptSteps < p.nck && ts < p.L, sc.abort)) {
+        if (!SUMMARY && ck_lane != nullptr && SSM_IN_RANGE(ts / kCkptSteps < p.nck && ts < p.L, sc.abort)) {
+          float* dst = ck_lane + (size_t)(ts / kCkptSteps) * ck_stride;
 #pragma unroll
           for (int k = 0; k < S / 4; ++k)
-            *reinterpret_cast<float4*>(p.ckpt + (((size_t)b * p.nck + ts / kCkptSteps) * D + c_own) * 16 + S * j + 4 * k) =
-                make_float4(h[2 * k].x, h[2 * k].y, h[2 * k + 1].x, h[2 * k + 1].y);
+            *reinterpret_cast<float4*>(dst + 128 * k) = make_float4(h[2 * k].x, h[2 * k].y, h[2 * k + 1].x, h[2 * k + 1].y);
         }
         if constexpr (ZOH) {
           // smallest step size of the live rows of the sub-block for this lane's channel

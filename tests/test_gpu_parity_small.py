@@ -170,3 +170,28 @@ def test_pointers_off_the_16_byte_grid_take_the_generic_kernels():
     dev2 = {k: (shifted(v) if v is not None else None) for k, v in dev.items()}
     got = U.gpu_fwd_bwd(dev2)
     U.assert_parity(got, U.oracle_fwd_bwd(inp), "bf16", "misaligned")
+
+
+@pytest.mark.parametrize("fwd_generic", [False, True])
+def test_saved_states_pass_between_tuned_and_generic_kernels(fwd_generic):
+    # the forward and the backward of one problem may take different kernels (the tuned ones need 16-byte aligned
+    # pointers): the checkpoint states one of them saves must be the ones the other reads.  D = 72 leaves the third
+    # group of 32 channels ragged.
+    import torch
+    from paper_2312_00752_b200 import binding as K
+    cfg, inp = _case(2, 150, 72, 16, "bf16")
+    dev = U.to_device(inp, "bf16")
+
+    def shifted(t):   # same values at an address that is 8 bytes past a 16-byte boundary
+        buf = torch.empty(t.numel() + 8, dtype=t.dtype, device=t.device)
+        v = buf[4:4 + t.numel()].view(t.shape)
+        v.copy_(t)
+        assert v.data_ptr() % 16 == 8
+        return v
+    args = lambda x: (x, dev["delta"], dev["A"], dev["B"], dev["C"], dev["D_skip"], dev["z"])
+    x_off = shifted(dev["x"])
+    out, saved = K.ssm_scan_fwd(*args(x_off if fwd_generic else dev["x"]), save_states=True)
+    g = K.ssm_scan_bwd(*args(dev["x"] if fwd_generic else x_off), dev["dout"], saved)
+    got = {"out": U.to_host(out)}
+    got.update({k: U.to_host(g[k]) for k in U.GRADS})
+    U.assert_parity(got, U.oracle_fwd_bwd(inp), "bf16", f"mixed kernels fwd_generic={fwd_generic}")
