@@ -68,7 +68,7 @@ __device__ __forceinline__ float bf16at(const uint32_t* row, int c) {
 }  // namespace
 
 template <int S, int MODE, bool SP, bool ZOH, int BC, int NST>
-__global__ void __launch_bounds__(kWarpsPerBlock * 32) ssm_fwd_warp_kernel(const FwdParams p, const WarpSched sc) {
+__global__ void __launch_bounds__(kWarpsPerBlock * 32, MODE == kFwdFull ? 1 : 0) ssm_fwd_warp_kernel(const FwdParams p, const WarpSched sc) {
   static_assert(NST == 2 || NST == 3, "ring stages");
   static_assert(S == 16 || S == 8, "one lane or a lane pair per channel");
   constexpr bool FULL = (MODE == kFwdFull);
