@@ -32,7 +32,8 @@
  *     anything is launched and reported by the return value; nothing is written in that case.  A failed kernel
  *     launch is reported as SSM_ERR_CUDA.
  *   - N must be 1, 2, 4, 8, 16 (the state sizes Table 10 ablates), 32 or 64 (larger states on the generic kernels;
- *     the tuned kernels are N = 16).  All io pointers must be
+ *     the tuned kernels are N = 16; bf16 problems with N < 16 and D % 8 == 0 run on them too, with A, B, C and the
+ *     state arrays widened inside the workspace by columns that stay zero).  All io pointers must be
  *     aligned to the element size; 16-byte aligned pointers together with D % 8 == 0 select the vector path.
  *   - Results are bitwise reproducible for fixed inputs, shape, flags and library build: every reduction (over n,
  *     over channels for dB/dC, over batch and time for dA/dD) has a fixed order and no floating-point atomics

@@ -25,6 +25,20 @@ int fwd_states_per_thread();
 int fwd_fast_channels_per_warp();
 int bwd_fast_channels_per_warp();
 bool bwd_fast_applicable(const ssm_problem_t& prob, const BwdParams& p);
+// ssm_repack.cu
+enum { kRepackBf16 = 0, kRepackF32 = 1, kRepackA = 2 };
+constexpr int kRepackMax = 6;
+struct RepackJob {
+  const void* src;
+  void* dst;
+  int rows, n_src, n_dst, kind;
+};
+struct RepackJobs {
+  RepackJob job[kRepackMax];
+  int count;
+};
+void repack_add(RepackJobs& jobs, const void* src, void* dst, long long rows, int n_src, int n_dst, int kind);
+cudaError_t repack_run(const RepackJobs& jobs, cudaStream_t s);
 size_t fwd_handoff_bytes_per_worker();
 size_t bwd_handoff_bytes_per_worker(bool static_B, bool static_C);
 
@@ -43,7 +57,52 @@ static int shared_workers(long long chains) {
   return (int)std::min<long long>(std::max<long long>(chains, 8LL * kNumSMs), (long long)kMaxWarpsPerSM * kNumSMs);
 }
 
+constexpr size_t kStatusBytes = 256;   // head of every workspace: the status word
 static inline size_t align_up(size_t v) { return (v + 255) & ~(size_t)255; }
+
+// bf16 problems with fewer than 16 states run as 16-state problems on the tuned kernels, with A, B, C (and the state
+// arrays) widened by columns that stay zero (ssm_repack.cu); `wide` is that problem.
+constexpr int kWideN = 16;
+static bool widen_route(const ssm_problem_t& p, ssm_problem_t* wide) {
+  if (p.io_dtype != SSM_BF16 || p.N >= kWideN || p.D % 8 != 0 || (p.flags & SSM_FLAG_COMPLEX)) return false;
+  if ((long long)p.batch * p.L > 0x7fffffffLL || (long long)p.batch * p.D > 0x7fffffffLL) return false;
+  if (wide) {
+    *wide = p;
+    wide->N = kWideN;
+  }
+  return true;
+}
+// Buffers of the widened arrays, placed behind the wide problem's own workspace (whose head holds the status word).
+struct WidenLayout {
+  size_t A, B, C, h0, h_last, dh_last, dA, dB, dC, dh0, total;
+};
+static WidenLayout widen_layout(const ssm_problem_t& p, size_t inner_bytes, bool bwd) {
+  WidenLayout w{};
+  size_t off = align_up(inner_bytes > (size_t)kStatusBytes ? inner_bytes : (size_t)kStatusBytes);
+  auto take = [&](size_t bytes) {
+    const size_t at = off;
+    off += align_up(bytes);
+    return at;
+  };
+  const size_t rows_t = (size_t)p.batch * p.L, rows_s = (size_t)p.batch * p.D;
+  const size_t bsz = (p.flags & SSM_FLAG_STATIC_B) ? (size_t)p.D * kWideN * sizeof(float) : rows_t * kWideN * 2;
+  const size_t csz = (p.flags & SSM_FLAG_STATIC_C) ? (size_t)p.D * kWideN * sizeof(float) : rows_t * kWideN * 2;
+  w.A = take((size_t)p.D * kWideN * sizeof(float));
+  w.B = take(bsz);
+  w.C = take(csz);
+  w.h0 = take(rows_s * kWideN * sizeof(float));
+  if (!bwd) {
+    w.h_last = take(rows_s * kWideN * sizeof(float));
+  } else {
+    w.dh_last = take(rows_s * kWideN * sizeof(float));
+    w.dA = take((size_t)p.D * kWideN * sizeof(float));
+    w.dB = take(bsz);
+    w.dC = take(csz);
+    w.dh0 = take(rows_s * kWideN * sizeof(float));
+  }
+  w.total = off;
+  return w;
+}
 
 static ssm_status_t validate_problem(const ssm_problem_t* p) {
   if (p == nullptr) return SSM_ERR_INVALID_ARG;
@@ -140,7 +199,6 @@ Plan make_bwd_plan(const ssm_problem_t& p) {
 }
 
 // Every non-empty workspace starts with a status block whose first word is the one ssm_scan_check_status reads.
-constexpr size_t kStatusBytes = 256;
 
 struct FwdWorkspace {
   size_t seg_end, seg_dsum, h_start, flags, handoff, total;
@@ -273,18 +331,24 @@ extern "C" {
 
 size_t ssm_scan_fwd_workspace_bytes(const ssm_problem_t* p) {
   if (validate_problem(p) != SSM_OK) return 0;
+  ssm_problem_t wide;
+  if (widen_route(*p, &wide)) return widen_layout(*p, ssm_scan_fwd_workspace_bytes(&wide), false).total;
   return fwd_layout(*p, make_plan(*p)).total;
 }
 
 size_t ssm_scan_bwd_workspace_bytes(const ssm_problem_t* p) {
   if (validate_problem(p) != SSM_OK) return 0;
   if (p->flags & SSM_FLAG_COMPLEX) return complex_bwd_workspace_bytes(*p);
+  ssm_problem_t wide;
+  if (widen_route(*p, &wide)) return widen_layout(*p, ssm_scan_bwd_workspace_bytes(&wide), true).total;
   return bwd_layout(*p, make_bwd_plan(*p), make_plan(*p)).total;
 }
 
 size_t ssm_scan_saved_state_bytes(const ssm_problem_t* p) {
   if (validate_problem(p) != SSM_OK) return 0;
   if (p->flags & SSM_FLAG_COMPLEX) return complex_saved_state_bytes(*p);
+  ssm_problem_t wide;
+  if (widen_route(*p, &wide)) return ssm_scan_saved_state_bytes(&wide);
   const size_t nck = (size_t)(p->L + kCkptSteps - 1) / kCkptSteps;
   return (size_t)p->batch * nck * ckpt_floats_per_step(tuned_shape(*p), p->D, p->N) * sizeof(float);
 }
@@ -320,6 +384,8 @@ ssm_status_t ssm_scan_plan(const ssm_problem_t* p, int32_t* n_segments, int32_t*
                            int32_t* channels_per_block, int32_t* states_per_thread) {
   const ssm_status_t st = validate_problem(p);
   if (st != SSM_OK) return st;
+  ssm_problem_t wide;
+  if (widen_route(*p, &wide)) return ssm_scan_plan(&wide, n_segments, segment_steps, channels_per_block, states_per_thread);
   const Plan pl = make_plan(*p);
   if (n_segments) *n_segments = pl.nseg;
   if (segment_steps) *segment_steps = pl.seg_steps;
@@ -332,6 +398,8 @@ ssm_status_t ssm_scan_bwd_plan(const ssm_problem_t* p, int32_t* n_segments, int3
                                int32_t* channels_per_group) {
   const ssm_status_t st = validate_problem(p);
   if (st != SSM_OK) return st;
+  ssm_problem_t wide;
+  if (widen_route(*p, &wide)) return ssm_scan_bwd_plan(&wide, n_segments, segment_steps, channels_per_group);
   const Plan pl = make_bwd_plan(*p);
   if (n_segments) *n_segments = pl.nseg;
   if (segment_steps) *segment_steps = pl.seg_steps;
@@ -362,6 +430,31 @@ static ssm_status_t fwd_impl(const ssm_problem_t* p, const void* x, const void* 
                        save ? saved_states : nullptr, static_cast<cudaStream_t>(stream)) == cudaSuccess
                ? SSM_OK
                : SSM_ERR_CUDA;
+  }
+  ssm_problem_t wide;
+  if (widen_route(*p, &wide)) {
+    const size_t inner = ssm_scan_fwd_workspace_bytes(&wide);
+    const WidenLayout wl = widen_layout(*p, inner, false);
+    st = check_ws(workspace, workspace_bytes, wl.total);
+    if (st != SSM_OK) return st;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    char* ws = static_cast<char*>(workspace);
+    const bool sb = p->flags & SSM_FLAG_STATIC_B, sc = p->flags & SSM_FLAG_STATIC_C;
+    const long long rows_t = (long long)p->batch * p->L, rows_s = (long long)p->batch * p->D;
+    if (cudaMemsetAsync(ws, 0, kStatusBytes, s) != cudaSuccess) return SSM_ERR_CUDA;
+    RepackJobs in{};
+    repack_add(in, A, ws + wl.A, p->D, p->N, kWideN, kRepackA);
+    repack_add(in, B, ws + wl.B, sb ? p->D : rows_t, p->N, kWideN, sb ? kRepackF32 : kRepackBf16);
+    repack_add(in, C, ws + wl.C, sc ? p->D : rows_t, p->N, kWideN, sc ? kRepackF32 : kRepackBf16);
+    repack_add(in, h0, ws + wl.h0, rows_s, p->N, kWideN, kRepackF32);
+    if (repack_run(in, s) != cudaSuccess) return SSM_ERR_CUDA;
+    st = fwd_impl(&wide, x, delta, delta_bias, reinterpret_cast<const float*>(ws + wl.A), ws + wl.B, ws + wl.C, D_skip, z,
+                  h0 ? reinterpret_cast<const float*>(ws + wl.h0) : nullptr, out,
+                  h_last ? reinterpret_cast<float*>(ws + wl.h_last) : nullptr, saved_states, workspace, inner, stream);
+    if (st != SSM_OK) return st;
+    RepackJobs outj{};
+    repack_add(outj, h_last ? ws + wl.h_last : nullptr, h_last, rows_s, kWideN, p->N, kRepackF32);
+    return repack_run(outj, s) == cudaSuccess ? SSM_OK : SSM_ERR_CUDA;
   }
   const Plan pl = make_plan(*p);
   st = check_ws(workspace, workspace_bytes, fwd_layout(*p, pl).total);
@@ -501,6 +594,36 @@ static ssm_status_t bwd_impl(const ssm_problem_t* p, const void* x, const void* 
                        static_cast<cudaStream_t>(stream)) == cudaSuccess
                ? SSM_OK
                : SSM_ERR_CUDA;
+  }
+  ssm_problem_t wide;
+  if (widen_route(*p, &wide)) {
+    const size_t inner = ssm_scan_bwd_workspace_bytes(&wide);
+    const WidenLayout wl = widen_layout(*p, inner, true);
+    st = check_ws(workspace, workspace_bytes, wl.total);
+    if (st != SSM_OK) return st;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    char* ws = static_cast<char*>(workspace);
+    const bool sb = p->flags & SSM_FLAG_STATIC_B, sc = p->flags & SSM_FLAG_STATIC_C;
+    const long long rows_t = (long long)p->batch * p->L, rows_s = (long long)p->batch * p->D;
+    RepackJobs in{};
+    repack_add(in, A, ws + wl.A, p->D, p->N, kWideN, kRepackA);
+    repack_add(in, B, ws + wl.B, sb ? p->D : rows_t, p->N, kWideN, sb ? kRepackF32 : kRepackBf16);
+    repack_add(in, C, ws + wl.C, sc ? p->D : rows_t, p->N, kWideN, sc ? kRepackF32 : kRepackBf16);
+    repack_add(in, h0, ws + wl.h0, rows_s, p->N, kWideN, kRepackF32);
+    repack_add(in, dh_last, ws + wl.dh_last, rows_s, p->N, kWideN, kRepackF32);
+    if (repack_run(in, s) != cudaSuccess) return SSM_ERR_CUDA;
+    st = bwd_impl(&wide, x, delta, delta_bias, reinterpret_cast<const float*>(ws + wl.A), ws + wl.B, ws + wl.C, D_skip, z,
+                  dout, h0 ? reinterpret_cast<const float*>(ws + wl.h0) : nullptr,
+                  dh_last ? reinterpret_cast<const float*>(ws + wl.dh_last) : nullptr, saved_states, dx, ddelta,
+                  ddelta_bias, reinterpret_cast<float*>(ws + wl.dA), ws + wl.dB, ws + wl.dC, dD, dz,
+                  dh0 ? reinterpret_cast<float*>(ws + wl.dh0) : nullptr, workspace, inner, stream);
+    if (st != SSM_OK) return st;
+    RepackJobs outj{};
+    repack_add(outj, ws + wl.dA, dA, p->D, kWideN, p->N, kRepackF32);
+    repack_add(outj, ws + wl.dB, dB, sb ? p->D : rows_t, kWideN, p->N, sb ? kRepackF32 : kRepackBf16);
+    repack_add(outj, ws + wl.dC, dC, sc ? p->D : rows_t, kWideN, p->N, sc ? kRepackF32 : kRepackBf16);
+    repack_add(outj, dh0 ? ws + wl.dh0 : nullptr, dh0, rows_s, kWideN, p->N, kRepackF32);
+    return repack_run(outj, s) == cudaSuccess ? SSM_OK : SSM_ERR_CUDA;
   }
   const Plan pl = make_bwd_plan(*p), pl_fwd = make_plan(*p);
   const BwdWorkspace w = bwd_layout(*p, pl, pl_fwd);
