@@ -549,6 +549,13 @@ def run_ours(args, cfg):
                 line["variants"][name] = time_shape(K, torch, dev, stream, cfg, peak, reps=5, **kw)
             except Exception as exc:
                 line["variants"][name] = {"error": str(exc)}
+        # other state sizes at the same (batch, L, D): N = 8 (bf16: the 16-state kernels on a widened problem) and
+        # N = 64 at a quarter of the batch (generic kernels)
+        for name, small in (("state_8", cfg.scaled(N=8)), ("state_64_batch_1", cfg.scaled(N=64, batch=1))):
+            try:
+                line["variants"][name] = time_shape(K, torch, dev, stream, small, peak, reps=5)
+            except Exception as exc:
+                line["variants"][name] = {"error": str(exc)}
         line["configs"] = {}
         for ci in (1, 2, 4):
             if ci == cfg.cfg_id:

@@ -26,6 +26,7 @@ def _host_tensors(inp, io, pin=True):
     (11, 64, 24, 8, "f32", True),        # six pieces, the last one smaller
     (1, 200, 16, 16, "bf16", True),      # a single piece
     (3, 130, 32, 16, "bf16", False),     # pageable host memory: same results, no overlap
+    (3, 90, 24, 4, "bf16", True),        # fewer than 16 states: the widened problem inside every piece
 ])
 def test_host_call_equals_device_calls_and_oracle(batch, L, D, N, io, pin):
     import torch
