@@ -184,8 +184,8 @@ SSM_API ssm_status_t ssm_scan_bwd_fused_dt_state(const ssm_problem_t* p, const v
 /*
  * One recurrent step (Eq. 2a/2b evaluated for a single t, the mode used for autoregressive inference): p->L must be
  * 1; x, delta, z, out are [batch][D], B, C are [batch][N] (io_dtype), A [D][N], D_skip [D]; the float32 state
- * h [batch][D][N] is read and overwritten with the state after the step (h and A 16-byte aligned when N >= 4).  Needs
- * no workspace.
+ * h [batch][D][N] is read and overwritten with the state after the step (when N >= 4: h and A 16-byte aligned, B and
+ * C aligned to four of their elements).  Needs no workspace.
  */
 SSM_API ssm_status_t ssm_step(const ssm_problem_t* p, const void* x, const void* delta, const float* A, const void* B,
                               const void* C, const float* D_skip, const void* z, float* h, void* out,

@@ -539,8 +539,12 @@ ssm_status_t ssm_step(const ssm_problem_t* p, const void* x, const void* delta, 
   if (!static_bc_aligned(*p, B, C, nullptr, nullptr)) return SSM_ERR_INVALID_ARG;
   for (const void* q : {(const void*)A, (const void*)D_skip, (const void*)h})
     if (q && !aligned_to(q, 4)) return SSM_ERR_INVALID_ARG;
-  // the state and A are accessed 16 bytes at a time when a channel has at least 4 states
+  // the state and A are accessed 16 bytes at a time when a channel has at least 4 states, B and C four values at a time
   if (p->N >= 4 && (!aligned_to(A, 16) || !aligned_to(h, 16))) return SSM_ERR_INVALID_ARG;
+  if (p->N >= 4 && !(p->flags & SSM_FLAG_COMPLEX)) {
+    const size_t ab = (p->flags & SSM_FLAG_STATIC_B) ? 16 : 4 * esz, ac = (p->flags & SSM_FLAG_STATIC_C) ? 16 : 4 * esz;
+    if (!aligned_to(B, ab) || !aligned_to(C, ac)) return SSM_ERR_INVALID_ARG;
+  }
   if (p->flags & SSM_FLAG_COMPLEX)
     return complex_step(*p, x, delta, A, B, C, has_d ? D_skip : nullptr, has_z ? z : nullptr, h, out,
                         static_cast<cudaStream_t>(stream)) == cudaSuccess

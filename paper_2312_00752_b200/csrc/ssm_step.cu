@@ -19,7 +19,26 @@ struct StepGeom {
   static constexpr int CH = 128 / LPC;       // channels per block of 128 threads
 };
 
-template <typename IO, int N>
+// this thread's S values of a row of N: io dtype (B, C of the batch entry; one 8-byte load for four bf16 values) or float
+template <typename IO, int S>
+__device__ __forceinline__ void load_io_row(const IO* __restrict__ src, float (&v)[S]) {
+  if constexpr (S == 4 && sizeof(IO) == 2) {
+    const uint2 w = __ldg(reinterpret_cast<const uint2*>(src));
+    v[0] = __uint_as_float(w.x << 16);
+    v[1] = __uint_as_float(w.x & 0xffff0000u);
+    v[2] = __uint_as_float(w.y << 16);
+    v[3] = __uint_as_float(w.y & 0xffff0000u);
+  } else if constexpr (S == 4) {
+    const float4 w = __ldg(reinterpret_cast<const float4*>(src));
+    v[0] = w.x; v[1] = w.y; v[2] = w.z; v[3] = w.w;
+  } else {
+#pragma unroll
+    for (int k = 0; k < S; ++k) v[k] = io_to_float<IO>(__ldg(src + k));
+  }
+}
+
+// ZOH: the B-bar rule of Eq. 4; SB / SC: B / C are float32 parameters [D][N] instead of inputs [batch][N]
+template <typename IO, int N, bool ZOH, bool SB, bool SC>
 __global__ void __launch_bounds__(128) ssm_step_kernel(const StepParams p) {
   constexpr int S = StepGeom<N>::S, LPC = StepGeom<N>::LPC, CH = StepGeom<N>::CH;
   const int j = threadIdx.x % LPC;
@@ -28,42 +47,36 @@ __global__ void __launch_bounds__(128) ssm_step_kernel(const StepParams p) {
   const bool valid = d < p.D;          // (whole lane groups are valid or not: the shuffles below stay inside a group)
   const int dc = valid ? d : 0;
   const size_t e = (size_t)b * p.D + dc;
-  const IO* __restrict__ gB = static_cast<const IO*>(p.B) + (size_t)b * N + j * S;
-  const IO* __restrict__ gC = static_cast<const IO*>(p.C) + (size_t)b * N + j * S;
-  const float* __restrict__ sB = static_cast<const float*>(p.B) + (size_t)dc * N + j * S;   // static B / C: float32 [D][N]
-  const float* __restrict__ sC = static_cast<const float*>(p.C) + (size_t)dc * N + j * S;
   const float dt = io_to_float<IO>(static_cast<const IO*>(p.delta)[e]);
   const float u = io_to_float<IO>(static_cast<const IO*>(p.x)[e]);
   const float du = dt * u;
   float* hrow = p.h + e * N + j * S;
-  const float* arow = p.A + (size_t)dc * N + j * S;
-  float hv[S], av[S];
+  float hv[S], av[S], Bv[S], Cv[S];
+  load_io_row<float, S>(p.A + (size_t)dc * N + j * S, av);
+  if constexpr (SB) load_io_row<float, S>(static_cast<const float*>(p.B) + (size_t)dc * N + j * S, Bv);
+  else load_io_row<IO, S>(static_cast<const IO*>(p.B) + (size_t)b * N + j * S, Bv);
+  if constexpr (SC) load_io_row<float, S>(static_cast<const float*>(p.C) + (size_t)dc * N + j * S, Cv);
+  else load_io_row<IO, S>(static_cast<const IO*>(p.C) + (size_t)b * N + j * S, Cv);
   if constexpr (S == 4) {
     const float4 h4 = *reinterpret_cast<const float4*>(hrow);
-    const float4 a4 = __ldg(reinterpret_cast<const float4*>(arow));
     hv[0] = h4.x; hv[1] = h4.y; hv[2] = h4.z; hv[3] = h4.w;
-    av[0] = a4.x; av[1] = a4.y; av[2] = a4.z; av[3] = a4.w;
   } else {
 #pragma unroll
-    for (int k = 0; k < S; ++k) {
-      hv[k] = hrow[k];
-      av[k] = __ldg(arow + k);
-    }
+    for (int k = 0; k < S; ++k) hv[k] = hrow[k];
   }
   float y = 0.f;
 #pragma unroll
   for (int k = 0; k < S; ++k) {
-    const float Bk = p.static_B ? __ldg(sB + k) : io_to_float<IO>(__ldg(gB + k));
-    float a, bx = du * Bk;
-    if (p.zoh) {
+    float a, bx = du * Bv[k];
+    if constexpr (ZOH) {
       float E;
       zoh_discretize(dt, av[k], a, E);
-      bx = E * u * Bk;
+      bx = E * u * Bv[k];
     } else {
       a = ex2_approx(dt * (av[k] * kLog2e));
     }
     hv[k] = fmaf(a, hv[k], bx);
-    y = fmaf(p.static_C ? __ldg(sC + k) : io_to_float<IO>(__ldg(gC + k)), hv[k], y);
+    y = fmaf(Cv[k], hv[k], y);
   }
   if (valid) {
     if constexpr (S == 4) {
@@ -86,17 +99,32 @@ __global__ void __launch_bounds__(128) ssm_step_kernel(const StepParams p) {
   }
 }
 
+template <typename IO, int N>
+static void launch_step_n(const StepParams& p, cudaStream_t s) {
+  const dim3 grid((unsigned)((p.D + StepGeom<N>::CH - 1) / StepGeom<N>::CH), (unsigned)p.batch);
+  const int v = (p.zoh ? 1 : 0) | (p.static_B ? 2 : 0) | (p.static_C ? 4 : 0);
+  switch (v) {
+    case 0: ssm_step_kernel<IO, N, false, false, false><<<grid, 128, 0, s>>>(p); break;
+    case 1: ssm_step_kernel<IO, N, true, false, false><<<grid, 128, 0, s>>>(p); break;
+    case 2: ssm_step_kernel<IO, N, false, true, false><<<grid, 128, 0, s>>>(p); break;
+    case 3: ssm_step_kernel<IO, N, true, true, false><<<grid, 128, 0, s>>>(p); break;
+    case 4: ssm_step_kernel<IO, N, false, false, true><<<grid, 128, 0, s>>>(p); break;
+    case 5: ssm_step_kernel<IO, N, true, false, true><<<grid, 128, 0, s>>>(p); break;
+    case 6: ssm_step_kernel<IO, N, false, true, true><<<grid, 128, 0, s>>>(p); break;
+    default: ssm_step_kernel<IO, N, true, true, true><<<grid, 128, 0, s>>>(p); break;
+  }
+}
+
 template <typename IO>
 static cudaError_t launch_step_io(const StepParams& p, cudaStream_t s) {
-  auto grid = [&](int ch) { return dim3((unsigned)((p.D + ch - 1) / ch), (unsigned)p.batch); };
   switch (p.N) {
-    case 64: ssm_step_kernel<IO, 64><<<grid(StepGeom<64>::CH), 128, 0, s>>>(p); break;
-    case 32: ssm_step_kernel<IO, 32><<<grid(StepGeom<32>::CH), 128, 0, s>>>(p); break;
-    case 16: ssm_step_kernel<IO, 16><<<grid(StepGeom<16>::CH), 128, 0, s>>>(p); break;
-    case 8: ssm_step_kernel<IO, 8><<<grid(StepGeom<8>::CH), 128, 0, s>>>(p); break;
-    case 4: ssm_step_kernel<IO, 4><<<grid(StepGeom<4>::CH), 128, 0, s>>>(p); break;
-    case 2: ssm_step_kernel<IO, 2><<<grid(StepGeom<2>::CH), 128, 0, s>>>(p); break;
-    case 1: ssm_step_kernel<IO, 1><<<grid(StepGeom<1>::CH), 128, 0, s>>>(p); break;
+    case 64: launch_step_n<IO, 64>(p, s); break;
+    case 32: launch_step_n<IO, 32>(p, s); break;
+    case 16: launch_step_n<IO, 16>(p, s); break;
+    case 8: launch_step_n<IO, 8>(p, s); break;
+    case 4: launch_step_n<IO, 4>(p, s); break;
+    case 2: launch_step_n<IO, 2>(p, s); break;
+    case 1: launch_step_n<IO, 1>(p, s); break;
     default: return cudaErrorInvalidValue;
   }
   return cudaGetLastError();
