@@ -31,8 +31,8 @@ FALLBACK_HBM_GBS = 6650.0
 # DRAM bytes (read + write) of one launch of the dominant kernel of each direction from ncu captures at the bench
 # workload itself (profiles/ssm_bwd_warp_kernel_mamba2p8b_layer.md, profiles/ssm_fwd_warp_kernel_mamba2p8b_layer.md);
 # None where no capture exists.
-NCU_TRAFFIC_BYTES = {3: 706.0e6 + 395.5e6}
-NCU_TRAFFIC_BYTES_FWD = {3: 265.0e6 + 368.3e6}
+NCU_TRAFFIC_BYTES = {3: 705.4e6 + 395.6e6}
+NCU_TRAFFIC_BYTES_FWD = {3: 265.7e6 + 368.4e6}
 
 
 def parse_args():

@@ -44,7 +44,8 @@ __device__ __forceinline__ void cp_async_wait_but_one() { asm volatile("cp.async
 }  // namespace
 
 // SP: `delta` holds the pre-activation and the step size is delta + bias, through the softplus if asked (Algorithm 2 step 4)
-template <bool SP, bool SC>
+// WHOLE: every tile and every channel group of the problem is whole, so the staging and the tile loop carry no range tests
+template <bool SP, bool SC, bool WHOLE = false>
 __global__ void __launch_bounds__(kLWarps * 32) ssm_bwd_local_warp_kernel(const BwdParams p, const WarpSched sc) {
   constexpr int H = 8;   // float2 pairs of states per thread
   using Smem = LocalWarpSmem<SP, SC>;
@@ -96,7 +97,7 @@ __global__ void __launch_bounds__(kLWarps * 32) ssm_bwd_local_warp_kernel(const 
 #pragma unroll
         for (int k = 0; k < 4; ++k) {
           const int tt = xrow + 8 * k;
-          const bool ok = xcol_ok && (t0 + tt < t_seg_end);
+          const bool ok = WHOLE || (xcol_ok && (t0 + tt < t_seg_end));
           const size_t go = ok ? (row0 + tt) * D + d_w + xcc * 8 : 0;
           cp_async16(&sm.d[st][tt][xcc * 4], gd + go, ok);
           cp_async16(&sm.z[st][tt][xcc * 4], (has_z ? gz : gd) + go, ok && has_z);
@@ -105,7 +106,7 @@ __global__ void __launch_bounds__(kLWarps * 32) ssm_bwd_local_warp_kernel(const 
 #pragma unroll
         for (int k = 0; k < 2; ++k) {
           const int tt = brow + 16 * k;
-          const bool ok = t0 + tt < t_seg_end;
+          const bool ok = WHOLE || t0 + tt < t_seg_end;
           const size_t go = ok ? (row0 + tt) * 16 + bhc * 8 : 0;
           if constexpr (!SC) cp_async16(&sm.rC[st][tt][bhc * 4], gC + go, ok);
         }
@@ -241,14 +242,14 @@ __global__ void __launch_bounds__(kLWarps * 32) ssm_bwd_local_warp_kernel(const 
           for (int r = 0; r < kLT; ++r) {
             float v = bf16_at(sm.d[st][r], lane) + bias_own;
             if (p.softplus) v = softplus_fast(v);
-            sm.dF[r][lane] = (t0 + r < t_seg_end) ? v : 0.f;
+            sm.dF[r][lane] = (WHOLE || t0 + r < t_seg_end) ? v : 0.f;
           }
         }
       }
       __syncwarp();
 #pragma unroll 1
       for (int sb = kLT / 8 - 1; sb >= 0; --sb) {
-        if (t0 + sb * 8 >= t_seg_end) continue;   // identity steps
+        if (!WHOLE && t0 + sb * 8 >= t_seg_end) continue;   // identity steps
         if (ap) eight_steps(st, sb * 8, std::true_type{});
         else eight_steps(st, sb * 8, std::false_type{});
       }
@@ -310,6 +311,15 @@ cudaError_t launch_local(const Plan& plan, const BwdParams& p, cudaStream_t s) {
   sc.abort = p.abort;
   sc.handoff = p.handoff;                     // (the hand-off slots are shared: the two kernels run one after the other)
   const unsigned grid = (unsigned)((sc.workers + kLWarps - 1) / kLWarps);
+  if constexpr (!SC) {
+    // no ragged tile or channel group anywhere: the instantiation without range tests (same launch shape)
+    if (p.L % kLT == 0 && plan.seg_steps % kLT == 0 && p.D % 32 == 0) {
+      auto whole = ssm_bwd_local_warp_kernel<SP, SC, true>;
+      if ((e = cudaFuncSetAttribute(whole, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess) return e;
+      whole<<<grid, kLWarps * 32, smem, s>>>(p, sc);
+      return cudaGetLastError();
+    }
+  }
   kern<<<grid, kLWarps * 32, smem, s>>>(p, sc);
   return cudaGetLastError();
 }

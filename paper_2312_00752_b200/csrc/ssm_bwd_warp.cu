@@ -502,7 +502,9 @@ __device__ __forceinline__ void sub_block(const Lane<S, CPT>& ln, ChainRegs<S, C
 
 }  // namespace
 
-template <int S, int CPT, bool SP, bool ZOH, int BC>
+// WHOLE: every tile and every channel group of the problem is whole (L and the segment length are multiples of the tile,
+// D of the chain width), so the staging, the sub-blocks and the output copy carry no range tests
+template <int S, int CPT, bool SP, bool ZOH, int BC, bool WHOLE = false>
 __global__ void __launch_bounds__(kBwdWarps * 32, (CPT == 16 / S) ? 2 : 3)
     ssm_bwd_warp_kernel(const BwdParams p, const WarpSched sc) {
   constexpr bool SB = BC & 1, SC = BC & 2;
@@ -553,7 +555,7 @@ __global__ void __launch_bounds__(kBwdWarps * 32, (CPT == 16 / S) ? 2 : 3)
     constexpr int CPR = CW / 8;                 // chunks per row
     constexpr int XCH = kBT * CPR;              // chunks per tensor and tile
     const int c_grp = d_w + g * CPT;            // first channel of this lane group
-    const bool valid = c_grp < D;               // (CPT channels: all valid or none, D is a multiple of 8)
+    const bool valid = WHOLE || c_grp < D;      // (CPT channels: all valid or none, D is a multiple of 8)
     auto chan = [&](int q) { return OWN ? c_grp + (j ^ q) : c_grp; };
     auto issue_tile = [&](int tile, int st) {
       if (tile >= tile_lo && tile >= 0) {
@@ -564,7 +566,7 @@ __global__ void __launch_bounds__(kBwdWarps * 32, (CPT == 16 / S) ? 2 : 3)
           const int c = lane + 32 * k;
           if (XCH % 32 == 0 || c < XCH) {
             const int tt = c / CPR, cc = c % CPR;
-            const bool ok = (d_w + cc * 8 < D) && (t0 + tt < t_seg_end);
+            const bool ok = WHOLE || ((d_w + cc * 8 < D) && (t0 + tt < t_seg_end));
             const size_t go = ok ? (row0 + tt) * D + d_w + cc * 8 : 0;
             cp_async16(&sm.x[st][tt][cc * 4], gx + go, ok);
             cp_async16(&sm.d[st][tt][cc * 4], gd + go, ok);
@@ -574,14 +576,14 @@ __global__ void __launch_bounds__(kBwdWarps * 32, (CPT == 16 / S) ? 2 : 3)
         }
         if (lane < kBT * 2) {
           const int tt = lane >> 1, hc = lane & 1;
-          const bool ok = t0 + tt < t_seg_end;
+          const bool ok = WHOLE || t0 + tt < t_seg_end;
           const size_t go = ok ? (row0 + tt) * 16 + hc * 8 : 0;
           if constexpr (!SB) cp_async16(&sm.rB[st][tt][hc * 4], gB + go, ok);
           if constexpr (!SC) cp_async16(&sm.rC[st][tt][hc * 4], gC + go, ok);
         }
 #pragma unroll
         for (int sb = 0; sb < kBT / kSB; ++sb) {
-          const bool ok = valid && (t0 + sb * kSB < t_seg_end);
+          const bool ok = WHOLE || (valid && (t0 + sb * kSB < t_seg_end));
 #pragma unroll
           for (int q = 0; q < CPT; ++q)
 #pragma unroll
@@ -710,7 +712,7 @@ __global__ void __launch_bounds__(kBwdWarps * 32, (CPT == 16 / S) ? 2 : 3)
       __syncwarp();                   // this tile landed for all lanes; all lanes are done with the previous one
       issue_tile(tile - 1, st ^ 1);   // prefetch the tile before in time
       const int t0 = t_seg0 + tile * kBT;
-      const int nlive = min(kBT, t_seg_end - t0);
+      const int nlive = WHOLE ? kBT : min(kBT, t_seg_end - t0);
       {
         // B and C of the tile to float: lane -> (row lane / 4, states 4 (lane % 4) ..)
 #pragma unroll
@@ -803,7 +805,7 @@ __global__ void __launch_bounds__(kBwdWarps * 32, (CPT == 16 / S) ? 2 : 3)
       for (int k = 0; k < (XCH + 31) / 32; ++k) {
         const int c = lane + 32 * k;
         const int tt = c / CPR, cc = c % CPR;
-        if ((XCH % 32 == 0 || c < XCH) && d_w + cc * 8 < D && tt < nlive &&
+        if ((XCH % 32 == 0 || c < XCH) && (WHOLE || (d_w + cc * 8 < D && tt < nlive)) &&
             SSM_IN_RANGE(row0 + tt < (size_t)p.batch * p.L && d_w + cc * 8 + 8 <= D, sc.abort)) {
           const size_t go = (row0 + tt) * D + d_w + cc * 8;
           *reinterpret_cast<uint4*>(gdx + go) = *reinterpret_cast<const uint4*>(&sm.ox[tt][cc * 4]);
@@ -910,6 +912,15 @@ cudaError_t launch_bwd_variant(const Plan& plan, const BwdParams& p, cudaStream_
   sc.abort = p.abort;
   sc.handoff = p.handoff;
   const unsigned grid = (unsigned)((sc.workers + kBwdWarps - 1) / kBwdWarps);
+  if constexpr (!ZOH && BC == 0) {
+    // no ragged tile or channel group anywhere: the instantiation without range tests (same launch shape)
+    if (p.L % kBT == 0 && plan.seg_steps % kBT == 0 && p.D % CW == 0) {
+      auto whole = ssm_bwd_warp_kernel<S, CPT, SP, ZOH, BC, true>;
+      if ((e = cudaFuncSetAttribute(whole, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess) return e;
+      whole<<<grid, kBwdWarps * 32, smem, s>>>(p, sc);
+      return cudaGetLastError();
+    }
+  }
   kern<<<grid, kBwdWarps * 32, smem, s>>>(p, sc);
   return cudaGetLastError();
 }

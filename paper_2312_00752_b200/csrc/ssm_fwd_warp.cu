@@ -67,7 +67,9 @@ __device__ __forceinline__ float bf16at(const uint32_t* row, int c) {
 
 }  // namespace
 
-template <int S, int MODE, bool SP, bool ZOH, int BC, int NST>
+// WHOLE: every tile and every channel group of the problem is whole (L and the segment length are multiples of the tile,
+// D of the chain width), so the staging, the sub-block loop and the output copy carry no range tests
+template <int S, int MODE, bool SP, bool ZOH, int BC, int NST, bool WHOLE = false>
 __global__ void __launch_bounds__(kWarpsPerBlock * 32, MODE == kFwdFull ? 1 : 0) ssm_fwd_warp_kernel(const FwdParams p, const WarpSched sc) {
   static_assert(NST == 2 || NST == 3, "ring stages");
   static_assert(S == 16 || S == 8, "one lane or a lane pair per channel");
@@ -138,7 +140,7 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, MODE == kFwdFull ? 1 : 0)
 #pragma unroll
         for (int k = 0; k < kWT / RP; ++k) {
           const int tt = xrow + RP * k;
-          const bool ok = xcol_ok && (t0 + tt < t_to);
+          const bool ok = WHOLE || (xcol_ok && (t0 + tt < t_to));
           const size_t go = ok ? xo + (size_t)k * RP * D : 0;
           cp_async16(&sm.x[st][tt][xcc * 4], gx + go, ok);
           cp_async16(&sm.d[st][tt][xcc * 4], gd + go, ok);
@@ -147,7 +149,7 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, MODE == kFwdFull ? 1 : 0)
 #pragma unroll
         for (int k = 0; k < 2; ++k) {
           const int tt = brow + 16 * k;
-          const bool ok = t0 + tt < t_to;
+          const bool ok = WHOLE || (t0 + tt < t_to);
           const size_t go = ok ? bo + (size_t)k * 16 * 16 : 0;
           if constexpr (TB) cp_async16(&sm.rB[st][tt][bhc * 4], gB + go, ok);
           if constexpr (TC) cp_async16(&sm.rC[st][tt][bhc * 4], gC + go, ok);
@@ -438,7 +440,7 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, MODE == kFwdFull ? 1 : 0)
 #pragma unroll 1
       for (int sb = 0; sb < kWT / kSub; ++sb) {
         const int ts = t0 + sb * kSub;
-        if (ts >= t_to) break;
+        if (!WHOLE && ts >= t_to) break;
         if (!SUMMARY && ck_lane != nullptr && SSM_IN_RANGE(ts / kCkptSteps < p.nck && ts < p.L, sc.abort)) {
           float* dst = ck_lane + (size_t)(ts / kCkptSteps) * ck_stride;
 #pragma unroll
@@ -468,7 +470,7 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, MODE == kFwdFull ? 1 : 0)
 #pragma unroll
         for (int k = 0; k < kWT / RP; ++k) {
           const int tt = xrow + RP * k;
-          if (xcol_ok && t0 + tt < t_to &&
+          if ((WHOLE || (xcol_ok && t0 + tt < t_to)) &&
               SSM_IN_RANGE(xo + (size_t)k * RP * D + 8 <= (size_t)p.batch * p.L * D && d_w + xcc * 8 + 8 <= D, sc.abort))
             *reinterpret_cast<uint4*>(gout + xo + (size_t)k * RP * D) = *reinterpret_cast<const uint4*>(&sm.o[tt][xcc * 4]);
         }
@@ -559,6 +561,22 @@ cudaError_t launch_variant_w(const Plan& plan, const FwdParams& p, cudaStream_t 
   sc.abort = p.abort;
   sc.handoff = p.handoff;
   const unsigned grid = (unsigned)((sc.workers + kWarpsPerBlock - 1) / kWarpsPerBlock);
+  if constexpr (!ZOH && BC == 0) {
+    // no ragged tile or channel group anywhere: the instantiations without range tests (same shared memory and launch
+    // shape as the ones the occupancy was taken from)
+    if (p.L % kWT == 0 && plan.seg_steps % kWT == 0 && p.D % CW == 0) {
+      auto go = [&](auto kern) {
+        const cudaError_t ea = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (ea != cudaSuccess) return ea;
+        kern<<<grid, kWarpsPerBlock * 32, smem, s>>>(p, sc);
+        return cudaGetLastError();
+      };
+      if constexpr (MODE != kFwdSummary) {
+        if (two_stage) return go(ssm_fwd_warp_kernel<S, MODE, SP, ZOH, BC, 2, true>);
+      }
+      return go(ssm_fwd_warp_kernel<S, MODE, SP, ZOH, BC, 3, true>);
+    }
+  }
   if constexpr (!ZOH && MODE != kFwdSummary && BC == 0) {
     if (two_stage) {
       ssm_fwd_warp_kernel<S, MODE, SP, ZOH, BC, 2><<<grid, kWarpsPerBlock * 32, smem, s>>>(p, sc);
