@@ -311,7 +311,7 @@ cudaError_t launch_local(const Plan& plan, const BwdParams& p, cudaStream_t s) {
   sc.abort = p.abort;
   sc.handoff = p.handoff;                     // (the hand-off slots are shared: the two kernels run one after the other)
   const unsigned grid = (unsigned)((sc.workers + kLWarps - 1) / kLWarps);
-  if constexpr (!SC) {
+  {
     // no ragged tile or channel group anywhere: the instantiation without range tests (same launch shape)
     if (p.L % kLT == 0 && plan.seg_steps % kLT == 0 && p.D % 32 == 0) {
       auto whole = ssm_bwd_local_warp_kernel<SP, SC, true>;

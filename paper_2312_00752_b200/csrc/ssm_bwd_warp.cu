@@ -912,7 +912,7 @@ cudaError_t launch_bwd_variant(const Plan& plan, const BwdParams& p, cudaStream_
   sc.abort = p.abort;
   sc.handoff = p.handoff;
   const unsigned grid = (unsigned)((sc.workers + kBwdWarps - 1) / kBwdWarps);
-  if constexpr (!ZOH && BC == 0) {
+  {
     // no ragged tile or channel group anywhere: the instantiation without range tests (same launch shape)
     if (p.L % kBT == 0 && plan.seg_steps % kBT == 0 && p.D % CW == 0) {
       auto whole = ssm_bwd_warp_kernel<S, CPT, SP, ZOH, BC, true>;

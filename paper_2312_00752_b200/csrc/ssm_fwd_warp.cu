@@ -561,7 +561,7 @@ cudaError_t launch_variant_w(const Plan& plan, const FwdParams& p, cudaStream_t 
   sc.abort = p.abort;
   sc.handoff = p.handoff;
   const unsigned grid = (unsigned)((sc.workers + kWarpsPerBlock - 1) / kWarpsPerBlock);
-  if constexpr (!ZOH && BC == 0) {
+  {
     // no ragged tile or channel group anywhere: the instantiations without range tests (same shared memory and launch
     // shape as the ones the occupancy was taken from)
     if (p.L % kWT == 0 && plan.seg_steps % kWT == 0 && p.D % CW == 0) {
@@ -571,7 +571,7 @@ cudaError_t launch_variant_w(const Plan& plan, const FwdParams& p, cudaStream_t 
         kern<<<grid, kWarpsPerBlock * 32, smem, s>>>(p, sc);
         return cudaGetLastError();
       };
-      if constexpr (MODE != kFwdSummary) {
+      if constexpr (!ZOH && MODE != kFwdSummary && BC == 0) {
         if (two_stage) return go(ssm_fwd_warp_kernel<S, MODE, SP, ZOH, BC, 2, true>);
       }
       return go(ssm_fwd_warp_kernel<S, MODE, SP, ZOH, BC, 3, true>);
