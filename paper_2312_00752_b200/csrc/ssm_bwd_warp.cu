@@ -706,6 +706,10 @@ __global__ void __launch_bounds__(kBwdWarps * 32, (CPT == 16 / S) ? 2 : 3)
         }
     }
 
+    // The sweep over the tiles exists once per kind of A (arithmetic progression or general), chosen once per chain, so
+    // that neither body carries the registers of the other.
+    auto sweep = [&](auto ap_tag) {
+    constexpr bool AP_ = decltype(ap_tag)::value;
     int st = 0;
     for (int tile = tile_hi; tile >= tile_lo; --tile, st ^= 1) {
       cp_async_wait_all();
@@ -780,22 +784,16 @@ __global__ void __launch_bounds__(kBwdWarps * 32, (CPT == 16 / S) ? 2 : 3)
           }
           zs = __any_sync(0xffffffffu, dmin * cr.minA < kZohSmall);
         }
-#define SSM_SUB_BLOCK(AP_, ZS_)                                                                                     \
+#define SSM_SUB_BLOCK(ZS_)                                                                                          \
   sub_block<S, CPT, SP, AP_, ZOH, ZS_, BC>(ln, cr, sb * kSB, nlive, has_z ? 1.f : 0.f, p.softplus != 0, &sm.x[st][0][0], \
                                        &sm.d[st][0][0], &sm.fB[0][0], &sm.fC[0][0], &sm.ds[0][0], &sm.gp[0][0],      \
                                        &sm.dF[0][0], &sm.ck[st][sb][0][0], &sm.ox[0][0], &sm.od[0][0], &sm.oz[0][0], \
                                        &sm.red[0][0][0], part_dB, part_dC, sc.abort)
         if constexpr (ZOH) {
-          if (zs) {
-            if (ap) SSM_SUB_BLOCK(true, true);
-            else SSM_SUB_BLOCK(false, true);
-          } else {
-            if (ap) SSM_SUB_BLOCK(true, false);
-            else SSM_SUB_BLOCK(false, false);
-          }
+          if (zs) SSM_SUB_BLOCK(true);
+          else SSM_SUB_BLOCK(false);
         } else {
-          if (ap) SSM_SUB_BLOCK(true, false);
-          else SSM_SUB_BLOCK(false, false);
+          SSM_SUB_BLOCK(false);
         }
 #undef SSM_SUB_BLOCK
       }
@@ -814,6 +812,9 @@ __global__ void __launch_bounds__(kBwdWarps * 32, (CPT == 16 / S) ? 2 : 3)
         }
       }
     }
+    };
+    if (ap) sweep(std::true_type{});
+    else sweep(std::false_type{});
     cp_async_wait_all();
     __syncwarp();
 
