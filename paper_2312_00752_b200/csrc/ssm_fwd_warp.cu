@@ -70,7 +70,7 @@ __device__ __forceinline__ float bf16at(const uint32_t* row, int c) {
 // WHOLE: every tile and every channel group of the problem is whole (L and the segment length are multiples of the tile,
 // D of the chain width), so the staging, the sub-block loop and the output copy carry no range tests
 template <int S, int MODE, bool SP, bool ZOH, int BC, int NST, bool WHOLE = false>
-__global__ void __launch_bounds__(kWarpsPerBlock * 32, MODE == kFwdFull ? 1 : 0) ssm_fwd_warp_kernel(const FwdParams p, const WarpSched sc) {
+__global__ void __launch_bounds__(kWarpsPerBlock * 32, MODE == kFwdFull ? 1 : 3) ssm_fwd_warp_kernel(const FwdParams p, const WarpSched sc) {
   static_assert(NST == 2 || NST == 3, "ring stages");
   static_assert(S == 16 || S == 8, "one lane or a lane pair per channel");
   constexpr bool FULL = (MODE == kFwdFull);
