@@ -52,6 +52,8 @@ def _oracle_static(inp, Bs, Cs, zoh=False):
     (1, 97, 72, 16, "bf16", False, True, False),     # tuned kernels: selective B only, channel blocks 32 + 32 + 8
     (1, 4200, 48, 16, "bf16", True, True, False),    # tuned kernels with a time split in both directions
     (2, 64, 32, 16, "bf16", True, True, True),       # ZOH with non-selective B / C stays on the generic kernels
+    (2, 128, 64, 16, "bf16", True, True, False),     # tuned kernels, whole tiles and channel groups (no range tests)
+    (1, 256, 96, 16, "bf16", False, True, False),    # the same with selective B only
 ])
 def test_static_b_and_c(batch, L, D, N, io, sB, sC, zoh):
     import torch
